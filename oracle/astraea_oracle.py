@@ -1,0 +1,165 @@
+"""ctypes front end of the CPU oracle (astraea_oracle.c).
+
+TEST INFRASTRUCTURE ONLY.  Importers: tests/, the smoke check and the CPU-baseline
+leg of the benchmark.  The CUDA library and its Python binding never import this
+module, and this module imports nothing from them.
+
+All floating-point arrays are float64 numpy arrays; bf16 inputs are upcast
+exactly by the caller before they get here.  `step()` chains the four stages in
+the order of Algorithm 1.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "astraea_oracle.c")
+_LIB = os.path.join(_HERE, "libastraea_oracle.so")
+
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (-O2 -fopenmp).  Returns the library path."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11",
+                               "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = ctypes.CDLL(_LIB)
+        _lib.oracle_select.restype = ctypes.c_int
+        _lib.oracle_budget_to_k.restype = ctypes.c_int
+    return _lib
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _f64(a):
+    return None if a is None else np.ascontiguousarray(a, dtype=np.float64)
+
+
+def _i32(a):
+    return None if a is None else np.ascontiguousarray(a, dtype=np.int32)
+
+
+def num_threads() -> int:
+    """Threads the OpenMP loops will use (OMP_NUM_THREADS or all cores)."""
+    v = os.environ.get("OMP_NUM_THREADS")
+    return int(v) if v else (os.cpu_count() or 1)
+
+
+def budget_to_k(n_sel: int, theta_permille: int) -> int:
+    return int(_load().oracle_budget_to_k(int(n_sel), int(theta_permille)))
+
+
+def score(x_cur, x_ref, lse=None, n_skip=None, n_sel=None, H=1, w_alpha=1.0, w_beta=1.0,
+          delta_mode=0, lse_mode=0):
+    """S_token for tokens [0, n_sel) of every batch row; returns float64 [B, n_sel]."""
+    x_cur, x_ref, lse, n_skip = _f64(x_cur), _f64(x_ref), _f64(lse), _i32(n_skip)
+    B, N, D = x_cur.shape
+    n_sel = N if n_sel is None else n_sel
+    if lse is not None:
+        H = lse.shape[1]
+        assert lse.shape == (B, H, N)
+    out = np.empty((B, n_sel), dtype=np.float64)
+    _load().oracle_score(_p(x_cur), _p(x_ref), _p(lse), _p(n_skip), _p(out),
+                         B, N, n_sel, D, H, ctypes.c_double(w_alpha), ctypes.c_double(w_beta),
+                         int(delta_mode), int(lse_mode))
+    return out
+
+
+def select(score_f32, k, n_always=0, n_skip=None):
+    """Top-k per batch row on float32 scores.  Returns (idx_sel, idx_rem, n_skip_new)."""
+    s = np.ascontiguousarray(score_f32, dtype=np.float32)
+    B, n_sel = s.shape
+    idx_sel = np.empty((B, k + n_always), dtype=np.int32)
+    idx_rem = np.empty((B, n_sel - k), dtype=np.int32)
+    n_new = None if n_skip is None else np.array(n_skip, dtype=np.int32, copy=True, order="C")
+    rc = _load().oracle_select(_p(s), B, n_sel, int(k), int(n_always), _p(idx_sel), _p(idx_rem), _p(n_new))
+    if rc != 0:
+        raise ValueError("oracle_select: bad k")
+    return idx_sel, idx_rem, n_new
+
+
+def sparse_attn(q, k, v, q_idx=None, kv_idx=None, scale=0.0, want_probs=False):
+    """Attention rows for the listed queries against all keys (or kv_idx).
+
+    q, k, v: [B, N, H, d].  Returns (o [B, M, H, d], lse [B, H, M], probs or None).
+    """
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    B, N, H, d = k.shape
+    assert q.shape == k.shape == v.shape
+    q_idx = _i32(q_idx)
+    kv_idx = _i32(kv_idx)
+    M = N if q_idx is None else q_idx.shape[1]
+    M_kv = 0 if kv_idx is None else kv_idx.shape[1]
+    Nk = N if kv_idx is None else M_kv
+    o = np.empty((B, M, H, d), dtype=np.float64)
+    lse = np.empty((B, H, M), dtype=np.float64)
+    probs = np.empty((B, H, M, Nk), dtype=np.float64) if want_probs else None
+    _load().oracle_sparse_attn(_p(q), _p(k), _p(v), _p(q_idx), M, _p(kv_idx), M_kv,
+                               _p(o), _p(lse), _p(probs), B, H, N, d, ctypes.c_double(scale))
+    return o, lse, probs
+
+
+def scatter_reuse(cache, rows, idx):
+    """Copy of `cache` [B, N, ...] with rows idx[b, r] replaced by rows[b, r]."""
+    out = np.array(cache, dtype=np.float64, copy=True, order="C")
+    rows = _f64(rows)
+    idx = _i32(idx)
+    B, N = out.shape[:2]
+    R = int(np.prod(out.shape[2:]))
+    M = idx.shape[1]
+    if M:
+        _load().oracle_scatter_reuse(_p(out), _p(rows), _p(idx), B, N, M, R)
+    return out
+
+
+def scatter_lse(lse_cache, lse_rows, idx):
+    out = np.array(lse_cache, dtype=np.float64, copy=True, order="C")
+    lse_rows, idx = _f64(lse_rows), _i32(idx)
+    B, H, N = out.shape
+    M = idx.shape[1]
+    if M:
+        _load().oracle_scatter_lse(_p(out), _p(lse_rows), _p(idx), B, H, N, M)
+    return out
+
+
+def step(x_cur, x_ref, lse_cache, n_skip, q, k, v, cache, k_keep, n_always=0,
+         w_alpha=1.0, w_beta=1.0, delta_mode=0, lse_mode=0, scale=0.0):
+    """One attention block at one denoising step (Algorithm 1), all in fp64.
+
+    Returns a dict with score (fp64), score_f32, idx_sel, idx_rem, n_skip (new),
+    out (new cache, [B,N,H,d]), lse (new lse cache, [B,H,N]), x_ref (refreshed at
+    the selected tokens: the "last computed" reference).
+    """
+    B, N = x_cur.shape[:2]
+    n_sel = N - n_always
+    s64 = score(x_cur, x_ref, lse_cache, n_skip, n_sel=n_sel, w_alpha=w_alpha, w_beta=w_beta,
+                delta_mode=delta_mode, lse_mode=lse_mode)
+    s32 = s64.astype(np.float32)
+    idx_sel, idx_rem, n_new = select(s32, k_keep, n_always, n_skip)
+    if idx_sel.shape[1]:
+        o, l, _ = sparse_attn(q, k, v, q_idx=idx_sel, scale=scale)
+        out = scatter_reuse(cache, o, idx_sel)
+        lse_new = scatter_lse(lse_cache, l, idx_sel)
+        xr = scatter_reuse(x_ref, np.take_along_axis(_f64(x_cur), idx_sel[:, :, None].astype(np.int64), axis=1), idx_sel)
+    else:
+        out = np.array(cache, dtype=np.float64, copy=True)
+        lse_new = np.array(lse_cache, dtype=np.float64, copy=True)
+        xr = np.array(x_ref, dtype=np.float64, copy=True)
+    return dict(score=s64, score_f32=s32, idx_sel=idx_sel, idx_rem=idx_rem, n_skip=n_new,
+                out=out, lse=lse_new, x_ref=xr)

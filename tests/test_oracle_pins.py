@@ -1,0 +1,323 @@
+"""Pins for the CPU oracle: each test checks it against something other than itself
+(a library routine, a closed form, brute force, an invariant), so that a dropped
+term, a wrong sign or index, or a transposed operand fails at least one of them.
+No GPU needed."""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2506_05096_b200 import synth
+
+
+def _rand(rng, *shape):
+    return rng.standard_normal(shape)
+
+
+# ---------------------------------------------------------------- attention pins
+def test_dense_special_case_matches_library_attention(oracle):
+    """Keep-ratio 1 (all queries) is plain Softmax(QK^T/sqrt(d))V (Section 3.1 equations):
+    compare with torch's fp64 scaled_dot_product_attention and a numpy einsum."""
+    rng = np.random.default_rng(1)
+    B, N, H, d = 2, 37, 3, 8
+    q, k, v = (_rand(rng, B, N, H, d) for _ in range(3))
+    o, lse, p = oracle.sparse_attn(q, k, v, want_probs=True)
+    tq, tk, tv = (torch.from_numpy(a).permute(0, 2, 1, 3) for a in (q, k, v))
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv).permute(0, 2, 1, 3).numpy()
+    assert np.abs(o - ref).max() < 1e-12
+    s = np.einsum("bihc,bjhc->bhij", q, k) / math.sqrt(d)
+    ref_lse = np.log(np.exp(s).sum(-1))
+    assert np.abs(lse - ref_lse).max() < 1e-12
+    ref_p = np.exp(s - ref_lse[..., None])
+    assert np.abs(p - ref_p).max() < 1e-13
+    assert np.abs(o - np.einsum("bhij,bjhc->bihc", ref_p, v)).max() < 1e-12
+
+
+def test_selected_rows_equal_rows_of_dense(oracle):
+    """Each selected output row depends only on its own query and all K/V."""
+    rng = np.random.default_rng(2)
+    B, N, H, d = 2, 50, 2, 16
+    q, k, v = (_rand(rng, B, N, H, d) for _ in range(3))
+    idx = np.stack([np.sort(rng.choice(N, 13, replace=False)) for _ in range(B)]).astype(np.int32)
+    o_all, lse_all, _ = oracle.sparse_attn(q, k, v)
+    o, lse, _ = oracle.sparse_attn(q, k, v, q_idx=idx)
+    for b in range(B):
+        assert np.array_equal(o[b], o_all[b, idx[b]])
+        assert np.array_equal(lse[b], lse_all[b][:, idx[b]])
+    # independence from the other queries: scrambling unselected q rows changes nothing
+    q2 = q.copy()
+    mask = np.ones((B, N), bool)
+    for b in range(B):
+        mask[b, idx[b]] = False
+    q2[mask] = 123.0
+    o2, _, _ = oracle.sparse_attn(q2, k, v, q_idx=idx)
+    assert np.array_equal(o, o2)
+
+
+def test_softmax_rows_sum_to_one_and_outputs_in_hull(oracle):
+    rng = np.random.default_rng(3)
+    B, N, H, d = 1, 64, 2, 8
+    q, k, v = (3.0 * _rand(rng, B, N, H, d) for _ in range(3))
+    idx = np.arange(0, N, 3, dtype=np.int32)[None]
+    o, _, p = oracle.sparse_attn(q, k, v, q_idx=idx, want_probs=True)
+    assert np.abs(p.sum(-1) - 1.0).max() < 1e-12
+    assert (p >= 0).all()
+    lo, hi = v.min(axis=1)[:, None], v.max(axis=1)[:, None]
+    assert (o >= lo - 1e-12).all() and (o <= hi + 1e-12).all()
+
+
+def test_zero_keys_give_mean_of_values_and_ln_n(oracle):
+    rng = np.random.default_rng(4)
+    B, N, H, d = 1, 33, 2, 8
+    q, v = _rand(rng, B, N, H, d), _rand(rng, B, N, H, d)
+    o, lse, _ = oracle.sparse_attn(q, np.zeros_like(q), v)
+    assert np.abs(o - v.mean(axis=1, keepdims=True)).max() < 1e-13
+    assert np.abs(lse - math.log(N)).max() < 1e-13
+    o, lse, _ = oracle.sparse_attn(np.zeros_like(q), q, v)
+    assert np.abs(o - v.mean(axis=1, keepdims=True)).max() < 1e-13
+
+
+def test_constant_value_row_is_returned(oracle):
+    rng = np.random.default_rng(5)
+    B, N, H, d = 1, 20, 2, 8
+    q, k = _rand(rng, B, N, H, d), _rand(rng, B, N, H, d)
+    row = _rand(rng, 1, 1, H, d)
+    o, _, _ = oracle.sparse_attn(q, k, np.broadcast_to(row, q.shape).copy())
+    assert np.abs(o - row).max() < 1e-13
+
+
+def test_dominant_key_selects_its_value(oracle):
+    """One key aligned with the query and scaled up takes all the softmax mass; the
+    scale is 1/sqrt(d): the logit gap is c*|q|^2/sqrt(d), which the LSE reveals."""
+    rng = np.random.default_rng(6)
+    B, N, H, d = 1, 16, 1, 4
+    q, v = _rand(rng, B, N, H, d), _rand(rng, B, N, H, d)
+    k = np.zeros_like(q)
+    i, j, c = 5, 11, 40.0
+    k[0, j] = c * q[0, i]
+    o, lse, _ = oracle.sparse_attn(q, k, v, q_idx=np.array([[i]], np.int32))
+    assert np.abs(o[0, 0] - v[0, j]).max() < 1e-9
+    top = c * (q[0, i, 0] ** 2).sum() / math.sqrt(d)
+    assert abs(lse[0, 0, 0] - top) < 1e-9
+    # an explicit scale overrides 1/sqrt(d)
+    _, lse2, _ = oracle.sparse_attn(q, k, v, q_idx=np.array([[i]], np.int32), scale=0.25)
+    assert abs(lse2[0, 0, 0] - 0.25 * c * (q[0, i, 0] ** 2).sum()) < 1e-5   # the other 15 keys weigh e^-15.7 each
+
+
+def test_joint_permutation_of_keys_and_values_is_invisible(oracle):
+    rng = np.random.default_rng(7)
+    B, N, H, d = 1, 40, 2, 8
+    q, k, v = (_rand(rng, B, N, H, d) for _ in range(3))
+    idx = np.array([[1, 4, 9, 30]], np.int32)
+    o, lse, _ = oracle.sparse_attn(q, k, v, q_idx=idx)
+    perm = rng.permutation(N)
+    inv = np.argsort(perm)
+    # permute tokens: query rows move with their tokens
+    o2, lse2, _ = oracle.sparse_attn(q[:, perm], k[:, perm], v[:, perm],
+                                     q_idx=np.sort(inv[idx[0]])[None].astype(np.int32))
+    order = np.argsort(inv[idx[0]])
+    assert np.abs(o2[0] - o[0, order]).max() < 1e-12
+    assert np.abs(lse2[0] - lse[0][:, order]).max() < 1e-12
+
+
+def test_select_q_and_k_ablation_is_attention_on_the_subset(oracle):
+    rng = np.random.default_rng(8)
+    B, N, H, d = 1, 24, 2, 8
+    q, k, v = (_rand(rng, B, N, H, d) for _ in range(3))
+    idx = np.array([[0, 3, 5, 8, 13, 21]], np.int32)
+    o, _, _ = oracle.sparse_attn(q, k, v, q_idx=idx, kv_idx=idx)
+    sub = lambda a: a[:, idx[0]]
+    o_ref, _, _ = oracle.sparse_attn(sub(q), sub(k), sub(v))
+    assert np.abs(o - o_ref).max() < 1e-13
+
+
+# ------------------------------------------------------------------ reuse pins
+def test_keep_ratio_zero_returns_cache_unchanged(oracle):
+    rng = np.random.default_rng(9)
+    B, N, H, d = 2, 12, 2, 4
+    cache = _rand(rng, B, N, H, d)
+    out = oracle.scatter_reuse(cache, np.empty((B, 0, H, d)), np.empty((B, 0), np.int32))
+    assert np.array_equal(out, cache)
+    x = _rand(rng, B, N, H * d)
+    lse = _rand(rng, B, H, N)
+    res = oracle.step(x, x + 0.1, lse, np.zeros((B, N), np.int32), *(_rand(rng, B, N, H, d) for _ in range(3)),
+                      cache, k_keep=0)
+    assert np.array_equal(res["out"], cache)
+    assert np.array_equal(res["lse"], lse)
+    assert (res["n_skip"] == 1).all()
+    assert res["idx_sel"].shape == (B, 0) and res["idx_rem"].shape == (B, N)
+
+
+def test_scatter_touches_only_selected_rows(oracle):
+    rng = np.random.default_rng(10)
+    B, N, R, M = 2, 17, 6, 5
+    cache = _rand(rng, B, N, R)
+    rows = _rand(rng, B, M, R)
+    idx = np.stack([np.sort(rng.choice(N, M, replace=False)) for _ in range(B)]).astype(np.int32)
+    out = oracle.scatter_reuse(cache, rows, idx)
+    for b in range(B):
+        for i in range(N):
+            if i in idx[b]:
+                assert np.array_equal(out[b, i], rows[b, list(idx[b]).index(i)])
+            else:
+                assert np.array_equal(out[b, i], cache[b, i])
+    # selected rows do not depend on the prior cache contents
+    out2 = oracle.scatter_reuse(np.zeros_like(cache), rows, idx)
+    for b in range(B):
+        assert np.array_equal(out2[b, idx[b]], out[b, idx[b]])
+
+
+def test_full_step_at_keep_ratio_one_is_dense_attention(oracle):
+    rng = np.random.default_rng(11)
+    B, N, H, d = 1, 30, 2, 8
+    x = _rand(rng, B, N, H * d)
+    q, k, v, cache = (_rand(rng, B, N, H, d) for _ in range(4))
+    res = oracle.step(x, x * 0.5, _rand(rng, B, H, N), np.zeros((B, N), np.int32), q, k, v, cache, k_keep=N)
+    tq, tk, tv = (torch.from_numpy(a).permute(0, 2, 1, 3) for a in (q, k, v))
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv).permute(0, 2, 1, 3).numpy()
+    assert np.abs(res["out"] - ref).max() < 1e-12
+    assert (res["n_skip"] == 0).all()
+    assert np.array_equal(res["x_ref"], x)
+
+
+# -------------------------------------------------------------- selection pins
+def _brute_select(s, k):
+    order = sorted(range(len(s)), key=lambda i: (-(s[i] if not math.isnan(s[i]) else -math.inf), i))
+    return sorted(order[:k]), sorted(order[k:])
+
+
+@pytest.mark.parametrize("n,levels", [(1, 2), (7, 3), (64, 4), (257, 5), (300, 1000)])
+def test_select_equals_brute_force_sort(oracle, n, levels):
+    for seed in range(4):
+        s = synth.integer_scores(2, n, seed, levels)
+        for k in sorted({0, 1, n // 3, n - 1, n} & set(range(n + 1))):
+            sel, rem, _ = oracle.select(s, k)
+            for b in range(2):
+                bs, br = _brute_select(list(map(float, s[b])), k)
+                assert list(sel[b]) == bs and list(rem[b]) == br
+
+
+def test_select_ties_nan_signed_zero_and_always_kept(oracle):
+    s = np.array([[1.0, 1.0, 1.0, 1.0, 1.0, 1.0]], np.float32)
+    sel, rem, _ = oracle.select(s, 2)
+    assert list(sel[0]) == [0, 1] and list(rem[0]) == [2, 3, 4, 5]
+    s = np.array([[0.0, -0.0, np.nan, -1.0, np.inf, -0.0]], np.float32)
+    sel, rem, _ = oracle.select(s, 3)          # inf, then the zeros by index (+0 == -0)
+    assert list(sel[0]) == [0, 1, 4]
+    sel, _, _ = oracle.select(s, 5)            # NaN ranks last
+    assert list(sel[0]) == [0, 1, 3, 4, 5]
+    sel, rem, n = oracle.select(np.array([[3.0, 1.0, 2.0]], np.float32), 1, n_always=2,
+                                n_skip=np.array([[5, 80, 0]], np.int32))
+    assert list(sel[0]) == [0, 3, 4] and list(rem[0]) == [1, 2]
+    assert list(n[0]) == [0, 80, 1]           # reset, clamp, increment
+
+
+def test_select_on_float_scores_matches_numpy_partition(oracle):
+    rng = np.random.default_rng(12)
+    s = rng.standard_normal((3, 1000)).astype(np.float32)
+    k = 333
+    sel, rem, _ = oracle.select(s, k)
+    for b in range(3):
+        ref = np.sort(np.argsort(-s[b], kind="stable")[:k])
+        assert np.array_equal(sel[b], ref)
+        assert np.array_equal(np.sort(np.concatenate([sel[b], rem[b]])), np.arange(1000))
+
+
+def test_budget_to_k_is_floor(oracle):
+    assert oracle.budget_to_k(17550, 250) == 4387       # 4387.5 floors
+    assert oracle.budget_to_k(17550, 500) == 8775
+    assert oracle.budget_to_k(16384, 400) == 6553
+    assert oracle.budget_to_k(118800, 600) == 71280
+    assert oracle.budget_to_k(100, 0) == 0 and oracle.budget_to_k(100, 1000) == 100
+
+
+# ------------------------------------------------------------------ score pins
+def test_score_constant_per_token_difference_closed_form(oracle):
+    """x_cur = x_ref + c_i: delta is |c_i|, c_i^2, c_i for the three reductions; the
+    score is w_a * mean_h exp(lse) * delta + w_b * e^{n} (selection-metric equations)."""
+    rng = np.random.default_rng(13)
+    B, N, D, H = 2, 9, 16, 3
+    x_ref = _rand(rng, B, N, D)
+    c = rng.choice([-0.5, 0.25, 0.125, -2.0, 1.0], size=(B, N))
+    x_cur = x_ref + c[..., None]
+    lse = 0.3 * _rand(rng, B, H, N)
+    n = rng.integers(0, 4, size=(B, N)).astype(np.int32)
+    s_lse = np.exp(lse).mean(axis=1)
+    for mode, delta in ((0, np.abs(c)), (1, c * c), (2, c)):
+        got = oracle.score(x_cur, x_ref, lse, n, w_alpha=0.7, w_beta=0.2, delta_mode=mode)
+        want = 0.7 * s_lse * delta + 0.2 * np.exp(n)
+        assert np.abs(got - want).max() < 1e-12
+    got = oracle.score(x_cur, x_ref, lse, n, w_alpha=1.0, w_beta=0.0, lse_mode=1)
+    assert np.abs(got - lse.mean(axis=1) * np.abs(c)).max() < 1e-12
+    # no LSE, no counters: S_LSE = 1, e^0 = 1
+    got = oracle.score(x_cur, x_ref, None, None, H=H, w_alpha=1.0, w_beta=1.0)
+    assert np.abs(got - (np.abs(c) + 1.0)).max() < 1e-12
+    # clamp of n at 80
+    big = oracle.score(x_ref, x_ref, None, np.full((B, N), 500, np.int32), w_alpha=0.0, w_beta=1.0)
+    assert np.allclose(big, math.exp(80.0), rtol=1e-15)
+
+
+def test_score_mixed_signs_distinguish_the_three_reductions(oracle):
+    x_ref = np.zeros((1, 1, 4))
+    x_cur = np.array([[[1.0, -1.0, 2.0, -4.0]]])
+    for mode, want in ((0, 2.0), (1, 5.5), (2, -0.5)):
+        got = oracle.score(x_cur, x_ref, None, None, w_alpha=1.0, w_beta=0.0, delta_mode=mode)
+        assert got[0, 0] == want
+
+
+def test_score_only_covers_selectable_tokens_and_permutes_with_tokens(oracle):
+    rng = np.random.default_rng(14)
+    B, N, D, H, n_sel = 1, 12, 8, 2, 9
+    x_ref, x_cur = _rand(rng, B, N, D), _rand(rng, B, N, D)
+    lse = _rand(rng, B, H, N)
+    n = rng.integers(0, 3, size=(B, n_sel)).astype(np.int32)
+    s = oracle.score(x_cur, x_ref, lse, n, n_sel=n_sel)
+    assert s.shape == (B, n_sel)
+    perm = rng.permutation(n_sel)
+    full = np.concatenate([perm, np.arange(n_sel, N)])
+    s2 = oracle.score(x_cur[:, full], x_ref[:, full], lse[:, :, full], n[:, perm], n_sel=n_sel)
+    assert np.array_equal(s2, s[:, perm])
+
+
+def test_penalty_only_schedule_is_round_robin(oracle):
+    """w_alpha = 0: scores are e^{n_i}; with ties to the lower index and n reset on selection
+    the selection cycles [0,k), [k,2k), ... with period N/k."""
+    N, k = 24, 6
+    n = np.zeros((1, N), np.int32)
+    x = np.zeros((1, N, 4))
+    for t in range(3 * N // k):
+        s = oracle.score(x, x, None, n, w_alpha=0.0, w_beta=1.0).astype(np.float32)
+        sel, _, n = oracle.select(s, k, n_skip=n)
+        start = (t * k) % N
+        assert list(sel[0]) == list(range(start, start + k))
+
+
+def test_drift_statistics_half_normal_mean(oracle):
+    """x_cur = x_ref + sigma*eps gives E[mean|delta|] = sigma*sqrt(2/pi)."""
+    rng = np.random.default_rng(15)
+    N, D, sigma = 64, 4096, 0.05
+    x_ref = _rand(rng, 1, N, D)
+    x_cur = x_ref + sigma * _rand(rng, 1, N, D)
+    s = oracle.score(x_cur, x_ref, None, None, w_alpha=1.0, w_beta=0.0)
+    want = sigma * math.sqrt(2 / math.pi)
+    assert abs(s.mean() - want) < 3e-4
+    assert np.abs(s - want).max() < 6 * sigma * math.sqrt(1 - 2 / math.pi) / math.sqrt(D)
+
+
+# -------------------------------------------------------- flop accounting pin
+def test_attention_flops_are_linear_in_selected_tokens_like_the_papers_tables():
+    from paper_2506_05096_b200 import accounting
+    path = os.path.join(os.path.dirname(__file__), "golden", "flops_tables.txt")
+    B, H, N, d = 1, 24, 118800, 128
+    full = accounting.attn_flops(B, H, N, N, d)
+    assert full == 4 * B * H * N * N * d                # 4*B*N^2*(H*d): the N^2 term of the FLOPs formula
+    for line in open(path):
+        if line.startswith("#") or not line.strip():
+            continue
+        name, orig, *rows = line.split()
+        for theta, val in zip((0.4, 0.5, 0.7), rows):
+            M = int(round(theta * N))
+            ratio = accounting.attn_flops(B, H, M, N, d) / full
+            assert abs(ratio - float(val) / float(orig)) < 2e-4, (name, theta)
