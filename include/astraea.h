@@ -1,0 +1,197 @@
+/*
+ * astraea.h -- C ABI of the B200 (sm_100a) hot path of Astraea's per-denoising-step
+ * token reduction for video diffusion transformers:
+ *
+ *     score -> select (budgeted top-k) -> sparse attention (selected queries x ALL
+ *     keys/values) -> scatter over the cached output (unselected tokens reuse it).
+ *
+ * Conventions
+ *   - Unless a parameter says "host", every data pointer is a DEVICE pointer owned by
+ *     the caller.  The library never frees or retains caller memory and keeps no state
+ *     between calls: all cross-step state (output cache, LSE cache, reference inputs,
+ *     skip counters) lives in caller buffers.
+ *   - Every call is asynchronous on `stream` (a cudaStream_t passed as void*; NULL is the
+ *     default stream), does no host synchronisation and no device->host copy, except
+ *     astraea_poll_error and astraea_step_host which say so.
+ *   - Token order is [selectable tokens 0..N_sel) | always-kept tokens N_sel..N).
+ *   - Hidden states and the cached attention output are [B, N, D] row-major bf16 with
+ *     D = H*d and head h in columns [h*d, (h+1)*d), i.e. [B, N, H, d].
+ *   - Return value: ASTRAEA_OK or a negative ASTRAEA_ERR_*.  Argument errors are found
+ *     on the host before any launch and leave the outputs untouched;
+ *     astraea_last_error() gives a text for the last failure on the calling thread.
+ *   - Rows must start on 16-byte boundaries (d*2 and D*2 bytes are multiples of 16).
+ *   - Inputs must not alias outputs except where "in place" is stated.
+ */
+#ifndef ASTRAEA_H
+#define ASTRAEA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ASTRAEA_OK                        0
+#define ASTRAEA_ERR_INVALID_ARG          -1  /* null/misaligned pointer, bad size, k outside [0,N_sel], D != H*d */
+#define ASTRAEA_ERR_UNSUPPORTED          -2  /* head_dim not in {64,72,128}, unsupported flag or mode            */
+#define ASTRAEA_ERR_WORKSPACE_TOO_SMALL  -3
+#define ASTRAEA_ERR_CUDA                 -4  /* a CUDA call or launch failed                                      */
+#define ASTRAEA_ERR_TIMEOUT              -5  /* a bounded device-side wait gave up (seen by astraea_poll_error)   */
+#define ASTRAEA_ERR_BAD_INDEX            -6  /* an index list was out of range or not strictly ascending          */
+
+#define ASTRAEA_N_SKIP_CLAMP 80              /* counters saturate here so that e^n stays finite in fp32 */
+
+/* delta_mode of astraea_score: how the per-token input difference is reduced over channels */
+#define ASTRAEA_DELTA_MEAN_ABS    0          /* default reading: mean absolute difference */
+#define ASTRAEA_DELTA_MEAN_SQ     1
+#define ASTRAEA_DELTA_MEAN_SIGNED 2
+/* lse_mode of astraea_score */
+#define ASTRAEA_LSE_SUM_EXP 0                /* S_LSE = mean over heads of exp(lse): the paper's literal sum of exponentials */
+#define ASTRAEA_LSE_LOG     1                /* S_LSE = mean over heads of lse itself */
+
+/* flags of astraea_sparse_attn */
+#define ASTRAEA_ATTN_COMPACT_OUT  1u         /* out is [B,M,H,d] and lse_out [B,H,M] (row r of the index list), not the caches */
+/* flags of astraea_scatter_reuse */
+#define ASTRAEA_SCATTER_SRC_FULL  1u         /* rows is [B,N,row_elems]; row idx[r] of it is copied to row idx[r] of cache */
+
+/* op codes of astraea_workspace_bytes */
+#define ASTRAEA_OP_SELECT       1
+#define ASTRAEA_OP_SPARSE_ATTN  2
+#define ASTRAEA_OP_STEP         3
+
+/*
+ * Selection metric (Section 3.2 "Selection Metric"; Algorithm 1 lines 1-2):
+ *     S_token = w_alpha * S_LSE,t-1 * Delta_token,t + w_beta * e^{n_i}
+ * for tokens [0, N_sel) of every batch row.  Delta_token is the difference between the
+ * current inputs x_cur and the reference inputs x_ref (the inputs of the step at which
+ * the token was last computed) reduced over the D channels as delta_mode says; S_LSE is
+ * the softmax normaliser of the token's attention row from an earlier step, carried in
+ * log domain and averaged over heads as lse_mode says; n_i counts the consecutive steps
+ * in which token i was not selected (values above ASTRAEA_N_SKIP_CLAMP count as the clamp).
+ *   x_cur, x_ref : bf16 [B, N, D]                 lse    : fp32 [B, H, N]; NULL => S_LSE = 1
+ *   n_skip       : int32 [B, N_sel]; NULL => 0    score  : out fp32 [B, N_sel]
+ * Arithmetic: bf16 inputs, fp32 accumulation and result.
+ * Errors: INVALID_ARG (null x/score, B,N,D,H <= 0, N_sel outside [0,N], D % 8 != 0,
+ * pointers not 16-byte aligned), UNSUPPORTED (unknown mode), CUDA.
+ */
+int32_t astraea_score(const void *x_cur, const void *x_ref, const float *lse, const int32_t *n_skip,
+                      float *score, int B, int N, int N_sel, int D, int H,
+                      float w_alpha, float w_beta, int delta_mode, int lse_mode, void *stream);
+
+/*
+ * TopK(S_token, theta) -> I_sel, I_remain (Algorithm 1 line 3): the k largest scores of
+ * each batch row.  Deterministic: equal scores go to the lower token index, -0 equals +0,
+ * NaN ranks below every number.  Both index lists come out ascending by token index; the
+ * always-kept span [N_sel, N_sel + n_always) is appended to idx_sel.  The skip counters
+ * are updated in the same pass: 0 for a selected token, min(n+1, ASTRAEA_N_SKIP_CLAMP) otherwise.
+ *   score   : fp32 [B, N_sel]
+ *   idx_sel : out int32 [B, k + n_always]           idx_rem : out int32 [B, N_sel - k]; may be NULL
+ *   n_skip  : in/out int32 [B, N_sel]; may be NULL
+ *   workspace : at least astraea_workspace_bytes(ASTRAEA_OP_SELECT, B, 0, N_sel, k, 0) bytes, 16-byte aligned
+ * k = 0 with n_always = 0 is valid (only the counters change).
+ * Errors: INVALID_ARG (k outside [0,N_sel], negative sizes, null score/idx_sel when needed),
+ * WORKSPACE_TOO_SMALL, CUDA.
+ */
+int32_t astraea_select(const float *score, int B, int N_sel, int k, int n_always,
+                       int32_t *idx_sel, int32_t *idx_rem, int32_t *n_skip,
+                       void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Sparse attention (Algorithm 1 line 6; Section 3.2 "Sparse Attention"; softmax and
+ * attention equations of Section 3.1): for each listed query row i, head h,
+ *     out[i] = Softmax(q_i K^T * scale) V   over ALL N keys/values,
+ *     lse[i] = ln sum_j exp(q_i . k_j * scale),
+ * written IN PLACE at row i of the caches (the reuse step of Algorithm 1 line 7 is thereby
+ * fused: rows that are not listed keep their previous contents), or compactly with
+ * ASTRAEA_ATTN_COMPACT_OUT.
+ *   q, k, v : bf16, head_dim contiguous; element strides (batch, head, token) given per tensor.
+ *             [B,N,H,d] has strides (N*H*d, d, H*d); [B,H,N,d] has (H*N*d, N*d, d).
+ *             Token strides must be multiples of 8 elements, bases 16-byte aligned.
+ *   q_idx   : int32 [B, M] strictly ascending token indices in [0,N); NULL => rows 0..M-1
+ *   kv_idx  : must be NULL (all keys, the paper's method); the select-Q-and-K ablation is not built
+ *   out     : bf16 [B, N, H, d]  (or [B, M, H, d] compact)
+ *   lse_out : fp32 [B, H, N]     (or [B, H, M] compact); may be NULL
+ *   scale   : 0 => 1/sqrt(d)
+ *   workspace : at least astraea_workspace_bytes(ASTRAEA_OP_SPARSE_ATTN, B, H, N, M, d) bytes,
+ *               256-byte aligned; its first word is an error word (see astraea_poll_error)
+ * Arithmetic: bf16 operands, fp32 logits, softmax and accumulation; probabilities are
+ * rounded to bf16 before the P.V product; outputs rounded to bf16.
+ * M = 0 is valid: nothing is launched and the caches are untouched.
+ * Errors: INVALID_ARG, UNSUPPORTED (d not in {64,72,128}, kv_idx != NULL), WORKSPACE_TOO_SMALL, CUDA.
+ */
+int32_t astraea_sparse_attn(const void *q, const void *k, const void *v,
+                            int64_t q_sb, int64_t q_sh, int64_t q_sn,
+                            int64_t k_sb, int64_t k_sh, int64_t k_sn,
+                            int64_t v_sb, int64_t v_sh, int64_t v_sn,
+                            const int32_t *q_idx, int M, const int32_t *kv_idx, int M_kv,
+                            void *out, float *lse_out,
+                            int B, int H, int N, int d, float scale, uint32_t flags,
+                            void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Reuse / cache update (Algorithm 1 lines 6-7; Section 3.2 "Execution Flow"):
+ *     cache[b, idx[b,r], :] = rows[b, r, :]      (rows compact [B, M, row_elems]), or
+ *     cache[b, idx[b,r], :] = rows[b, idx[b,r], :] with ASTRAEA_SCATTER_SRC_FULL;
+ * every row that is not listed is left untouched, i.e. keeps the earlier step's value.
+ * The second form refreshes the reference inputs of the tokens that were computed.
+ *   cache : bf16 [B, N, row_elems], in place      rows : bf16     idx : int32 [B, M], in [0,N), no duplicates
+ * M = 0 is valid.  Errors: INVALID_ARG (row_elems % 8 != 0, misaligned pointers, ...), CUDA.
+ */
+int32_t astraea_scatter_reuse(void *cache, const void *rows, const int32_t *idx,
+                              int B, int N, int M, int row_elems, uint32_t flags, void *stream);
+
+/*
+ * One whole step of one attention block on device buffers (Algorithm 1 with given Q, K, V):
+ * score -> select -> sparse attention with fused scatter -> refresh of x_ref at the
+ * selected tokens.  Equivalent to the four calls above in sequence on `stream`.
+ *   x_cur : bf16 [B,N,D]       x_ref : in/out bf16 [B,N,D]   lse_cache : in/out fp32 [B,H,N]
+ *   n_skip: in/out int32 [B,N_sel]                           q,k,v     : bf16 [B,N,H,d]
+ *   out_cache : in/out bf16 [B,N,H,d]
+ *   score : scratch/out fp32 [B,N_sel]   idx_sel : out int32 [B,k+n_always]   idx_rem : out int32 [B,N_sel-k] or NULL
+ *   workspace : astraea_workspace_bytes(ASTRAEA_OP_STEP, B, H, N, k + n_always, d) bytes
+ */
+int32_t astraea_step(const void *x_cur, void *x_ref, float *lse_cache, int32_t *n_skip,
+                     const void *q, const void *k, const void *v, void *out_cache,
+                     float *score, int32_t *idx_sel, int32_t *idx_rem,
+                     int B, int H, int N, int N_sel, int d, int k_keep,
+                     float w_alpha, float w_beta, int delta_mode, int lse_mode,
+                     void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Host-buffer session: the library owns the device-side state of one attention block
+ * (x_ref, LSE cache, counters, output cache) and staging buffers, and each step copies
+ * the HOST inputs to the device, runs astraea_step and copies the merged output back.
+ * astraea_session_create allocates device memory (cudaMalloc) on the current device;
+ * the first step of a session must be run with k_keep = N_sel (all tokens computed) to
+ * fill the caches, as the paper's denoising loop does at its first timestep.
+ *   x_cur, q, k, v : host bf16 [B,N,D] (pinned memory gives asynchronous copies)
+ *   out            : host bf16 [B,N,D], receives X_out,t (computed + cached rows)
+ * astraea_step_host synchronises the session's stream before it returns.
+ */
+typedef struct astraea_session astraea_session;
+int32_t astraea_session_create(astraea_session **session, int B, int H, int N, int N_sel, int d);
+void    astraea_session_destroy(astraea_session *session);
+int32_t astraea_step_host(astraea_session *session, const void *x_cur, const void *q, const void *k,
+                          const void *v, void *out, int k_keep,
+                          float w_alpha, float w_beta, int delta_mode, int lse_mode);
+
+/* Scratch size for an op (bytes); 0 for unknown ops.  H, d, M may be 0 where the op does not use them. */
+size_t  astraea_workspace_bytes(int op, int B, int H, int N, int M, int d);
+
+/* k = floor(n_sel * theta_permille / 1000) in integer arithmetic (budget theta in 1/1000). */
+int32_t astraea_budget_to_k(int n_sel, int theta_permille);
+
+/*
+ * Synchronises `stream`, reads the error word at the start of `workspace` and clears it.
+ * Returns ASTRAEA_OK, ASTRAEA_ERR_TIMEOUT, ASTRAEA_ERR_BAD_INDEX or ASTRAEA_ERR_CUDA.
+ */
+int32_t astraea_poll_error(void *workspace, void *stream);
+
+const char *astraea_last_error(void);
+const char *astraea_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ASTRAEA_H */

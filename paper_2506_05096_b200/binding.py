@@ -1,0 +1,183 @@
+"""ctypes binding of libastraea.so: same names as include/astraea.h, argument marshalling only.
+
+Tensors are torch CUDA tensors (torch is used for device memory and streams, nothing else);
+every step of the path runs in the library's kernels.  Loading fails loudly if the library
+has not been built (python -m paper_2506_05096_b200.build): there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libastraea.so")
+
+OK = 0
+ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_TIMEOUT, ERR_BAD_INDEX = -1, -2, -3, -4, -5, -6
+DELTA_MEAN_ABS, DELTA_MEAN_SQ, DELTA_MEAN_SIGNED = 0, 1, 2
+LSE_SUM_EXP, LSE_LOG = 0, 1
+ATTN_COMPACT_OUT = 1
+SCATTER_SRC_FULL = 1
+OP_SELECT, OP_SPARSE_ATTN, OP_STEP = 1, 2, 3
+N_SKIP_CLAMP = 80
+
+EXPORTS = [
+    "astraea_score", "astraea_select", "astraea_sparse_attn", "astraea_scatter_reuse", "astraea_step",
+    "astraea_session_create", "astraea_session_destroy", "astraea_step_host",
+    "astraea_workspace_bytes", "astraea_budget_to_k", "astraea_poll_error",
+    "astraea_last_error", "astraea_version",
+]
+
+
+class AstraeaError(RuntimeError):
+    def __init__(self, code: int, text: str):
+        super().__init__("astraea error %d: %s" % (code, text))
+        self.code = code
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError("libastraea.so is not built; run `python -m paper_2506_05096_b200.build` "
+                              "(the CUDA library is the only implementation: there is no fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        c_i, c_f, c_p, c_sz, c_i64, c_u = (ctypes.c_int, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t,
+                                           ctypes.c_int64, ctypes.c_uint32)
+        L.astraea_score.argtypes = [c_p, c_p, c_p, c_p, c_p, c_i, c_i, c_i, c_i, c_i, c_f, c_f, c_i, c_i, c_p]
+        L.astraea_select.argtypes = [c_p, c_i, c_i, c_i, c_i, c_p, c_p, c_p, c_p, c_sz, c_p]
+        L.astraea_sparse_attn.argtypes = [c_p, c_p, c_p] + [c_i64] * 9 + [c_p, c_i, c_p, c_i, c_p, c_p,
+                                                                         c_i, c_i, c_i, c_i, c_f, c_u, c_p, c_sz, c_p]
+        L.astraea_scatter_reuse.argtypes = [c_p, c_p, c_p, c_i, c_i, c_i, c_i, c_u, c_p]
+        L.astraea_step.argtypes = [c_p] * 11 + [c_i] * 6 + [c_f, c_f, c_i, c_i, c_p, c_sz, c_p]
+        L.astraea_session_create.argtypes = [ctypes.POINTER(c_p), c_i, c_i, c_i, c_i, c_i]
+        L.astraea_session_destroy.argtypes = [c_p]
+        L.astraea_session_destroy.restype = None
+        L.astraea_step_host.argtypes = [c_p, c_p, c_p, c_p, c_p, c_p, c_i, c_f, c_f, c_i, c_i]
+        L.astraea_workspace_bytes.argtypes = [c_i] * 6
+        L.astraea_workspace_bytes.restype = c_sz
+        L.astraea_budget_to_k.argtypes = [c_i, c_i]
+        L.astraea_poll_error.argtypes = [c_p, c_p]
+        L.astraea_last_error.restype = ctypes.c_char_p
+        L.astraea_version.restype = ctypes.c_char_p
+        for name in ("astraea_score", "astraea_select", "astraea_sparse_attn", "astraea_scatter_reuse",
+                     "astraea_step", "astraea_session_create", "astraea_step_host", "astraea_budget_to_k",
+                     "astraea_poll_error"):
+            getattr(L, name).restype = ctypes.c_int32
+        _lib = L
+    return _lib
+
+
+def _check(rc: int) -> None:
+    if rc != OK:
+        raise AstraeaError(rc, lib().astraea_last_error().decode())
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def astraea_version() -> str:
+    return lib().astraea_version().decode()
+
+
+def astraea_last_error() -> str:
+    return lib().astraea_last_error().decode()
+
+
+def astraea_budget_to_k(n_sel: int, theta_permille: int) -> int:
+    k = lib().astraea_budget_to_k(n_sel, theta_permille)
+    if k < 0:
+        raise AstraeaError(k, "bad budget")
+    return k
+
+
+def astraea_workspace_bytes(op: int, B: int, H: int, N: int, M: int, d: int) -> int:
+    return int(lib().astraea_workspace_bytes(op, B, H, N, M, d))
+
+
+def new_workspace(op: int, B: int, H: int, N: int, M: int, d: int, device="cuda") -> torch.Tensor:
+    """A zeroed workspace of the size the op asks for (caller-owned device memory)."""
+    return torch.zeros(max(256, astraea_workspace_bytes(op, B, H, N, M, d)), dtype=torch.uint8, device=device)
+
+
+def astraea_score(x_cur, x_ref, lse, n_skip, score, B, N, N_sel, D, H, w_alpha=1.0, w_beta=1.0,
+                  delta_mode=DELTA_MEAN_ABS, lse_mode=LSE_SUM_EXP, stream=None) -> None:
+    _check(lib().astraea_score(_ptr(x_cur), _ptr(x_ref), _ptr(lse), _ptr(n_skip), _ptr(score),
+                               B, N, N_sel, D, H, w_alpha, w_beta, delta_mode, lse_mode, _stream(stream)))
+
+
+def astraea_select(score, B, N_sel, k, n_always, idx_sel, idx_rem, n_skip, workspace, stream=None) -> None:
+    _check(lib().astraea_select(_ptr(score), B, N_sel, k, n_always, _ptr(idx_sel), _ptr(idx_rem), _ptr(n_skip),
+                                _ptr(workspace), workspace.numel() if workspace is not None else 0, _stream(stream)))
+
+
+def astraea_sparse_attn(q, k, v, q_strides, k_strides, v_strides, q_idx, M, out, lse_out, B, H, N, d,
+                        scale=0.0, flags=0, workspace=None, kv_idx=None, M_kv=0, stream=None) -> None:
+    """q_strides etc. are (batch, head, token) element strides."""
+    _check(lib().astraea_sparse_attn(_ptr(q), _ptr(k), _ptr(v), *q_strides, *k_strides, *v_strides,
+                                     _ptr(q_idx), M, _ptr(kv_idx), M_kv, _ptr(out), _ptr(lse_out),
+                                     B, H, N, d, scale, flags, _ptr(workspace),
+                                     workspace.numel() if workspace is not None else 0, _stream(stream)))
+
+
+def astraea_scatter_reuse(cache, rows, idx, B, N, M, row_elems, flags=0, stream=None) -> None:
+    _check(lib().astraea_scatter_reuse(_ptr(cache), _ptr(rows), _ptr(idx), B, N, M, row_elems, flags, _stream(stream)))
+
+
+def astraea_step(x_cur, x_ref, lse_cache, n_skip, q, k, v, out_cache, score, idx_sel, idx_rem,
+                 B, H, N, N_sel, d, k_keep, w_alpha=1.0, w_beta=1.0, delta_mode=DELTA_MEAN_ABS,
+                 lse_mode=LSE_SUM_EXP, workspace=None, stream=None) -> None:
+    _check(lib().astraea_step(_ptr(x_cur), _ptr(x_ref), _ptr(lse_cache), _ptr(n_skip), _ptr(q), _ptr(k), _ptr(v),
+                              _ptr(out_cache), _ptr(score), _ptr(idx_sel), _ptr(idx_rem),
+                              B, H, N, N_sel, d, k_keep, w_alpha, w_beta, delta_mode, lse_mode,
+                              _ptr(workspace), workspace.numel() if workspace is not None else 0, _stream(stream)))
+
+
+def astraea_poll_error(workspace, stream=None) -> None:
+    _check(lib().astraea_poll_error(_ptr(workspace), _stream(stream)))
+
+
+class Session:
+    """Host-buffer session (astraea_session_create / astraea_step_host / astraea_session_destroy)."""
+
+    def __init__(self, B: int, H: int, N: int, N_sel: int, d: int):
+        self._h = ctypes.c_void_p()
+        _check(lib().astraea_session_create(ctypes.byref(self._h), B, H, N, N_sel, d))
+        self.shape = (B, N, H, d)
+
+    def step_host(self, x_cur, q, k, v, out, k_keep, w_alpha=1.0, w_beta=1.0,
+                  delta_mode=DELTA_MEAN_ABS, lse_mode=LSE_SUM_EXP) -> None:
+        """All five tensors are HOST (ideally pinned) bf16 tensors of shape [B,N,H*d]."""
+        for t in (x_cur, q, k, v, out):
+            assert not t.is_cuda and t.is_contiguous()
+        _check(lib().astraea_step_host(self._h, _ptr(x_cur), _ptr(q), _ptr(k), _ptr(v), _ptr(out), k_keep,
+                                       w_alpha, w_beta, delta_mode, lse_mode))
+
+    def close(self) -> None:
+        if self._h:
+            lib().astraea_session_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def bhnd_strides(N: int, H: int, d: int):
+    """(batch, head, token) element strides of a contiguous [B, N, H, d] tensor."""
+    return (N * H * d, d, H * d)

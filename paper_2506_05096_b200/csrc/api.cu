@@ -1,0 +1,275 @@
+// extern "C" entry points of the astraea library: argument validation on the host, then the
+// kernel launchers.  No C++ exception crosses this boundary.
+#include <stdarg.h>
+#include <string.h>
+
+#include <new>
+
+#include "common.cuh"
+
+namespace astraea {
+
+static thread_local char g_err[512] = "";
+
+void set_error(const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+}
+
+int32_t fail(int32_t code, const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+int32_t check_launch(const char *what) {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+    return ASTRAEA_OK;
+}
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace astraea
+
+using namespace astraea;
+
+#define REQUIRE(cond, ...) do { if (!(cond)) return fail(ASTRAEA_ERR_INVALID_ARG, __VA_ARGS__); } while (0)
+
+extern "C" {
+
+const char *astraea_last_error(void) { return g_err; }
+const char *astraea_version(void) { return "astraea-b200 0.1 (sm_100a)"; }
+
+int32_t astraea_budget_to_k(int n_sel, int theta_permille) {
+    if (n_sel < 0 || theta_permille < 0 || theta_permille > 1000) return ASTRAEA_ERR_INVALID_ARG;
+    return (int32_t)(((int64_t)n_sel * theta_permille) / 1000);
+}
+
+size_t astraea_workspace_bytes(int op, int B, int H, int N, int M, int d) {
+    switch (op) {
+    case ASTRAEA_OP_SELECT: return select_workspace_bytes(B, N);
+    case ASTRAEA_OP_SPARSE_ATTN: return attn_workspace_bytes(B, H, N, M, d);
+    case ASTRAEA_OP_STEP: return attn_workspace_bytes(B, H, N, M, d) + align_up(select_workspace_bytes(B, N), 256);
+    default: return 0;
+    }
+}
+
+int32_t astraea_score(const void *x_cur, const void *x_ref, const float *lse, const int32_t *n_skip,
+                      float *score, int B, int N, int N_sel, int D, int H,
+                      float w_alpha, float w_beta, int delta_mode, int lse_mode, void *stream)
+{
+    REQUIRE(B > 0 && N > 0 && D > 0 && H > 0, "astraea_score: B, N, D, H must be positive");
+    REQUIRE(N_sel >= 0 && N_sel <= N, "astraea_score: N_sel=%d outside [0, N=%d]", N_sel, N);
+    REQUIRE(D % 8 == 0, "astraea_score: D=%d must be a multiple of 8 (16-byte rows)", D);
+    REQUIRE(x_cur && x_ref && score, "astraea_score: null x_cur, x_ref or score");
+    REQUIRE(aligned16(x_cur) && aligned16(x_ref), "astraea_score: x_cur / x_ref must be 16-byte aligned");
+    if (delta_mode < 0 || delta_mode > 2 || lse_mode < 0 || lse_mode > 1)
+        return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_score: unknown delta_mode %d or lse_mode %d", delta_mode, lse_mode);
+    return launch_score(x_cur, x_ref, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, delta_mode,
+                        lse_mode, (cudaStream_t)stream);
+}
+
+int32_t astraea_select(const float *score, int B, int N_sel, int k, int n_always,
+                       int32_t *idx_sel, int32_t *idx_rem, int32_t *n_skip,
+                       void *workspace, size_t workspace_bytes, void *stream)
+{
+    REQUIRE(B > 0 && N_sel >= 0 && n_always >= 0, "astraea_select: bad sizes");
+    REQUIRE(k >= 0 && k <= N_sel, "astraea_select: k=%d outside [0, N_sel=%d]", k, N_sel);
+    REQUIRE(score || N_sel == 0, "astraea_select: null score");
+    REQUIRE(idx_sel || (k + n_always) == 0, "astraea_select: null idx_sel");
+    if (workspace_bytes < select_workspace_bytes(B, N_sel) || !workspace)
+        return fail(ASTRAEA_ERR_WORKSPACE_TOO_SMALL, "astraea_select: workspace of %zu bytes, need %zu",
+                    workspace_bytes, select_workspace_bytes(B, N_sel));
+    REQUIRE(aligned16(workspace), "astraea_select: workspace must be 16-byte aligned");
+    return launch_select(score, B, N_sel, k, n_always, idx_sel, idx_rem, n_skip, workspace, (cudaStream_t)stream);
+}
+
+int32_t astraea_sparse_attn(const void *q, const void *k, const void *v,
+                            int64_t q_sb, int64_t q_sh, int64_t q_sn,
+                            int64_t k_sb, int64_t k_sh, int64_t k_sn,
+                            int64_t v_sb, int64_t v_sh, int64_t v_sn,
+                            const int32_t *q_idx, int M, const int32_t *kv_idx, int M_kv,
+                            void *out, float *lse_out,
+                            int B, int H, int N, int d, float scale, uint32_t flags,
+                            void *workspace, size_t workspace_bytes, void *stream)
+{
+    (void)M_kv;
+    REQUIRE(B > 0 && H > 0 && N > 0 && d > 0, "astraea_sparse_attn: B, H, N, d must be positive");
+    REQUIRE(M >= 0 && M <= N, "astraea_sparse_attn: M=%d outside [0, N=%d]", M, N);
+    if (d != 64 && d != 72 && d != 128)
+        return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_sparse_attn: head_dim %d not in {64, 72, 128}", d);
+    if (kv_idx) return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_sparse_attn: kv_idx (select-Q-and-K ablation) is not built");
+    if (flags & ~ASTRAEA_ATTN_COMPACT_OUT) return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_sparse_attn: unknown flags 0x%x", flags);
+    REQUIRE(q && k && v && out, "astraea_sparse_attn: null q, k, v or out");
+    REQUIRE(aligned16(q) && aligned16(k) && aligned16(v) && aligned16(out), "astraea_sparse_attn: q, k, v, out must be 16-byte aligned");
+    REQUIRE(q_sn % 8 == 0 && k_sn % 8 == 0 && v_sn % 8 == 0 && q_sh % 8 == 0 && k_sh % 8 == 0 && v_sh % 8 == 0 &&
+            q_sb % 8 == 0 && k_sb % 8 == 0 && v_sb % 8 == 0,
+            "astraea_sparse_attn: strides must be multiples of 8 elements (16 bytes)");
+    REQUIRE(q_sn >= d && k_sn >= d && v_sn >= d && q_sh > 0 && k_sh > 0 && v_sh > 0 && q_sb >= 0 && k_sb >= 0 && v_sb >= 0,
+            "astraea_sparse_attn: strides must be positive and token stride >= head_dim");
+    REQUIRE(scale >= 0.f, "astraea_sparse_attn: scale must be >= 0 (0 selects 1/sqrt(d))");
+    if (!workspace || workspace_bytes < attn_workspace_bytes(B, H, N, M, d))
+        return fail(ASTRAEA_ERR_WORKSPACE_TOO_SMALL, "astraea_sparse_attn: workspace of %zu bytes, need %zu",
+                    workspace_bytes, attn_workspace_bytes(B, H, N, M, d));
+    REQUIRE((reinterpret_cast<uintptr_t>(workspace) & 255u) == 0, "astraea_sparse_attn: workspace must be 256-byte aligned");
+    if (M == 0) return ASTRAEA_OK;
+    AttnArgs a;
+    a.q = q; a.k = k; a.v = v;
+    a.q_sb = q_sb; a.q_sh = q_sh; a.q_sn = q_sn;
+    a.k_sb = k_sb; a.k_sh = k_sh; a.k_sn = k_sn;
+    a.v_sb = v_sb; a.v_sh = v_sh; a.v_sn = v_sn;
+    a.q_idx = q_idx; a.M = M; a.out = out; a.lse_out = lse_out;
+    a.B = B; a.H = H; a.N = N; a.d = d;
+    a.scale = (scale == 0.f) ? 1.0f / sqrtf((float)d) : scale;
+    a.flags = flags;
+    a.err_word = reinterpret_cast<int *>(workspace);
+    return launch_sparse_attn(a, (cudaStream_t)stream);
+}
+
+int32_t astraea_scatter_reuse(void *cache, const void *rows, const int32_t *idx,
+                              int B, int N, int M, int row_elems, uint32_t flags, void *stream)
+{
+    REQUIRE(B > 0 && N > 0 && row_elems > 0, "astraea_scatter_reuse: B, N, row_elems must be positive");
+    REQUIRE(M >= 0 && M <= N, "astraea_scatter_reuse: M=%d outside [0, N=%d]", M, N);
+    REQUIRE(row_elems % 8 == 0, "astraea_scatter_reuse: row_elems=%d must be a multiple of 8", row_elems);
+    if (flags & ~ASTRAEA_SCATTER_SRC_FULL) return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_scatter_reuse: unknown flags 0x%x", flags);
+    if (M == 0) return ASTRAEA_OK;
+    REQUIRE(cache && rows && idx, "astraea_scatter_reuse: null cache, rows or idx");
+    REQUIRE(aligned16(cache) && aligned16(rows), "astraea_scatter_reuse: cache / rows must be 16-byte aligned");
+    return launch_scatter(cache, rows, idx, B, N, M, row_elems, flags, (cudaStream_t)stream);
+}
+
+int32_t astraea_step(const void *x_cur, void *x_ref, float *lse_cache, int32_t *n_skip,
+                     const void *q, const void *k, const void *v, void *out_cache,
+                     float *score, int32_t *idx_sel, int32_t *idx_rem,
+                     int B, int H, int N, int N_sel, int d, int k_keep,
+                     float w_alpha, float w_beta, int delta_mode, int lse_mode,
+                     void *workspace, size_t workspace_bytes, void *stream)
+{
+    REQUIRE(N_sel >= 0 && N_sel <= N, "astraea_step: N_sel=%d outside [0, N=%d]", N_sel, N);
+    REQUIRE(k_keep >= 0 && k_keep <= N_sel, "astraea_step: k_keep=%d outside [0, N_sel=%d]", k_keep, N_sel);
+    const int n_always = N - N_sel;
+    const int M = k_keep + n_always;
+    const int D = H * d;
+    const size_t attn_ws = attn_workspace_bytes(B, H, N, M, d);
+    if (!workspace || workspace_bytes < astraea_workspace_bytes(ASTRAEA_OP_STEP, B, H, N, M, d))
+        return fail(ASTRAEA_ERR_WORKSPACE_TOO_SMALL, "astraea_step: workspace of %zu bytes, need %zu", workspace_bytes,
+                    astraea_workspace_bytes(ASTRAEA_OP_STEP, B, H, N, M, d));
+    REQUIRE(score && (idx_sel || M == 0), "astraea_step: null score or idx_sel");
+    char *ws = reinterpret_cast<char *>(workspace);
+    int32_t rc = astraea_score(x_cur, x_ref, lse_cache, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta,
+                               delta_mode, lse_mode, stream);
+    if (rc != ASTRAEA_OK) return rc;
+    rc = astraea_select(score, B, N_sel, k_keep, n_always, idx_sel, idx_rem, n_skip, ws + attn_ws,
+                        workspace_bytes - attn_ws, stream);
+    if (rc != ASTRAEA_OK) return rc;
+    const int64_t sb = (int64_t)N * D, sh = d, sn = D;
+    rc = astraea_sparse_attn(q, k, v, sb, sh, sn, sb, sh, sn, sb, sh, sn, idx_sel, M, nullptr, 0, out_cache,
+                             lse_cache, B, H, N, d, 0.f, 0u, ws, attn_ws, stream);
+    if (rc != ASTRAEA_OK) return rc;
+    // the reference inputs of the tokens that were computed become the current inputs
+    return astraea_scatter_reuse(x_ref, x_cur, idx_sel, B, N, M, D, ASTRAEA_SCATTER_SRC_FULL, stream);
+}
+
+int32_t astraea_poll_error(void *workspace, void *stream)
+{
+    REQUIRE(workspace, "astraea_poll_error: null workspace");
+    int word = 0;
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaMemcpy(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_poll_error: %s", cudaGetErrorString(e));
+    if (word != 0) cudaMemset(workspace, 0, sizeof(int));
+    if (word == kErrTimeout) return fail(ASTRAEA_ERR_TIMEOUT, "a bounded device-side wait gave up");
+    if (word == kErrBadIndex) return fail(ASTRAEA_ERR_BAD_INDEX, "an index was out of range");
+    return ASTRAEA_OK;
+}
+
+// ------------------------------------------------------------------ host-buffer session
+struct astraea_session {
+    int B, H, N, N_sel, d;
+    size_t tensor_bytes;
+    void *x_cur, *x_ref, *q, *k, *v, *out_cache;
+    float *lse_cache, *score;
+    int32_t *n_skip, *idx_sel, *idx_rem;
+    void *workspace;
+    size_t workspace_bytes;
+    cudaStream_t stream;
+    int steps;
+};
+
+void astraea_session_destroy(astraea_session *s)
+{
+    if (!s) return;
+    void *bufs[] = {s->x_cur, s->x_ref, s->q, s->k, s->v, s->out_cache, s->lse_cache, s->score,
+                    s->n_skip, s->idx_sel, s->idx_rem, s->workspace};
+    for (void *p : bufs) if (p) cudaFree(p);
+    if (s->stream) cudaStreamDestroy(s->stream);
+    delete s;
+}
+
+int32_t astraea_session_create(astraea_session **session, int B, int H, int N, int N_sel, int d)
+{
+    REQUIRE(session, "astraea_session_create: null session pointer");
+    *session = nullptr;
+    REQUIRE(B > 0 && H > 0 && N > 0 && N_sel >= 0 && N_sel <= N, "astraea_session_create: bad sizes");
+    if (d != 64 && d != 72 && d != 128) return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_session_create: head_dim %d", d);
+    astraea_session *s = new (std::nothrow) astraea_session();
+    if (!s) return fail(ASTRAEA_ERR_CUDA, "astraea_session_create: out of host memory");
+    memset(s, 0, sizeof(*s));
+    s->B = B; s->H = H; s->N = N; s->N_sel = N_sel; s->d = d;
+    s->tensor_bytes = (size_t)B * N * H * d * 2;
+    s->workspace_bytes = astraea_workspace_bytes(ASTRAEA_OP_STEP, B, H, N, N, d);
+    cudaError_t e = cudaStreamCreateWithFlags(&s->stream, cudaStreamNonBlocking);
+    void **big[] = {&s->x_cur, &s->x_ref, &s->q, &s->k, &s->v, &s->out_cache};
+    for (void **p : big) if (e == cudaSuccess) e = cudaMalloc(p, s->tensor_bytes);
+    if (e == cudaSuccess) e = cudaMalloc((void **)&s->lse_cache, (size_t)B * H * N * 4);
+    if (e == cudaSuccess) e = cudaMalloc((void **)&s->score, (size_t)B * (N_sel + 1) * 4);
+    if (e == cudaSuccess) e = cudaMalloc((void **)&s->n_skip, (size_t)B * (N_sel + 1) * 4);
+    if (e == cudaSuccess) e = cudaMalloc((void **)&s->idx_sel, (size_t)B * N * 4);
+    if (e == cudaSuccess) e = cudaMalloc((void **)&s->idx_rem, (size_t)B * (N_sel + 1) * 4);
+    if (e == cudaSuccess) e = cudaMalloc(&s->workspace, s->workspace_bytes);
+    if (e == cudaSuccess) e = cudaMemsetAsync(s->workspace, 0, s->workspace_bytes, s->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(s->n_skip, 0, (size_t)B * (N_sel + 1) * 4, s->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(s->lse_cache, 0, (size_t)B * H * N * 4, s->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(s->out_cache, 0, s->tensor_bytes, s->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s->stream);
+    if (e != cudaSuccess) {
+        int32_t rc = fail(ASTRAEA_ERR_CUDA, "astraea_session_create: %s", cudaGetErrorString(e));
+        astraea_session_destroy(s);
+        return rc;
+    }
+    *session = s;
+    return ASTRAEA_OK;
+}
+
+int32_t astraea_step_host(astraea_session *s, const void *x_cur, const void *q, const void *k,
+                          const void *v, void *out, int k_keep,
+                          float w_alpha, float w_beta, int delta_mode, int lse_mode)
+{
+    REQUIRE(s && x_cur && q && k && v && out, "astraea_step_host: null argument");
+    REQUIRE(k_keep >= 0 && k_keep <= s->N_sel, "astraea_step_host: k_keep=%d outside [0, N_sel=%d]", k_keep, s->N_sel);
+    REQUIRE(s->steps > 0 || k_keep == s->N_sel, "astraea_step_host: the first step of a session must compute every token (k_keep = N_sel)");
+    cudaError_t e = cudaMemcpyAsync(s->x_cur, x_cur, s->tensor_bytes, cudaMemcpyHostToDevice, s->stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(s->q, q, s->tensor_bytes, cudaMemcpyHostToDevice, s->stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(s->k, k, s->tensor_bytes, cudaMemcpyHostToDevice, s->stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(s->v, v, s->tensor_bytes, cudaMemcpyHostToDevice, s->stream);
+    if (e == cudaSuccess && s->steps == 0)   // no earlier step: the reference inputs are the current ones
+        e = cudaMemcpyAsync(s->x_ref, s->x_cur, s->tensor_bytes, cudaMemcpyDeviceToDevice, s->stream);
+    if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_step_host (copy in): %s", cudaGetErrorString(e));
+    int32_t rc = astraea_step(s->x_cur, s->x_ref, s->lse_cache, s->n_skip, s->q, s->k, s->v, s->out_cache,
+                              s->score, s->idx_sel, s->idx_rem, s->B, s->H, s->N, s->N_sel, s->d, k_keep,
+                              w_alpha, w_beta, delta_mode, lse_mode, s->workspace, s->workspace_bytes, s->stream);
+    if (rc != ASTRAEA_OK) return rc;
+    e = cudaMemcpyAsync(out, s->out_cache, s->tensor_bytes, cudaMemcpyDeviceToHost, s->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s->stream);
+    if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_step_host (copy out): %s", cudaGetErrorString(e));
+    s->steps++;
+    return astraea_poll_error(s->workspace, s->stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,437 @@
+// astraea_sparse_attn: out[i] = Softmax(q_i K^T * scale) V for the selected query rows i
+// against ALL keys/values, written in place over the cached output (Algorithm 1 lines 6-7;
+// Section 3.2 "Sparse Attention").
+//
+// One CTA per (128 selected queries, head, batch).  Warp roles:
+//   warps 0-3  softmax: gather the CTA's Q rows into 128B-swizzled shared memory, then per
+//              key tile read S from TMEM (one thread per query row), online softmax in the
+//              log2 domain with lazy rescaling of O, write P (bf16) back to TMEM over S,
+//              and at the end normalise O and scatter it to the rows q_idx names;
+//   warp 4     TMA producer: K and V tiles (128 keys) into multi-stage swizzled buffers;
+//   warp 5     tcgen05.mma issuer: S = Q K^T (SS, K-major operands), O += P V (P from TMEM,
+//              V as an MN-major shared-memory operand); owns the TMEM allocation.
+// TMEM columns: S/P buffer 0 [0,128), S/P buffer 1 [128,256), O [256, 256+d).
+// Every mbarrier wait is bounded; on a timeout the CTA raises the error word and leaves.
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace astraea {
+namespace {
+
+using namespace ptx;
+
+constexpr int kBlockM = 128;
+constexpr int kBlockN = 128;
+constexpr int kThreads = 192;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColO = 256;
+constexpr float kRescaleThreshold = 8.0f;        // log2 units: P stays below 2^8
+constexpr uint64_t kWaitLimitNs = 1000000000ull; // bounded waits: one second
+
+template <int DH> struct Cfg {
+    static constexpr int kChunks = DH / 64;                       // 64-column (128-byte) swizzle chunks
+    static constexpr int kChunkBytes = 128 * 128;                 // 128 rows x 128 bytes
+    static constexpr int kTileBytes = kChunks * kChunkBytes;      // one Q / K / V tile
+    static constexpr int kStages = (DH == 128) ? 3 : 6;
+    static constexpr int kBarBytes = 256;
+    static constexpr int kSmemBytes = kTileBytes * (1 + 2 * kStages) + kBarBytes + 1024;
+};
+
+struct Params {
+    const __nv_bfloat16 *q;
+    int64_t q_sb, q_sh, q_sn;
+    const int32_t *q_idx;
+    int M;
+    __nv_bfloat16 *out;
+    float *lse_out;
+    int N, H;
+    float scale, scale_log2;
+    int compact;
+    int *err_word;
+};
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Bounded mbarrier wait.  Returns false after the limit or once another role has given up.
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err_word) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = globaltimer_ns();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 255u) == 0) {
+            if (*abort_flag) return false;
+            if (globaltimer_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                atomicExch(err_word, kErrTimeout);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+template <int DH>
+__global__ void __launch_bounds__(kThreads, 1)
+sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v, const Params p)
+{
+    using C = Cfg<DH>;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    const uint32_t sQ = smem_base;
+    const uint32_t sK = sQ + C::kTileBytes;
+    const uint32_t sV = sK + C::kStages * C::kTileBytes;
+    const uint32_t bars = sV + C::kStages * C::kTileBytes;
+    // barrier slots (8 bytes each)
+    const uint32_t bar_q = bars;
+    const uint32_t bar_s = bars + 8;                       // [2]
+    const uint32_t bar_p = bars + 24;                      // [2]
+    const uint32_t bar_o = bars + 40;
+    const uint32_t bar_kf = bars + 48;                     // [kStages]
+    const uint32_t bar_ke = bar_kf + 8 * C::kStages;
+    const uint32_t bar_vf = bar_ke + 8 * C::kStages;
+    const uint32_t bar_ve = bar_vf + 8 * C::kStages;
+    static_assert(48 + 32 * C::kStages <= C::kBarBytes, "barrier area too small");
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int m0 = blockIdx.x * kBlockM, h = blockIdx.y, b = blockIdx.z;
+    const int n_tiles = (p.N + kBlockN - 1) / kBlockN;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        mbar_init(bar_q, 128);
+        mbar_init(bar_s, 1); mbar_init(bar_s + 8, 1);
+        mbar_init(bar_p, 128); mbar_init(bar_p + 8, 128);
+        mbar_init(bar_o, 1);
+        for (int s = 0; s < C::kStages; ++s) {
+            mbar_init(bar_kf + 8 * s, 1); mbar_init(bar_ke + 8 * s, 1);
+            mbar_init(bar_vf + 8 * s, 1); mbar_init(bar_ve + 8 * s, 1);
+        }
+        fence_barrier_init();
+    }
+    if (warp == 5) {
+        tmem_alloc(smem_u32(&tmem_slot), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_slot;
+
+    if (warp < 4) {
+        // ------------------------------------------------ gather Q rows (swizzled, K-major)
+        constexpr int kVecPerRow = DH / 8;                 // 16-byte vectors per row
+        constexpr int kRowsPerIter = 32 / kVecPerRow;
+        const int sub = lane / kVecPerRow, c = lane % kVecPerRow;
+        for (int r0 = warp * kRowsPerIter; r0 < kBlockM; r0 += 4 * kRowsPerIter) {
+            const int r = r0 + sub;
+            const int m = m0 + r;
+            uint4 val = make_uint4(0, 0, 0, 0);
+            if (m < p.M) {
+                const int tok = p.q_idx ? __ldg(p.q_idx + (size_t)b * p.M + m) : m;
+                if ((unsigned)tok < (unsigned)p.N) {
+                    const __nv_bfloat16 *src = p.q + (size_t)b * p.q_sb + (size_t)tok * p.q_sn + (size_t)h * p.q_sh + c * 8;
+                    val = __ldg(reinterpret_cast<const uint4 *>(src));
+                }
+            }
+            const uint32_t off = (c >> 3) * C::kChunkBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
+            *reinterpret_cast<uint4 *>(smem_gen + off) = val;
+        }
+        fence_proxy_async_smem();
+        mbar_arrive(bar_q);
+
+        // ------------------------------------------------ online softmax, one thread per query row
+        const int row = tid;                               // TMEM lane
+        const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);
+        const int m = m0 + row;
+        int tok = -1;
+        if (m < p.M) {
+            tok = p.q_idx ? __ldg(p.q_idx + (size_t)b * p.M + m) : m;
+            if ((unsigned)tok >= (unsigned)p.N) { atomicExch(p.err_word, kErrBadIndex); tok = -1; }
+        }
+        const float sl2 = p.scale_log2;
+        float m_ref = -INFINITY, l_sum = 0.f;
+        bool ok = true;
+
+        for (int j = 0; j < n_tiles && ok; ++j) {
+            const int buf = j & 1;
+            ok = wait_bar(bar_s + 8 * buf, (j >> 1) & 1, &abort_flag, p.err_word);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            float s[kBlockN];
+            {
+                uint32_t t0[32], t1[32], t2[32], t3[32];
+                tmem_ld32(t_row + buf * 128, t0);
+                tmem_ld32(t_row + buf * 128 + 32, t1);
+                tmem_ld32(t_row + buf * 128 + 64, t2);
+                tmem_ld32(t_row + buf * 128 + 96, t3);
+                tc_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    s[i] = __uint_as_float(t0[i]);
+                    s[32 + i] = __uint_as_float(t1[i]);
+                    s[64 + i] = __uint_as_float(t2[i]);
+                    s[96 + i] = __uint_as_float(t3[i]);
+                }
+            }
+            const int valid = p.N - j * kBlockN;           // keys of this tile that exist
+            if (valid < kBlockN) {
+#pragma unroll
+                for (int i = 0; i < kBlockN; ++i) if (i >= valid) s[i] = -INFINITY;
+            }
+            float mx = s[0];
+#pragma unroll
+            for (int i = 1; i < kBlockN; ++i) mx = fmaxf(mx, s[i]);
+
+            if (j == 0) {
+                m_ref = mx;
+            } else {
+                const bool need = (mx - m_ref) * sl2 > kRescaleThreshold;
+                if (__any_sync(0xffffffffu, need)) {
+                    float alpha = 1.0f;
+                    if (need) { alpha = ex2((m_ref - mx) * sl2); m_ref = mx; l_sum *= alpha; }
+                    ok = wait_bar(bar_o, (j - 1) & 1, &abort_flag, p.err_word);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int cc = 0; cc < DH / 32; ++cc) {
+                        uint32_t o[32];
+                        tmem_ld32(t_row + kColO + cc * 32, o);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st32(t_row + kColO + cc * 32, o);
+                    }
+                    tc_wait_st();
+                }
+            }
+            const float neg = -m_ref * sl2;
+            float sum = 0.f;
+#pragma unroll
+            for (int i = 0; i < kBlockN; ++i) { s[i] = ex2(fmaf(s[i], sl2, neg)); sum += s[i]; }
+            l_sum += sum;
+            // P as bf16 pairs over the first 64 columns of this S buffer (element 2c in the low half)
+#pragma unroll
+            for (int cc = 0; cc < 2; ++cc) {
+                uint32_t pk[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    __nv_bfloat162 v2 = __floats2bfloat162_rn(s[cc * 64 + 2 * i], s[cc * 64 + 2 * i + 1]);
+                    pk[i] = *reinterpret_cast<uint32_t *>(&v2);
+                }
+                tmem_st32(t_row + buf * 128 + cc * 32, pk);
+            }
+            tc_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar_p + 8 * buf);
+        }
+
+        // ------------------------------------------------ epilogue: normalise and scatter
+        if (ok) {
+            ok = wait_bar(bar_o, (n_tiles - 1) & 1, &abort_flag, p.err_word);
+            ok = __all_sync(0xffffffffu, ok);
+        }
+        if (ok) {
+            tc_fence_after();
+            const float inv_l = 1.0f / l_sum;
+            __nv_bfloat16 *dst = nullptr;
+            if (tok >= 0) {
+                const size_t orow = p.compact ? ((size_t)b * p.M + m) : ((size_t)b * p.N + tok);
+                dst = p.out + (orow * p.H + h) * DH;
+                if (p.lse_out) {
+                    const size_t li = p.compact ? (((size_t)b * p.H + h) * p.M + m) : (((size_t)b * p.H + h) * p.N + tok);
+                    p.lse_out[li] = m_ref * p.scale + logf(l_sum);
+                }
+            }
+#pragma unroll
+            for (int cc = 0; cc < DH / 32; ++cc) {
+                uint32_t o[32];
+                tmem_ld32(t_row + kColO + cc * 32, o);
+                tc_wait_ld();
+                if (dst) {
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(o[v * 8 + 2 * i]) * inv_l,
+                                                                      __uint_as_float(o[v * 8 + 2 * i + 1]) * inv_l);
+                            w[i] = *reinterpret_cast<uint32_t *>(&v2);
+                        }
+                        *reinterpret_cast<uint4 *>(dst + cc * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                }
+            }
+        }
+    } else if (warp == 4) {
+        // ------------------------------------------------ TMA producer
+        if (lane == 0) {
+            prefetch_tensormap(&tmap_k);
+            prefetch_tensormap(&tmap_v);
+            int issued_k = 0, issued_v = 0;
+            bool ok = true;
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const int st = j % C::kStages;
+                const uint32_t ph = (j / C::kStages) & 1;
+                ok = wait_bar(bar_ke + 8 * st, ph ^ 1, &abort_flag, p.err_word);
+                if (!ok) break;
+                mbar_arrive_expect_tx(bar_kf + 8 * st, C::kTileBytes);
+#pragma unroll
+                for (int ch = 0; ch < C::kChunks; ++ch)
+                    tma_load_4d(sK + st * C::kTileBytes + ch * C::kChunkBytes, &tmap_k, bar_kf + 8 * st,
+                                ch * 64, j * kBlockN, h, b);
+                issued_k = j + 1;
+                ok = wait_bar(bar_ve + 8 * st, ph ^ 1, &abort_flag, p.err_word);
+                if (!ok) break;
+                mbar_arrive_expect_tx(bar_vf + 8 * st, C::kTileBytes);
+#pragma unroll
+                for (int ch = 0; ch < C::kChunks; ++ch)
+                    tma_load_4d(sV + st * C::kTileBytes + ch * C::kChunkBytes, &tmap_v, bar_vf + 8 * st,
+                                ch * 64, j * kBlockN, h, b);
+                issued_v = j + 1;
+            }
+            if (!ok) {
+                // leaving early: let the copies already issued land before the CTA's shared memory is released
+                for (int j = (issued_k > C::kStages ? issued_k - C::kStages : 0); j < issued_k; ++j)
+                    wait_bar(bar_kf + 8 * (j % C::kStages), (j / C::kStages) & 1, &abort_flag, p.err_word);
+                for (int j = (issued_v > C::kStages ? issued_v - C::kStages : 0); j < issued_v; ++j)
+                    wait_bar(bar_vf + 8 * (j % C::kStages), (j / C::kStages) & 1, &abort_flag, p.err_word);
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_qk = idesc_bf16(kBlockM, kBlockN, false);
+            constexpr uint32_t idesc_pv = idesc_bf16(kBlockM, DH, true);
+            bool ok = wait_bar(bar_q, 0, &abort_flag, p.err_word);
+            auto issue_qk = [&](int j) -> bool {
+                const int st = j % C::kStages;
+                if (!wait_bar(bar_kf + 8 * st, (j / C::kStages) & 1, &abort_flag, p.err_word)) return false;
+                tc_fence_after();
+                const uint32_t d_s = tmem + (j & 1) * 128;
+#pragma unroll
+                for (int ks = 0; ks < DH / 16; ++ks) {
+                    const uint32_t off = (ks >> 2) * C::kChunkBytes + (ks & 3) * 32;
+                    mma_ss(d_s, smem_desc(sQ + off, 16, 1024, kSwizzle128B),
+                           smem_desc(sK + st * C::kTileBytes + off, 16, 1024, kSwizzle128B), idesc_qk, ks > 0);
+                }
+                tc_commit(bar_s + 8 * (j & 1));
+                tc_commit(bar_ke + 8 * st);
+                return true;
+            };
+            if (ok) ok = issue_qk(0);
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                if (j + 1 < n_tiles) { ok = issue_qk(j + 1); if (!ok) break; }
+                ok = wait_bar(bar_p + 8 * (j & 1), (j >> 1) & 1, &abort_flag, p.err_word);
+                if (!ok) break;
+                const int st = j % C::kStages;
+                ok = wait_bar(bar_vf + 8 * st, (j / C::kStages) & 1, &abort_flag, p.err_word);
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < kBlockN / 16; ++ks) {
+                    mma_ts(tmem + kColO, tmem + (j & 1) * 128 + ks * 8,
+                           smem_desc(sV + st * C::kTileBytes + ks * 2048, C::kChunkBytes, 1024, kSwizzle128B),
+                           idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+                }
+                tc_commit(bar_o);
+                tc_commit(bar_ve + 8 * st);
+            }
+        }
+        __syncwarp();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) tmem_dealloc(tmem, kTmemCols);
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// K or V as a 4-D tensor (d, N, H, B) with 128-byte-swizzled boxes of 64 columns x 128 tokens
+int32_t make_kv_map(CUtensorMap *map, const void *base, int B, int H, int N, int d,
+                    int64_t sb, int64_t sh, int64_t sn)
+{
+    EncodeTiledFn enc = get_encode_fn();
+    if (!enc) return fail(ASTRAEA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)H, (cuuint64_t)B};
+    cuuint64_t strides[3] = {(cuuint64_t)sn * 2, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)kBlockN, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(ASTRAEA_ERR_INVALID_ARG, "tensor map rejected (CUresult %d): check K/V strides and alignment", (int)r);
+    return ASTRAEA_OK;
+}
+
+template <int DH>
+int32_t launch_dh(const AttnArgs &a, cudaStream_t stream)
+{
+    using C = Cfg<DH>;
+    CUtensorMap mk, mv;
+    int32_t rc = make_kv_map(&mk, a.k, a.B, a.H, a.N, a.d, a.k_sb, a.k_sh, a.k_sn);
+    if (rc != ASTRAEA_OK) return rc;
+    rc = make_kv_map(&mv, a.v, a.B, a.H, a.N, a.d, a.v_sb, a.v_sh, a.v_sn);
+    if (rc != ASTRAEA_OK) return rc;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(sparse_attn_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
+            return check_launch("astraea_sparse_attn (shared memory attribute)");
+        attr_set = true;
+    }
+    Params p;
+    p.q = reinterpret_cast<const __nv_bfloat16 *>(a.q);
+    p.q_sb = a.q_sb; p.q_sh = a.q_sh; p.q_sn = a.q_sn;
+    p.q_idx = a.q_idx; p.M = a.M;
+    p.out = reinterpret_cast<__nv_bfloat16 *>(a.out);
+    p.lse_out = a.lse_out;
+    p.N = a.N; p.H = a.H;
+    p.scale = a.scale;
+    p.scale_log2 = a.scale * 1.4426950408889634f;
+    p.compact = (a.flags & ASTRAEA_ATTN_COMPACT_OUT) ? 1 : 0;
+    p.err_word = a.err_word;
+    dim3 grid((a.M + kBlockM - 1) / kBlockM, a.H, a.B);
+    sparse_attn_kernel<DH><<<grid, kThreads, C::kSmemBytes, stream>>>(mk, mv, p);
+    return check_launch("astraea_sparse_attn");
+}
+
+}  // namespace
+
+size_t attn_workspace_bytes(int, int, int, int, int) { return 256; }
+
+int32_t launch_sparse_attn(const AttnArgs &a, cudaStream_t stream)
+{
+    switch (a.d) {
+    case 64: return launch_dh<64>(a, stream);
+    case 128: return launch_dh<128>(a, stream);
+    default: return fail(ASTRAEA_ERR_UNSUPPORTED, "head_dim %d is not supported", a.d);
+    }
+}
+
+}  // namespace astraea

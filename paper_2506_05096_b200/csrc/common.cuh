@@ -1,0 +1,49 @@
+// Shared host/device helpers of the astraea library (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include "../../include/astraea.h"
+
+namespace astraea {
+
+constexpr int kNumSMs = 148;            // B200: 2 dies x 74 SMs
+constexpr int kErrTimeout = 1;          // values of the device-side error word
+constexpr int kErrBadIndex = 2;
+
+// thread-local text of the last failure
+void set_error(const char *fmt, ...);
+int32_t fail(int32_t code, const char *fmt, ...);
+int32_t check_launch(const char *what);
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// kernel launchers (one per .cu file)
+int32_t launch_score(const void *x_cur, const void *x_ref, const float *lse, const int32_t *n_skip,
+                     float *score, int B, int N, int N_sel, int D, int H, float w_alpha, float w_beta,
+                     int delta_mode, int lse_mode, cudaStream_t stream);
+int32_t launch_select(const float *score, int B, int N_sel, int k, int n_always, int32_t *idx_sel,
+                      int32_t *idx_rem, int32_t *n_skip, void *workspace, cudaStream_t stream);
+size_t select_workspace_bytes(int B, int N_sel);
+int32_t launch_scatter(void *cache, const void *rows, const int32_t *idx, int B, int N, int M,
+                       int row_elems, uint32_t flags, cudaStream_t stream);
+
+struct AttnArgs {
+    const void *q, *k, *v;
+    int64_t q_sb, q_sh, q_sn, k_sb, k_sh, k_sn, v_sb, v_sh, v_sn;
+    const int32_t *q_idx;
+    int M;
+    void *out;
+    float *lse_out;
+    int B, H, N, d;
+    float scale;
+    uint32_t flags;
+    int *err_word;
+};
+int32_t launch_sparse_attn(const AttnArgs &a, cudaStream_t stream);
+size_t attn_workspace_bytes(int B, int H, int N, int M, int d);
+
+}  // namespace astraea

@@ -1,0 +1,345 @@
+"""Parity of the CUDA library (through its C ABI) with the CPU oracle, element by element,
+on the same seeded inputs.  Integer / index results must be bit-exact; floating-point
+results within the stated tolerances (attention: max-abs 2e-2, mean-abs 2e-3 against the
+fp64 oracle on the bf16-rounded inputs; LSE 1e-3; scores 1e-5 relative)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2506_05096_b200 import binding as A
+from paper_2506_05096_b200 import synth
+from helpers import bf16_dev_to_f64, dev, f64, to_dev_bf16
+
+pytestmark = pytest.mark.gpu
+
+ATTN_MAX_ABS, ATTN_MEAN_ABS, LSE_ABS, SCORE_RTOL = 2e-2, 2e-3, 1e-3, 1e-5
+
+
+# ---------------------------------------------------------------------- score
+def _score_case(oracle, w, seed, n_sel, delta_mode, lse_mode, use_lse=True, use_n=True, w_alpha=1.0, w_beta=1.0):
+    inp = synth.make_step_inputs(w, seed, parts=("x_ref", "x_cur"))
+    B, N, D, H = w.B, w.N, w.D, w.H
+    lse = inp["lse"] if use_lse else None
+    if lse is not None and lse_mode == A.LSE_SUM_EXP:
+        lse = (lse - np.float32(math.log(N))).astype(np.float32)      # keep exp() moderate for any N
+    n_skip = inp["n_skip"][:, :n_sel].copy() if use_n else None
+    want = oracle.score(f64(inp["x_cur"]), f64(inp["x_ref"]), lse, n_skip, n_sel=n_sel, H=H, w_alpha=w_alpha,
+                        w_beta=w_beta, delta_mode=delta_mode, lse_mode=lse_mode)
+    out = torch.full((B, n_sel), float("nan"), device="cuda")
+    A.astraea_score(to_dev_bf16(inp["x_cur"]), to_dev_bf16(inp["x_ref"]),
+                    None if lse is None else dev(lse), None if n_skip is None else dev(n_skip), out,
+                    B, N, n_sel, D, H, w_alpha, w_beta, delta_mode, lse_mode)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy().astype(np.float64)
+    err = np.abs(got - want) / np.maximum(np.abs(want), 1e-30)
+    assert err.max() < SCORE_RTOL, err.max()
+    return got, want
+
+
+@pytest.mark.parametrize("delta_mode", [A.DELTA_MEAN_ABS, A.DELTA_MEAN_SQ, A.DELTA_MEAN_SIGNED])
+@pytest.mark.parametrize("lse_mode", [A.LSE_SUM_EXP, A.LSE_LOG])
+def test_score_tiny_all_modes(oracle, delta_mode, lse_mode):
+    w = synth.scaled(synth.WORKLOADS["tiny"], n_skip_max=5)
+    # the signed mean cancels to ~0: compare it in absolute terms through a w_beta = 1 offset
+    _score_case(oracle, w, 0, w.N_v, delta_mode, lse_mode, w_alpha=0.5, w_beta=1.0)
+
+
+@pytest.mark.parametrize("name,N_v,N_t", [("cogvideox", 1013, 26), ("opensora", 777, 0), ("hunyuan", 530, 0)])
+def test_score_workload_shapes_ragged(oracle, name, N_v, N_t):
+    w = synth.scaled(synth.WORKLOADS[name], N_v=N_v, N_t=N_t)
+    _score_case(oracle, w, 1, N_v, A.DELTA_MEAN_ABS, A.LSE_SUM_EXP)
+
+
+def test_score_without_lse_and_counters_and_odd_width(oracle):
+    w = synth.Workload("odd", B=2, H=3, d=24, N_v=70, N_t=3)      # D = 72: 9 vectors per row, a ragged tail
+    _score_case(oracle, w, 2, 70, A.DELTA_MEAN_ABS, A.LSE_SUM_EXP, use_lse=False, use_n=False)
+    w = synth.Workload("wide", B=1, H=5, d=200, N_v=33, N_t=0)    # D = 1000: 125 vectors, unrolled body + tail
+    _score_case(oracle, w, 3, 33, A.DELTA_MEAN_SQ, A.LSE_LOG)
+
+
+def test_score_counter_clamp(oracle):
+    B, N, D = 1, 8, 64
+    x = torch.zeros(B, N, D, dtype=torch.bfloat16, device="cuda")
+    n = torch.tensor([[0, 1, 2, 79, 80, 81, 1000, 2 ** 30]], dtype=torch.int32, device="cuda")
+    out = torch.empty(B, N, device="cuda")
+    A.astraea_score(x, x, None, n, out, B, N, N, D, 1, 1.0, 1.0)
+    want = np.exp(np.minimum(n.cpu().numpy().astype(np.float64), 80.0))
+    got = out.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    assert (np.abs(got - want) / want).max() < 1e-5
+
+
+# --------------------------------------------------------------------- select
+def _select_case(oracle, s, k, n_always=0, with_n=True, with_rem=True, seed=0):
+    B, n_sel = s.shape
+    rng = np.random.default_rng(seed)
+    n0 = rng.integers(0, 85, size=(B, n_sel)).astype(np.int32) if with_n else None
+    want_sel, want_rem, want_n = oracle.select(s, k, n_always, n0)
+    idx_sel = torch.full((B, k + n_always), -7, dtype=torch.int32, device="cuda")
+    idx_rem = torch.full((B, n_sel - k), -7, dtype=torch.int32, device="cuda") if with_rem else None
+    n_dev = dev(n0) if with_n else None
+    ws = A.new_workspace(A.OP_SELECT, B, 0, n_sel, k, 0)
+    A.astraea_select(dev(s), B, n_sel, k, n_always, idx_sel, idx_rem, n_dev, ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(idx_sel.cpu().numpy(), want_sel)
+    if with_rem:
+        assert np.array_equal(idx_rem.cpu().numpy(), want_rem)
+    if with_n:
+        assert np.array_equal(n_dev.cpu().numpy(), want_n)
+
+
+@pytest.mark.parametrize("n_sel", [1, 5, 256, 1000, 4096, 4097, 9000])
+def test_select_integer_scores_bit_exact(oracle, n_sel):
+    for seed, levels in ((0, 2), (1, 7), (2, 64), (3, 100000)):
+        s = synth.integer_scores(2, n_sel, seed, levels)
+        for k in sorted({0, 1, n_sel // 4, n_sel // 2, n_sel - 1, n_sel}):
+            if 0 <= k <= n_sel:
+                _select_case(oracle, s, k, seed=seed)
+
+
+def test_select_all_equal_and_special_values(oracle):
+    _select_case(oracle, np.ones((2, 5000), np.float32), 1234)
+    s = np.random.default_rng(4).standard_normal((1, 3000)).astype(np.float32)
+    s[0, ::7] = 0.0
+    s[0, 3::7] = -0.0
+    s[0, 5::97] = np.nan
+    s[0, 11::101] = np.inf
+    s[0, 13::103] = -np.inf
+    s[0, 17::89] = 1e-42           # denormal
+    for k in (0, 10, 100, 1500, 2900, 2999, 3000):
+        _select_case(oracle, s, k)
+
+
+def test_select_always_kept_span_and_optional_outputs(oracle):
+    s = synth.integer_scores(2, 700, 5, 9)
+    _select_case(oracle, s, 300, n_always=26)
+    _select_case(oracle, s, 0, n_always=26)
+    _select_case(oracle, s, 300, n_always=26, with_n=False, with_rem=False)
+
+
+@pytest.mark.parametrize("name", ["cogvideox", "opensora", "hunyuan", "sweep"])
+def test_select_full_size_float_scores(oracle, name):
+    w = synth.WORKLOADS[name]
+    rng = np.random.default_rng(6)
+    s = np.exp(rng.standard_normal((w.B, w.N_v))).astype(np.float32) * 8000 + np.exp(rng.integers(0, 4, (w.B, w.N_v))).astype(np.float32)
+    for th in w.thetas_permille[:3]:
+        _select_case(oracle, s, w.k_of(th), n_always=w.N_t)
+    _select_case(oracle, synth.integer_scores(w.B, w.N_v, 7, 50), w.k_of(w.thetas_permille[0]), n_always=w.N_t)
+
+
+# -------------------------------------------------------------------- scatter
+@pytest.mark.parametrize("B,N,M,R", [(1, 256, 128, 128), (2, 301, 77, 3072), (1, 64, 64, 72), (2, 50, 1, 1152)])
+def test_scatter_reuse_bit_exact(oracle, B, N, M, R):
+    rng = np.random.default_rng(8)
+    cache = synth.f32_to_bf16_bits(rng.standard_normal((B, N, R)).astype(np.float32))
+    rows = synth.f32_to_bf16_bits(rng.standard_normal((B, M, R)).astype(np.float32))
+    full = synth.f32_to_bf16_bits(rng.standard_normal((B, N, R)).astype(np.float32))
+    idx = np.stack([np.sort(rng.choice(N, M, replace=False)) for _ in range(B)]).astype(np.int32)
+    c = to_dev_bf16(cache)
+    A.astraea_scatter_reuse(c, to_dev_bf16(rows), dev(idx), B, N, M, R)
+    want = oracle.scatter_reuse(f64(cache), f64(rows), idx)
+    assert np.array_equal(bf16_dev_to_f64(c), want)
+    c = to_dev_bf16(cache)
+    A.astraea_scatter_reuse(c, to_dev_bf16(full), dev(idx), B, N, M, R, A.SCATTER_SRC_FULL)
+    want = oracle.scatter_reuse(f64(cache), np.take_along_axis(f64(full), idx[:, :, None].astype(np.int64), 1), idx)
+    assert np.array_equal(bf16_dev_to_f64(c), want)
+
+
+def test_scatter_with_no_rows_leaves_cache_alone():
+    c = torch.randn(1, 16, 64, device="cuda").bfloat16()
+    before = c.clone()
+    A.astraea_scatter_reuse(c, c, torch.empty(1, 0, dtype=torch.int32, device="cuda"), 1, 16, 0, 64)
+    assert torch.equal(c, before)
+
+
+# ------------------------------------------------------------------ attention
+def _attn_case(oracle, B, H, N, d, M, seed, layout="bnhd", compact=False, dense=False, scale=0.0, amp=1.0):
+    rng = np.random.default_rng(seed)
+    q, k, v, cache = (synth.f32_to_bf16_bits((amp * rng.standard_normal((B, N, H, d))).astype(np.float32)) for _ in range(4))
+    idx = None if dense else np.stack([np.sort(rng.choice(N, M, replace=False)) for _ in range(B)]).astype(np.int32)
+    M = N if dense else M
+    want_o, want_lse, _ = oracle.sparse_attn(f64(q), f64(k), f64(v), q_idx=idx, scale=scale)
+
+    def place(bits):
+        t = to_dev_bf16(bits)
+        if layout == "bhnd":
+            t = t.permute(0, 2, 1, 3).contiguous()
+            return t, (H * N * d, N * d, d)
+        return t, A.bhnd_strides(N, H, d)
+
+    (qd, qs), (kd, ks), (vd, vs) = place(q), place(k), place(v)
+    lse_cache0 = rng.standard_normal((B, H, N)).astype(np.float32)
+    if compact:
+        out = torch.zeros(B, M, H, d, dtype=torch.bfloat16, device="cuda")
+        lse = torch.zeros(B, H, M, device="cuda")
+    else:
+        out = to_dev_bf16(cache)
+        lse = dev(lse_cache0)
+    ws = A.new_workspace(A.OP_SPARSE_ATTN, B, H, N, M, d)
+    A.astraea_sparse_attn(qd, kd, vd, qs, ks, vs, None if idx is None else dev(idx), M, out, lse, B, H, N, d,
+                          scale=scale, flags=A.ATTN_COMPACT_OUT if compact else 0, workspace=ws)
+    A.astraea_poll_error(ws)
+    got = bf16_dev_to_f64(out)
+    got_lse = lse.cpu().numpy().astype(np.float64)
+    if idx is None:
+        idx = np.broadcast_to(np.arange(N, dtype=np.int32), (B, N))
+    if compact:
+        got_rows, got_lse_rows = got, got_lse
+    else:
+        got_rows = np.take_along_axis(got, idx[:, :, None, None].astype(np.int64), 1)
+        got_lse_rows = np.take_along_axis(got_lse, idx[:, None, :].astype(np.int64), 2)
+        # rows that were not selected are bit-identical to the cache (reuse)
+        mask = np.ones((B, N), bool)
+        for b in range(B):
+            mask[b, idx[b]] = False
+        assert np.array_equal(got[mask], f64(cache)[mask])
+        assert np.array_equal(got_lse.transpose(0, 2, 1)[mask], lse_cache0.astype(np.float64).transpose(0, 2, 1)[mask])
+    err = np.abs(got_rows - want_o)
+    assert err.max() < ATTN_MAX_ABS and err.mean() < ATTN_MEAN_ABS, (err.max(), err.mean())
+    assert np.abs(got_lse_rows - want_lse).max() < LSE_ABS, np.abs(got_lse_rows - want_lse).max()
+
+
+def test_attn_tiny_config(oracle):
+    _attn_case(oracle, 1, 2, 256, 64, 128, seed=0)
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_attn_single_tile(oracle, d):
+    _attn_case(oracle, 1, 1, 128, d, 128, seed=1, dense=True)
+
+
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("N,M", [(300, 77), (1000, 333), (129, 129), (1, 1), (127, 5)])
+def test_attn_ragged_tiles(oracle, d, N, M):
+    _attn_case(oracle, 2, 3, N, d, M, seed=2)
+
+
+def test_attn_many_key_tiles_exercise_every_stage_phase(oracle):
+    _attn_case(oracle, 1, 2, 128 * 19 + 16, 128, 200, seed=3)
+    _attn_case(oracle, 1, 2, 128 * 27 + 112, 64, 130, seed=4)
+
+
+def test_attn_head_major_layout_compact_output_and_scale(oracle):
+    _attn_case(oracle, 2, 2, 400, 64, 100, seed=5, layout="bhnd")
+    _attn_case(oracle, 2, 2, 400, 128, 100, seed=6, compact=True)
+    _attn_case(oracle, 1, 2, 400, 128, 100, seed=7, scale=0.05)
+
+
+def test_attn_dense_equals_all_rows(oracle):
+    _attn_case(oracle, 1, 2, 517, 64, 517, seed=8, dense=True)
+
+
+def test_attn_peaked_softmax_triggers_rescaling(oracle):
+    # logits of order +-40: the running maximum moves by more than the lazy-rescale threshold
+    _attn_case(oracle, 1, 2, 900, 64, 128, seed=9, amp=2.5)
+    _attn_case(oracle, 1, 1, 900, 128, 128, seed=10, amp=2.0)
+
+
+def test_attn_closed_forms_on_device():
+    """Zero keys: every selected output is the mean of all value rows and LSE = ln N; this
+    catches phantom keys from the zero-filled tail of the last key tile."""
+    B, H, N, d, M = 1, 2, 333, 64, 50
+    g = torch.Generator(device="cpu").manual_seed(0)
+    q = torch.randn(B, N, H, d, generator=g).bfloat16().cuda()
+    v = torch.randn(B, N, H, d, generator=g).bfloat16().cuda()
+    k = torch.zeros_like(q)
+    idx = torch.arange(0, 2 * M, 2, dtype=torch.int32, device="cuda")[None].contiguous()
+    out = torch.zeros(B, M, H, d, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros(B, H, M, device="cuda")
+    ws = A.new_workspace(A.OP_SPARSE_ATTN, B, H, N, M, d)
+    s = A.bhnd_strides(N, H, d)
+    A.astraea_sparse_attn(q, k, v, s, s, s, idx, M, out, lse, B, H, N, d, flags=A.ATTN_COMPACT_OUT, workspace=ws)
+    A.astraea_poll_error(ws)
+    mean_v = v.double().mean(dim=1, keepdim=True)
+    assert (out.double() - mean_v).abs().max().item() < 4e-3
+    assert (lse.double() - math.log(N)).abs().max().item() < 1e-5
+
+
+def test_attn_bad_index_is_reported_not_dereferenced():
+    B, H, N, d, M = 1, 1, 64, 64, 4
+    q = torch.zeros(B, N, H, d, dtype=torch.bfloat16, device="cuda")
+    out = torch.ones(B, N, H, d, dtype=torch.bfloat16, device="cuda")
+    idx = torch.tensor([[0, 1, 64, 2 ** 30]], dtype=torch.int32, device="cuda")
+    ws = A.new_workspace(A.OP_SPARSE_ATTN, B, H, N, M, d)
+    s = A.bhnd_strides(N, H, d)
+    A.astraea_sparse_attn(q, q, q, s, s, s, idx, M, out, None, B, H, N, d, workspace=ws)
+    with pytest.raises(A.AstraeaError) as e:
+        A.astraea_poll_error(ws)
+    assert e.value.code == A.ERR_BAD_INDEX
+    A.astraea_poll_error(ws)                 # the word was cleared
+    assert torch.equal(out[0, 2:], torch.ones_like(out[0, 2:]))
+
+
+# ------------------------------------------------------------- the whole step
+def _step_case(oracle, w, seed, theta, steps=1):
+    inp = synth.make_step_inputs(w, seed)
+    B, N, H, d, D, N_sel, n_always = w.B, w.N, w.H, w.d, w.D, w.N_v, w.N_t
+    k_keep = w.k_of(theta)
+    M = k_keep + n_always
+    # state on the device
+    x_ref = to_dev_bf16(inp["x_ref"])
+    lse = dev(inp["lse"] - np.float32(math.log(N)))
+    n_skip = dev(inp["n_skip"])
+    out = to_dev_bf16(inp["cache"])
+    score = torch.empty(B, N_sel, device="cuda")
+    idx_sel = torch.empty(B, M, dtype=torch.int32, device="cuda")
+    idx_rem = torch.empty(B, N_sel - k_keep, dtype=torch.int32, device="cuda")
+    ws = A.new_workspace(A.OP_STEP, B, H, N, M, d)
+    # state of the oracle
+    o_xref, o_lse, o_n, o_out = f64(inp["x_ref"]), lse.cpu().numpy().astype(np.float64), inp["n_skip"].copy(), f64(inp["cache"])
+    x_bits, q_bits, k_bits, v_bits = inp["x_cur"], inp["q"], inp["k"], inp["v"]
+    for t in range(steps):
+        if t > 0:
+            x_bits = synth.drift_step(x_bits, 100 + t, 0.05, False)
+            q_bits, k_bits, v_bits = (synth.drift_step(a, 200 + 10 * t + i, 0.05, True) for i, a in enumerate((q_bits, k_bits, v_bits)))
+        A.astraea_step(to_dev_bf16(x_bits), x_ref, lse, n_skip, to_dev_bf16(q_bits), to_dev_bf16(k_bits),
+                       to_dev_bf16(v_bits), out, score, idx_sel, idx_rem, B, H, N, N_sel, d, k_keep, workspace=ws)
+        A.astraea_poll_error(ws)
+        # teacher forcing: the oracle starts each step from the state the device had (bf16 / fp32 values)
+        res = oracle.step(f64(x_bits), o_xref, o_lse, o_n, f64(q_bits), f64(k_bits), f64(v_bits), o_out, k_keep, n_always)
+        got_score = score.cpu().numpy()
+        rel = np.abs(got_score.astype(np.float64) - res["score"]) / np.abs(res["score"])
+        assert rel.max() < SCORE_RTOL
+        got_sel = idx_sel.cpu().numpy()
+        if not np.array_equal(got_sel, res["idx_sel"]):
+            # allowed only where a score is within 1e-6 relative of the k-th largest
+            for b in range(B):
+                kth = np.sort(res["score"][b])[::-1][k_keep - 1]
+                diff = np.setxor1d(got_sel[b], res["idx_sel"][b])
+                assert (np.abs(res["score"][b][diff] - kth) <= 1e-6 * abs(kth)).all()
+            return      # the two chains diverge legitimately from here on
+        assert np.array_equal(idx_rem.cpu().numpy(), res["idx_rem"])
+        assert np.array_equal(n_skip.cpu().numpy(), res["n_skip"])
+        got_out = bf16_dev_to_f64(out)
+        err = np.abs(got_out - res["out"])
+        assert err.max() < ATTN_MAX_ABS and err.mean() < ATTN_MEAN_ABS
+        sel_mask = np.zeros((B, N), bool)
+        for b in range(B):
+            sel_mask[b, res["idx_sel"][b]] = True
+        assert np.array_equal(got_out[~sel_mask], o_out[~sel_mask])            # reuse is bit-exact
+        assert np.abs(lse.cpu().numpy() - res["lse"]).max() < LSE_ABS
+        assert np.array_equal(bf16_dev_to_f64(x_ref), res["x_ref"])
+        # next step starts from the device state
+        o_xref, o_lse, o_n, o_out = res["x_ref"], lse.cpu().numpy().astype(np.float64), res["n_skip"], got_out
+
+
+def test_step_tiny_config(oracle):
+    _step_case(oracle, synth.WORKLOADS["tiny"], 0, 500)
+
+
+def test_step_keep_ratio_zero_and_one(oracle):
+    w = synth.scaled(synth.WORKLOADS["tiny"], drift_sigma=0.05, n_skip_max=3)
+    _step_case(oracle, w, 1, 0)
+    _step_case(oracle, w, 1, 1000)
+
+
+def test_step_with_text_tokens_and_batch(oracle):
+    w = synth.Workload("mini-cog", B=2, H=4, d=64, N_v=450, N_t=26)
+    _step_case(oracle, w, 2, 250)
+
+
+def test_step_chain_of_three_steps_d128(oracle):
+    w = synth.Workload("mini-hy", B=1, H=2, d=128, N_v=8 * 12 * 20, N_t=0)
+    _step_case(oracle, w, 3, 600, steps=3)
