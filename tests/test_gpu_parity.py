@@ -157,7 +157,8 @@ def test_scatter_with_no_rows_leaves_cache_alone():
 # ------------------------------------------------------------------ attention
 def _attn_case(oracle, B, H, N, d, M, seed, layout="bnhd", compact=False, dense=False, scale=0.0, amp=1.0):
     rng = np.random.default_rng(seed)
-    q, k, v, cache = (synth.f32_to_bf16_bits((amp * rng.standard_normal((B, N, H, d))).astype(np.float32)) for _ in range(4))
+    # amp sharpens the logits only (q, k); values and the cache stay N(0,1)
+    q, k, v, cache = (synth.f32_to_bf16_bits((a * rng.standard_normal((B, N, H, d))).astype(np.float32)) for a in (amp, amp, 1.0, 1.0))
     idx = None if dense else np.stack([np.sort(rng.choice(N, M, replace=False)) for _ in range(B)]).astype(np.int32)
     M = N if dense else M
     want_o, want_lse, _ = oracle.sparse_attn(f64(q), f64(k), f64(v), q_idx=idx, scale=scale)
