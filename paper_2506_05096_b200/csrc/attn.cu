@@ -2,15 +2,18 @@
 // against ALL keys/values, written in place over the cached output (Algorithm 1 lines 6-7;
 // Section 3.2 "Sparse Attention").
 //
-// One CTA per (128 selected queries, head, batch).  Warp roles:
-//   warps 0-3  softmax: gather the CTA's Q rows into 128B-swizzled shared memory, then per
-//              key tile read S from TMEM (one thread per query row), online softmax in the
-//              log2 domain with lazy rescaling of O, write P (bf16) back to TMEM over S,
-//              and at the end normalise O and scatter it to the rows q_idx names;
-//   warp 4     TMA producer: K and V tiles (128 keys) into multi-stage swizzled buffers;
-//   warp 5     tcgen05.mma issuer: S = Q K^T (SS, K-major operands), O += P V (P from TMEM,
+// One CTA per (256 selected queries, head, batch): two 128-row query tiles A and B that
+// share every K/V tile and alternate on the tensor core, so that one tile's softmax runs
+// while the other tile's MMAs execute.  Warp roles (384 threads, three warpgroups):
+//   warpgroup 0 / 1  softmax of tile A / B: gather the tile's Q rows into 128B-swizzled shared
+//              memory, then per key tile read S from TMEM (one thread per query row), online
+//              softmax in the log2 domain with lazy rescaling of O, write P (bf16) back to
+//              TMEM over S, and at the end normalise O and scatter it to the rows q_idx names;
+//   warp 8     TMA producer: K and V tiles (128 keys) into multi-stage swizzled buffers;
+//   warp 9     tcgen05.mma issuer: S = Q K^T (SS, K-major operands), O += P V (P from TMEM,
 //              V as an MN-major shared-memory operand); owns the TMEM allocation.
-// TMEM columns: S/P buffer 0 [0,128), S/P buffer 1 [128,256), O [256, 256+d).
+// Registers are rebalanced with setmaxnreg (softmax warpgroups up, the third one down).
+// TMEM columns: S/P of tile A [0,128), of tile B [128,256), O of A [256,256+d), of B [384,384+d).
 // Every mbarrier wait is bounded; on a timeout the CTA raises the error word and leaves.
 #include "common.cuh"
 #include "sm100_ptx.cuh"
@@ -20,9 +23,10 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kBlockM = 128;
+constexpr int kBlockM = 128;                     // rows of one query tile
+constexpr int kTilesM = 2;                       // query tiles per CTA
 constexpr int kBlockN = 128;
-constexpr int kThreads = 192;
+constexpr int kThreads = 384;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColO = 256;
 constexpr float kRescaleThreshold = 8.0f;        // log2 units: P stays below 2^8
@@ -32,9 +36,10 @@ template <int DH> struct Cfg {
     static constexpr int kChunks = DH / 64;                       // 64-column (128-byte) swizzle chunks
     static constexpr int kChunkBytes = 128 * 128;                 // 128 rows x 128 bytes
     static constexpr int kTileBytes = kChunks * kChunkBytes;      // one Q / K / V tile
-    static constexpr int kStages = (DH == 128) ? 3 : 6;
+    static constexpr int kStagesK = (DH == 128) ? 3 : 5;
+    static constexpr int kStagesV = (DH == 128) ? 2 : 5;
     static constexpr int kBarBytes = 256;
-    static constexpr int kSmemBytes = kTileBytes * (1 + 2 * kStages) + kBarBytes + 1024;
+    static constexpr int kSmemBytes = kTileBytes * (kTilesM + kStagesK + kStagesV) + kBarBytes + 1024;
 };
 
 struct Params {
@@ -74,6 +79,177 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     return true;
 }
 
+struct Bars {
+    uint32_t q, s, p, o;            // [kTilesM] each
+    uint32_t kf, ke, vf, ve;        // [stages]
+};
+
+// ---------------------------------------------------------------- softmax warpgroup (one query tile)
+template <int DH>
+__device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, int tile, uint8_t *sQ_gen, uint32_t tmem,
+                                             int m_base, int h, int b, int n_tiles, volatile int *abort_flag)
+{
+    using C = Cfg<DH>;
+    const int wtid = threadIdx.x & 127, warp = wtid >> 5, lane = wtid & 31;
+    // gather this tile's Q rows (swizzled, K-major)
+    constexpr int kVecPerRow = DH / 8;                 // 16-byte vectors per row
+    constexpr int kRowsPerIter = 32 / kVecPerRow;
+    {
+        const int sub = lane / kVecPerRow, c = lane % kVecPerRow;
+#pragma unroll 4
+        for (int r0 = warp * kRowsPerIter; r0 < kBlockM; r0 += 4 * kRowsPerIter) {
+            const int r = r0 + sub;
+            const int m = m_base + r;
+            uint4 val = make_uint4(0, 0, 0, 0);
+            if (m < p.M) {
+                const int tok = p.q_idx ? __ldg(p.q_idx + (size_t)b * p.M + m) : m;
+                if ((unsigned)tok < (unsigned)p.N) {
+                    const __nv_bfloat16 *src = p.q + (size_t)b * p.q_sb + (size_t)tok * p.q_sn + (size_t)h * p.q_sh + c * 8;
+                    val = __ldg(reinterpret_cast<const uint4 *>(src));
+                }
+            }
+            const uint32_t off = (c >> 3) * C::kChunkBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
+            *reinterpret_cast<uint4 *>(sQ_gen + off) = val;
+        }
+    }
+    fence_proxy_async_smem();
+    mbar_arrive(bar.q + 8 * tile);
+
+    const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);
+    const uint32_t t_s = t_row + tile * 128;
+    const uint32_t t_o = t_row + kColO + tile * 128;
+    const uint32_t bar_s = bar.s + 8 * tile, bar_p = bar.p + 8 * tile, bar_o = bar.o + 8 * tile;
+    const int m = m_base + wtid;
+    int tok = -1;
+    if (m < p.M) {
+        tok = p.q_idx ? __ldg(p.q_idx + (size_t)b * p.M + m) : m;
+        if ((unsigned)tok >= (unsigned)p.N) { atomicExch(p.err_word, kErrBadIndex); tok = -1; }
+    }
+    const float sl2 = p.scale_log2;
+    float m_ref = -INFINITY, l_sum = 0.f;
+    bool ok = true;
+
+    for (int j = 0; j < n_tiles; ++j) {
+        ok = wait_bar(bar_s, j & 1, abort_flag, p.err_word);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        float s[kBlockN];
+        {
+            uint32_t t0[32], t1[32], t2[32], t3[32];
+            tmem_ld32(t_s, t0);
+            tmem_ld32(t_s + 32, t1);
+            tmem_ld32(t_s + 64, t2);
+            tmem_ld32(t_s + 96, t3);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                s[i] = __uint_as_float(t0[i]);
+                s[32 + i] = __uint_as_float(t1[i]);
+                s[64 + i] = __uint_as_float(t2[i]);
+                s[96 + i] = __uint_as_float(t3[i]);
+            }
+        }
+        const int valid = p.N - j * kBlockN;           // keys of this tile that exist
+        if (valid < kBlockN) {
+#pragma unroll
+            for (int i = 0; i < kBlockN; ++i) if (i >= valid) s[i] = -INFINITY;
+        }
+        // row maximum: independent partial maxima keep the dependency chains short
+        float mx4[4] = {s[0], s[1], s[2], s[3]};
+#pragma unroll
+        for (int i = 4; i < kBlockN; i += 4) {
+            mx4[0] = fmaxf(mx4[0], s[i]); mx4[1] = fmaxf(mx4[1], s[i + 1]);
+            mx4[2] = fmaxf(mx4[2], s[i + 2]); mx4[3] = fmaxf(mx4[3], s[i + 3]);
+        }
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+
+        if (j == 0) {
+            m_ref = mx;
+        } else {
+            const bool need = (mx - m_ref) * sl2 > kRescaleThreshold;
+            if (__any_sync(0xffffffffu, need)) {
+                float alpha = 1.0f;
+                if (need) { alpha = ex2((m_ref - mx) * sl2); m_ref = mx; l_sum *= alpha; }
+                ok = wait_bar(bar_o, (j - 1) & 1, abort_flag, p.err_word);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int cc = 0; cc < DH / 32; ++cc) {
+                    uint32_t o[32];
+                    tmem_ld32(t_o + cc * 32, o);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                    tmem_st32(t_o + cc * 32, o);
+                }
+                tc_wait_st();
+            }
+        }
+        const float neg = -m_ref * sl2;
+        float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int i = 0; i < kBlockN; i += 4) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { s[i + u] = ex2(fmaf(s[i + u], sl2, neg)); sum4[u] += s[i + u]; }
+        }
+        l_sum += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+        // P as bf16 pairs over the first 64 columns of this S buffer (element 2c in the low half)
+#pragma unroll
+        for (int cc = 0; cc < 2; ++cc) {
+            uint32_t pk[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                __nv_bfloat162 v2 = __floats2bfloat162_rn(s[cc * 64 + 2 * i], s[cc * 64 + 2 * i + 1]);
+                pk[i] = *reinterpret_cast<uint32_t *>(&v2);
+            }
+            tmem_st32(t_s + cc * 32, pk);
+        }
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar_p);
+    }
+
+    // epilogue: normalise and scatter
+    if (ok) {
+        ok = wait_bar(bar_o, (n_tiles - 1) & 1, abort_flag, p.err_word);
+        ok = __all_sync(0xffffffffu, ok);
+    }
+    if (ok) {
+        tc_fence_after();
+        const float inv_l = 1.0f / l_sum;
+        __nv_bfloat16 *dst = nullptr;
+        if (tok >= 0) {
+            const size_t orow = p.compact ? ((size_t)b * p.M + m) : ((size_t)b * p.N + tok);
+            dst = p.out + (orow * p.H + h) * DH;
+            if (p.lse_out) {
+                const size_t li = p.compact ? (((size_t)b * p.H + h) * p.M + m) : (((size_t)b * p.H + h) * p.N + tok);
+                p.lse_out[li] = m_ref * p.scale + logf(l_sum);
+            }
+        }
+#pragma unroll
+        for (int cc = 0; cc < DH / 32; ++cc) {
+            uint32_t o[32];
+            tmem_ld32(t_o + cc * 32, o);
+            tc_wait_ld();
+            if (dst) {
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                    uint32_t w[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(o[v * 8 + 2 * i]) * inv_l,
+                                                                  __uint_as_float(o[v * 8 + 2 * i + 1]) * inv_l);
+                        w[i] = *reinterpret_cast<uint32_t *>(&v2);
+                    }
+                    *reinterpret_cast<uint4 *>(dst + cc * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+            }
+        }
+    }
+}
+
 template <int DH>
 __global__ void __launch_bounds__(kThreads, 1)
 sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v, const Params p)
@@ -86,37 +262,32 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const uint32_t sQ = smem_base;
-    const uint32_t sK = sQ + C::kTileBytes;
-    const uint32_t sV = sK + C::kStages * C::kTileBytes;
-    const uint32_t bars = sV + C::kStages * C::kTileBytes;
-    // barrier slots (8 bytes each)
-    const uint32_t bar_q = bars;
-    const uint32_t bar_s = bars + 8;                       // [2]
-    const uint32_t bar_p = bars + 24;                      // [2]
-    const uint32_t bar_o = bars + 40;
-    const uint32_t bar_kf = bars + 48;                     // [kStages]
-    const uint32_t bar_ke = bar_kf + 8 * C::kStages;
-    const uint32_t bar_vf = bar_ke + 8 * C::kStages;
-    const uint32_t bar_ve = bar_vf + 8 * C::kStages;
-    static_assert(48 + 32 * C::kStages <= C::kBarBytes, "barrier area too small");
+    const uint32_t sK = sQ + kTilesM * C::kTileBytes;
+    const uint32_t sV = sK + C::kStagesK * C::kTileBytes;
+    const uint32_t bars = sV + C::kStagesV * C::kTileBytes;
+    Bars bar;
+    bar.q = bars; bar.s = bars + 16; bar.p = bars + 32; bar.o = bars + 48;
+    bar.kf = bars + 64;
+    bar.ke = bar.kf + 8 * C::kStagesK;
+    bar.vf = bar.ke + 8 * C::kStagesK;
+    bar.ve = bar.vf + 8 * C::kStagesV;
+    static_assert(64 + 16 * (C::kStagesK + C::kStagesV) <= C::kBarBytes, "barrier area too small");
 
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int m0 = blockIdx.x * kBlockM, h = blockIdx.y, b = blockIdx.z;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, wg = tid >> 7;
+    const int m0 = blockIdx.x * (kTilesM * kBlockM), h = blockIdx.y, b = blockIdx.z;
     const int n_tiles = (p.N + kBlockN - 1) / kBlockN;
 
     if (tid == 0) {
         abort_flag = 0;
-        mbar_init(bar_q, 128);
-        mbar_init(bar_s, 1); mbar_init(bar_s + 8, 1);
-        mbar_init(bar_p, 128); mbar_init(bar_p + 8, 128);
-        mbar_init(bar_o, 1);
-        for (int s = 0; s < C::kStages; ++s) {
-            mbar_init(bar_kf + 8 * s, 1); mbar_init(bar_ke + 8 * s, 1);
-            mbar_init(bar_vf + 8 * s, 1); mbar_init(bar_ve + 8 * s, 1);
+        for (int t = 0; t < kTilesM; ++t) {
+            mbar_init(bar.q + 8 * t, 128); mbar_init(bar.s + 8 * t, 1);
+            mbar_init(bar.p + 8 * t, 128); mbar_init(bar.o + 8 * t, 1);
         }
+        for (int s = 0; s < C::kStagesK; ++s) { mbar_init(bar.kf + 8 * s, 1); mbar_init(bar.ke + 8 * s, 1); }
+        for (int s = 0; s < C::kStagesV; ++s) { mbar_init(bar.vf + 8 * s, 1); mbar_init(bar.ve + 8 * s, 1); }
         fence_barrier_init();
     }
-    if (warp == 5) {
+    if (warp == 9) {
         tmem_alloc(smem_u32(&tmem_slot), kTmemCols);
         tmem_relinquish();
     }
@@ -125,227 +296,101 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
 
-    if (warp < 4) {
-        // ------------------------------------------------ gather Q rows (swizzled, K-major)
-        constexpr int kVecPerRow = DH / 8;                 // 16-byte vectors per row
-        constexpr int kRowsPerIter = 32 / kVecPerRow;
-        const int sub = lane / kVecPerRow, c = lane % kVecPerRow;
-        for (int r0 = warp * kRowsPerIter; r0 < kBlockM; r0 += 4 * kRowsPerIter) {
-            const int r = r0 + sub;
-            const int m = m0 + r;
-            uint4 val = make_uint4(0, 0, 0, 0);
-            if (m < p.M) {
-                const int tok = p.q_idx ? __ldg(p.q_idx + (size_t)b * p.M + m) : m;
-                if ((unsigned)tok < (unsigned)p.N) {
-                    const __nv_bfloat16 *src = p.q + (size_t)b * p.q_sb + (size_t)tok * p.q_sn + (size_t)h * p.q_sh + c * 8;
-                    val = __ldg(reinterpret_cast<const uint4 *>(src));
-                }
-            }
-            const uint32_t off = (c >> 3) * C::kChunkBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
-            *reinterpret_cast<uint4 *>(smem_gen + off) = val;
-        }
-        fence_proxy_async_smem();
-        mbar_arrive(bar_q);
-
-        // ------------------------------------------------ online softmax, one thread per query row
-        const int row = tid;                               // TMEM lane
-        const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);
-        const int m = m0 + row;
-        int tok = -1;
-        if (m < p.M) {
-            tok = p.q_idx ? __ldg(p.q_idx + (size_t)b * p.M + m) : m;
-            if ((unsigned)tok >= (unsigned)p.N) { atomicExch(p.err_word, kErrBadIndex); tok = -1; }
-        }
-        const float sl2 = p.scale_log2;
-        float m_ref = -INFINITY, l_sum = 0.f;
-        bool ok = true;
-
-        for (int j = 0; j < n_tiles && ok; ++j) {
-            const int buf = j & 1;
-            ok = wait_bar(bar_s + 8 * buf, (j >> 1) & 1, &abort_flag, p.err_word);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-            float s[kBlockN];
-            {
-                uint32_t t0[32], t1[32], t2[32], t3[32];
-                tmem_ld32(t_row + buf * 128, t0);
-                tmem_ld32(t_row + buf * 128 + 32, t1);
-                tmem_ld32(t_row + buf * 128 + 64, t2);
-                tmem_ld32(t_row + buf * 128 + 96, t3);
-                tc_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    s[i] = __uint_as_float(t0[i]);
-                    s[32 + i] = __uint_as_float(t1[i]);
-                    s[64 + i] = __uint_as_float(t2[i]);
-                    s[96 + i] = __uint_as_float(t3[i]);
-                }
-            }
-            const int valid = p.N - j * kBlockN;           // keys of this tile that exist
-            if (valid < kBlockN) {
-#pragma unroll
-                for (int i = 0; i < kBlockN; ++i) if (i >= valid) s[i] = -INFINITY;
-            }
-            float mx = s[0];
-#pragma unroll
-            for (int i = 1; i < kBlockN; ++i) mx = fmaxf(mx, s[i]);
-
-            if (j == 0) {
-                m_ref = mx;
-            } else {
-                const bool need = (mx - m_ref) * sl2 > kRescaleThreshold;
-                if (__any_sync(0xffffffffu, need)) {
-                    float alpha = 1.0f;
-                    if (need) { alpha = ex2((m_ref - mx) * sl2); m_ref = mx; l_sum *= alpha; }
-                    ok = wait_bar(bar_o, (j - 1) & 1, &abort_flag, p.err_word);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    tc_fence_after();
-#pragma unroll
-                    for (int cc = 0; cc < DH / 32; ++cc) {
-                        uint32_t o[32];
-                        tmem_ld32(t_row + kColO + cc * 32, o);
-                        tc_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                        tmem_st32(t_row + kColO + cc * 32, o);
-                    }
-                    tc_wait_st();
-                }
-            }
-            const float neg = -m_ref * sl2;
-            float sum = 0.f;
-#pragma unroll
-            for (int i = 0; i < kBlockN; ++i) { s[i] = ex2(fmaf(s[i], sl2, neg)); sum += s[i]; }
-            l_sum += sum;
-            // P as bf16 pairs over the first 64 columns of this S buffer (element 2c in the low half)
-#pragma unroll
-            for (int cc = 0; cc < 2; ++cc) {
-                uint32_t pk[32];
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    __nv_bfloat162 v2 = __floats2bfloat162_rn(s[cc * 64 + 2 * i], s[cc * 64 + 2 * i + 1]);
-                    pk[i] = *reinterpret_cast<uint32_t *>(&v2);
-                }
-                tmem_st32(t_row + buf * 128 + cc * 32, pk);
-            }
-            tc_wait_st();
-            tc_fence_before();
-            mbar_arrive(bar_p + 8 * buf);
-        }
-
-        // ------------------------------------------------ epilogue: normalise and scatter
-        if (ok) {
-            ok = wait_bar(bar_o, (n_tiles - 1) & 1, &abort_flag, p.err_word);
-            ok = __all_sync(0xffffffffu, ok);
-        }
-        if (ok) {
-            tc_fence_after();
-            const float inv_l = 1.0f / l_sum;
-            __nv_bfloat16 *dst = nullptr;
-            if (tok >= 0) {
-                const size_t orow = p.compact ? ((size_t)b * p.M + m) : ((size_t)b * p.N + tok);
-                dst = p.out + (orow * p.H + h) * DH;
-                if (p.lse_out) {
-                    const size_t li = p.compact ? (((size_t)b * p.H + h) * p.M + m) : (((size_t)b * p.H + h) * p.N + tok);
-                    p.lse_out[li] = m_ref * p.scale + logf(l_sum);
-                }
-            }
-#pragma unroll
-            for (int cc = 0; cc < DH / 32; ++cc) {
-                uint32_t o[32];
-                tmem_ld32(t_row + kColO + cc * 32, o);
-                tc_wait_ld();
-                if (dst) {
-#pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        uint32_t w[4];
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(o[v * 8 + 2 * i]) * inv_l,
-                                                                      __uint_as_float(o[v * 8 + 2 * i + 1]) * inv_l);
-                            w[i] = *reinterpret_cast<uint32_t *>(&v2);
-                        }
-                        *reinterpret_cast<uint4 *>(dst + cc * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-                    }
-                }
-            }
-        }
-    } else if (warp == 4) {
-        // ------------------------------------------------ TMA producer
-        if (lane == 0) {
+    if (wg < 2) {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
+        softmax_role<DH>(p, bar, wg, smem_gen + wg * C::kTileBytes, tmem, m0 + wg * kBlockM, h, b, n_tiles, &abort_flag);
+    } else {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+        if (warp == 8 && lane == 0) {
+            // ------------------------------------------------ TMA producer
             prefetch_tensormap(&tmap_k);
             prefetch_tensormap(&tmap_v);
             int issued_k = 0, issued_v = 0;
             bool ok = true;
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                const int st = j % C::kStages;
-                const uint32_t ph = (j / C::kStages) & 1;
-                ok = wait_bar(bar_ke + 8 * st, ph ^ 1, &abort_flag, p.err_word);
-                if (!ok) break;
-                mbar_arrive_expect_tx(bar_kf + 8 * st, C::kTileBytes);
+            auto load_k = [&](int j) -> bool {
+                const int st = j % C::kStagesK;
+                if (!wait_bar(bar.ke + 8 * st, ((j / C::kStagesK) & 1) ^ 1, &abort_flag, p.err_word)) return false;
+                mbar_arrive_expect_tx(bar.kf + 8 * st, C::kTileBytes);
 #pragma unroll
                 for (int ch = 0; ch < C::kChunks; ++ch)
-                    tma_load_4d(sK + st * C::kTileBytes + ch * C::kChunkBytes, &tmap_k, bar_kf + 8 * st,
-                                ch * 64, j * kBlockN, h, b);
+                    tma_load_4d(sK + st * C::kTileBytes + ch * C::kChunkBytes, &tmap_k, bar.kf + 8 * st, ch * 64, j * kBlockN, h, b);
                 issued_k = j + 1;
-                ok = wait_bar(bar_ve + 8 * st, ph ^ 1, &abort_flag, p.err_word);
-                if (!ok) break;
-                mbar_arrive_expect_tx(bar_vf + 8 * st, C::kTileBytes);
+                return true;
+            };
+            auto load_v = [&](int j) -> bool {
+                const int st = j % C::kStagesV;
+                if (!wait_bar(bar.ve + 8 * st, ((j / C::kStagesV) & 1) ^ 1, &abort_flag, p.err_word)) return false;
+                mbar_arrive_expect_tx(bar.vf + 8 * st, C::kTileBytes);
 #pragma unroll
                 for (int ch = 0; ch < C::kChunks; ++ch)
-                    tma_load_4d(sV + st * C::kTileBytes + ch * C::kChunkBytes, &tmap_v, bar_vf + 8 * st,
-                                ch * 64, j * kBlockN, h, b);
+                    tma_load_4d(sV + st * C::kTileBytes + ch * C::kChunkBytes, &tmap_v, bar.vf + 8 * st, ch * 64, j * kBlockN, h, b);
                 issued_v = j + 1;
+                return true;
+            };
+            // K runs one tile ahead of V: K_{j+1} is needed before V_j
+            ok = load_k(0);
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                if (j + 1 < n_tiles) ok = load_k(j + 1);
+                if (ok) ok = load_v(j);
             }
             if (!ok) {
                 // leaving early: let the copies already issued land before the CTA's shared memory is released
-                for (int j = (issued_k > C::kStages ? issued_k - C::kStages : 0); j < issued_k; ++j)
-                    wait_bar(bar_kf + 8 * (j % C::kStages), (j / C::kStages) & 1, &abort_flag, p.err_word);
-                for (int j = (issued_v > C::kStages ? issued_v - C::kStages : 0); j < issued_v; ++j)
-                    wait_bar(bar_vf + 8 * (j % C::kStages), (j / C::kStages) & 1, &abort_flag, p.err_word);
+                for (int j = (issued_k > C::kStagesK ? issued_k - C::kStagesK : 0); j < issued_k; ++j)
+                    wait_bar(bar.kf + 8 * (j % C::kStagesK), (j / C::kStagesK) & 1, &abort_flag, p.err_word);
+                for (int j = (issued_v > C::kStagesV ? issued_v - C::kStagesV : 0); j < issued_v; ++j)
+                    wait_bar(bar.vf + 8 * (j % C::kStagesV), (j / C::kStagesV) & 1, &abort_flag, p.err_word);
             }
-        }
-        __syncwarp();
-    } else {
-        // ------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        } else if (warp == 9 && lane == 0) {
+            // ------------------------------------------------ MMA issuer
             constexpr uint32_t idesc_qk = idesc_bf16(kBlockM, kBlockN, false);
             constexpr uint32_t idesc_pv = idesc_bf16(kBlockM, DH, true);
-            bool ok = wait_bar(bar_q, 0, &abort_flag, p.err_word);
-            auto issue_qk = [&](int j) -> bool {
-                const int st = j % C::kStages;
-                if (!wait_bar(bar_kf + 8 * st, (j / C::kStages) & 1, &abort_flag, p.err_word)) return false;
-                tc_fence_after();
-                const uint32_t d_s = tmem + (j & 1) * 128;
+            auto issue_qk = [&](int t, int st) {          // S_t = Q_t K^T
 #pragma unroll
                 for (int ks = 0; ks < DH / 16; ++ks) {
                     const uint32_t off = (ks >> 2) * C::kChunkBytes + (ks & 3) * 32;
-                    mma_ss(d_s, smem_desc(sQ + off, 16, 1024, kSwizzle128B),
+                    mma_ss(tmem + t * 128, smem_desc(sQ + t * C::kTileBytes + off, 16, 1024, kSwizzle128B),
                            smem_desc(sK + st * C::kTileBytes + off, 16, 1024, kSwizzle128B), idesc_qk, ks > 0);
                 }
-                tc_commit(bar_s + 8 * (j & 1));
-                tc_commit(bar_ke + 8 * st);
-                return true;
+                tc_commit(bar.s + 8 * t);
             };
-            if (ok) ok = issue_qk(0);
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                if (j + 1 < n_tiles) { ok = issue_qk(j + 1); if (!ok) break; }
-                ok = wait_bar(bar_p + 8 * (j & 1), (j >> 1) & 1, &abort_flag, p.err_word);
-                if (!ok) break;
-                const int st = j % C::kStages;
-                ok = wait_bar(bar_vf + 8 * st, (j / C::kStages) & 1, &abort_flag, p.err_word);
-                if (!ok) break;
-                tc_fence_after();
+            auto issue_pv = [&](int t, int st, int j) {   // O_t += P_t V
 #pragma unroll
-                for (int ks = 0; ks < kBlockN / 16; ++ks) {
-                    mma_ts(tmem + kColO, tmem + (j & 1) * 128 + ks * 8,
+                for (int ks = 0; ks < kBlockN / 16; ++ks)
+                    mma_ts(tmem + kColO + t * 128, tmem + t * 128 + ks * 8,
                            smem_desc(sV + st * C::kTileBytes + ks * 2048, C::kChunkBytes, 1024, kSwizzle128B),
                            idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+                tc_commit(bar.o + 8 * t);
+            };
+            bool ok = wait_bar(bar.kf, 0, &abort_flag, p.err_word);
+            for (int t = 0; t < kTilesM && ok; ++t) {
+                ok = wait_bar(bar.q + 8 * t, 0, &abort_flag, p.err_word);
+                if (!ok) break;
+                tc_fence_after();
+                issue_qk(t, 0);
+            }
+            if (ok) tc_commit(bar.ke);
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const int sv = j % C::kStagesV;
+                const int sk = (j + 1) % C::kStagesK;
+                const bool more = j + 1 < n_tiles;
+                for (int t = 0; t < kTilesM; ++t) {
+                    ok = wait_bar(bar.p + 8 * t, j & 1, &abort_flag, p.err_word);
+                    if (ok && t == 0) ok = wait_bar(bar.vf + 8 * sv, (j / C::kStagesV) & 1, &abort_flag, p.err_word);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv(t, sv, j);
+                    if (more) {
+                        if (t == 0) {
+                            ok = wait_bar(bar.kf + 8 * sk, ((j + 1) / C::kStagesK) & 1, &abort_flag, p.err_word);
+                            if (!ok) break;
+                            tc_fence_after();
+                        }
+                        issue_qk(t, sk);          // overwrites S_t / P_t after the PV above has read it (in-order pipe)
+                    }
                 }
-                tc_commit(bar_o);
-                tc_commit(bar_ve + 8 * st);
+                if (!ok) break;
+                tc_commit(bar.ve + 8 * sv);
+                if (more) tc_commit(bar.ke + 8 * sk);
             }
         }
         __syncwarp();
@@ -353,7 +398,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) tmem_dealloc(tmem, kTmemCols);
+    if (warp == 9) tmem_dealloc(tmem, kTmemCols);
 }
 
 // ------------------------------------------------------------------ host side
@@ -416,7 +461,7 @@ int32_t launch_dh(const AttnArgs &a, cudaStream_t stream)
     p.scale_log2 = a.scale * 1.4426950408889634f;
     p.compact = (a.flags & ASTRAEA_ATTN_COMPACT_OUT) ? 1 : 0;
     p.err_word = a.err_word;
-    dim3 grid((a.M + kBlockM - 1) / kBlockM, a.H, a.B);
+    dim3 grid((a.M + kTilesM * kBlockM - 1) / (kTilesM * kBlockM), a.H, a.B);
     sparse_attn_kernel<DH><<<grid, kThreads, C::kSmemBytes, stream>>>(mk, mv, p);
     return check_launch("astraea_sparse_attn");
 }
