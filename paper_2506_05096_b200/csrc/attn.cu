@@ -2,19 +2,22 @@
 // against ALL keys/values, written in place over the cached output (Algorithm 1 lines 6-7;
 // Section 3.2 "Sparse Attention").
 //
-// One CTA per (256 selected queries, head, batch): two 128-row query tiles A and B that
-// share every K/V tile and alternate on the tensor core, so that one tile's softmax runs
-// while the other tile's MMAs execute.  Warp roles (384 threads, three warpgroups):
-//   warpgroup 0 / 1  softmax of tile A / B: gather the tile's Q rows into 128B-swizzled shared
-//              memory, then per key tile read S from TMEM (one thread per query row), online
-//              softmax in the log2 domain with lazy rescaling of O, write P (bf16) back to
-//              TMEM over S, and at the end normalise O and scatter it to the rows q_idx names;
-//   warp 8     TMA producer: K and V tiles (128 keys) into multi-stage swizzled buffers;
+// One CTA per (256 selected queries, head, batch): two 128-row query tiles that share every
+// K/V tile of 64 keys.  Warp roles (320 threads):
+//   warps 0-3 / 4-7  softmax of query tile 0 / 1: gather the tile's Q rows into 128B-swizzled
+//              shared memory, then per key tile read S from TMEM (one thread per query row),
+//              online softmax in the log2 domain with lazy rescaling of O, write P (bf16) back
+//              to TMEM over S, and at the end normalise O and scatter it to the rows q_idx names;
+//   warp 8     TMA producer: K and V tiles into multi-stage swizzled buffers;
 //   warp 9     tcgen05.mma issuer: S = Q K^T (SS, K-major operands), O += P V (P from TMEM,
 //              V as an MN-major shared-memory operand); owns the TMEM allocation.
-// Registers are rebalanced with setmaxnreg (softmax warpgroups up, the third one down).
-// TMEM columns: S/P of tile A [0,128), of tile B [128,256), O of A [256,256+d), of B [384,384+d).
-// Every mbarrier wait is bounded; on a timeout the CTA raises the error word and leaves.
+// S is double-buffered per query tile, so the QK^T of key tile j+1 is already in TMEM while the
+// softmax of tile j runs: the softmax warps never wait for the tensor core in steady state.
+// TMEM columns: S/P of (tile t, buffer u) at (2t+u)*64; O of tile t at 256 + 128 t.
+// The producer and issuer warps run warp-uniform code and elect one lane per instruction, so
+// that descriptors and addresses stay in uniform registers (a lone diverged thread issues
+// tcgen05.mma several times slower).  Every mbarrier wait is bounded; on a timeout the CTA
+// raises the error word, the remaining waits return at once, and the CTA runs out.
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -25,8 +28,8 @@ using namespace ptx;
 
 constexpr int kBlockM = 128;                     // rows of one query tile
 constexpr int kTilesM = 2;                       // query tiles per CTA
-constexpr int kBlockN = 128;
-constexpr int kThreads = 384;
+constexpr int kBlockN = 64;                      // keys per K/V tile
+constexpr int kThreads = 320;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColO = 256;
 constexpr float kRescaleThreshold = 8.0f;        // log2 units: P stays below 2^8
@@ -34,12 +37,14 @@ constexpr uint64_t kWaitLimitNs = 1000000000ull; // bounded waits: one second
 
 template <int DH> struct Cfg {
     static constexpr int kChunks = DH / 64;                       // 64-column (128-byte) swizzle chunks
-    static constexpr int kChunkBytes = 128 * 128;                 // 128 rows x 128 bytes
-    static constexpr int kTileBytes = kChunks * kChunkBytes;      // one Q / K / V tile
-    static constexpr int kStagesK = (DH == 128) ? 3 : 5;
-    static constexpr int kStagesV = (DH == 128) ? 2 : 5;
-    static constexpr int kBarBytes = 256;
-    static constexpr int kSmemBytes = kTileBytes * (kTilesM + kStagesK + kStagesV) + kBarBytes + 1024;
+    static constexpr int kQChunkBytes = kBlockM * 128;            // 128 query rows x 128 bytes
+    static constexpr int kQTileBytes = kChunks * kQChunkBytes;
+    static constexpr int kChunkBytes = kBlockN * 128;             // 64 keys x 128 bytes
+    static constexpr int kTileBytes = kChunks * kChunkBytes;      // one K or V tile
+    static constexpr int kStagesK = (DH == 128) ? 5 : 6;
+    static constexpr int kStagesV = (DH == 128) ? 5 : 6;
+    static constexpr int kBarBytes = 512;
+    static constexpr int kSmemBytes = kQTileBytes * kTilesM + kTileBytes * (kStagesK + kStagesV) + kBarBytes + 1024;
 };
 
 struct Params {
@@ -61,26 +66,34 @@ __device__ __forceinline__ float ex2(float x) {
     return y;
 }
 
-// Bounded mbarrier wait.  Returns false after the limit or once another role has given up.
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err_word) {
-    if (mbar_try_wait(bar, parity)) return true;
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred px;\n\telect.sync _|px, 0xffffffff;\n\tselp.u32 %0, 1, 0, px;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
+
+// Bounded mbarrier wait.  Gives up after the limit, or at once when another wait of this CTA
+// already gave up; the caller carries on (its results are void, the error word says so).
+__device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err_word) {
+    if (mbar_try_wait(bar, parity)) return;
+    if (*abort_flag) return;
     const uint64_t t0 = globaltimer_ns();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 255u) == 0) {
-            if (*abort_flag) return false;
+            if (*abort_flag) return;
             if (globaltimer_ns() - t0 > kWaitLimitNs) {
                 *abort_flag = 1;
                 atomicExch(err_word, kErrTimeout);
-                return false;
+                return;
             }
         }
     }
-    return true;
 }
 
 struct Bars {
-    uint32_t q, s, p, o;            // [kTilesM] each
+    uint32_t q, o;                  // [kTilesM]
+    uint32_t s, p;                  // [kTilesM][2]
     uint32_t kf, ke, vf, ve;        // [stages]
 };
 
@@ -90,7 +103,8 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
                                              int m_base, int h, int b, int n_tiles, volatile int *abort_flag)
 {
     using C = Cfg<DH>;
-    const int wtid = threadIdx.x & 127, warp = wtid >> 5, lane = wtid & 31;
+    const int wtid = threadIdx.x & 127, lane = wtid & 31;
+    const int warp = __shfl_sync(0xffffffffu, wtid >> 5, 0);       // warp-uniform
     // gather this tile's Q rows (swizzled, K-major)
     constexpr int kVecPerRow = DH / 8;                 // 16-byte vectors per row
     constexpr int kRowsPerIter = 32 / kVecPerRow;
@@ -108,7 +122,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
                     val = __ldg(reinterpret_cast<const uint4 *>(src));
                 }
             }
-            const uint32_t off = (c >> 3) * C::kChunkBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
+            const uint32_t off = (c >> 3) * C::kQChunkBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
             *reinterpret_cast<uint4 *>(sQ_gen + off) = val;
         }
     }
@@ -116,9 +130,9 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     mbar_arrive(bar.q + 8 * tile);
 
     const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);
-    const uint32_t t_s = t_row + tile * 128;
+    const uint32_t t_s0 = t_row + tile * 128;
     const uint32_t t_o = t_row + kColO + tile * 128;
-    const uint32_t bar_s = bar.s + 8 * tile, bar_p = bar.p + 8 * tile, bar_o = bar.o + 8 * tile;
+    const uint32_t bar_s = bar.s + 16 * tile, bar_p = bar.p + 16 * tile, bar_o = bar.o + 8 * tile;
     const int m = m_base + wtid;
     int tok = -1;
     if (m < p.M) {
@@ -127,27 +141,22 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     }
     const float sl2 = p.scale_log2;
     float m_ref = -INFINITY, l_sum = 0.f;
-    bool ok = true;
 
     for (int j = 0; j < n_tiles; ++j) {
-        ok = wait_bar(bar_s, j & 1, abort_flag, p.err_word);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
+        const int buf = j & 1;
+        const uint32_t t_s = t_s0 + buf * kBlockN;
+        wait_bar(bar_s + 8 * buf, (j >> 1) & 1, abort_flag, p.err_word);
         tc_fence_after();
         float s[kBlockN];
         {
-            uint32_t t0[32], t1[32], t2[32], t3[32];
+            uint32_t t0[32], t1[32];
             tmem_ld32(t_s, t0);
             tmem_ld32(t_s + 32, t1);
-            tmem_ld32(t_s + 64, t2);
-            tmem_ld32(t_s + 96, t3);
             tc_wait_ld();
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
                 s[i] = __uint_as_float(t0[i]);
                 s[32 + i] = __uint_as_float(t1[i]);
-                s[64 + i] = __uint_as_float(t2[i]);
-                s[96 + i] = __uint_as_float(t3[i]);
             }
         }
         const int valid = p.N - j * kBlockN;           // keys of this tile that exist
@@ -171,9 +180,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
             if (__any_sync(0xffffffffu, need)) {
                 float alpha = 1.0f;
                 if (need) { alpha = ex2((m_ref - mx) * sl2); m_ref = mx; l_sum *= alpha; }
-                ok = wait_bar(bar_o, (j - 1) & 1, abort_flag, p.err_word);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
+                wait_bar(bar_o, (j - 1) & 1, abort_flag, p.err_word);     // P V of the previous key tile has landed
                 tc_fence_after();
 #pragma unroll
                 for (int cc = 0; cc < DH / 32; ++cc) {
@@ -195,56 +202,50 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
             for (int u = 0; u < 4; ++u) { s[i + u] = ex2(fmaf(s[i + u], sl2, neg)); sum4[u] += s[i + u]; }
         }
         l_sum += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-        // P as bf16 pairs over the first 64 columns of this S buffer (element 2c in the low half)
-#pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {
+        // P as bf16 pairs over the first 32 columns of this S buffer (element 2c in the low half)
+        {
             uint32_t pk[32];
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
-                __nv_bfloat162 v2 = __floats2bfloat162_rn(s[cc * 64 + 2 * i], s[cc * 64 + 2 * i + 1]);
+                __nv_bfloat162 v2 = __floats2bfloat162_rn(s[2 * i], s[2 * i + 1]);
                 pk[i] = *reinterpret_cast<uint32_t *>(&v2);
             }
-            tmem_st32(t_s + cc * 32, pk);
+            tmem_st32(t_s, pk);
         }
         tc_wait_st();
         tc_fence_before();
-        mbar_arrive(bar_p);
+        mbar_arrive(bar_p + 8 * buf);
     }
 
     // epilogue: normalise and scatter
-    if (ok) {
-        ok = wait_bar(bar_o, (n_tiles - 1) & 1, abort_flag, p.err_word);
-        ok = __all_sync(0xffffffffu, ok);
-    }
-    if (ok) {
-        tc_fence_after();
-        const float inv_l = 1.0f / l_sum;
-        __nv_bfloat16 *dst = nullptr;
-        if (tok >= 0) {
-            const size_t orow = p.compact ? ((size_t)b * p.M + m) : ((size_t)b * p.N + tok);
-            dst = p.out + (orow * p.H + h) * DH;
-            if (p.lse_out) {
-                const size_t li = p.compact ? (((size_t)b * p.H + h) * p.M + m) : (((size_t)b * p.H + h) * p.N + tok);
-                p.lse_out[li] = m_ref * p.scale + logf(l_sum);
-            }
+    wait_bar(bar_o, (n_tiles - 1) & 1, abort_flag, p.err_word);
+    tc_fence_after();
+    const float inv_l = 1.0f / l_sum;
+    __nv_bfloat16 *dst = nullptr;
+    if (tok >= 0 && !*abort_flag) {
+        const size_t orow = p.compact ? ((size_t)b * p.M + m) : ((size_t)b * p.N + tok);
+        dst = p.out + (orow * p.H + h) * DH;
+        if (p.lse_out) {
+            const size_t li = p.compact ? (((size_t)b * p.H + h) * p.M + m) : (((size_t)b * p.H + h) * p.N + tok);
+            p.lse_out[li] = m_ref * p.scale + logf(l_sum);
         }
+    }
 #pragma unroll
-        for (int cc = 0; cc < DH / 32; ++cc) {
-            uint32_t o[32];
-            tmem_ld32(t_o + cc * 32, o);
-            tc_wait_ld();
-            if (dst) {
+    for (int cc = 0; cc < DH / 32; ++cc) {
+        uint32_t o[32];
+        tmem_ld32(t_o + cc * 32, o);
+        tc_wait_ld();
+        if (dst) {
 #pragma unroll
-                for (int v = 0; v < 4; ++v) {
-                    uint32_t w[4];
+            for (int v = 0; v < 4; ++v) {
+                uint32_t w[4];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(o[v * 8 + 2 * i]) * inv_l,
-                                                                  __uint_as_float(o[v * 8 + 2 * i + 1]) * inv_l);
-                        w[i] = *reinterpret_cast<uint32_t *>(&v2);
-                    }
-                    *reinterpret_cast<uint4 *>(dst + cc * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                for (int i = 0; i < 4; ++i) {
+                    __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(o[v * 8 + 2 * i]) * inv_l,
+                                                              __uint_as_float(o[v * 8 + 2 * i + 1]) * inv_l);
+                    w[i] = *reinterpret_cast<uint32_t *>(&v2);
                 }
+                *reinterpret_cast<uint4 *>(dst + cc * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
             }
         }
     }
@@ -262,26 +263,27 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const uint32_t sQ = smem_base;
-    const uint32_t sK = sQ + kTilesM * C::kTileBytes;
+    const uint32_t sK = sQ + kTilesM * C::kQTileBytes;
     const uint32_t sV = sK + C::kStagesK * C::kTileBytes;
     const uint32_t bars = sV + C::kStagesV * C::kTileBytes;
     Bars bar;
-    bar.q = bars; bar.s = bars + 16; bar.p = bars + 32; bar.o = bars + 48;
-    bar.kf = bars + 64;
+    bar.q = bars; bar.o = bars + 16; bar.s = bars + 32; bar.p = bars + 64;
+    bar.kf = bars + 96;
     bar.ke = bar.kf + 8 * C::kStagesK;
     bar.vf = bar.ke + 8 * C::kStagesK;
     bar.ve = bar.vf + 8 * C::kStagesV;
-    static_assert(64 + 16 * (C::kStagesK + C::kStagesV) <= C::kBarBytes, "barrier area too small");
+    static_assert(96 + 16 * (C::kStagesK + C::kStagesV) <= C::kBarBytes, "barrier area too small");
 
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, wg = tid >> 7;
+    const int tid = threadIdx.x;
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);        // warp-uniform
     const int m0 = blockIdx.x * (kTilesM * kBlockM), h = blockIdx.y, b = blockIdx.z;
     const int n_tiles = (p.N + kBlockN - 1) / kBlockN;
 
     if (tid == 0) {
         abort_flag = 0;
         for (int t = 0; t < kTilesM; ++t) {
-            mbar_init(bar.q + 8 * t, 128); mbar_init(bar.s + 8 * t, 1);
-            mbar_init(bar.p + 8 * t, 128); mbar_init(bar.o + 8 * t, 1);
+            mbar_init(bar.q + 8 * t, 128); mbar_init(bar.o + 8 * t, 1);
+            for (int u = 0; u < 2; ++u) { mbar_init(bar.s + 16 * t + 8 * u, 1); mbar_init(bar.p + 16 * t + 8 * u, 128); }
         }
         for (int s = 0; s < C::kStagesK; ++s) { mbar_init(bar.kf + 8 * s, 1); mbar_init(bar.ke + 8 * s, 1); }
         for (int s = 0; s < C::kStagesV; ++s) { mbar_init(bar.vf + 8 * s, 1); mbar_init(bar.ve + 8 * s, 1); }
@@ -296,104 +298,95 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
 
-    if (wg < 2) {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
-        softmax_role<DH>(p, bar, wg, smem_gen + wg * C::kTileBytes, tmem, m0 + wg * kBlockM, h, b, n_tiles, &abort_flag);
-    } else {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
-        if (warp == 8 && lane == 0) {
-            // ------------------------------------------------ TMA producer
-            prefetch_tensormap(&tmap_k);
-            prefetch_tensormap(&tmap_v);
-            int issued_k = 0, issued_v = 0;
-            bool ok = true;
-            auto load_k = [&](int j) -> bool {
-                const int st = j % C::kStagesK;
-                if (!wait_bar(bar.ke + 8 * st, ((j / C::kStagesK) & 1) ^ 1, &abort_flag, p.err_word)) return false;
+    if (warp < 8) {
+        const int tile = warp >> 2;
+        softmax_role<DH>(p, bar, tile, smem_gen + tile * C::kQTileBytes, tmem, m0 + tile * kBlockM, h, b, n_tiles, &abort_flag);
+    } else if (warp == 8) {
+        // ------------------------------------------------ TMA producer (warp-uniform, one elected lane issues)
+        if (elect_one()) { prefetch_tensormap(&tmap_k); prefetch_tensormap(&tmap_v); }
+        auto load_k = [&](int j) {
+            const int st = j % C::kStagesK;
+            wait_bar(bar.ke + 8 * st, ((j / C::kStagesK) & 1) ^ 1, &abort_flag, p.err_word);
+            if (elect_one()) {
                 mbar_arrive_expect_tx(bar.kf + 8 * st, C::kTileBytes);
 #pragma unroll
                 for (int ch = 0; ch < C::kChunks; ++ch)
                     tma_load_4d(sK + st * C::kTileBytes + ch * C::kChunkBytes, &tmap_k, bar.kf + 8 * st, ch * 64, j * kBlockN, h, b);
-                issued_k = j + 1;
-                return true;
-            };
-            auto load_v = [&](int j) -> bool {
-                const int st = j % C::kStagesV;
-                if (!wait_bar(bar.ve + 8 * st, ((j / C::kStagesV) & 1) ^ 1, &abort_flag, p.err_word)) return false;
+            }
+            __syncwarp();
+        };
+        auto load_v = [&](int j) {
+            const int st = j % C::kStagesV;
+            wait_bar(bar.ve + 8 * st, ((j / C::kStagesV) & 1) ^ 1, &abort_flag, p.err_word);
+            if (elect_one()) {
                 mbar_arrive_expect_tx(bar.vf + 8 * st, C::kTileBytes);
 #pragma unroll
                 for (int ch = 0; ch < C::kChunks; ++ch)
                     tma_load_4d(sV + st * C::kTileBytes + ch * C::kChunkBytes, &tmap_v, bar.vf + 8 * st, ch * 64, j * kBlockN, h, b);
-                issued_v = j + 1;
-                return true;
-            };
-            // K runs one tile ahead of V: K_{j+1} is needed before V_j
-            ok = load_k(0);
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                if (j + 1 < n_tiles) ok = load_k(j + 1);
-                if (ok) ok = load_v(j);
             }
-            if (!ok) {
-                // leaving early: let the copies already issued land before the CTA's shared memory is released
-                for (int j = (issued_k > C::kStagesK ? issued_k - C::kStagesK : 0); j < issued_k; ++j)
-                    wait_bar(bar.kf + 8 * (j % C::kStagesK), (j / C::kStagesK) & 1, &abort_flag, p.err_word);
-                for (int j = (issued_v > C::kStagesV ? issued_v - C::kStagesV : 0); j < issued_v; ++j)
-                    wait_bar(bar.vf + 8 * (j % C::kStagesV), (j / C::kStagesV) & 1, &abort_flag, p.err_word);
-            }
-        } else if (warp == 9 && lane == 0) {
-            // ------------------------------------------------ MMA issuer
-            constexpr uint32_t idesc_qk = idesc_bf16(kBlockM, kBlockN, false);
-            constexpr uint32_t idesc_pv = idesc_bf16(kBlockM, DH, true);
-            auto issue_qk = [&](int t, int st) {          // S_t = Q_t K^T
+            __syncwarp();
+        };
+        // K runs one tile ahead of V: K_{j+1} is needed before V_j
+        load_k(0);
+        for (int j = 0; j < n_tiles; ++j) {
+            if (j + 1 < n_tiles) load_k(j + 1);
+            load_v(j);
+        }
+        // every copy issued above must have landed before the CTA's shared memory is released
+        for (int j = (n_tiles > C::kStagesK ? n_tiles - C::kStagesK : 0); j < n_tiles; ++j)
+            wait_bar(bar.kf + 8 * (j % C::kStagesK), (j / C::kStagesK) & 1, &abort_flag, p.err_word);
+        for (int j = (n_tiles > C::kStagesV ? n_tiles - C::kStagesV : 0); j < n_tiles; ++j)
+            wait_bar(bar.vf + 8 * (j % C::kStagesV), (j / C::kStagesV) & 1, &abort_flag, p.err_word);
+    } else {
+        // ------------------------------------------------ MMA issuer (warp-uniform, one elected lane issues)
+        constexpr uint32_t idesc_qk = idesc_bf16(kBlockM, kBlockN, false);
+        constexpr uint32_t idesc_pv = idesc_bf16(kBlockM, DH, true);
+        auto issue_qk = [&](int j) {                  // S[t][j&1] = Q_t K_j^T for both query tiles
+            const int st = j % C::kStagesK;
+            const uint32_t kbase = sK + st * C::kTileBytes;
+            const uint32_t sbuf = (j & 1) * kBlockN;
+            wait_bar(bar.kf + 8 * st, (j / C::kStagesK) & 1, &abort_flag, p.err_word);
+            tc_fence_after();
+            if (elect_one()) {
 #pragma unroll
-                for (int ks = 0; ks < DH / 16; ++ks) {
-                    const uint32_t off = (ks >> 2) * C::kChunkBytes + (ks & 3) * 32;
-                    mma_ss(tmem + t * 128, smem_desc(sQ + t * C::kTileBytes + off, 16, 1024, kSwizzle128B),
-                           smem_desc(sK + st * C::kTileBytes + off, 16, 1024, kSwizzle128B), idesc_qk, ks > 0);
-                }
-                tc_commit(bar.s + 8 * t);
-            };
-            auto issue_pv = [&](int t, int st, int j) {   // O_t += P_t V
-#pragma unroll
-                for (int ks = 0; ks < kBlockN / 16; ++ks)
-                    mma_ts(tmem + kColO + t * 128, tmem + t * 128 + ks * 8,
-                           smem_desc(sV + st * C::kTileBytes + ks * 2048, C::kChunkBytes, 1024, kSwizzle128B),
-                           idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
-                tc_commit(bar.o + 8 * t);
-            };
-            bool ok = wait_bar(bar.kf, 0, &abort_flag, p.err_word);
-            for (int t = 0; t < kTilesM && ok; ++t) {
-                ok = wait_bar(bar.q + 8 * t, 0, &abort_flag, p.err_word);
-                if (!ok) break;
-                tc_fence_after();
-                issue_qk(t, 0);
-            }
-            if (ok) tc_commit(bar.ke);
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                const int sv = j % C::kStagesV;
-                const int sk = (j + 1) % C::kStagesK;
-                const bool more = j + 1 < n_tiles;
                 for (int t = 0; t < kTilesM; ++t) {
-                    ok = wait_bar(bar.p + 8 * t, j & 1, &abort_flag, p.err_word);
-                    if (ok && t == 0) ok = wait_bar(bar.vf + 8 * sv, (j / C::kStagesV) & 1, &abort_flag, p.err_word);
-                    if (!ok) break;
-                    tc_fence_after();
-                    issue_pv(t, sv, j);
-                    if (more) {
-                        if (t == 0) {
-                            ok = wait_bar(bar.kf + 8 * sk, ((j + 1) / C::kStagesK) & 1, &abort_flag, p.err_word);
-                            if (!ok) break;
-                            tc_fence_after();
-                        }
-                        issue_qk(t, sk);          // overwrites S_t / P_t after the PV above has read it (in-order pipe)
-                    }
+#pragma unroll
+                    for (int ks = 0; ks < DH / 16; ++ks)
+                        mma_ss(tmem + t * 128 + sbuf,
+                               smem_desc(sQ + t * C::kQTileBytes + (ks >> 2) * C::kQChunkBytes + (ks & 3) * 32, 16, 1024, kSwizzle128B),
+                               smem_desc(kbase + (ks >> 2) * C::kChunkBytes + (ks & 3) * 32, 16, 1024, kSwizzle128B),
+                               idesc_qk, ks > 0);
+                    tc_commit(bar.s + 16 * t + 8 * (j & 1));
                 }
-                if (!ok) break;
-                tc_commit(bar.ve + 8 * sv);
-                if (more) tc_commit(bar.ke + 8 * sk);
+                tc_commit(bar.ke + 8 * st);
+            }
+            __syncwarp();
+        };
+        wait_bar(bar.q, 0, &abort_flag, p.err_word);
+        wait_bar(bar.q + 8, 0, &abort_flag, p.err_word);
+        issue_qk(0);
+        for (int j = 0; j < n_tiles; ++j) {
+            if (j + 1 < n_tiles) issue_qk(j + 1);     // its S buffer held P of tile j-1, already consumed in order
+            const int sv = j % C::kStagesV;
+            const uint32_t vbase = sV + sv * C::kTileBytes;
+            const uint32_t sbuf = (j & 1) * kBlockN;
+            wait_bar(bar.vf + 8 * sv, (j / C::kStagesV) & 1, &abort_flag, p.err_word);
+#pragma unroll
+            for (int t = 0; t < kTilesM; ++t) {
+                wait_bar(bar.p + 16 * t + 8 * (j & 1), (j >> 1) & 1, &abort_flag, p.err_word);
+                tc_fence_after();
+                if (elect_one()) {
+#pragma unroll
+                    for (int ks = 0; ks < kBlockN / 16; ++ks)
+                        mma_ts(tmem + kColO + t * 128, tmem + t * 128 + sbuf + ks * 8,
+                               smem_desc(vbase + ks * 2048, C::kChunkBytes, 1024, kSwizzle128B),
+                               idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+                    tc_commit(bar.o + 8 * t);
+                    if (t == kTilesM - 1) tc_commit(bar.ve + 8 * sv);
+                }
+                __syncwarp();
             }
         }
-        __syncwarp();
     }
 
     tc_fence_before();
@@ -426,7 +419,7 @@ int32_t make_kv_map(CUtensorMap *map, const void *base, int B, int H, int N, int
     if (!enc) return fail(ASTRAEA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
     cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)H, (cuuint64_t)B};
     cuuint64_t strides[3] = {(cuuint64_t)sn * 2, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
-    cuuint32_t box[4] = {64, (cuuint32_t)kBlockN, 1, 1};
+    cuuint32_t box[4] = {64, (cuuint32_t)kBlockN, 1, 1};   // 64 columns x one key tile
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
