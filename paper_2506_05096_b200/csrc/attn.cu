@@ -3,21 +3,32 @@
 // Section 3.2 "Sparse Attention").
 //
 // One CTA per (256 selected queries, head, batch): two 128-row query tiles that share every
-// K/V tile of 64 keys.  Warp roles (320 threads):
-//   warps 0-3 / 4-7  softmax of query tile 0 / 1: gather the tile's Q rows into 128B-swizzled
-//              shared memory, then per key tile read S from TMEM (one thread per query row),
-//              online softmax in the log2 domain with lazy rescaling of O, write P (bf16) back
-//              to TMEM over S, and at the end normalise O and scatter it to the rows q_idx names;
-//   warp 8     TMA producer: K and V tiles into multi-stage swizzled buffers;
-//   warp 9     tcgen05.mma issuer: S = Q K^T (SS, K-major operands), O += P V (P from TMEM,
+// K/V tile of 64 keys.  Warp roles:
+//   softmax warpgroups (one thread per query row): gather the tile's Q rows into 128B-swizzled
+//              shared memory, then per key tile read S from TMEM, online softmax in the log2 domain
+//              with lazy rescaling of O, write P (bf16) back to TMEM over S, and at the end
+//              normalise O and scatter it to the rows q_idx names;
+//   one warp   TMA producer: K and V tiles into multi-stage swizzled buffers;
+//   one warp   tcgen05.mma issuer: S = Q K^T (SS, K-major operands), O += P V (P from TMEM,
 //              V as an MN-major shared-memory operand); owns the TMEM allocation.
-// S is double-buffered per query tile, so the QK^T of key tile j+1 is already in TMEM while the
-// softmax of tile j runs: the softmax warps never wait for the tensor core in steady state.
-// TMEM columns: S/P of (tile t, buffer u) at (2t+u)*64; O of tile t at 256 + 128 t.
+// S is double-buffered per query tile and refilled with key tile j+2 as soon as P of tile j has
+// been consumed.
+//
+// The exponentials (XU pipe, 16 per clock per SM) bound the softmax.  One warp alone cannot keep
+// its XU sub-pipe busy, and at head_dim 64 the MMAs of a key tile are much shorter than its
+// exponentials.  So at head_dim 64 every query tile has TWO softmax warpgroups: even key tiles go
+// to one, odd ones to the other, each with its own running maximum, row sum and O accumulator in
+// TMEM (a split over keys inside the CTA), merged once in the epilogue.  That gives four softmax
+// warps per SM sub-partition.  At head_dim 128 the MMAs are as long as the exponentials and TMEM
+// has no room for four accumulators: one warpgroup per query tile, which prefetches S of the next
+// key tile and reduces its maximum while the current tile's exponentials execute.
+//
+// TMEM columns: S/P of (tile t, buffer u) at (2t+u)*64; O accumulators from column 256.
 // The producer and issuer warps run warp-uniform code and elect one lane per instruction, so
 // that descriptors and addresses stay in uniform registers (a lone diverged thread issues
-// tcgen05.mma several times slower).  Every mbarrier wait is bounded; on a timeout the CTA
-// raises the error word, the remaining waits return at once, and the CTA runs out.
+// tcgen05.mma several times slower).  setmaxnreg moves registers from the last warpgroup to the
+// softmax warpgroups.  Every mbarrier wait is bounded; on a timeout the CTA raises the error
+// word, the remaining waits return at once, and the CTA runs out.
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -29,13 +40,22 @@ using namespace ptx;
 constexpr int kBlockM = 128;                     // rows of one query tile
 constexpr int kTilesM = 2;                       // query tiles per CTA
 constexpr int kBlockN = 64;                      // keys per K/V tile
-constexpr int kThreads = 320;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColO = 256;
 constexpr float kRescaleThreshold = 8.0f;        // log2 units: P stays below 2^8
 constexpr uint64_t kWaitLimitNs = 1000000000ull; // bounded waits: one second
 
 template <int DH> struct Cfg {
+    static constexpr int kSplit = 1;              // softmax warpgroups per query tile
+    static constexpr int kSoftmaxWarps = 4 * kTilesM * kSplit;
+    static constexpr int kThreads = (kSoftmaxWarps + 4) * 32;     // + producer, issuer, two register donors
+    // setmaxnreg only redistributes what the CTA got at launch (kRegsLaunch per thread): an increase
+    // that the decreases of the last warpgroup cannot cover would block forever
+    static constexpr int kRegsLaunch = (65536 / kThreads) / 8 * 8;
+    static constexpr int kRegsSoftmax = (kSplit == 2) ? 112 : 232;
+    static constexpr int kRegsOther = (kSplit == 2) ? 32 : 40;
+    static_assert(kRegsSoftmax * kSoftmaxWarps * 32 + kRegsOther * 128 <= kRegsLaunch * kThreads, "setmaxnreg budget");
+    static constexpr uint32_t kOStride = 128 / kSplit;            // TMEM columns between O accumulators
     static constexpr int kChunks = DH / 64;                       // 64-column (128-byte) swizzle chunks
     static constexpr int kQChunkBytes = kBlockM * 128;            // 128 query rows x 128 bytes
     static constexpr int kQTileBytes = kChunks * kQChunkBytes;
@@ -45,6 +65,7 @@ template <int DH> struct Cfg {
     static constexpr int kStagesV = (DH == 128) ? 5 : 6;
     static constexpr int kBarBytes = 512;
     static constexpr int kSmemBytes = kQTileBytes * kTilesM + kTileBytes * (kStagesK + kStagesV) + kBarBytes + 1024;
+    static_assert(kColO + kTilesM * kSplit * kOStride <= kTmemCols && DH <= (int)kOStride, "TMEM budget");
 };
 
 struct Params {
@@ -64,6 +85,12 @@ __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
 }
 
 __device__ __forceinline__ bool elect_one() {
@@ -92,26 +119,150 @@ __device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, volatile
 }
 
 struct Bars {
-    uint32_t q, o;                  // [kTilesM]
-    uint32_t s, p;                  // [kTilesM][2]
+    uint32_t q;                     // [kTilesM]
+    uint32_t s, p, o;               // [kTilesM][2]
     uint32_t kf, ke, vf, ve;        // [stages]
 };
 
-// ---------------------------------------------------------------- softmax warpgroup (one query tile)
+struct SoftmaxState {
+    float sl2, m_ref, l_sum;
+    uint32_t t_s0, t_o, bar_s, bar_p, bar_o;
+    int N, n_tiles;
+    volatile int *abort_flag;
+    int *err_word;
+};
+
+// 64 columns of one S buffer into registers (asynchronous: wait_s_regs before using them)
+__device__ __forceinline__ void load_s(uint32_t t_s, float (&s)[kBlockN]) {
+    tmem_ld32(t_s, reinterpret_cast<uint32_t (&)[32]>(s[0]));
+    tmem_ld32(t_s + 32, reinterpret_cast<uint32_t (&)[32]>(s[32]));
+}
+// tcgen05.wait::ld that names the loaded registers, so that no use of them can move above it
+__device__ __forceinline__ void wait_s_regs(float (&s)[kBlockN]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+        : "+f"(s[0]), "+f"(s[1]), "+f"(s[2]), "+f"(s[3]), "+f"(s[4]), "+f"(s[5]), "+f"(s[6]), "+f"(s[7]),
+          "+f"(s[8]), "+f"(s[9]), "+f"(s[10]), "+f"(s[11]), "+f"(s[12]), "+f"(s[13]), "+f"(s[14]), "+f"(s[15]),
+          "+f"(s[16]), "+f"(s[17]), "+f"(s[18]), "+f"(s[19]), "+f"(s[20]), "+f"(s[21]), "+f"(s[22]), "+f"(s[23]),
+          "+f"(s[24]), "+f"(s[25]), "+f"(s[26]), "+f"(s[27]), "+f"(s[28]), "+f"(s[29]), "+f"(s[30]), "+f"(s[31])
+        :: "memory");
+    asm volatile(""
+        : "+f"(s[32]), "+f"(s[33]), "+f"(s[34]), "+f"(s[35]), "+f"(s[36]), "+f"(s[37]), "+f"(s[38]), "+f"(s[39]),
+          "+f"(s[40]), "+f"(s[41]), "+f"(s[42]), "+f"(s[43]), "+f"(s[44]), "+f"(s[45]), "+f"(s[46]), "+f"(s[47]),
+          "+f"(s[48]), "+f"(s[49]), "+f"(s[50]), "+f"(s[51]), "+f"(s[52]), "+f"(s[53]), "+f"(s[54]), "+f"(s[55]),
+          "+f"(s[56]), "+f"(s[57]), "+f"(s[58]), "+f"(s[59]), "+f"(s[60]), "+f"(s[61]), "+f"(s[62]), "+f"(s[63])
+        :: "memory");
+}
+
+// maximum of the row's logits in one key tile; keys beyond `valid` (zero-filled tail) become -inf
+__device__ __forceinline__ float row_max(float (&s)[kBlockN], int valid) {
+    if (valid < kBlockN) {
+#pragma unroll
+        for (int i = 0; i < kBlockN; ++i) if (i >= valid) s[i] = -INFINITY;
+    }
+    float mx4[4] = {max3(s[0], s[1], s[2]), max3(s[3], s[4], s[5]), max3(s[6], s[7], s[8]), max3(s[9], s[10], s[11])};
+#pragma unroll
+    for (int i = 12; i + 7 < kBlockN; i += 8) {
+        mx4[0] = max3(mx4[0], s[i], s[i + 1]); mx4[1] = max3(mx4[1], s[i + 2], s[i + 3]);
+        mx4[2] = max3(mx4[2], s[i + 4], s[i + 5]); mx4[3] = max3(mx4[3], s[i + 6], s[i + 7]);
+    }
+    static_assert((kBlockN - 12) % 8 == 4, "tail of the max tree");
+    mx4[0] = max3(mx4[0], s[kBlockN - 4], s[kBlockN - 3]);
+    mx4[1] = max3(mx4[1], s[kBlockN - 2], s[kBlockN - 1]);
+    return fmaxf(max3(mx4[0], mx4[1], mx4[2]), mx4[3]);
+}
+
+// Moves the running maximum to mx when it has grown by more than the threshold, rescaling the row
+// sum and (once the previous P V of this accumulator has landed: o_parity) the O accumulator.
 template <int DH>
-__device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, int tile, uint8_t *sQ_gen, uint32_t tmem,
-                                             int m_base, int h, int b, int n_tiles, volatile int *abort_flag)
+__device__ __forceinline__ void maybe_rescale(SoftmaxState &st, float mx, bool first, uint32_t o_parity) {
+    if (first) { st.m_ref = mx; return; }
+    const bool need = (mx - st.m_ref) * st.sl2 > kRescaleThreshold;
+    if (__any_sync(0xffffffffu, need)) {
+        float alpha = 1.0f;
+        if (need) { alpha = ex2((st.m_ref - mx) * st.sl2); st.m_ref = mx; st.l_sum *= alpha; }
+        wait_bar(st.bar_o, o_parity, st.abort_flag, st.err_word);
+        tc_fence_after();
+#pragma unroll
+        for (int cc = 0; cc < DH / 32; ++cc) {
+            uint32_t o[32];
+            tmem_ld32(st.t_o + cc * 32, o);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+            tmem_st32(st.t_o + cc * 32, o);
+        }
+        tc_wait_st();
+    }
+}
+
+// exponentials of one key tile in place, their sum added to the row sum, P (bf16 pairs, element 2c
+// in the low half) stored over the first 32 columns of the S buffer, then the P barrier
+__device__ __forceinline__ void finish_tile(SoftmaxState &st, float (&cur)[kBlockN], int buf) {
+    float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int i = 0; i < kBlockN; i += 4) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) sum4[u] += cur[i + u];
+    }
+    st.l_sum += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+    uint32_t pk[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        __nv_bfloat162 v2 = __floats2bfloat162_rn(cur[2 * i], cur[2 * i + 1]);
+        pk[i] = *reinterpret_cast<uint32_t *>(&v2);
+    }
+    tmem_st32(st.t_s0 + buf * kBlockN, pk);
+    tc_wait_st();
+    tc_fence_before();
+    mbar_arrive(st.bar_p + 8 * buf);
+}
+
+// One key tile of the online softmax, one warpgroup per query tile.  `cur` holds S of tile j (row
+// maximum mx); S of tile j+1 is fetched into `nxt` and reduced while the exponentials of tile j
+// execute.  Returns the row maximum of tile j+1.
+template <int DH>
+__device__ __forceinline__ float softmax_step_prefetch(SoftmaxState &st, float (&cur)[kBlockN], float (&nxt)[kBlockN], int j, float mx)
+{
+    const int buf = j & 1;
+    const float sl2 = st.sl2;
+    maybe_rescale<DH>(st, mx, j == 0, (j - 1) & 1);
+    const bool more = j + 1 < st.n_tiles;
+    const float neg = -st.m_ref * sl2;
+#pragma unroll
+    for (int i = 0; i < kBlockN / 2; ++i) cur[i] = ex2(fmaf(cur[i], sl2, neg));
+    if (more) {
+        wait_bar(st.bar_s + 8 * (buf ^ 1), ((j + 1) >> 1) & 1, st.abort_flag, st.err_word);
+        tc_fence_after();
+        load_s(st.t_s0 + (buf ^ 1) * kBlockN, nxt);
+    }
+#pragma unroll
+    for (int i = kBlockN / 2; i < kBlockN; ++i) cur[i] = ex2(fmaf(cur[i], sl2, neg));
+    float mx_next = 0.f;
+    if (more) {
+        wait_s_regs(nxt);
+        mx_next = row_max(nxt, st.N - (j + 1) * kBlockN);
+    }
+    finish_tile(st, cur, buf);
+    return mx_next;
+}
+
+// ---------------------------------------------------------------- softmax warpgroup
+// tile: query tile of this warpgroup; par: which key tiles it takes (j = par, par + kSplit, ...)
+template <int DH>
+__device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, int tile, int par, uint8_t *sQ_gen, uint32_t tmem,
+                                             int m_base, int h, int b, int n_tiles, volatile int *abort_flag, float2 *xchg)
 {
     using C = Cfg<DH>;
+    constexpr int kSplit = C::kSplit;
     const int wtid = threadIdx.x & 127, lane = wtid & 31;
     const int warp = __shfl_sync(0xffffffffu, wtid >> 5, 0);       // warp-uniform
-    // gather this tile's Q rows (swizzled, K-major)
+    // gather this tile's Q rows (swizzled, K-major); the warpgroups of a tile share the rows
     constexpr int kVecPerRow = DH / 8;                 // 16-byte vectors per row
     constexpr int kRowsPerIter = 32 / kVecPerRow;
     {
         const int sub = lane / kVecPerRow, c = lane % kVecPerRow;
 #pragma unroll 4
-        for (int r0 = warp * kRowsPerIter; r0 < kBlockM; r0 += 4 * kRowsPerIter) {
+        for (int r0 = (par * 4 + warp) * kRowsPerIter; r0 < kBlockM; r0 += 4 * kSplit * kRowsPerIter) {
             const int r = r0 + sub;
             const int m = m_base + r;
             uint4 val = make_uint4(0, 0, 0, 0);
@@ -130,97 +281,77 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     mbar_arrive(bar.q + 8 * tile);
 
     const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);
-    const uint32_t t_s0 = t_row + tile * 128;
-    const uint32_t t_o = t_row + kColO + tile * 128;
-    const uint32_t bar_s = bar.s + 16 * tile, bar_p = bar.p + 16 * tile, bar_o = bar.o + 8 * tile;
+    SoftmaxState st;
+    st.sl2 = p.scale_log2;
+    st.m_ref = -INFINITY;
+    st.l_sum = 0.f;
+    st.t_s0 = t_row + tile * 128;
+    st.t_o = t_row + kColO + (tile * kSplit + par) * C::kOStride;
+    st.bar_s = bar.s + 16 * tile; st.bar_p = bar.p + 16 * tile; st.bar_o = bar.o + 16 * tile + 8 * par;
+    st.N = p.N; st.n_tiles = n_tiles; st.abort_flag = abort_flag; st.err_word = p.err_word;
+
     const int m = m_base + wtid;
     int tok = -1;
     if (m < p.M) {
         tok = p.q_idx ? __ldg(p.q_idx + (size_t)b * p.M + m) : m;
-        if ((unsigned)tok >= (unsigned)p.N) { atomicExch(p.err_word, kErrBadIndex); tok = -1; }
+        if ((unsigned)tok >= (unsigned)p.N) { if (par == 0) atomicExch(p.err_word, kErrBadIndex); tok = -1; }
     }
-    const float sl2 = p.scale_log2;
-    float m_ref = -INFINITY, l_sum = 0.f;
 
-    for (int j = 0; j < n_tiles; ++j) {
-        const int buf = j & 1;
-        const uint32_t t_s = t_s0 + buf * kBlockN;
-        wait_bar(bar_s + 8 * buf, (j >> 1) & 1, abort_flag, p.err_word);
+    int my_tiles;                                      // key tiles this warpgroup has processed
+    if constexpr (kSplit == 1) {
+        float sa[kBlockN], sb[kBlockN];
+        wait_bar(st.bar_s, 0, abort_flag, p.err_word);
         tc_fence_after();
-        float s[kBlockN];
-        {
-            uint32_t t0[32], t1[32];
-            tmem_ld32(t_s, t0);
-            tmem_ld32(t_s + 32, t1);
-            tc_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                s[i] = __uint_as_float(t0[i]);
-                s[32 + i] = __uint_as_float(t1[i]);
-            }
+        load_s(st.t_s0, sa);
+        wait_s_regs(sa);
+        float mx = row_max(sa, p.N);
+        for (int j = 0; j < n_tiles; j += 2) {
+            mx = softmax_step_prefetch<DH>(st, sa, sb, j, mx);
+            if (j + 1 < n_tiles) mx = softmax_step_prefetch<DH>(st, sb, sa, j + 1, mx);
         }
-        const int valid = p.N - j * kBlockN;           // keys of this tile that exist
-        if (valid < kBlockN) {
+        my_tiles = n_tiles;
+    } else {
+        my_tiles = 0;
+        for (int j = par; j < n_tiles; j += kSplit, ++my_tiles) {
+            float s[kBlockN];
+            wait_bar(st.bar_s + 8 * par, (j >> 1) & 1, abort_flag, p.err_word);
+            tc_fence_after();
+            load_s(st.t_s0 + par * kBlockN, s);
+            wait_s_regs(s);
+            const float mx = row_max(s, p.N - j * kBlockN);
+            maybe_rescale<DH>(st, mx, my_tiles == 0, (my_tiles - 1) & 1);
+            const float neg = -st.m_ref * st.sl2;
 #pragma unroll
-            for (int i = 0; i < kBlockN; ++i) if (i >= valid) s[i] = -INFINITY;
+            for (int i = 0; i < kBlockN; ++i) s[i] = ex2(fmaf(s[i], st.sl2, neg));
+            finish_tile(st, s, par);
         }
-        // row maximum: independent partial maxima keep the dependency chains short
-        float mx4[4] = {s[0], s[1], s[2], s[3]};
-#pragma unroll
-        for (int i = 4; i < kBlockN; i += 4) {
-            mx4[0] = fmaxf(mx4[0], s[i]); mx4[1] = fmaxf(mx4[1], s[i + 1]);
-            mx4[2] = fmaxf(mx4[2], s[i + 2]); mx4[3] = fmaxf(mx4[3], s[i + 3]);
-        }
-        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-
-        if (j == 0) {
-            m_ref = mx;
-        } else {
-            const bool need = (mx - m_ref) * sl2 > kRescaleThreshold;
-            if (__any_sync(0xffffffffu, need)) {
-                float alpha = 1.0f;
-                if (need) { alpha = ex2((m_ref - mx) * sl2); m_ref = mx; l_sum *= alpha; }
-                wait_bar(bar_o, (j - 1) & 1, abort_flag, p.err_word);     // P V of the previous key tile has landed
-                tc_fence_after();
-#pragma unroll
-                for (int cc = 0; cc < DH / 32; ++cc) {
-                    uint32_t o[32];
-                    tmem_ld32(t_o + cc * 32, o);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                    tmem_st32(t_o + cc * 32, o);
-                }
-                tc_wait_st();
-            }
-        }
-        const float neg = -m_ref * sl2;
-        float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int i = 0; i < kBlockN; i += 4) {
-#pragma unroll
-            for (int u = 0; u < 4; ++u) { s[i + u] = ex2(fmaf(s[i + u], sl2, neg)); sum4[u] += s[i + u]; }
-        }
-        l_sum += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-        // P as bf16 pairs over the first 32 columns of this S buffer (element 2c in the low half)
-        {
-            uint32_t pk[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                __nv_bfloat162 v2 = __floats2bfloat162_rn(s[2 * i], s[2 * i + 1]);
-                pk[i] = *reinterpret_cast<uint32_t *>(&v2);
-            }
-            tmem_st32(t_s, pk);
-        }
-        tc_wait_st();
-        tc_fence_before();
-        mbar_arrive(bar_p + 8 * buf);
     }
 
-    // epilogue: normalise and scatter
-    wait_bar(bar_o, (n_tiles - 1) & 1, abort_flag, p.err_word);
+    // ------------------------------------------------ epilogue: (merge,) normalise and scatter
+    if (my_tiles > 0) wait_bar(st.bar_o, (my_tiles - 1) & 1, abort_flag, p.err_word);
     tc_fence_after();
+    float w_own = 1.0f, w_other = 0.f, l_sum = st.l_sum, m_ref = st.m_ref;
+    uint32_t t_other = 0;
+    if constexpr (kSplit == 2) {
+        // the odd-tile warpgroup hands its maximum and row sum to the even-tile one, which merges
+        if (par == 1) xchg[wtid] = make_float2(st.m_ref, my_tiles > 0 ? st.l_sum : 0.f);
+        tc_fence_before();
+        if (tile == 0) asm volatile("bar.sync 1, 256;" ::: "memory");
+        else asm volatile("bar.sync 2, 256;" ::: "memory");
+        if (par == 1) return;
+        tc_fence_after();
+        const float2 other = xchg[wtid];
+        if (other.y > 0.f) {
+            m_ref = fmaxf(st.m_ref, other.x);
+            w_own = ex2((st.m_ref - m_ref) * st.sl2);
+            w_other = ex2((other.x - m_ref) * st.sl2);
+            l_sum = st.l_sum * w_own + other.y * w_other;
+            t_other = t_row + kColO + (tile * kSplit + 1) * C::kOStride;
+        }
+    }
     const float inv_l = 1.0f / l_sum;
+    w_own *= inv_l;
+    w_other *= inv_l;
     __nv_bfloat16 *dst = nullptr;
     if (tok >= 0 && !*abort_flag) {
         const size_t orow = p.compact ? ((size_t)b * p.M + m) : ((size_t)b * p.N + tok);
@@ -230,19 +361,28 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
             p.lse_out[li] = m_ref * p.scale + logf(l_sum);
         }
     }
+    const bool merge = __any_sync(0xffffffffu, w_other != 0.f);     // warp-uniform: the partner has tiles or not
 #pragma unroll
     for (int cc = 0; cc < DH / 32; ++cc) {
         uint32_t o[32];
-        tmem_ld32(t_o + cc * 32, o);
+        tmem_ld32(st.t_o + cc * 32, o);
         tc_wait_ld();
+        float f[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(o[i]) * w_own;
+        if (kSplit == 2 && merge) {
+            tmem_ld32(t_other + cc * 32, o);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) f[i] = fmaf(__uint_as_float(o[i]), w_other, f[i]);
+        }
         if (dst) {
 #pragma unroll
             for (int v = 0; v < 4; ++v) {
                 uint32_t w[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(o[v * 8 + 2 * i]) * inv_l,
-                                                              __uint_as_float(o[v * 8 + 2 * i + 1]) * inv_l);
+                    __nv_bfloat162 v2 = __floats2bfloat162_rn(f[v * 8 + 2 * i], f[v * 8 + 2 * i + 1]);
                     w[i] = *reinterpret_cast<uint32_t *>(&v2);
                 }
                 *reinterpret_cast<uint4 *>(dst + cc * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -252,13 +392,15 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
 }
 
 template <int DH>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(Cfg<DH>::kThreads, 1)
 sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v, const Params p)
 {
     using C = Cfg<DH>;
+    constexpr int kSplit = C::kSplit;
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    __shared__ float2 xchg[kTilesM][kBlockM];
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -267,29 +409,32 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     const uint32_t sV = sK + C::kStagesK * C::kTileBytes;
     const uint32_t bars = sV + C::kStagesV * C::kTileBytes;
     Bars bar;
-    bar.q = bars; bar.o = bars + 16; bar.s = bars + 32; bar.p = bars + 64;
-    bar.kf = bars + 96;
+    bar.q = bars; bar.s = bars + 16; bar.p = bars + 48; bar.o = bars + 80;
+    bar.kf = bars + 112;
     bar.ke = bar.kf + 8 * C::kStagesK;
     bar.vf = bar.ke + 8 * C::kStagesK;
     bar.ve = bar.vf + 8 * C::kStagesV;
-    static_assert(96 + 16 * (C::kStagesK + C::kStagesV) <= C::kBarBytes, "barrier area too small");
+    static_assert(112 + 16 * (C::kStagesK + C::kStagesV) <= C::kBarBytes, "barrier area too small");
 
     const int tid = threadIdx.x;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);        // warp-uniform
     const int m0 = blockIdx.x * (kTilesM * kBlockM), h = blockIdx.y, b = blockIdx.z;
     const int n_tiles = (p.N + kBlockN - 1) / kBlockN;
+    constexpr int kProducerWarp = C::kSoftmaxWarps, kIssuerWarp = C::kSoftmaxWarps + 1;
 
     if (tid == 0) {
         abort_flag = 0;
         for (int t = 0; t < kTilesM; ++t) {
-            mbar_init(bar.q + 8 * t, 128); mbar_init(bar.o + 8 * t, 1);
-            for (int u = 0; u < 2; ++u) { mbar_init(bar.s + 16 * t + 8 * u, 1); mbar_init(bar.p + 16 * t + 8 * u, 128); }
+            mbar_init(bar.q + 8 * t, 128 * kSplit);
+            for (int u = 0; u < 2; ++u) {
+                mbar_init(bar.s + 16 * t + 8 * u, 1); mbar_init(bar.p + 16 * t + 8 * u, 128); mbar_init(bar.o + 16 * t + 8 * u, 1);
+            }
         }
         for (int s = 0; s < C::kStagesK; ++s) { mbar_init(bar.kf + 8 * s, 1); mbar_init(bar.ke + 8 * s, 1); }
         for (int s = 0; s < C::kStagesV; ++s) { mbar_init(bar.vf + 8 * s, 1); mbar_init(bar.ve + 8 * s, 1); }
         fence_barrier_init();
     }
-    if (warp == 9) {
+    if (warp == kIssuerWarp) {
         tmem_alloc(smem_u32(&tmem_slot), kTmemCols);
         tmem_relinquish();
     }
@@ -298,10 +443,14 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
 
-    if (warp < 8) {
-        const int tile = warp >> 2;
-        softmax_role<DH>(p, bar, tile, smem_gen + tile * C::kQTileBytes, tmem, m0 + tile * kBlockM, h, b, n_tiles, &abort_flag);
-    } else if (warp == 8) {
+    if (warp < C::kSoftmaxWarps) {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(C::kRegsSoftmax));
+        const int wg = warp >> 2;
+        const int tile = wg / kSplit, par = wg % kSplit;
+        softmax_role<DH>(p, bar, tile, par, smem_gen + tile * C::kQTileBytes, tmem, m0 + tile * kBlockM, h, b, n_tiles,
+                         &abort_flag, xchg[tile]);
+    } else if (warp == kProducerWarp) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
         // ------------------------------------------------ TMA producer (warp-uniform, one elected lane issues)
         if (elect_one()) { prefetch_tensormap(&tmap_k); prefetch_tensormap(&tmap_v); }
         auto load_k = [&](int j) {
@@ -326,10 +475,11 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             }
             __syncwarp();
         };
-        // K runs one tile ahead of V: K_{j+1} is needed before V_j
+        // K runs two tiles ahead of V: K_{j+2} is consumed right after V_j
         load_k(0);
+        if (n_tiles > 1) load_k(1);
         for (int j = 0; j < n_tiles; ++j) {
-            if (j + 1 < n_tiles) load_k(j + 1);
+            if (j + 2 < n_tiles) load_k(j + 2);
             load_v(j);
         }
         // every copy issued above must have landed before the CTA's shared memory is released
@@ -337,40 +487,43 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             wait_bar(bar.kf + 8 * (j % C::kStagesK), (j / C::kStagesK) & 1, &abort_flag, p.err_word);
         for (int j = (n_tiles > C::kStagesV ? n_tiles - C::kStagesV : 0); j < n_tiles; ++j)
             wait_bar(bar.vf + 8 * (j % C::kStagesV), (j / C::kStagesV) & 1, &abort_flag, p.err_word);
-    } else {
+    } else if (warp == kIssuerWarp) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
         // ------------------------------------------------ MMA issuer (warp-uniform, one elected lane issues)
         constexpr uint32_t idesc_qk = idesc_bf16(kBlockM, kBlockN, false);
         constexpr uint32_t idesc_pv = idesc_bf16(kBlockM, DH, true);
-        auto issue_qk = [&](int j) {                  // S[t][j&1] = Q_t K_j^T for both query tiles
+        auto issue_qk = [&](int t, int j, uint32_t kbase) {        // S[t][j&1] = Q_t K_j^T  (one elected lane)
+#pragma unroll
+            for (int ks = 0; ks < DH / 16; ++ks)
+                mma_ss(tmem + t * 128 + (j & 1) * kBlockN,
+                       smem_desc(sQ + t * C::kQTileBytes + (ks >> 2) * C::kQChunkBytes + (ks & 3) * 32, 16, 1024, kSwizzle128B),
+                       smem_desc(kbase + (ks >> 2) * C::kChunkBytes + (ks & 3) * 32, 16, 1024, kSwizzle128B),
+                       idesc_qk, ks > 0);
+            tc_commit(bar.s + 16 * t + 8 * (j & 1));
+        };
+        // prologue: S of key tiles 0 and 1 for both query tiles
+        wait_bar(bar.q, 0, &abort_flag, p.err_word);
+        wait_bar(bar.q + 8, 0, &abort_flag, p.err_word);
+        for (int j = 0; j < 2 && j < n_tiles; ++j) {
             const int st = j % C::kStagesK;
-            const uint32_t kbase = sK + st * C::kTileBytes;
-            const uint32_t sbuf = (j & 1) * kBlockN;
             wait_bar(bar.kf + 8 * st, (j / C::kStagesK) & 1, &abort_flag, p.err_word);
             tc_fence_after();
             if (elect_one()) {
-#pragma unroll
-                for (int t = 0; t < kTilesM; ++t) {
-#pragma unroll
-                    for (int ks = 0; ks < DH / 16; ++ks)
-                        mma_ss(tmem + t * 128 + sbuf,
-                               smem_desc(sQ + t * C::kQTileBytes + (ks >> 2) * C::kQChunkBytes + (ks & 3) * 32, 16, 1024, kSwizzle128B),
-                               smem_desc(kbase + (ks >> 2) * C::kChunkBytes + (ks & 3) * 32, 16, 1024, kSwizzle128B),
-                               idesc_qk, ks > 0);
-                    tc_commit(bar.s + 16 * t + 8 * (j & 1));
-                }
+                issue_qk(0, j, sK + st * C::kTileBytes);
+                issue_qk(1, j, sK + st * C::kTileBytes);
                 tc_commit(bar.ke + 8 * st);
             }
             __syncwarp();
-        };
-        wait_bar(bar.q, 0, &abort_flag, p.err_word);
-        wait_bar(bar.q + 8, 0, &abort_flag, p.err_word);
-        issue_qk(0);
+        }
         for (int j = 0; j < n_tiles; ++j) {
-            if (j + 1 < n_tiles) issue_qk(j + 1);     // its S buffer held P of tile j-1, already consumed in order
             const int sv = j % C::kStagesV;
             const uint32_t vbase = sV + sv * C::kTileBytes;
             const uint32_t sbuf = (j & 1) * kBlockN;
+            const uint32_t acc = (kSplit == 2) ? (uint32_t)(j & 1) : 0u;      // which O accumulator of the tile
+            const bool more = j + 2 < n_tiles;
+            const int sk = (j + 2) % C::kStagesK;
             wait_bar(bar.vf + 8 * sv, (j / C::kStagesV) & 1, &abort_flag, p.err_word);
+            if (more) wait_bar(bar.kf + 8 * sk, ((j + 2) / C::kStagesK) & 1, &abort_flag, p.err_word);
 #pragma unroll
             for (int t = 0; t < kTilesM; ++t) {
                 wait_bar(bar.p + 16 * t + 8 * (j & 1), (j >> 1) & 1, &abort_flag, p.err_word);
@@ -378,20 +531,27 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                 if (elect_one()) {
 #pragma unroll
                     for (int ks = 0; ks < kBlockN / 16; ++ks)
-                        mma_ts(tmem + kColO + t * 128, tmem + t * 128 + sbuf + ks * 8,
+                        mma_ts(tmem + kColO + (t * kSplit + acc) * C::kOStride, tmem + t * 128 + sbuf + ks * 8,
                                smem_desc(vbase + ks * 2048, C::kChunkBytes, 1024, kSwizzle128B),
-                               idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
-                    tc_commit(bar.o + 8 * t);
+                               idesc_pv, (j >= kSplit || ks > 0) ? 1u : 0u);
+                    tc_commit(bar.o + 16 * t + 8 * acc);
                     if (t == kTilesM - 1) tc_commit(bar.ve + 8 * sv);
+                    // the S buffer just consumed as P is free again (in-order pipe): refill it with key tile j+2
+                    if (more) {
+                        issue_qk(t, j + 2, sK + sk * C::kTileBytes);
+                        if (t == kTilesM - 1) tc_commit(bar.ke + 8 * sk);
+                    }
                 }
                 __syncwarp();
             }
         }
+    } else {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
     }
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 9) tmem_dealloc(tmem, kTmemCols);
+    if (warp == kIssuerWarp) tmem_dealloc(tmem, kTmemCols);
 }
 
 // ------------------------------------------------------------------ host side
@@ -455,7 +615,7 @@ int32_t launch_dh(const AttnArgs &a, cudaStream_t stream)
     p.compact = (a.flags & ASTRAEA_ATTN_COMPACT_OUT) ? 1 : 0;
     p.err_word = a.err_word;
     dim3 grid((a.M + kTilesM * kBlockM - 1) / (kTilesM * kBlockM), a.H, a.B);
-    sparse_attn_kernel<DH><<<grid, kThreads, C::kSmemBytes, stream>>>(mk, mv, p);
+    sparse_attn_kernel<DH><<<grid, C::kThreads, C::kSmemBytes, stream>>>(mk, mv, p);
     return check_launch("astraea_sparse_attn");
 }
 
