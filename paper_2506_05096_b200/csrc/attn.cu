@@ -3,32 +3,31 @@
 // Section 3.2 "Sparse Attention").
 //
 // One CTA per (256 selected queries, head, batch): two 128-row query tiles that share every
-// K/V tile of 64 keys.  Warp roles:
-//   softmax warpgroups (one thread per query row): gather the tile's Q rows into 128B-swizzled
-//              shared memory, then per key tile read S from TMEM, online softmax in the log2 domain
-//              with lazy rescaling of O, write P (bf16) back to TMEM over S, and at the end
-//              normalise O and scatter it to the rows q_idx names;
-//   one warp   TMA producer: K and V tiles into multi-stage swizzled buffers;
-//   one warp   tcgen05.mma issuer: S = Q K^T (SS, K-major operands), O += P V (P from TMEM,
-//              V as an MN-major shared-memory operand); owns the TMEM allocation.
-// S is double-buffered per query tile and refilled with key tile j+2 as soon as P of tile j has
-// been consumed.
+// K/V tile of 64 keys.  Warp roles (384 threads):
+//   warps 0-3 / 4-7  softmax of query tile 0 / 1 (one thread per query row): gather the tile's Q rows
+//              into 128B-swizzled shared memory, then per key tile read S from TMEM, exponentiate
+//              in the log2 domain against a running reference maximum, write P (bf16) back to TMEM
+//              over S, and at the end normalise O and scatter it to the rows q_idx names;
+//   warp 8     TMA producer: K and V tiles into multi-stage swizzled buffers;
+//   warp 9     tcgen05.mma issuer: S = Q K^T (SS, K-major operands), O += P V (P from TMEM,
+//              V as an MN-major shared-memory operand); owns the TMEM allocation;
+//   warps 10-11 only donate registers (setmaxnreg moves them to the softmax warps).
+// S has kSBufs buffers per query tile; a buffer is refilled with key tile j+kSBufs as soon as P of
+// tile j has been consumed, so S of the next tiles is in TMEM while the softmax of tile j runs.
 //
-// The exponentials (XU pipe, 16 per clock per SM) bound the softmax.  One warp alone cannot keep
-// its XU sub-pipe busy, and at head_dim 64 the MMAs of a key tile are much shorter than its
-// exponentials.  So at head_dim 64 every query tile has TWO softmax warpgroups: even key tiles go
-// to one, odd ones to the other, each with its own running maximum, row sum and O accumulator in
-// TMEM (a split over keys inside the CTA), merged once in the epilogue.  That gives four softmax
-// warps per SM sub-partition.  At head_dim 128 the MMAs are as long as the exponentials and TMEM
-// has no room for four accumulators: one warpgroup per query tile, which prefetches S of the next
-// key tile and reduces its maximum while the current tile's exponentials execute.
+// The softmax is bound by the exponentials (XU pipe, 16 per clock per SM) and by the latencies of
+// its own chain, so the common path of a key tile is kept to: load S, one FFMA + ex2 per element,
+// sum, pack, store.  The reference maximum is the exact row maximum of the first key tile and is
+// then only checked through the tile's sum of exponentials: while that sum stays below 2^16 the
+// tile is accepted as it is (the probabilities are relative to a stale maximum, which the final
+// normalisation cancels; fp32 has the range).  Otherwise the exact maximum is taken and the row
+// sum and the O accumulator are rescaled before the tile is redone.
 //
-// TMEM columns: S/P of (tile t, buffer u) at (2t+u)*64; O accumulators from column 256.
+// TMEM columns: S/P of (tile t, buffer u) at (t*kSBufs+u)*64; O of tile t behind them.
 // The producer and issuer warps run warp-uniform code and elect one lane per instruction, so
 // that descriptors and addresses stay in uniform registers (a lone diverged thread issues
-// tcgen05.mma several times slower).  setmaxnreg moves registers from the last warpgroup to the
-// softmax warpgroups.  Every mbarrier wait is bounded; on a timeout the CTA raises the error
-// word, the remaining waits return at once, and the CTA runs out.
+// tcgen05.mma several times slower).  Every mbarrier wait is bounded; on a timeout the CTA raises
+// the error word, the remaining waits return at once, and the CTA runs out.
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -40,22 +39,21 @@ using namespace ptx;
 constexpr int kBlockM = 128;                     // rows of one query tile
 constexpr int kTilesM = 2;                       // query tiles per CTA
 constexpr int kBlockN = 64;                      // keys per K/V tile
+constexpr int kThreads = 384;
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColO = 256;
-constexpr float kRescaleThreshold = 8.0f;        // log2 units: P stays below 2^8
+constexpr float kTileSumLimit = 65536.0f;        // a tile's sum of exponentials above this forces an exact maximum
 constexpr uint64_t kWaitLimitNs = 1000000000ull; // bounded waits: one second
 
 template <int DH> struct Cfg {
-    static constexpr int kSplit = 1;              // softmax warpgroups per query tile
-    static constexpr int kSoftmaxWarps = 4 * kTilesM * kSplit;
-    static constexpr int kThreads = (kSoftmaxWarps + 4) * 32;     // + producer, issuer, two register donors
-    // setmaxnreg only redistributes what the CTA got at launch (kRegsLaunch per thread): an increase
-    // that the decreases of the last warpgroup cannot cover would block forever
+    static constexpr int kSBufs = (DH == 128) ? 2 : 3;            // S buffers per query tile
+    static constexpr uint32_t kColO = kTilesM * kSBufs * kBlockN; // first O column
+    static constexpr uint32_t kOStride = (DH == 128) ? 128 : 64;
+    static_assert(kColO + kTilesM * kOStride <= kTmemCols && DH <= (int)kOStride, "TMEM budget");
+    // setmaxnreg only redistributes what the CTA got at launch: an increase that the decreases of
+    // the last warpgroup cannot cover would block forever
     static constexpr int kRegsLaunch = (65536 / kThreads) / 8 * 8;
-    static constexpr int kRegsSoftmax = (kSplit == 2) ? 112 : 232;
-    static constexpr int kRegsOther = (kSplit == 2) ? 32 : 40;
-    static_assert(kRegsSoftmax * kSoftmaxWarps * 32 + kRegsOther * 128 <= kRegsLaunch * kThreads, "setmaxnreg budget");
-    static constexpr uint32_t kOStride = 128 / kSplit;            // TMEM columns between O accumulators
+    static constexpr int kRegsSoftmax = 232, kRegsOther = 40;
+    static_assert(kRegsSoftmax * 256 + kRegsOther * 128 <= kRegsLaunch * kThreads, "setmaxnreg budget");
     static constexpr int kChunks = DH / 64;                       // 64-column (128-byte) swizzle chunks
     static constexpr int kQChunkBytes = kBlockM * 128;            // 128 query rows x 128 bytes
     static constexpr int kQTileBytes = kChunks * kQChunkBytes;
@@ -63,9 +61,9 @@ template <int DH> struct Cfg {
     static constexpr int kTileBytes = kChunks * kChunkBytes;      // one K or V tile
     static constexpr int kStagesK = (DH == 128) ? 5 : 6;
     static constexpr int kStagesV = (DH == 128) ? 5 : 6;
+    static_assert(kStagesK > kSBufs, "K runs kSBufs tiles ahead");
     static constexpr int kBarBytes = 512;
     static constexpr int kSmemBytes = kQTileBytes * kTilesM + kTileBytes * (kStagesK + kStagesV) + kBarBytes + 1024;
-    static_assert(kColO + kTilesM * kSplit * kOStride <= kTmemCols && DH <= (int)kOStride, "TMEM budget");
 };
 
 struct Params {
@@ -120,11 +118,11 @@ __device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, volatile
 
 struct Bars {
     uint32_t q;                     // [kTilesM]
-    uint32_t s, p, o;               // [kTilesM][2]
+    uint32_t s, p, o;               // [kTilesM][4]: one per S buffer (o: P V of the tile in that buffer has landed)
     uint32_t kf, ke, vf, ve;        // [stages]
 };
 
-struct SoftmaxState {
+template <int DH> struct SoftmaxState {
     float sl2, m_ref, l_sum;
     uint32_t t_s0, t_o, bar_s, bar_p, bar_o;
     int N, n_tiles;
@@ -153,12 +151,15 @@ __device__ __forceinline__ void wait_s_regs(float (&s)[kBlockN]) {
         :: "memory");
 }
 
-// maximum of the row's logits in one key tile; keys beyond `valid` (zero-filled tail) become -inf
-__device__ __forceinline__ float row_max(float (&s)[kBlockN], int valid) {
+// keys beyond `valid` (zero-filled tail of the last key tile) get logit -inf
+__device__ __forceinline__ void mask_tail(float (&s)[kBlockN], int valid) {
     if (valid < kBlockN) {
 #pragma unroll
         for (int i = 0; i < kBlockN; ++i) if (i >= valid) s[i] = -INFINITY;
     }
+}
+
+__device__ __forceinline__ float row_max(const float (&s)[kBlockN]) {
     float mx4[4] = {max3(s[0], s[1], s[2]), max3(s[3], s[4], s[5]), max3(s[6], s[7], s[8]), max3(s[9], s[10], s[11])};
 #pragma unroll
     for (int i = 12; i + 7 < kBlockN; i += 8) {
@@ -171,98 +172,102 @@ __device__ __forceinline__ float row_max(float (&s)[kBlockN], int valid) {
     return fmaxf(max3(mx4[0], mx4[1], mx4[2]), mx4[3]);
 }
 
-// Moves the running maximum to mx when it has grown by more than the threshold, rescaling the row
-// sum and (once the previous P V of this accumulator has landed: o_parity) the O accumulator.
-template <int DH>
-__device__ __forceinline__ void maybe_rescale(SoftmaxState &st, float mx, bool first, uint32_t o_parity) {
-    if (first) { st.m_ref = mx; return; }
-    const bool need = (mx - st.m_ref) * st.sl2 > kRescaleThreshold;
-    if (__any_sync(0xffffffffu, need)) {
-        float alpha = 1.0f;
-        if (need) { alpha = ex2((st.m_ref - mx) * st.sl2); st.m_ref = mx; st.l_sum *= alpha; }
-        wait_bar(st.bar_o, o_parity, st.abort_flag, st.err_word);
-        tc_fence_after();
+__device__ __forceinline__ float row_sum(const float (&s)[kBlockN]) {
+    float a[8];
 #pragma unroll
-        for (int cc = 0; cc < DH / 32; ++cc) {
-            uint32_t o[32];
-            tmem_ld32(st.t_o + cc * 32, o);
-            tc_wait_ld();
+    for (int u = 0; u < 8; ++u) a[u] = s[u];
 #pragma unroll
-            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-            tmem_st32(st.t_o + cc * 32, o);
-        }
-        tc_wait_st();
+    for (int i = 8; i < kBlockN; i += 8) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) a[u] += s[i + u];
     }
+    return ((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7]));
 }
 
-// exponentials of one key tile in place, their sum added to the row sum, P (bf16 pairs, element 2c
-// in the low half) stored over the first 32 columns of the S buffer, then the P barrier
-__device__ __forceinline__ void finish_tile(SoftmaxState &st, float (&cur)[kBlockN], int buf) {
-    float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+// P has been stored: make it visible to the issuer warp
+__device__ __forceinline__ void publish_p(uint32_t bar) {
+    tc_wait_st();
+    tc_fence_before();
+    mbar_arrive(bar);
+}
+
+// One key tile of the online softmax.
+template <int DH>
+__device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j)
+{
+    constexpr int kSBufs = Cfg<DH>::kSBufs;
+    const int buf = j % kSBufs;
+    const uint32_t t_s = st.t_s0 + buf * kBlockN;
+    const float sl2 = st.sl2;
+    float cur[kBlockN];
+    // S of this tile has been in TMEM for a while (kSBufs buffers); the load is waited for at once:
+    // registers of a tcgen05.ld in flight must not be touched, and the compiler cannot know that
+    wait_bar(st.bar_s + 8 * buf, (j / kSBufs) & 1, st.abort_flag, st.err_word);
+    tc_fence_after();
+    load_s(t_s, cur);
+    wait_s_regs(cur);
+    mask_tail(cur, st.N - j * kBlockN);
+    if (j == 0) st.m_ref = row_max(cur);          // the reference starts as the exact maximum of the first key tile
+    float neg = -st.m_ref * sl2;
+    float e[kBlockN];
 #pragma unroll
-    for (int i = 0; i < kBlockN; i += 4) {
+    for (int i = 0; i < kBlockN; ++i) e[i] = ex2(fmaf(cur[i], sl2, neg));
+    float tile_sum = row_sum(e);
+    if (__any_sync(0xffffffffu, !(tile_sum <= kTileSumLimit))) {
+        // rare: the reference maximum is too low for this tile: take the exact maximum, rescale what
+        // has been accumulated, and redo the tile
+        const float mx = row_max(cur);
+        float alpha = 1.0f;
+        if (mx > st.m_ref) { alpha = ex2((st.m_ref - mx) * sl2); st.m_ref = mx; st.l_sum *= alpha; }
+        if (j > 0) {
+            // P V of the previous key tile has landed.  The o barrier of a buffer cannot be a whole phase
+            // behind: S of this tile was seen, so every MMA issued before its Q K^T is complete, and
+            // that includes the P V that last used the previous tile's buffer.
+            wait_bar(st.bar_o + 8 * ((j - 1) % kSBufs), ((j - 1) / kSBufs) & 1, st.abort_flag, st.err_word);
+            tc_fence_after();
 #pragma unroll
-        for (int u = 0; u < 4; ++u) sum4[u] += cur[i + u];
+            for (int cc = 0; cc < DH / 32; ++cc) {
+                uint32_t o[32];
+                tmem_ld32(st.t_o + cc * 32, o);
+                tc_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                tmem_st32(st.t_o + cc * 32, o);
+            }
+            tc_wait_st();
+        }
+        neg = -st.m_ref * sl2;
+#pragma unroll
+        for (int i = 0; i < kBlockN; ++i) e[i] = ex2(fmaf(cur[i], sl2, neg));
+        tile_sum = row_sum(e);
     }
-    st.l_sum += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+    st.l_sum += tile_sum;
+    // P as bf16 pairs (element 2c in the low half) over the first 32 columns of this S buffer
     uint32_t pk[32];
 #pragma unroll
     for (int i = 0; i < 32; ++i) {
-        __nv_bfloat162 v2 = __floats2bfloat162_rn(cur[2 * i], cur[2 * i + 1]);
+        __nv_bfloat162 v2 = __floats2bfloat162_rn(e[2 * i], e[2 * i + 1]);
         pk[i] = *reinterpret_cast<uint32_t *>(&v2);
     }
-    tmem_st32(st.t_s0 + buf * kBlockN, pk);
-    tc_wait_st();
-    tc_fence_before();
-    mbar_arrive(st.bar_p + 8 * buf);
+    tmem_st32(t_s, pk);
+    publish_p(st.bar_p + 8 * buf);
 }
 
-// One key tile of the online softmax, one warpgroup per query tile.  `cur` holds S of tile j (row
-// maximum mx); S of tile j+1 is fetched into `nxt` and reduced while the exponentials of tile j
-// execute.  Returns the row maximum of tile j+1.
+// ---------------------------------------------------------------- softmax warpgroup (one query tile)
 template <int DH>
-__device__ __forceinline__ float softmax_step_prefetch(SoftmaxState &st, float (&cur)[kBlockN], float (&nxt)[kBlockN], int j, float mx)
-{
-    const int buf = j & 1;
-    const float sl2 = st.sl2;
-    maybe_rescale<DH>(st, mx, j == 0, (j - 1) & 1);
-    const bool more = j + 1 < st.n_tiles;
-    const float neg = -st.m_ref * sl2;
-#pragma unroll
-    for (int i = 0; i < kBlockN / 2; ++i) cur[i] = ex2(fmaf(cur[i], sl2, neg));
-    if (more) {
-        wait_bar(st.bar_s + 8 * (buf ^ 1), ((j + 1) >> 1) & 1, st.abort_flag, st.err_word);
-        tc_fence_after();
-        load_s(st.t_s0 + (buf ^ 1) * kBlockN, nxt);
-    }
-#pragma unroll
-    for (int i = kBlockN / 2; i < kBlockN; ++i) cur[i] = ex2(fmaf(cur[i], sl2, neg));
-    float mx_next = 0.f;
-    if (more) {
-        wait_s_regs(nxt);
-        mx_next = row_max(nxt, st.N - (j + 1) * kBlockN);
-    }
-    finish_tile(st, cur, buf);
-    return mx_next;
-}
-
-// ---------------------------------------------------------------- softmax warpgroup
-// tile: query tile of this warpgroup; par: which key tiles it takes (j = par, par + kSplit, ...)
-template <int DH>
-__device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, int tile, int par, uint8_t *sQ_gen, uint32_t tmem,
-                                             int m_base, int h, int b, int n_tiles, volatile int *abort_flag, float2 *xchg)
+__device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, int tile, uint8_t *sQ_gen, uint32_t tmem,
+                                             int m_base, int h, int b, int n_tiles, volatile int *abort_flag)
 {
     using C = Cfg<DH>;
-    constexpr int kSplit = C::kSplit;
     const int wtid = threadIdx.x & 127, lane = wtid & 31;
     const int warp = __shfl_sync(0xffffffffu, wtid >> 5, 0);       // warp-uniform
-    // gather this tile's Q rows (swizzled, K-major); the warpgroups of a tile share the rows
+    // gather this tile's Q rows (swizzled, K-major)
     constexpr int kVecPerRow = DH / 8;                 // 16-byte vectors per row
     constexpr int kRowsPerIter = 32 / kVecPerRow;
     {
         const int sub = lane / kVecPerRow, c = lane % kVecPerRow;
 #pragma unroll 4
-        for (int r0 = (par * 4 + warp) * kRowsPerIter; r0 < kBlockM; r0 += 4 * kSplit * kRowsPerIter) {
+        for (int r0 = warp * kRowsPerIter; r0 < kBlockM; r0 += 4 * kRowsPerIter) {
             const int r = r0 + sub;
             const int m = m_base + r;
             uint4 val = make_uint4(0, 0, 0, 0);
@@ -281,108 +286,50 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     mbar_arrive(bar.q + 8 * tile);
 
     const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);
-    SoftmaxState st;
+    SoftmaxState<DH> st;
     st.sl2 = p.scale_log2;
-    st.m_ref = -INFINITY;
     st.l_sum = 0.f;
-    st.t_s0 = t_row + tile * 128;
-    st.t_o = t_row + kColO + (tile * kSplit + par) * C::kOStride;
-    st.bar_s = bar.s + 16 * tile; st.bar_p = bar.p + 16 * tile; st.bar_o = bar.o + 16 * tile + 8 * par;
+    st.t_s0 = t_row + tile * C::kSBufs * kBlockN;
+    st.t_o = t_row + C::kColO + tile * C::kOStride;
+    st.bar_s = bar.s + 32 * tile; st.bar_p = bar.p + 32 * tile; st.bar_o = bar.o + 32 * tile;
     st.N = p.N; st.n_tiles = n_tiles; st.abort_flag = abort_flag; st.err_word = p.err_word;
 
     const int m = m_base + wtid;
     int tok = -1;
     if (m < p.M) {
         tok = p.q_idx ? __ldg(p.q_idx + (size_t)b * p.M + m) : m;
-        if ((unsigned)tok >= (unsigned)p.N) { if (par == 0) atomicExch(p.err_word, kErrBadIndex); tok = -1; }
+        if ((unsigned)tok >= (unsigned)p.N) { atomicExch(p.err_word, kErrBadIndex); tok = -1; }
     }
 
-    int my_tiles;                                      // key tiles this warpgroup has processed
-    if constexpr (kSplit == 1) {
-        float sa[kBlockN], sb[kBlockN];
-        wait_bar(st.bar_s, 0, abort_flag, p.err_word);
-        tc_fence_after();
-        load_s(st.t_s0, sa);
-        wait_s_regs(sa);
-        float mx = row_max(sa, p.N);
-        for (int j = 0; j < n_tiles; j += 2) {
-            mx = softmax_step_prefetch<DH>(st, sa, sb, j, mx);
-            if (j + 1 < n_tiles) mx = softmax_step_prefetch<DH>(st, sb, sa, j + 1, mx);
-        }
-        my_tiles = n_tiles;
-    } else {
-        my_tiles = 0;
-        for (int j = par; j < n_tiles; j += kSplit, ++my_tiles) {
-            float s[kBlockN];
-            wait_bar(st.bar_s + 8 * par, (j >> 1) & 1, abort_flag, p.err_word);
-            tc_fence_after();
-            load_s(st.t_s0 + par * kBlockN, s);
-            wait_s_regs(s);
-            const float mx = row_max(s, p.N - j * kBlockN);
-            maybe_rescale<DH>(st, mx, my_tiles == 0, (my_tiles - 1) & 1);
-            const float neg = -st.m_ref * st.sl2;
-#pragma unroll
-            for (int i = 0; i < kBlockN; ++i) s[i] = ex2(fmaf(s[i], st.sl2, neg));
-            finish_tile(st, s, par);
-        }
-    }
+    st.m_ref = -INFINITY;
+    for (int j = 0; j < n_tiles; ++j) softmax_step<DH>(st, j);
 
-    // ------------------------------------------------ epilogue: (merge,) normalise and scatter
-    if (my_tiles > 0) wait_bar(st.bar_o, (my_tiles - 1) & 1, abort_flag, p.err_word);
+    // ------------------------------------------------ epilogue: normalise and scatter
+    wait_bar(st.bar_o + 8 * ((n_tiles - 1) % C::kSBufs), ((n_tiles - 1) / C::kSBufs) & 1, abort_flag, p.err_word);
     tc_fence_after();
-    float w_own = 1.0f, w_other = 0.f, l_sum = st.l_sum, m_ref = st.m_ref;
-    uint32_t t_other = 0;
-    if constexpr (kSplit == 2) {
-        // the odd-tile warpgroup hands its maximum and row sum to the even-tile one, which merges
-        if (par == 1) xchg[wtid] = make_float2(st.m_ref, my_tiles > 0 ? st.l_sum : 0.f);
-        tc_fence_before();
-        if (tile == 0) asm volatile("bar.sync 1, 256;" ::: "memory");
-        else asm volatile("bar.sync 2, 256;" ::: "memory");
-        if (par == 1) return;
-        tc_fence_after();
-        const float2 other = xchg[wtid];
-        if (other.y > 0.f) {
-            m_ref = fmaxf(st.m_ref, other.x);
-            w_own = ex2((st.m_ref - m_ref) * st.sl2);
-            w_other = ex2((other.x - m_ref) * st.sl2);
-            l_sum = st.l_sum * w_own + other.y * w_other;
-            t_other = t_row + kColO + (tile * kSplit + 1) * C::kOStride;
-        }
-    }
-    const float inv_l = 1.0f / l_sum;
-    w_own *= inv_l;
-    w_other *= inv_l;
+    const float inv_l = 1.0f / st.l_sum;
     __nv_bfloat16 *dst = nullptr;
     if (tok >= 0 && !*abort_flag) {
         const size_t orow = p.compact ? ((size_t)b * p.M + m) : ((size_t)b * p.N + tok);
         dst = p.out + (orow * p.H + h) * DH;
         if (p.lse_out) {
             const size_t li = p.compact ? (((size_t)b * p.H + h) * p.M + m) : (((size_t)b * p.H + h) * p.N + tok);
-            p.lse_out[li] = m_ref * p.scale + logf(l_sum);
+            p.lse_out[li] = st.m_ref * p.scale + logf(st.l_sum);
         }
     }
-    const bool merge = __any_sync(0xffffffffu, w_other != 0.f);     // warp-uniform: the partner has tiles or not
 #pragma unroll
     for (int cc = 0; cc < DH / 32; ++cc) {
         uint32_t o[32];
         tmem_ld32(st.t_o + cc * 32, o);
         tc_wait_ld();
-        float f[32];
-#pragma unroll
-        for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(o[i]) * w_own;
-        if (kSplit == 2 && merge) {
-            tmem_ld32(t_other + cc * 32, o);
-            tc_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) f[i] = fmaf(__uint_as_float(o[i]), w_other, f[i]);
-        }
         if (dst) {
 #pragma unroll
             for (int v = 0; v < 4; ++v) {
                 uint32_t w[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    __nv_bfloat162 v2 = __floats2bfloat162_rn(f[v * 8 + 2 * i], f[v * 8 + 2 * i + 1]);
+                    __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(o[v * 8 + 2 * i]) * inv_l,
+                                                              __uint_as_float(o[v * 8 + 2 * i + 1]) * inv_l);
                     w[i] = *reinterpret_cast<uint32_t *>(&v2);
                 }
                 *reinterpret_cast<uint4 *>(dst + cc * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -392,15 +339,14 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
 }
 
 template <int DH>
-__global__ void __launch_bounds__(Cfg<DH>::kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 1)
 sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v, const Params p)
 {
     using C = Cfg<DH>;
-    constexpr int kSplit = C::kSplit;
+    constexpr int kSBufs = C::kSBufs;
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
-    __shared__ float2 xchg[kTilesM][kBlockM];
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -409,32 +355,31 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     const uint32_t sV = sK + C::kStagesK * C::kTileBytes;
     const uint32_t bars = sV + C::kStagesV * C::kTileBytes;
     Bars bar;
-    bar.q = bars; bar.s = bars + 16; bar.p = bars + 48; bar.o = bars + 80;
-    bar.kf = bars + 112;
+    bar.q = bars; bar.s = bars + 16; bar.p = bars + 80; bar.o = bars + 144;
+    bar.kf = bars + 208;
     bar.ke = bar.kf + 8 * C::kStagesK;
     bar.vf = bar.ke + 8 * C::kStagesK;
     bar.ve = bar.vf + 8 * C::kStagesV;
-    static_assert(112 + 16 * (C::kStagesK + C::kStagesV) <= C::kBarBytes, "barrier area too small");
+    static_assert(208 + 16 * (C::kStagesK + C::kStagesV) <= C::kBarBytes, "barrier area too small");
 
     const int tid = threadIdx.x;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);        // warp-uniform
     const int m0 = blockIdx.x * (kTilesM * kBlockM), h = blockIdx.y, b = blockIdx.z;
     const int n_tiles = (p.N + kBlockN - 1) / kBlockN;
-    constexpr int kProducerWarp = C::kSoftmaxWarps, kIssuerWarp = C::kSoftmaxWarps + 1;
 
     if (tid == 0) {
         abort_flag = 0;
         for (int t = 0; t < kTilesM; ++t) {
-            mbar_init(bar.q + 8 * t, 128 * kSplit);
-            for (int u = 0; u < 2; ++u) {
-                mbar_init(bar.s + 16 * t + 8 * u, 1); mbar_init(bar.p + 16 * t + 8 * u, 128); mbar_init(bar.o + 16 * t + 8 * u, 1);
+            mbar_init(bar.q + 8 * t, 128);
+            for (int u = 0; u < 4; ++u) {
+                mbar_init(bar.s + 32 * t + 8 * u, 1); mbar_init(bar.p + 32 * t + 8 * u, 128); mbar_init(bar.o + 32 * t + 8 * u, 1);
             }
         }
         for (int s = 0; s < C::kStagesK; ++s) { mbar_init(bar.kf + 8 * s, 1); mbar_init(bar.ke + 8 * s, 1); }
         for (int s = 0; s < C::kStagesV; ++s) { mbar_init(bar.vf + 8 * s, 1); mbar_init(bar.ve + 8 * s, 1); }
         fence_barrier_init();
     }
-    if (warp == kIssuerWarp) {
+    if (warp == 9) {
         tmem_alloc(smem_u32(&tmem_slot), kTmemCols);
         tmem_relinquish();
     }
@@ -443,13 +388,11 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
 
-    if (warp < C::kSoftmaxWarps) {
+    if (warp < 8) {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(C::kRegsSoftmax));
-        const int wg = warp >> 2;
-        const int tile = wg / kSplit, par = wg % kSplit;
-        softmax_role<DH>(p, bar, tile, par, smem_gen + tile * C::kQTileBytes, tmem, m0 + tile * kBlockM, h, b, n_tiles,
-                         &abort_flag, xchg[tile]);
-    } else if (warp == kProducerWarp) {
+        const int tile = warp >> 2;
+        softmax_role<DH>(p, bar, tile, smem_gen + tile * C::kQTileBytes, tmem, m0 + tile * kBlockM, h, b, n_tiles, &abort_flag);
+    } else if (warp == 8) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
         // ------------------------------------------------ TMA producer (warp-uniform, one elected lane issues)
         if (elect_one()) { prefetch_tensormap(&tmap_k); prefetch_tensormap(&tmap_v); }
@@ -475,11 +418,10 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             }
             __syncwarp();
         };
-        // K runs two tiles ahead of V: K_{j+2} is consumed right after V_j
-        load_k(0);
-        if (n_tiles > 1) load_k(1);
+        // K runs kSBufs tiles ahead of V: K_{j+kSBufs} is consumed right after V_j
+        for (int j = 0; j < kSBufs && j < n_tiles; ++j) load_k(j);
         for (int j = 0; j < n_tiles; ++j) {
-            if (j + 2 < n_tiles) load_k(j + 2);
+            if (j + kSBufs < n_tiles) load_k(j + kSBufs);
             load_v(j);
         }
         // every copy issued above must have landed before the CTA's shared memory is released
@@ -487,24 +429,25 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             wait_bar(bar.kf + 8 * (j % C::kStagesK), (j / C::kStagesK) & 1, &abort_flag, p.err_word);
         for (int j = (n_tiles > C::kStagesV ? n_tiles - C::kStagesV : 0); j < n_tiles; ++j)
             wait_bar(bar.vf + 8 * (j % C::kStagesV), (j / C::kStagesV) & 1, &abort_flag, p.err_word);
-    } else if (warp == kIssuerWarp) {
+    } else if (warp == 9) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
         // ------------------------------------------------ MMA issuer (warp-uniform, one elected lane issues)
         constexpr uint32_t idesc_qk = idesc_bf16(kBlockM, kBlockN, false);
         constexpr uint32_t idesc_pv = idesc_bf16(kBlockM, DH, true);
-        auto issue_qk = [&](int t, int j, uint32_t kbase) {        // S[t][j&1] = Q_t K_j^T  (one elected lane)
+        auto issue_qk = [&](int t, int j, uint32_t kbase) {        // S[t][j % kSBufs] = Q_t K_j^T  (one elected lane)
+            const int u = j % kSBufs;
 #pragma unroll
             for (int ks = 0; ks < DH / 16; ++ks)
-                mma_ss(tmem + t * 128 + (j & 1) * kBlockN,
+                mma_ss(tmem + (t * kSBufs + u) * kBlockN,
                        smem_desc(sQ + t * C::kQTileBytes + (ks >> 2) * C::kQChunkBytes + (ks & 3) * 32, 16, 1024, kSwizzle128B),
                        smem_desc(kbase + (ks >> 2) * C::kChunkBytes + (ks & 3) * 32, 16, 1024, kSwizzle128B),
                        idesc_qk, ks > 0);
-            tc_commit(bar.s + 16 * t + 8 * (j & 1));
+            tc_commit(bar.s + 32 * t + 8 * u);
         };
-        // prologue: S of key tiles 0 and 1 for both query tiles
+        // prologue: S of the first kSBufs key tiles for both query tiles
         wait_bar(bar.q, 0, &abort_flag, p.err_word);
         wait_bar(bar.q + 8, 0, &abort_flag, p.err_word);
-        for (int j = 0; j < 2 && j < n_tiles; ++j) {
+        for (int j = 0; j < kSBufs && j < n_tiles; ++j) {
             const int st = j % C::kStagesK;
             wait_bar(bar.kf + 8 * st, (j / C::kStagesK) & 1, &abort_flag, p.err_word);
             tc_fence_after();
@@ -518,27 +461,26 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         for (int j = 0; j < n_tiles; ++j) {
             const int sv = j % C::kStagesV;
             const uint32_t vbase = sV + sv * C::kTileBytes;
-            const uint32_t sbuf = (j & 1) * kBlockN;
-            const uint32_t acc = (kSplit == 2) ? (uint32_t)(j & 1) : 0u;      // which O accumulator of the tile
-            const bool more = j + 2 < n_tiles;
-            const int sk = (j + 2) % C::kStagesK;
+            const int u = j % kSBufs;
+            const bool more = j + kSBufs < n_tiles;
+            const int sk = (j + kSBufs) % C::kStagesK;
             wait_bar(bar.vf + 8 * sv, (j / C::kStagesV) & 1, &abort_flag, p.err_word);
-            if (more) wait_bar(bar.kf + 8 * sk, ((j + 2) / C::kStagesK) & 1, &abort_flag, p.err_word);
+            if (more) wait_bar(bar.kf + 8 * sk, ((j + kSBufs) / C::kStagesK) & 1, &abort_flag, p.err_word);
 #pragma unroll
             for (int t = 0; t < kTilesM; ++t) {
-                wait_bar(bar.p + 16 * t + 8 * (j & 1), (j >> 1) & 1, &abort_flag, p.err_word);
+                wait_bar(bar.p + 32 * t + 8 * u, (j / kSBufs) & 1, &abort_flag, p.err_word);
                 tc_fence_after();
                 if (elect_one()) {
 #pragma unroll
                     for (int ks = 0; ks < kBlockN / 16; ++ks)
-                        mma_ts(tmem + kColO + (t * kSplit + acc) * C::kOStride, tmem + t * 128 + sbuf + ks * 8,
+                        mma_ts(tmem + C::kColO + t * C::kOStride, tmem + (t * kSBufs + u) * kBlockN + ks * 8,
                                smem_desc(vbase + ks * 2048, C::kChunkBytes, 1024, kSwizzle128B),
-                               idesc_pv, (j >= kSplit || ks > 0) ? 1u : 0u);
-                    tc_commit(bar.o + 16 * t + 8 * acc);
+                               idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+                    tc_commit(bar.o + 32 * t + 8 * u);
                     if (t == kTilesM - 1) tc_commit(bar.ve + 8 * sv);
-                    // the S buffer just consumed as P is free again (in-order pipe): refill it with key tile j+2
+                    // the S buffer just consumed as P is free again (in-order pipe): refill it with key tile j+kSBufs
                     if (more) {
-                        issue_qk(t, j + 2, sK + sk * C::kTileBytes);
+                        issue_qk(t, j + kSBufs, sK + sk * C::kTileBytes);
                         if (t == kTilesM - 1) tc_commit(bar.ke + 8 * sk);
                     }
                 }
@@ -551,7 +493,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 
     tc_fence_before();
     __syncthreads();
-    if (warp == kIssuerWarp) tmem_dealloc(tmem, kTmemCols);
+    if (warp == 9) tmem_dealloc(tmem, kTmemCols);
 }
 
 // ------------------------------------------------------------------ host side
@@ -615,7 +557,7 @@ int32_t launch_dh(const AttnArgs &a, cudaStream_t stream)
     p.compact = (a.flags & ASTRAEA_ATTN_COMPACT_OUT) ? 1 : 0;
     p.err_word = a.err_word;
     dim3 grid((a.M + kTilesM * kBlockM - 1) / (kTilesM * kBlockM), a.H, a.B);
-    sparse_attn_kernel<DH><<<grid, C::kThreads, C::kSmemBytes, stream>>>(mk, mv, p);
+    sparse_attn_kernel<DH><<<grid, kThreads, C::kSmemBytes, stream>>>(mk, mv, p);
     return check_launch("astraea_sparse_attn");
 }
 
