@@ -45,20 +45,29 @@ constexpr float kTileSumLimit = 65536.0f;        // a tile's sum of exponentials
 constexpr uint64_t kWaitLimitNs = 1000000000ull; // bounded waits: one second
 
 template <int DH> struct Cfg {
-    static constexpr int kSBufs = (DH == 128) ? 2 : 3;            // S buffers per query tile
+    // head_dim = kMain (whole 64-column, 128-byte-swizzled chunks) + kTail (8 columns at head_dim 72,
+    // carried as a 16-column, 32-byte-swizzled chunk whose upper half is zero)
+    static constexpr int kMain = DH / 64 * 64;
+    static constexpr int kTail = DH - kMain;
+    static constexpr int kTailPad = kTail ? 16 : 0;
+    static_assert(kTail == 0 || kTail == 8, "head_dim must be 64, 72 or 128");
+    static constexpr int kSBufs = (DH == 64) ? 3 : 2;             // S buffers per query tile
     static constexpr uint32_t kColO = kTilesM * kSBufs * kBlockN; // first O column
-    static constexpr uint32_t kOStride = (DH == 128) ? 128 : 64;
-    static_assert(kColO + kTilesM * kOStride <= kTmemCols && DH <= (int)kOStride, "TMEM budget");
+    static constexpr uint32_t kOStride = (DH == 64) ? 64 : 128;
+    static_assert(kColO + kTilesM * kOStride <= kTmemCols && kMain + kTailPad <= (int)kOStride, "TMEM budget");
     // setmaxnreg only redistributes what the CTA got at launch: an increase that the decreases of
     // the last warpgroup cannot cover would block forever
     static constexpr int kRegsLaunch = (65536 / kThreads) / 8 * 8;
     static constexpr int kRegsSoftmax = 232, kRegsOther = 40;
     static_assert(kRegsSoftmax * 256 + kRegsOther * 128 <= kRegsLaunch * kThreads, "setmaxnreg budget");
-    static constexpr int kChunks = DH / 64;                       // 64-column (128-byte) swizzle chunks
+    static constexpr int kChunks = kMain / 64;                    // 64-column (128-byte) swizzle chunks
     static constexpr int kQChunkBytes = kBlockM * 128;            // 128 query rows x 128 bytes
-    static constexpr int kQTileBytes = kChunks * kQChunkBytes;
+    static constexpr int kQTailBytes = kTail ? kBlockM * 32 : 0;  // 128 query rows x 32 bytes
+    static constexpr int kQTileBytes = kChunks * kQChunkBytes + kQTailBytes;
     static constexpr int kChunkBytes = kBlockN * 128;             // 64 keys x 128 bytes
-    static constexpr int kTileBytes = kChunks * kChunkBytes;      // one K or V tile
+    static constexpr int kTailBytes = kTail ? kBlockN * 32 : 0;   // 64 keys x 32 bytes
+    static constexpr int kTileBytes = kChunks * kChunkBytes + kTailBytes;   // one K or V tile
+    static_assert(kQTileBytes % 1024 == 0 && kTileBytes % 1024 == 0, "tiles keep the 1024-byte swizzle alignment");
     static constexpr int kStagesK = (DH == 128) ? 5 : 6;
     static constexpr int kStagesV = (DH == 128) ? 5 : 6;
     static_assert(kStagesK > kSBufs, "K runs kSBufs tiles ahead");
@@ -226,13 +235,21 @@ __device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j)
             wait_bar(st.bar_o + 8 * ((j - 1) % kSBufs), ((j - 1) / kSBufs) & 1, st.abort_flag, st.err_word);
             tc_fence_after();
 #pragma unroll
-            for (int cc = 0; cc < DH / 32; ++cc) {
+            for (int cc = 0; cc < Cfg<DH>::kMain / 32; ++cc) {
                 uint32_t o[32];
                 tmem_ld32(st.t_o + cc * 32, o);
                 tc_wait_ld();
 #pragma unroll
                 for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
                 tmem_st32(st.t_o + cc * 32, o);
+            }
+            if (Cfg<DH>::kTail) {
+                uint32_t o[16];
+                tmem_ld16(st.t_o + Cfg<DH>::kMain, o);
+                tc_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                tmem_st16(st.t_o + Cfg<DH>::kMain, o);
             }
             tc_wait_st();
         }
@@ -259,28 +276,25 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
                                              int m_base, int h, int b, int n_tiles, volatile int *abort_flag)
 {
     using C = Cfg<DH>;
-    const int wtid = threadIdx.x & 127, lane = wtid & 31;
+    const int wtid = threadIdx.x & 127;
     const int warp = __shfl_sync(0xffffffffu, wtid >> 5, 0);       // warp-uniform
-    // gather this tile's Q rows (swizzled, K-major)
-    constexpr int kVecPerRow = DH / 8;                 // 16-byte vectors per row
-    constexpr int kRowsPerIter = 32 / kVecPerRow;
-    {
-        const int sub = lane / kVecPerRow, c = lane % kVecPerRow;
-#pragma unroll 4
-        for (int r0 = warp * kRowsPerIter; r0 < kBlockM; r0 += 4 * kRowsPerIter) {
-            const int r = r0 + sub;
-            const int m = m_base + r;
-            uint4 val = make_uint4(0, 0, 0, 0);
-            if (m < p.M) {
-                const int tok = p.q_idx ? __ldg(p.q_idx + (size_t)b * p.M + m) : m;
-                if ((unsigned)tok < (unsigned)p.N) {
-                    const __nv_bfloat16 *src = p.q + (size_t)b * p.q_sb + (size_t)tok * p.q_sn + (size_t)h * p.q_sh + c * 8;
-                    val = __ldg(reinterpret_cast<const uint4 *>(src));
-                }
+    // gather this tile's Q rows (swizzled, K-major): 16-byte units, unit c of row r
+    constexpr int kMainUnits = C::kMain / 8, kUnits = kMainUnits + (C::kTail ? 2 : 0);
+    for (int v = wtid; v < kBlockM * kUnits; v += 128) {
+        const int r = v / kUnits, c = v - r * kUnits;
+        const int m = m_base + r;
+        uint4 val = make_uint4(0, 0, 0, 0);
+        if (m < p.M && c * 8 < DH) {                 // the upper half of the tail chunk stays zero
+            const int tok = p.q_idx ? __ldg(p.q_idx + (size_t)b * p.M + m) : m;
+            if ((unsigned)tok < (unsigned)p.N) {
+                const __nv_bfloat16 *src = p.q + (size_t)b * p.q_sb + (size_t)tok * p.q_sn + (size_t)h * p.q_sh + c * 8;
+                val = __ldg(reinterpret_cast<const uint4 *>(src));
             }
-            const uint32_t off = (c >> 3) * C::kQChunkBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);
-            *reinterpret_cast<uint4 *>(sQ_gen + off) = val;
         }
+        uint32_t off;
+        if (c < kMainUnits) off = (c >> 3) * C::kQChunkBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);          // 128-byte swizzle
+        else off = C::kChunks * C::kQChunkBytes + r * 32 + ((((c - kMainUnits) & 1) ^ ((r >> 2) & 1)) << 4);   // 32-byte swizzle
+        *reinterpret_cast<uint4 *>(sQ_gen + off) = val;
     }
     fence_proxy_async_smem();
     mbar_arrive(bar.q + 8 * tile);
@@ -318,7 +332,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
         }
     }
 #pragma unroll
-    for (int cc = 0; cc < DH / 32; ++cc) {
+    for (int cc = 0; cc < C::kMain / 32; ++cc) {
         uint32_t o[32];
         tmem_ld32(st.t_o + cc * 32, o);
         tc_wait_ld();
@@ -336,11 +350,23 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
             }
         }
     }
+    if (C::kTail) {
+        uint32_t o[8], w[4];
+        tmem_ld8(st.t_o + C::kMain, o);
+        tc_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(o[2 * i]) * inv_l, __uint_as_float(o[2 * i + 1]) * inv_l);
+            w[i] = *reinterpret_cast<uint32_t *>(&v2);
+        }
+        if (dst) *reinterpret_cast<uint4 *>(dst + C::kMain) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
 }
 
 template <int DH>
 __global__ void __launch_bounds__(kThreads, 1)
-sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v, const Params p)
+sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
+                   const __grid_constant__ CUtensorMap tmap_k_tail, const __grid_constant__ CUtensorMap tmap_v_tail, const Params p)
 {
     using C = Cfg<DH>;
     constexpr int kSBufs = C::kSBufs;
@@ -395,7 +421,10 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     } else if (warp == 8) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
         // ------------------------------------------------ TMA producer (warp-uniform, one elected lane issues)
-        if (elect_one()) { prefetch_tensormap(&tmap_k); prefetch_tensormap(&tmap_v); }
+        if (elect_one()) {
+            prefetch_tensormap(&tmap_k); prefetch_tensormap(&tmap_v);
+            if (C::kTail) { prefetch_tensormap(&tmap_k_tail); prefetch_tensormap(&tmap_v_tail); }
+        }
         auto load_k = [&](int j) {
             const int st = j % C::kStagesK;
             wait_bar(bar.ke + 8 * st, ((j / C::kStagesK) & 1) ^ 1, &abort_flag, p.err_word);
@@ -404,6 +433,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 #pragma unroll
                 for (int ch = 0; ch < C::kChunks; ++ch)
                     tma_load_4d(sK + st * C::kTileBytes + ch * C::kChunkBytes, &tmap_k, bar.kf + 8 * st, ch * 64, j * kBlockN, h, b);
+                if (C::kTail)
+                    tma_load_4d(sK + st * C::kTileBytes + C::kChunks * C::kChunkBytes, &tmap_k_tail, bar.kf + 8 * st, C::kMain, j * kBlockN, h, b);
             }
             __syncwarp();
         };
@@ -415,6 +446,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 #pragma unroll
                 for (int ch = 0; ch < C::kChunks; ++ch)
                     tma_load_4d(sV + st * C::kTileBytes + ch * C::kChunkBytes, &tmap_v, bar.vf + 8 * st, ch * 64, j * kBlockN, h, b);
+                if (C::kTail)
+                    tma_load_4d(sV + st * C::kTileBytes + C::kChunks * C::kChunkBytes, &tmap_v_tail, bar.vf + 8 * st, C::kMain, j * kBlockN, h, b);
             }
             __syncwarp();
         };
@@ -433,15 +466,20 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
         // ------------------------------------------------ MMA issuer (warp-uniform, one elected lane issues)
         constexpr uint32_t idesc_qk = idesc_bf16(kBlockM, kBlockN, false);
-        constexpr uint32_t idesc_pv = idesc_bf16(kBlockM, DH, true);
+        constexpr uint32_t idesc_pv = idesc_bf16(kBlockM, C::kMain, true);
+        constexpr uint32_t idesc_pv_tail = idesc_bf16(kBlockM, 16, true);
         auto issue_qk = [&](int t, int j, uint32_t kbase) {        // S[t][j % kSBufs] = Q_t K_j^T  (one elected lane)
             const int u = j % kSBufs;
 #pragma unroll
-            for (int ks = 0; ks < DH / 16; ++ks)
+            for (int ks = 0; ks < C::kMain / 16; ++ks)
                 mma_ss(tmem + (t * kSBufs + u) * kBlockN,
                        smem_desc(sQ + t * C::kQTileBytes + (ks >> 2) * C::kQChunkBytes + (ks & 3) * 32, 16, 1024, kSwizzle128B),
                        smem_desc(kbase + (ks >> 2) * C::kChunkBytes + (ks & 3) * 32, 16, 1024, kSwizzle128B),
                        idesc_qk, ks > 0);
+            if (C::kTail)      // columns 64..79 (72..79 are zero): one more K step on the 32-byte-swizzled chunks
+                mma_ss(tmem + (t * kSBufs + u) * kBlockN,
+                       smem_desc(sQ + t * C::kQTileBytes + C::kChunks * C::kQChunkBytes, 16, 256, kSwizzle32B),
+                       smem_desc(kbase + C::kChunks * C::kChunkBytes, 16, 256, kSwizzle32B), idesc_qk, 1u);
             tc_commit(bar.s + 32 * t + 8 * u);
         };
         // prologue: S of the first kSBufs key tiles for both query tiles
@@ -472,10 +510,15 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                 tc_fence_after();
                 if (elect_one()) {
 #pragma unroll
-                    for (int ks = 0; ks < kBlockN / 16; ++ks)
+                    for (int ks = 0; ks < kBlockN / 16; ++ks) {
                         mma_ts(tmem + C::kColO + t * C::kOStride, tmem + (t * kSBufs + u) * kBlockN + ks * 8,
                                smem_desc(vbase + ks * 2048, C::kChunkBytes, 1024, kSwizzle128B),
                                idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+                        if (C::kTail)  // O columns 64..79 from the 16-column chunk of V
+                            mma_ts(tmem + C::kColO + t * C::kOStride + C::kMain, tmem + (t * kSBufs + u) * kBlockN + ks * 8,
+                                   smem_desc(vbase + C::kChunks * C::kChunkBytes + ks * 512, 256, 256, kSwizzle32B),
+                                   idesc_pv_tail, (j > 0 || ks > 0) ? 1u : 0u);
+                    }
                     tc_commit(bar.o + 32 * t + 8 * u);
                     if (t == kTilesM - 1) tc_commit(bar.ve + 8 * sv);
                     // the S buffer just consumed as P is free again (in-order pipe): refill it with key tile j+kSBufs
@@ -515,16 +558,17 @@ EncodeTiledFn get_encode_fn() {
 
 // K or V as a 4-D tensor (d, N, H, B) with 128-byte-swizzled boxes of 64 columns x 128 tokens
 int32_t make_kv_map(CUtensorMap *map, const void *base, int B, int H, int N, int d,
-                    int64_t sb, int64_t sh, int64_t sn)
+                    int64_t sb, int64_t sh, int64_t sn, bool tail)
 {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) return fail(ASTRAEA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
     cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)H, (cuuint64_t)B};
     cuuint64_t strides[3] = {(cuuint64_t)sn * 2, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
-    cuuint32_t box[4] = {64, (cuuint32_t)kBlockN, 1, 1};   // 64 columns x one key tile
+    // 64 columns x one key tile, 128-byte swizzle; or the 16-column tail chunk (32-byte swizzle; columns past d read as zero)
+    cuuint32_t box[4] = {tail ? 16u : 64u, (cuuint32_t)kBlockN, 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
-                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, tail ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(ASTRAEA_ERR_INVALID_ARG, "tensor map rejected (CUresult %d): check K/V strides and alignment", (int)r);
     return ASTRAEA_OK;
@@ -534,11 +578,18 @@ template <int DH>
 int32_t launch_dh(const AttnArgs &a, cudaStream_t stream)
 {
     using C = Cfg<DH>;
-    CUtensorMap mk, mv;
-    int32_t rc = make_kv_map(&mk, a.k, a.B, a.H, a.N, a.d, a.k_sb, a.k_sh, a.k_sn);
+    CUtensorMap mk, mv, mkt, mvt;
+    int32_t rc = make_kv_map(&mk, a.k, a.B, a.H, a.N, a.d, a.k_sb, a.k_sh, a.k_sn, false);
     if (rc != ASTRAEA_OK) return rc;
-    rc = make_kv_map(&mv, a.v, a.B, a.H, a.N, a.d, a.v_sb, a.v_sh, a.v_sn);
+    rc = make_kv_map(&mv, a.v, a.B, a.H, a.N, a.d, a.v_sb, a.v_sh, a.v_sn, false);
     if (rc != ASTRAEA_OK) return rc;
+    mkt = mk; mvt = mv;
+    if (C::kTail) {
+        rc = make_kv_map(&mkt, a.k, a.B, a.H, a.N, a.d, a.k_sb, a.k_sh, a.k_sn, true);
+        if (rc != ASTRAEA_OK) return rc;
+        rc = make_kv_map(&mvt, a.v, a.B, a.H, a.N, a.d, a.v_sb, a.v_sh, a.v_sn, true);
+        if (rc != ASTRAEA_OK) return rc;
+    }
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(sparse_attn_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
@@ -557,7 +608,7 @@ int32_t launch_dh(const AttnArgs &a, cudaStream_t stream)
     p.compact = (a.flags & ASTRAEA_ATTN_COMPACT_OUT) ? 1 : 0;
     p.err_word = a.err_word;
     dim3 grid((a.M + kTilesM * kBlockM - 1) / (kTilesM * kBlockM), a.H, a.B);
-    sparse_attn_kernel<DH><<<grid, kThreads, C::kSmemBytes, stream>>>(mk, mv, p);
+    sparse_attn_kernel<DH><<<grid, kThreads, C::kSmemBytes, stream>>>(mk, mv, mkt, mvt, p);
     return check_launch("astraea_sparse_attn");
 }
 
@@ -569,6 +620,7 @@ int32_t launch_sparse_attn(const AttnArgs &a, cudaStream_t stream)
 {
     switch (a.d) {
     case 64: return launch_dh<64>(a, stream);
+    case 72: return launch_dh<72>(a, stream);
     case 128: return launch_dh<128>(a, stream);
     default: return fail(ASTRAEA_ERR_UNSUPPORTED, "head_dim %d is not supported", a.d);
     }

@@ -206,13 +206,13 @@ def test_attn_tiny_config(oracle):
     _attn_case(oracle, 1, 2, 256, 64, 128, seed=0)
 
 
-@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("d", [64, 72, 128])
 def test_attn_single_tile(oracle, d):
     _attn_case(oracle, 1, 1, 128, d, 128, seed=1, dense=True)
 
 
-@pytest.mark.parametrize("d", [64, 128])
-@pytest.mark.parametrize("N,M", [(300, 77), (1000, 333), (129, 129), (1, 1), (127, 5)])
+@pytest.mark.parametrize("d", [64, 72, 128])
+@pytest.mark.parametrize("N,M", [(300, 77), (1000, 333), (129, 129), (1, 1), (127, 5), (64, 64), (65, 3)])
 def test_attn_ragged_tiles(oracle, d, N, M):
     _attn_case(oracle, 2, 3, N, d, M, seed=2)
 
@@ -220,6 +220,13 @@ def test_attn_ragged_tiles(oracle, d, N, M):
 def test_attn_many_key_tiles_exercise_every_stage_phase(oracle):
     _attn_case(oracle, 1, 2, 128 * 19 + 16, 128, 200, seed=3)
     _attn_case(oracle, 1, 2, 128 * 27 + 112, 64, 130, seed=4)
+    _attn_case(oracle, 1, 2, 128 * 23 + 40, 72, 260, seed=5)
+
+
+def test_attn_head_dim_72_layouts(oracle):
+    _attn_case(oracle, 2, 2, 400, 72, 100, seed=11, layout="bhnd")
+    _attn_case(oracle, 2, 3, 400, 72, 100, seed=12, compact=True)
+    _attn_case(oracle, 1, 2, 900, 72, 128, seed=13, amp=2.5)
 
 
 def test_attn_head_major_layout_compact_output_and_scale(oracle):
@@ -314,7 +321,9 @@ def _step_case(oracle, w, seed, theta, steps=1):
         assert np.array_equal(idx_rem.cpu().numpy(), res["idx_rem"])
         assert np.array_equal(n_skip.cpu().numpy(), res["n_skip"])
         got_out = bf16_dev_to_f64(out)
-        err = np.abs(got_out - res["out"])
+        # the tolerances are stated for N(0,1) values; where the workload scales the value rows
+        # (per-token lognormal norms) they scale with the output's magnitude
+        err = np.abs(got_out - res["out"]) / np.maximum(1.0, np.abs(res["out"]))
         assert err.max() < ATTN_MAX_ABS and err.mean() < ATTN_MEAN_ABS
         sel_mask = np.zeros((B, N), bool)
         for b in range(B):
@@ -339,6 +348,11 @@ def test_step_keep_ratio_zero_and_one(oracle):
 def test_step_with_text_tokens_and_batch(oracle):
     w = synth.Workload("mini-cog", B=2, H=4, d=64, N_v=450, N_t=26)
     _step_case(oracle, w, 2, 250)
+
+
+def test_step_opensora_shaped_reduced(oracle):
+    w = synth.scaled(synth.WORKLOADS["opensora"], N_v=8 * 16 * 16, H=4)
+    _step_case(oracle, w, 4, 400)
 
 
 def test_step_chain_of_three_steps_d128(oracle):
