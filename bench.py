@@ -27,14 +27,14 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from paper_2506_05096_b200 import accounting, synth  # noqa: E402
+from paper_2506_05096_b200 import accounting, replicas, synth  # noqa: E402
 
 METRIC = "sparse_attn_effective_tflops"
 UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the attention kernel, from the ncu
 # capture summarised in profiles/ (workload -> theta_permille -> bytes); None where not captured.
-NCU_TRAFFIC_BYTES = {"cogvideox": {500: 326806272}}
+NCU_TRAFFIC_BYTES = {"cogvideox": {500: 324956160}, "sweep": {250: 1315367968}}
 
 
 def measured_peaks():
@@ -182,7 +182,7 @@ def main():
 
     # two input sets (step t and t+1 of a drifting latent), alternated so that the reference
     # inputs keep differing from the current ones; replicas use different seeds
-    inp = synth.make_step_inputs(w, seed=rank)
+    inp = synth.make_step_inputs(w, seed=replicas.rank_seed(0, rank))
     sets = [{n: bf(inp[n]) for n in ("x_cur", "q", "k", "v")}]
     sets.append({"x_cur": bf(synth.drift_step(inp["x_cur"], 1000 + rank, 0.05, False)),
                  **{n: bf(synth.drift_step(inp[n], 1001 + i + rank, 0.05, True)) for i, n in enumerate(("q", "k", "v"))}})
@@ -245,13 +245,10 @@ def main():
     M = k_keep + n_always
     total_ms, parts = timed(k_keep, args.steps, args.warmup, 1)
     A.astraea_poll_error(ws)
-    if world > 1:
-        tt = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
-    ms_per_step = total_ms / args.steps
     flops = accounting.attn_flops(B, H, M, N, d)
-    value = world * flops / (ms_per_step * 1e-3) / 1e12
+    total_ms, job_flops = replicas.aggregate(total_ms, flops * args.steps, device="cuda")
+    ms_per_step = total_ms / args.steps
+    value = replicas.throughput(job_flops, total_ms) / 1e12
 
     peaks = measured_peaks()
     attn_ms = float(parts[2])
@@ -309,12 +306,10 @@ def main():
             sess.step_host(host["x_cur"], host["q"], host["k"], host["v"], host_out, k_keep, w_alpha, 1.0)
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
-        if world > 1:
-            tt = torch.tensor([dt], device="cuda", dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            dt = float(tt.item())
+        dt_ms, e2e_flops = replicas.aggregate(dt * 1e3, flops * n_e2e, device="cuda")
+        dt = dt_ms * 1e-3
         sess.close()
-        e2e = {"value": world * flops / (dt / n_e2e) / 1e12, "unit": UNIT, "h2d_bytes_per_step": 4 * tb,
+        e2e = {"value": replicas.throughput(e2e_flops, dt_ms) / 1e12, "unit": UNIT, "h2d_bytes_per_step": 4 * tb,
                "d2h_bytes_per_step": tb, "ms_per_step": 1e3 * dt / n_e2e, "steps": n_e2e,
                "api": "astraea_step_host (pinned host buffers)"}
 
