@@ -130,6 +130,37 @@ int32_t astraea_sparse_attn(const void *q, const void *k, const void *v,
                             void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The same attention for callers that must not allocate.  (The paper has no counterpart: this is a
+ * property of the library, not of the method.)  astraea_sparse_attn takes its scratch from the
+ * caller, which some callers cannot provide: code that runs while a CUDA memory pool or a framework
+ * allocator is locked, inside a region where cudaMalloc would synchronise the device, or in a
+ * process whose device memory has been handed out in full to other owners.  This entry point keeps
+ * its scratch in a fixed array inside the library image instead (ASTRAEA_NOALLOC_SCRATCH_BYTES per
+ * GPU that loads the library, held until the process exits) and calls no cudaMalloc, cudaFree or
+ * other allocating routine.  Arguments, arithmetic and results are those of astraea_sparse_attn
+ * without the workspace pair.
+ *   - Problems whose scratch need (astraea_workspace_bytes(ASTRAEA_OP_SPARSE_ATTN, ...)) exceeds
+ *     ASTRAEA_NOALLOC_SCRATCH_BYTES are rejected with ASTRAEA_ERR_WORKSPACE_TOO_SMALL.
+ *   - The first call on a device resolves the array's device address (with that device current);
+ *     make that first call before any stream capture.
+ *   - All calls on a device share the one array.  It keeps the last call's contents, so each call
+ *     first clears the part it uses on `stream`; calls that overlap on the GPU (different streams)
+ *     race on it and must be serialised by the caller.
+ *   - The error word lives in that array, so astraea_poll_error cannot be pointed at it: a device-side
+ *     timeout or bad index in this variant is not reported.  Callers that need the report use
+ *     astraea_sparse_attn.
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE_TOO_SMALL (see above), CUDA.
+ */
+#define ASTRAEA_NOALLOC_SCRATCH_BYTES 4096
+int32_t astraea_sparse_attn_noalloc(const void *q, const void *k, const void *v,
+                                    int64_t q_sb, int64_t q_sh, int64_t q_sn,
+                                    int64_t k_sb, int64_t k_sh, int64_t k_sn,
+                                    int64_t v_sb, int64_t v_sh, int64_t v_sn,
+                                    const int32_t *q_idx, int M, const int32_t *kv_idx, int M_kv,
+                                    void *out, float *lse_out,
+                                    int B, int H, int N, int d, float scale, uint32_t flags, void *stream);
+
+/*
  * Reuse / cache update (Algorithm 1 lines 6-7; Section 3.2 "Execution Flow"):
  *     cache[b, idx[b,r], :] = rows[b, r, :]      (rows compact [B, M, row_elems]), or
  *     cache[b, idx[b,r], :] = rows[b, idx[b,r], :] with ASTRAEA_SCATTER_SRC_FULL;

@@ -23,9 +23,10 @@ ATTN_COMPACT_OUT = 1
 SCATTER_SRC_FULL = 1
 OP_SELECT, OP_SPARSE_ATTN, OP_STEP = 1, 2, 3
 N_SKIP_CLAMP = 80
+NOALLOC_SCRATCH_BYTES = 4096
 
 EXPORTS = [
-    "astraea_score", "astraea_select", "astraea_sparse_attn", "astraea_scatter_reuse", "astraea_step",
+    "astraea_score", "astraea_select", "astraea_sparse_attn", "astraea_sparse_attn_noalloc", "astraea_scatter_reuse", "astraea_step",
     "astraea_session_create", "astraea_session_destroy", "astraea_step_host",
     "astraea_workspace_bytes", "astraea_budget_to_k", "astraea_poll_error",
     "astraea_last_error", "astraea_version",
@@ -54,6 +55,8 @@ def lib() -> ctypes.CDLL:
         L.astraea_select.argtypes = [c_p, c_i, c_i, c_i, c_i, c_p, c_p, c_p, c_p, c_sz, c_p]
         L.astraea_sparse_attn.argtypes = [c_p, c_p, c_p] + [c_i64] * 9 + [c_p, c_i, c_p, c_i, c_p, c_p,
                                                                          c_i, c_i, c_i, c_i, c_f, c_u, c_p, c_sz, c_p]
+        L.astraea_sparse_attn_noalloc.argtypes = [c_p, c_p, c_p] + [c_i64] * 9 + [c_p, c_i, c_p, c_i, c_p, c_p,
+                                                                                 c_i, c_i, c_i, c_i, c_f, c_u, c_p]
         L.astraea_scatter_reuse.argtypes = [c_p, c_p, c_p, c_i, c_i, c_i, c_i, c_u, c_p]
         L.astraea_step.argtypes = [c_p] * 11 + [c_i] * 6 + [c_f, c_f, c_i, c_i, c_p, c_sz, c_p]
         L.astraea_session_create.argtypes = [ctypes.POINTER(c_p), c_i, c_i, c_i, c_i, c_i]
@@ -66,7 +69,7 @@ def lib() -> ctypes.CDLL:
         L.astraea_poll_error.argtypes = [c_p, c_p]
         L.astraea_last_error.restype = ctypes.c_char_p
         L.astraea_version.restype = ctypes.c_char_p
-        for name in ("astraea_score", "astraea_select", "astraea_sparse_attn", "astraea_scatter_reuse",
+        for name in ("astraea_score", "astraea_select", "astraea_sparse_attn", "astraea_sparse_attn_noalloc", "astraea_scatter_reuse",
                      "astraea_step", "astraea_session_create", "astraea_step_host", "astraea_budget_to_k",
                      "astraea_poll_error"):
             getattr(L, name).restype = ctypes.c_int32
@@ -131,6 +134,15 @@ def astraea_sparse_attn(q, k, v, q_strides, k_strides, v_strides, q_idx, M, out,
                                      _ptr(q_idx), M, _ptr(kv_idx), M_kv, _ptr(out), _ptr(lse_out),
                                      B, H, N, d, scale, flags, _ptr(workspace),
                                      workspace.numel() if workspace is not None else 0, _stream(stream)))
+
+
+def astraea_sparse_attn_noalloc(q, k, v, q_strides, k_strides, v_strides, q_idx, M, out, lse_out, B, H, N, d,
+                                scale=0.0, flags=0, kv_idx=None, M_kv=0, stream=None) -> None:
+    """astraea_sparse_attn for callers that cannot allocate: the scratch is a fixed array inside the
+    library (NOALLOC_SCRATCH_BYTES per GPU), shared by all calls on the device, so overlapping calls race."""
+    _check(lib().astraea_sparse_attn_noalloc(_ptr(q), _ptr(k), _ptr(v), *q_strides, *k_strides, *v_strides,
+                                             _ptr(q_idx), M, _ptr(kv_idx), M_kv, _ptr(out), _ptr(lse_out),
+                                             B, H, N, d, scale, flags, _stream(stream)))
 
 
 def astraea_scatter_reuse(cache, rows, idx, B, N, M, row_elems, flags=0, stream=None) -> None:

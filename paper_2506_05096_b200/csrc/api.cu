@@ -131,6 +131,43 @@ int32_t astraea_sparse_attn(const void *q, const void *k, const void *v,
     return launch_sparse_attn(a, (cudaStream_t)stream);
 }
 
+int32_t astraea_sparse_attn_noalloc(const void *q, const void *k, const void *v,
+                                    int64_t q_sb, int64_t q_sh, int64_t q_sn,
+                                    int64_t k_sb, int64_t k_sh, int64_t k_sn,
+                                    int64_t v_sb, int64_t v_sh, int64_t v_sn,
+                                    const int32_t *q_idx, int M, const int32_t *kv_idx, int M_kv,
+                                    void *out, float *lse_out,
+                                    int B, int H, int N, int d, float scale, uint32_t flags, void *stream)
+{
+    (void)M_kv;
+    REQUIRE(B > 0 && H > 0 && N > 0 && d > 0, "astraea_sparse_attn_noalloc: B, H, N, d must be positive");
+    REQUIRE(M >= 0 && M <= N, "astraea_sparse_attn_noalloc: M=%d outside [0, N=%d]", M, N);
+    if (d != 64 && d != 72 && d != 128)
+        return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_sparse_attn_noalloc: head_dim %d not in {64, 72, 128}", d);
+    if (kv_idx) return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_sparse_attn_noalloc: kv_idx (select-Q-and-K ablation) is not built");
+    if (flags & ~ASTRAEA_ATTN_COMPACT_OUT) return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_sparse_attn_noalloc: unknown flags 0x%x", flags);
+    REQUIRE(q && k && v && out, "astraea_sparse_attn_noalloc: null q, k, v or out");
+    REQUIRE(aligned16(q) && aligned16(k) && aligned16(v) && aligned16(out), "astraea_sparse_attn_noalloc: q, k, v, out must be 16-byte aligned");
+    REQUIRE(q_sn % 8 == 0 && k_sn % 8 == 0 && v_sn % 8 == 0 && q_sh % 8 == 0 && k_sh % 8 == 0 && v_sh % 8 == 0 &&
+            q_sb % 8 == 0 && k_sb % 8 == 0 && v_sb % 8 == 0,
+            "astraea_sparse_attn_noalloc: strides must be multiples of 8 elements (16 bytes)");
+    REQUIRE(q_sn >= d && k_sn >= d && v_sn >= d && q_sh > 0 && k_sh > 0 && v_sh > 0 && q_sb >= 0 && k_sb >= 0 && v_sb >= 0,
+            "astraea_sparse_attn_noalloc: strides must be positive and token stride >= head_dim");
+    REQUIRE(scale >= 0.f, "astraea_sparse_attn_noalloc: scale must be >= 0 (0 selects 1/sqrt(d))");
+    if (M == 0) return ASTRAEA_OK;
+    AttnArgs a;
+    a.q = q; a.k = k; a.v = v;
+    a.q_sb = q_sb; a.q_sh = q_sh; a.q_sn = q_sn;
+    a.k_sb = k_sb; a.k_sh = k_sh; a.k_sn = k_sn;
+    a.v_sb = v_sb; a.v_sh = v_sh; a.v_sn = v_sn;
+    a.q_idx = q_idx; a.M = M; a.out = out; a.lse_out = lse_out;
+    a.B = B; a.H = H; a.N = N; a.d = d;
+    a.scale = (scale == 0.f) ? 1.0f / sqrtf((float)d) : scale;
+    a.flags = flags;
+    a.err_word = nullptr;
+    return launch_sparse_attn_noalloc(a, (cudaStream_t)stream);
+}
+
 int32_t astraea_scatter_reuse(void *cache, const void *rows, const int32_t *idx,
                               int B, int N, int M, int row_elems, uint32_t flags, void *stream)
 {

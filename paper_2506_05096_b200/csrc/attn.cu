@@ -28,6 +28,8 @@
 // that descriptors and addresses stay in uniform registers (a lone diverged thread issues
 // tcgen05.mma several times slower).  Every mbarrier wait is bounded; on a timeout the CTA raises
 // the error word, the remaining waits return at once, and the CTA runs out.
+#include <mutex>
+
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -615,6 +617,45 @@ int32_t launch_dh(const AttnArgs &a, cudaStream_t stream)
 }  // namespace
 
 size_t attn_workspace_bytes(int, int, int, int, int) { return 256; }
+
+// Scratch of astraea_sparse_attn_noalloc: lives in the library image, so every GPU that loads the
+// library holds these bytes until the process exits.  In host code this name is only a handle of
+// the symbol, never a device address: the address comes from cudaGetSymbolAddress, per device.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[ASTRAEA_NOALLOC_SCRATCH_BYTES];
+
+int32_t launch_sparse_attn_noalloc(AttnArgs a, cudaStream_t stream)
+{
+    const size_t need = attn_workspace_bytes(a.B, a.H, a.N, a.M, a.d);
+    if (need > ASTRAEA_NOALLOC_SCRATCH_BYTES)
+        return fail(ASTRAEA_ERR_WORKSPACE_TOO_SMALL,
+                    "astraea_sparse_attn_noalloc: this problem needs %zu bytes of scratch, the built-in scratch holds %d; "
+                    "use astraea_sparse_attn with a caller workspace", need, ASTRAEA_NOALLOC_SCRATCH_BYTES);
+    // one-time set-up per device (with that device current): resolve the symbol to its device address
+    constexpr int kMaxDevices = 64;
+    static void *scratch_of_device[kMaxDevices] = {};
+    static std::mutex mu;
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices)
+        return fail(ASTRAEA_ERR_CUDA, "astraea_sparse_attn_noalloc: no usable current device (%s)", cudaGetErrorString(e));
+    void *scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!scratch_of_device[dev]) {
+            void *ptr = nullptr;
+            e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+            if (e != cudaSuccess || !ptr)
+                return fail(ASTRAEA_ERR_CUDA, "astraea_sparse_attn_noalloc: cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
+            scratch_of_device[dev] = ptr;
+        }
+        scratch = scratch_of_device[dev];
+    }
+    // the array keeps what the last call left: the error word must start at zero
+    e = cudaMemsetAsync(scratch, 0, need, stream);
+    if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_sparse_attn_noalloc: clearing the scratch failed: %s", cudaGetErrorString(e));
+    a.err_word = reinterpret_cast<int *>(scratch);
+    return launch_sparse_attn(a, stream);
+}
 
 int32_t launch_sparse_attn(const AttnArgs &a, cudaStream_t stream)
 {

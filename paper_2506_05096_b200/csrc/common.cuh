@@ -45,5 +45,6 @@ struct AttnArgs {
 };
 int32_t launch_sparse_attn(const AttnArgs &a, cudaStream_t stream);
 size_t attn_workspace_bytes(int B, int H, int N, int M, int d);
+int32_t launch_sparse_attn_noalloc(AttnArgs a, cudaStream_t stream);   // scratch in a static device array
 
 }  // namespace astraea

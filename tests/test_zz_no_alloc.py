@@ -1,0 +1,51 @@
+"""astraea_sparse_attn_noalloc, the entry point for callers that cannot allocate device memory (their
+allocator is locked, or they run where cudaMalloc would stall the device): it must give what
+astraea_sparse_attn gives while taking its scratch from a fixed array inside the library.  Two calls in
+a row share that array, so the second call also checks that nothing stale from the first one leaks in.
+This file sorts last on purpose: a run that stops at the first failure has then run everything else."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2506_05096_b200 import binding as A
+
+pytestmark = pytest.mark.gpu
+
+
+def _inputs(seed, B, H, N, d, M):
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    q, k, v, cache = (torch.randn(B, N, H, d, generator=g).bfloat16().cuda() for _ in range(4))
+    idx = torch.stack([torch.sort(torch.randperm(N, generator=g)[:M])[0] for _ in range(B)]).int().cuda()
+    return q, k, v, cache, idx
+
+
+def test_noalloc_entry_matches_the_workspace_entry_on_two_calls_in_a_row():
+    for call, (seed, B, H, N, d, M) in enumerate([(1, 2, 3, 700, 64, 300), (2, 1, 2, 1500, 128, 260)]):
+        q, k, v, cache, idx = _inputs(seed, B, H, N, d, M)
+        s = A.bhnd_strides(N, H, d)
+        want, want_lse = cache.clone(), torch.zeros(B, H, N, device="cuda")
+        ws = A.new_workspace(A.OP_SPARSE_ATTN, B, H, N, M, d)
+        A.astraea_sparse_attn(q, k, v, s, s, s, idx, M, want, want_lse, B, H, N, d, workspace=ws)
+        A.astraea_poll_error(ws)
+        got, got_lse = cache.clone(), torch.zeros(B, H, N, device="cuda")
+        A.astraea_sparse_attn_noalloc(q, k, v, s, s, s, idx, M, got, got_lse, B, H, N, d)
+        torch.cuda.synchronize()
+        err = (got.float() - want.float()).abs()
+        assert err.max().item() < 2e-2 and err.mean().item() < 2e-3, (call, err.max().item())
+        assert (got_lse - want_lse).abs().max().item() < 1e-3
+        # rows that were not selected keep the cache, exactly as with the workspace entry
+        mask = torch.ones(B, N, dtype=torch.bool, device="cuda")
+        for b in range(B):
+            mask[b, idx[b].long()] = False
+        assert torch.equal(got[mask], cache[mask])
+
+
+def test_noalloc_entry_rejects_bad_arguments_like_the_workspace_entry():
+    z = torch.zeros(1, 64, 1, 64, dtype=torch.bfloat16, device="cuda")
+    s = A.bhnd_strides(64, 1, 64)
+    with pytest.raises(A.AstraeaError) as e:
+        A.astraea_sparse_attn_noalloc(z, z, z, s, s, s, None, 65, z, None, 1, 1, 64, 64)
+    assert e.value.code == A.ERR_INVALID_ARG
+    with pytest.raises(A.AstraeaError) as e:
+        A.astraea_sparse_attn_noalloc(z, z, z, s, s, s, None, 64, z, None, 1, 1, 64, 96)
+    assert e.value.code == A.ERR_UNSUPPORTED
