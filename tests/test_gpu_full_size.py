@@ -1,0 +1,92 @@
+"""Parity at the full sizes of the workloads, in the launch configuration bench.py times (the four calls of a
+step on one stream): scores and selection against the oracle at full size; attention on sampled selected rows
+(each output row depends only on its own query and all keys/values, so a sampled row is an exact check) for a few
+heads; every unselected row bit-identical to the cache."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2506_05096_b200 import binding as A
+from paper_2506_05096_b200 import synth
+from helpers import bf16_dev_to_f64, dev, f64, to_dev_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+def _full_size_case(oracle, name, theta, rows=48, score_rows=4096, seed=0):
+    w = synth.WORKLOADS[name]
+    inp = synth.make_step_inputs(w, seed)
+    B, N, H, d, D, N_sel, n_always = w.B, w.N, w.H, w.d, w.D, w.N_v, w.N_t
+    k_keep = w.k_of(theta)
+    M = k_keep + n_always
+    lse0 = (inp["lse"] - np.float32(math.log(N))).astype(np.float32)
+    x_cur, x_ref = to_dev_bf16(inp["x_cur"]), to_dev_bf16(inp["x_ref"])
+    q, k, v = (to_dev_bf16(inp[n]) for n in ("q", "k", "v"))
+    out, lse, n_skip = to_dev_bf16(inp["cache"]), dev(lse0), dev(inp["n_skip"])
+    score = torch.empty(B, N_sel, device="cuda")
+    idx_sel = torch.empty(B, M, dtype=torch.int32, device="cuda")
+    idx_rem = torch.empty(B, N_sel - k_keep, dtype=torch.int32, device="cuda")
+    ws = A.new_workspace(A.OP_STEP, B, H, N, M, d)
+    ws_sel = A.new_workspace(A.OP_SELECT, B, 0, N_sel, k_keep, 0)
+    s = A.bhnd_strides(N, H, d)
+    A.astraea_score(x_cur, x_ref, lse, n_skip, score, B, N, N_sel, D, H, 1.0, 1.0)
+    A.astraea_select(score, B, N_sel, k_keep, n_always, idx_sel, idx_rem, n_skip, ws_sel)
+    A.astraea_sparse_attn(q, k, v, s, s, s, idx_sel, M, out, lse, B, H, N, d, workspace=ws)
+    A.astraea_scatter_reuse(x_ref, x_cur, idx_sel, B, N, M, D, A.SCATTER_SRC_FULL)
+    A.astraea_poll_error(ws)
+
+    rng = np.random.default_rng(seed + 1)
+    # scores: a sample of tokens against the oracle (rows are independent)
+    got_score = score.cpu().numpy()
+    pick = np.sort(rng.choice(N_sel, min(score_rows, N_sel), replace=False))
+    full = np.concatenate([pick, np.arange(N_sel, N)])           # keep the [selectable | always] structure
+    want = oracle.score(f64(inp["x_cur"][:, full]), f64(inp["x_ref"][:, full]), lse0[:, :, full],
+                        inp["n_skip"][:, pick], n_sel=len(pick))
+    rel = np.abs(got_score[:, pick].astype(np.float64) - want) / np.abs(want)
+    assert rel.max() < 1e-5
+    # selection: bit-exact on the scores the device produced
+    want_sel, want_rem, want_n = oracle.select(got_score, k_keep, n_always, inp["n_skip"])
+    got_sel = idx_sel.cpu().numpy()
+    assert np.array_equal(got_sel, want_sel)
+    assert np.array_equal(idx_rem.cpu().numpy(), want_rem)
+    assert np.array_equal(n_skip.cpu().numpy(), want_n)
+    # attention: sampled selected rows, a few heads, all keys
+    heads = sorted({0, H // 2, H - 1})
+    r = min(rows, M)
+    rows_pick = np.stack([np.sort(rng.choice(got_sel[b], r, replace=False)) for b in range(B)]).astype(np.int32)
+    qh, kh, vh = (f64(np.ascontiguousarray(inp[n][:, :, heads])) for n in ("q", "k", "v"))
+    want_o, want_l, _ = oracle.sparse_attn(qh, kh, vh, q_idx=rows_pick)
+    got_out = out[:, :, heads].float().cpu().numpy().astype(np.float64)
+    got_rows = np.take_along_axis(got_out, rows_pick[:, :, None, None].astype(np.int64), 1)
+    err = np.abs(got_rows - want_o) / np.maximum(1.0, np.abs(want_o))
+    assert err.max() < 2e-2 and err.mean() < 2e-3, (err.max(), err.mean())
+    got_l = np.take_along_axis(lse[:, heads].cpu().numpy().astype(np.float64), rows_pick[:, None, :].astype(np.int64), 2)
+    assert np.abs(got_l - want_l).max() < 1e-3
+    # reuse: unselected rows keep the cache bit for bit; the LSE cache too; x_ref refreshed only where selected
+    unsel = torch.ones(B, N, dtype=torch.bool, device="cuda")
+    for b in range(B):
+        unsel[b, idx_sel[b].long()] = False
+    cache = to_dev_bf16(inp["cache"])
+    assert torch.equal(out[unsel], cache[unsel])
+    assert torch.equal(lse.transpose(1, 2)[unsel], dev(lse0).transpose(1, 2)[unsel])
+    x_ref0 = to_dev_bf16(inp["x_ref"])
+    assert torch.equal(x_ref[unsel], x_ref0[unsel]) and torch.equal(x_ref[~unsel], x_cur[~unsel])
+
+
+@pytest.mark.parametrize("theta", [500, 250])
+def test_cogvideox_shaped_full_size(oracle, theta):
+    _full_size_case(oracle, "cogvideox", theta)
+
+
+def test_opensora_shaped_full_size(oracle):
+    _full_size_case(oracle, "opensora", 400)
+
+
+def test_sweep_shaped_full_size(oracle):
+    _full_size_case(oracle, "sweep", 300, rows=32)
+
+
+def test_hunyuan_shaped_full_size(oracle):
+    _full_size_case(oracle, "hunyuan", 600, rows=24, score_rows=2048)
