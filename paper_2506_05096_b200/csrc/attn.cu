@@ -41,7 +41,6 @@ using namespace ptx;
 constexpr int kBlockM = 128;                     // rows of one query tile
 constexpr int kTilesM = 2;                       // query tiles per CTA
 constexpr int kBlockN = 64;                      // keys per K/V tile
-constexpr int kThreads = 384;
 constexpr uint32_t kTmemCols = 512;
 constexpr float kTileSumLimit = 65536.0f;        // a tile's sum of exponentials above this forces an exact maximum
 constexpr uint64_t kWaitLimitNs = 1000000000ull; // bounded waits: one second
@@ -53,15 +52,21 @@ template <int DH> struct Cfg {
     static constexpr int kTail = DH - kMain;
     static constexpr int kTailPad = kTail ? 16 : 0;
     static_assert(kTail == 0 || kTail == 8, "head_dim must be 64, 72 or 128");
-    static constexpr int kSBufs = (DH == 64) ? 3 : 2;             // S buffers per query tile
+    // softmax warpgroups per query tile: at head_dim 64 even key tiles go to one and odd ones to the other,
+    // each with its own running reference, row sum and O accumulator (merged in the epilogue)
+    static constexpr int kSplit = (DH == 64) ? 2 : 1;
+    static constexpr int kSBufs = 2;                              // S buffers per query tile
+    static constexpr int kSoftmaxWarps = 4 * kTilesM * kSplit;
+    static constexpr int kThreads = (kSoftmaxWarps + 4) * 32;     // + producer, issuer and two register donors
     static constexpr uint32_t kColO = kTilesM * kSBufs * kBlockN; // first O column
-    static constexpr uint32_t kOStride = (DH == 64) ? 64 : 128;
-    static_assert(kColO + kTilesM * kOStride <= kTmemCols && kMain + kTailPad <= (int)kOStride, "TMEM budget");
+    static constexpr uint32_t kOStride = (DH == 64) ? 64 : 128;   // columns between O accumulators
+    static_assert(kColO + kTilesM * kSplit * kOStride <= kTmemCols && kMain + kTailPad <= (int)kOStride, "TMEM budget");
+    static_assert(kSplit == 1 || kSplit == kSBufs, "a split warpgroup owns one S buffer");
     // setmaxnreg only redistributes what the CTA got at launch: an increase that the decreases of
     // the last warpgroup cannot cover would block forever
     static constexpr int kRegsLaunch = (65536 / kThreads) / 8 * 8;
-    static constexpr int kRegsSoftmax = 232, kRegsOther = 40;
-    static_assert(kRegsSoftmax * 256 + kRegsOther * 128 <= kRegsLaunch * kThreads, "setmaxnreg budget");
+    static constexpr int kRegsSoftmax = (kSplit == 2) ? 112 : 232, kRegsOther = (kSplit == 2) ? 32 : 40;
+    static_assert(kRegsSoftmax * kSoftmaxWarps * 32 + kRegsOther * 128 <= kRegsLaunch * kThreads, "setmaxnreg budget");
     static constexpr int kChunks = kMain / 64;                    // 64-column (128-byte) swizzle chunks
     static constexpr int kQChunkBytes = kBlockM * 128;            // 128 query rows x 128 bytes
     static constexpr int kQTailBytes = kTail ? kBlockM * 32 : 0;  // 128 query rows x 32 bytes
@@ -202,42 +207,46 @@ __device__ __forceinline__ void publish_p(uint32_t bar) {
     mbar_arrive(bar);
 }
 
-// One key tile of the online softmax.
+// One key tile of the online softmax.  `first`: this warpgroup's first tile.
 template <int DH>
-__device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j)
+__device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j, bool first)
 {
-    constexpr int kSBufs = Cfg<DH>::kSBufs;
+    using C = Cfg<DH>;
+    constexpr int kSBufs = C::kSBufs;
     const int buf = j % kSBufs;
     const uint32_t t_s = st.t_s0 + buf * kBlockN;
     const float sl2 = st.sl2;
     float cur[kBlockN];
-    // S of this tile has been in TMEM for a while (kSBufs buffers); the load is waited for at once:
-    // registers of a tcgen05.ld in flight must not be touched, and the compiler cannot know that
+    // the load is waited for at once: registers of a tcgen05.ld in flight must not be touched, and the
+    // compiler cannot know that
     wait_bar(st.bar_s + 8 * buf, (j / kSBufs) & 1, st.abort_flag, st.err_word);
     tc_fence_after();
     load_s(t_s, cur);
     wait_s_regs(cur);
     mask_tail(cur, st.N - j * kBlockN);
-    if (j == 0) st.m_ref = row_max(cur);          // the reference starts as the exact maximum of the first key tile
+    if (first) st.m_ref = row_max(cur);           // the reference starts as the exact maximum of the first key tile
     float neg = -st.m_ref * sl2;
-    float e[kBlockN];
 #pragma unroll
-    for (int i = 0; i < kBlockN; ++i) e[i] = ex2(fmaf(cur[i], sl2, neg));
-    float tile_sum = row_sum(e);
+    for (int i = 0; i < kBlockN; ++i) cur[i] = ex2(fmaf(cur[i], sl2, neg));
+    float tile_sum = row_sum(cur);
     if (__any_sync(0xffffffffu, !(tile_sum <= kTileSumLimit))) {
-        // rare: the reference maximum is too low for this tile: take the exact maximum, rescale what
-        // has been accumulated, and redo the tile
+        // rare: the reference maximum is too low for this tile.  S is still intact in TMEM (P is not stored
+        // yet): take the exact maximum, rescale what has been accumulated, and redo the tile
+        load_s(t_s, cur);
+        wait_s_regs(cur);
+        mask_tail(cur, st.N - j * kBlockN);
         const float mx = row_max(cur);
         float alpha = 1.0f;
         if (mx > st.m_ref) { alpha = ex2((st.m_ref - mx) * sl2); st.m_ref = mx; st.l_sum *= alpha; }
-        if (j > 0) {
-            // P V of the previous key tile has landed.  The o barrier of a buffer cannot be a whole phase
-            // behind: S of this tile was seen, so every MMA issued before its Q K^T is complete, and
-            // that includes the P V that last used the previous tile's buffer.
-            wait_bar(st.bar_o + 8 * ((j - 1) % kSBufs), ((j - 1) / kSBufs) & 1, st.abort_flag, st.err_word);
+        if (!first) {
+            // P V of this accumulator's previous key tile has landed.  Its o barrier cannot be a whole phase
+            // behind: S of this tile was seen, so every MMA issued before its Q K^T is complete, and that
+            // includes the P V that last used the previous tile's buffer.
+            const int jp = j - C::kSplit;
+            wait_bar(st.bar_o + 8 * (jp % kSBufs), (jp / kSBufs) & 1, st.abort_flag, st.err_word);
             tc_fence_after();
 #pragma unroll
-            for (int cc = 0; cc < Cfg<DH>::kMain / 32; ++cc) {
+            for (int cc = 0; cc < C::kMain / 32; ++cc) {
                 uint32_t o[32];
                 tmem_ld32(st.t_o + cc * 32, o);
                 tc_wait_ld();
@@ -245,44 +254,45 @@ __device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j)
                 for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
                 tmem_st32(st.t_o + cc * 32, o);
             }
-            if (Cfg<DH>::kTail) {
+            if (C::kTail) {
                 uint32_t o[16];
-                tmem_ld16(st.t_o + Cfg<DH>::kMain, o);
+                tmem_ld16(st.t_o + C::kMain, o);
                 tc_wait_ld();
 #pragma unroll
                 for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                tmem_st16(st.t_o + Cfg<DH>::kMain, o);
+                tmem_st16(st.t_o + C::kMain, o);
             }
             tc_wait_st();
         }
         neg = -st.m_ref * sl2;
 #pragma unroll
-        for (int i = 0; i < kBlockN; ++i) e[i] = ex2(fmaf(cur[i], sl2, neg));
-        tile_sum = row_sum(e);
+        for (int i = 0; i < kBlockN; ++i) cur[i] = ex2(fmaf(cur[i], sl2, neg));
+        tile_sum = row_sum(cur);
     }
     st.l_sum += tile_sum;
     // P as bf16 pairs (element 2c in the low half) over the first 32 columns of this S buffer
     uint32_t pk[32];
 #pragma unroll
     for (int i = 0; i < 32; ++i) {
-        __nv_bfloat162 v2 = __floats2bfloat162_rn(e[2 * i], e[2 * i + 1]);
+        __nv_bfloat162 v2 = __floats2bfloat162_rn(cur[2 * i], cur[2 * i + 1]);
         pk[i] = *reinterpret_cast<uint32_t *>(&v2);
     }
     tmem_st32(t_s, pk);
     publish_p(st.bar_p + 8 * buf);
 }
 
-// ---------------------------------------------------------------- softmax warpgroup (one query tile)
+// ---------------------------------------------------------------- softmax warpgroup
+// tile: its query tile; par: which key tiles it takes (j = par, par + kSplit, ...)
 template <int DH>
-__device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, int tile, uint8_t *sQ_gen, uint32_t tmem,
-                                             int m_base, int h, int b, int n_tiles, volatile int *abort_flag)
+__device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, int tile, int par, uint8_t *sQ_gen, uint32_t tmem,
+                                             int m_base, int h, int b, int n_tiles, volatile int *abort_flag, float2 *xchg)
 {
     using C = Cfg<DH>;
     const int wtid = threadIdx.x & 127;
     const int warp = __shfl_sync(0xffffffffu, wtid >> 5, 0);       // warp-uniform
     // gather this tile's Q rows (swizzled, K-major): 16-byte units, unit c of row r
     constexpr int kMainUnits = C::kMain / 8, kUnits = kMainUnits + (C::kTail ? 2 : 0);
-    for (int v = wtid; v < kBlockM * kUnits; v += 128) {
+    for (int v = par * 128 + wtid; v < kBlockM * kUnits; v += 128 * C::kSplit) {     // the warpgroups of a tile share the rows
         const int r = v / kUnits, c = v - r * kUnits;
         const int m = m_base + r;
         uint4 val = make_uint4(0, 0, 0, 0);
@@ -306,7 +316,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     st.sl2 = p.scale_log2;
     st.l_sum = 0.f;
     st.t_s0 = t_row + tile * C::kSBufs * kBlockN;
-    st.t_o = t_row + C::kColO + tile * C::kOStride;
+    st.t_o = t_row + C::kColO + (tile * C::kSplit + par) * C::kOStride;
     st.bar_s = bar.s + 32 * tile; st.bar_p = bar.p + 32 * tile; st.bar_o = bar.o + 32 * tile;
     st.N = p.N; st.n_tiles = n_tiles; st.abort_flag = abort_flag; st.err_word = p.err_word;
 
@@ -314,23 +324,46 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     int tok = -1;
     if (m < p.M) {
         tok = p.q_idx ? __ldg(p.q_idx + (size_t)b * p.M + m) : m;
-        if ((unsigned)tok >= (unsigned)p.N) { atomicExch(p.err_word, kErrBadIndex); tok = -1; }
+        if ((unsigned)tok >= (unsigned)p.N) { if (par == 0) atomicExch(p.err_word, kErrBadIndex); tok = -1; }
     }
 
     st.m_ref = -INFINITY;
-    for (int j = 0; j < n_tiles; ++j) softmax_step<DH>(st, j);
+    int j_last = -1;
+    for (int j = par; j < n_tiles; j += C::kSplit) { softmax_step<DH>(st, j, j == par); j_last = j; }
 
-    // ------------------------------------------------ epilogue: normalise and scatter
-    wait_bar(st.bar_o + 8 * ((n_tiles - 1) % C::kSBufs), ((n_tiles - 1) / C::kSBufs) & 1, abort_flag, p.err_word);
+    // ------------------------------------------------ epilogue: (merge,) normalise and scatter
+    if (j_last >= 0) wait_bar(st.bar_o + 8 * (j_last % C::kSBufs), (j_last / C::kSBufs) & 1, abort_flag, p.err_word);
     tc_fence_after();
-    const float inv_l = 1.0f / st.l_sum;
+    float w_own = 1.0f, w_other = 0.f, l_sum = st.l_sum, m_ref = st.m_ref;
+    uint32_t t_other = st.t_o;
+    if constexpr (C::kSplit == 2) {
+        // the odd-tile warpgroup hands its reference and row sum to the even-tile one, which merges both accumulators
+        if (par == 1) xchg[wtid] = make_float2(st.m_ref, j_last >= 0 ? st.l_sum : 0.f);
+        tc_fence_before();
+        if (tile == 0) asm volatile("bar.sync 1, 256;" ::: "memory");
+        else asm volatile("bar.sync 2, 256;" ::: "memory");
+        if (par == 1) return;
+        tc_fence_after();
+        const float2 other = xchg[wtid];
+        if (other.y > 0.f) {
+            m_ref = fmaxf(st.m_ref, other.x);
+            w_own = ex2((st.m_ref - m_ref) * st.sl2);
+            w_other = ex2((other.x - m_ref) * st.sl2);
+            l_sum = st.l_sum * w_own + other.y * w_other;
+            t_other = t_row + C::kColO + (tile * C::kSplit + 1) * C::kOStride;
+        }
+    }
+    const bool merge = C::kSplit == 2 && __any_sync(0xffffffffu, w_other != 0.f);   // warp-uniform: the partner has tiles or not
+    const float inv_l = 1.0f / l_sum;
+    w_own *= inv_l;
+    w_other *= inv_l;
     __nv_bfloat16 *dst = nullptr;
     if (tok >= 0 && !*abort_flag) {
         const size_t orow = p.compact ? ((size_t)b * p.M + m) : ((size_t)b * p.N + tok);
         dst = p.out + (orow * p.H + h) * DH;
         if (p.lse_out) {
             const size_t li = p.compact ? (((size_t)b * p.H + h) * p.M + m) : (((size_t)b * p.H + h) * p.N + tok);
-            p.lse_out[li] = st.m_ref * p.scale + logf(st.l_sum);
+            p.lse_out[li] = m_ref * p.scale + logf(l_sum);
         }
     }
 #pragma unroll
@@ -338,14 +371,22 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
         uint32_t o[32];
         tmem_ld32(st.t_o + cc * 32, o);
         tc_wait_ld();
+        float f[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(o[i]) * w_own;
+        if (merge) {
+            tmem_ld32(t_other + cc * 32, o);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) f[i] = fmaf(__uint_as_float(o[i]), w_other, f[i]);
+        }
         if (dst) {
 #pragma unroll
             for (int v = 0; v < 4; ++v) {
                 uint32_t w[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(o[v * 8 + 2 * i]) * inv_l,
-                                                              __uint_as_float(o[v * 8 + 2 * i + 1]) * inv_l);
+                    __nv_bfloat162 v2 = __floats2bfloat162_rn(f[v * 8 + 2 * i], f[v * 8 + 2 * i + 1]);
                     w[i] = *reinterpret_cast<uint32_t *>(&v2);
                 }
                 *reinterpret_cast<uint4 *>(dst + cc * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -358,7 +399,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
         tc_wait_ld();
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(o[2 * i]) * inv_l, __uint_as_float(o[2 * i + 1]) * inv_l);
+            __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(o[2 * i]) * w_own, __uint_as_float(o[2 * i + 1]) * w_own);
             w[i] = *reinterpret_cast<uint32_t *>(&v2);
         }
         if (dst) *reinterpret_cast<uint4 *>(dst + C::kMain) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -366,7 +407,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
 }
 
 template <int DH>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(Cfg<DH>::kThreads, 1)
 sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                    const __grid_constant__ CUtensorMap tmap_k_tail, const __grid_constant__ CUtensorMap tmap_v_tail, const Params p)
 {
@@ -375,6 +416,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    __shared__ float2 xchg[kTilesM][kBlockM];
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -398,7 +440,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     if (tid == 0) {
         abort_flag = 0;
         for (int t = 0; t < kTilesM; ++t) {
-            mbar_init(bar.q + 8 * t, 128);
+            mbar_init(bar.q + 8 * t, 128 * C::kSplit);
             for (int u = 0; u < 4; ++u) {
                 mbar_init(bar.s + 32 * t + 8 * u, 1); mbar_init(bar.p + 32 * t + 8 * u, 128); mbar_init(bar.o + 32 * t + 8 * u, 1);
             }
@@ -407,7 +449,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         for (int s = 0; s < C::kStagesV; ++s) { mbar_init(bar.vf + 8 * s, 1); mbar_init(bar.ve + 8 * s, 1); }
         fence_barrier_init();
     }
-    if (warp == 9) {
+    constexpr int kProducerWarp = C::kSoftmaxWarps, kIssuerWarp = C::kSoftmaxWarps + 1;
+    if (warp == kIssuerWarp) {
         tmem_alloc(smem_u32(&tmem_slot), kTmemCols);
         tmem_relinquish();
     }
@@ -416,11 +459,13 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
 
-    if (warp < 8) {
+    if (warp < C::kSoftmaxWarps) {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(C::kRegsSoftmax));
-        const int tile = warp >> 2;
-        softmax_role<DH>(p, bar, tile, smem_gen + tile * C::kQTileBytes, tmem, m0 + tile * kBlockM, h, b, n_tiles, &abort_flag);
-    } else if (warp == 8) {
+        const int wg = warp >> 2;
+        const int tile = wg / C::kSplit, par = wg % C::kSplit;
+        softmax_role<DH>(p, bar, tile, par, smem_gen + tile * C::kQTileBytes, tmem, m0 + tile * kBlockM, h, b, n_tiles,
+                         &abort_flag, xchg[tile]);
+    } else if (warp == kProducerWarp) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
         // ------------------------------------------------ TMA producer (warp-uniform, one elected lane issues)
         if (elect_one()) {
@@ -464,7 +509,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             wait_bar(bar.kf + 8 * (j % C::kStagesK), (j / C::kStagesK) & 1, &abort_flag, p.err_word);
         for (int j = (n_tiles > C::kStagesV ? n_tiles - C::kStagesV : 0); j < n_tiles; ++j)
             wait_bar(bar.vf + 8 * (j % C::kStagesV), (j / C::kStagesV) & 1, &abort_flag, p.err_word);
-    } else if (warp == 9) {
+    } else if (warp == kIssuerWarp) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
         // ------------------------------------------------ MMA issuer (warp-uniform, one elected lane issues)
         constexpr uint32_t idesc_qk = idesc_bf16(kBlockM, kBlockN, false);
@@ -510,16 +555,17 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             for (int t = 0; t < kTilesM; ++t) {
                 wait_bar(bar.p + 32 * t + 8 * u, (j / kSBufs) & 1, &abort_flag, p.err_word);
                 tc_fence_after();
+                const uint32_t o_col = C::kColO + (t * C::kSplit + (j % C::kSplit)) * C::kOStride;   // this tile's accumulator
                 if (elect_one()) {
 #pragma unroll
                     for (int ks = 0; ks < kBlockN / 16; ++ks) {
-                        mma_ts(tmem + C::kColO + t * C::kOStride, tmem + (t * kSBufs + u) * kBlockN + ks * 8,
+                        mma_ts(tmem + o_col, tmem + (t * kSBufs + u) * kBlockN + ks * 8,
                                smem_desc(vbase + ks * 2048, C::kChunkBytes, 1024, kSwizzle128B),
-                               idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+                               idesc_pv, (j >= C::kSplit || ks > 0) ? 1u : 0u);
                         if (C::kTail)  // O columns 64..79 from the 16-column chunk of V
-                            mma_ts(tmem + C::kColO + t * C::kOStride + C::kMain, tmem + (t * kSBufs + u) * kBlockN + ks * 8,
+                            mma_ts(tmem + o_col + C::kMain, tmem + (t * kSBufs + u) * kBlockN + ks * 8,
                                    smem_desc(vbase + C::kChunks * C::kChunkBytes + ks * 512, 256, 256, kSwizzle32B),
-                                   idesc_pv_tail, (j > 0 || ks > 0) ? 1u : 0u);
+                                   idesc_pv_tail, (j >= C::kSplit || ks > 0) ? 1u : 0u);
                     }
                     tc_commit(bar.o + 32 * t + 8 * u);
                     if (t == kTilesM - 1) tc_commit(bar.ve + 8 * sv);
@@ -538,7 +584,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 9) tmem_dealloc(tmem, kTmemCols);
+    if (warp == kIssuerWarp) tmem_dealloc(tmem, kTmemCols);
 }
 
 // ------------------------------------------------------------------ host side
@@ -610,7 +656,7 @@ int32_t launch_dh(const AttnArgs &a, cudaStream_t stream)
     p.compact = (a.flags & ASTRAEA_ATTN_COMPACT_OUT) ? 1 : 0;
     p.err_word = a.err_word;
     dim3 grid((a.M + kTilesM * kBlockM - 1) / (kTilesM * kBlockM), a.H, a.B);
-    sparse_attn_kernel<DH><<<grid, kThreads, C::kSmemBytes, stream>>>(mk, mv, mkt, mvt, p);
+    sparse_attn_kernel<DH><<<grid, C::kThreads, C::kSmemBytes, stream>>>(mk, mv, mkt, mvt, p);
     return check_launch("astraea_sparse_attn");
 }
 
