@@ -436,6 +436,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);        // warp-uniform
     const int m0 = blockIdx.x * (kTilesM * kBlockM), h = blockIdx.y, b = blockIdx.z;
     const int n_tiles = (p.N + kBlockN - 1) / kBlockN;
+    // the last CTA of a head may have rows in its first query tile only: the second tile's warps and MMAs are skipped
+    const int q_tiles = (m0 + kBlockM < p.M) ? kTilesM : 1;
 
     if (tid == 0) {
         abort_flag = 0;
@@ -463,8 +465,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(C::kRegsSoftmax));
         const int wg = warp >> 2;
         const int tile = wg / C::kSplit, par = wg % C::kSplit;
-        softmax_role<DH>(p, bar, tile, par, smem_gen + tile * C::kQTileBytes, tmem, m0 + tile * kBlockM, h, b, n_tiles,
-                         &abort_flag, xchg[tile]);
+        if (tile < q_tiles)
+            softmax_role<DH>(p, bar, tile, par, smem_gen + tile * C::kQTileBytes, tmem, m0 + tile * kBlockM, h, b, n_tiles,
+                             &abort_flag, xchg[tile]);
     } else if (warp == kProducerWarp) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
         // ------------------------------------------------ TMA producer (warp-uniform, one elected lane issues)
@@ -531,14 +534,14 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         };
         // prologue: S of the first kSBufs key tiles for both query tiles
         wait_bar(bar.q, 0, &abort_flag, p.err_word);
-        wait_bar(bar.q + 8, 0, &abort_flag, p.err_word);
+        if (q_tiles > 1) wait_bar(bar.q + 8, 0, &abort_flag, p.err_word);
         for (int j = 0; j < kSBufs && j < n_tiles; ++j) {
             const int st = j % C::kStagesK;
             wait_bar(bar.kf + 8 * st, (j / C::kStagesK) & 1, &abort_flag, p.err_word);
             tc_fence_after();
             if (elect_one()) {
                 issue_qk(0, j, sK + st * C::kTileBytes);
-                issue_qk(1, j, sK + st * C::kTileBytes);
+                if (q_tiles > 1) issue_qk(1, j, sK + st * C::kTileBytes);
                 tc_commit(bar.ke + 8 * st);
             }
             __syncwarp();
@@ -553,6 +556,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             if (more) wait_bar(bar.kf + 8 * sk, ((j + kSBufs) / C::kStagesK) & 1, &abort_flag, p.err_word);
 #pragma unroll
             for (int t = 0; t < kTilesM; ++t) {
+                if (t >= q_tiles) break;
                 wait_bar(bar.p + 32 * t + 8 * u, (j / kSBufs) & 1, &abort_flag, p.err_word);
                 tc_fence_after();
                 const uint32_t o_col = C::kColO + (t * C::kSplit + (j % C::kSplit)) * C::kOStride;   // this tile's accumulator
@@ -568,11 +572,11 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                                    idesc_pv_tail, (j >= C::kSplit || ks > 0) ? 1u : 0u);
                     }
                     tc_commit(bar.o + 32 * t + 8 * u);
-                    if (t == kTilesM - 1) tc_commit(bar.ve + 8 * sv);
+                    if (t == q_tiles - 1) tc_commit(bar.ve + 8 * sv);
                     // the S buffer just consumed as P is free again (in-order pipe): refill it with key tile j+kSBufs
                     if (more) {
                         issue_qk(t, j + kSBufs, sK + sk * C::kTileBytes);
-                        if (t == kTilesM - 1) tc_commit(bar.ke + 8 * sk);
+                        if (t == q_tiles - 1) tc_commit(bar.ke + 8 * sk);
                     }
                 }
                 __syncwarp();
