@@ -3,17 +3,21 @@
 // Section 3.2 "Sparse Attention").
 //
 // One CTA per (256 selected queries, head, batch): two 128-row query tiles that share every
-// K/V tile of 64 keys.  Warp roles (384 threads):
-//   warps 0-3 / 4-7  softmax of query tile 0 / 1 (one thread per query row): gather the tile's Q rows
-//              into 128B-swizzled shared memory, then per key tile read S from TMEM, exponentiate
-//              in the log2 domain against a running reference maximum, write P (bf16) back to TMEM
-//              over S, and at the end normalise O and scatter it to the rows q_idx names;
-//   warp 8     TMA producer: K and V tiles into multi-stage swizzled buffers;
-//   warp 9     tcgen05.mma issuer: S = Q K^T (SS, K-major operands), O += P V (P from TMEM,
-//              V as an MN-major shared-memory operand); owns the TMEM allocation;
-//   warps 10-11 only donate registers (setmaxnreg moves them to the softmax warps).
-// S has kSBufs buffers per query tile; a buffer is refilled with key tile j+kSBufs as soon as P of
-// tile j has been consumed, so S of the next tiles is in TMEM while the softmax of tile j runs.
+// K/V tile of 64 keys.  Warp roles:
+//   softmax warpgroups (one thread per query row): gather the tile's Q rows into 128B-swizzled shared
+//              memory, then per key tile read S from TMEM, exponentiate in the log2 domain against a
+//              running reference maximum, write P (bf16) back to TMEM over S, and at the end normalise
+//              O and scatter it to the rows q_idx names.  head_dim 72 / 128: one warpgroup per query
+//              tile.  head_dim 64: two per query tile; even key tiles go to one and odd ones to the
+//              other, each with its own reference, row sum and O accumulator (a split over keys inside
+//              the CTA, merged in the epilogue), which puts four softmax warps on every SM sub-partition
+//              and hides the serial chain of a key tile (wait, load, exponentials, sum, pack, publish);
+//   one warp   TMA producer: K and V tiles into multi-stage swizzled buffers;
+//   two warps  tcgen05.mma issuers, one per query tile: S = Q K^T (SS, K-major operands), O += P V (P from
+//              TMEM, V as an MN-major shared-memory operand); the first owns the TMEM allocation;
+//   one warp   only donates registers (setmaxnreg moves registers to the softmax warps).
+// Every query tile has two S buffers; a buffer is refilled with key tile j+2 as soon as P of tile j has
+// been consumed (the tensor pipe executes one thread's MMAs in order).
 //
 // The softmax is bound by the exponentials (XU pipe, 16 per clock per SM) and by the latencies of
 // its own chain, so the common path of a key tile is kept to: load S, one FFMA + ex2 per element,
@@ -23,7 +27,7 @@
 // normalisation cancels; fp32 has the range).  Otherwise the exact maximum is taken and the row
 // sum and the O accumulator are rescaled before the tile is redone.
 //
-// TMEM columns: S/P of (tile t, buffer u) at (t*kSBufs+u)*64; O of tile t behind them.
+// TMEM columns: S/P of (tile t, buffer u) at (2t+u)*64; the O accumulators from column 256.
 // The producer and issuer warps run warp-uniform code and elect one lane per instruction, so
 // that descriptors and addresses stay in uniform registers (a lone diverged thread issues
 // tcgen05.mma several times slower).  Every mbarrier wait is bounded; on a timeout the CTA raises
@@ -57,7 +61,7 @@ template <int DH> struct Cfg {
     static constexpr int kSplit = (DH == 64) ? 2 : 1;
     static constexpr int kSBufs = 2;                              // S buffers per query tile
     static constexpr int kSoftmaxWarps = 4 * kTilesM * kSplit;
-    static constexpr int kThreads = (kSoftmaxWarps + 4) * 32;     // + producer, issuer and two register donors
+    static constexpr int kThreads = (kSoftmaxWarps + 4) * 32;     // + producer, two issuers, one register donor
     static constexpr uint32_t kColO = kTilesM * kSBufs * kBlockN; // first O column
     static constexpr uint32_t kOStride = (DH == 64) ? 64 : 128;   // columns between O accumulators
     static_assert(kColO + kTilesM * kSplit * kOStride <= kTmemCols && kMain + kTailPad <= (int)kOStride, "TMEM budget");
@@ -447,8 +451,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                 mbar_init(bar.s + 32 * t + 8 * u, 1); mbar_init(bar.p + 32 * t + 8 * u, 128); mbar_init(bar.o + 32 * t + 8 * u, 1);
             }
         }
-        for (int s = 0; s < C::kStagesK; ++s) { mbar_init(bar.kf + 8 * s, 1); mbar_init(bar.ke + 8 * s, 1); }
-        for (int s = 0; s < C::kStagesV; ++s) { mbar_init(bar.vf + 8 * s, 1); mbar_init(bar.ve + 8 * s, 1); }
+        // a K/V stage is free once the issuer of every active query tile has committed its MMAs on it
+        for (int s = 0; s < C::kStagesK; ++s) { mbar_init(bar.kf + 8 * s, 1); mbar_init(bar.ke + 8 * s, q_tiles); }
+        for (int s = 0; s < C::kStagesV; ++s) { mbar_init(bar.vf + 8 * s, 1); mbar_init(bar.ve + 8 * s, q_tiles); }
         fence_barrier_init();
     }
     constexpr int kProducerWarp = C::kSoftmaxWarps, kIssuerWarp = C::kSoftmaxWarps + 1;
@@ -512,7 +517,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             wait_bar(bar.kf + 8 * (j % C::kStagesK), (j / C::kStagesK) & 1, &abort_flag, p.err_word);
         for (int j = (n_tiles > C::kStagesV ? n_tiles - C::kStagesV : 0); j < n_tiles; ++j)
             wait_bar(bar.vf + 8 * (j % C::kStagesV), (j / C::kStagesV) & 1, &abort_flag, p.err_word);
-    } else if (warp == kIssuerWarp) {
+    } else if (warp == kIssuerWarp || warp == kIssuerWarp + 1) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
         // ------------------------------------------------ MMA issuer (warp-uniform, one elected lane issues)
         constexpr uint32_t idesc_qk = idesc_bf16(kBlockM, kBlockN, false);
@@ -532,34 +537,34 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                        smem_desc(kbase + C::kChunks * C::kChunkBytes, 16, 256, kSwizzle32B), idesc_qk, 1u);
             tc_commit(bar.s + 32 * t + 8 * u);
         };
-        // prologue: S of the first kSBufs key tiles for both query tiles
-        wait_bar(bar.q, 0, &abort_flag, p.err_word);
-        if (q_tiles > 1) wait_bar(bar.q + 8, 0, &abort_flag, p.err_word);
-        for (int j = 0; j < kSBufs && j < n_tiles; ++j) {
-            const int st = j % C::kStagesK;
-            wait_bar(bar.kf + 8 * st, (j / C::kStagesK) & 1, &abort_flag, p.err_word);
-            tc_fence_after();
-            if (elect_one()) {
-                issue_qk(0, j, sK + st * C::kTileBytes);
-                if (q_tiles > 1) issue_qk(1, j, sK + st * C::kTileBytes);
-                tc_commit(bar.ke + 8 * st);
+        // One issuer warp per query tile, on different SM sub-partitions: the tcgen05 instructions of a
+        // sub-partition's issuer slow the exponentials of the softmax warps that live there, so the load is spread.
+        // All MMAs that touch one S buffer / O accumulator come from one thread, in order.
+        const int t = warp - kIssuerWarp;
+        if (t < q_tiles) {
+            // prologue: S of the first kSBufs key tiles
+            wait_bar(bar.q + 8 * t, 0, &abort_flag, p.err_word);
+            for (int j = 0; j < kSBufs && j < n_tiles; ++j) {
+                const int st = j % C::kStagesK;
+                wait_bar(bar.kf + 8 * st, (j / C::kStagesK) & 1, &abort_flag, p.err_word);
+                tc_fence_after();
+                if (elect_one()) {
+                    issue_qk(t, j, sK + st * C::kTileBytes);
+                    tc_commit(bar.ke + 8 * st);
+                }
+                __syncwarp();
             }
-            __syncwarp();
-        }
-        for (int j = 0; j < n_tiles; ++j) {
-            const int sv = j % C::kStagesV;
-            const uint32_t vbase = sV + sv * C::kTileBytes;
-            const int u = j % kSBufs;
-            const bool more = j + kSBufs < n_tiles;
-            const int sk = (j + kSBufs) % C::kStagesK;
-            wait_bar(bar.vf + 8 * sv, (j / C::kStagesV) & 1, &abort_flag, p.err_word);
-            if (more) wait_bar(bar.kf + 8 * sk, ((j + kSBufs) / C::kStagesK) & 1, &abort_flag, p.err_word);
-#pragma unroll
-            for (int t = 0; t < kTilesM; ++t) {
-                if (t >= q_tiles) break;
+            for (int j = 0; j < n_tiles; ++j) {
+                const int sv = j % C::kStagesV;
+                const uint32_t vbase = sV + sv * C::kTileBytes;
+                const int u = j % kSBufs;
+                const bool more = j + kSBufs < n_tiles;
+                const int sk = (j + kSBufs) % C::kStagesK;
+                const uint32_t o_col = C::kColO + (t * C::kSplit + (j % C::kSplit)) * C::kOStride;   // this tile's accumulator
+                wait_bar(bar.vf + 8 * sv, (j / C::kStagesV) & 1, &abort_flag, p.err_word);
+                if (more) wait_bar(bar.kf + 8 * sk, ((j + kSBufs) / C::kStagesK) & 1, &abort_flag, p.err_word);
                 wait_bar(bar.p + 32 * t + 8 * u, (j / kSBufs) & 1, &abort_flag, p.err_word);
                 tc_fence_after();
-                const uint32_t o_col = C::kColO + (t * C::kSplit + (j % C::kSplit)) * C::kOStride;   // this tile's accumulator
                 if (elect_one()) {
 #pragma unroll
                     for (int ks = 0; ks < kBlockN / 16; ++ks) {
@@ -572,11 +577,11 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                                    idesc_pv_tail, (j >= C::kSplit || ks > 0) ? 1u : 0u);
                     }
                     tc_commit(bar.o + 32 * t + 8 * u);
-                    if (t == q_tiles - 1) tc_commit(bar.ve + 8 * sv);
+                    tc_commit(bar.ve + 8 * sv);
                     // the S buffer just consumed as P is free again (in-order pipe): refill it with key tile j+kSBufs
                     if (more) {
                         issue_qk(t, j + kSBufs, sK + sk * C::kTileBytes);
-                        if (t == q_tiles - 1) tc_commit(bar.ke + 8 * sk);
+                        tc_commit(bar.ke + 8 * sk);
                     }
                 }
                 __syncwarp();
