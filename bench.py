@@ -150,7 +150,7 @@ def main():
     ap.add_argument("--theta", type=int, default=500, help="keep-ratio in permille")
     ap.add_argument("--ref-rows", type=int, default=256, help="sampled query rows per step of the reference arm")
     ap.add_argument("--ref-heads", type=int, default=8)
-    ap.add_argument("--cpu-rows", type=int, default=2048, help="sampled query rows of the cpu_baseline leg (all heads)")
+    ap.add_argument("--cpu-rows", type=int, default=1024, help="sampled query rows of the cpu_baseline leg (all heads)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
