@@ -112,6 +112,14 @@ def test_select_all_equal_and_special_values(oracle):
         _select_case(oracle, s, k)
 
 
+def test_select_rows_longer_than_a_cluster_holds(oracle):
+    """Rows above 131072 tokens take the one-CTA path that re-reads the row in every pass."""
+    s = np.random.default_rng(9).standard_normal((2, 140001)).astype(np.float32)
+    s[:, ::5] = 0.25                     # plenty of ties
+    for k in (0, 1, 70000, 140001):
+        _select_case(oracle, s, k, n_always=3)
+
+
 def test_select_always_kept_span_and_optional_outputs(oracle):
     s = synth.integer_scores(2, 700, 5, 9)
     _select_case(oracle, s, 300, n_always=26)
