@@ -366,3 +366,12 @@ def test_step_opensora_shaped_reduced(oracle):
 def test_step_chain_of_three_steps_d128(oracle):
     w = synth.Workload("mini-hy", B=1, H=2, d=128, N_v=8 * 12 * 20, N_t=0)
     _step_case(oracle, w, 3, 600, steps=3)
+
+
+def test_step_chain_of_fifty_steps_reduced_hunyuan_shape(oracle):
+    """The 50-step drifting-latent workload at a reduced shape (8x12x20 tokens, 2 heads, head_dim 128):
+    every step is checked against the oracle started from the device's state of the step before."""
+    w = synth.Workload("mini-hy-50", B=1, H=2, d=128, N_v=8 * 12 * 20, N_t=0)
+    _step_case(oracle, w, 5, 600, steps=50)
+    _step_case(oracle, w, 6, 300, steps=12)
+
