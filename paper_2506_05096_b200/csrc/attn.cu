@@ -44,7 +44,6 @@ using namespace ptx;
 
 constexpr int kBlockM = 128;                     // rows of one query tile
 constexpr int kTilesM = 2;                       // query tiles per CTA
-constexpr int kBlockN = 64;                      // keys per K/V tile
 constexpr uint32_t kTmemCols = 512;
 constexpr float kTileSumLimit = 65536.0f;        // a tile's sum of exponentials above this forces an exact maximum
 constexpr uint64_t kWaitLimitNs = 1000000000ull; // bounded waits: one second
@@ -58,12 +57,15 @@ template <int DH> struct Cfg {
     static_assert(kTail == 0 || kTail == 8, "head_dim must be 64, 72 or 128");
     // softmax warpgroups per query tile: at head_dim 64 even key tiles go to one and odd ones to the other,
     // each with its own running reference, row sum and O accumulator (merged in the epilogue)
-    static constexpr int kSplit = (DH == 64) ? 2 : 1;
+    static constexpr int kSplit = (DH == 128) ? 1 : 2;
+    // keys per K/V tile = columns of an S buffer.  64, but 48 at head_dim 72: four O accumulators of 80 columns
+    // leave 192 TMEM columns for the four S buffers
+    static constexpr int kBlockN = (DH == 72) ? 48 : 64;
     static constexpr int kSBufs = 2;                              // S buffers per query tile
     static constexpr int kSoftmaxWarps = 4 * kTilesM * kSplit;
     static constexpr int kThreads = (kSoftmaxWarps + 4) * 32;     // + producer, two issuers, one register donor
     static constexpr uint32_t kColO = kTilesM * kSBufs * kBlockN; // first O column
-    static constexpr uint32_t kOStride = (DH == 64) ? 64 : 128;   // columns between O accumulators
+    static constexpr uint32_t kOStride = (DH == 64) ? 64 : (DH == 72) ? 80 : 128;   // columns between O accumulators
     static_assert(kColO + kTilesM * kSplit * kOStride <= kTmemCols && kMain + kTailPad <= (int)kOStride, "TMEM budget");
     static_assert(kSplit == 1 || kSplit == kSBufs, "a split warpgroup owns one S buffer");
     // setmaxnreg only redistributes what the CTA got at launch: an increase that the decreases of
@@ -75,9 +77,10 @@ template <int DH> struct Cfg {
     static constexpr int kQChunkBytes = kBlockM * 128;            // 128 query rows x 128 bytes
     static constexpr int kQTailBytes = kTail ? kBlockM * 32 : 0;  // 128 query rows x 32 bytes
     static constexpr int kQTileBytes = kChunks * kQChunkBytes + kQTailBytes;
-    static constexpr int kChunkBytes = kBlockN * 128;             // 64 keys x 128 bytes
-    static constexpr int kTailBytes = kTail ? kBlockN * 32 : 0;   // 64 keys x 32 bytes
-    static constexpr int kTileBytes = kChunks * kChunkBytes + kTailBytes;   // one K or V tile
+    static constexpr int kChunkBytes = kBlockN * 128;             // one key tile x 128 bytes
+    static constexpr int kTailBytes = kTail ? kBlockN * 32 : 0;   // one key tile x 32 bytes
+    static constexpr int kLoadBytes = kChunks * kChunkBytes + kTailBytes;   // what TMA delivers per K or V tile
+    static constexpr int kTileBytes = (kLoadBytes + 1023) / 1024 * 1024;    // stage size (keeps the swizzle alignment)
     static_assert(kQTileBytes % 1024 == 0 && kTileBytes % 1024 == 0, "tiles keep the 1024-byte swizzle alignment");
     static constexpr int kStagesK = (DH == 128) ? 5 : 6;
     static constexpr int kStagesV = (DH == 128) ? 5 : 6;
@@ -150,58 +153,72 @@ template <int DH> struct SoftmaxState {
     int *err_word;
 };
 
-// 64 columns of one S buffer into registers (asynchronous: wait_s_regs before using them)
-__device__ __forceinline__ void load_s(uint32_t t_s, float (&s)[kBlockN]) {
+// NS (48 or 64) columns of one S buffer into registers (asynchronous: wait_s_regs before using them)
+template <int NS>
+__device__ __forceinline__ void load_s(uint32_t t_s, float (&s)[NS]) {
     tmem_ld32(t_s, reinterpret_cast<uint32_t (&)[32]>(s[0]));
-    tmem_ld32(t_s + 32, reinterpret_cast<uint32_t (&)[32]>(s[32]));
+    if constexpr (NS == 64) tmem_ld32(t_s + 32, reinterpret_cast<uint32_t (&)[32]>(s[32]));
+    else tmem_ld16(t_s + 32, reinterpret_cast<uint32_t (&)[16]>(s[32]));
 }
 // tcgen05.wait::ld that names the loaded registers, so that no use of them can move above it
-__device__ __forceinline__ void wait_s_regs(float (&s)[kBlockN]) {
+__device__ __forceinline__ void wait_regs16(float *s) {
     asm volatile("tcgen05.wait::ld.sync.aligned;"
         : "+f"(s[0]), "+f"(s[1]), "+f"(s[2]), "+f"(s[3]), "+f"(s[4]), "+f"(s[5]), "+f"(s[6]), "+f"(s[7]),
-          "+f"(s[8]), "+f"(s[9]), "+f"(s[10]), "+f"(s[11]), "+f"(s[12]), "+f"(s[13]), "+f"(s[14]), "+f"(s[15]),
-          "+f"(s[16]), "+f"(s[17]), "+f"(s[18]), "+f"(s[19]), "+f"(s[20]), "+f"(s[21]), "+f"(s[22]), "+f"(s[23]),
-          "+f"(s[24]), "+f"(s[25]), "+f"(s[26]), "+f"(s[27]), "+f"(s[28]), "+f"(s[29]), "+f"(s[30]), "+f"(s[31])
+          "+f"(s[8]), "+f"(s[9]), "+f"(s[10]), "+f"(s[11]), "+f"(s[12]), "+f"(s[13]), "+f"(s[14]), "+f"(s[15])
         :: "memory");
-    asm volatile(""
-        : "+f"(s[32]), "+f"(s[33]), "+f"(s[34]), "+f"(s[35]), "+f"(s[36]), "+f"(s[37]), "+f"(s[38]), "+f"(s[39]),
-          "+f"(s[40]), "+f"(s[41]), "+f"(s[42]), "+f"(s[43]), "+f"(s[44]), "+f"(s[45]), "+f"(s[46]), "+f"(s[47]),
-          "+f"(s[48]), "+f"(s[49]), "+f"(s[50]), "+f"(s[51]), "+f"(s[52]), "+f"(s[53]), "+f"(s[54]), "+f"(s[55]),
-          "+f"(s[56]), "+f"(s[57]), "+f"(s[58]), "+f"(s[59]), "+f"(s[60]), "+f"(s[61]), "+f"(s[62]), "+f"(s[63])
-        :: "memory");
+}
+template <int NS>
+__device__ __forceinline__ void wait_s_regs(float (&s)[NS]) {
+    static_assert(NS % 16 == 0, "sixteen registers per wait");
+#pragma unroll
+    for (int i = 0; i < NS; i += 16) wait_regs16(&s[i]);      // waits after the first are free; they only tie registers
 }
 
 // keys beyond `valid` (zero-filled tail of the last key tile) get logit -inf
-__device__ __forceinline__ void mask_tail(float (&s)[kBlockN], int valid) {
-    if (valid < kBlockN) {
+template <int NS>
+__device__ __forceinline__ void mask_tail(float (&s)[NS], int valid) {
+    if (valid < NS) {
 #pragma unroll
-        for (int i = 0; i < kBlockN; ++i) if (i >= valid) s[i] = -INFINITY;
+        for (int i = 0; i < NS; ++i) if (i >= valid) s[i] = -INFINITY;
     }
 }
 
-__device__ __forceinline__ float row_max(const float (&s)[kBlockN]) {
+template <int NS>
+__device__ __forceinline__ float row_max(const float (&s)[NS]) {
     float mx4[4] = {max3(s[0], s[1], s[2]), max3(s[3], s[4], s[5]), max3(s[6], s[7], s[8]), max3(s[9], s[10], s[11])};
 #pragma unroll
-    for (int i = 12; i + 7 < kBlockN; i += 8) {
+    for (int i = 12; i + 7 < NS; i += 8) {
         mx4[0] = max3(mx4[0], s[i], s[i + 1]); mx4[1] = max3(mx4[1], s[i + 2], s[i + 3]);
         mx4[2] = max3(mx4[2], s[i + 4], s[i + 5]); mx4[3] = max3(mx4[3], s[i + 6], s[i + 7]);
     }
-    static_assert((kBlockN - 12) % 8 == 4, "tail of the max tree");
-    mx4[0] = max3(mx4[0], s[kBlockN - 4], s[kBlockN - 3]);
-    mx4[1] = max3(mx4[1], s[kBlockN - 2], s[kBlockN - 1]);
+    static_assert((NS - 12) % 8 == 4, "tail of the max tree");
+    mx4[0] = max3(mx4[0], s[NS - 4], s[NS - 3]);
+    mx4[1] = max3(mx4[1], s[NS - 2], s[NS - 1]);
     return fmaxf(max3(mx4[0], mx4[1], mx4[2]), mx4[3]);
 }
 
-__device__ __forceinline__ float row_sum(const float (&s)[kBlockN]) {
+template <int NS>
+__device__ __forceinline__ float row_sum(const float (&s)[NS]) {
     float a[8];
 #pragma unroll
     for (int u = 0; u < 8; ++u) a[u] = s[u];
 #pragma unroll
-    for (int i = 8; i < kBlockN; i += 8) {
+    for (int i = 8; i < NS; i += 8) {
 #pragma unroll
         for (int u = 0; u < 8; ++u) a[u] += s[i + u];
     }
     return ((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7]));
+}
+
+// P of one key tile: NS/2 packed bf16 pairs over the first NS/2 columns of the S buffer
+template <int NS>
+__device__ __forceinline__ void store_p(uint32_t t_s, const uint32_t (&pk)[NS / 2]) {
+    if constexpr (NS == 64) {
+        tmem_st32(t_s, pk);
+    } else {
+        tmem_st16(t_s, reinterpret_cast<const uint32_t (&)[16]>(pk[0]));
+        tmem_st8(t_s + 16, reinterpret_cast<const uint32_t (&)[8]>(pk[16]));
+    }
 }
 
 // P has been stored: make it visible to the issuer warp
@@ -216,30 +233,30 @@ template <int DH>
 __device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j, bool first)
 {
     using C = Cfg<DH>;
-    constexpr int kSBufs = C::kSBufs;
+    constexpr int kSBufs = C::kSBufs, NS = C::kBlockN;
     const int buf = j % kSBufs;
-    const uint32_t t_s = st.t_s0 + buf * kBlockN;
+    const uint32_t t_s = st.t_s0 + buf * NS;
     const float sl2 = st.sl2;
-    float cur[kBlockN];
+    float cur[NS];
     // the load is waited for at once: registers of a tcgen05.ld in flight must not be touched, and the
     // compiler cannot know that
     wait_bar(st.bar_s + 8 * buf, (j / kSBufs) & 1, st.abort_flag, st.err_word);
     tc_fence_after();
-    load_s(t_s, cur);
-    wait_s_regs(cur);
-    mask_tail(cur, st.N - j * kBlockN);
-    if (first) st.m_ref = row_max(cur);           // the reference starts as the exact maximum of the first key tile
+    load_s<NS>(t_s, cur);
+    wait_s_regs<NS>(cur);
+    mask_tail<NS>(cur, st.N - j * NS);
+    if (first) st.m_ref = row_max<NS>(cur);           // the reference starts as the exact maximum of the first key tile
     float neg = -st.m_ref * sl2;
 #pragma unroll
-    for (int i = 0; i < kBlockN; ++i) cur[i] = ex2(fmaf(cur[i], sl2, neg));
-    float tile_sum = row_sum(cur);
+    for (int i = 0; i < NS; ++i) cur[i] = ex2(fmaf(cur[i], sl2, neg));
+    float tile_sum = row_sum<NS>(cur);
     if (__any_sync(0xffffffffu, !(tile_sum <= kTileSumLimit))) {
         // rare: the reference maximum is too low for this tile.  S is still intact in TMEM (P is not stored
         // yet): take the exact maximum, rescale what has been accumulated, and redo the tile
-        load_s(t_s, cur);
-        wait_s_regs(cur);
-        mask_tail(cur, st.N - j * kBlockN);
-        const float mx = row_max(cur);
+        load_s<NS>(t_s, cur);
+        wait_s_regs<NS>(cur);
+        mask_tail<NS>(cur, st.N - j * NS);
+        const float mx = row_max<NS>(cur);
         float alpha = 1.0f;
         if (mx > st.m_ref) { alpha = ex2((st.m_ref - mx) * sl2); st.m_ref = mx; st.l_sum *= alpha; }
         if (!first) {
@@ -270,18 +287,18 @@ __device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j, bool f
         }
         neg = -st.m_ref * sl2;
 #pragma unroll
-        for (int i = 0; i < kBlockN; ++i) cur[i] = ex2(fmaf(cur[i], sl2, neg));
-        tile_sum = row_sum(cur);
+        for (int i = 0; i < NS; ++i) cur[i] = ex2(fmaf(cur[i], sl2, neg));
+        tile_sum = row_sum<NS>(cur);
     }
     st.l_sum += tile_sum;
-    // P as bf16 pairs (element 2c in the low half) over the first 32 columns of this S buffer
-    uint32_t pk[32];
+    // P as bf16 pairs (element 2c in the low half) over the first NS/2 columns of this S buffer
+    uint32_t pk[NS / 2];
 #pragma unroll
-    for (int i = 0; i < 32; ++i) {
+    for (int i = 0; i < NS / 2; ++i) {
         __nv_bfloat162 v2 = __floats2bfloat162_rn(cur[2 * i], cur[2 * i + 1]);
         pk[i] = *reinterpret_cast<uint32_t *>(&v2);
     }
-    tmem_st32(t_s, pk);
+    store_p<NS>(t_s, pk);
     publish_p(st.bar_p + 8 * buf);
 }
 
@@ -319,7 +336,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     SoftmaxState<DH> st;
     st.sl2 = p.scale_log2;
     st.l_sum = 0.f;
-    st.t_s0 = t_row + tile * C::kSBufs * kBlockN;
+    st.t_s0 = t_row + tile * C::kSBufs * C::kBlockN;
     st.t_o = t_row + C::kColO + (tile * C::kSplit + par) * C::kOStride;
     st.bar_s = bar.s + 32 * tile; st.bar_p = bar.p + 32 * tile; st.bar_o = bar.o + 32 * tile;
     st.N = p.N; st.n_tiles = n_tiles; st.abort_flag = abort_flag; st.err_word = p.err_word;
@@ -401,9 +418,18 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
         uint32_t o[8], w[4];
         tmem_ld8(st.t_o + C::kMain, o);
         tc_wait_ld();
+        float f[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(o[i]) * w_own;
+        if (merge) {
+            tmem_ld8(t_other + C::kMain, o);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 8; ++i) f[i] = fmaf(__uint_as_float(o[i]), w_other, f[i]);
+        }
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(o[2 * i]) * w_own, __uint_as_float(o[2 * i + 1]) * w_own);
+            __nv_bfloat162 v2 = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
             w[i] = *reinterpret_cast<uint32_t *>(&v2);
         }
         if (dst) *reinterpret_cast<uint4 *>(dst + C::kMain) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -439,6 +465,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     const int tid = threadIdx.x;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);        // warp-uniform
     const int m0 = blockIdx.x * (kTilesM * kBlockM), h = blockIdx.y, b = blockIdx.z;
+    constexpr int kBlockN = C::kBlockN;
     const int n_tiles = (p.N + kBlockN - 1) / kBlockN;
     // the last CTA of a head may have rows in its first query tile only: the second tile's warps and MMAs are skipped
     const int q_tiles = (m0 + kBlockM < p.M) ? kTilesM : 1;
@@ -484,7 +511,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             const int st = j % C::kStagesK;
             wait_bar(bar.ke + 8 * st, ((j / C::kStagesK) & 1) ^ 1, &abort_flag, p.err_word);
             if (elect_one()) {
-                mbar_arrive_expect_tx(bar.kf + 8 * st, C::kTileBytes);
+                mbar_arrive_expect_tx(bar.kf + 8 * st, C::kLoadBytes);
 #pragma unroll
                 for (int ch = 0; ch < C::kChunks; ++ch)
                     tma_load_4d(sK + st * C::kTileBytes + ch * C::kChunkBytes, &tmap_k, bar.kf + 8 * st, ch * 64, j * kBlockN, h, b);
@@ -497,7 +524,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             const int st = j % C::kStagesV;
             wait_bar(bar.ve + 8 * st, ((j / C::kStagesV) & 1) ^ 1, &abort_flag, p.err_word);
             if (elect_one()) {
-                mbar_arrive_expect_tx(bar.vf + 8 * st, C::kTileBytes);
+                mbar_arrive_expect_tx(bar.vf + 8 * st, C::kLoadBytes);
 #pragma unroll
                 for (int ch = 0; ch < C::kChunks; ++ch)
                     tma_load_4d(sV + st * C::kTileBytes + ch * C::kChunkBytes, &tmap_v, bar.vf + 8 * st, ch * 64, j * kBlockN, h, b);
@@ -615,14 +642,14 @@ EncodeTiledFn get_encode_fn() {
 
 // K or V as a 4-D tensor (d, N, H, B) with 128-byte-swizzled boxes of 64 columns x 128 tokens
 int32_t make_kv_map(CUtensorMap *map, const void *base, int B, int H, int N, int d,
-                    int64_t sb, int64_t sh, int64_t sn, bool tail)
+                    int64_t sb, int64_t sh, int64_t sn, bool tail, int tile_keys)
 {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) return fail(ASTRAEA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
     cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)H, (cuuint64_t)B};
     cuuint64_t strides[3] = {(cuuint64_t)sn * 2, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
     // 64 columns x one key tile, 128-byte swizzle; or the 16-column tail chunk (32-byte swizzle; columns past d read as zero)
-    cuuint32_t box[4] = {tail ? 16u : 64u, (cuuint32_t)kBlockN, 1, 1};
+    cuuint32_t box[4] = {tail ? 16u : 64u, (cuuint32_t)tile_keys, 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, tail ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -636,15 +663,15 @@ int32_t launch_dh(const AttnArgs &a, cudaStream_t stream)
 {
     using C = Cfg<DH>;
     CUtensorMap mk, mv, mkt, mvt;
-    int32_t rc = make_kv_map(&mk, a.k, a.B, a.H, a.N, a.d, a.k_sb, a.k_sh, a.k_sn, false);
+    int32_t rc = make_kv_map(&mk, a.k, a.B, a.H, a.N, a.d, a.k_sb, a.k_sh, a.k_sn, false, C::kBlockN);
     if (rc != ASTRAEA_OK) return rc;
-    rc = make_kv_map(&mv, a.v, a.B, a.H, a.N, a.d, a.v_sb, a.v_sh, a.v_sn, false);
+    rc = make_kv_map(&mv, a.v, a.B, a.H, a.N, a.d, a.v_sb, a.v_sh, a.v_sn, false, C::kBlockN);
     if (rc != ASTRAEA_OK) return rc;
     mkt = mk; mvt = mv;
     if (C::kTail) {
-        rc = make_kv_map(&mkt, a.k, a.B, a.H, a.N, a.d, a.k_sb, a.k_sh, a.k_sn, true);
+        rc = make_kv_map(&mkt, a.k, a.B, a.H, a.N, a.d, a.k_sb, a.k_sh, a.k_sn, true, C::kBlockN);
         if (rc != ASTRAEA_OK) return rc;
-        rc = make_kv_map(&mvt, a.v, a.B, a.H, a.N, a.d, a.v_sb, a.v_sh, a.v_sn, true);
+        rc = make_kv_map(&mvt, a.v, a.B, a.H, a.N, a.d, a.v_sb, a.v_sh, a.v_sn, true, C::kBlockN);
         if (rc != ASTRAEA_OK) return rc;
     }
     static bool attr_set = false;
