@@ -210,6 +210,15 @@ __device__ __forceinline__ float row_sum(const float (&s)[NS]) {
     return ((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7]));
 }
 
+template <int NS>
+__device__ __forceinline__ void pack_p(const float (&e)[NS], uint32_t (&pk)[NS / 2]) {
+#pragma unroll
+    for (int i = 0; i < NS / 2; ++i) {
+        __nv_bfloat162 v2 = __floats2bfloat162_rn(e[2 * i], e[2 * i + 1]);
+        pk[i] = *reinterpret_cast<uint32_t *>(&v2);
+    }
+}
+
 // P of one key tile: NS/2 packed bf16 pairs over the first NS/2 columns of the S buffer
 template <int NS>
 __device__ __forceinline__ void store_p(uint32_t t_s, const uint32_t (&pk)[NS / 2]) {
@@ -250,6 +259,10 @@ __device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j, bool f
 #pragma unroll
     for (int i = 0; i < NS; ++i) cur[i] = ex2(fmaf(cur[i], sl2, neg));
     float tile_sum = row_sum<NS>(cur);
+    // P as bf16 pairs (element 2c in the low half); packed before the check below so that the conversions run
+    // in the shadow of the sum and the vote
+    uint32_t pk[NS / 2];
+    pack_p<NS>(cur, pk);
     if (__any_sync(0xffffffffu, !(tile_sum <= kTileSumLimit))) {
         // rare: the reference maximum is too low for this tile.  S is still intact in TMEM (P is not stored
         // yet): take the exact maximum, rescale what has been accumulated, and redo the tile
@@ -289,16 +302,10 @@ __device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j, bool f
 #pragma unroll
         for (int i = 0; i < NS; ++i) cur[i] = ex2(fmaf(cur[i], sl2, neg));
         tile_sum = row_sum<NS>(cur);
+        pack_p<NS>(cur, pk);
     }
     st.l_sum += tile_sum;
-    // P as bf16 pairs (element 2c in the low half) over the first NS/2 columns of this S buffer
-    uint32_t pk[NS / 2];
-#pragma unroll
-    for (int i = 0; i < NS / 2; ++i) {
-        __nv_bfloat162 v2 = __floats2bfloat162_rn(cur[2 * i], cur[2 * i + 1]);
-        pk[i] = *reinterpret_cast<uint32_t *>(&v2);
-    }
-    store_p<NS>(t_s, pk);
+    store_p<NS>(t_s, pk);                         // over the first NS/2 columns of this S buffer
     publish_p(st.bar_p + 8 * buf);
 }
 
