@@ -108,6 +108,22 @@ __device__ __forceinline__ float ex2(float x) {
     return y;
 }
 
+// packed fp32 pairs: one issue slot for two FMAs / adds
+__device__ __forceinline__ void ffma2(float &x0, float &x1, float m, float c) {
+    unsigned long long a, b, d, r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(a) : "f"(x0), "f"(x1));
+    asm("mov.b64 %0, {%1, %1};" : "=l"(b) : "f"(m));
+    asm("mov.b64 %0, {%1, %1};" : "=l"(d) : "f"(c));
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(d));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(x0), "=f"(x1) : "l"(r));
+}
+__device__ __forceinline__ unsigned long long fadd2(unsigned long long a, float x0, float x1) {
+    unsigned long long b, r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(b) : "f"(x0), "f"(x1));
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float r;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
@@ -257,8 +273,22 @@ __device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j, bool f
     if (first) st.m_ref = row_max<NS>(cur);           // the reference starts as the exact maximum of the first key tile
     float neg = -st.m_ref * sl2;
 #pragma unroll
-    for (int i = 0; i < NS; ++i) cur[i] = ex2(fmaf(cur[i], sl2, neg));
-    float tile_sum = row_sum<NS>(cur);
+    for (int i = 0; i < NS; i += 2) ffma2(cur[i], cur[i + 1], sl2, neg);
+#pragma unroll
+    for (int i = 0; i < NS; ++i) cur[i] = ex2(cur[i]);
+    float tile_sum;
+    {
+        unsigned long long a[4] = {0ull, 0ull, 0ull, 0ull};
+#pragma unroll
+        for (int i = 0; i < NS; i += 8) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) a[u] = fadd2(a[u], cur[i + 2 * u], cur[i + 2 * u + 1]);
+        }
+        float f[8];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) asm("mov.b64 {%0, %1}, %2;" : "=f"(f[2 * u]), "=f"(f[2 * u + 1]) : "l"(a[u]));
+        tile_sum = ((f[0] + f[1]) + (f[2] + f[3])) + ((f[4] + f[5]) + (f[6] + f[7]));
+    }
     // P as bf16 pairs (element 2c in the low half); packed before the check below so that the conversions run
     // in the shadow of the sum and the vote
     uint32_t pk[NS / 2];
