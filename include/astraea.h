@@ -59,6 +59,7 @@ extern "C" {
 #define ASTRAEA_OP_SELECT       1
 #define ASTRAEA_OP_SPARSE_ATTN  2
 #define ASTRAEA_OP_STEP         3
+#define ASTRAEA_OP_SPARSE_ATTN_KV 4          /* astraea_sparse_attn with kv_idx: pass M_kv as the M argument */
 
 /*
  * Selection metric (Section 3.2 "Selection Metric"; Algorithm 1 lines 1-2):
@@ -109,7 +110,10 @@ int32_t astraea_select(const float *score, int B, int N_sel, int k, int n_always
  *             [B,N,H,d] has strides (N*H*d, d, H*d); [B,H,N,d] has (H*N*d, N*d, d).
  *             Token strides must be multiples of 8 elements, bases 16-byte aligned.
  *   q_idx   : int32 [B, M] strictly ascending token indices in [0,N); NULL => rows 0..M-1
- *   kv_idx  : must be NULL (all keys, the paper's method); the select-Q-and-K ablation is not built
+ *   kv_idx  : NULL (all keys: the paper's method), or int32 [B, M_kv] token indices in [0,N): the softmax then
+ *             runs over the listed keys/values only (the SelectQ&K variant of the paper's ablation study, Table 2).  Their
+ *             rows are gathered into the workspace first, which must then hold
+ *             astraea_workspace_bytes(ASTRAEA_OP_SPARSE_ATTN_KV, B, H, N, M_kv, d) bytes.
  *   out     : bf16 [B, N, H, d]  (or [B, M, H, d] compact)
  *   lse_out : fp32 [B, H, N]     (or [B, H, M] compact); may be NULL
  *   scale   : 0 => 1/sqrt(d)
@@ -118,7 +122,7 @@ int32_t astraea_select(const float *score, int B, int N_sel, int k, int n_always
  * Arithmetic: bf16 operands, fp32 logits, softmax and accumulation; probabilities are
  * rounded to bf16 before the P.V product; outputs rounded to bf16.
  * M = 0 is valid: nothing is launched and the caches are untouched.
- * Errors: INVALID_ARG, UNSUPPORTED (d not in {64,72,128}, kv_idx != NULL), WORKSPACE_TOO_SMALL, CUDA.
+ * Errors: INVALID_ARG, UNSUPPORTED (d not in {64,72,128}), WORKSPACE_TOO_SMALL, CUDA.
  */
 int32_t astraea_sparse_attn(const void *q, const void *k, const void *v,
                             int64_t q_sb, int64_t q_sh, int64_t q_sn,

@@ -54,6 +54,7 @@ size_t astraea_workspace_bytes(int op, int B, int H, int N, int M, int d) {
     switch (op) {
     case ASTRAEA_OP_SELECT: return select_workspace_bytes(B, N);
     case ASTRAEA_OP_SPARSE_ATTN: return attn_workspace_bytes(B, H, N, M, d);
+    case ASTRAEA_OP_SPARSE_ATTN_KV: return attn_kv_workspace_bytes(B, H, M, d);
     case ASTRAEA_OP_STEP: return attn_workspace_bytes(B, H, N, M, d) + align_up(select_workspace_bytes(B, N), 256);
     default: return 0;
     }
@@ -98,12 +99,11 @@ int32_t astraea_sparse_attn(const void *q, const void *k, const void *v,
                             int B, int H, int N, int d, float scale, uint32_t flags,
                             void *workspace, size_t workspace_bytes, void *stream)
 {
-    (void)M_kv;
     REQUIRE(B > 0 && H > 0 && N > 0 && d > 0, "astraea_sparse_attn: B, H, N, d must be positive");
+    REQUIRE(!kv_idx || (M_kv > 0 && M_kv <= N), "astraea_sparse_attn: M_kv=%d outside [1, N=%d]", M_kv, N);
     REQUIRE(M >= 0 && M <= N, "astraea_sparse_attn: M=%d outside [0, N=%d]", M, N);
     if (d != 64 && d != 72 && d != 128)
         return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_sparse_attn: head_dim %d not in {64, 72, 128}", d);
-    if (kv_idx) return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_sparse_attn: kv_idx (select-Q-and-K ablation) is not built");
     if (flags & ~ASTRAEA_ATTN_COMPACT_OUT) return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_sparse_attn: unknown flags 0x%x", flags);
     REQUIRE(q && k && v && out, "astraea_sparse_attn: null q, k, v or out");
     REQUIRE(aligned16(q) && aligned16(k) && aligned16(v) && aligned16(out), "astraea_sparse_attn: q, k, v, out must be 16-byte aligned");
@@ -113,9 +113,10 @@ int32_t astraea_sparse_attn(const void *q, const void *k, const void *v,
     REQUIRE(q_sn >= d && k_sn >= d && v_sn >= d && q_sh > 0 && k_sh > 0 && v_sh > 0 && q_sb >= 0 && k_sb >= 0 && v_sb >= 0,
             "astraea_sparse_attn: strides must be positive and token stride >= head_dim");
     REQUIRE(scale >= 0.f, "astraea_sparse_attn: scale must be >= 0 (0 selects 1/sqrt(d))");
-    if (!workspace || workspace_bytes < attn_workspace_bytes(B, H, N, M, d))
+    const size_t ws_need = kv_idx ? attn_kv_workspace_bytes(B, H, M_kv, d) : attn_workspace_bytes(B, H, N, M, d);
+    if (!workspace || workspace_bytes < ws_need)
         return fail(ASTRAEA_ERR_WORKSPACE_TOO_SMALL, "astraea_sparse_attn: workspace of %zu bytes, need %zu",
-                    workspace_bytes, attn_workspace_bytes(B, H, N, M, d));
+                    workspace_bytes, ws_need);
     REQUIRE((reinterpret_cast<uintptr_t>(workspace) & 255u) == 0, "astraea_sparse_attn: workspace must be 256-byte aligned");
     if (M == 0) return ASTRAEA_OK;
     AttnArgs a;
@@ -128,6 +129,8 @@ int32_t astraea_sparse_attn(const void *q, const void *k, const void *v,
     a.scale = (scale == 0.f) ? 1.0f / sqrtf((float)d) : scale;
     a.flags = flags;
     a.err_word = reinterpret_cast<int *>(workspace);
+    a.N_tok = N;
+    if (kv_idx) return launch_sparse_attn_kv(a, kv_idx, M_kv, workspace, (cudaStream_t)stream);
     return launch_sparse_attn(a, (cudaStream_t)stream);
 }
 
@@ -165,6 +168,7 @@ int32_t astraea_sparse_attn_noalloc(const void *q, const void *k, const void *v,
     a.scale = (scale == 0.f) ? 1.0f / sqrtf((float)d) : scale;
     a.flags = flags;
     a.err_word = nullptr;
+    a.N_tok = N;
     return launch_sparse_attn_noalloc(a, (cudaStream_t)stream);
 }
 

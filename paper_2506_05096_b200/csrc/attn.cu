@@ -96,7 +96,8 @@ struct Params {
     int M;
     __nv_bfloat16 *out;
     float *lse_out;
-    int N, H;
+    int N, H;                    // N: keys
+    int N_tok;                   // tokens of q / out / lse_out (N_tok == N unless the keys were gathered)
     float scale, scale_log2;
     int compact;
     int *err_word;
@@ -356,7 +357,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
         uint4 val = make_uint4(0, 0, 0, 0);
         if (m < p.M && c * 8 < DH) {                 // the upper half of the tail chunk stays zero
             const int tok = p.q_idx ? __ldg(p.q_idx + (size_t)b * p.M + m) : m;
-            if ((unsigned)tok < (unsigned)p.N) {
+            if ((unsigned)tok < (unsigned)p.N_tok) {
                 const __nv_bfloat16 *src = p.q + (size_t)b * p.q_sb + (size_t)tok * p.q_sn + (size_t)h * p.q_sh + c * 8;
                 val = __ldg(reinterpret_cast<const uint4 *>(src));
             }
@@ -382,7 +383,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     int tok = -1;
     if (m < p.M) {
         tok = p.q_idx ? __ldg(p.q_idx + (size_t)b * p.M + m) : m;
-        if ((unsigned)tok >= (unsigned)p.N) { if (par == 0) atomicExch(p.err_word, kErrBadIndex); tok = -1; }
+        if ((unsigned)tok >= (unsigned)p.N_tok) { if (par == 0) atomicExch(p.err_word, kErrBadIndex); tok = -1; }
     }
 
     st.m_ref = -INFINITY;
@@ -417,10 +418,10 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     w_other *= inv_l;
     __nv_bfloat16 *dst = nullptr;
     if (tok >= 0 && !*abort_flag) {
-        const size_t orow = p.compact ? ((size_t)b * p.M + m) : ((size_t)b * p.N + tok);
+        const size_t orow = p.compact ? ((size_t)b * p.M + m) : ((size_t)b * p.N_tok + tok);
         dst = p.out + (orow * p.H + h) * DH;
         if (p.lse_out) {
-            const size_t li = p.compact ? (((size_t)b * p.H + h) * p.M + m) : (((size_t)b * p.H + h) * p.N + tok);
+            const size_t li = p.compact ? (((size_t)b * p.H + h) * p.M + m) : (((size_t)b * p.H + h) * p.N_tok + tok);
             p.lse_out[li] = m_ref * p.scale + logf(l_sum);
         }
     }
@@ -723,7 +724,7 @@ int32_t launch_dh(const AttnArgs &a, cudaStream_t stream)
     p.q_idx = a.q_idx; p.M = a.M;
     p.out = reinterpret_cast<__nv_bfloat16 *>(a.out);
     p.lse_out = a.lse_out;
-    p.N = a.N; p.H = a.H;
+    p.N = a.N; p.H = a.H; p.N_tok = a.N_tok;
     p.scale = a.scale;
     p.scale_log2 = a.scale * 1.4426950408889634f;
     p.compact = (a.flags & ASTRAEA_ATTN_COMPACT_OUT) ? 1 : 0;
@@ -736,6 +737,57 @@ int32_t launch_dh(const AttnArgs &a, cudaStream_t stream)
 }  // namespace
 
 size_t attn_workspace_bytes(int, int, int, int, int) { return 256; }
+
+// ---------------------------------------------------------------- gathered keys / values
+// The "select Q and K" ablation of the paper restricts keys and values to listed tokens.  The listed K and V
+// rows are gathered into compact [B, M_kv, H, d] buffers in the workspace, and the attention kernel runs on them.
+namespace {
+__global__ void __launch_bounds__(256)
+gather_kv_kernel(uint4 *__restrict__ dst, const __nv_bfloat16 *__restrict__ src, int64_t sb, int64_t sh, int64_t sn,
+                 const int32_t *__restrict__ idx, int B, int H, int N, int M_kv, int vec_per_row, int *err_word)
+{
+    const long long total = (long long)B * M_kv * H * vec_per_row;
+    for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (long long)gridDim.x * blockDim.x) {
+        const int v = (int)(t % vec_per_row);
+        long long r = t / vec_per_row;
+        const int h = (int)(r % H); r /= H;
+        const int m = (int)(r % M_kv);
+        const int b = (int)(r / M_kv);
+        const int tok = __ldg(idx + (size_t)b * M_kv + m);
+        uint4 val = make_uint4(0, 0, 0, 0);
+        if ((unsigned)tok < (unsigned)N) val = __ldg(reinterpret_cast<const uint4 *>(src + b * sb + tok * sn + h * sh) + v);
+        else if (v == 0 && h == 0) atomicExch(err_word, kErrBadIndex);
+        dst[t] = val;
+    }
+}
+}  // namespace
+
+size_t attn_kv_workspace_bytes(int B, int H, int M_kv, int d) {
+    const size_t one = ((size_t)B * M_kv * H * d * 2 + 255) / 256 * 256;
+    return 256 + 2 * one;
+}
+
+int32_t launch_sparse_attn_kv(AttnArgs a, const int32_t *kv_idx, int M_kv, void *workspace, cudaStream_t stream)
+{
+    const size_t one = ((size_t)a.B * M_kv * a.H * a.d * 2 + 255) / 256 * 256;
+    char *ws = reinterpret_cast<char *>(workspace);
+    uint4 *kc = reinterpret_cast<uint4 *>(ws + 256), *vc = reinterpret_cast<uint4 *>(ws + 256 + one);
+    const int vec = a.d / 8;
+    const long long total = (long long)a.B * M_kv * a.H * vec;
+    const int grid = (int)((total + 255) / 256 < (long long)kNumSMs * 16 ? (total + 255) / 256 : (long long)kNumSMs * 16);
+    gather_kv_kernel<<<grid, 256, 0, stream>>>(kc, reinterpret_cast<const __nv_bfloat16 *>(a.k), a.k_sb, a.k_sh, a.k_sn,
+                                               kv_idx, a.B, a.H, a.N, M_kv, vec, a.err_word);
+    gather_kv_kernel<<<grid, 256, 0, stream>>>(vc, reinterpret_cast<const __nv_bfloat16 *>(a.v), a.v_sb, a.v_sh, a.v_sn,
+                                               kv_idx, a.B, a.H, a.N, M_kv, vec, a.err_word);
+    int32_t rc = check_launch("astraea_sparse_attn (gather of K/V)");
+    if (rc != ASTRAEA_OK) return rc;
+    a.k = kc; a.v = vc;
+    a.k_sb = a.v_sb = (int64_t)M_kv * a.H * a.d;
+    a.k_sh = a.v_sh = a.d;
+    a.k_sn = a.v_sn = (int64_t)a.H * a.d;
+    a.N = M_kv;                       // keys; a.N_tok stays the token count of q / out
+    return launch_sparse_attn(a, stream);
+}
 
 // Scratch of astraea_sparse_attn_noalloc: lives in the library image, so every GPU that loads the
 // library holds these bytes until the process exits.  In host code this name is only a handle of

@@ -38,13 +38,16 @@ struct AttnArgs {
     int M;
     void *out;
     float *lse_out;
-    int B, H, N, d;
+    int B, H, N, d;          // N: keys
+    int N_tok;               // tokens of q / out / lse_out
     float scale;
     uint32_t flags;
     int *err_word;
 };
 int32_t launch_sparse_attn(const AttnArgs &a, cudaStream_t stream);
 size_t attn_workspace_bytes(int B, int H, int N, int M, int d);
-int32_t launch_sparse_attn_noalloc(AttnArgs a, cudaStream_t stream);   // scratch in a static device array
+int32_t launch_sparse_attn_noalloc(AttnArgs a, cudaStream_t stream);
+size_t attn_kv_workspace_bytes(int B, int H, int M_kv, int d);
+int32_t launch_sparse_attn_kv(AttnArgs a, const int32_t *kv_idx, int M_kv, void *workspace, cudaStream_t stream);   // scratch in a static device array
 
 }  // namespace astraea

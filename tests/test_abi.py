@@ -58,7 +58,7 @@ def test_argument_errors_are_reported_before_any_launch(L):
     args = lambda d, kv=None, ws=p, wsb=4096, flags=0, qsn=64: (p, p, p, s[0], s[1], qsn, *s, *s, None, 16, kv, 0, p, None,
                                                                1, 1, 16, d, 0.0, flags, ws, wsb, None)
     assert L.astraea_sparse_attn(*args(96)) == binding.ERR_UNSUPPORTED
-    assert L.astraea_sparse_attn(*args(64, kv=p)) == binding.ERR_UNSUPPORTED
+    assert L.astraea_sparse_attn(*args(64, kv=p)) == binding.ERR_INVALID_ARG      # kv_idx with M_kv = 0
     assert L.astraea_sparse_attn(*args(64, flags=8)) == binding.ERR_UNSUPPORTED
     assert L.astraea_sparse_attn(*args(64, wsb=8)) == binding.ERR_WORKSPACE_TOO_SMALL
     assert L.astraea_sparse_attn(*args(64, qsn=60)) == binding.ERR_INVALID_ARG

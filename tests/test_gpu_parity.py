@@ -253,6 +253,37 @@ def test_attn_peaked_softmax_triggers_rescaling(oracle):
     _attn_case(oracle, 1, 1, 900, 128, 128, seed=10, amp=2.0)
 
 
+@pytest.mark.parametrize("d", [64, 72, 128])
+def test_attn_select_q_and_k_ablation(oracle, d):
+    """kv_idx: the softmax runs over the listed keys/values only (the ablation that also masks K and V)."""
+    rng = np.random.default_rng(20 + d)
+    B, H, N, M, M_kv = 2, 2, 500, 90, 217
+    q, k, v, cache = (synth.f32_to_bf16_bits(rng.standard_normal((B, N, H, d)).astype(np.float32)) for _ in range(4))
+    q_idx = np.stack([np.sort(rng.choice(N, M, replace=False)) for _ in range(B)]).astype(np.int32)
+    kv_idx = np.stack([np.sort(rng.choice(N, M_kv, replace=False)) for _ in range(B)]).astype(np.int32)
+    want_o, want_lse, _ = oracle.sparse_attn(f64(q), f64(k), f64(v), q_idx=q_idx, kv_idx=kv_idx)
+    out, lse = to_dev_bf16(cache), torch.zeros(B, H, N, device="cuda")
+    ws = A.new_workspace(A.OP_SPARSE_ATTN_KV, B, H, N, M_kv, d)
+    s = A.bhnd_strides(N, H, d)
+    A.astraea_sparse_attn(to_dev_bf16(q), to_dev_bf16(k), to_dev_bf16(v), s, s, s, dev(q_idx), M, out, lse, B, H, N, d,
+                          workspace=ws, kv_idx=dev(kv_idx), M_kv=M_kv)
+    A.astraea_poll_error(ws)
+    got = np.take_along_axis(bf16_dev_to_f64(out), q_idx[:, :, None, None].astype(np.int64), 1)
+    err = np.abs(got - want_o)
+    assert err.max() < ATTN_MAX_ABS and err.mean() < ATTN_MEAN_ABS, (err.max(), err.mean())
+    got_lse = np.take_along_axis(lse.cpu().numpy().astype(np.float64), q_idx[:, None, :].astype(np.int64), 2)
+    assert np.abs(got_lse - want_lse).max() < LSE_ABS
+    mask = np.ones((B, N), bool)
+    for b in range(B):
+        mask[b, q_idx[b]] = False
+    assert np.array_equal(bf16_dev_to_f64(out)[mask], f64(cache)[mask])
+    # too small a workspace for the gathered rows is refused
+    with pytest.raises(A.AstraeaError) as e:
+        A.astraea_sparse_attn(to_dev_bf16(q), to_dev_bf16(k), to_dev_bf16(v), s, s, s, dev(q_idx), M, out, lse, B, H, N, d,
+                              workspace=A.new_workspace(A.OP_SPARSE_ATTN, B, H, N, M, d), kv_idx=dev(kv_idx), M_kv=M_kv)
+    assert e.value.code == A.ERR_WORKSPACE_TOO_SMALL
+
+
 def test_attn_closed_forms_on_device():
     """Zero keys: every selected output is the mean of all value rows and LSE = ln N; this
     catches phantom keys from the zero-filled tail of the last key tile."""
