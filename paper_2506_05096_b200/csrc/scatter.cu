@@ -9,8 +9,8 @@ namespace astraea {
 namespace {
 
 constexpr int kWarpsPerBlock = 8;
-constexpr int kBlocksPerSM = 8;
-constexpr int kUnroll = 4;
+constexpr int kBlocksPerSM = 16;
+constexpr int kUnroll = 6;
 
 __device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
     uint4 r;
@@ -34,15 +34,13 @@ scatter_kernel(uint4 *__restrict__ cache, const uint4 *__restrict__ rows, const 
         if ((unsigned)i >= (unsigned)N) continue;           // never write outside the cache
         const uint4 *src = rows + ((size_t)b * (src_full ? N : M) + (src_full ? i : r)) * vec_per_row;
         uint4 *dst = cache + ((size_t)b * N + i) * vec_per_row;
-        int v = lane;
-        for (; v + 32 * (kUnroll - 1) < vec_per_row; v += 32 * kUnroll) {
+        for (int v = lane; v < vec_per_row; v += 32 * kUnroll) {
             uint4 a[kUnroll];
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) a[u] = ld_stream(src + v + 32 * u);
+            for (int u = 0; u < kUnroll; ++u) if (v + 32 * u < vec_per_row) a[u] = ld_stream(src + v + 32 * u);
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) dst[v + 32 * u] = a[u];
+            for (int u = 0; u < kUnroll; ++u) if (v + 32 * u < vec_per_row) dst[v + 32 * u] = a[u];
         }
-        for (; v < vec_per_row; v += 32) dst[v] = ld_stream(src + v);
     }
 }
 

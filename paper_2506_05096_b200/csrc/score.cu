@@ -2,7 +2,7 @@
 // (selection-metric equations of Section 3.2; Algorithm 1 lines 1-2).
 //
 // HBM-bound: 2 * D bf16 per token are read once.  One warp owns one token row and
-// streams it with 16-byte loads, several in flight per lane; the channel reduction is a
+// streams it with 16-byte loads, six per tensor in flight per lane; the channel reduction is a
 // per-lane fp32 partial sum followed by a warp shuffle tree.  The per-head LSE values of
 // the token (a strided gather of H floats, 1/d of the traffic) are averaged by the same
 // warp.  The grid is a multiple of the SM count and walks the tokens with a grid stride.
@@ -12,8 +12,8 @@ namespace astraea {
 namespace {
 
 constexpr int kWarpsPerBlock = 8;
-constexpr int kBlocksPerSM = 8;
-constexpr int kUnroll = 4;
+constexpr int kBlocksPerSM = 16;     // twice what is resident: the second half evens out the tail
+constexpr int kUnroll = 6;           // 16-byte loads in flight per lane and tensor
 
 __device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
     uint4 r;
@@ -65,20 +65,19 @@ score_kernel(const uint4 *__restrict__ x_cur, const uint4 *__restrict__ x_ref,
         const uint4 *pr = x_ref + row;
 
         float acc0 = 0.f, acc1 = 0.f;
-        int v = lane;
-        for (; v + 32 * (kUnroll - 1) < vec_per_row; v += 32 * kUnroll) {
+        for (int v = lane; v < vec_per_row; v += 32 * kUnroll) {
             uint4 a[kUnroll], r[kUnroll];
+            // loads past the end of the row are skipped; zeros add nothing in any of the three reductions
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) a[u] = ld_stream(pc + v + 32 * u);
+            for (int u = 0; u < kUnroll; ++u) a[u] = (v + 32 * u < vec_per_row) ? ld_stream(pc + v + 32 * u) : make_uint4(0, 0, 0, 0);
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) r[u] = ld_stream(pr + v + 32 * u);
+            for (int u = 0; u < kUnroll; ++u) r[u] = (v + 32 * u < vec_per_row) ? ld_stream(pr + v + 32 * u) : make_uint4(0, 0, 0, 0);
 #pragma unroll
             for (int u = 0; u < kUnroll; u += 2) {
                 acc0 = accum_vec<MODE>(a[u], r[u], acc0);
                 acc1 = accum_vec<MODE>(a[u + 1], r[u + 1], acc1);
             }
         }
-        for (; v < vec_per_row; v += 32) acc0 = accum_vec<MODE>(ld_stream(pc + v), ld_stream(pr + v), acc0);
         float acc = acc0 + acc1;
 
         // S_LSE: mean over heads of exp(lse[b,h,i]) (or of lse itself)
