@@ -45,7 +45,6 @@ using namespace ptx;
 constexpr int kBlockM = 128;                     // rows of one query tile
 constexpr int kTilesM = 2;                       // query tiles per CTA
 constexpr uint32_t kTmemCols = 512;
-constexpr float kTileSumLimit = 65536.0f;        // a tile's sum of exponentials above this forces an exact maximum
 constexpr uint64_t kWaitLimitNs = 1000000000ull; // bounded waits: one second
 
 template <int DH> struct Cfg {
@@ -61,13 +60,22 @@ template <int DH> struct Cfg {
     // keys per K/V tile = columns of an S buffer.  64, but 48 at head_dim 72: four O accumulators of 80 columns
     // leave 192 TMEM columns for the four S buffers
     static constexpr int kBlockN = (DH == 72) ? 48 : 64;
-    static constexpr int kSBufs = 2;                              // S buffers per query tile
+    // S buffers per query tile.  Split: three, used round-robin by the two warpgroups, so that S of key tile j+2
+    // is produced while tiles j and j+1 are in the softmax; the warpgroups then share one O accumulator
+    static constexpr int kSBufs = (kSplit == 2) ? 3 : 2;
+    // exponentials per 16 that are computed on the FMA pipe instead of the XU (measured: 6 is best at head_dim 64,
+    // none at 72 and 128, where the tensor pipe has less slack)
+    static constexpr int kPolyOf16 = (DH == 64) ? 6 : 0;
+    // a tile's sum of exponentials above this means the reference maximum is too low.  fp32 and bf16 share the
+    // exponent range, so the limit only has to keep row sums and accumulators far from overflow; with the
+    // split it is as high as that allows, because a redo costs the CTA two more passes over the keys
+    static constexpr float kTileSumLimit = (kSplit == 2) ? 1152921504606846976.0f /* 2^60 */ : 65536.0f;
+    static constexpr int kAhead = 2;                              // Q K^T runs this many key tiles ahead of P V
     static constexpr int kSoftmaxWarps = 4 * kTilesM * kSplit;
     static constexpr int kThreads = (kSoftmaxWarps + 4) * 32;     // + producer, two issuers, one register donor
     static constexpr uint32_t kColO = kTilesM * kSBufs * kBlockN; // first O column
     static constexpr uint32_t kOStride = (DH == 64) ? 64 : (DH == 72) ? 80 : 128;   // columns between O accumulators
-    static_assert(kColO + kTilesM * kSplit * kOStride <= kTmemCols && kMain + kTailPad <= (int)kOStride, "TMEM budget");
-    static_assert(kSplit == 1 || kSplit == kSBufs, "a split warpgroup owns one S buffer");
+    static_assert(kColO + kTilesM * kOStride <= kTmemCols && kMain + kTailPad <= (int)kOStride, "TMEM budget");
     // setmaxnreg only redistributes what the CTA got at launch: an increase that the decreases of
     // the last warpgroup cannot cover would block forever
     static constexpr int kRegsLaunch = (65536 / kThreads) / 8 * 8;
@@ -84,7 +92,7 @@ template <int DH> struct Cfg {
     static_assert(kQTileBytes % 1024 == 0 && kTileBytes % 1024 == 0, "tiles keep the 1024-byte swizzle alignment");
     static constexpr int kStagesK = (DH == 128) ? 5 : 6;
     static constexpr int kStagesV = (DH == 128) ? 5 : 6;
-    static_assert(kStagesK > kSBufs, "K runs kSBufs tiles ahead");
+    static_assert(kStagesK > kAhead, "K runs kAhead tiles ahead");
     static constexpr int kBarBytes = 512;
     static constexpr int kSmemBytes = kQTileBytes * kTilesM + kTileBytes * (kStagesK + kStagesV) + kBarBytes + 1024;
 };
@@ -123,6 +131,34 @@ __device__ __forceinline__ unsigned long long fadd2(unsigned long long a, float 
     asm("mov.b64 %0, {%1, %2};" : "=l"(b) : "f"(x0), "f"(x1));
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
     return r;
+}
+
+// 2^x for a pair, without the XU pipe: x = n + f with n = floor(x) taken by adding 1.5 * 2^23 rounded down, a
+// cubic for 2^f on [0, 1) (relative error 8.6e-5, well below the bf16 rounding of P), and n added to the
+// exponent field.  x is clamped to the normal range first.
+__device__ __forceinline__ void exp2_poly2(float &x0, float &x1) {
+    x0 = fmaxf(x0, -126.0f);
+    x1 = fmaxf(x1, -126.0f);
+    unsigned long long x, t, pl;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(x) : "f"(x0), "f"(x1));
+    asm("{\n\t.reg .b64 mg, c1, c2, c3, one, fr;\n\t"
+        "mov.b64 mg, 0x4B4000004B400000;\n\t"        // 1.5 * 2^23, twice
+        "mov.b64 c3, 0x3D9DD4DF3D9DD4DF;\n\t"        // 2^f ~ 1 + f (c1 + f (c2 + f c3))
+        "mov.b64 c2, 0x3E691C043E691C04;\n\t"
+        "mov.b64 c1, 0x3F31F3293F31F329;\n\t"
+        "mov.b64 one, 0x3F8000003F800000;\n\t"
+        "add.rm.f32x2 %0, %2, mg;\n\t"               // low mantissa bits of t = floor(x)
+        "sub.rn.f32x2 fr, %0, mg;\n\t"
+        "sub.rn.f32x2 fr, %2, fr;\n\t"               // f = x - floor(x)
+        "fma.rn.f32x2 %1, fr, c3, c2;\n\t"
+        "fma.rn.f32x2 %1, %1, fr, c1;\n\t"
+        "fma.rn.f32x2 %1, %1, fr, one;\n\t}"
+        : "=&l"(t), "=&l"(pl) : "l"(x));
+    uint32_t t0, t1, p0, p1;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(t0), "=r"(t1) : "l"(t));
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(p0), "=r"(p1) : "l"(pl));
+    x0 = __uint_as_float(p0 + (t0 << 23));
+    x1 = __uint_as_float(p1 + (t1 << 23));
 }
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -166,6 +202,9 @@ template <int DH> struct SoftmaxState {
     float sl2, m_ref, l_sum;
     uint32_t t_s0, t_o, bar_s, bar_p, bar_o;
     int N, n_tiles;
+    float *ref_x;                   // split: the reference of this thread's row, shared by the tile's two warpgroups
+    int ref_bar;                    // split: named barrier on which the reference is handed over
+    volatile int *redo_flag;
     volatile int *abort_flag;
     int *err_word;
 };
@@ -254,29 +293,59 @@ __device__ __forceinline__ void publish_p(uint32_t bar) {
     mbar_arrive(bar);
 }
 
-// One key tile of the online softmax.  `first`: this warpgroup's first tile.
-template <int DH>
-__device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j, bool first)
+// What a pass over the keys does (split configurations only know kSpeculate unless a tile overflowed):
+//   kSpeculate  exponentials against the exact row maximum of key tile 0; a tile whose sum of exponentials passes
+//               the limit is, without the split, redone after rescaling the accumulator in place, and with the
+//               split (where the accumulator is shared) raises the CTA's redo flag;
+//   kMaxOnly    first pass of a redo: only the exact row maxima over all keys are taken;
+//   kExact      second pass of a redo: exponentials against those maxima, nothing can overflow.
+enum { kSpeculate = 0, kMaxOnly = 1, kExact = 2 };
+
+// One key tile of the softmax.  j: key tile; g: running count of S-buffer uses of this query tile (buffer
+// g % kSBufs, barrier phase (g / kSBufs) & 1), which keeps counting across the passes.
+template <int DH, int MODE>
+__device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j, int g)
 {
     using C = Cfg<DH>;
     constexpr int kSBufs = C::kSBufs, NS = C::kBlockN;
-    const int buf = j % kSBufs;
+    const int buf = g % kSBufs;
     const uint32_t t_s = st.t_s0 + buf * NS;
     const float sl2 = st.sl2;
     float cur[NS];
     // the load is waited for at once: registers of a tcgen05.ld in flight must not be touched, and the
     // compiler cannot know that
-    wait_bar(st.bar_s + 8 * buf, (j / kSBufs) & 1, st.abort_flag, st.err_word);
+    wait_bar(st.bar_s + 8 * buf, (g / kSBufs) & 1, st.abort_flag, st.err_word);
     tc_fence_after();
     load_s<NS>(t_s, cur);
     wait_s_regs<NS>(cur);
     mask_tail<NS>(cur, st.N - j * NS);
-    if (first) st.m_ref = row_max<NS>(cur);           // the reference starts as the exact maximum of the first key tile
+    if constexpr (MODE == kMaxOnly) {
+        st.m_ref = fmaxf(st.m_ref, row_max<NS>(cur));
+        tc_fence_before();
+        mbar_arrive(st.bar_p + 8 * buf);              // S has been read: the buffer may be refilled
+        return;
+    }
+    const bool first = MODE == kSpeculate && j == 0;
+    if (first) {                                      // the reference starts as the exact maximum of the first key tile
+        st.m_ref = row_max<NS>(cur);
+        if constexpr (C::kSplit == 2) {               // ... and the other warpgroup of this query tile takes the same one
+            *st.ref_x = st.m_ref;
+            if (st.ref_bar == 3) asm volatile("bar.arrive 3, 256;" ::: "memory");
+            else asm volatile("bar.arrive 4, 256;" ::: "memory");
+        }
+    }
     float neg = -st.m_ref * sl2;
 #pragma unroll
     for (int i = 0; i < NS; i += 2) ffma2(cur[i], cur[i + 1], sl2, neg);
+    // kPolyOf16 of every 16 exponentials go to the FMA pipe, the rest to the XU
 #pragma unroll
-    for (int i = 0; i < NS; ++i) cur[i] = ex2(cur[i]);
+    for (int i = 0; i < NS; i += 16) {
+#pragma unroll
+        for (int u = 0; u < 16; u += 2) {
+            if (u >= 16 - C::kPolyOf16) exp2_poly2(cur[i + u], cur[i + u + 1]);
+            else { cur[i + u] = ex2(cur[i + u]); cur[i + u + 1] = ex2(cur[i + u + 1]); }
+        }
+    }
     float tile_sum;
     {
         unsigned long long a[4] = {0ull, 0ull, 0ull, 0ull};
@@ -294,7 +363,11 @@ __device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j, bool f
     // in the shadow of the sum and the vote
     uint32_t pk[NS / 2];
     pack_p<NS>(cur, pk);
-    if (__any_sync(0xffffffffu, !(tile_sum <= kTileSumLimit))) {
+    if constexpr (MODE == kSpeculate && C::kSplit == 2) {
+        // rare: the reference is too low for this tile.  The accumulator is shared with the other warpgroup, so
+        // nothing is repaired here: the CTA finishes the pass and redoes its work with exact maxima
+        if (__any_sync(0xffffffffu, !(tile_sum <= C::kTileSumLimit))) *st.redo_flag = 1;
+    } else if (MODE == kSpeculate && __any_sync(0xffffffffu, !(tile_sum <= C::kTileSumLimit))) {
         // rare: the reference maximum is too low for this tile.  S is still intact in TMEM (P is not stored
         // yet): take the exact maximum, rescale what has been accumulated, and redo the tile
         load_s<NS>(t_s, cur);
@@ -304,11 +377,11 @@ __device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j, bool f
         float alpha = 1.0f;
         if (mx > st.m_ref) { alpha = ex2((st.m_ref - mx) * sl2); st.m_ref = mx; st.l_sum *= alpha; }
         if (!first) {
-            // P V of this accumulator's previous key tile has landed.  Its o barrier cannot be a whole phase
-            // behind: S of this tile was seen, so every MMA issued before its Q K^T is complete, and that
-            // includes the P V that last used the previous tile's buffer.
-            const int jp = j - C::kSplit;
-            wait_bar(st.bar_o + 8 * (jp % kSBufs), (jp / kSBufs) & 1, st.abort_flag, st.err_word);
+            // P V of the previous key tile has landed.  Its o barrier cannot be a whole phase behind: S of this
+            // tile was seen, so every MMA issued before its Q K^T is complete, and that includes the P V that
+            // last used the previous tile's buffer.
+            const int gp = g - 1;
+            wait_bar(st.bar_o + 8 * (gp % kSBufs), (gp / kSBufs) & 1, st.abort_flag, st.err_word);
             tc_fence_after();
 #pragma unroll
             for (int cc = 0; cc < C::kMain / 32; ++cc) {
@@ -318,14 +391,6 @@ __device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j, bool f
 #pragma unroll
                 for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
                 tmem_st32(st.t_o + cc * 32, o);
-            }
-            if (C::kTail) {
-                uint32_t o[16];
-                tmem_ld16(st.t_o + C::kMain, o);
-                tc_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                tmem_st16(st.t_o + C::kMain, o);
             }
             tc_wait_st();
         }
@@ -340,11 +405,17 @@ __device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j, bool f
     publish_p(st.bar_p + 8 * buf);
 }
 
+// All warps of the CTA meet after the speculative pass and then agree on the redo flag.
+template <int DH>
+__device__ __forceinline__ void pass_sync() {
+    asm volatile("bar.sync 5, %0;" ::"n"(Cfg<DH>::kThreads) : "memory");
+}
+
 // ---------------------------------------------------------------- softmax warpgroup
 // tile: its query tile; par: which key tiles it takes (j = par, par + kSplit, ...)
 template <int DH>
 __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, int tile, int par, uint8_t *sQ_gen, uint32_t tmem,
-                                             int m_base, int h, int b, int n_tiles, volatile int *abort_flag, float2 *xchg)
+                                             int m_base, int h, int b, int n_tiles, volatile int *abort_flag, volatile int *redo_flag, float2 *xchg)
 {
     using C = Cfg<DH>;
     const int wtid = threadIdx.x & 127;
@@ -375,9 +446,10 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     st.sl2 = p.scale_log2;
     st.l_sum = 0.f;
     st.t_s0 = t_row + tile * C::kSBufs * C::kBlockN;
-    st.t_o = t_row + C::kColO + (tile * C::kSplit + par) * C::kOStride;
+    st.t_o = t_row + C::kColO + tile * C::kOStride;
     st.bar_s = bar.s + 32 * tile; st.bar_p = bar.p + 32 * tile; st.bar_o = bar.o + 32 * tile;
     st.N = p.N; st.n_tiles = n_tiles; st.abort_flag = abort_flag; st.err_word = p.err_word;
+    st.ref_x = &xchg[wtid].x; st.ref_bar = 3 + tile; st.redo_flag = redo_flag;
 
     const int m = m_base + wtid;
     int tok = -1;
@@ -387,87 +459,77 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     }
 
     st.m_ref = -INFINITY;
-    int j_last = -1;
-    for (int j = par; j < n_tiles; j += C::kSplit) { softmax_step<DH>(st, j, j == par); j_last = j; }
-
-    // ------------------------------------------------ epilogue: (merge,) normalise and scatter
-    if (j_last >= 0) wait_bar(st.bar_o + 8 * (j_last % C::kSBufs), (j_last / C::kSBufs) & 1, abort_flag, p.err_word);
-    tc_fence_after();
-    float w_own = 1.0f, w_other = 0.f, l_sum = st.l_sum, m_ref = st.m_ref;
-    uint32_t t_other = st.t_o;
+    if (C::kSplit == 2 && par == 1) {
+        // the even-tile warpgroup takes the exact row maxima of key tile 0 and hands them over
+        if (tile == 0) asm volatile("bar.sync 3, 256;" ::: "memory");
+        else asm volatile("bar.sync 4, 256;" ::: "memory");
+        st.m_ref = *st.ref_x;
+    }
+    for (int j = par; j < n_tiles; j += C::kSplit) softmax_step<DH, kSpeculate>(st, j, j);
+    wait_bar(st.bar_o + 24, 0, abort_flag, p.err_word);          // every P V of this query tile has landed
     if constexpr (C::kSplit == 2) {
-        // the odd-tile warpgroup hands its reference and row sum to the even-tile one, which merges both accumulators
-        if (par == 1) xchg[wtid] = make_float2(st.m_ref, j_last >= 0 ? st.l_sum : 0.f);
-        tc_fence_before();
-        if (tile == 0) asm volatile("bar.sync 1, 256;" ::: "memory");
-        else asm volatile("bar.sync 2, 256;" ::: "memory");
-        if (par == 1) return;
-        tc_fence_after();
-        const float2 other = xchg[wtid];
-        if (other.y > 0.f) {
-            m_ref = fmaxf(st.m_ref, other.x);
-            w_own = ex2((st.m_ref - m_ref) * st.sl2);
-            w_other = ex2((other.x - m_ref) * st.sl2);
-            l_sum = st.l_sum * w_own + other.y * w_other;
-            t_other = t_row + C::kColO + (tile * C::kSplit + 1) * C::kOStride;
+        pass_sync<DH>();
+        if (*redo_flag) {
+            // a tile overflowed somewhere in the CTA: exact row maxima first, then the whole pass again
+            st.m_ref = -INFINITY;
+            for (int j = par; j < n_tiles; j += C::kSplit) softmax_step<DH, kMaxOnly>(st, j, n_tiles + j);
+            xchg[wtid + par * kBlockM].x = st.m_ref;
+            if (tile == 0) asm volatile("bar.sync 1, 256;" ::: "memory");
+            else asm volatile("bar.sync 2, 256;" ::: "memory");
+            st.m_ref = fmaxf(xchg[wtid].x, xchg[wtid + kBlockM].x);
+            st.l_sum = 0.f;
+            for (int j = par; j < n_tiles; j += C::kSplit) softmax_step<DH, kExact>(st, j, 2 * n_tiles + j);
+            wait_bar(st.bar_o + 24, 1, abort_flag, p.err_word);
         }
     }
-    const bool merge = C::kSplit == 2 && __any_sync(0xffffffffu, w_other != 0.f);   // warp-uniform: the partner has tiles or not
+
+    // ------------------------------------------------ epilogue: normalise and scatter
+    tc_fence_after();
+    float l_sum = st.l_sum;
+    int col0 = 0, ncol = C::kMain;                               // O columns this thread writes
+    if constexpr (C::kSplit == 2) {
+        // both warpgroups accumulated into one O against one reference: add the row sums, split the columns
+        xchg[wtid + par * kBlockM].y = st.l_sum;
+        if (tile == 0) asm volatile("bar.sync 1, 256;" ::: "memory");
+        else asm volatile("bar.sync 2, 256;" ::: "memory");
+        l_sum = xchg[wtid].y + xchg[wtid + kBlockM].y;
+        ncol = C::kMain / 2;
+        col0 = par * ncol;
+    }
     const float inv_l = 1.0f / l_sum;
-    w_own *= inv_l;
-    w_other *= inv_l;
     __nv_bfloat16 *dst = nullptr;
     if (tok >= 0 && !*abort_flag) {
         const size_t orow = p.compact ? ((size_t)b * p.M + m) : ((size_t)b * p.N_tok + tok);
         dst = p.out + (orow * p.H + h) * DH;
-        if (p.lse_out) {
+        if (p.lse_out && par == 0) {
             const size_t li = p.compact ? (((size_t)b * p.H + h) * p.M + m) : (((size_t)b * p.H + h) * p.N_tok + tok);
-            p.lse_out[li] = m_ref * p.scale + logf(l_sum);
+            p.lse_out[li] = st.m_ref * p.scale + logf(l_sum);
         }
     }
-#pragma unroll
-    for (int cc = 0; cc < C::kMain / 32; ++cc) {
+    for (int c = col0; c < col0 + ncol; c += 32) {
         uint32_t o[32];
-        tmem_ld32(st.t_o + cc * 32, o);
+        tmem_ld32(st.t_o + c, o);
         tc_wait_ld();
-        float f[32];
-#pragma unroll
-        for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(o[i]) * w_own;
-        if (merge) {
-            tmem_ld32(t_other + cc * 32, o);
-            tc_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) f[i] = fmaf(__uint_as_float(o[i]), w_other, f[i]);
-        }
         if (dst) {
 #pragma unroll
             for (int v = 0; v < 4; ++v) {
                 uint32_t w[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    __nv_bfloat162 v2 = __floats2bfloat162_rn(f[v * 8 + 2 * i], f[v * 8 + 2 * i + 1]);
+                    __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(o[v * 8 + 2 * i]) * inv_l, __uint_as_float(o[v * 8 + 2 * i + 1]) * inv_l);
                     w[i] = *reinterpret_cast<uint32_t *>(&v2);
                 }
-                *reinterpret_cast<uint4 *>(dst + cc * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                *reinterpret_cast<uint4 *>(dst + c + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
             }
         }
     }
-    if (C::kTail) {
+    if (C::kTail && par == C::kSplit - 1) {
         uint32_t o[8], w[4];
         tmem_ld8(st.t_o + C::kMain, o);
         tc_wait_ld();
-        float f[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(o[i]) * w_own;
-        if (merge) {
-            tmem_ld8(t_other + C::kMain, o);
-            tc_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 8; ++i) f[i] = fmaf(__uint_as_float(o[i]), w_other, f[i]);
-        }
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            __nv_bfloat162 v2 = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+            __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(o[2 * i]) * inv_l, __uint_as_float(o[2 * i + 1]) * inv_l);
             w[i] = *reinterpret_cast<uint32_t *>(&v2);
         }
         if (dst) *reinterpret_cast<uint4 *>(dst + C::kMain) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -480,11 +542,12 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                    const __grid_constant__ CUtensorMap tmap_k_tail, const __grid_constant__ CUtensorMap tmap_v_tail, const Params p)
 {
     using C = Cfg<DH>;
-    constexpr int kSBufs = C::kSBufs;
+    constexpr int kSBufs = C::kSBufs, kAhead = C::kAhead;
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
-    __shared__ float2 xchg[kTilesM][kBlockM];
+    __shared__ volatile int redo_flag;
+    __shared__ float2 xchg[kTilesM][2 * kBlockM];
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -510,6 +573,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 
     if (tid == 0) {
         abort_flag = 0;
+        redo_flag = 0;
         for (int t = 0; t < kTilesM; ++t) {
             mbar_init(bar.q + 8 * t, 128 * C::kSplit);
             for (int u = 0; u < 4; ++u) {
@@ -537,7 +601,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         const int tile = wg / C::kSplit, par = wg % C::kSplit;
         if (tile < q_tiles)
             softmax_role<DH>(p, bar, tile, par, smem_gen + tile * C::kQTileBytes, tmem, m0 + tile * kBlockM, h, b, n_tiles,
-                             &abort_flag, xchg[tile]);
+                             &abort_flag, &redo_flag, xchg[tile]);
+        else if constexpr (C::kSplit == 2) pass_sync<DH>();
     } else if (warp == kProducerWarp) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
         // ------------------------------------------------ TMA producer (warp-uniform, one elected lane issues)
@@ -545,9 +610,10 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             prefetch_tensormap(&tmap_k); prefetch_tensormap(&tmap_v);
             if (C::kTail) { prefetch_tensormap(&tmap_k_tail); prefetch_tensormap(&tmap_v_tail); }
         }
-        auto load_k = [&](int j) {
-            const int st = j % C::kStagesK;
-            wait_bar(bar.ke + 8 * st, ((j / C::kStagesK) & 1) ^ 1, &abort_flag, p.err_word);
+        // g: running count of K (or V) tiles over all passes: stage g % kStages, phase (g / kStages) & 1
+        auto load_k = [&](int g, int j) {
+            const int st = g % C::kStagesK;
+            wait_bar(bar.ke + 8 * st, ((g / C::kStagesK) & 1) ^ 1, &abort_flag, p.err_word);
             if (elect_one()) {
                 mbar_arrive_expect_tx(bar.kf + 8 * st, C::kLoadBytes);
 #pragma unroll
@@ -558,9 +624,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             }
             __syncwarp();
         };
-        auto load_v = [&](int j) {
-            const int st = j % C::kStagesV;
-            wait_bar(bar.ve + 8 * st, ((j / C::kStagesV) & 1) ^ 1, &abort_flag, p.err_word);
+        auto load_v = [&](int g, int j) {
+            const int st = g % C::kStagesV;
+            wait_bar(bar.ve + 8 * st, ((g / C::kStagesV) & 1) ^ 1, &abort_flag, p.err_word);
             if (elect_one()) {
                 mbar_arrive_expect_tx(bar.vf + 8 * st, C::kLoadBytes);
 #pragma unroll
@@ -571,25 +637,40 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             }
             __syncwarp();
         };
-        // K runs kSBufs tiles ahead of V: K_{j+kSBufs} is consumed right after V_j
-        for (int j = 0; j < kSBufs && j < n_tiles; ++j) load_k(j);
-        for (int j = 0; j < n_tiles; ++j) {
-            if (j + kSBufs < n_tiles) load_k(j + kSBufs);
-            load_v(j);
+        // K runs kAhead tiles ahead of V: K_{j+kAhead} is consumed next to V_j.  The max-only pass needs no V.
+        auto produce_pass = [&](int pass) {
+            const int gk0 = pass * n_tiles, gv0 = (pass == kExact) ? n_tiles : 0;
+            for (int j = 0; j < kAhead && j < n_tiles; ++j) load_k(gk0 + j, j);
+            for (int j = 0; j < n_tiles; ++j) {
+                if (j + kAhead < n_tiles) load_k(gk0 + j + kAhead, j + kAhead);
+                if (pass != kMaxOnly) load_v(gv0 + j, j);
+            }
+        };
+        produce_pass(kSpeculate);
+        int k_loads = n_tiles, v_loads = n_tiles;
+        if constexpr (C::kSplit == 2) {
+            pass_sync<DH>();
+            if (redo_flag) {
+                produce_pass(kMaxOnly);
+                produce_pass(kExact);
+                k_loads = 3 * n_tiles; v_loads = 2 * n_tiles;
+            }
         }
         // every copy issued above must have landed before the CTA's shared memory is released
-        for (int j = (n_tiles > C::kStagesK ? n_tiles - C::kStagesK : 0); j < n_tiles; ++j)
-            wait_bar(bar.kf + 8 * (j % C::kStagesK), (j / C::kStagesK) & 1, &abort_flag, p.err_word);
-        for (int j = (n_tiles > C::kStagesV ? n_tiles - C::kStagesV : 0); j < n_tiles; ++j)
-            wait_bar(bar.vf + 8 * (j % C::kStagesV), (j / C::kStagesV) & 1, &abort_flag, p.err_word);
+        for (int g = (k_loads > C::kStagesK ? k_loads - C::kStagesK : 0); g < k_loads; ++g)
+            wait_bar(bar.kf + 8 * (g % C::kStagesK), (g / C::kStagesK) & 1, &abort_flag, p.err_word);
+        for (int g = (v_loads > C::kStagesV ? v_loads - C::kStagesV : 0); g < v_loads; ++g)
+            wait_bar(bar.vf + 8 * (g % C::kStagesV), (g / C::kStagesV) & 1, &abort_flag, p.err_word);
     } else if (warp == kIssuerWarp || warp == kIssuerWarp + 1) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
         // ------------------------------------------------ MMA issuer (warp-uniform, one elected lane issues)
         constexpr uint32_t idesc_qk = idesc_bf16(kBlockM, kBlockN, false);
         constexpr uint32_t idesc_pv = idesc_bf16(kBlockM, C::kMain, true);
         constexpr uint32_t idesc_pv_tail = idesc_bf16(kBlockM, 16, true);
-        auto issue_qk = [&](int t, int j, uint32_t kbase) {        // S[t][j % kSBufs] = Q_t K_j^T  (one elected lane)
-            const int u = j % kSBufs;
+        // S[t][g % kSBufs] = Q_t K^T of the key tile in shared memory at kbase (one elected lane); g counts the
+        // S-buffer uses of the query tile over all passes
+        auto issue_qk = [&](int t, int g, uint32_t kbase) {
+            const int u = g % kSBufs;
 #pragma unroll
             for (int ks = 0; ks < C::kMain / 16; ++ks)
                 mma_ss(tmem + (t * kSBufs + u) * kBlockN,
@@ -606,54 +687,81 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         // sub-partition's issuer slow the exponentials of the softmax warps that live there, so the load is spread.
         // All MMAs that touch one S buffer / O accumulator come from one thread, in order.
         const int t = warp - kIssuerWarp;
-        if (t < q_tiles) {
-            // prologue: S of the first kSBufs key tiles
-            wait_bar(bar.q + 8 * t, 0, &abort_flag, p.err_word);
-            for (int j = 0; j < kSBufs && j < n_tiles; ++j) {
-                const int st = j % C::kStagesK;
-                wait_bar(bar.kf + 8 * st, (j / C::kStagesK) & 1, &abort_flag, p.err_word);
+        const uint32_t o_col = C::kColO + t * C::kOStride;
+        auto issue_pass = [&](int pass) {
+            const bool with_v = pass != kMaxOnly;
+            const int gs0 = pass * n_tiles, gk0 = pass * n_tiles, gv0 = (pass == kExact) ? n_tiles : 0;
+            // prologue: S of the first kAhead key tiles
+            for (int j = 0; j < kAhead && j < n_tiles; ++j) {
+                const int st = (gk0 + j) % C::kStagesK;
+                wait_bar(bar.kf + 8 * st, ((gk0 + j) / C::kStagesK) & 1, &abort_flag, p.err_word);
                 tc_fence_after();
                 if (elect_one()) {
-                    issue_qk(t, j, sK + st * C::kTileBytes);
+                    issue_qk(t, gs0 + j, sK + st * C::kTileBytes);
                     tc_commit(bar.ke + 8 * st);
                 }
                 __syncwarp();
             }
             for (int j = 0; j < n_tiles; ++j) {
-                const int sv = j % C::kStagesV;
+                const int sv = (gv0 + j) % C::kStagesV;
                 const uint32_t vbase = sV + sv * C::kTileBytes;
-                const int u = j % kSBufs;
-                const bool more = j + kSBufs < n_tiles;
-                const int sk = (j + kSBufs) % C::kStagesK;
-                const uint32_t o_col = C::kColO + (t * C::kSplit + (j % C::kSplit)) * C::kOStride;   // this tile's accumulator
-                wait_bar(bar.vf + 8 * sv, (j / C::kStagesV) & 1, &abort_flag, p.err_word);
-                if (more) wait_bar(bar.kf + 8 * sk, ((j + kSBufs) / C::kStagesK) & 1, &abort_flag, p.err_word);
-                wait_bar(bar.p + 32 * t + 8 * u, (j / kSBufs) & 1, &abort_flag, p.err_word);
+                const int u = (gs0 + j) % kSBufs;
+                const bool more = j + kAhead < n_tiles;
+                const int sk = (gk0 + j + kAhead) % C::kStagesK;
+                if (more) wait_bar(bar.kf + 8 * sk, ((gk0 + j + kAhead) / C::kStagesK) & 1, &abort_flag, p.err_word);
+                if constexpr (kSBufs > kAhead) {
+                    // a third S buffer: the one of key tile j-1 was consumed by the P V issued last (in-order pipe),
+                    // so S of key tile j+2 is started before waiting for P of tile j
+                    tc_fence_after();
+                    if (more && elect_one()) {
+                        issue_qk(t, gs0 + j + kAhead, sK + sk * C::kTileBytes);
+                        tc_commit(bar.ke + 8 * sk);
+                    }
+                    __syncwarp();
+                }
+                if (with_v) wait_bar(bar.vf + 8 * sv, ((gv0 + j) / C::kStagesV) & 1, &abort_flag, p.err_word);
+                // P of key tile j is in TMEM (max-only pass: S of key tile j has been read)
+                wait_bar(bar.p + 32 * t + 8 * u, ((gs0 + j) / kSBufs) & 1, &abort_flag, p.err_word);
                 tc_fence_after();
                 if (elect_one()) {
+                    if (with_v) {
 #pragma unroll
-                    for (int ks = 0; ks < kBlockN / 16; ++ks) {
-                        mma_ts(tmem + o_col, tmem + (t * kSBufs + u) * kBlockN + ks * 8,
-                               smem_desc(vbase + ks * 2048, C::kChunkBytes, 1024, kSwizzle128B),
-                               idesc_pv, (j >= C::kSplit || ks > 0) ? 1u : 0u);
-                        if (C::kTail)  // O columns 64..79 from the 16-column chunk of V
-                            mma_ts(tmem + o_col + C::kMain, tmem + (t * kSBufs + u) * kBlockN + ks * 8,
-                                   smem_desc(vbase + C::kChunks * C::kChunkBytes + ks * 512, 256, 256, kSwizzle32B),
-                                   idesc_pv_tail, (j >= C::kSplit || ks > 0) ? 1u : 0u);
+                        for (int ks = 0; ks < kBlockN / 16; ++ks) {
+                            mma_ts(tmem + o_col, tmem + (t * kSBufs + u) * kBlockN + ks * 8,
+                                   smem_desc(vbase + ks * 2048, C::kChunkBytes, 1024, kSwizzle128B),
+                                   idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+                            if (C::kTail)  // O columns 64..79 from the 16-column chunk of V
+                                mma_ts(tmem + o_col + C::kMain, tmem + (t * kSBufs + u) * kBlockN + ks * 8,
+                                       smem_desc(vbase + C::kChunks * C::kChunkBytes + ks * 512, 256, 256, kSwizzle32B),
+                                       idesc_pv_tail, (j > 0 || ks > 0) ? 1u : 0u);
+                        }
+                        if (kSBufs == kAhead) tc_commit(bar.o + 32 * t + 8 * u);
+                        tc_commit(bar.ve + 8 * sv);
+                        if (j == n_tiles - 1) tc_commit(bar.o + 32 * t + 24);      // the pass is done for this query tile
                     }
-                    tc_commit(bar.o + 32 * t + 8 * u);
-                    tc_commit(bar.ve + 8 * sv);
-                    // the S buffer just consumed as P is free again (in-order pipe): refill it with key tile j+kSBufs
-                    if (more) {
-                        issue_qk(t, j + kSBufs, sK + sk * C::kTileBytes);
+                    // two S buffers: the one just consumed as P is free again (in-order pipe), refill it with key tile j+2
+                    if (kSBufs == kAhead && more) {
+                        issue_qk(t, gs0 + j + kAhead, sK + sk * C::kTileBytes);
                         tc_commit(bar.ke + 8 * sk);
                     }
                 }
                 __syncwarp();
             }
+        };
+        if (t < q_tiles) {
+            wait_bar(bar.q + 8 * t, 0, &abort_flag, p.err_word);
+            issue_pass(kSpeculate);
+        }
+        if constexpr (C::kSplit == 2) {
+            pass_sync<DH>();
+            if (redo_flag && t < q_tiles) {
+                issue_pass(kMaxOnly);
+                issue_pass(kExact);
+            }
         }
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
+        if constexpr (C::kSplit == 2) pass_sync<DH>();
     }
 
     tc_fence_before();

@@ -254,6 +254,17 @@ def test_attn_peaked_softmax_triggers_rescaling(oracle):
 
 
 @pytest.mark.parametrize("d", [64, 72, 128])
+def test_attn_reference_maximum_far_too_low_is_repaired_exactly(oracle, d):
+    # logits of order +-250: in most rows a later key tile beats the first tile's maximum by more than 60 nats,
+    # past every speculation limit of the kernel (in-place rescale at 128, a redo of the whole CTA at 64 / 72);
+    # three CTAs per head, the last one with a single query tile, ragged last key tile
+    _attn_case(oracle, 1, 2, 900, d, 600, seed=20 + d, amp=8.0)
+    # a single key tile and exactly two: the odd-tile warpgroup has nothing, or one tile, to contribute
+    _attn_case(oracle, 1, 1, 40, d, 40, seed=21 + d, amp=8.0)
+    _attn_case(oracle, 2, 1, 100, d, 70, seed=22 + d, amp=8.0)
+
+
+@pytest.mark.parametrize("d", [64, 72, 128])
 def test_attn_select_q_and_k_ablation(oracle, d):
     """kv_idx: the softmax runs over the listed keys/values only (the ablation that also masks K and V)."""
     rng = np.random.default_rng(20 + d)
