@@ -3,31 +3,36 @@
 // Section 3.2 "Sparse Attention").
 //
 // One CTA per (256 selected queries, head, batch): two 128-row query tiles that share every
-// K/V tile of 64 keys.  Warp roles:
+// K/V tile of 64 keys (48 at head_dim 72).  Warp roles:
 //   softmax warpgroups (one thread per query row): gather the tile's Q rows into 128B-swizzled shared
 //              memory, then per key tile read S from TMEM, exponentiate in the log2 domain against a
-//              running reference maximum, write P (bf16) back to TMEM over S, and at the end normalise
-//              O and scatter it to the rows q_idx names.  head_dim 72 / 128: one warpgroup per query
-//              tile.  head_dim 64: two per query tile; even key tiles go to one and odd ones to the
-//              other, each with its own reference, row sum and O accumulator (a split over keys inside
-//              the CTA, merged in the epilogue), which puts four softmax warps on every SM sub-partition
-//              and hides the serial chain of a key tile (wait, load, exponentials, sum, pack, publish);
+//              reference maximum, write P (bf16) back to TMEM over S, and at the end normalise O and
+//              scatter it to the rows q_idx names;
 //   one warp   TMA producer: K and V tiles into multi-stage swizzled buffers;
 //   two warps  tcgen05.mma issuers, one per query tile: S = Q K^T (SS, K-major operands), O += P V (P from
 //              TMEM, V as an MN-major shared-memory operand); the first owns the TMEM allocation;
 //   one warp   only donates registers (setmaxnreg moves registers to the softmax warps).
-// Every query tile has two S buffers; a buffer is refilled with key tile j+2 as soon as P of tile j has
-// been consumed (the tensor pipe executes one thread's MMAs in order).
 //
-// The softmax is bound by the exponentials (XU pipe, 16 per clock per SM) and by the latencies of
-// its own chain, so the common path of a key tile is kept to: load S, one FFMA + ex2 per element,
-// sum, pack, store.  The reference maximum is the exact row maximum of the first key tile and is
-// then only checked through the tile's sum of exponentials: while that sum stays below 2^16 the
-// tile is accepted as it is (the probabilities are relative to a stale maximum, which the final
-// normalisation cancels; fp32 has the range).  Otherwise the exact maximum is taken and the row
-// sum and the O accumulator are rescaled before the tile is redone.
+// head_dim 128: one softmax warpgroup and two S buffers per query tile; a buffer is refilled with key
+// tile j+2 as soon as P of tile j has been consumed (the tensor pipe executes one thread's MMAs in order).
+// head_dim 64 / 72: two softmax warpgroups per query tile, which puts four softmax warps on every SM
+// sub-partition and hides the serial chain of a key tile (wait, load, exponentials, sum, pack, publish).
+// Even key tiles go to one warpgroup and odd ones to the other; both work against the same reference
+// maximum and their P tiles accumulate into ONE O accumulator, which leaves TMEM room for three S buffers
+// per query tile: S of key tile j+2 is computed while tiles j and j+1 are in the softmax.
 //
-// TMEM columns: S/P of (tile t, buffer u) at (2t+u)*64; the O accumulators from column 256.
+// The softmax is bound by the exponentials (XU pipe, 16 per clock per SM), by the issue slots and by the
+// latencies of its own chain, so the common path of a key tile is kept to: load S, one FFMA + one
+// exponential per element, sum, pack, store.  At head_dim 64 six of every sixteen exponentials are a
+// cubic on the FMA pipe instead of ex2 on the XU.  The reference maximum is the exact row maximum of key
+// tile 0 and is then only checked through each tile's sum of exponentials: while that sum stays below a
+// limit the tile is accepted as it is (the probabilities are relative to a stale maximum, which the final
+// normalisation cancels; fp32 and bf16 have the range).  Otherwise, at head_dim 128 the exact maximum is
+// taken and the row sum and the O accumulator are rescaled in place before the tile is redone; at 64 / 72,
+// where the accumulator is shared, the CTA raises a flag, finishes the pass, and redoes its work in two
+// more passes over the keys: exact row maxima first, then the softmax against them.
+//
+// TMEM columns: S/P of (tile t, buffer u) at (kSBufs t + u) * kBlockN; the O accumulators behind them.
 // The producer and issuer warps run warp-uniform code and elect one lane per instruction, so
 // that descriptors and addresses stay in uniform registers (a lone diverged thread issues
 // tcgen05.mma several times slower).  Every mbarrier wait is bounded; on a timeout the CTA raises
