@@ -4,22 +4,22 @@
 //
 // One CTA per (256 selected queries, head, batch): two 128-row query tiles that share every
 // K/V tile of 64 keys (48 at head_dim 72).  Warp roles:
-//   softmax warpgroups (one thread per query row): gather the tile's Q rows into 128B-swizzled shared
-//              memory, then per key tile read S from TMEM, exponentiate in the log2 domain against a
-//              reference maximum, write P (bf16) back to TMEM over S, and at the end normalise O and
-//              scatter it to the rows q_idx names;
+//   softmax warpgroups (one thread per query row), two per query tile: gather the tile's Q rows into
+//              128B-swizzled shared memory, then per key tile read S from TMEM, exponentiate in the log2
+//              domain against a reference maximum, write P (bf16) back to TMEM over S, and at the end
+//              normalise O and scatter it to the rows q_idx names;
 //   one warp   TMA producer: K and V tiles into multi-stage swizzled buffers;
 //   two warps  tcgen05.mma issuers, one per query tile: S = Q K^T (SS, K-major operands), O += P V (P from
 //              TMEM, V as an MN-major shared-memory operand); the first owns the TMEM allocation;
 //   one warp   only donates registers (setmaxnreg moves registers to the softmax warps).
 //
-// head_dim 128: one softmax warpgroup and two S buffers per query tile; a buffer is refilled with key
-// tile j+2 as soon as P of tile j has been consumed (the tensor pipe executes one thread's MMAs in order).
-// head_dim 64 / 72: two softmax warpgroups per query tile, which puts four softmax warps on every SM
-// sub-partition and hides the serial chain of a key tile (wait, load, exponentials, sum, pack, publish).
-// Even key tiles go to one warpgroup and odd ones to the other; both work against the same reference
-// maximum and their P tiles accumulate into ONE O accumulator, which leaves TMEM room for three S buffers
-// per query tile: S of key tile j+2 is computed while tiles j and j+1 are in the softmax.
+// Two softmax warpgroups per query tile put four softmax warps on every SM sub-partition, which hides the
+// serial chain of a key tile (wait, load, exponentials, sum, pack, publish).  Even key tiles go to one
+// warpgroup and odd ones to the other; both work against the same reference maximum and their P tiles
+// accumulate into ONE O accumulator per query tile.  That leaves TMEM room for three S buffers per query
+// tile at head_dim 64 / 72 (S of key tile j+2 is computed while tiles j and j+1 are in the softmax) and
+// for two at head_dim 128 (a buffer is refilled with key tile j+2 as soon as P of tile j has been
+// consumed; the tensor pipe executes one thread's MMAs in order).
 //
 // The softmax is bound by the exponentials (XU pipe, 16 per clock per SM), by the issue slots and by the
 // latencies of its own chain, so the common path of a key tile is kept to: load S, one FFMA + one
@@ -27,10 +27,9 @@
 // cubic on the FMA pipe instead of ex2 on the XU.  The reference maximum is the exact row maximum of key
 // tile 0 and is then only checked through each tile's sum of exponentials: while that sum stays below a
 // limit the tile is accepted as it is (the probabilities are relative to a stale maximum, which the final
-// normalisation cancels; fp32 and bf16 have the range).  Otherwise, at head_dim 128 the exact maximum is
-// taken and the row sum and the O accumulator are rescaled in place before the tile is redone; at 64 / 72,
-// where the accumulator is shared, the CTA raises a flag, finishes the pass, and redoes its work in two
-// more passes over the keys: exact row maxima first, then the softmax against them.
+// normalisation cancels; fp32 and bf16 have the range).  Otherwise the CTA raises a flag, finishes the
+// pass, and redoes its work in two more passes over the keys: exact row maxima first, then the softmax
+// against them (the accumulator is shared by two warpgroups, so it is not rescaled in place).
 //
 // TMEM columns: S/P of (tile t, buffer u) at (kSBufs t + u) * kBlockN; the O accumulators behind them.
 // The producer and issuer warps run warp-uniform code and elect one lane per instruction, so
@@ -49,6 +48,11 @@ using namespace ptx;
 
 constexpr int kBlockM = 128;                     // rows of one query tile
 constexpr int kTilesM = 2;                       // query tiles per CTA
+constexpr int kSplit = 2;                        // softmax warpgroups per query tile: one takes the even key tiles, one the odd
+// A tile's sum of exponentials above this means that the reference maximum is too low.  fp32 and bf16 share the
+// exponent range, so the limit only has to keep row sums and accumulators far from overflow; it is as high as that
+// allows, because a redo costs the CTA two more passes over the keys.
+constexpr float kTileSumLimit = 1152921504606846976.0f;   // 2^60
 constexpr uint32_t kTmemCols = 512;
 constexpr uint64_t kWaitLimitNs = 1000000000ull; // bounded waits: one second
 
@@ -59,24 +63,17 @@ template <int DH> struct Cfg {
     static constexpr int kTail = DH - kMain;
     static constexpr int kTailPad = kTail ? 16 : 0;
     static_assert(kTail == 0 || kTail == 8, "head_dim must be 64, 72 or 128");
-    // softmax warpgroups per query tile: at head_dim 64 even key tiles go to one and odd ones to the other,
-    // each with its own running reference, row sum and O accumulator (merged in the epilogue)
-    static constexpr int kSplit = (DH == 128) ? 1 : 2;
-    // keys per K/V tile = columns of an S buffer.  64, but 48 at head_dim 72: four O accumulators of 80 columns
-    // leave 192 TMEM columns for the four S buffers
+    // keys per K/V tile = columns of an S buffer.  64, but 48 at head_dim 72 (two O accumulators of 80 columns leave
+    // 352 TMEM columns for the S buffers)
     static constexpr int kBlockN = (DH == 72) ? 48 : 64;
-    // S buffers per query tile.  Split: three, used round-robin by the two warpgroups, so that S of key tile j+2
-    // is produced while tiles j and j+1 are in the softmax; the warpgroups then share one O accumulator
-    static constexpr int kSBufs = (kSplit == 2) ? 3 : 2;
+    // S buffers per query tile, used round-robin by its two softmax warpgroups.  Three where TMEM has the room: S
+    // of key tile j+2 is then produced while tiles j and j+1 are in the softmax.  head_dim 128 has room for two.
+    static constexpr int kSBufs = (DH == 128) ? 2 : 3;
     // exponentials per 16 that are computed on the FMA pipe instead of the XU (measured: 6 is best at head_dim 64,
     // none at 72 and 128, where the tensor pipe has less slack)
     static constexpr int kPolyOf16 = (DH == 64) ? 6 : 0;
-    // a tile's sum of exponentials above this means the reference maximum is too low.  fp32 and bf16 share the
-    // exponent range, so the limit only has to keep row sums and accumulators far from overflow; with the
-    // split it is as high as that allows, because a redo costs the CTA two more passes over the keys
-    static constexpr float kTileSumLimit = (kSplit == 2) ? 1152921504606846976.0f /* 2^60 */ : 65536.0f;
-    static constexpr int kAhead = 2;                              // Q K^T runs this many key tiles ahead of P V
     static constexpr int kSoftmaxWarps = 4 * kTilesM * kSplit;
+    static constexpr int kAhead = 2;                              // Q K^T runs this many key tiles ahead of P V
     static constexpr int kThreads = (kSoftmaxWarps + 4) * 32;     // + producer, two issuers, one register donor
     static constexpr uint32_t kColO = kTilesM * kSBufs * kBlockN; // first O column
     static constexpr uint32_t kOStride = (DH == 64) ? 64 : (DH == 72) ? 80 : 128;   // columns between O accumulators
@@ -84,7 +81,7 @@ template <int DH> struct Cfg {
     // setmaxnreg only redistributes what the CTA got at launch: an increase that the decreases of
     // the last warpgroup cannot cover would block forever
     static constexpr int kRegsLaunch = (65536 / kThreads) / 8 * 8;
-    static constexpr int kRegsSoftmax = (kSplit == 2) ? 112 : 232, kRegsOther = (kSplit == 2) ? 32 : 40;
+    static constexpr int kRegsSoftmax = 112, kRegsOther = 32;
     static_assert(kRegsSoftmax * kSoftmaxWarps * 32 + kRegsOther * 128 <= kRegsLaunch * kThreads, "setmaxnreg budget");
     static constexpr int kChunks = kMain / 64;                    // 64-column (128-byte) swizzle chunks
     static constexpr int kQChunkBytes = kBlockM * 128;            // 128 query rows x 128 bytes
@@ -96,7 +93,7 @@ template <int DH> struct Cfg {
     static constexpr int kTileBytes = (kLoadBytes + 1023) / 1024 * 1024;    // stage size (keeps the swizzle alignment)
     static_assert(kQTileBytes % 1024 == 0 && kTileBytes % 1024 == 0, "tiles keep the 1024-byte swizzle alignment");
     static constexpr int kStagesK = (DH == 128) ? 5 : 6;
-    static constexpr int kStagesV = (DH == 128) ? 5 : 6;
+    static constexpr int kStagesV = (DH == 128) ? 4 : 6;
     static_assert(kStagesK > kAhead, "K runs kAhead tiles ahead");
     static constexpr int kBarBytes = 512;
     static constexpr int kSmemBytes = kQTileBytes * kTilesM + kTileBytes * (kStagesK + kStagesV) + kBarBytes + 1024;
@@ -199,13 +196,14 @@ __device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, volatile
 
 struct Bars {
     uint32_t q;                     // [kTilesM]
-    uint32_t s, p, o;               // [kTilesM][4]: one per S buffer (o: P V of the tile in that buffer has landed)
+    uint32_t s, p;                  // [kTilesM][4]: one per S buffer (S is there; P is there)
+    uint32_t done;                  // [kTilesM]: every P V of the pass has landed
     uint32_t kf, ke, vf, ve;        // [stages]
 };
 
 template <int DH> struct SoftmaxState {
     float sl2, m_ref, l_sum;
-    uint32_t t_s0, t_o, bar_s, bar_p, bar_o;
+    uint32_t t_s0, t_o, bar_s, bar_p, bar_done;
     int N, n_tiles;
     float *ref_x;                   // split: the reference of this thread's row, shared by the tile's two warpgroups
     int ref_bar;                    // split: named barrier on which the reference is handed over
@@ -259,19 +257,6 @@ __device__ __forceinline__ float row_max(const float (&s)[NS]) {
 }
 
 template <int NS>
-__device__ __forceinline__ float row_sum(const float (&s)[NS]) {
-    float a[8];
-#pragma unroll
-    for (int u = 0; u < 8; ++u) a[u] = s[u];
-#pragma unroll
-    for (int i = 8; i < NS; i += 8) {
-#pragma unroll
-        for (int u = 0; u < 8; ++u) a[u] += s[i + u];
-    }
-    return ((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7]));
-}
-
-template <int NS>
 __device__ __forceinline__ void pack_p(const float (&e)[NS], uint32_t (&pk)[NS / 2]) {
 #pragma unroll
     for (int i = 0; i < NS / 2; ++i) {
@@ -298,10 +283,10 @@ __device__ __forceinline__ void publish_p(uint32_t bar) {
     mbar_arrive(bar);
 }
 
-// What a pass over the keys does (split configurations only know kSpeculate unless a tile overflowed):
+// What a pass over the keys does (only kSpeculate unless a tile overflowed):
 //   kSpeculate  exponentials against the exact row maximum of key tile 0; a tile whose sum of exponentials passes
-//               the limit is, without the split, redone after rescaling the accumulator in place, and with the
-//               split (where the accumulator is shared) raises the CTA's redo flag;
+//               the limit raises the CTA's redo flag (the accumulator is shared by two warpgroups, so nothing
+//               is repaired in place);
 //   kMaxOnly    first pass of a redo: only the exact row maxima over all keys are taken;
 //   kExact      second pass of a redo: exponentials against those maxima, nothing can overflow.
 enum { kSpeculate = 0, kMaxOnly = 1, kExact = 2 };
@@ -330,16 +315,14 @@ __device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j, int g)
         mbar_arrive(st.bar_p + 8 * buf);              // S has been read: the buffer may be refilled
         return;
     }
-    const bool first = MODE == kSpeculate && j == 0;
-    if (first) {                                      // the reference starts as the exact maximum of the first key tile
+    if (MODE == kSpeculate && j == 0) {
+        // the reference is the exact maximum of the first key tile; the other warpgroup of this query tile takes the same one
         st.m_ref = row_max<NS>(cur);
-        if constexpr (C::kSplit == 2) {               // ... and the other warpgroup of this query tile takes the same one
-            *st.ref_x = st.m_ref;
-            if (st.ref_bar == 3) asm volatile("bar.arrive 3, 256;" ::: "memory");
-            else asm volatile("bar.arrive 4, 256;" ::: "memory");
-        }
+        *st.ref_x = st.m_ref;
+        if (st.ref_bar == 3) asm volatile("bar.arrive 3, 256;" ::: "memory");
+        else asm volatile("bar.arrive 4, 256;" ::: "memory");
     }
-    float neg = -st.m_ref * sl2;
+    const float neg = -st.m_ref * sl2;
 #pragma unroll
     for (int i = 0; i < NS; i += 2) ffma2(cur[i], cur[i + 1], sl2, neg);
     // kPolyOf16 of every 16 exponentials go to the FMA pipe, the rest to the XU
@@ -368,42 +351,9 @@ __device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j, int g)
     // in the shadow of the sum and the vote
     uint32_t pk[NS / 2];
     pack_p<NS>(cur, pk);
-    if constexpr (MODE == kSpeculate && C::kSplit == 2) {
-        // rare: the reference is too low for this tile.  The accumulator is shared with the other warpgroup, so
-        // nothing is repaired here: the CTA finishes the pass and redoes its work with exact maxima
-        if (__any_sync(0xffffffffu, !(tile_sum <= C::kTileSumLimit))) *st.redo_flag = 1;
-    } else if (MODE == kSpeculate && __any_sync(0xffffffffu, !(tile_sum <= C::kTileSumLimit))) {
-        // rare: the reference maximum is too low for this tile.  S is still intact in TMEM (P is not stored
-        // yet): take the exact maximum, rescale what has been accumulated, and redo the tile
-        load_s<NS>(t_s, cur);
-        wait_s_regs<NS>(cur);
-        mask_tail<NS>(cur, st.N - j * NS);
-        const float mx = row_max<NS>(cur);
-        float alpha = 1.0f;
-        if (mx > st.m_ref) { alpha = ex2((st.m_ref - mx) * sl2); st.m_ref = mx; st.l_sum *= alpha; }
-        if (!first) {
-            // P V of the previous key tile has landed.  Its o barrier cannot be a whole phase behind: S of this
-            // tile was seen, so every MMA issued before its Q K^T is complete, and that includes the P V that
-            // last used the previous tile's buffer.
-            const int gp = g - 1;
-            wait_bar(st.bar_o + 8 * (gp % kSBufs), (gp / kSBufs) & 1, st.abort_flag, st.err_word);
-            tc_fence_after();
-#pragma unroll
-            for (int cc = 0; cc < C::kMain / 32; ++cc) {
-                uint32_t o[32];
-                tmem_ld32(st.t_o + cc * 32, o);
-                tc_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                tmem_st32(st.t_o + cc * 32, o);
-            }
-            tc_wait_st();
-        }
-        neg = -st.m_ref * sl2;
-#pragma unroll
-        for (int i = 0; i < NS; ++i) cur[i] = ex2(fmaf(cur[i], sl2, neg));
-        tile_sum = row_sum<NS>(cur);
-        pack_p<NS>(cur, pk);
+    if constexpr (MODE == kSpeculate) {
+        // rare: the reference is too low for this tile.  The CTA finishes the pass and redoes its work with exact maxima
+        if (__any_sync(0xffffffffu, !(tile_sum <= kTileSumLimit))) *st.redo_flag = 1;
     }
     st.l_sum += tile_sum;
     store_p<NS>(t_s, pk);                         // over the first NS/2 columns of this S buffer
@@ -427,7 +377,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     const int warp = __shfl_sync(0xffffffffu, wtid >> 5, 0);       // warp-uniform
     // gather this tile's Q rows (swizzled, K-major): 16-byte units, unit c of row r
     constexpr int kMainUnits = C::kMain / 8, kUnits = kMainUnits + (C::kTail ? 2 : 0);
-    for (int v = par * 128 + wtid; v < kBlockM * kUnits; v += 128 * C::kSplit) {     // the warpgroups of a tile share the rows
+    for (int v = par * 128 + wtid; v < kBlockM * kUnits; v += 128 * kSplit) {     // the warpgroups of a tile share the rows
         const int r = v / kUnits, c = v - r * kUnits;
         const int m = m_base + r;
         uint4 val = make_uint4(0, 0, 0, 0);
@@ -452,7 +402,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     st.l_sum = 0.f;
     st.t_s0 = t_row + tile * C::kSBufs * C::kBlockN;
     st.t_o = t_row + C::kColO + tile * C::kOStride;
-    st.bar_s = bar.s + 32 * tile; st.bar_p = bar.p + 32 * tile; st.bar_o = bar.o + 32 * tile;
+    st.bar_s = bar.s + 32 * tile; st.bar_p = bar.p + 32 * tile; st.bar_done = bar.done + 8 * tile;
     st.N = p.N; st.n_tiles = n_tiles; st.abort_flag = abort_flag; st.err_word = p.err_word;
     st.ref_x = &xchg[wtid].x; st.ref_bar = 3 + tile; st.redo_flag = redo_flag;
 
@@ -464,43 +414,37 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     }
 
     st.m_ref = -INFINITY;
-    if (C::kSplit == 2 && par == 1) {
+    if (par == 1) {
         // the even-tile warpgroup takes the exact row maxima of key tile 0 and hands them over
         if (tile == 0) asm volatile("bar.sync 3, 256;" ::: "memory");
         else asm volatile("bar.sync 4, 256;" ::: "memory");
         st.m_ref = *st.ref_x;
     }
-    for (int j = par; j < n_tiles; j += C::kSplit) softmax_step<DH, kSpeculate>(st, j, j);
-    wait_bar(st.bar_o + 24, 0, abort_flag, p.err_word);          // every P V of this query tile has landed
-    if constexpr (C::kSplit == 2) {
-        pass_sync<DH>();
-        if (*redo_flag) {
-            // a tile overflowed somewhere in the CTA: exact row maxima first, then the whole pass again
-            st.m_ref = -INFINITY;
-            for (int j = par; j < n_tiles; j += C::kSplit) softmax_step<DH, kMaxOnly>(st, j, n_tiles + j);
-            xchg[wtid + par * kBlockM].x = st.m_ref;
-            if (tile == 0) asm volatile("bar.sync 1, 256;" ::: "memory");
-            else asm volatile("bar.sync 2, 256;" ::: "memory");
-            st.m_ref = fmaxf(xchg[wtid].x, xchg[wtid + kBlockM].x);
-            st.l_sum = 0.f;
-            for (int j = par; j < n_tiles; j += C::kSplit) softmax_step<DH, kExact>(st, j, 2 * n_tiles + j);
-            wait_bar(st.bar_o + 24, 1, abort_flag, p.err_word);
-        }
+    for (int j = par; j < n_tiles; j += kSplit) softmax_step<DH, kSpeculate>(st, j, j);
+    wait_bar(st.bar_done, 0, abort_flag, p.err_word);            // every P V of this query tile has landed
+    pass_sync<DH>();
+    if (*redo_flag) {
+        // a tile overflowed somewhere in the CTA: exact row maxima first, then the whole pass again
+        st.m_ref = -INFINITY;
+        for (int j = par; j < n_tiles; j += kSplit) softmax_step<DH, kMaxOnly>(st, j, n_tiles + j);
+        xchg[wtid + par * kBlockM].x = st.m_ref;
+        if (tile == 0) asm volatile("bar.sync 1, 256;" ::: "memory");
+        else asm volatile("bar.sync 2, 256;" ::: "memory");
+        st.m_ref = fmaxf(xchg[wtid].x, xchg[wtid + kBlockM].x);
+        st.l_sum = 0.f;
+        for (int j = par; j < n_tiles; j += kSplit) softmax_step<DH, kExact>(st, j, 2 * n_tiles + j);
+        wait_bar(st.bar_done, 1, abort_flag, p.err_word);
     }
 
     // ------------------------------------------------ epilogue: normalise and scatter
     tc_fence_after();
-    float l_sum = st.l_sum;
-    int col0 = 0, ncol = C::kMain;                               // O columns this thread writes
-    if constexpr (C::kSplit == 2) {
-        // both warpgroups accumulated into one O against one reference: add the row sums, split the columns
-        xchg[wtid + par * kBlockM].y = st.l_sum;
-        if (tile == 0) asm volatile("bar.sync 1, 256;" ::: "memory");
-        else asm volatile("bar.sync 2, 256;" ::: "memory");
-        l_sum = xchg[wtid].y + xchg[wtid + kBlockM].y;
-        ncol = C::kMain / 2;
-        col0 = par * ncol;
-    }
+    // both warpgroups accumulated into one O against one reference: add the row sums, split the columns
+    xchg[wtid + par * kBlockM].y = st.l_sum;
+    if (tile == 0) asm volatile("bar.sync 1, 256;" ::: "memory");
+    else asm volatile("bar.sync 2, 256;" ::: "memory");
+    const float l_sum = xchg[wtid].y + xchg[wtid + kBlockM].y;
+    constexpr int ncol = C::kMain / 2;                           // O columns this thread writes
+    const int col0 = par * ncol;
     const float inv_l = 1.0f / l_sum;
     __nv_bfloat16 *dst = nullptr;
     if (tok >= 0 && !*abort_flag) {
@@ -511,7 +455,9 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
             p.lse_out[li] = st.m_ref * p.scale + logf(l_sum);
         }
     }
-    for (int c = col0; c < col0 + ncol; c += 32) {
+#pragma unroll
+    for (int cc = 0; cc < ncol; cc += 32) {
+        const int c = col0 + cc;
         uint32_t o[32];
         tmem_ld32(st.t_o + c, o);
         tc_wait_ld();
@@ -528,7 +474,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
             }
         }
     }
-    if (C::kTail && par == C::kSplit - 1) {
+    if (C::kTail && par == kSplit - 1) {
         uint32_t o[8], w[4];
         tmem_ld8(st.t_o + C::kMain, o);
         tc_wait_ld();
@@ -561,12 +507,12 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     const uint32_t sV = sK + C::kStagesK * C::kTileBytes;
     const uint32_t bars = sV + C::kStagesV * C::kTileBytes;
     Bars bar;
-    bar.q = bars; bar.s = bars + 16; bar.p = bars + 80; bar.o = bars + 144;
-    bar.kf = bars + 208;
+    bar.q = bars; bar.s = bars + 16; bar.p = bars + 80; bar.done = bars + 144;
+    bar.kf = bars + 160;
     bar.ke = bar.kf + 8 * C::kStagesK;
     bar.vf = bar.ke + 8 * C::kStagesK;
     bar.ve = bar.vf + 8 * C::kStagesV;
-    static_assert(208 + 16 * (C::kStagesK + C::kStagesV) <= C::kBarBytes, "barrier area too small");
+    static_assert(160 + 16 * (C::kStagesK + C::kStagesV) <= C::kBarBytes, "barrier area too small");
 
     const int tid = threadIdx.x;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);        // warp-uniform
@@ -580,10 +526,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         abort_flag = 0;
         redo_flag = 0;
         for (int t = 0; t < kTilesM; ++t) {
-            mbar_init(bar.q + 8 * t, 128 * C::kSplit);
-            for (int u = 0; u < 4; ++u) {
-                mbar_init(bar.s + 32 * t + 8 * u, 1); mbar_init(bar.p + 32 * t + 8 * u, 128); mbar_init(bar.o + 32 * t + 8 * u, 1);
-            }
+            mbar_init(bar.q + 8 * t, 128 * kSplit);
+            mbar_init(bar.done + 8 * t, 1);
+            for (int u = 0; u < 4; ++u) { mbar_init(bar.s + 32 * t + 8 * u, 1); mbar_init(bar.p + 32 * t + 8 * u, 128); }
         }
         // a K/V stage is free once the issuer of every active query tile has committed its MMAs on it
         for (int s = 0; s < C::kStagesK; ++s) { mbar_init(bar.kf + 8 * s, 1); mbar_init(bar.ke + 8 * s, q_tiles); }
@@ -603,11 +548,11 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     if (warp < C::kSoftmaxWarps) {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(C::kRegsSoftmax));
         const int wg = warp >> 2;
-        const int tile = wg / C::kSplit, par = wg % C::kSplit;
+        const int tile = wg / kSplit, par = wg % kSplit;
         if (tile < q_tiles)
             softmax_role<DH>(p, bar, tile, par, smem_gen + tile * C::kQTileBytes, tmem, m0 + tile * kBlockM, h, b, n_tiles,
                              &abort_flag, &redo_flag, xchg[tile]);
-        else if constexpr (C::kSplit == 2) pass_sync<DH>();
+        else pass_sync<DH>();
     } else if (warp == kProducerWarp) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
         // ------------------------------------------------ TMA producer (warp-uniform, one elected lane issues)
@@ -653,13 +598,11 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         };
         produce_pass(kSpeculate);
         int k_loads = n_tiles, v_loads = n_tiles;
-        if constexpr (C::kSplit == 2) {
-            pass_sync<DH>();
-            if (redo_flag) {
-                produce_pass(kMaxOnly);
-                produce_pass(kExact);
-                k_loads = 3 * n_tiles; v_loads = 2 * n_tiles;
-            }
+        pass_sync<DH>();
+        if (redo_flag) {
+            produce_pass(kMaxOnly);
+            produce_pass(kExact);
+            k_loads = 3 * n_tiles; v_loads = 2 * n_tiles;
         }
         // every copy issued above must have landed before the CTA's shared memory is released
         for (int g = (k_loads > C::kStagesK ? k_loads - C::kStagesK : 0); g < k_loads; ++g)
@@ -740,9 +683,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                                        smem_desc(vbase + C::kChunks * C::kChunkBytes + ks * 512, 256, 256, kSwizzle32B),
                                        idesc_pv_tail, (j > 0 || ks > 0) ? 1u : 0u);
                         }
-                        if (kSBufs == kAhead) tc_commit(bar.o + 32 * t + 8 * u);
                         tc_commit(bar.ve + 8 * sv);
-                        if (j == n_tiles - 1) tc_commit(bar.o + 32 * t + 24);      // the pass is done for this query tile
+                        if (j == n_tiles - 1) tc_commit(bar.done + 8 * t);        // the pass is done for this query tile
                     }
                     // two S buffers: the one just consumed as P is free again (in-order pipe), refill it with key tile j+2
                     if (kSBufs == kAhead && more) {
@@ -757,16 +699,14 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             wait_bar(bar.q + 8 * t, 0, &abort_flag, p.err_word);
             issue_pass(kSpeculate);
         }
-        if constexpr (C::kSplit == 2) {
-            pass_sync<DH>();
-            if (redo_flag && t < q_tiles) {
-                issue_pass(kMaxOnly);
-                issue_pass(kExact);
-            }
+        pass_sync<DH>();
+        if (redo_flag && t < q_tiles) {
+            issue_pass(kMaxOnly);
+            issue_pass(kExact);
         }
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
-        if constexpr (C::kSplit == 2) pass_sync<DH>();
+        pass_sync<DH>();
     }
 
     tc_fence_before();
