@@ -34,7 +34,7 @@ UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the attention kernel, from the ncu
 # capture summarised in profiles/ (workload -> theta_permille -> bytes); None where not captured.
-NCU_TRAFFIC_BYTES = {"cogvideox": {500: 324246784}, "sweep": {250: 1312009224}}
+NCU_TRAFFIC_BYTES = {"cogvideox": {500: 324246784}, "sweep": {250: 1285133616}}
 
 
 def measured_peaks():
