@@ -3,7 +3,7 @@
 // Section 3.2 "Sparse Attention").
 //
 // One CTA per (256 selected queries, head, batch): two 128-row query tiles that share every
-// K/V tile of 64 keys (48 at head_dim 72).  Warp roles:
+// K/V tile of 64 keys.  Warp roles:
 //   softmax warpgroups (one thread per query row), two per query tile: gather the tile's Q rows into
 //              128B-swizzled shared memory, then per key tile read S from TMEM, exponentiate in the log2
 //              domain against a reference maximum, write P (bf16) back to TMEM over S, and at the end
@@ -17,14 +17,14 @@
 // serial chain of a key tile (wait, load, exponentials, sum, pack, publish).  Even key tiles go to one
 // warpgroup and odd ones to the other; both work against the same reference maximum and their P tiles
 // accumulate into ONE O accumulator per query tile.  That leaves TMEM room for three S buffers per query
-// tile at head_dim 64 / 72 (S of key tile j+2 is computed while tiles j and j+1 are in the softmax) and
-// for two at head_dim 128 (a buffer is refilled with key tile j+2 as soon as P of tile j has been
+// tile at head_dim 64 (S of key tile j+2 is computed while tiles j and j+1 are in the softmax) and for
+// two at head_dim 72 / 128 (a buffer is refilled with key tile j+2 as soon as P of tile j has been
 // consumed; the tensor pipe executes one thread's MMAs in order).
 //
 // The softmax is bound by the exponentials (XU pipe, 16 per clock per SM), by the issue slots and by the
 // latencies of its own chain, so the common path of a key tile is kept to: load S, one FFMA + one
-// exponential per element, sum, pack, store.  At head_dim 64 six of every sixteen exponentials are a
-// cubic on the FMA pipe instead of ex2 on the XU.  The reference maximum is the exact row maximum of key
+// exponential per element, sum, pack, store.  At head_dim 64 / 72 six / four of every sixteen exponentials
+// are a cubic on the FMA pipe instead of ex2 on the XU.  The reference maximum is the exact row maximum of key
 // tile 0 and is then only checked through each tile's sum of exponentials: while that sum stays below a
 // limit the tile is accepted as it is (the probabilities are relative to a stale maximum, which the final
 // normalisation cancels; fp32 and bf16 have the range).  Otherwise the CTA raises a flag, finishes the
@@ -63,15 +63,13 @@ template <int DH> struct Cfg {
     static constexpr int kTail = DH - kMain;
     static constexpr int kTailPad = kTail ? 16 : 0;
     static_assert(kTail == 0 || kTail == 8, "head_dim must be 64, 72 or 128");
-    // keys per K/V tile = columns of an S buffer.  64, but 48 at head_dim 72 (two O accumulators of 80 columns leave
-    // 352 TMEM columns for the S buffers)
-    static constexpr int kBlockN = (DH == 72) ? 48 : 64;
-    // S buffers per query tile, used round-robin by its two softmax warpgroups.  Three where TMEM has the room: S
-    // of key tile j+2 is then produced while tiles j and j+1 are in the softmax.  head_dim 128 has room for two.
-    static constexpr int kSBufs = (DH == 128) ? 2 : 3;
-    // exponentials per 16 that are computed on the FMA pipe instead of the XU (measured: 6 is best at head_dim 64,
-    // none at 72 and 128, where the tensor pipe has less slack)
-    static constexpr int kPolyOf16 = (DH == 64) ? 6 : 0;
+    static constexpr int kBlockN = 64;                            // keys per K/V tile = columns of an S buffer
+    // S buffers per query tile, used round-robin by its two softmax warpgroups.  Three where TMEM has the room
+    // (head_dim 64): S of key tile j+2 is then produced while tiles j and j+1 are in the softmax.
+    static constexpr int kSBufs = (DH == 64) ? 3 : 2;
+    // exponentials per 16 that are computed on the FMA pipe instead of the XU (measured best: 6 at head_dim 64, 4 at
+    // 72, none at 128, where the tensor pipe is as busy as the XU)
+    static constexpr int kPolyOf16 = (DH == 64) ? 6 : (DH == 72) ? 4 : 0;
     static constexpr int kSoftmaxWarps = 4 * kTilesM * kSplit;
     static constexpr int kAhead = 2;                              // Q K^T runs this many key tiles ahead of P V
     static constexpr int kThreads = (kSoftmaxWarps + 4) * 32;     // + producer, two issuers, one register donor
@@ -212,12 +210,12 @@ template <int DH> struct SoftmaxState {
     int *err_word;
 };
 
-// NS (48 or 64) columns of one S buffer into registers (asynchronous: wait_s_regs before using them)
+// the 64 columns of one S buffer into registers (asynchronous: wait_s_regs before using them)
 template <int NS>
 __device__ __forceinline__ void load_s(uint32_t t_s, float (&s)[NS]) {
+    static_assert(NS == 64, "an S buffer has 64 columns");
     tmem_ld32(t_s, reinterpret_cast<uint32_t (&)[32]>(s[0]));
-    if constexpr (NS == 64) tmem_ld32(t_s + 32, reinterpret_cast<uint32_t (&)[32]>(s[32]));
-    else tmem_ld16(t_s + 32, reinterpret_cast<uint32_t (&)[16]>(s[32]));
+    tmem_ld32(t_s + 32, reinterpret_cast<uint32_t (&)[32]>(s[32]));
 }
 // tcgen05.wait::ld that names the loaded registers, so that no use of them can move above it
 __device__ __forceinline__ void wait_regs16(float *s) {
@@ -268,12 +266,8 @@ __device__ __forceinline__ void pack_p(const float (&e)[NS], uint32_t (&pk)[NS /
 // P of one key tile: NS/2 packed bf16 pairs over the first NS/2 columns of the S buffer
 template <int NS>
 __device__ __forceinline__ void store_p(uint32_t t_s, const uint32_t (&pk)[NS / 2]) {
-    if constexpr (NS == 64) {
-        tmem_st32(t_s, pk);
-    } else {
-        tmem_st16(t_s, reinterpret_cast<const uint32_t (&)[16]>(pk[0]));
-        tmem_st8(t_s + 16, reinterpret_cast<const uint32_t (&)[8]>(pk[16]));
-    }
+    static_assert(NS == 64, "an S buffer has 64 columns");
+    tmem_st32(t_s, pk);
 }
 
 // P has been stored: make it visible to the issuer warp
