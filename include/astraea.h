@@ -196,13 +196,17 @@ int32_t astraea_step(const void *x_cur, void *x_ref, float *lse_cache, int32_t *
 /*
  * Host-buffer session: the library owns the device-side state of one attention block
  * (x_ref, LSE cache, counters, output cache) and staging buffers, and each step copies
- * the HOST inputs to the device, runs astraea_step and copies the merged output back.
+ * the HOST inputs to the device, runs the step (score, select, refresh of x_ref,
+ * sparse attention) and copies the merged output back.  The copies run on streams of
+ * their own: x_cur goes first, q / k / v follow in four groups of heads, the attention
+ * of a group starts when its heads have arrived, and the group's columns of the output
+ * go back while the next group is computed.  The results are those of astraea_step.
  * astraea_session_create allocates device memory (cudaMalloc) on the current device;
  * the first step of a session must be run with k_keep = N_sel (all tokens computed) to
  * fill the caches, as the paper's denoising loop does at its first timestep.
  *   x_cur, q, k, v : host bf16 [B,N,D] (pinned memory gives asynchronous copies)
  *   out            : host bf16 [B,N,D], receives X_out,t (computed + cached rows)
- * astraea_step_host synchronises the session's stream before it returns.
+ * astraea_step_host synchronises the session's streams before it returns.
  */
 typedef struct astraea_session astraea_session;
 int32_t astraea_session_create(astraea_session **session, int B, int H, int N, int N_sel, int d);

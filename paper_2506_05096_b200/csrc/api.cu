@@ -231,6 +231,10 @@ int32_t astraea_poll_error(void *workspace, void *stream)
 }
 
 // ------------------------------------------------------------------ host-buffer session
+// astraea_step_host moves q, k, v in and the output back in groups of heads, so that the copies of one group run
+// under the attention of another.
+constexpr int kHostGroups = 4;
+
 struct astraea_session {
     int B, H, N, N_sel, d;
     size_t tensor_bytes;
@@ -239,7 +243,11 @@ struct astraea_session {
     int32_t *n_skip, *idx_sel, *idx_rem;
     void *workspace;
     size_t workspace_bytes;
-    cudaStream_t stream;
+    cudaStream_t stream;            // score, select, attention, refresh
+    cudaStream_t copy_in, copy_out; // host -> device and device -> host copies, overlapped with the compute stream
+    cudaEvent_t ev_x;               // x_cur has arrived
+    cudaEvent_t ev_in[kHostGroups]; // q, k, v of a head group have arrived
+    cudaEvent_t ev_attn[kHostGroups];   // attention of a head group is done
     int steps;
 };
 
@@ -249,7 +257,13 @@ void astraea_session_destroy(astraea_session *s)
     void *bufs[] = {s->x_cur, s->x_ref, s->q, s->k, s->v, s->out_cache, s->lse_cache, s->score,
                     s->n_skip, s->idx_sel, s->idx_rem, s->workspace};
     for (void *p : bufs) if (p) cudaFree(p);
-    if (s->stream) cudaStreamDestroy(s->stream);
+    if (s->ev_x) cudaEventDestroy(s->ev_x);
+    for (int g = 0; g < kHostGroups; ++g) {
+        if (s->ev_in[g]) cudaEventDestroy(s->ev_in[g]);
+        if (s->ev_attn[g]) cudaEventDestroy(s->ev_attn[g]);
+    }
+    cudaStream_t streams[] = {s->stream, s->copy_in, s->copy_out};
+    for (cudaStream_t st : streams) if (st) cudaStreamDestroy(st);
     delete s;
 }
 
@@ -266,6 +280,13 @@ int32_t astraea_session_create(astraea_session **session, int B, int H, int N, i
     s->tensor_bytes = (size_t)B * N * H * d * 2;
     s->workspace_bytes = astraea_workspace_bytes(ASTRAEA_OP_STEP, B, H, N, N, d);
     cudaError_t e = cudaStreamCreateWithFlags(&s->stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&s->copy_in, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&s->copy_out, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&s->ev_x, cudaEventDisableTiming);
+    for (int g = 0; g < kHostGroups; ++g) {
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&s->ev_in[g], cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&s->ev_attn[g], cudaEventDisableTiming);
+    }
     void **big[] = {&s->x_cur, &s->x_ref, &s->q, &s->k, &s->v, &s->out_cache};
     for (void **p : big) if (e == cudaSuccess) e = cudaMalloc(p, s->tensor_bytes);
     if (e == cudaSuccess) e = cudaMalloc((void **)&s->lse_cache, (size_t)B * H * N * 4);
@@ -295,19 +316,70 @@ int32_t astraea_step_host(astraea_session *s, const void *x_cur, const void *q, 
     REQUIRE(s && x_cur && q && k && v && out, "astraea_step_host: null argument");
     REQUIRE(k_keep >= 0 && k_keep <= s->N_sel, "astraea_step_host: k_keep=%d outside [0, N_sel=%d]", k_keep, s->N_sel);
     REQUIRE(s->steps > 0 || k_keep == s->N_sel, "astraea_step_host: the first step of a session must compute every token (k_keep = N_sel)");
-    cudaError_t e = cudaMemcpyAsync(s->x_cur, x_cur, s->tensor_bytes, cudaMemcpyHostToDevice, s->stream);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(s->q, q, s->tensor_bytes, cudaMemcpyHostToDevice, s->stream);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(s->k, k, s->tensor_bytes, cudaMemcpyHostToDevice, s->stream);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(s->v, v, s->tensor_bytes, cudaMemcpyHostToDevice, s->stream);
+    const int B = s->B, H = s->H, N = s->N, N_sel = s->N_sel, d = s->d, D = H * d;
+    const int n_always = N - N_sel, M = k_keep + n_always;
+    const size_t pitch = (size_t)D * 2, rows = (size_t)B * N;
+    const size_t attn_ws = attn_workspace_bytes(B, H, N, M, d);
+    char *ws = reinterpret_cast<char *>(s->workspace);
+    const int groups = H < kHostGroups ? H : kHostGroups;
+    auto head_lo = [&](int g) { return (int)((long long)H * g / groups); };
+
+    // copy-in stream: x_cur first (the score needs nothing else), then q, k, v by head group
+    cudaError_t e = cudaMemcpyAsync(s->x_cur, x_cur, s->tensor_bytes, cudaMemcpyHostToDevice, s->copy_in);
+    if (e == cudaSuccess) e = cudaEventRecord(s->ev_x, s->copy_in);
+    for (int g = 0; g < groups && e == cudaSuccess; ++g) {
+        const size_t off = (size_t)head_lo(g) * d * 2, width = (size_t)(head_lo(g + 1) - head_lo(g)) * d * 2;
+        const void *src[3] = {q, k, v};
+        void *dst[3] = {s->q, s->k, s->v};
+        for (int i = 0; i < 3 && e == cudaSuccess; ++i)
+            e = cudaMemcpy2DAsync(static_cast<char *>(dst[i]) + off, pitch, static_cast<const char *>(src[i]) + off, pitch,
+                                  width, rows, cudaMemcpyHostToDevice, s->copy_in);
+        if (e == cudaSuccess) e = cudaEventRecord(s->ev_in[g], s->copy_in);
+    }
+    if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_step_host (copy in): %s", cudaGetErrorString(e));
+
+    // compute stream: score -> select -> refresh of x_ref, then the attention of each head group as it arrives
+    e = cudaStreamWaitEvent(s->stream, s->ev_x, 0);
     if (e == cudaSuccess && s->steps == 0)   // no earlier step: the reference inputs are the current ones
         e = cudaMemcpyAsync(s->x_ref, s->x_cur, s->tensor_bytes, cudaMemcpyDeviceToDevice, s->stream);
-    if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_step_host (copy in): %s", cudaGetErrorString(e));
-    int32_t rc = astraea_step(s->x_cur, s->x_ref, s->lse_cache, s->n_skip, s->q, s->k, s->v, s->out_cache,
-                              s->score, s->idx_sel, s->idx_rem, s->B, s->H, s->N, s->N_sel, s->d, k_keep,
-                              w_alpha, w_beta, delta_mode, lse_mode, s->workspace, s->workspace_bytes, s->stream);
+    if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_step_host: %s", cudaGetErrorString(e));
+    int32_t rc = astraea_score(s->x_cur, s->x_ref, s->lse_cache, s->n_skip, s->score, B, N, N_sel, D, H, w_alpha, w_beta,
+                               delta_mode, lse_mode, s->stream);
+    if (rc == ASTRAEA_OK)
+        rc = astraea_select(s->score, B, N_sel, k_keep, n_always, s->idx_sel, s->idx_rem, s->n_skip, ws + attn_ws,
+                            s->workspace_bytes - attn_ws, s->stream);
+    if (rc == ASTRAEA_OK)
+        rc = astraea_scatter_reuse(s->x_ref, s->x_cur, s->idx_sel, B, N, M, D, ASTRAEA_SCATTER_SRC_FULL, s->stream);
     if (rc != ASTRAEA_OK) return rc;
-    e = cudaMemcpyAsync(out, s->out_cache, s->tensor_bytes, cudaMemcpyDeviceToHost, s->stream);
-    if (e == cudaSuccess) e = cudaStreamSynchronize(s->stream);
+    for (int g = 0; g < groups; ++g) {
+        e = cudaStreamWaitEvent(s->stream, s->ev_in[g], 0);
+        if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_step_host: %s", cudaGetErrorString(e));
+        if (M > 0) {
+            AttnArgs a;
+            a.q = s->q; a.k = s->k; a.v = s->v;
+            a.q_sb = a.k_sb = a.v_sb = (int64_t)N * D;
+            a.q_sh = a.k_sh = a.v_sh = d;
+            a.q_sn = a.k_sn = a.v_sn = D;
+            a.q_idx = s->idx_sel; a.M = M; a.out = s->out_cache; a.lse_out = s->lse_cache;
+            a.B = B; a.H = H; a.N = N; a.d = d; a.N_tok = N;
+            a.scale = 1.0f / sqrtf((float)d);
+            a.flags = 0;
+            a.err_word = reinterpret_cast<int *>(s->workspace);
+            a.head_begin = head_lo(g); a.head_count = head_lo(g + 1) - head_lo(g);
+            rc = launch_sparse_attn(a, s->stream);
+            if (rc != ASTRAEA_OK) return rc;
+        }
+        e = cudaEventRecord(s->ev_attn[g], s->stream);
+        // copy-out stream: the group's columns of the output cache (computed and reused rows alike)
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(s->copy_out, s->ev_attn[g], 0);
+        const size_t off = (size_t)head_lo(g) * d * 2, width = (size_t)(head_lo(g + 1) - head_lo(g)) * d * 2;
+        if (e == cudaSuccess)
+            e = cudaMemcpy2DAsync(static_cast<char *>(out) + off, pitch, static_cast<const char *>(s->out_cache) + off, pitch,
+                                  width, rows, cudaMemcpyDeviceToHost, s->copy_out);
+        if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_step_host (copy out): %s", cudaGetErrorString(e));
+    }
+    e = cudaStreamSynchronize(s->copy_out);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s->copy_in);
     if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_step_host (copy out): %s", cudaGetErrorString(e));
     s->steps++;
     return astraea_poll_error(s->workspace, s->stream);

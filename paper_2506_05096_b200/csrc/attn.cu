@@ -108,6 +108,7 @@ struct Params {
     int N_tok;                   // tokens of q / out / lse_out (N_tok == N unless the keys were gathered)
     float scale, scale_log2;
     int compact;
+    int h0;                      // first head of this launch
     int *err_word;
 };
 
@@ -510,7 +511,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 
     const int tid = threadIdx.x;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);        // warp-uniform
-    const int m0 = blockIdx.x * (kTilesM * kBlockM), h = blockIdx.y, b = blockIdx.z;
+    const int m0 = blockIdx.x * (kTilesM * kBlockM), h = p.h0 + blockIdx.y, b = blockIdx.z;
     constexpr int kBlockN = C::kBlockN;
     const int n_tiles = (p.N + kBlockN - 1) / kBlockN;
     // the last CTA of a head may have rows in its first query tile only: the second tile's warps and MMAs are skipped
@@ -776,7 +777,8 @@ int32_t launch_dh(const AttnArgs &a, cudaStream_t stream)
     p.scale_log2 = a.scale * 1.4426950408889634f;
     p.compact = (a.flags & ASTRAEA_ATTN_COMPACT_OUT) ? 1 : 0;
     p.err_word = a.err_word;
-    dim3 grid((a.M + kTilesM * kBlockM - 1) / (kTilesM * kBlockM), a.H, a.B);
+    p.h0 = a.head_begin;
+    dim3 grid((a.M + kTilesM * kBlockM - 1) / (kTilesM * kBlockM), a.head_count > 0 ? a.head_count : a.H, a.B);
     sparse_attn_kernel<DH><<<grid, C::kThreads, C::kSmemBytes, stream>>>(mk, mv, mkt, mvt, p);
     return check_launch("astraea_sparse_attn");
 }

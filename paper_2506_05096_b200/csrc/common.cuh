@@ -43,6 +43,7 @@ struct AttnArgs {
     float scale;
     uint32_t flags;
     int *err_word;
+    int head_begin = 0, head_count = 0;   // a sub-range of the H heads (head_count 0: all); strides and H stay those of the full tensors
 };
 int32_t launch_sparse_attn(const AttnArgs &a, cudaStream_t stream);
 size_t attn_workspace_bytes(int B, int H, int N, int M, int d);

@@ -231,9 +231,15 @@ select_cluster_kernel(const float *__restrict__ score, int N_sel, int k, int n_a
                 const bool live = (base + u < N_sel) && ((key[u] & mask) == prefix);
                 const uint32_t bin = (key[u] >> shift) & 255u;
                 const uint32_t act = __ballot_sync(0xffffffffu, live);
-                if (live) {                      // one shared-memory atomic per distinct bin per warp
-                    const uint32_t peers = __match_any_sync(act, bin);
-                    if (lane == (__ffs(peers) - 1)) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
+                if (act == 0) continue;
+                // the leading digits of the scores are nearly all equal: one atomic for the warp when its live keys
+                // share the bin, else one per key (the later digits are spread out, so those rarely collide)
+                const int leader = __ffs(act) - 1;
+                const uint32_t lbin = __shfl_sync(0xffffffffu, bin, leader);
+                if (__all_sync(0xffffffffu, !live || bin == lbin)) {
+                    if (lane == leader) atomicAdd(&hist[lbin], (uint32_t)__popc(act));
+                } else if (live) {
+                    atomicAdd(&hist[bin], 1u);
                 }
             }
             __syncthreads();
@@ -357,6 +363,9 @@ int32_t launch_select(const float *score, int B, int N_sel, int k, int n_always,
                       int32_t *idx_rem, int32_t *n_skip, void *, cudaStream_t stream)
 {
     if (B == 0 || (N_sel == 0 && n_always == 0)) return ASTRAEA_OK;
+#ifdef SEL_FORCE
+    if (N_sel > 0 && N_sel <= SEL_FORCE * kThreads * kMaxCluster) return launch_cluster<SEL_FORCE>(score, B, N_sel, k, n_always, idx_sel, idx_rem, n_skip, stream);
+#endif
     if (N_sel > 0 && N_sel <= 4 * kThreads * kMaxCluster)
         return launch_cluster<4>(score, B, N_sel, k, n_always, idx_sel, idx_rem, n_skip, stream);
     if (N_sel > 0 && N_sel <= 8 * kThreads * kMaxCluster)

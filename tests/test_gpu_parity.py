@@ -417,3 +417,42 @@ def test_step_chain_of_fifty_steps_reduced_hunyuan_shape(oracle):
     _step_case(oracle, w, 5, 600, steps=50)
     _step_case(oracle, w, 6, 300, steps=12)
 
+
+
+# ------------------------------------------------------------- host-buffer session
+def test_session_step_host_equals_the_device_path_and_the_oracle(oracle):
+    """astraea_step_host (pinned host buffers, copies overlapped with the attention by head group) against
+    astraea_step on device buffers from the same initial state: bit-identical outputs over three steps; the first,
+    dense step also against the oracle."""
+    w = synth.Workload("mini-session", B=2, H=6, d=64, N_v=700, N_t=30)
+    inp = synth.make_step_inputs(w, 11)
+    B, N, H, d, N_sel, n_always = w.B, w.N, w.H, w.d, w.N_v, w.N_t
+    sess = A.Session(B, H, N, N_sel, d)
+    # device path, same initial state as a fresh session: zero caches and counters, x_ref = first x_cur
+    x_ref = to_dev_bf16(inp["x_cur"])
+    lse = torch.zeros(B, H, N, device="cuda")
+    n_skip = torch.zeros(B, N_sel, dtype=torch.int32, device="cuda")
+    out = torch.zeros(B, N, H, d, dtype=torch.bfloat16, device="cuda")
+    score = torch.empty(B, N_sel, device="cuda")
+    x_bits, q_bits, k_bits, v_bits = inp["x_cur"], inp["q"], inp["k"], inp["v"]
+    host_out = torch.empty(B, N, H, d, dtype=torch.bfloat16).pin_memory()
+    for t, theta in enumerate((1000, 400, 250)):
+        if t > 0:
+            x_bits = synth.drift_step(x_bits, 300 + t, 0.05, False)
+            q_bits, k_bits, v_bits = (synth.drift_step(a, 400 + 10 * t + i, 0.05, True) for i, a in enumerate((q_bits, k_bits, v_bits)))
+        k_keep = w.k_of(theta)
+        M = k_keep + n_always
+        host = [torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).pin_memory() for a in (x_bits, q_bits, k_bits, v_bits)]
+        sess.step_host(host[0], host[1], host[2], host[3], host_out, k_keep)
+        idx_sel = torch.empty(B, M, dtype=torch.int32, device="cuda")
+        idx_rem = torch.empty(B, N_sel - k_keep, dtype=torch.int32, device="cuda")
+        ws = A.new_workspace(A.OP_STEP, B, H, N, M, d)
+        A.astraea_step(to_dev_bf16(x_bits), x_ref, lse, n_skip, to_dev_bf16(q_bits), to_dev_bf16(k_bits),
+                       to_dev_bf16(v_bits), out, score, idx_sel, idx_rem, B, H, N, N_sel, d, k_keep, workspace=ws)
+        A.astraea_poll_error(ws)
+        assert torch.equal(host_out.view(torch.int16), out.cpu().view(torch.int16)), "step %d" % t
+        if t == 0:
+            want_o, _, _ = oracle.sparse_attn(f64(q_bits), f64(k_bits), f64(v_bits), q_idx=None, scale=0.0)
+            err = np.abs(bf16_dev_to_f64(out) - want_o)
+            assert err.max() < ATTN_MAX_ABS and err.mean() < ATTN_MEAN_ABS
+    sess.close()
