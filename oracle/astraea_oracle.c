@@ -25,7 +25,8 @@
  * library softmax-attention; keep-ratio 0 identity; brute-force selection;
  * softmax rows sum to 1; closed forms for zero keys, constant values, a dominant
  * key, constant per-token differences, the round-robin penalty schedule;
- * permutation invariances; half-normal drift statistics.
+ * permutation invariances; half-normal drift statistics; the linear layer on listed rows
+ * vs a library matmul, a one-hot weight, a zero weight and pure-Python brute force.
  * parity unpinned: absolute score values under the paper's own (unpublished)
  * w_alpha, w_beta and its intended reading of [R1]-[R4].
  */
@@ -226,6 +227,31 @@ void oracle_scatter_lse(double *lse_cache, const double *lse_rows, const int32_t
 }
 
 /* floor(theta * N_sel) in integer arithmetic from a permille budget [R9]. */
+/*
+ * Linear layer on the selected rows (Algorithm 1 lines 4-5 and Section 3.2, "the same strategy
+ * applies to the other layers of the block"): y[b, i, :] = x[b, i, :] W^T + bias for the listed
+ * rows i = idx[b, r]; every other row of y keeps what it held (the cached result).  W is
+ * [N_out, K] (out features x in features).  idx == NULL: all N rows.  Plain triple loop.
+ */
+void oracle_gathered_linear(const double *x, const int32_t *idx, int M, const double *w,
+                            const double *bias, double *y, int B, int N, int K, int N_out)
+{
+    const int rows = idx ? M : N;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int b = 0; b < B; ++b)
+        for (int r = 0; r < rows; ++r) {
+            const int i = idx ? idx[(size_t)b * M + r] : r;
+            const double *xr = x + ((size_t)b * N + i) * K;
+            double *yr = y + ((size_t)b * N + i) * N_out;
+            for (int n = 0; n < N_out; ++n) {
+                double acc = bias ? bias[n] : 0.0;
+                const double *wr = w + (size_t)n * K;
+                for (int c = 0; c < K; ++c) acc += xr[c] * wr[c];
+                yr[n] = acc;
+            }
+        }
+}
+
 int oracle_budget_to_k(int n_sel, int theta_permille)
 {
     return (int)(((int64_t)n_sel * theta_permille) / 1000);

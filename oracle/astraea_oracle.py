@@ -128,6 +128,26 @@ def scatter_reuse(cache, rows, idx):
     return out
 
 
+def gathered_linear(x, w, bias=None, idx=None, y_cache=None):
+    """y = copy of y_cache [B, N, N_out] (zeros if None) with rows idx[b, r] (all rows if idx is None)
+    replaced by x[b, i, :] @ w.T + bias; w is [N_out, K]."""
+    x, w = _f64(x), _f64(w)
+    B, N, K = x.shape
+    N_out = w.shape[0]
+    assert w.shape == (N_out, K)
+    y = np.zeros((B, N, N_out)) if y_cache is None else np.array(y_cache, dtype=np.float64, copy=True, order="C")
+    assert y.shape == (B, N, N_out)
+    bias = None if bias is None else _f64(bias)
+    M = 0
+    if idx is not None:
+        idx = _i32(idx)
+        M = idx.shape[1]
+        if M == 0:
+            return y
+    _load().oracle_gathered_linear(_p(x), _p(idx), M, _p(w), _p(bias), _p(y), B, N, K, N_out)
+    return y
+
+
 def scatter_lse(lse_cache, lse_rows, idx):
     out = np.array(lse_cache, dtype=np.float64, copy=True, order="C")
     lse_rows, idx = _f64(lse_rows), _i32(idx)

@@ -307,6 +307,45 @@ def test_drift_statistics_half_normal_mean(oracle):
 
 
 # -------------------------------------------------------- flop accounting pin
+# ---------------------------------------------------------------- linear layers on selected rows
+def test_gathered_linear_matches_a_library_matmul_and_leaves_other_rows_alone(oracle):
+    """All rows: the textbook x W^T + b (numpy matmul).  Listed rows only: those rows equal the full product,
+    the others are bit-identical to the cache (Algorithm 1 lines 4-7 applied to a linear layer)."""
+    rng = np.random.default_rng(21)
+    B, N, K, N_out, M = 2, 29, 24, 17, 11
+    x, w, bias, cache = _rand(rng, B, N, K), _rand(rng, N_out, K), _rand(rng, N_out), _rand(rng, B, N, N_out)
+    full = x @ w.T + bias
+    assert np.abs(oracle.gathered_linear(x, w, bias) - full).max() < 1e-12
+    idx = np.stack([np.sort(rng.choice(N, M, replace=False)) for _ in range(B)]).astype(np.int32)
+    y = oracle.gathered_linear(x, w, bias, idx, cache)
+    for b in range(B):
+        mask = np.zeros(N, bool)
+        mask[idx[b]] = True
+        assert np.abs(y[b, mask] - full[b, mask]).max() < 1e-12
+        assert np.array_equal(y[b, ~mask], cache[b, ~mask])
+    assert np.array_equal(oracle.gathered_linear(x, w, bias, np.zeros((B, 0), np.int32), cache), cache)
+
+
+def test_gathered_linear_closed_forms_catch_a_transposed_weight_or_a_dropped_bias(oracle):
+    rng = np.random.default_rng(22)
+    B, N, K = 1, 7, 5
+    x = _rand(rng, B, N, K)
+    # a non-square one-hot weight: output feature n copies input feature sel[n] (a transposed operand cannot do this)
+    sel = np.array([3, 0, 4, 4, 1, 2, 0])
+    w = np.zeros((len(sel), K))
+    w[np.arange(len(sel)), sel] = 1.0
+    assert np.array_equal(oracle.gathered_linear(x, w), x[:, :, sel])
+    # zero weight: every computed row is the bias; brute force in pure Python for a dense random case
+    bias = _rand(rng, len(sel))
+    assert np.array_equal(oracle.gathered_linear(x, np.zeros_like(w), bias), np.broadcast_to(bias, (B, N, len(sel))))
+    w2 = _rand(rng, 3, K)
+    got = oracle.gathered_linear(x, w2, bias[:3])
+    for i in range(N):
+        for n in range(3):
+            want = bias[n] + sum(x[0, i, c] * w2[n, c] for c in range(K))
+            assert abs(got[0, i, n] - want) < 1e-13
+
+
 def test_attention_flops_are_linear_in_selected_tokens_like_the_papers_tables():
     from paper_2506_05096_b200 import accounting
     path = os.path.join(os.path.dirname(__file__), "golden", "flops_tables.txt")
