@@ -52,6 +52,8 @@ extern "C" {
 
 /* flags of astraea_sparse_attn */
 #define ASTRAEA_ATTN_COMPACT_OUT  1u         /* out is [B,M,H,d] and lse_out [B,H,M] (row r of the index list), not the caches */
+/* flags of astraea_gathered_linear */
+#define ASTRAEA_LINEAR_COMPACT_OUT 1u        /* y is [B,M,N_out] (row r of the index list), not the cache [B,N,N_out] */
 /* flags of astraea_scatter_reuse */
 #define ASTRAEA_SCATTER_SRC_FULL  1u         /* rows is [B,N,row_elems]; row idx[r] of it is copied to row idx[r] of cache */
 
@@ -60,6 +62,7 @@ extern "C" {
 #define ASTRAEA_OP_SPARSE_ATTN  2
 #define ASTRAEA_OP_STEP         3
 #define ASTRAEA_OP_SPARSE_ATTN_KV 4          /* astraea_sparse_attn with kv_idx: pass M_kv as the M argument */
+#define ASTRAEA_OP_GATHERED_LINEAR 5        /* astraea_gathered_linear (the size arguments are ignored) */
 
 /*
  * Selection metric (Section 3.2 "Selection Metric"; Algorithm 1 lines 1-2):
@@ -175,6 +178,27 @@ int32_t astraea_sparse_attn_noalloc(const void *q, const void *k, const void *v,
  */
 int32_t astraea_scatter_reuse(void *cache, const void *rows, const int32_t *idx,
                               int B, int N, int M, int row_elems, uint32_t flags, void *stream);
+
+/*
+ * A linear layer of the compute block on the selected tokens only (Algorithm 1 lines 4-5: the query
+ * projection X_in[I_sel] W_Q of the gathered rows, the key / value projections of all rows; Section 3.2:
+ * the other layers of the block follow the same gather - compute - scatter pattern):
+ *     y[b, idx[b,r], :] = x[b, idx[b,r], :] W^T + bias        for r in [0, M)
+ * and every row of y that is not listed is left untouched, i.e. keeps the cached result of the earlier
+ * step.  The gather of the rows of x and the scatter of the rows of y are fused into the GEMM.
+ *   x    : bf16 [B, N, K]            idx : int32 [B, M] in [0,N), no duplicates; NULL => all N rows (M ignored)
+ *   w    : bf16 [N_out, K] row-major (out features x in features)        bias : bf16 [N_out] or NULL
+ *   y    : bf16 [B, N, N_out], rows at idx written in place; with ASTRAEA_LINEAR_COMPACT_OUT bf16 [B, M, N_out]
+ *   workspace : at least astraea_workspace_bytes(ASTRAEA_OP_GATHERED_LINEAR, 0, 0, 0, 0, 0) bytes, 256-byte
+ *               aligned, zero before the first use (holds the error word read by astraea_poll_error).
+ * bf16 operands, fp32 accumulation, one rounding to bf16 at the end.  K must be a multiple of 64, N_out
+ * a multiple of 8; x, w, y 16-byte aligned.  M = 0 is valid (nothing is launched).  An index outside
+ * [0,N) is not dereferenced: its row is skipped and astraea_poll_error reports BAD_INDEX.
+ * Errors: INVALID_ARG, UNSUPPORTED (unknown flags), WORKSPACE_TOO_SMALL, CUDA.
+ */
+int32_t astraea_gathered_linear(const void *x, const int32_t *idx, int M, const void *w, const void *bias,
+                                void *y, int B, int N, int K, int N_out, uint32_t flags,
+                                void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * One whole step of one attention block on device buffers (Algorithm 1 with given Q, K, V):

@@ -21,13 +21,14 @@ DELTA_MEAN_ABS, DELTA_MEAN_SQ, DELTA_MEAN_SIGNED = 0, 1, 2
 LSE_SUM_EXP, LSE_LOG = 0, 1
 ATTN_COMPACT_OUT = 1
 SCATTER_SRC_FULL = 1
-OP_SELECT, OP_SPARSE_ATTN, OP_STEP, OP_SPARSE_ATTN_KV = 1, 2, 3, 4
+LINEAR_COMPACT_OUT = 1
+OP_SELECT, OP_SPARSE_ATTN, OP_STEP, OP_SPARSE_ATTN_KV, OP_GATHERED_LINEAR = 1, 2, 3, 4, 5
 N_SKIP_CLAMP = 80
 NOALLOC_SCRATCH_BYTES = 4096
 
 EXPORTS = [
     "astraea_score", "astraea_select", "astraea_sparse_attn", "astraea_sparse_attn_noalloc", "astraea_scatter_reuse", "astraea_step",
-    "astraea_session_create", "astraea_session_destroy", "astraea_step_host",
+    "astraea_gathered_linear", "astraea_session_create", "astraea_session_destroy", "astraea_step_host",
     "astraea_workspace_bytes", "astraea_budget_to_k", "astraea_poll_error",
     "astraea_last_error", "astraea_version",
 ]
@@ -58,6 +59,7 @@ def lib() -> ctypes.CDLL:
         L.astraea_sparse_attn_noalloc.argtypes = [c_p, c_p, c_p] + [c_i64] * 9 + [c_p, c_i, c_p, c_i, c_p, c_p,
                                                                                  c_i, c_i, c_i, c_i, c_f, c_u, c_p]
         L.astraea_scatter_reuse.argtypes = [c_p, c_p, c_p, c_i, c_i, c_i, c_i, c_u, c_p]
+        L.astraea_gathered_linear.argtypes = [c_p, c_p, c_i, c_p, c_p, c_p, c_i, c_i, c_i, c_i, c_u, c_p, c_sz, c_p]
         L.astraea_step.argtypes = [c_p] * 11 + [c_i] * 6 + [c_f, c_f, c_i, c_i, c_p, c_sz, c_p]
         L.astraea_session_create.argtypes = [ctypes.POINTER(c_p), c_i, c_i, c_i, c_i, c_i]
         L.astraea_session_destroy.argtypes = [c_p]
@@ -70,7 +72,7 @@ def lib() -> ctypes.CDLL:
         L.astraea_last_error.restype = ctypes.c_char_p
         L.astraea_version.restype = ctypes.c_char_p
         for name in ("astraea_score", "astraea_select", "astraea_sparse_attn", "astraea_sparse_attn_noalloc", "astraea_scatter_reuse",
-                     "astraea_step", "astraea_session_create", "astraea_step_host", "astraea_budget_to_k",
+                     "astraea_step", "astraea_gathered_linear", "astraea_session_create", "astraea_step_host", "astraea_budget_to_k",
                      "astraea_poll_error"):
             getattr(L, name).restype = ctypes.c_int32
         _lib = L
@@ -147,6 +149,14 @@ def astraea_sparse_attn_noalloc(q, k, v, q_strides, k_strides, v_strides, q_idx,
 
 def astraea_scatter_reuse(cache, rows, idx, B, N, M, row_elems, flags=0, stream=None) -> None:
     _check(lib().astraea_scatter_reuse(_ptr(cache), _ptr(rows), _ptr(idx), B, N, M, row_elems, flags, _stream(stream)))
+
+
+def astraea_gathered_linear(x, idx, M, w, bias, y, B, N, K, N_out, flags=0, workspace=None, stream=None) -> None:
+    """y[b, idx[b,r], :] = x[b, idx[b,r], :] @ w.T + bias (idx None: all rows); other rows of y are left alone."""
+    if idx is not None and M == 0:
+        return          # an empty index tensor has a null data pointer, which the C ABI reads as "all rows"
+    _check(lib().astraea_gathered_linear(_ptr(x), _ptr(idx), M, _ptr(w), _ptr(bias), _ptr(y), B, N, K, N_out, flags,
+                                         _ptr(workspace), workspace.numel() if workspace is not None else 0, _stream(stream)))
 
 
 def astraea_step(x_cur, x_ref, lse_cache, n_skip, q, k, v, out_cache, score, idx_sel, idx_rem,

@@ -56,6 +56,7 @@ size_t astraea_workspace_bytes(int op, int B, int H, int N, int M, int d) {
     case ASTRAEA_OP_SPARSE_ATTN: return attn_workspace_bytes(B, H, N, M, d);
     case ASTRAEA_OP_SPARSE_ATTN_KV: return attn_kv_workspace_bytes(B, H, M, d);
     case ASTRAEA_OP_STEP: return attn_workspace_bytes(B, H, N, M, d) + align_up(select_workspace_bytes(B, N), 256);
+    case ASTRAEA_OP_GATHERED_LINEAR: return linear_workspace_bytes();
     default: return 0;
     }
 }
@@ -183,6 +184,27 @@ int32_t astraea_scatter_reuse(void *cache, const void *rows, const int32_t *idx,
     REQUIRE(cache && rows && idx, "astraea_scatter_reuse: null cache, rows or idx");
     REQUIRE(aligned16(cache) && aligned16(rows), "astraea_scatter_reuse: cache / rows must be 16-byte aligned");
     return launch_scatter(cache, rows, idx, B, N, M, row_elems, flags, (cudaStream_t)stream);
+}
+
+int32_t astraea_gathered_linear(const void *x, const int32_t *idx, int M, const void *w, const void *bias,
+                                void *y, int B, int N, int K, int N_out, uint32_t flags,
+                                void *workspace, size_t workspace_bytes, void *stream)
+{
+    REQUIRE(B > 0 && N > 0 && K > 0 && N_out > 0, "astraea_gathered_linear: B, N, K, N_out must be positive");
+    REQUIRE(!idx || (M >= 0 && M <= N), "astraea_gathered_linear: M=%d outside [0, N=%d]", M, N);
+    REQUIRE(K % 64 == 0, "astraea_gathered_linear: K=%d must be a multiple of 64", K);
+    REQUIRE(N_out % 8 == 0, "astraea_gathered_linear: N_out=%d must be a multiple of 8", N_out);
+    if (flags & ~ASTRAEA_LINEAR_COMPACT_OUT) return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_gathered_linear: unknown flags 0x%x", flags);
+    REQUIRE(!(flags & ASTRAEA_LINEAR_COMPACT_OUT) || idx, "astraea_gathered_linear: a compact output needs an index list");
+    if (!workspace || workspace_bytes < linear_workspace_bytes())
+        return fail(ASTRAEA_ERR_WORKSPACE_TOO_SMALL, "astraea_gathered_linear: workspace of %zu bytes, need %zu",
+                    workspace_bytes, linear_workspace_bytes());
+    REQUIRE((reinterpret_cast<uintptr_t>(workspace) & 255u) == 0, "astraea_gathered_linear: workspace must be 256-byte aligned");
+    if (idx && M == 0) return ASTRAEA_OK;
+    REQUIRE(x && w && y, "astraea_gathered_linear: null x, w or y");
+    REQUIRE(aligned16(x) && aligned16(w) && aligned16(y) && aligned16(bias), "astraea_gathered_linear: x, w, bias, y must be 16-byte aligned");
+    return launch_gathered_linear(x, idx, M, w, bias, y, B, N, K, N_out, flags, reinterpret_cast<int *>(workspace),
+                                  (cudaStream_t)stream);
 }
 
 int32_t astraea_step(const void *x_cur, void *x_ref, float *lse_cache, int32_t *n_skip,

@@ -40,6 +40,7 @@
 
 #include "common.cuh"
 #include "sm100_ptx.cuh"
+#include "bounded_wait.cuh"
 
 namespace astraea {
 namespace {
@@ -54,7 +55,6 @@ constexpr int kSplit = 2;                        // softmax warpgroups per query
 // allows, because a redo costs the CTA two more passes over the keys.
 constexpr float kTileSumLimit = 1152921504606846976.0f;   // 2^60
 constexpr uint32_t kTmemCols = 512;
-constexpr uint64_t kWaitLimitNs = 1000000000ull; // bounded waits: one second
 
 template <int DH> struct Cfg {
     // head_dim = kMain (whole 64-column, 128-byte-swizzled chunks) + kTail (8 columns at head_dim 72,
@@ -166,31 +166,6 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     float r;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
     return r;
-}
-
-__device__ __forceinline__ bool elect_one() {
-    uint32_t pred;
-    asm volatile("{\n\t.reg .pred px;\n\telect.sync _|px, 0xffffffff;\n\tselp.u32 %0, 1, 0, px;\n\t}" : "=r"(pred));
-    return pred != 0;
-}
-
-// Bounded mbarrier wait.  Gives up after the limit, or at once when another wait of this CTA
-// already gave up; the caller carries on (its results are void, the error word says so).
-__device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err_word) {
-    if (mbar_try_wait(bar, parity)) return;
-    if (*abort_flag) return;
-    const uint64_t t0 = globaltimer_ns();
-    uint32_t spins = 0;
-    while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 255u) == 0) {
-            if (*abort_flag) return;
-            if (globaltimer_ns() - t0 > kWaitLimitNs) {
-                *abort_flag = 1;
-                atomicExch(err_word, kErrTimeout);
-                return;
-            }
-        }
-    }
 }
 
 struct Bars {

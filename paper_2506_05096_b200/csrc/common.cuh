@@ -31,6 +31,10 @@ size_t select_workspace_bytes(int B, int N_sel);
 int32_t launch_scatter(void *cache, const void *rows, const int32_t *idx, int B, int N, int M,
                        int row_elems, uint32_t flags, cudaStream_t stream);
 
+size_t linear_workspace_bytes();
+int32_t launch_gathered_linear(const void *x, const int32_t *idx, int M, const void *w, const void *bias, void *y,
+                               int B, int N, int K, int N_out, uint32_t flags, int *err_word, cudaStream_t stream);
+
 struct AttnArgs {
     const void *q, *k, *v;
     int64_t q_sb, q_sh, q_sn, k_sb, k_sh, k_sn, v_sb, v_sh, v_sn;

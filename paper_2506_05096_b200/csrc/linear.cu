@@ -1,0 +1,295 @@
+// astraea_gathered_linear: y[b, i, :] = x[b, i, :] W^T + bias for the listed token rows i = idx[b, r];
+// the other rows of y keep the cached result (Algorithm 1 lines 4-7 applied to a linear layer of the
+// block: the query projection of the selected tokens, the output projection and the MLP on selected
+// rows; with idx == NULL the key / value projections of all tokens).
+//
+// A dense contraction, so it runs on the tcgen05 tensor cores.  Persistent CTAs, one per SM, walk over
+// 128-row x 256-column output tiles (column tiles of one row tile are neighbours in the walk, so the
+// gathered rows stay in L2 while W, which is small, lives there anyway).  Warp roles:
+//   warps 0-3  epilogue: one thread per output row; TMEM -> registers -> (+ bias) -> bf16 -> the row of y
+//              that idx names (fused scatter).  Two accumulators of 256 TMEM columns, so the epilogue of a
+//              tile runs under the main loop of the next;
+//   warps 4-7  gather of the A operand: the listed rows of x, 64 columns (128 bytes) per pipeline stage,
+//              by 16-byte cp.async into the 128-byte-swizzled layout the MMA reads (rows past the end
+//              are zero-filled);
+//   warp 8     TMA producer of the B operand: a 256 x 64 tile of W per stage (rows past N_out read as zero);
+//   warp 9     tcgen05.mma issuer: four 128 x 256 x 16 SS MMAs per stage into the tile's accumulator.
+// Stages: 4 x (16 KB of A + 32 KB of W).  Every mbarrier wait is bounded; on a timeout the CTA raises the
+// error word, the remaining waits return at once, and the CTA runs out.
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+#include "bounded_wait.cuh"
+
+namespace astraea {
+namespace {
+
+using namespace ptx;
+
+constexpr int kBM = 128, kBN = 256, kBK = 64;
+constexpr int kStages = 4;
+constexpr int kLag = 2;                                  // stages a gather thread keeps in flight
+constexpr int kABytes = kBM * kBK * 2, kBBytes = kBN * kBK * 2;
+constexpr int kEpiWarps = 4, kGatherWarps = 4;
+constexpr int kThreads = (kEpiWarps + kGatherWarps + 2) * 32;
+constexpr int kTmaWarp = kEpiWarps + kGatherWarps, kMmaWarp = kTmaWarp + 1;
+constexpr int kSmemBytes = kStages * (kABytes + kBBytes) + 256 + 1024;
+constexpr uint32_t kAccCols = kBN, kTmemCols = 2 * kBN;
+
+struct LinParams {
+    const __nv_bfloat16 *x;
+    const int32_t *idx;
+    int M;                       // rows listed per batch element (N when idx == nullptr)
+    const __nv_bfloat16 *bias;
+    __nv_bfloat16 *y;
+    int B, N, K, N_out;
+    int compact;
+    int *err_word;
+};
+
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, bool valid) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(valid ? 16 : 0) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// 2-D tiled load global -> shared, completion counted in bytes on an mbarrier
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *m, uint32_t bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(m), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+
+// token row of the g-th listed row (all batch elements in one list), or -1
+__device__ __forceinline__ long long source_row(const LinParams &p, long long g, long long total, long long *out_row) {
+    if (g >= total) return -1;
+    const int b = (int)(g / p.M), r = (int)(g - (long long)b * p.M);
+    const int tok = p.idx ? __ldg(p.idx + g) : r;
+    if ((unsigned)tok >= (unsigned)p.N) return -2;
+    if (out_row) *out_row = p.compact ? g : (long long)b * p.N + tok;
+    return (long long)b * p.N + tok;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+gathered_linear_kernel(const __grid_constant__ CUtensorMap tmap_w, const LinParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sA = smem_base, sB = sA + kStages * kABytes, bars = sB + kStages * kBBytes;
+    const uint32_t bar_full = bars, bar_empty = bars + 8 * kStages, bar_acc_full = bars + 16 * kStages,
+                   bar_acc_empty = bar_acc_full + 16;
+
+    const int tid = threadIdx.x;
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);        // warp-uniform
+    const int lane = tid & 31;
+    const long long total_rows = (long long)p.B * p.M;
+    const int tiles_m = (int)((total_rows + kBM - 1) / kBM), tiles_n = (p.N_out + kBN - 1) / kBN;
+    const int total_tiles = tiles_m * tiles_n, k_steps = p.K / kBK;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(bar_full + 8 * s, kGatherWarps * 32 + 1);     // every gather thread + the TMA producer
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int a = 0; a < 2; ++a) { mbar_init(bar_acc_full + 8 * a, 1); mbar_init(bar_acc_empty + 8 * a, kEpiWarps * 32); }
+        fence_barrier_init();
+    }
+    if (warp == kMmaWarp) {
+        tmem_alloc(smem_u32(&tmem_slot), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_slot;
+
+    if (warp < kEpiWarps) {
+        // ------------------------------------------------ epilogue
+        const int row = warp * 32 + lane;
+        const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);
+        int it = 0;
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
+            const int tm = tile / tiles_n, tn = tile - tm * tiles_n;
+            const int acc = it & 1, n0 = tn * kBN;
+            long long out_row = -1;
+            const long long src = source_row(p, (long long)tm * kBM + row, total_rows, &out_row);
+            if (src == -2 && tn == 0) atomicExch(p.err_word, kErrBadIndex);
+            __nv_bfloat16 *dst = (src >= 0) ? p.y + out_row * p.N_out + n0 : nullptr;
+            wait_bar(bar_acc_full + 8 * acc, (it >> 1) & 1, &abort_flag, p.err_word);
+            tc_fence_after();
+            if (abort_flag) dst = nullptr;
+#pragma unroll 1
+            for (int c = 0; c < kBN; c += 32) {
+                uint32_t o[32];
+                tmem_ld32(t_row + acc * kAccCols + c, o);
+                tc_wait_ld();
+                if (c + 32 == kBN) {                     // the accumulator has been read: the MMA warp may reuse it
+                    tc_fence_before();
+                    mbar_arrive(bar_acc_empty + 8 * acc);
+                }
+                if (dst == nullptr) continue;
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                    const int col = n0 + c + v * 8;
+                    if (col >= p.N_out) break;           // N_out is a multiple of 8
+                    float f[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(o[v * 8 + i]);
+                    if (p.bias) {
+                        const uint4 bb = __ldg(reinterpret_cast<const uint4 *>(p.bias + col));
+                        const uint32_t bw[4] = {bb.x, bb.y, bb.z, bb.w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            f[2 * i] += __uint_as_float(bw[i] << 16);
+                            f[2 * i + 1] += __uint_as_float(bw[i] & 0xffff0000u);
+                        }
+                    }
+                    uint32_t w[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        __nv_bfloat162 v2 = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+                        w[i] = *reinterpret_cast<uint32_t *>(&v2);
+                    }
+                    *reinterpret_cast<uint4 *>(dst + c + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+            }
+        }
+    } else if (warp < kEpiWarps + kGatherWarps) {
+        // ------------------------------------------------ gather of the A rows (cp.async, 128-byte swizzle)
+        const int t = tid - kEpiWarps * 32;                   // 0..127
+        const int chunk = t & 7, row0 = t >> 3;               // this thread: 16-byte chunk `chunk` of rows row0 + 16 i
+        int g = 0;                                            // running stage count over all tiles
+        auto publish = [&](int gs) {                          // the copies of stage gs have landed
+            fence_proxy_async_smem();
+            mbar_arrive(bar_full + 8 * (gs % kStages));
+        };
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+            const int tm = tile / tiles_n;
+            const __nv_bfloat16 *src[8];
+            uint32_t off[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int r = row0 + 16 * i;
+                const long long s = source_row(p, (long long)tm * kBM + r, total_rows, nullptr);
+                src[i] = (s >= 0) ? p.x + s * p.K + chunk * 8 : nullptr;
+                off[i] = r * 128 + ((chunk ^ (r & 7)) << 4);
+            }
+            for (int ks = 0; ks < k_steps; ++ks, ++g) {
+                const int st = g % kStages;
+                wait_bar(bar_empty + 8 * st, ((g / kStages) & 1) ^ 1, &abort_flag, p.err_word);
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    cp_async_16(sA + st * kABytes + off[i], src[i] ? (const void *)(src[i] + ks * kBK) : (const void *)p.x, src[i] != nullptr);
+                cp_async_commit();
+                if (g >= kLag) { cp_async_wait<kLag>(); publish(g - kLag); }
+            }
+        }
+        // drain
+        cp_async_wait<0>();
+        for (int gs = (g > kLag ? g - kLag : 0); gs < g; ++gs) publish(gs);
+    } else if (warp == kTmaWarp) {
+        // ------------------------------------------------ TMA producer of the W tiles
+        if (elect_one()) prefetch_tensormap(&tmap_w);
+        int g = 0;
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+            const int tn = tile % tiles_n;
+            for (int ks = 0; ks < k_steps; ++ks, ++g) {
+                const int st = g % kStages;
+                wait_bar(bar_empty + 8 * st, ((g / kStages) & 1) ^ 1, &abort_flag, p.err_word);
+                if (elect_one()) {
+                    mbar_arrive_expect_tx(bar_full + 8 * st, kBBytes);
+                    tma_load_2d(sB + st * kBBytes, &tmap_w, bar_full + 8 * st, ks * kBK, tn * kBN);
+                }
+                __syncwarp();
+            }
+        }
+        // every copy issued above must have landed before the CTA's shared memory is released
+        for (int gs = (g > kStages ? g - kStages : 0); gs < g; ++gs)
+            wait_bar(bar_full + 8 * (gs % kStages), (gs / kStages) & 1, &abort_flag, p.err_word);
+    } else {
+        // ------------------------------------------------ MMA issuer
+        constexpr uint32_t idesc = idesc_bf16(kBM, kBN, false);
+        int g = 0, it = 0;
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
+            const int acc = it & 1;
+            wait_bar(bar_acc_empty + 8 * acc, ((it >> 1) & 1) ^ 1, &abort_flag, p.err_word);
+            for (int ks = 0; ks < k_steps; ++ks, ++g) {
+                const int st = g % kStages;
+                wait_bar(bar_full + 8 * st, (g / kStages) & 1, &abort_flag, p.err_word);
+                tc_fence_after();
+                if (elect_one()) {
+#pragma unroll
+                    for (int kk = 0; kk < kBK / 16; ++kk)
+                        mma_ss(tmem + acc * kAccCols,
+                               smem_desc(sA + st * kABytes + kk * 32, 16, 1024, kSwizzle128B),
+                               smem_desc(sB + st * kBBytes + kk * 32, 16, 1024, kSwizzle128B),
+                               idesc, (ks > 0 || kk > 0) ? 1u : 0u);
+                    tc_commit(bar_empty + 8 * st);
+                    if (ks == k_steps - 1) tc_commit(bar_acc_full + 8 * acc);
+                }
+                __syncwarp();
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kMmaWarp) tmem_dealloc(tmem, kTmemCols);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+}  // namespace
+
+size_t linear_workspace_bytes() { return 256; }
+
+int32_t launch_gathered_linear(const void *x, const int32_t *idx, int M, const void *w, const void *bias, void *y,
+                               int B, int N, int K, int N_out, uint32_t flags, int *err_word, cudaStream_t stream)
+{
+    static EncodeTiledFn enc = nullptr;
+    if (!enc) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            enc = reinterpret_cast<EncodeTiledFn>(ptr);
+        if (!enc) return fail(ASTRAEA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    }
+    // W as a 2-D tensor (K, N_out) with 128-byte-swizzled boxes of 64 columns x 256 rows
+    CUtensorMap mw;
+    cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)N_out};
+    cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)kBN};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(&mw, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(w), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(ASTRAEA_ERR_INVALID_ARG, "astraea_gathered_linear: tensor map of W rejected (CUresult %d)", (int)r);
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(gathered_linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+            return check_launch("astraea_gathered_linear (shared memory attribute)");
+        attr_set = true;
+    }
+    LinParams p;
+    p.x = reinterpret_cast<const __nv_bfloat16 *>(x);
+    p.idx = idx;
+    p.M = idx ? M : N;
+    p.bias = reinterpret_cast<const __nv_bfloat16 *>(bias);
+    p.y = reinterpret_cast<__nv_bfloat16 *>(y);
+    p.B = B; p.N = N; p.K = K; p.N_out = N_out;
+    p.compact = (flags & ASTRAEA_LINEAR_COMPACT_OUT) ? 1 : 0;
+    p.err_word = err_word;
+    const long long rows = (long long)B * p.M;
+    const long long tiles = ((rows + kBM - 1) / kBM) * ((N_out + kBN - 1) / kBN);
+    const int grid = (int)(tiles < kNumSMs ? tiles : kNumSMs);
+    gathered_linear_kernel<<<grid, kThreads, kSmemBytes, stream>>>(mw, p);
+    return check_launch("astraea_gathered_linear");
+}
+
+}  // namespace astraea

@@ -456,3 +456,64 @@ def test_session_step_host_equals_the_device_path_and_the_oracle(oracle):
             err = np.abs(bf16_dev_to_f64(out) - want_o)
             assert err.max() < ATTN_MAX_ABS and err.mean() < ATTN_MEAN_ABS
     sess.close()
+
+
+# ------------------------------------------------------------- linear layers on the selected rows
+LINEAR_MAX_ABS = 2e-2        # one bf16 rounding of outputs of magnitude <= ~5 (2^-8 relative) on top of fp32 sums
+LINEAR_MEAN_ABS = 2e-3
+
+
+def _linear_case(oracle, B, N, K, N_out, M, seed, bias=True, compact=False, dense=False):
+    rng = np.random.default_rng(seed)
+    x = synth.f32_to_bf16_bits(rng.standard_normal((B, N, K)).astype(np.float32))
+    w = synth.f32_to_bf16_bits((rng.standard_normal((N_out, K)) / math.sqrt(K)).astype(np.float32))
+    bb = synth.f32_to_bf16_bits(rng.standard_normal(N_out).astype(np.float32)) if bias else None
+    cache = synth.f32_to_bf16_bits(rng.standard_normal((B, N, N_out)).astype(np.float32))
+    idx = None if dense else np.stack([np.sort(rng.choice(N, M, replace=False)) for _ in range(B)]).astype(np.int32)
+    want = oracle.gathered_linear(f64(x), f64(w), None if bb is None else f64(bb), idx, f64(cache))
+    y = torch.zeros(B, M, N_out, dtype=torch.bfloat16, device="cuda") if compact else to_dev_bf16(cache)
+    ws = A.new_workspace(A.OP_GATHERED_LINEAR, 0, 0, 0, 0, 0)
+    A.astraea_gathered_linear(to_dev_bf16(x), None if idx is None else dev(idx), M, to_dev_bf16(w),
+                              None if bb is None else to_dev_bf16(bb), y, B, N, K, N_out,
+                              flags=A.LINEAR_COMPACT_OUT if compact else 0, workspace=ws)
+    A.astraea_poll_error(ws)
+    got = bf16_dev_to_f64(y)
+    if compact:
+        want = np.take_along_axis(want, idx[:, :, None].astype(np.int64), 1)
+    elif idx is not None:
+        mask = np.ones((B, N), bool)
+        for b in range(B):
+            mask[b, idx[b]] = False
+        assert np.array_equal(got[mask], f64(cache)[mask])          # rows that were not listed keep the cache, bit for bit
+    err = np.abs(got - want)
+    assert err.max() < LINEAR_MAX_ABS and err.mean() < LINEAR_MEAN_ABS, (err.max(), err.mean())
+
+
+@pytest.mark.parametrize("N,K,N_out,M", [(300, 64, 256, 77), (1000, 192, 512, 333), (129, 128, 264, 129), (40, 64, 8, 1),
+                                         (700, 320, 1160, 450)])
+def test_gathered_linear_ragged_tiles(oracle, N, K, N_out, M):
+    _linear_case(oracle, 2, N, K, N_out, M, seed=31)
+
+
+def test_gathered_linear_all_rows_no_bias_compact_and_many_k_steps(oracle):
+    _linear_case(oracle, 1, 260, 64, 256, 0, seed=32, dense=True)
+    _linear_case(oracle, 2, 200, 128, 320, 90, seed=33, bias=False)
+    _linear_case(oracle, 2, 200, 128, 320, 90, seed=34, compact=True)
+    _linear_case(oracle, 1, 150, 64 * 23, 256, 100, seed=35)           # every pipeline stage several times over
+    _linear_case(oracle, 1, 128 * 5 + 3, 64, 256 * 3, 128 * 5 + 3, seed=36)   # more tiles than fit one pass of two accumulators
+
+
+def test_gathered_linear_bad_index_and_no_rows():
+    B, N, K, N_out = 1, 64, 64, 64
+    x = torch.ones(B, N, K, dtype=torch.bfloat16, device="cuda")
+    w = torch.ones(N_out, K, dtype=torch.bfloat16, device="cuda")
+    y = torch.zeros(B, N, N_out, dtype=torch.bfloat16, device="cuda")
+    ws = A.new_workspace(A.OP_GATHERED_LINEAR, 0, 0, 0, 0, 0)
+    A.astraea_gathered_linear(x, torch.empty(1, 0, dtype=torch.int32, device="cuda"), 0, w, None, y, B, N, K, N_out, workspace=ws)
+    assert float(y.abs().sum()) == 0.0
+    idx = torch.tensor([[1, 64, 2 ** 30]], dtype=torch.int32, device="cuda")
+    A.astraea_gathered_linear(x, idx, 3, w, None, y, B, N, K, N_out, workspace=ws)
+    with pytest.raises(A.AstraeaError) as e:
+        A.astraea_poll_error(ws)
+    assert e.value.code == A.ERR_BAD_INDEX
+    assert float(y[0, 1, 0]) == 64.0 and float(y[0, 2:].abs().sum()) == 0.0
