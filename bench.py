@@ -154,6 +154,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-next", action="store_true", help="skip the query projection of the selected rows (astraea_gathered_linear)")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
     theta = args.theta
@@ -285,7 +286,34 @@ def main():
             sweep[str(th)] = {"ms_per_step": tot / n_st, "attn_ms": float(pp[2]), "tflops": f / (tot / n_st * 1e-3) / 1e12,
                               "attn_tflops": f / (pp[2] * 1e-3) / 1e12}
         A.astraea_poll_error(ws)
-    clocks = sampler.stop()      # covers warm-up, the timed steps and the keep-ratio sweep
+    # ---- the next layer of the block on the same selection: query projection of the selected rows
+    nxt = None
+    if not args.no_next and rank == 0 and world == 1 and M > 0:
+        g = torch.Generator(device="cuda").manual_seed(7)
+        w_q = (torch.randn(D, D, device="cuda", generator=g) / math.sqrt(D)).to(torch.bfloat16)
+        ys = [torch.zeros(B, N, D, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+        ws_lin = A.new_workspace(A.OP_GATHERED_LINEAR, 0, 0, 0, 0, 0)
+        step(0, k_keep)          # the selection of the timed keep-ratio (the sweep left another one behind)
+        idx_now = idx_sel[:, :M] if B == 1 else idx_sel.view(-1)[:B * M].view(B, M)
+        reps = 10
+        for t in range(3):
+            A.astraea_gathered_linear(sets[t & 1]["x_cur"], idx_now, M, w_q, None, ys[t & 1], B, N, D, D, workspace=ws_lin)
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+        torch.cuda.synchronize()
+        evs[0].record()
+        for t in range(reps):     # two alternating x / y sets: 2 x (M rows of x and y) + W > 126 MB L2 on every workload but tiny
+            A.astraea_gathered_linear(sets[t & 1]["x_cur"], idx_now, M, w_q, None, ys[t & 1], B, N, D, D, workspace=ws_lin)
+            evs[t + 1].record()
+        torch.cuda.synchronize()
+        A.astraea_poll_error(ws_lin)
+        lin_ms = float(np.median([evs[i].elapsed_time(evs[i + 1]) for i in range(reps)]))
+        lin_flops = 2.0 * B * M * D * D
+        nxt = {"gathered_linear(q projection of the selected rows)": {
+            "ms": lin_ms, "TFLOP/s": lin_flops / (lin_ms * 1e-3) / 1e12,
+            "frac_bf16_peak": lin_flops / (lin_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+            "shape": {"rows": B * M, "K": D, "N_out": D}}}
+        del ys, w_q
+    clocks = sampler.stop()      # covers warm-up, the timed steps, the keep-ratio sweep and the projection
 
     # ---- end to end through the host-buffer session
     e2e = None
@@ -328,7 +356,7 @@ def main():
                            "l2": "two alternating input sets, %.0f MB touched per step > 126 MB L2"
                                  % ((6 * B * N * D * 2) / 1e6)},
                 "gpu_launches": 4 * args.steps, "clocks": clocks, "roofline": roofline, "kernels": kernels,
-                "keep_ratio_sweep": sweep, "e2e": e2e, "cpu_baseline": cpu}
+                "keep_ratio_sweep": sweep, "next": nxt, "e2e": e2e, "cpu_baseline": cpu}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -50,10 +50,16 @@ using namespace ptx;
 constexpr int kBlockM = 128;                     // rows of one query tile
 constexpr int kTilesM = 2;                       // query tiles per CTA
 constexpr int kSplit = 2;                        // softmax warpgroups per query tile: one takes the even key tiles, one the odd
-// A tile's sum of exponentials above this means that the reference maximum is too low.  fp32 and bf16 share the
-// exponent range, so the limit only has to keep row sums and accumulators far from overflow; it is as high as that
-// allows, because a redo costs the CTA two more passes over the keys.
-constexpr float kTileSumLimit = 1152921504606846976.0f;   // 2^60
+// The speculative reference of a row is the exact maximum of its first key tile plus kRefShift (log2 domain), and
+// a tile whose sum of exponentials passes kTileSumLimit means that this reference is too low.  fp32 and bf16 share
+// the exponent range and keep their relative precision across it, so the reference may sit anywhere in a wide
+// window: the shift leaves 2^-48 .. 2^-126 for the terms below a maximum that IS in the first tile (78 bits), and
+// the limit leaves 2^27 of head room above 2^100 for the number of keys times the magnitude of the values.
+// Together a later key may beat the first tile's maximum by 148 * ln 2 = 102 nats before the CTA has to redo its
+// work, which costs two more passes over the keys: heavy-tailed logits (per-token norms) reach 40-60 nats in some
+// row of most CTAs, but not 100.
+constexpr float kRefShift = 48.0f;
+constexpr float kTileSumLimit = 1267650600228229401496703205376.0f;   // 2^100
 constexpr uint32_t kTmemCols = 512;
 
 template <int DH> struct Cfg {
@@ -177,6 +183,7 @@ struct Bars {
 
 template <int DH> struct SoftmaxState {
     float sl2, m_ref, l_sum;
+    float shift;                    // the exponentials are taken against m_ref * sl2 + shift (log2 domain)
     uint32_t t_s0, t_o, bar_s, bar_p, bar_done;
     int N, n_tiles;
     float *ref_x;                   // split: the reference of this thread's row, shared by the tile's two warpgroups
@@ -292,7 +299,7 @@ __device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j, int g)
         if (st.ref_bar == 3) asm volatile("bar.arrive 3, 256;" ::: "memory");
         else asm volatile("bar.arrive 4, 256;" ::: "memory");
     }
-    const float neg = -st.m_ref * sl2;
+    const float neg = -st.m_ref * sl2 - st.shift;
 #pragma unroll
     for (int i = 0; i < NS; i += 2) ffma2(cur[i], cur[i + 1], sl2, neg);
     // kPolyOf16 of every 16 exponentials go to the FMA pipe, the rest to the XU
@@ -384,6 +391,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     }
 
     st.m_ref = -INFINITY;
+    st.shift = kRefShift;
     if (par == 1) {
         // the even-tile warpgroup takes the exact row maxima of key tile 0 and hands them over
         if (tile == 0) asm volatile("bar.sync 3, 256;" ::: "memory");
@@ -401,6 +409,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
         if (tile == 0) asm volatile("bar.sync 1, 256;" ::: "memory");
         else asm volatile("bar.sync 2, 256;" ::: "memory");
         st.m_ref = fmaxf(xchg[wtid].x, xchg[wtid + kBlockM].x);
+        st.shift = 0.f;
         st.l_sum = 0.f;
         for (int j = par; j < n_tiles; j += kSplit) softmax_step<DH, kExact>(st, j, 2 * n_tiles + j);
         wait_bar(st.bar_done, 1, abort_flag, p.err_word);
@@ -422,7 +431,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
         dst = p.out + (orow * p.H + h) * DH;
         if (p.lse_out && par == 0) {
             const size_t li = p.compact ? (((size_t)b * p.H + h) * p.M + m) : (((size_t)b * p.H + h) * p.N_tok + tok);
-            p.lse_out[li] = st.m_ref * p.scale + logf(l_sum);
+            p.lse_out[li] = st.m_ref * p.scale + st.shift * 0.6931471805599453f + logf(l_sum);
         }
     }
 #pragma unroll

@@ -11,7 +11,8 @@
 //              tile runs under the main loop of the next;
 //   warps 4-7  gather of the A operand: the listed rows of x, 64 columns (128 bytes) per pipeline stage,
 //              by 16-byte cp.async into the 128-byte-swizzled layout the MMA reads (rows past the end
-//              are zero-filled);
+//              are zero-filled); the copies arrive on the stage's barrier by themselves, so a thread never
+//              waits for its own copies, only for a free stage;
 //   warp 8     TMA producer of the B operand: a 256 x 64 tile of W per stage (rows past N_out read as zero);
 //   warp 9     tcgen05.mma issuer: four 128 x 256 x 16 SS MMAs per stage into the tile's accumulator.
 // Stages: 4 x (16 KB of A + 32 KB of W).  Every mbarrier wait is bounded; on a timeout the CTA raises the
@@ -27,7 +28,6 @@ using namespace ptx;
 
 constexpr int kBM = 128, kBN = 256, kBK = 64;
 constexpr int kStages = 4;
-constexpr int kLag = 2;                                  // stages a gather thread keeps in flight
 constexpr int kABytes = kBM * kBK * 2, kBBytes = kBN * kBK * 2;
 constexpr int kEpiWarps = 4, kGatherWarps = 4;
 constexpr int kThreads = (kEpiWarps + kGatherWarps + 2) * 32;
@@ -49,8 +49,11 @@ struct LinParams {
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, bool valid) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(valid ? 16 : 0) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+// arrive on the mbarrier once every cp.async this thread has issued so far has landed (the arrival is one of
+// those the barrier was initialised to expect)
+__device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
 
 // 2-D tiled load global -> shared, completion counted in bytes on an mbarrier
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *m, uint32_t bar, int c0, int c1) {
@@ -162,10 +165,6 @@ gathered_linear_kernel(const __grid_constant__ CUtensorMap tmap_w, const LinPara
         const int t = tid - kEpiWarps * 32;                   // 0..127
         const int chunk = t & 7, row0 = t >> 3;               // this thread: 16-byte chunk `chunk` of rows row0 + 16 i
         int g = 0;                                            // running stage count over all tiles
-        auto publish = [&](int gs) {                          // the copies of stage gs have landed
-            fence_proxy_async_smem();
-            mbar_arrive(bar_full + 8 * (gs % kStages));
-        };
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
             const int tm = tile / tiles_n;
             const __nv_bfloat16 *src[8];
@@ -183,13 +182,9 @@ gathered_linear_kernel(const __grid_constant__ CUtensorMap tmap_w, const LinPara
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
                     cp_async_16(sA + st * kABytes + off[i], src[i] ? (const void *)(src[i] + ks * kBK) : (const void *)p.x, src[i] != nullptr);
-                cp_async_commit();
-                if (g >= kLag) { cp_async_wait<kLag>(); publish(g - kLag); }
+                cp_async_arrive(bar_full + 8 * st);           // asynchronous: the thread goes on to the next free stage
             }
         }
-        // drain
-        cp_async_wait<0>();
-        for (int gs = (g > kLag ? g - kLag : 0); gs < g; ++gs) publish(gs);
     } else if (warp == kTmaWarp) {
         // ------------------------------------------------ TMA producer of the W tiles
         if (elect_one()) prefetch_tensormap(&tmap_w);
@@ -219,6 +214,7 @@ gathered_linear_kernel(const __grid_constant__ CUtensorMap tmap_w, const LinPara
             for (int ks = 0; ks < k_steps; ++ks, ++g) {
                 const int st = g % kStages;
                 wait_bar(bar_full + 8 * st, (g / kStages) & 1, &abort_flag, p.err_word);
+                fence_proxy_async_smem();             // the gathered rows were written through the generic proxy
                 tc_fence_after();
                 if (elect_one()) {
 #pragma unroll

@@ -255,13 +255,13 @@ def test_attn_peaked_softmax(oracle):
 
 @pytest.mark.parametrize("d", [64, 72, 128])
 def test_attn_reference_maximum_far_too_low_is_repaired_exactly(oracle, d):
-    # logits of order +-250: in most rows a later key tile beats the first tile's maximum by more than 60 nats,
+    # logits of order +-600: in most rows a later key tile beats the first tile's maximum by more than 100 nats,
     # past the speculation limit of the kernel, so that the CTAs redo their work against exact row maxima;
     # three CTAs per head, the last one with a single query tile, ragged last key tile
-    _attn_case(oracle, 1, 2, 900, d, 600, seed=20 + d, amp=8.0)
+    _attn_case(oracle, 1, 2, 900, d, 600, seed=20 + d, amp=12.0)
     # a single key tile and exactly two: the odd-tile warpgroup has nothing, or one tile, to contribute
-    _attn_case(oracle, 1, 1, 40, d, 40, seed=21 + d, amp=8.0)
-    _attn_case(oracle, 2, 1, 100, d, 70, seed=22 + d, amp=8.0)
+    _attn_case(oracle, 1, 1, 40, d, 40, seed=21 + d, amp=12.0)
+    _attn_case(oracle, 2, 1, 100, d, 70, seed=22 + d, amp=12.0)
 
 
 @pytest.mark.parametrize("d", [64, 72, 128])
