@@ -313,6 +313,22 @@ def main():
             "frac_bf16_peak": lin_flops / (lin_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
             "shape": {"rows": B * M, "K": D, "N_out": D}}}
         del ys, w_q
+        # the same steps recorded once as a CUDA graph (a fixed budget schedule) and replayed with one launch
+        T = 10
+        sched = A.Schedule([k_keep] * T, [sets[t & 1]["x_cur"] for t in range(T)], [sets[t & 1]["q"] for t in range(T)],
+                           [sets[t & 1]["k"] for t in range(T)], [sets[t & 1]["v"] for t in range(T)], x_ref, lse, n_skip,
+                           out, score, idx_sel, idx_rem, B, H, N, N_sel, d, w_alpha, 1.0, workspace=ws)
+        sched.launch()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        sched.launch()
+        e1.record()
+        torch.cuda.synchronize()
+        A.astraea_poll_error(ws)
+        nxt["schedule_graph(%d steps, one launch)" % T] = {"ms_per_step": e0.elapsed_time(e1) / T,
+                                                          "ms_per_step_separate_launches": ms_per_step}
+        sched.close()
     clocks = sampler.stop()      # covers warm-up, the timed steps, the keep-ratio sweep and the projection
 
     # ---- end to end through the host-buffer session

@@ -218,6 +218,33 @@ int32_t astraea_step(const void *x_cur, void *x_ref, float *lse_cache, int32_t *
                      void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * A schedule of T denoising steps of one attention block as ONE CUDA graph (the per-step token budgets
+ * theta_t of Section 3.3 are fixed before the generation starts, so the whole loop of Algorithm 1 can be
+ * recorded once and replayed): step t runs astraea_step with budget k_keep[t] on the inputs x_cur[t], q[t],
+ * k[t], v[t] and the shared state.  A budget of 0 with no always-kept tokens skips the attention of that step
+ * (scores and counters are still updated); the first step of a generation should carry k_keep = N_sel.
+ * astraea_schedule_create captures and instantiates the graph (host work only, nothing runs on the device);
+ * astraea_schedule_launch enqueues all T steps on `stream` with a single graph launch, asynchronously.
+ *   k_keep            : HOST int32 [T]
+ *   x_cur, q, k, v    : HOST arrays of T DEVICE pointers (bf16 [B,N,D] each; the producers of those tensors,
+ *                       i.e. the rest of the model, are outside this library)
+ *   x_ref ... idx_rem, workspace : device buffers as for astraea_step; idx_sel holds at least B*N entries,
+ *                       idx_rem at least B*N_sel (or NULL), workspace the ASTRAEA_OP_STEP size for M = N
+ * The graph keeps the pointers, not the data: the buffers must stay allocated while the schedule exists and
+ * may be refilled between launches.  Errors: as astraea_step, plus CUDA for a failed capture.
+ */
+typedef struct astraea_schedule astraea_schedule;
+int32_t astraea_schedule_create(astraea_schedule **schedule, int T, const int32_t *k_keep,
+                                const void *const *x_cur, const void *const *q, const void *const *k,
+                                const void *const *v, void *x_ref, float *lse_cache, int32_t *n_skip,
+                                void *out_cache, float *score, int32_t *idx_sel, int32_t *idx_rem,
+                                int B, int H, int N, int N_sel, int d,
+                                float w_alpha, float w_beta, int delta_mode, int lse_mode,
+                                void *workspace, size_t workspace_bytes);
+int32_t astraea_schedule_launch(astraea_schedule *schedule, void *stream);
+void    astraea_schedule_destroy(astraea_schedule *schedule);
+
+/*
  * Host-buffer session: the library owns the device-side state of one attention block
  * (x_ref, LSE cache, counters, output cache) and staging buffers, and each step copies
  * the HOST inputs to the device, runs the step (score, select, refresh of x_ref,

@@ -28,7 +28,8 @@ NOALLOC_SCRATCH_BYTES = 4096
 
 EXPORTS = [
     "astraea_score", "astraea_select", "astraea_sparse_attn", "astraea_sparse_attn_noalloc", "astraea_scatter_reuse", "astraea_step",
-    "astraea_gathered_linear", "astraea_session_create", "astraea_session_destroy", "astraea_step_host",
+    "astraea_gathered_linear", "astraea_schedule_create", "astraea_schedule_launch", "astraea_schedule_destroy",
+    "astraea_session_create", "astraea_session_destroy", "astraea_step_host",
     "astraea_workspace_bytes", "astraea_budget_to_k", "astraea_poll_error",
     "astraea_last_error", "astraea_version",
 ]
@@ -61,6 +62,11 @@ def lib() -> ctypes.CDLL:
         L.astraea_scatter_reuse.argtypes = [c_p, c_p, c_p, c_i, c_i, c_i, c_i, c_u, c_p]
         L.astraea_gathered_linear.argtypes = [c_p, c_p, c_i, c_p, c_p, c_p, c_i, c_i, c_i, c_i, c_u, c_p, c_sz, c_p]
         L.astraea_step.argtypes = [c_p] * 11 + [c_i] * 6 + [c_f, c_f, c_i, c_i, c_p, c_sz, c_p]
+        L.astraea_schedule_create.argtypes = [ctypes.POINTER(c_p), c_i, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p,
+                                              c_i, c_i, c_i, c_i, c_i, c_f, c_f, c_i, c_i, c_p, c_sz]
+        L.astraea_schedule_launch.argtypes = [c_p, c_p]
+        L.astraea_schedule_destroy.argtypes = [c_p]
+        L.astraea_schedule_destroy.restype = None
         L.astraea_session_create.argtypes = [ctypes.POINTER(c_p), c_i, c_i, c_i, c_i, c_i]
         L.astraea_session_destroy.argtypes = [c_p]
         L.astraea_session_destroy.restype = None
@@ -72,7 +78,8 @@ def lib() -> ctypes.CDLL:
         L.astraea_last_error.restype = ctypes.c_char_p
         L.astraea_version.restype = ctypes.c_char_p
         for name in ("astraea_score", "astraea_select", "astraea_sparse_attn", "astraea_sparse_attn_noalloc", "astraea_scatter_reuse",
-                     "astraea_step", "astraea_gathered_linear", "astraea_session_create", "astraea_step_host", "astraea_budget_to_k",
+                     "astraea_step", "astraea_gathered_linear", "astraea_schedule_create", "astraea_schedule_launch",
+                     "astraea_session_create", "astraea_step_host", "astraea_budget_to_k",
                      "astraea_poll_error"):
             getattr(L, name).restype = ctypes.c_int32
         _lib = L
@@ -170,6 +177,40 @@ def astraea_step(x_cur, x_ref, lse_cache, n_skip, q, k, v, out_cache, score, idx
 
 def astraea_poll_error(workspace, stream=None) -> None:
     _check(lib().astraea_poll_error(_ptr(workspace), _stream(stream)))
+
+
+class Schedule:
+    """T steps of one attention block as one CUDA graph (astraea_schedule_create / _launch / _destroy).
+    x_cur, q, k, v are lists of T device tensors; the state tensors are those of astraea_step."""
+
+    def __init__(self, k_keep, x_cur, q, k, v, x_ref, lse_cache, n_skip, out_cache, score, idx_sel, idx_rem,
+                 B, H, N, N_sel, d, w_alpha=1.0, w_beta=1.0, delta_mode=DELTA_MEAN_ABS, lse_mode=LSE_SUM_EXP,
+                 workspace=None):
+        T = len(k_keep)
+        assert len(x_cur) == len(q) == len(k) == len(v) == T
+        # the graph keeps pointers: hold on to the tensors for as long as the schedule lives
+        self._keep = (list(x_cur), list(q), list(k), list(v), x_ref, lse_cache, n_skip, out_cache, score, idx_sel, idx_rem, workspace)
+        kk = (ctypes.c_int32 * T)(*[int(a) for a in k_keep])
+        arrs = [(ctypes.c_void_p * T)(*[t.data_ptr() for t in lst]) for lst in (x_cur, q, k, v)]
+        self._h = ctypes.c_void_p()
+        _check(lib().astraea_schedule_create(ctypes.byref(self._h), T, kk, *arrs, _ptr(x_ref), _ptr(lse_cache), _ptr(n_skip),
+                                             _ptr(out_cache), _ptr(score), _ptr(idx_sel), _ptr(idx_rem), B, H, N, N_sel, d,
+                                             w_alpha, w_beta, delta_mode, lse_mode, _ptr(workspace),
+                                             workspace.numel() if workspace is not None else 0))
+
+    def launch(self, stream=None) -> None:
+        _check(lib().astraea_schedule_launch(self._h, _stream(stream)))
+
+    def close(self) -> None:
+        if getattr(self, "_h", None):
+            lib().astraea_schedule_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 class Session:

@@ -252,6 +252,75 @@ int32_t astraea_poll_error(void *workspace, void *stream)
     return ASTRAEA_OK;
 }
 
+// ------------------------------------------------------------------ a schedule of steps as one CUDA graph
+struct astraea_schedule {
+    cudaGraph_t graph;
+    cudaGraphExec_t exec;
+    int T;
+};
+
+void astraea_schedule_destroy(astraea_schedule *s)
+{
+    if (!s) return;
+    if (s->exec) cudaGraphExecDestroy(s->exec);
+    if (s->graph) cudaGraphDestroy(s->graph);
+    delete s;
+}
+
+int32_t astraea_schedule_create(astraea_schedule **schedule, int T, const int32_t *k_keep,
+                                const void *const *x_cur, const void *const *q, const void *const *k,
+                                const void *const *v, void *x_ref, float *lse_cache, int32_t *n_skip,
+                                void *out_cache, float *score, int32_t *idx_sel, int32_t *idx_rem,
+                                int B, int H, int N, int N_sel, int d,
+                                float w_alpha, float w_beta, int delta_mode, int lse_mode,
+                                void *workspace, size_t workspace_bytes)
+{
+    REQUIRE(schedule, "astraea_schedule_create: null schedule pointer");
+    *schedule = nullptr;
+    REQUIRE(T > 0 && k_keep && x_cur && q && k && v, "astraea_schedule_create: T must be positive and the per-step arrays non-null");
+    REQUIRE(N_sel >= 0 && N_sel <= N, "astraea_schedule_create: N_sel=%d outside [0, N=%d]", N_sel, N);
+    for (int t = 0; t < T; ++t) {
+        REQUIRE(k_keep[t] >= 0 && k_keep[t] <= N_sel, "astraea_schedule_create: k_keep[%d]=%d outside [0, N_sel=%d]", t, k_keep[t], N_sel);
+        REQUIRE(x_cur[t] && q[t] && k[t] && v[t], "astraea_schedule_create: null input pointer at step %d", t);
+    }
+    if (!workspace || workspace_bytes < astraea_workspace_bytes(ASTRAEA_OP_STEP, B, H, N, N, d))
+        return fail(ASTRAEA_ERR_WORKSPACE_TOO_SMALL, "astraea_schedule_create: workspace of %zu bytes, need %zu",
+                    workspace_bytes, astraea_workspace_bytes(ASTRAEA_OP_STEP, B, H, N, N, d));
+    astraea_schedule *s = new (std::nothrow) astraea_schedule();
+    if (!s) return fail(ASTRAEA_ERR_CUDA, "astraea_schedule_create: out of host memory");
+    s->graph = nullptr; s->exec = nullptr; s->T = T;
+    cudaStream_t cap = nullptr;
+    cudaError_t e = cudaStreamCreateWithFlags(&cap, cudaStreamNonBlocking);
+    if (e != cudaSuccess) { delete s; return fail(ASTRAEA_ERR_CUDA, "astraea_schedule_create: %s", cudaGetErrorString(e)); }
+    // a thread-local capture: other threads of the process may keep using CUDA meanwhile
+    e = cudaStreamBeginCapture(cap, cudaStreamCaptureModeThreadLocal);
+    int32_t rc = ASTRAEA_OK;
+    if (e == cudaSuccess) {
+        for (int t = 0; t < T && rc == ASTRAEA_OK; ++t)
+            rc = astraea_step(x_cur[t], x_ref, lse_cache, n_skip, q[t], k[t], v[t], out_cache, score, idx_sel, idx_rem,
+                              B, H, N, N_sel, d, k_keep[t], w_alpha, w_beta, delta_mode, lse_mode,
+                              workspace, workspace_bytes, cap);
+        e = cudaStreamEndCapture(cap, &s->graph);          // also ends a capture that a failed step left open
+    }
+    if (e == cudaSuccess && rc == ASTRAEA_OK) e = cudaGraphInstantiate(&s->exec, s->graph, 0);
+    cudaStreamDestroy(cap);
+    if (rc != ASTRAEA_OK) { astraea_schedule_destroy(s); return rc; }
+    if (e != cudaSuccess) {
+        astraea_schedule_destroy(s);
+        return fail(ASTRAEA_ERR_CUDA, "astraea_schedule_create (graph capture): %s", cudaGetErrorString(e));
+    }
+    *schedule = s;
+    return ASTRAEA_OK;
+}
+
+int32_t astraea_schedule_launch(astraea_schedule *s, void *stream)
+{
+    REQUIRE(s && s->exec, "astraea_schedule_launch: null schedule");
+    cudaError_t e = cudaGraphLaunch(s->exec, (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_schedule_launch: %s", cudaGetErrorString(e));
+    return ASTRAEA_OK;
+}
+
 // ------------------------------------------------------------------ host-buffer session
 // astraea_step_host moves q, k, v in and the output back in groups of heads, so that the copies of one group run
 // under the attention of another.

@@ -186,8 +186,8 @@ template <int DH> struct SoftmaxState {
     float shift;                    // the exponentials are taken against m_ref * sl2 + shift (log2 domain)
     uint32_t t_s0, t_o, bar_s, bar_p, bar_done;
     int N, n_tiles;
-    float *ref_x;                   // split: the reference of this thread's row, shared by the tile's two warpgroups
-    int ref_bar;                    // split: named barrier on which the reference is handed over
+    float *ref_x;                   // the reference of this thread's row, shared by the tile's two warpgroups
+    int ref_bar;                    // named barrier on which the reference is handed over
     volatile int *redo_flag;
     volatile int *abort_flag;
     int *err_word;

@@ -517,3 +517,49 @@ def test_gathered_linear_bad_index_and_no_rows():
         A.astraea_poll_error(ws)
     assert e.value.code == A.ERR_BAD_INDEX
     assert float(y[0, 1, 0]) == 64.0 and float(y[0, 2:].abs().sum()) == 0.0
+
+
+# ------------------------------------------------------------- a schedule of steps as one CUDA graph
+def test_schedule_graph_equals_step_by_step():
+    """Four steps with budgets (all, 40 %, none, 25 %) recorded as one graph against the same four astraea_step calls
+    (each of which the step tests check against the oracle): every piece of state ends bit-identical."""
+    w = synth.Workload("mini-schedule", B=2, H=4, d=64, N_v=600, N_t=0)
+    inp = synth.make_step_inputs(w, 17)
+    B, N, H, d, N_sel = w.B, w.N, w.H, w.d, w.N_v
+    budgets = [N_sel, w.k_of(400), 0, w.k_of(250)]
+    xs, qs, ks, vs = [inp["x_cur"]], [inp["q"]], [inp["k"]], [inp["v"]]
+    for t in range(1, len(budgets)):
+        xs.append(synth.drift_step(xs[-1], 500 + t, 0.05, False))
+        qs.append(synth.drift_step(qs[-1], 510 + t, 0.05, True))
+        ks.append(synth.drift_step(ks[-1], 520 + t, 0.05, True))
+        vs.append(synth.drift_step(vs[-1], 530 + t, 0.05, True))
+    dx, dq, dk, dv = ([to_dev_bf16(a) for a in lst] for lst in (xs, qs, ks, vs))
+
+    def fresh_state():
+        return dict(x_ref=to_dev_bf16(inp["x_cur"]), lse=torch.zeros(B, H, N, device="cuda"),
+                    n_skip=torch.zeros(B, N_sel, dtype=torch.int32, device="cuda"),
+                    out=torch.zeros(B, N, H, d, dtype=torch.bfloat16, device="cuda"),
+                    score=torch.empty(B, N_sel, device="cuda"),
+                    idx_sel=torch.zeros(B, N, dtype=torch.int32, device="cuda"),
+                    idx_rem=torch.zeros(B, N_sel, dtype=torch.int32, device="cuda"),
+                    ws=A.new_workspace(A.OP_STEP, B, H, N, N, d))
+
+    a, b = fresh_state(), fresh_state()
+    for t, kk in enumerate(budgets):
+        A.astraea_step(dx[t], a["x_ref"], a["lse"], a["n_skip"], dq[t], dk[t], dv[t], a["out"], a["score"], a["idx_sel"],
+                       a["idx_rem"], B, H, N, N_sel, d, kk, workspace=a["ws"])
+    A.astraea_poll_error(a["ws"])
+    sched = A.Schedule(budgets, dx, dq, dk, dv, b["x_ref"], b["lse"], b["n_skip"], b["out"], b["score"], b["idx_sel"],
+                       b["idx_rem"], B, H, N, N_sel, d, workspace=b["ws"])
+    sched.launch()
+    A.astraea_poll_error(b["ws"])
+    for name in ("x_ref", "lse", "n_skip", "out", "score"):
+        ta, tb = a[name], b[name]
+        assert torch.equal(ta.view(torch.int16) if ta.dtype == torch.bfloat16 else ta,
+                           tb.view(torch.int16) if tb.dtype == torch.bfloat16 else tb), name
+    assert int((b["n_skip"] > 0).sum()) > 0 and float(b["out"].float().abs().sum()) > 0
+    sched.close()
+    with pytest.raises(A.AstraeaError) as e:
+        A.Schedule([N_sel + 1], dx[:1], dq[:1], dk[:1], dv[:1], b["x_ref"], b["lse"], b["n_skip"], b["out"], b["score"],
+                   b["idx_sel"], b["idx_rem"], B, H, N, N_sel, d, workspace=b["ws"])
+    assert e.value.code == A.ERR_INVALID_ARG
