@@ -232,22 +232,26 @@ void oracle_scatter_lse(double *lse_cache, const double *lse_rows, const int32_t
  * applies to the other layers of the block"): y[b, i, :] = x[b, i, :] W^T + bias for the listed
  * rows i = idx[b, r]; every other row of y keeps what it held (the cached result).  W is
  * [N_out, K] (out features x in features).  idx == NULL: all N rows.  Plain triple loop.
+ * compact_in: x is [B, M, K] and its row r belongs to token idx[b, r] (the output of an earlier layer
+ * that was computed on the selected rows only).  gelu: y = GELU(x W^T + bias) with the exact (erf)
+ * definition GELU(u) = u/2 (1 + erf(u / sqrt 2)), the activation between the two MLP layers.
  */
 void oracle_gathered_linear(const double *x, const int32_t *idx, int M, const double *w,
-                            const double *bias, double *y, int B, int N, int K, int N_out)
+                            const double *bias, double *y, int B, int N, int K, int N_out,
+                            int compact_in, int gelu)
 {
     const int rows = idx ? M : N;
 #pragma omp parallel for collapse(2) schedule(static)
     for (int b = 0; b < B; ++b)
         for (int r = 0; r < rows; ++r) {
             const int i = idx ? idx[(size_t)b * M + r] : r;
-            const double *xr = x + ((size_t)b * N + i) * K;
+            const double *xr = compact_in ? x + ((size_t)b * M + r) * K : x + ((size_t)b * N + i) * K;
             double *yr = y + ((size_t)b * N + i) * N_out;
             for (int n = 0; n < N_out; ++n) {
                 double acc = bias ? bias[n] : 0.0;
                 const double *wr = w + (size_t)n * K;
                 for (int c = 0; c < K; ++c) acc += xr[c] * wr[c];
-                yr[n] = acc;
+                yr[n] = gelu ? 0.5 * acc * (1.0 + erf(acc * 0.70710678118654752440)) : acc;
             }
         }
 }

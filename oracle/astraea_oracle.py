@@ -128,11 +128,17 @@ def scatter_reuse(cache, rows, idx):
     return out
 
 
-def gathered_linear(x, w, bias=None, idx=None, y_cache=None):
+def gathered_linear(x, w, bias=None, idx=None, y_cache=None, compact_in=False, gelu=False, N=None):
     """y = copy of y_cache [B, N, N_out] (zeros if None) with rows idx[b, r] (all rows if idx is None)
-    replaced by x[b, i, :] @ w.T + bias; w is [N_out, K]."""
+    replaced by act(x[b, i, :] @ w.T + bias); w is [N_out, K].  compact_in: x is [B, M, K], row r belongs to
+    token idx[b, r] (pass N, the number of tokens, or y_cache).  gelu: act = exact GELU, else identity."""
     x, w = _f64(x), _f64(w)
-    B, N, K = x.shape
+    B, rows_x, K = x.shape
+    if compact_in:
+        assert idx is not None and (y_cache is not None or N is not None)
+        N = N if y_cache is None else np.asarray(y_cache).shape[1]
+    else:
+        N = rows_x
     N_out = w.shape[0]
     assert w.shape == (N_out, K)
     y = np.zeros((B, N, N_out)) if y_cache is None else np.array(y_cache, dtype=np.float64, copy=True, order="C")
@@ -144,7 +150,8 @@ def gathered_linear(x, w, bias=None, idx=None, y_cache=None):
         M = idx.shape[1]
         if M == 0:
             return y
-    _load().oracle_gathered_linear(_p(x), _p(idx), M, _p(w), _p(bias), _p(y), B, N, K, N_out)
+    assert not compact_in or x.shape[1] == M
+    _load().oracle_gathered_linear(_p(x), _p(idx), M, _p(w), _p(bias), _p(y), B, N, K, N_out, int(compact_in), int(gelu))
     return y
 
 

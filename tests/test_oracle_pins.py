@@ -346,6 +346,32 @@ def test_gathered_linear_closed_forms_catch_a_transposed_weight_or_a_dropped_bia
             assert abs(got[0, i, n] - want) < 1e-13
 
 
+def test_gathered_linear_gelu_and_compact_input_match_library_routines(oracle):
+    """The MLP of a block on the selected rows: GELU(x[idx] W1^T + b1) kept compact, then W2 applied to the compact
+    rows and scattered to the tokens.  Checked against torch's fp64 gelu / linear and plain indexing."""
+    rng = np.random.default_rng(23)
+    B, N, K, Hd, M = 2, 19, 6, 10, 7
+    x, w1, b1, w2, b2, cache = (_rand(rng, B, N, K), _rand(rng, Hd, K), _rand(rng, Hd), _rand(rng, K, Hd), _rand(rng, K),
+                                _rand(rng, B, N, K))
+    idx = np.stack([np.sort(rng.choice(N, M, replace=False)) for _ in range(B)]).astype(np.int32)
+    hid_full = oracle.gathered_linear(x, w1, b1, idx, gelu=True)                    # [B, N, Hd], rows off the list are zero
+    hid = np.take_along_axis(hid_full, idx[:, :, None].astype(np.int64), 1)         # compact [B, M, Hd]
+    t = torch.from_numpy
+    want_hid = torch.nn.functional.gelu(torch.nn.functional.linear(t(x), t(w1), t(b1))).numpy()
+    assert np.abs(hid - np.take_along_axis(want_hid, idx[:, :, None].astype(np.int64), 1)).max() < 1e-12
+    assert np.abs(oracle.gathered_linear(np.array([[[0.0], [1.0], [-1.0]]]), np.ones((1, 1)), gelu=True).ravel()
+                  - np.array([0.0, 0.8413447460685429, -0.15865525393145707])).max() < 1e-15     # x Phi(x) at 0, 1, -1
+    y = oracle.gathered_linear(hid, w2, b2, idx, cache, compact_in=True)
+    want = np.array(cache)
+    for b in range(B):
+        want[b, idx[b]] = hid[b] @ w2.T + b2
+    assert np.abs(y - want).max() < 1e-12
+    mask = np.ones((B, N), bool)
+    for b in range(B):
+        mask[b, idx[b]] = False
+    assert np.array_equal(y[mask], cache[mask])
+
+
 def test_attention_flops_are_linear_in_selected_tokens_like_the_papers_tables():
     from paper_2506_05096_b200 import accounting
     path = os.path.join(os.path.dirname(__file__), "golden", "flops_tables.txt")
