@@ -54,6 +54,8 @@ extern "C" {
 #define ASTRAEA_ATTN_COMPACT_OUT  1u         /* out is [B,M,H,d] and lse_out [B,H,M] (row r of the index list), not the caches */
 /* flags of astraea_gathered_linear */
 #define ASTRAEA_LINEAR_COMPACT_OUT 1u        /* y is [B,M,N_out] (row r of the index list), not the cache [B,N,N_out] */
+#define ASTRAEA_LINEAR_COMPACT_IN  2u        /* x is [B,M,K]: row r is the row of token idx[b,r] (output of a layer run with COMPACT_OUT) */
+#define ASTRAEA_LINEAR_GELU        4u        /* y = GELU(x W^T + bias), GELU(u) = u/2 (1 + erf(u / sqrt 2)): the first MLP layer */
 /* flags of astraea_scatter_reuse */
 #define ASTRAEA_SCATTER_SRC_FULL  1u         /* rows is [B,N,row_elems]; row idx[r] of it is copied to row idx[r] of cache */
 
@@ -186,12 +188,15 @@ int32_t astraea_scatter_reuse(void *cache, const void *rows, const int32_t *idx,
  *     y[b, idx[b,r], :] = x[b, idx[b,r], :] W^T + bias        for r in [0, M)
  * and every row of y that is not listed is left untouched, i.e. keeps the cached result of the earlier
  * step.  The gather of the rows of x and the scatter of the rows of y are fused into the GEMM.
- *   x    : bf16 [B, N, K]            idx : int32 [B, M] in [0,N), no duplicates; NULL => all N rows (M ignored)
+ *   x    : bf16 [B, N, K] (with ASTRAEA_LINEAR_COMPACT_IN bf16 [B, M, K])
+ *   idx  : int32 [B, M] in [0,N), no duplicates; NULL => all N rows (M ignored)
  *   w    : bf16 [N_out, K] row-major (out features x in features)        bias : bf16 [N_out] or NULL
  *   y    : bf16 [B, N, N_out], rows at idx written in place; with ASTRAEA_LINEAR_COMPACT_OUT bf16 [B, M, N_out]
  *   workspace : at least astraea_workspace_bytes(ASTRAEA_OP_GATHERED_LINEAR, 0, 0, 0, 0, 0) bytes, 256-byte
  *               aligned, zero before the first use (holds the error word read by astraea_poll_error).
- * bf16 operands, fp32 accumulation, one rounding to bf16 at the end.  K must be a multiple of 64, N_out
+ * With ASTRAEA_LINEAR_COMPACT_OUT on the first and ASTRAEA_LINEAR_COMPACT_IN on the second layer the hidden
+ * activations of the MLP exist for the selected rows only.
+ * bf16 operands, fp32 accumulation (and fp32 GELU), one rounding to bf16 at the end.  K must be a multiple of 64, N_out
  * a multiple of 8; x, w, y 16-byte aligned.  M = 0 is valid (nothing is launched).  An index outside
  * [0,N) is not dereferenced: its row is skipped and astraea_poll_error reports BAD_INDEX.
  * Errors: INVALID_ARG, UNSUPPORTED (unknown flags), WORKSPACE_TOO_SMALL, CUDA.

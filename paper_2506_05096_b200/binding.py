@@ -21,7 +21,7 @@ DELTA_MEAN_ABS, DELTA_MEAN_SQ, DELTA_MEAN_SIGNED = 0, 1, 2
 LSE_SUM_EXP, LSE_LOG = 0, 1
 ATTN_COMPACT_OUT = 1
 SCATTER_SRC_FULL = 1
-LINEAR_COMPACT_OUT = 1
+LINEAR_COMPACT_OUT, LINEAR_COMPACT_IN, LINEAR_GELU = 1, 2, 4
 OP_SELECT, OP_SPARSE_ATTN, OP_STEP, OP_SPARSE_ATTN_KV, OP_GATHERED_LINEAR = 1, 2, 3, 4, 5
 N_SKIP_CLAMP = 80
 NOALLOC_SCRATCH_BYTES = 4096

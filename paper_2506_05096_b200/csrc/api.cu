@@ -194,8 +194,9 @@ int32_t astraea_gathered_linear(const void *x, const int32_t *idx, int M, const 
     REQUIRE(!idx || (M >= 0 && M <= N), "astraea_gathered_linear: M=%d outside [0, N=%d]", M, N);
     REQUIRE(K % 64 == 0, "astraea_gathered_linear: K=%d must be a multiple of 64", K);
     REQUIRE(N_out % 8 == 0, "astraea_gathered_linear: N_out=%d must be a multiple of 8", N_out);
-    if (flags & ~ASTRAEA_LINEAR_COMPACT_OUT) return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_gathered_linear: unknown flags 0x%x", flags);
-    REQUIRE(!(flags & ASTRAEA_LINEAR_COMPACT_OUT) || idx, "astraea_gathered_linear: a compact output needs an index list");
+    if (flags & ~(ASTRAEA_LINEAR_COMPACT_OUT | ASTRAEA_LINEAR_COMPACT_IN | ASTRAEA_LINEAR_GELU))
+        return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_gathered_linear: unknown flags 0x%x", flags);
+    REQUIRE(!(flags & (ASTRAEA_LINEAR_COMPACT_OUT | ASTRAEA_LINEAR_COMPACT_IN)) || idx, "astraea_gathered_linear: compact rows need an index list");
     if (!workspace || workspace_bytes < linear_workspace_bytes())
         return fail(ASTRAEA_ERR_WORKSPACE_TOO_SMALL, "astraea_gathered_linear: workspace of %zu bytes, need %zu",
                     workspace_bytes, linear_workspace_bytes());

@@ -42,7 +42,9 @@ struct LinParams {
     const __nv_bfloat16 *bias;
     __nv_bfloat16 *y;
     int B, N, K, N_out;
-    int compact;
+    int compact;                 // y is [B, M, N_out]
+    int compact_in;              // x is [B, M, K]
+    int gelu;                    // y = GELU(x W^T + bias), exact (erf) form
     int *err_word;
 };
 
@@ -62,14 +64,15 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *m, 
         ::"r"(dst), "l"(m), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
 
-// token row of the g-th listed row (all batch elements in one list), or -1
+// row of x that holds the g-th listed row (all batch elements in one list): -1 past the end, -2 for an index
+// outside [0, N); *out_row is the row of y it goes to
 __device__ __forceinline__ long long source_row(const LinParams &p, long long g, long long total, long long *out_row) {
     if (g >= total) return -1;
     const int b = (int)(g / p.M), r = (int)(g - (long long)b * p.M);
     const int tok = p.idx ? __ldg(p.idx + g) : r;
     if ((unsigned)tok >= (unsigned)p.N) return -2;
     if (out_row) *out_row = p.compact ? g : (long long)b * p.N + tok;
-    return (long long)b * p.N + tok;
+    return p.compact_in ? g : (long long)b * p.N + tok;
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -149,6 +152,10 @@ gathered_linear_kernel(const __grid_constant__ CUtensorMap tmap_w, const LinPara
                             f[2 * i] += __uint_as_float(bw[i] << 16);
                             f[2 * i + 1] += __uint_as_float(bw[i] & 0xffff0000u);
                         }
+                    }
+                    if (p.gelu) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) f[i] = 0.5f * f[i] * (1.0f + erff(f[i] * 0.70710678118654752f));
                     }
                     uint32_t w[4];
 #pragma unroll
@@ -280,6 +287,8 @@ int32_t launch_gathered_linear(const void *x, const int32_t *idx, int M, const v
     p.y = reinterpret_cast<__nv_bfloat16 *>(y);
     p.B = B; p.N = N; p.K = K; p.N_out = N_out;
     p.compact = (flags & ASTRAEA_LINEAR_COMPACT_OUT) ? 1 : 0;
+    p.compact_in = (flags & ASTRAEA_LINEAR_COMPACT_IN) ? 1 : 0;
+    p.gelu = (flags & ASTRAEA_LINEAR_GELU) ? 1 : 0;
     p.err_word = err_word;
     const long long rows = (long long)B * p.M;
     const long long tiles = ((rows + kBM - 1) / kBM) * ((N_out + kBN - 1) / kBN);

@@ -563,3 +563,40 @@ def test_schedule_graph_equals_step_by_step():
         A.Schedule([N_sel + 1], dx[:1], dq[:1], dk[:1], dv[:1], b["x_ref"], b["lse"], b["n_skip"], b["out"], b["score"],
                    b["idx_sel"], b["idx_rem"], B, H, N, N_sel, d, workspace=b["ws"])
     assert e.value.code == A.ERR_INVALID_ARG
+
+
+def test_gathered_linear_mlp_on_selected_rows_hidden_state_stays_compact(oracle):
+    """The MLP of a block: GELU(x[idx] W1^T + b1) into a compact [B, M, 4K] buffer, then W2 on the compact rows with
+    the result scattered over the cached output.  Both layers against the oracle (the second one fed with the
+    device's bf16 hidden state, so that each layer is checked on its own)."""
+    rng = np.random.default_rng(41)
+    B, N, K, M = 2, 300, 128, 170
+    Hd = 4 * K
+    x = synth.f32_to_bf16_bits(rng.standard_normal((B, N, K)).astype(np.float32))
+    w1 = synth.f32_to_bf16_bits((rng.standard_normal((Hd, K)) / math.sqrt(K)).astype(np.float32))
+    b1 = synth.f32_to_bf16_bits(rng.standard_normal(Hd).astype(np.float32))
+    w2 = synth.f32_to_bf16_bits((rng.standard_normal((K, Hd)) / math.sqrt(Hd)).astype(np.float32))
+    b2 = synth.f32_to_bf16_bits(rng.standard_normal(K).astype(np.float32))
+    cache = synth.f32_to_bf16_bits(rng.standard_normal((B, N, K)).astype(np.float32))
+    idx = np.stack([np.sort(rng.choice(N, M, replace=False)) for _ in range(B)]).astype(np.int32)
+    ws = A.new_workspace(A.OP_GATHERED_LINEAR, 0, 0, 0, 0, 0)
+    hid = torch.zeros(B, M, Hd, dtype=torch.bfloat16, device="cuda")
+    A.astraea_gathered_linear(to_dev_bf16(x), dev(idx), M, to_dev_bf16(w1), to_dev_bf16(b1), hid, B, N, K, Hd,
+                              flags=A.LINEAR_COMPACT_OUT | A.LINEAR_GELU, workspace=ws)
+    want_hid = np.take_along_axis(oracle.gathered_linear(f64(x), f64(w1), f64(b1), idx, gelu=True),
+                                  idx[:, :, None].astype(np.int64), 1)
+    got_hid = bf16_dev_to_f64(hid)
+    err = np.abs(got_hid - want_hid)
+    assert err.max() < LINEAR_MAX_ABS and err.mean() < LINEAR_MEAN_ABS, (err.max(), err.mean())
+    y = to_dev_bf16(cache)
+    A.astraea_gathered_linear(hid, dev(idx), M, to_dev_bf16(w2), to_dev_bf16(b2), y, B, N, Hd, K,
+                              flags=A.LINEAR_COMPACT_IN, workspace=ws)
+    A.astraea_poll_error(ws)
+    want = oracle.gathered_linear(got_hid, f64(w2), f64(b2), idx, f64(cache), compact_in=True)
+    got = bf16_dev_to_f64(y)
+    err = np.abs(got - want)
+    assert err.max() < LINEAR_MAX_ABS and err.mean() < LINEAR_MEAN_ABS, (err.max(), err.mean())
+    mask = np.ones((B, N), bool)
+    for b in range(B):
+        mask[b, idx[b]] = False
+    assert np.array_equal(got[mask], f64(cache)[mask])
