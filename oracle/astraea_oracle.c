@@ -159,9 +159,11 @@ void oracle_sparse_attn(const double *q, const double *k, const double *v,
                         const int32_t *q_idx, int M,
                         const int32_t *kv_idx, int M_kv,
                         double *o, double *lse, double *p_out,
-                        int B, int H, int N, int d, double scale)
+                        int B, int H, int N, int N_kv, int d, double scale)
 {
-    const int Nk = kv_idx ? M_kv : N;
+    /* N: tokens of q; N_kv: tokens of k and v (self-attention: N_kv == N; cross-attention of the
+     * selected rows against another sequence, e.g. the text tokens: N_kv != N) */
+    const int Nk = kv_idx ? M_kv : N_kv;
     if (scale == 0.0) scale = 1.0 / sqrt((double)d);
 #pragma omp parallel
     {
@@ -175,7 +177,7 @@ void oracle_sparse_attn(const double *q, const double *k, const double *v,
                 double m = -INFINITY;
                 for (int jj = 0; jj < Nk; ++jj) {
                     int j = kv_idx ? kv_idx[(size_t)b * M_kv + jj] : jj;
-                    const double *kj = k + (((size_t)b * N + j) * H + h) * d;
+                    const double *kj = k + (((size_t)b * N_kv + j) * H + h) * d;
                     double dot = 0.0;
                     for (int c = 0; c < d; ++c) dot += qi[c] * kj[c];
                     s[jj] = dot * scale;
@@ -187,7 +189,7 @@ void oracle_sparse_attn(const double *q, const double *k, const double *v,
                 for (int c = 0; c < d; ++c) oi[c] = 0.0;
                 for (int jj = 0; jj < Nk; ++jj) {
                     int j = kv_idx ? kv_idx[(size_t)b * M_kv + jj] : jj;
-                    const double *vj = v + (((size_t)b * N + j) * H + h) * d;
+                    const double *vj = v + (((size_t)b * N_kv + j) * H + h) * d;
                     double p = s[jj] / Z;
                     if (p_out) p_out[(((size_t)b * H + h) * M + r) * Nk + jj] = p;
                     for (int c = 0; c < d; ++c) oi[c] += p * vj[c];

@@ -97,21 +97,23 @@ def select(score_f32, k, n_always=0, n_skip=None):
 def sparse_attn(q, k, v, q_idx=None, kv_idx=None, scale=0.0, want_probs=False):
     """Attention rows for the listed queries against all keys (or kv_idx).
 
-    q, k, v: [B, N, H, d].  Returns (o [B, M, H, d], lse [B, H, M], probs or None).
+    q: [B, N, H, d]; k, v: [B, N_kv, H, d] (N_kv = N for self-attention; another length for the cross-attention
+    of the listed rows against a second sequence).  Returns (o [B, M, H, d], lse [B, H, M], probs or None).
     """
     q, k, v = _f64(q), _f64(k), _f64(v)
-    B, N, H, d = k.shape
-    assert q.shape == k.shape == v.shape
+    B, N, H, d = q.shape
+    N_kv = k.shape[1]
+    assert k.shape == v.shape == (B, N_kv, H, d)
     q_idx = _i32(q_idx)
     kv_idx = _i32(kv_idx)
     M = N if q_idx is None else q_idx.shape[1]
     M_kv = 0 if kv_idx is None else kv_idx.shape[1]
-    Nk = N if kv_idx is None else M_kv
+    Nk = N_kv if kv_idx is None else M_kv
     o = np.empty((B, M, H, d), dtype=np.float64)
     lse = np.empty((B, H, M), dtype=np.float64)
     probs = np.empty((B, H, M, Nk), dtype=np.float64) if want_probs else None
     _load().oracle_sparse_attn(_p(q), _p(k), _p(v), _p(q_idx), M, _p(kv_idx), M_kv,
-                               _p(o), _p(lse), _p(probs), B, H, N, d, ctypes.c_double(scale))
+                               _p(o), _p(lse), _p(probs), B, H, N, N_kv, d, ctypes.c_double(scale))
     return o, lse, probs
 
 

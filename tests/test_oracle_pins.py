@@ -307,6 +307,24 @@ def test_drift_statistics_half_normal_mean(oracle):
 
 
 # -------------------------------------------------------- flop accounting pin
+def test_cross_attention_of_listed_rows_matches_a_library_softmax(oracle):
+    """Queries from one sequence, keys / values from another (the block's cross-attention on the selected rows):
+    numpy softmax over the second sequence, rows picked by the list."""
+    rng = np.random.default_rng(24)
+    B, N, N_kv, H, d, M = 2, 23, 9, 2, 8, 6
+    q, k, v = _rand(rng, B, N, H, d), _rand(rng, B, N_kv, H, d), _rand(rng, B, N_kv, H, d)
+    idx = np.stack([np.sort(rng.choice(N, M, replace=False)) for _ in range(B)]).astype(np.int32)
+    o, lse, p = oracle.sparse_attn(q, k, v, q_idx=idx, want_probs=True)
+    s = np.einsum("bihc,bjhc->bhij", q, k) / math.sqrt(d)
+    pr = np.exp(s - s.max(-1, keepdims=True))
+    pr /= pr.sum(-1, keepdims=True)
+    ref = np.einsum("bhij,bjhc->bihc", pr, v)
+    for b in range(B):
+        assert np.abs(o[b] - ref[b, idx[b]]).max() < 1e-12
+        assert np.abs(lse[b] - np.log(np.exp(s[b]).sum(-1))[:, idx[b]]).max() < 1e-12
+    assert p.shape == (B, H, M, N_kv) and np.abs(p.sum(-1) - 1).max() < 1e-12
+
+
 # ---------------------------------------------------------------- linear layers on selected rows
 def test_gathered_linear_matches_a_library_matmul_and_leaves_other_rows_alone(oracle):
     """All rows: the textbook x W^T + b (numpy matmul).  Listed rows only: those rows equal the full product,
