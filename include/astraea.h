@@ -139,6 +139,22 @@ int32_t astraea_sparse_attn(const void *q, const void *k, const void *v,
                             void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Cross-attention of the selected rows (Section 3.2: the layers of a block other than self-attention are
+ * computed for the selected tokens only and their cached results reused for the rest): as
+ * astraea_sparse_attn, but keys and values come from another sequence of N_kv tokens (the text tokens),
+ *     out[b, i, h, :] = Softmax(q[b, i, h, :] K[b, :, h, :]^T * scale) V[b, :, h, :]   for i in q_idx,
+ * k, v : bf16 [B, N_kv, H, d] through their stride triples; q, out, lse_out, q_idx, M, flags, workspace as above
+ * (N is the token count of q and out).  There is no kv_idx form.  Errors as astraea_sparse_attn.
+ */
+int32_t astraea_sparse_cross_attn(const void *q, const void *k, const void *v,
+                                  int64_t q_sb, int64_t q_sh, int64_t q_sn,
+                                  int64_t k_sb, int64_t k_sh, int64_t k_sn,
+                                  int64_t v_sb, int64_t v_sh, int64_t v_sn,
+                                  const int32_t *q_idx, int M, void *out, float *lse_out,
+                                  int B, int H, int N, int N_kv, int d, float scale, uint32_t flags,
+                                  void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * The same attention for callers that must not allocate.  (The paper has no counterpart: this is a
  * property of the library, not of the method.)  astraea_sparse_attn takes its scratch from the
  * caller, which some callers cannot provide: code that runs while a CUDA memory pool or a framework

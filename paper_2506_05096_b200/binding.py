@@ -27,7 +27,7 @@ N_SKIP_CLAMP = 80
 NOALLOC_SCRATCH_BYTES = 4096
 
 EXPORTS = [
-    "astraea_score", "astraea_select", "astraea_sparse_attn", "astraea_sparse_attn_noalloc", "astraea_scatter_reuse", "astraea_step",
+    "astraea_score", "astraea_select", "astraea_sparse_attn", "astraea_sparse_cross_attn", "astraea_sparse_attn_noalloc", "astraea_scatter_reuse", "astraea_step",
     "astraea_gathered_linear", "astraea_schedule_create", "astraea_schedule_launch", "astraea_schedule_destroy",
     "astraea_session_create", "astraea_session_destroy", "astraea_step_host",
     "astraea_workspace_bytes", "astraea_budget_to_k", "astraea_poll_error",
@@ -57,6 +57,8 @@ def lib() -> ctypes.CDLL:
         L.astraea_select.argtypes = [c_p, c_i, c_i, c_i, c_i, c_p, c_p, c_p, c_p, c_sz, c_p]
         L.astraea_sparse_attn.argtypes = [c_p, c_p, c_p] + [c_i64] * 9 + [c_p, c_i, c_p, c_i, c_p, c_p,
                                                                          c_i, c_i, c_i, c_i, c_f, c_u, c_p, c_sz, c_p]
+        L.astraea_sparse_cross_attn.argtypes = [c_p, c_p, c_p] + [c_i64] * 9 + [c_p, c_i, c_p, c_p,
+                                                                               c_i, c_i, c_i, c_i, c_i, c_f, c_u, c_p, c_sz, c_p]
         L.astraea_sparse_attn_noalloc.argtypes = [c_p, c_p, c_p] + [c_i64] * 9 + [c_p, c_i, c_p, c_i, c_p, c_p,
                                                                                  c_i, c_i, c_i, c_i, c_f, c_u, c_p]
         L.astraea_scatter_reuse.argtypes = [c_p, c_p, c_p, c_i, c_i, c_i, c_i, c_u, c_p]
@@ -77,7 +79,7 @@ def lib() -> ctypes.CDLL:
         L.astraea_poll_error.argtypes = [c_p, c_p]
         L.astraea_last_error.restype = ctypes.c_char_p
         L.astraea_version.restype = ctypes.c_char_p
-        for name in ("astraea_score", "astraea_select", "astraea_sparse_attn", "astraea_sparse_attn_noalloc", "astraea_scatter_reuse",
+        for name in ("astraea_score", "astraea_select", "astraea_sparse_attn", "astraea_sparse_cross_attn", "astraea_sparse_attn_noalloc", "astraea_scatter_reuse",
                      "astraea_step", "astraea_gathered_linear", "astraea_schedule_create", "astraea_schedule_launch",
                      "astraea_session_create", "astraea_step_host", "astraea_budget_to_k",
                      "astraea_poll_error"):
@@ -152,6 +154,14 @@ def astraea_sparse_attn_noalloc(q, k, v, q_strides, k_strides, v_strides, q_idx,
     _check(lib().astraea_sparse_attn_noalloc(_ptr(q), _ptr(k), _ptr(v), *q_strides, *k_strides, *v_strides,
                                              _ptr(q_idx), M, _ptr(kv_idx), M_kv, _ptr(out), _ptr(lse_out),
                                              B, H, N, d, scale, flags, _stream(stream)))
+
+
+def astraea_sparse_cross_attn(q, k, v, q_strides, k_strides, v_strides, q_idx, M, out, lse_out, B, H, N, N_kv, d,
+                              scale=0.0, flags=0, workspace=None, stream=None) -> None:
+    """As astraea_sparse_attn with keys / values of another sequence (N_kv tokens)."""
+    _check(lib().astraea_sparse_cross_attn(_ptr(q), _ptr(k), _ptr(v), *q_strides, *k_strides, *v_strides,
+                                           _ptr(q_idx), M, _ptr(out), _ptr(lse_out), B, H, N, N_kv, d, scale, flags,
+                                           _ptr(workspace), workspace.numel() if workspace is not None else 0, _stream(stream)))
 
 
 def astraea_scatter_reuse(cache, rows, idx, B, N, M, row_elems, flags=0, stream=None) -> None:

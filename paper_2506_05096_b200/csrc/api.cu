@@ -91,7 +91,7 @@ int32_t astraea_select(const float *score, int B, int N_sel, int k, int n_always
     return launch_select(score, B, N_sel, k, n_always, idx_sel, idx_rem, n_skip, workspace, (cudaStream_t)stream);
 }
 
-int32_t astraea_sparse_attn(const void *q, const void *k, const void *v,
+static int32_t sparse_attn_entry(const char *fn, int N_kv, const void *q, const void *k, const void *v,
                             int64_t q_sb, int64_t q_sh, int64_t q_sn,
                             int64_t k_sb, int64_t k_sh, int64_t k_sn,
                             int64_t v_sb, int64_t v_sh, int64_t v_sn,
@@ -100,25 +100,25 @@ int32_t astraea_sparse_attn(const void *q, const void *k, const void *v,
                             int B, int H, int N, int d, float scale, uint32_t flags,
                             void *workspace, size_t workspace_bytes, void *stream)
 {
-    REQUIRE(B > 0 && H > 0 && N > 0 && d > 0, "astraea_sparse_attn: B, H, N, d must be positive");
-    REQUIRE(!kv_idx || (M_kv > 0 && M_kv <= N), "astraea_sparse_attn: M_kv=%d outside [1, N=%d]", M_kv, N);
-    REQUIRE(M >= 0 && M <= N, "astraea_sparse_attn: M=%d outside [0, N=%d]", M, N);
+    REQUIRE(B > 0 && H > 0 && N > 0 && d > 0 && N_kv >= 0, "%s: B, H, N, d must be positive", fn);
+    REQUIRE(!kv_idx || (M_kv > 0 && M_kv <= N), "%s: M_kv=%d outside [1, N=%d]", fn, M_kv, N);
+    REQUIRE(M >= 0 && M <= N, "%s: M=%d outside [0, N=%d]", fn, M, N);
     if (d != 64 && d != 72 && d != 128)
-        return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_sparse_attn: head_dim %d not in {64, 72, 128}", d);
-    if (flags & ~ASTRAEA_ATTN_COMPACT_OUT) return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_sparse_attn: unknown flags 0x%x", flags);
-    REQUIRE(q && k && v && out, "astraea_sparse_attn: null q, k, v or out");
-    REQUIRE(aligned16(q) && aligned16(k) && aligned16(v) && aligned16(out), "astraea_sparse_attn: q, k, v, out must be 16-byte aligned");
+        return fail(ASTRAEA_ERR_UNSUPPORTED, "%s: head_dim %d not in {64, 72, 128}", fn, d);
+    if (flags & ~ASTRAEA_ATTN_COMPACT_OUT) return fail(ASTRAEA_ERR_UNSUPPORTED, "%s: unknown flags 0x%x", fn, flags);
+    REQUIRE(q && k && v && out, "%s: null q, k, v or out", fn);
+    REQUIRE(aligned16(q) && aligned16(k) && aligned16(v) && aligned16(out), "%s: q, k, v, out must be 16-byte aligned", fn);
     REQUIRE(q_sn % 8 == 0 && k_sn % 8 == 0 && v_sn % 8 == 0 && q_sh % 8 == 0 && k_sh % 8 == 0 && v_sh % 8 == 0 &&
             q_sb % 8 == 0 && k_sb % 8 == 0 && v_sb % 8 == 0,
-            "astraea_sparse_attn: strides must be multiples of 8 elements (16 bytes)");
+            "%s: strides must be multiples of 8 elements (16 bytes)", fn);
     REQUIRE(q_sn >= d && k_sn >= d && v_sn >= d && q_sh > 0 && k_sh > 0 && v_sh > 0 && q_sb >= 0 && k_sb >= 0 && v_sb >= 0,
-            "astraea_sparse_attn: strides must be positive and token stride >= head_dim");
-    REQUIRE(scale >= 0.f, "astraea_sparse_attn: scale must be >= 0 (0 selects 1/sqrt(d))");
+            "%s: strides must be positive and token stride >= head_dim", fn);
+    REQUIRE(scale >= 0.f, "%s: scale must be >= 0 (0 selects 1/sqrt(d))", fn);
     const size_t ws_need = kv_idx ? attn_kv_workspace_bytes(B, H, M_kv, d) : attn_workspace_bytes(B, H, N, M, d);
     if (!workspace || workspace_bytes < ws_need)
-        return fail(ASTRAEA_ERR_WORKSPACE_TOO_SMALL, "astraea_sparse_attn: workspace of %zu bytes, need %zu",
+        return fail(ASTRAEA_ERR_WORKSPACE_TOO_SMALL, "%s: workspace of %zu bytes, need %zu", fn,
                     workspace_bytes, ws_need);
-    REQUIRE((reinterpret_cast<uintptr_t>(workspace) & 255u) == 0, "astraea_sparse_attn: workspace must be 256-byte aligned");
+    REQUIRE((reinterpret_cast<uintptr_t>(workspace) & 255u) == 0, "%s: workspace must be 256-byte aligned", fn);
     if (M == 0) return ASTRAEA_OK;
     AttnArgs a;
     a.q = q; a.k = k; a.v = v;
@@ -131,8 +131,35 @@ int32_t astraea_sparse_attn(const void *q, const void *k, const void *v,
     a.flags = flags;
     a.err_word = reinterpret_cast<int *>(workspace);
     a.N_tok = N;
+    if (N_kv > 0) a.N = N_kv;          // keys and values of another sequence: N stays the token count of q / out
     if (kv_idx) return launch_sparse_attn_kv(a, kv_idx, M_kv, workspace, (cudaStream_t)stream);
     return launch_sparse_attn(a, (cudaStream_t)stream);
+}
+
+int32_t astraea_sparse_attn(const void *q, const void *k, const void *v,
+                            int64_t q_sb, int64_t q_sh, int64_t q_sn,
+                            int64_t k_sb, int64_t k_sh, int64_t k_sn,
+                            int64_t v_sb, int64_t v_sh, int64_t v_sn,
+                            const int32_t *q_idx, int M, const int32_t *kv_idx, int M_kv,
+                            void *out, float *lse_out,
+                            int B, int H, int N, int d, float scale, uint32_t flags,
+                            void *workspace, size_t workspace_bytes, void *stream)
+{
+    return sparse_attn_entry("astraea_sparse_attn", 0, q, k, v, q_sb, q_sh, q_sn, k_sb, k_sh, k_sn, v_sb, v_sh, v_sn,
+                             q_idx, M, kv_idx, M_kv, out, lse_out, B, H, N, d, scale, flags, workspace, workspace_bytes, stream);
+}
+
+int32_t astraea_sparse_cross_attn(const void *q, const void *k, const void *v,
+                                  int64_t q_sb, int64_t q_sh, int64_t q_sn,
+                                  int64_t k_sb, int64_t k_sh, int64_t k_sn,
+                                  int64_t v_sb, int64_t v_sh, int64_t v_sn,
+                                  const int32_t *q_idx, int M, void *out, float *lse_out,
+                                  int B, int H, int N, int N_kv, int d, float scale, uint32_t flags,
+                                  void *workspace, size_t workspace_bytes, void *stream)
+{
+    REQUIRE(N_kv > 0, "astraea_sparse_cross_attn: N_kv=%d must be positive", N_kv);
+    return sparse_attn_entry("astraea_sparse_cross_attn", N_kv, q, k, v, q_sb, q_sh, q_sn, k_sb, k_sh, k_sn, v_sb, v_sh, v_sn,
+                             q_idx, M, nullptr, 0, out, lse_out, B, H, N, d, scale, flags, workspace, workspace_bytes, stream);
 }
 
 int32_t astraea_sparse_attn_noalloc(const void *q, const void *k, const void *v,

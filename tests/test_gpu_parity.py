@@ -600,3 +600,31 @@ def test_gathered_linear_mlp_on_selected_rows_hidden_state_stays_compact(oracle)
     for b in range(B):
         mask[b, idx[b]] = False
     assert np.array_equal(got[mask], f64(cache)[mask])
+
+
+# ------------------------------------------------------------- cross-attention of the selected rows
+@pytest.mark.parametrize("d,N_kv", [(64, 226), (72, 77), (128, 300), (64, 1)])
+def test_cross_attention_of_selected_rows(oracle, d, N_kv):
+    rng = np.random.default_rng(50 + d)
+    B, H, N, M = 2, 3, 500, 333
+    q, cache = (synth.f32_to_bf16_bits(rng.standard_normal((B, N, H, d)).astype(np.float32)) for _ in range(2))
+    k, v = (synth.f32_to_bf16_bits(rng.standard_normal((B, N_kv, H, d)).astype(np.float32)) for _ in range(2))
+    idx = np.stack([np.sort(rng.choice(N, M, replace=False)) for _ in range(B)]).astype(np.int32)
+    want_o, want_lse, _ = oracle.sparse_attn(f64(q), f64(k), f64(v), q_idx=idx)
+    out = to_dev_bf16(cache)
+    lse = torch.zeros(B, H, N, device="cuda")
+    ws = A.new_workspace(A.OP_SPARSE_ATTN, B, H, N, M, d)
+    A.astraea_sparse_cross_attn(to_dev_bf16(q), to_dev_bf16(k), to_dev_bf16(v), A.bhnd_strides(N, H, d),
+                                A.bhnd_strides(N_kv, H, d), A.bhnd_strides(N_kv, H, d), dev(idx), M, out, lse,
+                                B, H, N, N_kv, d, workspace=ws)
+    A.astraea_poll_error(ws)
+    got = bf16_dev_to_f64(out)
+    got_rows = np.take_along_axis(got, idx[:, :, None, None].astype(np.int64), 1)
+    err = np.abs(got_rows - want_o)
+    assert err.max() < ATTN_MAX_ABS and err.mean() < ATTN_MEAN_ABS, (err.max(), err.mean())
+    got_lse = np.take_along_axis(lse.cpu().numpy().astype(np.float64), idx[:, None, :].astype(np.int64), 2)
+    assert np.abs(got_lse - want_lse).max() < LSE_ABS
+    mask = np.ones((B, N), bool)
+    for b in range(B):
+        mask[b, idx[b]] = False
+    assert np.array_equal(got[mask], f64(cache)[mask])
