@@ -142,10 +142,12 @@ __device__ __forceinline__ unsigned long long fadd2(unsigned long long a, float 
 
 // 2^x for a pair, without the XU pipe: x = n + f with n = floor(x) taken by adding 1.5 * 2^23 rounded down, a
 // cubic for 2^f on [0, 1) (relative error 8.6e-5, well below the bf16 rounding of P), and n added to the
-// exponent field.  x is clamped to the normal range first.
+// exponent field.  x is clamped to the normal range first: below it the result is 2^-126 instead of 0, which no sum
+// notices; above it the exponent field would wrap around to a small number and hide the overflow from the check
+// on the tile's sum, so x stops at 127, whose 2^127 trips that check as surely as the XU's +inf does.
 __device__ __forceinline__ void exp2_poly2(float &x0, float &x1) {
-    x0 = fmaxf(x0, -126.0f);
-    x1 = fmaxf(x1, -126.0f);
+    x0 = fminf(fmaxf(x0, -126.0f), 127.0f);
+    x1 = fminf(fmaxf(x1, -126.0f), 127.0f);
     unsigned long long x, t, pl;
     asm("mov.b64 %0, {%1, %2};" : "=l"(x) : "f"(x0), "f"(x1));
     asm("{\n\t.reg .b64 mg, c1, c2, c3, one, fr;\n\t"

@@ -265,6 +265,34 @@ def test_attn_reference_maximum_far_too_low_is_repaired_exactly(oracle, d):
 
 
 @pytest.mark.parametrize("d", [64, 72, 128])
+@pytest.mark.parametrize("col", [3, 12, 30, 47, 63])
+def test_attn_single_overflowing_key_in_any_column_of_a_later_tile(oracle, d, col):
+    """One key of the second tile beats everything in the first by 128 nats and nothing else is large: the only
+    exponential that overflows sits in column `col` of its tile, whichever pipe computes that column.  The rows
+    must come out as that key's value row (and the LSE as its logit)."""
+    B, H, N, M = 1, 1, 129, 20
+    rng = np.random.default_rng(60 + col)
+    q = np.zeros((B, N, H, d), np.float32)
+    k = np.zeros((B, N, H, d), np.float32)
+    q[..., 0] = 32.0
+    k[0, 64 + col, 0, 0] = 32.0 * math.sqrt(d) / 8.0          # logit 128 * sqrt(d) / sqrt(d) ... = 128 at that key, 0 elsewhere
+    v = rng.standard_normal((B, N, H, d)).astype(np.float32)
+    qb, kb, vb = (synth.f32_to_bf16_bits(a) for a in (q, k, v))
+    idx = np.sort(rng.choice(N, M, replace=False)).astype(np.int32)[None]
+    want_o, want_lse, _ = oracle.sparse_attn(f64(qb), f64(kb), f64(vb), q_idx=idx)
+    out = torch.zeros(B, M, H, d, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros(B, H, M, device="cuda")
+    ws = A.new_workspace(A.OP_SPARSE_ATTN, B, H, N, M, d)
+    s_ = A.bhnd_strides(N, H, d)
+    A.astraea_sparse_attn(to_dev_bf16(qb), to_dev_bf16(kb), to_dev_bf16(vb), s_, s_, s_, dev(idx), M, out, lse, B, H, N, d,
+                          flags=A.ATTN_COMPACT_OUT, workspace=ws)
+    A.astraea_poll_error(ws)
+    assert np.abs(bf16_dev_to_f64(out) - want_o).max() < ATTN_MAX_ABS
+    assert np.abs(lse.cpu().numpy() - want_lse).max() < 2e-2 * 1e-2 * 128          # relative 2e-4 of a logit of ~128
+    assert np.abs(want_o - f64(vb)[0, 64 + col][None, None]).max() < 1e-9            # the oracle agrees: one-hot rows
+
+
+@pytest.mark.parametrize("d", [64, 72, 128])
 def test_attn_select_q_and_k_ablation(oracle, d):
     """kv_idx: the softmax runs over the listed keys/values only (the ablation that also masks K and V)."""
     rng = np.random.default_rng(20 + d)
