@@ -182,11 +182,6 @@ __device__ __forceinline__ uint32_t map_to_rank(const void *p, uint32_t rank) {
 __device__ __forceinline__ void remote_add(uint32_t addr, uint32_t v) {
     asm volatile("red.relaxed.cluster.shared::cluster.add.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
-__device__ __forceinline__ uint32_t remote_load(uint32_t addr) {
-    uint32_t v;
-    asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
-    return v;
-}
 __device__ __forceinline__ void remote_store(uint32_t addr, uint32_t v) {
     asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
@@ -196,8 +191,8 @@ __global__ void __launch_bounds__(kThreads)
 select_cluster_kernel(const float *__restrict__ score, int N_sel, int k, int n_always,
                       int32_t *__restrict__ idx_sel, int32_t *__restrict__ idx_rem, int32_t *__restrict__ n_skip)
 {
-    __shared__ uint32_t hist[256];
-    __shared__ uint32_t ghist[4][256];          // summed histograms of the four passes (used in CTA 0 only)
+    __shared__ uint32_t hist[4][256];           // this CTA's histograms of the four passes
+    __shared__ uint32_t ghist[4][256];          // the cluster's histograms: every CTA adds its counts into every CTA's copy
     __shared__ uint32_t cta_tot[kMaxCluster];   // packed (greater | equal << 16) totals of every CTA
     __shared__ uint32_t warp_tot[32];
     __shared__ uint32_t s_prefix, s_kk;
@@ -215,8 +210,8 @@ select_cluster_kernel(const float *__restrict__ score, int N_sel, int k, int n_a
 #pragma unroll
     for (int u = 0; u < ITEMS; ++u) key[u] = (base + u < N_sel) ? score_key(__ldg(s + base + u)) : 0u;
 
-    for (int i = tid; i < 4 * 256; i += kThreads) (&ghist[0][0])[i] = 0;
-    cluster_sync_all();                          // CTA 0's histograms are zero before anyone adds to them
+    for (int i = tid; i < 4 * 256; i += kThreads) { (&ghist[0][0])[i] = 0; (&hist[0][0])[i] = 0; }
+    cluster_sync_all();                          // every CTA's histograms are zero before anyone adds to them
 
     uint32_t T = 0xffffffffu, need_eq = 0;       // no key reaches 0xffffffff
     if (k > 0) {
@@ -224,8 +219,6 @@ select_cluster_kernel(const float *__restrict__ score, int N_sel, int k, int n_a
 #pragma unroll 1
         for (int pass = 0; pass < 4; ++pass) {
             const int shift = 24 - 8 * pass;
-            for (int i = tid; i < 256; i += kThreads) hist[i] = 0;
-            __syncthreads();
 #pragma unroll
             for (int u = 0; u < ITEMS; ++u) {
                 const bool live = (base + u < N_sel) && ((key[u] & mask) == prefix);
@@ -237,20 +230,23 @@ select_cluster_kernel(const float *__restrict__ score, int N_sel, int k, int n_a
                 const int leader = __ffs(act) - 1;
                 const uint32_t lbin = __shfl_sync(0xffffffffu, bin, leader);
                 if (__all_sync(0xffffffffu, !live || bin == lbin)) {
-                    if (lane == leader) atomicAdd(&hist[lbin], (uint32_t)__popc(act));
+                    if (lane == leader) atomicAdd(&hist[pass][lbin], (uint32_t)__popc(act));
                 } else if (live) {
-                    atomicAdd(&hist[bin], 1u);
+                    atomicAdd(&hist[pass][bin], 1u);
                 }
             }
             __syncthreads();
-            if (tid < 256 && hist[tid] != 0) remote_add(map_to_rank(&ghist[pass][tid], 0), hist[tid]);
+            // thread (r, bin) adds this CTA's count of the bin into CTA r's copy, so that every CTA searches its own copy
+            for (int i = tid; i < 256 * (int)csize; i += kThreads) {
+                const uint32_t c = hist[pass][i & 255];
+                if (c != 0) remote_add(map_to_rank(&ghist[pass][i & 255], (uint32_t)i >> 8), c);
+            }
             cluster_sync_all();
             if (warp == 0) {
                 // lane l owns bins 255-8l .. 248-8l (descending); find where the count from the top reaches kk
-                const uint32_t g0 = map_to_rank(&ghist[pass][0], 0);
                 uint32_t c[8], tot = 0;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) { c[j] = remote_load(g0 + 4 * (255 - 8 * lane - j)); tot += c[j]; }
+                for (int j = 0; j < 8; ++j) { c[j] = ghist[pass][255 - 8 * lane - j]; tot += c[j]; }
                 uint32_t inc = tot;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
@@ -330,7 +326,7 @@ select_cluster_kernel(const float *__restrict__ score, int N_sel, int k, int n_a
         pe += eq[u];
     }
     if (rank == 0) for (int t = tid; t < n_always; t += kThreads) sel[k + t] = N_sel + t;
-    cluster_sync_all();                          // no CTA leaves while its shared memory may still be addressed
+    // no barrier at the end: the last remote accesses (the totals above) were complete at the barrier before the placement
 }
 
 template <int ITEMS>
