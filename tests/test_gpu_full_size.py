@@ -90,3 +90,48 @@ def test_sweep_shaped_full_size(oracle):
 
 def test_hunyuan_shaped_full_size(oracle):
     _full_size_case(oracle, "hunyuan", 600, rows=24, score_rows=2048)
+
+
+def test_cogvideox_shaped_projection_and_cross_attention_full_size(oracle):
+    """The layers next to the self-attention at the CogVideoX shape, keep-ratio 0.5: the query projection of the
+    9001 selected rows (K = N_out = 3072) and their cross-attention against 226 keys; sampled rows against the oracle,
+    all rows that were not listed bit-identical to what they held."""
+    w = synth.WORKLOADS["cogvideox"]
+    rng = np.random.default_rng(9)
+    B, N, H, d, D = w.B, w.N, w.H, w.d, w.D
+    M = w.k_of(500) + w.N_t
+    idx = np.stack([np.sort(rng.choice(N, M, replace=False)) for _ in range(B)]).astype(np.int32)
+    x = synth.f32_to_bf16_bits(rng.standard_normal((B, N, D)).astype(np.float32))
+    wq = synth.f32_to_bf16_bits((rng.standard_normal((D, D)) / math.sqrt(D)).astype(np.float32))
+    bq = synth.f32_to_bf16_bits(rng.standard_normal(D).astype(np.float32))
+    cache = synth.f32_to_bf16_bits(rng.standard_normal((B, N, D)).astype(np.float32))
+    y = to_dev_bf16(cache)
+    ws = A.new_workspace(A.OP_GATHERED_LINEAR, 0, 0, 0, 0, 0)
+    A.astraea_gathered_linear(to_dev_bf16(x), dev(idx), M, to_dev_bf16(wq), to_dev_bf16(bq), y, B, N, D, D, workspace=ws)
+    A.astraea_poll_error(ws)
+    pick = np.stack([np.sort(rng.choice(idx[b], 96, replace=False)) for b in range(B)]).astype(np.int32)
+    want = oracle.gathered_linear(f64(x), f64(wq), f64(bq), pick)
+    got = bf16_dev_to_f64(y)
+    err = np.abs(np.take_along_axis(got, pick[:, :, None].astype(np.int64), 1) - np.take_along_axis(want, pick[:, :, None].astype(np.int64), 1))
+    assert err.max() < 2e-2 and err.mean() < 2e-3, (err.max(), err.mean())
+    unsel = np.ones((B, N), bool)
+    for b in range(B):
+        unsel[b, idx[b]] = False
+    assert np.array_equal(got[unsel], f64(cache)[unsel])
+    # cross-attention of the same rows (as heads of the projected queries) against N_kv = 226 other tokens
+    N_kv = w.N_t
+    kx, vx = (synth.f32_to_bf16_bits(rng.standard_normal((B, N_kv, H, d)).astype(np.float32)) for _ in range(2))
+    q_bits = synth.f32_to_bf16_bits(got.astype(np.float32)).reshape(B, N, H, d)
+    out = to_dev_bf16(cache.reshape(B, N, H, d))
+    ws2 = A.new_workspace(A.OP_SPARSE_ATTN, B, H, N, M, d)
+    A.astraea_sparse_cross_attn(to_dev_bf16(q_bits), to_dev_bf16(kx), to_dev_bf16(vx), A.bhnd_strides(N, H, d),
+                                A.bhnd_strides(N_kv, H, d), A.bhnd_strides(N_kv, H, d), dev(idx), M, out, None,
+                                B, H, N, N_kv, d, workspace=ws2)
+    A.astraea_poll_error(ws2)
+    heads = [0, H // 2, H - 1]
+    want_o, _, _ = oracle.sparse_attn(f64(np.ascontiguousarray(q_bits[:, :, heads])), f64(np.ascontiguousarray(kx[:, :, heads])),
+                                      f64(np.ascontiguousarray(vx[:, :, heads])), q_idx=pick)
+    got_o = np.take_along_axis(bf16_dev_to_f64(out)[:, :, heads], pick[:, :, None, None].astype(np.int64), 1)
+    err = np.abs(got_o - want_o)
+    assert err.max() < 2e-2 and err.mean() < 2e-3, (err.max(), err.mean())
+    assert np.array_equal(bf16_dev_to_f64(out)[unsel], f64(cache.reshape(B, N, H, d))[unsel])
