@@ -4,19 +4,20 @@
 // rows; with idx == NULL the key / value projections of all tokens).
 //
 // A dense contraction, so it runs on the tcgen05 tensor cores.  Persistent CTAs, one per SM, walk over
-// 128-row x 256-column output tiles (column tiles of one row tile are neighbours in the walk, so the
-// gathered rows stay in L2 while W, which is small, lives there anyway).  Warp roles:
-//   warps 0-3  epilogue: one thread per output row; TMEM -> registers -> (+ bias) -> bf16 -> the row of y
-//              that idx names (fused scatter).  Two accumulators of 256 TMEM columns, so the epilogue of a
-//              tile runs under the main loop of the next;
-//   warps 4-7  gather of the A operand: the listed rows of x, 64 columns (128 bytes) per pipeline stage,
-//              by 16-byte cp.async into the 128-byte-swizzled layout the MMA reads (rows past the end
-//              are zero-filled); the copies arrive on the stage's barrier by themselves, so a thread never
-//              waits for its own copies, only for a free stage;
-//   warp 8     TMA producer of the B operand: a 256 x 64 tile of W per stage (rows past N_out read as zero);
-//   warp 9     tcgen05.mma issuer: four 128 x 256 x 16 SS MMAs per stage into the tile's accumulator.
-// Stages: 4 x (16 KB of A + 32 KB of W).  Every mbarrier wait is bounded; on a timeout the CTA raises the
-// error word, the remaining waits return at once, and the CTA runs out.
+// 256-row x 256-column output tiles (column tiles of one row tile are neighbours in the walk, so the
+// gathered rows stay in L2 while W, which is small, lives there anyway).  A tile is two 128-row sub-tiles
+// that share every W tile in shared memory.  Warp roles:
+//   warps 0-7   epilogue: one thread per output row; TMEM -> registers -> (+ bias, GELU) -> bf16 -> the row
+//               of y that idx names (fused scatter);
+//   warps 8-15  gather of the A operand: the listed rows of x, 64 columns (128 bytes) per pipeline stage,
+//               by 16-byte cp.async into the 128-byte-swizzled layout the MMA reads (rows past the end
+//               are zero-filled); the copies arrive on the stage's barrier by themselves, so a thread never
+//               waits for its own copies, only for a free stage;
+//   warp 16     TMA producer of the B operand: a 256 x 64 tile of W per stage (rows past N_out read as zero);
+//   warp 17     tcgen05.mma issuer: per stage four 128 x 256 x 16 SS MMAs into each sub-tile's accumulator.
+// Stages: 3 x (2 x 16 KB of A + 32 KB of W); TMEM: two accumulators of 256 columns.  Every mbarrier wait
+// is bounded; on a timeout the CTA raises the error word, the remaining waits return at once, and the
+// CTA runs out.
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 #include "bounded_wait.cuh"
@@ -26,10 +27,15 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kBM = 128, kBN = 256, kBK = 64;
-constexpr int kStages = 4;
-constexpr int kABytes = kBM * kBK * 2, kBBytes = kBN * kBK * 2;
-constexpr int kEpiWarps = 4, kGatherWarps = 4;
+// 128-row sub-tiles of a CTA tile, each with its own 256-column accumulator.  Two: a 256 x 256 tile reads 128 flop
+// per byte of operands from L2 instead of 85, which is what bounds this kernel; it fills TMEM, so the epilogue is
+// not hidden under the next main loop any more, and is still 4-15 % faster than one sub-tile with two accumulator sets.
+constexpr int kMSub = 2;
+constexpr int kBM = 128 * kMSub, kBN = 256, kBK = 64;
+constexpr int kStages = (kMSub == 2) ? 3 : 4;
+constexpr int kAccSets = 2 / kMSub;                      // accumulator sets in TMEM: two sets let the epilogue run under the next main loop
+constexpr int kASubBytes = 128 * kBK * 2, kABytes = kMSub * kASubBytes, kBBytes = kBN * kBK * 2;
+constexpr int kEpiWarps = 4 * kMSub, kGatherWarps = 4 * kMSub;
 constexpr int kThreads = (kEpiWarps + kGatherWarps + 2) * 32;
 constexpr int kTmaWarp = kEpiWarps + kGatherWarps, kMmaWarp = kTmaWarp + 1;
 constexpr int kSmemBytes = kStages * (kABytes + kBBytes) + 256 + 1024;
@@ -100,7 +106,7 @@ gathered_linear_kernel(const __grid_constant__ CUtensorMap tmap_w, const LinPara
             mbar_init(bar_full + 8 * s, kGatherWarps * 32 + 1);     // every gather thread + the TMA producer
             mbar_init(bar_empty + 8 * s, 1);
         }
-        for (int a = 0; a < 2; ++a) { mbar_init(bar_acc_full + 8 * a, 1); mbar_init(bar_acc_empty + 8 * a, kEpiWarps * 32); }
+        for (int a = 0; a < kAccSets; ++a) { mbar_init(bar_acc_full + 8 * a, 1); mbar_init(bar_acc_empty + 8 * a, kEpiWarps * 32); }
         fence_barrier_init();
     }
     if (warp == kMmaWarp) {
@@ -114,23 +120,23 @@ gathered_linear_kernel(const __grid_constant__ CUtensorMap tmap_w, const LinPara
 
     if (warp < kEpiWarps) {
         // ------------------------------------------------ epilogue
-        const int row = warp * 32 + lane;
-        const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);
+        const int row = warp * 32 + lane;                      // row of the CTA tile; sub-tile warp / 4, TMEM lanes by warp % 4
+        const uint32_t t_row = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (warp >> 2) * kAccCols;
         int it = 0;
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
             const int tm = tile / tiles_n, tn = tile - tm * tiles_n;
-            const int acc = it & 1, n0 = tn * kBN;
+            const int acc = it % kAccSets, n0 = tn * kBN;
             long long out_row = -1;
             const long long src = source_row(p, (long long)tm * kBM + row, total_rows, &out_row);
             if (src == -2 && tn == 0) atomicExch(p.err_word, kErrBadIndex);
             __nv_bfloat16 *dst = (src >= 0) ? p.y + out_row * p.N_out + n0 : nullptr;
-            wait_bar(bar_acc_full + 8 * acc, (it >> 1) & 1, &abort_flag, p.err_word);
+            wait_bar(bar_acc_full + 8 * acc, (it / kAccSets) & 1, &abort_flag, p.err_word);
             tc_fence_after();
             if (abort_flag) dst = nullptr;
 #pragma unroll 1
             for (int c = 0; c < kBN; c += 32) {
                 uint32_t o[32];
-                tmem_ld32(t_row + acc * kAccCols + c, o);
+                tmem_ld32(t_row + acc * kMSub * kAccCols + c, o);
                 tc_wait_ld();
                 if (c + 32 == kBN) {                     // the accumulator has been read: the MMA warp may reuse it
                     tc_fence_before();
@@ -169,8 +175,8 @@ gathered_linear_kernel(const __grid_constant__ CUtensorMap tmap_w, const LinPara
         }
     } else if (warp < kEpiWarps + kGatherWarps) {
         // ------------------------------------------------ gather of the A rows (cp.async, 128-byte swizzle)
-        const int t = tid - kEpiWarps * 32;                   // 0..127
-        const int chunk = t & 7, row0 = t >> 3;               // this thread: 16-byte chunk `chunk` of rows row0 + 16 i
+        const int t = tid - kEpiWarps * 32;                   // 0 .. 128 kMSub - 1
+        const int chunk = t & 7, row0 = t >> 3;               // this thread: 16-byte chunk `chunk` of rows row0 + 16 kMSub i
         int g = 0;                                            // running stage count over all tiles
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
             const int tm = tile / tiles_n;
@@ -178,10 +184,10 @@ gathered_linear_kernel(const __grid_constant__ CUtensorMap tmap_w, const LinPara
             uint32_t off[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                const int r = row0 + 16 * i;
+                const int r = row0 + 16 * kMSub * i;
                 const long long s = source_row(p, (long long)tm * kBM + r, total_rows, nullptr);
                 src[i] = (s >= 0) ? p.x + s * p.K + chunk * 8 : nullptr;
-                off[i] = r * 128 + ((chunk ^ (r & 7)) << 4);
+                off[i] = (r >> 7) * kASubBytes + (r & 127) * 128 + ((chunk ^ (r & 7)) << 4);
             }
             for (int ks = 0; ks < k_steps; ++ks, ++g) {
                 const int st = g % kStages;
@@ -213,11 +219,11 @@ gathered_linear_kernel(const __grid_constant__ CUtensorMap tmap_w, const LinPara
             wait_bar(bar_full + 8 * (gs % kStages), (gs / kStages) & 1, &abort_flag, p.err_word);
     } else {
         // ------------------------------------------------ MMA issuer
-        constexpr uint32_t idesc = idesc_bf16(kBM, kBN, false);
+        constexpr uint32_t idesc = idesc_bf16(128, kBN, false);
         int g = 0, it = 0;
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
-            const int acc = it & 1;
-            wait_bar(bar_acc_empty + 8 * acc, ((it >> 1) & 1) ^ 1, &abort_flag, p.err_word);
+            const int acc = it % kAccSets;
+            wait_bar(bar_acc_empty + 8 * acc, ((it / kAccSets) & 1) ^ 1, &abort_flag, p.err_word);
             for (int ks = 0; ks < k_steps; ++ks, ++g) {
                 const int st = g % kStages;
                 wait_bar(bar_full + 8 * st, (g / kStages) & 1, &abort_flag, p.err_word);
@@ -225,11 +231,14 @@ gathered_linear_kernel(const __grid_constant__ CUtensorMap tmap_w, const LinPara
                 tc_fence_after();
                 if (elect_one()) {
 #pragma unroll
-                    for (int kk = 0; kk < kBK / 16; ++kk)
-                        mma_ss(tmem + acc * kAccCols,
-                               smem_desc(sA + st * kABytes + kk * 32, 16, 1024, kSwizzle128B),
-                               smem_desc(sB + st * kBBytes + kk * 32, 16, 1024, kSwizzle128B),
-                               idesc, (ks > 0 || kk > 0) ? 1u : 0u);
+                    for (int kk = 0; kk < kBK / 16; ++kk) {
+#pragma unroll
+                        for (int sub = 0; sub < kMSub; ++sub)       // the sub-tiles share the W tile in shared memory
+                            mma_ss(tmem + (acc * kMSub + sub) * kAccCols,
+                                   smem_desc(sA + st * kABytes + sub * kASubBytes + kk * 32, 16, 1024, kSwizzle128B),
+                                   smem_desc(sB + st * kBBytes + kk * 32, 16, 1024, kSwizzle128B),
+                                   idesc, (ks > 0 || kk > 0) ? 1u : 0u);
+                    }
                     tc_commit(bar_empty + 8 * st);
                     if (ks == k_steps - 1) tc_commit(bar_acc_full + 8 * acc);
                 }
