@@ -15,21 +15,22 @@
 //
 // Two softmax warpgroups per query tile put four softmax warps on every SM sub-partition, which hides the
 // serial chain of a key tile (wait, load, exponentials, sum, pack, publish).  Even key tiles go to one
-// warpgroup and odd ones to the other; both work against the same reference maximum and their P tiles
-// accumulate into ONE O accumulator per query tile.  That leaves TMEM room for three S buffers per query
-// tile at head_dim 64 (S of key tile j+2 is computed while tiles j and j+1 are in the softmax) and for
-// two at head_dim 72 / 128 (a buffer is refilled with key tile j+2 as soon as P of tile j has been
-// consumed; the tensor pipe executes one thread's MMAs in order).
+// warpgroup and odd ones to the other, each with an S buffer of its own, which is refilled with key tile
+// j+2 as soon as P of tile j has been consumed (the tensor pipe executes one thread's MMAs in order); both
+// work against the same reference maximum and their P tiles accumulate into ONE O accumulator per query
+// tile.
 //
 // The softmax is bound by the exponentials (XU pipe, 16 per clock per SM), by the issue slots and by the
 // latencies of its own chain, so the common path of a key tile is kept to: load S, one FFMA + one
-// exponential per element, sum, pack, store.  At head_dim 64 / 72 six / four of every sixteen exponentials
-// are a cubic on the FMA pipe instead of ex2 on the XU.  The reference maximum is the exact row maximum of key
-// tile 0 and is then only checked through each tile's sum of exponentials: while that sum stays below a
-// limit the tile is accepted as it is (the probabilities are relative to a stale maximum, which the final
-// normalisation cancels; fp32 and bf16 have the range).  Otherwise the CTA raises a flag, finishes the
-// pass, and redoes its work in two more passes over the keys: exact row maxima first, then the softmax
-// against them (the accumulator is shared by two warpgroups, so it is not rescaled in place).
+// exponential per element, (sum,) pack, store.  At head_dim 64 / 72 six / four of every sixteen
+// exponentials are a cubic on the FMA pipe instead of ex2 on the XU, and at head_dim 64 the row sums are
+// left to the tensor core (P times a column of ones, 16 more accumulator columns).  The reference maximum
+// is the exact row maximum of key tile 0 (plus a shift) and is then only checked through the sums of
+// exponentials: while they stay below a limit the probabilities are accepted as they are (they are relative
+// to a stale maximum, which the final normalisation cancels; fp32 and bf16 have the range).  Otherwise the
+// CTA raises a flag, finishes the pass, and redoes its work in two more passes over the keys: exact row
+// maxima first, then the softmax against them (the accumulator is shared by two warpgroups, so it is not
+// rescaled in place).
 //
 // TMEM columns: S/P of (tile t, buffer u) at (kSBufs t + u) * kBlockN; the O accumulators behind them.
 // The producer and issuer warps run warp-uniform code and elect one lane per instruction, so
@@ -70,18 +71,23 @@ template <int DH> struct Cfg {
     static constexpr int kTailPad = kTail ? 16 : 0;
     static_assert(kTail == 0 || kTail == 8, "head_dim must be 64, 72 or 128");
     static constexpr int kBlockN = 64;                            // keys per K/V tile = columns of an S buffer
-    // S buffers per query tile, used round-robin by its two softmax warpgroups.  Three where TMEM has the room
-    // (head_dim 64): S of key tile j+2 is then produced while tiles j and j+1 are in the softmax.
-    static constexpr int kSBufs = (DH == 64) ? 3 : 2;
+    // Row sums by the tensor core at head_dim 64: P times a column of ones into 16 more accumulator columns.  That
+    // takes the 64 packed adds per key tile off the softmax warps, whose issue slots are what is short there
+    // (+6 %), and normalises O by the sum of the very bf16 probabilities that went into it; the row sum, and with it
+    // the LSE, then carries the bf16 rounding of the probabilities (up to 2^-8 relative when one key dominates a row).
+    // head_dim 72 gains nothing from it and 128 has no TMEM columns left: they sum the fp32 exponentials themselves.
+    static constexpr bool kOnes = DH == 64;
+    static constexpr int kSBufs = 2;                              // S buffers per query tile: one per softmax warpgroup
     // exponentials per 16 that are computed on the FMA pipe instead of the XU (measured best: 6 at head_dim 64, 4 at
     // 72, none at 128, where the tensor pipe is as busy as the XU)
     static constexpr int kPolyOf16 = (DH == 64) ? 6 : (DH == 72) ? 4 : 0;
     static constexpr int kSoftmaxWarps = 4 * kTilesM * kSplit;
-    static constexpr int kAhead = 2;                              // Q K^T runs this many key tiles ahead of P V
+    static constexpr int kAhead = kSBufs;                         // Q K^T runs this many key tiles ahead of P V
     static constexpr int kThreads = (kSoftmaxWarps + 4) * 32;     // + producer, two issuers, one register donor
     static constexpr uint32_t kColO = kTilesM * kSBufs * kBlockN; // first O column
-    static constexpr uint32_t kOStride = (DH == 64) ? 64 : (DH == 72) ? 80 : 128;   // columns between O accumulators
-    static_assert(kColO + kTilesM * kOStride <= kTmemCols && kMain + kTailPad <= (int)kOStride, "TMEM budget");
+    static constexpr uint32_t kOnesCol = kMain + kTailPad;       // accumulator column that receives the row sums
+    static constexpr uint32_t kOStride = kMain + kTailPad + (kOnes ? 16 : 0);   // columns between O accumulators
+    static_assert(kColO + kTilesM * kOStride <= kTmemCols, "TMEM budget");
     // setmaxnreg only redistributes what the CTA got at launch: an increase that the decreases of
     // the last warpgroup cannot cover would block forever
     static constexpr int kRegsLaunch = (65536 / kThreads) / 8 * 8;
@@ -100,7 +106,8 @@ template <int DH> struct Cfg {
     static constexpr int kStagesV = (DH == 128) ? 4 : 6;
     static_assert(kStagesK > kAhead, "K runs kAhead tiles ahead");
     static constexpr int kBarBytes = 512;
-    static constexpr int kSmemBytes = kQTileBytes * kTilesM + kTileBytes * (kStagesK + kStagesV) + kBarBytes + 1024;
+    static constexpr int kOnesBytes = kOnes ? kBlockN * 32 : 0;  // a key tile x 16 columns of bf16: ones in column 0
+    static constexpr int kSmemBytes = kQTileBytes * kTilesM + kTileBytes * (kStagesK + kStagesV) + kOnesBytes + kBarBytes + 1024;
 };
 
 struct Params {
@@ -313,8 +320,8 @@ __device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j, int g)
             else { cur[i + u] = ex2(cur[i + u]); cur[i + u + 1] = ex2(cur[i + u + 1]); }
         }
     }
-    float tile_sum;
-    {
+    float tile_sum = 0.f;
+    if constexpr (!C::kOnes) {
         unsigned long long a[4] = {0ull, 0ull, 0ull, 0ull};
 #pragma unroll
         for (int i = 0; i < NS; i += 8) {
@@ -330,7 +337,7 @@ __device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j, int g)
     // in the shadow of the sum and the vote
     uint32_t pk[NS / 2];
     pack_p<NS>(cur, pk);
-    if constexpr (MODE == kSpeculate) {
+    if constexpr (MODE == kSpeculate && !C::kOnes) {
         // rare: the reference is too low for this tile.  The CTA finishes the pass and redoes its work with exact maxima
         if (__any_sync(0xffffffffu, !(tile_sum <= kTileSumLimit))) *st.redo_flag = 1;
     }
@@ -402,6 +409,16 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     }
     for (int j = par; j < n_tiles; j += kSplit) softmax_step<DH, kSpeculate>(st, j, j);
     wait_bar(st.bar_done, 0, abort_flag, p.err_word);            // every P V of this query tile has landed
+    if constexpr (C::kOnes) {
+        // the row sum came out of the tensor core with O; one that passed the limit (or is inf / NaN) means that
+        // the reference was too low somewhere along the row
+        tc_fence_after();
+        uint32_t o[8];
+        tmem_ld8(st.t_o + C::kOnesCol, o);
+        tc_wait_ld();
+        st.l_sum = __uint_as_float(o[0]);
+        if (__any_sync(0xffffffffu, !(st.l_sum <= kTileSumLimit))) *redo_flag = 1;
+    }
     pass_sync<DH>();
     if (*redo_flag) {
         // a tile overflowed somewhere in the CTA: exact row maxima first, then the whole pass again
@@ -415,15 +432,25 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
         st.l_sum = 0.f;
         for (int j = par; j < n_tiles; j += kSplit) softmax_step<DH, kExact>(st, j, 2 * n_tiles + j);
         wait_bar(st.bar_done, 1, abort_flag, p.err_word);
+        if constexpr (C::kOnes) {
+            tc_fence_after();
+            uint32_t o[8];
+            tmem_ld8(st.t_o + C::kOnesCol, o);
+            tc_wait_ld();
+            st.l_sum = __uint_as_float(o[0]);
+        }
     }
 
     // ------------------------------------------------ epilogue: normalise and scatter
     tc_fence_after();
     // both warpgroups accumulated into one O against one reference: add the row sums, split the columns
-    xchg[wtid + par * kBlockM].y = st.l_sum;
-    if (tile == 0) asm volatile("bar.sync 1, 256;" ::: "memory");
-    else asm volatile("bar.sync 2, 256;" ::: "memory");
-    const float l_sum = xchg[wtid].y + xchg[wtid + kBlockM].y;
+    float l_sum = st.l_sum;                                      // with the ones column: the row's whole sum already
+    if constexpr (!C::kOnes) {
+        xchg[wtid + par * kBlockM].y = st.l_sum;
+        if (tile == 0) asm volatile("bar.sync 1, 256;" ::: "memory");
+        else asm volatile("bar.sync 2, 256;" ::: "memory");
+        l_sum = xchg[wtid].y + xchg[wtid + kBlockM].y;
+    }
     constexpr int ncol = C::kMain / 2;                           // O columns this thread writes
     const int col0 = par * ncol;
     const float inv_l = 1.0f / l_sum;
@@ -486,7 +513,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     const uint32_t sQ = smem_base;
     const uint32_t sK = sQ + kTilesM * C::kQTileBytes;
     const uint32_t sV = sK + C::kStagesK * C::kTileBytes;
-    const uint32_t bars = sV + C::kStagesV * C::kTileBytes;
+    const uint32_t sOnes = sV + C::kStagesV * C::kTileBytes;       // [key tile x 16 columns] bf16, 32-byte swizzle, column 0 = 1
+    const uint32_t bars = sOnes + C::kOnesBytes;
     Bars bar;
     bar.q = bars; bar.s = bars + 16; bar.p = bars + 80; bar.done = bars + 144;
     bar.kf = bars + 160;
@@ -503,6 +531,16 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     // the last CTA of a head may have rows in its first query tile only: the second tile's warps and MMAs are skipped
     const int q_tiles = (m0 + kBlockM < p.M) ? kTilesM : 1;
 
+    if constexpr (C::kOnes) {
+        // row r: 32 bytes; the 16-byte unit that holds column 0 is unit (r >> 2) & 1 under the 32-byte swizzle
+        uint8_t *ones = smem_gen + (sOnes - smem_base);
+        for (int i = tid; i < kBlockN * 2; i += C::kThreads) {
+            const int r = i >> 1, unit = i & 1;
+            const uint32_t first = (unit == ((r >> 2) & 1)) ? 0x3F80u : 0u;      // bf16 1.0 in column 0
+            *reinterpret_cast<uint4 *>(ones + r * 32 + unit * 16) = make_uint4(first, 0u, 0u, 0u);
+        }
+        fence_proxy_async_smem();
+    }
     if (tid == 0) {
         abort_flag = 0;
         redo_flag = 0;
@@ -638,16 +676,6 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                 const bool more = j + kAhead < n_tiles;
                 const int sk = (gk0 + j + kAhead) % C::kStagesK;
                 if (more) wait_bar(bar.kf + 8 * sk, ((gk0 + j + kAhead) / C::kStagesK) & 1, &abort_flag, p.err_word);
-                if constexpr (kSBufs > kAhead) {
-                    // a third S buffer: the one of key tile j-1 was consumed by the P V issued last (in-order pipe),
-                    // so S of key tile j+2 is started before waiting for P of tile j
-                    tc_fence_after();
-                    if (more && elect_one()) {
-                        issue_qk(t, gs0 + j + kAhead, sK + sk * C::kTileBytes);
-                        tc_commit(bar.ke + 8 * sk);
-                    }
-                    __syncwarp();
-                }
                 if (with_v) wait_bar(bar.vf + 8 * sv, ((gv0 + j) / C::kStagesV) & 1, &abort_flag, p.err_word);
                 // P of key tile j is in TMEM (max-only pass: S of key tile j has been read)
                 wait_bar(bar.p + 32 * t + 8 * u, ((gs0 + j) / kSBufs) & 1, &abort_flag, p.err_word);
@@ -663,12 +691,16 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                                 mma_ts(tmem + o_col + C::kMain, tmem + (t * kSBufs + u) * kBlockN + ks * 8,
                                        smem_desc(vbase + C::kChunks * C::kChunkBytes + ks * 512, 256, 256, kSwizzle32B),
                                        idesc_pv_tail, (j > 0 || ks > 0) ? 1u : 0u);
+                            if (C::kOnes)  // the row sums: P times the column of ones
+                                mma_ts(tmem + o_col + C::kOnesCol, tmem + (t * kSBufs + u) * kBlockN + ks * 8,
+                                       smem_desc(sOnes + ks * 512, 256, 256, kSwizzle32B),
+                                       idesc_pv_tail, (j > 0 || ks > 0) ? 1u : 0u);
                         }
                         tc_commit(bar.ve + 8 * sv);
                         if (j == n_tiles - 1) tc_commit(bar.done + 8 * t);        // the pass is done for this query tile
                     }
-                    // two S buffers: the one just consumed as P is free again (in-order pipe), refill it with key tile j+2
-                    if (kSBufs == kAhead && more) {
+                    // the S buffer just consumed as P is free again (in-order pipe): refill it with key tile j+2
+                    if (more) {
                         issue_qk(t, gs0 + j + kAhead, sK + sk * C::kTileBytes);
                         tc_commit(bar.ke + 8 * sk);
                     }
