@@ -67,3 +67,33 @@ def test_argument_errors_are_reported_before_any_launch(L):
     assert L.astraea_scatter_reuse(p, p, p, 1, 16, 17, 16, 0, None) == binding.ERR_INVALID_ARG
     assert L.astraea_scatter_reuse(p, p, p, 1, 16, 0, 16, 0, None) == binding.OK     # M = 0: nothing to do
     assert L.astraea_poll_error(None, None) == binding.ERR_INVALID_ARG
+
+
+def test_argument_errors_of_the_next_layer_entry_points(L):
+    p = ctypes.c_void_p(0x1000)
+    lin = lambda K=64, N_out=64, M=4, flags=0, ws=p, wsb=4096, idx=p, x=p: L.astraea_gathered_linear(
+        x, idx, M, p, None, p, 1, 16, K, N_out, flags, ws, wsb, None)
+    assert lin(K=60) == binding.ERR_INVALID_ARG and b"multiple of 64" in L.astraea_last_error()
+    assert lin(N_out=12) == binding.ERR_INVALID_ARG
+    assert lin(M=17) == binding.ERR_INVALID_ARG
+    assert lin(flags=64) == binding.ERR_UNSUPPORTED
+    assert lin(flags=binding.LINEAR_COMPACT_OUT, idx=None) == binding.ERR_INVALID_ARG     # compact rows need a list
+    assert lin(wsb=8) == binding.ERR_WORKSPACE_TOO_SMALL
+    assert lin(ws=ctypes.c_void_p(0x1010)) == binding.ERR_INVALID_ARG
+    assert lin(x=None) == binding.ERR_INVALID_ARG
+    assert lin(M=0) == binding.OK                                                         # an empty list: nothing to do
+    s = (64 * 16, 64, 64)
+    cross = lambda N_kv=8, d=64: L.astraea_sparse_cross_attn(p, p, p, *s, *s, *s, None, 16, p, None, 1, 1, 16, N_kv, d, 0.0, 0,
+                                                             p, 4096, None)
+    assert cross(N_kv=0) == binding.ERR_INVALID_ARG and b"N_kv" in L.astraea_last_error()
+    assert cross(d=80) == binding.ERR_UNSUPPORTED and b"astraea_sparse_cross_attn" in L.astraea_last_error()
+    h = ctypes.c_void_p()
+    kk = (ctypes.c_int32 * 2)(4, 99)
+    arr = (ctypes.c_void_p * 2)(0x1000, 0x1000)
+    sched = lambda T=2, keep=kk, wsb=1 << 20: L.astraea_schedule_create(ctypes.byref(h), T, keep, arr, arr, arr, arr, p, p, p, p, p, p, None,
+                                                                         1, 1, 16, 16, 64, 1.0, 1.0, 0, 0, p, wsb)
+    assert sched() == binding.ERR_INVALID_ARG and b"k_keep[1]=99" in L.astraea_last_error() and not h.value
+    assert sched(T=0) == binding.ERR_INVALID_ARG
+    assert sched(keep=(ctypes.c_int32 * 2)(4, 4), wsb=8) == binding.ERR_WORKSPACE_TOO_SMALL
+    assert L.astraea_schedule_launch(None, None) == binding.ERR_INVALID_ARG
+    L.astraea_schedule_destroy(None)                                                       # a null handle is ignored
