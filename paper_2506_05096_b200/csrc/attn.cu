@@ -194,7 +194,7 @@ template <int DH> struct SoftmaxState {
     float sl2, m_ref, l_sum;
     float shift;                    // the exponentials are taken against m_ref * sl2 + shift (log2 domain)
     uint32_t t_s0, t_o, bar_s, bar_p, bar_done;
-    int N, n_tiles;
+    int N;                          // keys
     float *ref_x;                   // the reference of this thread's row, shared by the tile's two warpgroups
     int ref_bar;                    // named barrier on which the reference is handed over
     volatile int *redo_flag;
@@ -389,7 +389,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     st.t_s0 = t_row + tile * C::kSBufs * C::kBlockN;
     st.t_o = t_row + C::kColO + tile * C::kOStride;
     st.bar_s = bar.s + 32 * tile; st.bar_p = bar.p + 32 * tile; st.bar_done = bar.done + 8 * tile;
-    st.N = p.N; st.n_tiles = n_tiles; st.abort_flag = abort_flag; st.err_word = p.err_word;
+    st.N = p.N; st.abort_flag = abort_flag; st.err_word = p.err_word;
     st.ref_x = &xchg[wtid].x; st.ref_bar = 3 + tile; st.redo_flag = redo_flag;
 
     const int m = m_base + wtid;
