@@ -52,6 +52,8 @@ extern "C" {
 
 /* flags of astraea_sparse_attn */
 #define ASTRAEA_ATTN_COMPACT_OUT  1u         /* out is [B,M,H,d] and lse_out [B,H,M] (row r of the index list), not the caches */
+#define ASTRAEA_ATTN_SMALL_CTAS   2u         /* head_dim 64 / 72: one 128-row query tile per CTA, two CTAs per SM, whatever the
+                                              * launch-time estimate says (without the flag the library picks the faster shape) */
 /* flags of astraea_gathered_linear */
 #define ASTRAEA_LINEAR_COMPACT_OUT 1u        /* y is [B,M,N_out] (row r of the index list), not the cache [B,N,N_out] */
 #define ASTRAEA_LINEAR_COMPACT_IN  2u        /* x is [B,M,K]: row r is the row of token idx[b,r] (output of a layer run with COMPACT_OUT) */

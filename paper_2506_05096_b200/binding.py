@@ -20,6 +20,7 @@ ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_TIMEOUT
 DELTA_MEAN_ABS, DELTA_MEAN_SQ, DELTA_MEAN_SIGNED = 0, 1, 2
 LSE_SUM_EXP, LSE_LOG = 0, 1
 ATTN_COMPACT_OUT = 1
+ATTN_SMALL_CTAS = 2
 SCATTER_SRC_FULL = 1
 LINEAR_COMPACT_OUT, LINEAR_COMPACT_IN, LINEAR_GELU = 1, 2, 4
 OP_SELECT, OP_SPARSE_ATTN, OP_STEP, OP_SPARSE_ATTN_KV, OP_GATHERED_LINEAR = 1, 2, 3, 4, 5

@@ -105,7 +105,7 @@ static int32_t sparse_attn_entry(const char *fn, int N_kv, const void *q, const 
     REQUIRE(M >= 0 && M <= N, "%s: M=%d outside [0, N=%d]", fn, M, N);
     if (d != 64 && d != 72 && d != 128)
         return fail(ASTRAEA_ERR_UNSUPPORTED, "%s: head_dim %d not in {64, 72, 128}", fn, d);
-    if (flags & ~ASTRAEA_ATTN_COMPACT_OUT) return fail(ASTRAEA_ERR_UNSUPPORTED, "%s: unknown flags 0x%x", fn, flags);
+    if (flags & ~(ASTRAEA_ATTN_COMPACT_OUT | ASTRAEA_ATTN_SMALL_CTAS)) return fail(ASTRAEA_ERR_UNSUPPORTED, "%s: unknown flags 0x%x", fn, flags);
     REQUIRE(q && k && v && out, "%s: null q, k, v or out", fn);
     REQUIRE(aligned16(q) && aligned16(k) && aligned16(v) && aligned16(out), "%s: q, k, v, out must be 16-byte aligned", fn);
     REQUIRE(q_sn % 8 == 0 && k_sn % 8 == 0 && v_sn % 8 == 0 && q_sh % 8 == 0 && k_sh % 8 == 0 && v_sh % 8 == 0 &&

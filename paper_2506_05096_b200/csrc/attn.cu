@@ -49,7 +49,6 @@ namespace {
 using namespace ptx;
 
 constexpr int kBlockM = 128;                     // rows of one query tile
-constexpr int kTilesM = 2;                       // query tiles per CTA
 constexpr int kSplit = 2;                        // softmax warpgroups per query tile: one takes the even key tiles, one the odd
 // The speculative reference of a row is the exact maximum of its first key tile plus kRefShift (log2 domain), and
 // a tile whose sum of exponentials passes kTileSumLimit means that this reference is too low.  fp32 and bf16 share
@@ -61,9 +60,16 @@ constexpr int kSplit = 2;                        // softmax warpgroups per query
 // row of most CTAs, but not 100.
 constexpr float kRefShift = 48.0f;
 constexpr float kTileSumLimit = 1267650600228229401496703205376.0f;   // 2^100
-constexpr uint32_t kTmemCols = 512;
 
-template <int DH> struct Cfg {
+// DH: head_dim.  TM: 128-row query tiles per CTA.  Two share every K/V tile in shared memory and run one CTA per SM;
+// one (head_dim 64 / 72 only) lets two CTAs share an SM, which costs ~5 % of throughput per SM but halves the
+// granularity of the schedule: launches of only a few rounds of CTAs are faster with it.
+template <int DH, int TM> struct Cfg {
+    static constexpr int kDH = DH;
+    static constexpr int kTilesM = TM;
+    static constexpr int kCtasPerSM = (TM == 1) ? 2 : 1;
+    static constexpr uint32_t kTmemCols = 512 / kCtasPerSM;
+    static_assert(TM == 2 || DH != 128, "head_dim 128 needs the whole SM");
     // head_dim = kMain (whole 64-column, 128-byte-swizzled chunks) + kTail (8 columns at head_dim 72,
     // carried as a 16-column, 32-byte-swizzled chunk whose upper half is zero)
     static constexpr int kMain = DH / 64 * 64;
@@ -90,8 +96,8 @@ template <int DH> struct Cfg {
     static_assert(kColO + kTilesM * kOStride <= kTmemCols, "TMEM budget");
     // setmaxnreg only redistributes what the CTA got at launch: an increase that the decreases of
     // the last warpgroup cannot cover would block forever
-    static constexpr int kRegsLaunch = (65536 / kThreads) / 8 * 8;
-    static constexpr int kRegsSoftmax = 112, kRegsOther = 32;
+    static constexpr int kRegsLaunch = (65536 / kCtasPerSM / kThreads) / 8 * 8;
+    static constexpr int kRegsSoftmax = (kCtasPerSM == 2) ? 104 : 112, kRegsOther = 32;
     static_assert(kRegsSoftmax * kSoftmaxWarps * 32 + kRegsOther * 128 <= kRegsLaunch * kThreads, "setmaxnreg budget");
     static constexpr int kChunks = kMain / 64;                    // 64-column (128-byte) swizzle chunks
     static constexpr int kQChunkBytes = kBlockM * 128;            // 128 query rows x 128 bytes
@@ -102,8 +108,8 @@ template <int DH> struct Cfg {
     static constexpr int kLoadBytes = kChunks * kChunkBytes + kTailBytes;   // what TMA delivers per K or V tile
     static constexpr int kTileBytes = (kLoadBytes + 1023) / 1024 * 1024;    // stage size (keeps the swizzle alignment)
     static_assert(kQTileBytes % 1024 == 0 && kTileBytes % 1024 == 0, "tiles keep the 1024-byte swizzle alignment");
-    static constexpr int kStagesK = (DH == 128) ? 5 : 6;
-    static constexpr int kStagesV = (DH == 128) ? 4 : 6;
+    static constexpr int kStagesK = (kCtasPerSM == 2) ? 4 : (DH == 128) ? 5 : 6;     // two CTAs per SM: <= 113 KB each
+    static constexpr int kStagesV = (kCtasPerSM == 2) ? 4 : (DH == 128) ? 4 : 6;
     static_assert(kStagesK > kAhead, "K runs kAhead tiles ahead");
     static constexpr int kBarBytes = 512;
     static constexpr int kOnesBytes = kOnes ? kBlockN * 32 : 0;  // a key tile x 16 columns of bf16: ones in column 0
@@ -190,7 +196,7 @@ struct Bars {
     uint32_t kf, ke, vf, ve;        // [stages]
 };
 
-template <int DH> struct SoftmaxState {
+struct SoftmaxState {
     float sl2, m_ref, l_sum;
     float shift;                    // the exponentials are taken against m_ref * sl2 + shift (log2 domain)
     uint32_t t_s0, t_o, bar_s, bar_p, bar_done;
@@ -279,10 +285,9 @@ enum { kSpeculate = 0, kMaxOnly = 1, kExact = 2 };
 
 // One key tile of the softmax.  j: key tile; g: running count of S-buffer uses of this query tile (buffer
 // g % kSBufs, barrier phase (g / kSBufs) & 1), which keeps counting across the passes.
-template <int DH, int MODE>
-__device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j, int g)
+template <class C, int MODE>
+__device__ __forceinline__ void softmax_step(SoftmaxState &st, int j, int g)
 {
-    using C = Cfg<DH>;
     constexpr int kSBufs = C::kSBufs, NS = C::kBlockN;
     const int buf = g % kSBufs;
     const uint32_t t_s = st.t_s0 + buf * NS;
@@ -347,18 +352,17 @@ __device__ __forceinline__ void softmax_step(SoftmaxState<DH> &st, int j, int g)
 }
 
 // All warps of the CTA meet after the speculative pass and then agree on the redo flag.
-template <int DH>
+template <class C>
 __device__ __forceinline__ void pass_sync() {
-    asm volatile("bar.sync 5, %0;" ::"n"(Cfg<DH>::kThreads) : "memory");
+    asm volatile("bar.sync 5, %0;" ::"n"(C::kThreads) : "memory");
 }
 
 // ---------------------------------------------------------------- softmax warpgroup
 // tile: its query tile; par: which key tiles it takes (j = par, par + kSplit, ...)
-template <int DH>
+template <class C>
 __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, int tile, int par, uint8_t *sQ_gen, uint32_t tmem,
                                              int m_base, int h, int b, int n_tiles, volatile int *abort_flag, volatile int *redo_flag, float2 *xchg)
 {
-    using C = Cfg<DH>;
     const int wtid = threadIdx.x & 127;
     const int warp = __shfl_sync(0xffffffffu, wtid >> 5, 0);       // warp-uniform
     // gather this tile's Q rows (swizzled, K-major): 16-byte units, unit c of row r
@@ -367,7 +371,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
         const int r = v / kUnits, c = v - r * kUnits;
         const int m = m_base + r;
         uint4 val = make_uint4(0, 0, 0, 0);
-        if (m < p.M && c * 8 < DH) {                 // the upper half of the tail chunk stays zero
+        if (m < p.M && c * 8 < C::kDH) {                 // the upper half of the tail chunk stays zero
             const int tok = p.q_idx ? __ldg(p.q_idx + (size_t)b * p.M + m) : m;
             if ((unsigned)tok < (unsigned)p.N_tok) {
                 const __nv_bfloat16 *src = p.q + (size_t)b * p.q_sb + (size_t)tok * p.q_sn + (size_t)h * p.q_sh + c * 8;
@@ -383,7 +387,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     mbar_arrive(bar.q + 8 * tile);
 
     const uint32_t t_row = tmem + ((uint32_t)(warp * 32) << 16);
-    SoftmaxState<DH> st;
+    SoftmaxState st;
     st.sl2 = p.scale_log2;
     st.l_sum = 0.f;
     st.t_s0 = t_row + tile * C::kSBufs * C::kBlockN;
@@ -407,7 +411,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
         else asm volatile("bar.sync 4, 256;" ::: "memory");
         st.m_ref = *st.ref_x;
     }
-    for (int j = par; j < n_tiles; j += kSplit) softmax_step<DH, kSpeculate>(st, j, j);
+    for (int j = par; j < n_tiles; j += kSplit) softmax_step<C, kSpeculate>(st, j, j);
     wait_bar(st.bar_done, 0, abort_flag, p.err_word);            // every P V of this query tile has landed
     if constexpr (C::kOnes) {
         // the row sum came out of the tensor core with O; one that passed the limit (or is inf / NaN) means that
@@ -419,18 +423,18 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
         st.l_sum = __uint_as_float(o[0]);
         if (__any_sync(0xffffffffu, !(st.l_sum <= kTileSumLimit))) *redo_flag = 1;
     }
-    pass_sync<DH>();
+    pass_sync<C>();
     if (*redo_flag) {
         // a tile overflowed somewhere in the CTA: exact row maxima first, then the whole pass again
         st.m_ref = -INFINITY;
-        for (int j = par; j < n_tiles; j += kSplit) softmax_step<DH, kMaxOnly>(st, j, n_tiles + j);
+        for (int j = par; j < n_tiles; j += kSplit) softmax_step<C, kMaxOnly>(st, j, n_tiles + j);
         xchg[wtid + par * kBlockM].x = st.m_ref;
         if (tile == 0) asm volatile("bar.sync 1, 256;" ::: "memory");
         else asm volatile("bar.sync 2, 256;" ::: "memory");
         st.m_ref = fmaxf(xchg[wtid].x, xchg[wtid + kBlockM].x);
         st.shift = 0.f;
         st.l_sum = 0.f;
-        for (int j = par; j < n_tiles; j += kSplit) softmax_step<DH, kExact>(st, j, 2 * n_tiles + j);
+        for (int j = par; j < n_tiles; j += kSplit) softmax_step<C, kExact>(st, j, 2 * n_tiles + j);
         wait_bar(st.bar_done, 1, abort_flag, p.err_word);
         if constexpr (C::kOnes) {
             tc_fence_after();
@@ -457,7 +461,7 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     __nv_bfloat16 *dst = nullptr;
     if (tok >= 0 && !*abort_flag) {
         const size_t orow = p.compact ? ((size_t)b * p.M + m) : ((size_t)b * p.N_tok + tok);
-        dst = p.out + (orow * p.H + h) * DH;
+        dst = p.out + (orow * p.H + h) * C::kDH;
         if (p.lse_out && par == 0) {
             const size_t li = p.compact ? (((size_t)b * p.H + h) * p.M + m) : (((size_t)b * p.H + h) * p.N_tok + tok);
             p.lse_out[li] = st.m_ref * p.scale + st.shift * 0.6931471805599453f + logf(l_sum);
@@ -495,18 +499,19 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     }
 }
 
-template <int DH>
-__global__ void __launch_bounds__(Cfg<DH>::kThreads, 1)
+template <class C>
+__global__ void __launch_bounds__(C::kThreads, C::kCtasPerSM)
 sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                    const __grid_constant__ CUtensorMap tmap_k_tail, const __grid_constant__ CUtensorMap tmap_v_tail, const Params p)
 {
-    using C = Cfg<DH>;
+    constexpr int kTilesM = C::kTilesM;
+    constexpr uint32_t kTmemCols = C::kTmemCols;
     constexpr int kSBufs = C::kSBufs, kAhead = C::kAhead;
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ volatile int redo_flag;
-    __shared__ float2 xchg[kTilesM][2 * kBlockM];
+    __shared__ float2 xchg[C::kTilesM][2 * kBlockM];
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -569,9 +574,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         const int wg = warp >> 2;
         const int tile = wg / kSplit, par = wg % kSplit;
         if (tile < q_tiles)
-            softmax_role<DH>(p, bar, tile, par, smem_gen + tile * C::kQTileBytes, tmem, m0 + tile * kBlockM, h, b, n_tiles,
+            softmax_role<C>(p, bar, tile, par, smem_gen + tile * C::kQTileBytes, tmem, m0 + tile * kBlockM, h, b, n_tiles,
                              &abort_flag, &redo_flag, xchg[tile]);
-        else pass_sync<DH>();
+        else pass_sync<C>();
     } else if (warp == kProducerWarp) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
         // ------------------------------------------------ TMA producer (warp-uniform, one elected lane issues)
@@ -617,7 +622,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         };
         produce_pass(kSpeculate);
         int k_loads = n_tiles, v_loads = n_tiles;
-        pass_sync<DH>();
+        pass_sync<C>();
         if (redo_flag) {
             produce_pass(kMaxOnly);
             produce_pass(kExact);
@@ -712,14 +717,14 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             wait_bar(bar.q + 8 * t, 0, &abort_flag, p.err_word);
             issue_pass(kSpeculate);
         }
-        pass_sync<DH>();
+        pass_sync<C>();
         if (redo_flag && t < q_tiles) {
             issue_pass(kMaxOnly);
             issue_pass(kExact);
         }
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
-        pass_sync<DH>();
+        pass_sync<C>();
     }
 
     tc_fence_before();
@@ -762,10 +767,10 @@ int32_t make_kv_map(CUtensorMap *map, const void *base, int B, int H, int N, int
     return ASTRAEA_OK;
 }
 
-template <int DH>
+template <int DH, int TM>
 int32_t launch_dh(const AttnArgs &a, cudaStream_t stream)
 {
-    using C = Cfg<DH>;
+    using C = Cfg<DH, TM>;
     CUtensorMap mk, mv, mkt, mvt;
     int32_t rc = make_kv_map(&mk, a.k, a.B, a.H, a.N, a.d, a.k_sb, a.k_sh, a.k_sn, false, C::kBlockN);
     if (rc != ASTRAEA_OK) return rc;
@@ -780,7 +785,8 @@ int32_t launch_dh(const AttnArgs &a, cudaStream_t stream)
     }
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(sparse_attn_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(sparse_attn_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(sparse_attn_kernel<C>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess)
             return check_launch("astraea_sparse_attn (shared memory attribute)");
         attr_set = true;
     }
@@ -796,8 +802,8 @@ int32_t launch_dh(const AttnArgs &a, cudaStream_t stream)
     p.compact = (a.flags & ASTRAEA_ATTN_COMPACT_OUT) ? 1 : 0;
     p.err_word = a.err_word;
     p.h0 = a.head_begin;
-    dim3 grid((a.M + kTilesM * kBlockM - 1) / (kTilesM * kBlockM), a.head_count > 0 ? a.head_count : a.H, a.B);
-    sparse_attn_kernel<DH><<<grid, C::kThreads, C::kSmemBytes, stream>>>(mk, mv, mkt, mvt, p);
+    dim3 grid((a.M + TM * kBlockM - 1) / (TM * kBlockM), a.head_count > 0 ? a.head_count : a.H, a.B);
+    sparse_attn_kernel<C><<<grid, C::kThreads, C::kSmemBytes, stream>>>(mk, mv, mkt, mvt, p);
     return check_launch("astraea_sparse_attn");
 }
 
@@ -895,12 +901,43 @@ int32_t launch_sparse_attn_noalloc(AttnArgs a, cudaStream_t stream)
     return launch_sparse_attn(a, stream);
 }
 
+// Which CTA shape finishes first.  Large CTAs (two query tiles, one per SM) are dispatched in launch order onto 148
+// SMs; the last one of every (head, batch) is cheaper when it holds one query tile only (0.68 of a full one,
+// measured).  Small CTAs (one query tile, two per SM) all cost the same: `slowdown` times a large one, because two
+// share the SM (measured: 1.05 at head_dim 64, 1.17 at 72).  The difference matters for launches of a few rounds.
+static bool small_ctas_pay(const AttnArgs &a, double slowdown)
+{
+    const long long hb = (long long)(a.head_count > 0 ? a.head_count : a.H) * a.B;
+    const int pairs = (a.M + 2 * kBlockM - 1) / (2 * kBlockM), tiles = (a.M + kBlockM - 1) / kBlockM;
+    const bool light_last = a.M - (pairs - 1) * 2 * kBlockM <= kBlockM;
+    if (hb * pairs > 16 * kNumSMs) return false;                 // many rounds: the granularity does not matter
+    // a denoising loop repeats a few shapes: remember the last answer
+    thread_local long long last_hb = -1;
+    thread_local int last_M = -1;
+    thread_local double last_slowdown = 0.0;
+    thread_local bool last_answer = false;
+    if (hb == last_hb && a.M == last_M && slowdown == last_slowdown) return last_answer;
+    double sm_busy[kNumSMs] = {};
+    for (long long c = 0; c < hb * pairs; ++c) {                 // greedy dispatch in launch order
+        int best = 0;
+        for (int s = 1; s < kNumSMs; ++s) if (sm_busy[s] < sm_busy[best]) best = s;
+        sm_busy[best] += (light_last && c % pairs == pairs - 1) ? 0.68 : 1.0;
+    }
+    double large = 0.0;
+    for (int s = 0; s < kNumSMs; ++s) large = sm_busy[s] > large ? sm_busy[s] : large;
+    const double small = slowdown * (double)((hb * tiles + 2 * kNumSMs - 1) / (2 * kNumSMs));
+    last_hb = hb; last_M = a.M; last_slowdown = slowdown;
+    last_answer = small < 0.97 * large;
+    return last_answer;
+}
+
 int32_t launch_sparse_attn(const AttnArgs &a, cudaStream_t stream)
 {
+    const bool force_small = (a.flags & ASTRAEA_ATTN_SMALL_CTAS) != 0;
     switch (a.d) {
-    case 64: return launch_dh<64>(a, stream);
-    case 72: return launch_dh<72>(a, stream);
-    case 128: return launch_dh<128>(a, stream);
+    case 64: return (force_small || small_ctas_pay(a, 1.05)) ? launch_dh<64, 1>(a, stream) : launch_dh<64, 2>(a, stream);
+    case 72: return (force_small || small_ctas_pay(a, 1.17)) ? launch_dh<72, 1>(a, stream) : launch_dh<72, 2>(a, stream);
+    case 128: return launch_dh<128, 2>(a, stream);
     default: return fail(ASTRAEA_ERR_UNSUPPORTED, "head_dim %d is not supported", a.d);
     }
 }

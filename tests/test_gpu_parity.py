@@ -163,7 +163,7 @@ def test_scatter_with_no_rows_leaves_cache_alone():
 
 
 # ------------------------------------------------------------------ attention
-def _attn_case(oracle, B, H, N, d, M, seed, layout="bnhd", compact=False, dense=False, scale=0.0, amp=1.0):
+def _attn_case(oracle, B, H, N, d, M, seed, layout="bnhd", compact=False, dense=False, scale=0.0, amp=1.0, small_ctas=False):
     rng = np.random.default_rng(seed)
     # amp sharpens the logits only (q, k); values and the cache stay N(0,1)
     q, k, v, cache = (synth.f32_to_bf16_bits((a * rng.standard_normal((B, N, H, d))).astype(np.float32)) for a in (amp, amp, 1.0, 1.0))
@@ -188,7 +188,8 @@ def _attn_case(oracle, B, H, N, d, M, seed, layout="bnhd", compact=False, dense=
         lse = dev(lse_cache0)
     ws = A.new_workspace(A.OP_SPARSE_ATTN, B, H, N, M, d)
     A.astraea_sparse_attn(qd, kd, vd, qs, ks, vs, None if idx is None else dev(idx), M, out, lse, B, H, N, d,
-                          scale=scale, flags=A.ATTN_COMPACT_OUT if compact else 0, workspace=ws)
+                          scale=scale, flags=(A.ATTN_COMPACT_OUT if compact else 0) | (A.ATTN_SMALL_CTAS if small_ctas else 0),
+                          workspace=ws)
     A.astraea_poll_error(ws)
     got = bf16_dev_to_f64(out)
     got_lse = lse.cpu().numpy().astype(np.float64)
@@ -226,6 +227,20 @@ def test_attn_single_tile(oracle, d):
 @pytest.mark.parametrize("N,M", [(300, 77), (1000, 333), (129, 129), (1, 1), (127, 5), (64, 64), (65, 3)])
 def test_attn_ragged_tiles(oracle, d, N, M):
     _attn_case(oracle, 2, 3, N, d, M, seed=2)
+
+
+@pytest.mark.parametrize("d", [64, 72])
+def test_attn_one_query_tile_per_cta_shape(oracle, d):
+    """The CTA shape that the library picks for launches of a few rounds (one 128-row query tile, two CTAs per SM),
+    forced here on small cases: ragged tiles, several CTAs per head, many key tiles (every stage phase), a compact
+    output, and logits that make the CTAs redo their work."""
+    _attn_case(oracle, 2, 3, 300, d, 77, seed=70, small_ctas=True)
+    _attn_case(oracle, 2, 2, 1000, d, 333, seed=71, small_ctas=True)
+    _attn_case(oracle, 1, 2, 64 * 27 + 40, d, 130, seed=72, small_ctas=True)
+    _attn_case(oracle, 2, 2, 400, d, 100, seed=73, compact=True, small_ctas=True)
+    _attn_case(oracle, 1, 2, 129, d, 129, seed=74, dense=True, small_ctas=True)
+    _attn_case(oracle, 1, 2, 900, d, 600, seed=75, amp=12.0, small_ctas=True)
+    _attn_case(oracle, 1, 1, 1, d, 1, seed=76, small_ctas=True)
 
 
 def test_attn_many_key_tiles_exercise_every_stage_phase(oracle):

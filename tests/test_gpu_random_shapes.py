@@ -29,6 +29,7 @@ def test_random_attention_cases(oracle, seed):
         M = rnd.randint(1, N)
         mode = rnd.choice(["self", "self", "cross", "kv"])
         N_kv = rnd.choice([1, 5, 64, 100, 226, 300]) if mode == "cross" else N
+        fl = A.ATTN_SMALL_CTAS if (d != 128 and rnd.random() < 0.4) else 0   # the other CTA shape of head_dim 64 / 72
         sig = rnd.choice([0.0, 0.0, 0.5, 1.0])                       # per-token lognormal norms: heavy-tailed logits
         amp = rnd.choice([1.0, 1.0, 2.0, 12.0])                      # 12: the speculation limit is passed, the CTAs redo
         sq, sk = np.exp(sig * rng.standard_normal((B, N, 1, 1))), np.exp(sig * rng.standard_normal((B, N_kv, 1, 1)))
@@ -46,19 +47,19 @@ def test_random_attention_cases(oracle, seed):
         if mode == "cross":
             ws = A.new_workspace(A.OP_SPARSE_ATTN, B, H, N, M, d)
             A.astraea_sparse_cross_attn(to_dev_bf16(q), to_dev_bf16(k), to_dev_bf16(v), sq_, sk_, sk_, dev(idx), M, out, lse,
-                                        B, H, N, N_kv, d, workspace=ws)
+                                        B, H, N, N_kv, d, flags=fl, workspace=ws)
         elif mode == "kv":
             ws = A.new_workspace(A.OP_SPARSE_ATTN_KV, B, H, N, kv.shape[1], d)
             A.astraea_sparse_attn(to_dev_bf16(q), to_dev_bf16(k), to_dev_bf16(v), sq_, sq_, sq_, dev(idx), M, out, lse, B, H, N, d,
-                                  workspace=ws, kv_idx=dev(kv), M_kv=kv.shape[1])
+                                  flags=fl, workspace=ws, kv_idx=dev(kv), M_kv=kv.shape[1])
         else:
             ws = A.new_workspace(A.OP_SPARSE_ATTN, B, H, N, M, d)
             A.astraea_sparse_attn(to_dev_bf16(q), to_dev_bf16(k), to_dev_bf16(v), sq_, sq_, sq_, dev(idx), M, out, lse, B, H, N, d,
-                                  workspace=ws)
+                                  flags=fl, workspace=ws)
         A.astraea_poll_error(ws)
         got = bf16_dev_to_f64(out)
         rows = np.take_along_axis(got, idx[:, :, None, None].astype(np.int64), 1)
-        case = (d, B, H, N, M, mode, N_kv, sig, amp)
+        case = (d, B, H, N, M, mode, N_kv, sig, amp, fl)
         # one bf16 rounding of the output and of P: absolute for values of order one, relative beyond
         err = np.abs(rows - want_o) / np.maximum(1.0, np.abs(want_o))
         assert err.max() < 2e-2 and err.mean() < 2e-3, (case, err.max(), err.mean())
