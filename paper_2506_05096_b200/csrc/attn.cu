@@ -32,6 +32,10 @@
 // maxima first, then the softmax against them (the accumulator is shared by two warpgroups, so it is not
 // rescaled in place).
 //
+// At head_dim 64 / 72 the kernel also exists with ONE query tile per CTA and two CTAs per SM (half the TMEM, at
+// most 113 KB of shared memory each): per SM that is 5-17 % slower, but its CTAs are half as long, so a launch of
+// only a few rounds of CTAs finishes earlier with it; the launch estimates both and picks.
+//
 // TMEM columns: S/P of (tile t, buffer u) at (kSBufs t + u) * kBlockN; the O accumulators behind them.
 // The producer and issuer warps run warp-uniform code and elect one lane per instruction, so
 // that descriptors and addresses stay in uniform registers (a lone diverged thread issues
