@@ -34,6 +34,7 @@ UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the attention kernel, from the ncu
 # capture summarised in profiles/ (workload -> theta_permille -> bytes); None where not captured.
+NOMINAL_BF16_TFLOPS, NOMINAL_HBM_GBS = 2250.0, 8000.0     # the part's nominal dense bf16 and HBM3e figures, for context
 NCU_TRAFFIC_BYTES = {"cogvideox": {500: 324246784}, "sweep": {250: 1285133616}}
 
 
@@ -259,18 +260,26 @@ def main():
                 "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
                 "peak_kind": "%s burst bf16 (MEASURED_PEAKS.json)" % peaks["source"] if peaks["source"] == "measured"
                 else "fallback burst bf16", "traffic": traffic, "kernel_ms": attn_ms,
-                "min_bytes": accounting.attn_min_bytes(B, H, M, N, d)}
+                "min_bytes": accounting.attn_min_bytes(B, H, M, N, d),
+                # for context only: the nominal dense bf16 figure of the part, and the credit for the rows that were skipped
+                "frac_of_nominal_2250_tflops": achieved / NOMINAL_BF16_TFLOPS,
+                "dense_equivalent_tflops(speed-up credit, not a roofline figure)":
+                    accounting.attn_flops(B, H, N, N, d) / (attn_ms * 1e-3) / 1e12}
     hbm = peaks["hbm_gbs"]
     sb = accounting.score_bytes(B, N, N_sel, D, H)
     cb = accounting.scatter_bytes(B, M, D)
     selb = accounting.select_bytes(B, N_sel, k_keep)
     kernels = {
-        "score": {"ms": float(parts[0]), "GB/s": sb / parts[0] / 1e6, "frac_hbm": sb / parts[0] / 1e6 / hbm},
+        "hbm_peaks_gbs": {"measured": hbm, "nominal": NOMINAL_HBM_GBS},
+        "score": {"ms": float(parts[0]), "GB/s": sb / parts[0] / 1e6, "frac_hbm": sb / parts[0] / 1e6 / hbm,
+                  "frac_hbm_nominal": sb / parts[0] / 1e6 / NOMINAL_HBM_GBS},
         "select": {"ms": float(parts[1]), "GB/s": selb / parts[1] / 1e6, "note": "latency-bound"},
         "score+select": {"ms": float(parts[0] + parts[1]), "GB/s": (sb + selb) / (parts[0] + parts[1]) / 1e6,
-                         "frac_hbm": (sb + selb) / (parts[0] + parts[1]) / 1e6 / hbm},
+                         "frac_hbm": (sb + selb) / (parts[0] + parts[1]) / 1e6 / hbm,
+                         "frac_hbm_nominal": (sb + selb) / (parts[0] + parts[1]) / 1e6 / NOMINAL_HBM_GBS},
         "sparse_attn": {"ms": attn_ms, "TFLOP/s": achieved},
-        "scatter_reuse(x_ref)": {"ms": float(parts[3]), "GB/s": cb / parts[3] / 1e6, "frac_hbm": cb / parts[3] / 1e6 / hbm},
+        "scatter_reuse(x_ref)": {"ms": float(parts[3]), "GB/s": cb / parts[3] / 1e6, "frac_hbm": cb / parts[3] / 1e6 / hbm,
+                                 "frac_hbm_nominal": cb / parts[3] / 1e6 / NOMINAL_HBM_GBS},
     }
 
     sweep = {}
