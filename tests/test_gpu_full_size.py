@@ -135,3 +135,60 @@ def test_cogvideox_shaped_projection_and_cross_attention_full_size(oracle):
     err = np.abs(got_o - want_o)
     assert err.max() < 2e-2 and err.mean() < 2e-3, (err.max(), err.mean())
     assert np.array_equal(bf16_dev_to_f64(out)[unsel], f64(cache.reshape(B, N, H, d))[unsel])
+
+
+def test_hunyuan_shaped_consecutive_steps_full_size(oracle):
+    """Steps 0 and 1 of the drifting-latent workload at the full HunyuanVideo shape: step 0 computes every token and
+    fills the output and LSE caches from real data; step 1 (keep-ratio 0.6) is checked with the oracle started from the
+    device's state after step 0 (scores from the device's LSE cache, selection on the device's scores, sampled
+    attention rows, reuse of step 0's outputs bit for bit, refresh of x_ref where selected)."""
+    w = synth.WORKLOADS["hunyuan"]
+    inp = synth.make_step_inputs(w, 3)
+    B, N, H, d, D, N_sel = w.B, w.N, w.H, w.d, w.D, w.N_v
+    rng = np.random.default_rng(4)
+    x0, q0, k0, v0 = inp["x_cur"], inp["q"], inp["k"], inp["v"]
+    x1 = synth.drift_step(x0, 901, 0.05, False)
+    q1, k1, v1 = (synth.drift_step(a, 902 + i, 0.05, True) for i, a in enumerate((q0, k0, v0)))
+    x_ref = to_dev_bf16(x0)                                   # no earlier step: the reference inputs are the first ones
+    out = torch.zeros(B, N, H, d, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros(B, H, N, device="cuda")
+    n_skip = torch.zeros(B, N_sel, dtype=torch.int32, device="cuda")
+    score = torch.empty(B, N_sel, device="cuda")
+    idx_sel = torch.empty(B, N, dtype=torch.int32, device="cuda")
+    idx_rem = torch.empty(B, N_sel, dtype=torch.int32, device="cuda")
+    ws = A.new_workspace(A.OP_STEP, B, H, N, N, d)
+    w_alpha = 1.0 / N
+    A.astraea_step(to_dev_bf16(x0), x_ref, lse, n_skip, to_dev_bf16(q0), to_dev_bf16(k0), to_dev_bf16(v0), out, score,
+                   idx_sel, idx_rem, B, H, N, N_sel, d, N_sel, w_alpha=w_alpha, workspace=ws)
+    A.astraea_poll_error(ws)
+    out0, lse0 = out.clone(), lse.clone()
+    # step 0, sampled: dense attention rows and their LSE
+    heads = [0, H - 1]
+    pick0 = np.sort(rng.choice(N, 16, replace=False)).astype(np.int32)[None]
+    want_o, want_l, _ = oracle.sparse_attn(*(f64(np.ascontiguousarray(a[:, :, heads])) for a in (q0, k0, v0)), q_idx=pick0)
+    got = np.take_along_axis(out0[:, :, heads].float().cpu().numpy().astype(np.float64), pick0[:, :, None, None].astype(np.int64), 1)
+    assert np.abs(got - want_o).max() < 2e-2
+    assert np.abs(np.take_along_axis(lse0[:, heads].cpu().numpy().astype(np.float64), pick0[:, None, :].astype(np.int64), 2) - want_l).max() < 1e-3
+    # step 1
+    k_keep = w.k_of(600)
+    A.astraea_step(to_dev_bf16(x1), x_ref, lse, n_skip, to_dev_bf16(q1), to_dev_bf16(k1), to_dev_bf16(v1), out, score,
+                   idx_sel, idx_rem, B, H, N, N_sel, d, k_keep, w_alpha=w_alpha, workspace=ws)
+    A.astraea_poll_error(ws)
+    got_score = score.cpu().numpy()
+    pick = np.sort(rng.choice(N_sel, 2048, replace=False))
+    want_s = oracle.score(f64(x1[:, pick]), f64(x0[:, pick]), lse0.cpu().numpy()[:, :, pick], np.zeros((B, len(pick)), np.int32),
+                          n_sel=len(pick), w_alpha=w_alpha)
+    assert (np.abs(got_score[:, pick].astype(np.float64) - want_s) / np.abs(want_s)).max() < 1e-5
+    want_sel, want_rem, want_n = oracle.select(got_score, k_keep, 0, np.zeros((B, N_sel), np.int32))
+    got_sel = idx_sel.cpu().numpy()[:, :k_keep] if B == 1 else None
+    assert np.array_equal(got_sel, want_sel)
+    assert np.array_equal(n_skip.cpu().numpy(), want_n)
+    rows = np.sort(rng.choice(want_sel[0], 16, replace=False)).astype(np.int32)[None]
+    want_o, want_l, _ = oracle.sparse_attn(*(f64(np.ascontiguousarray(a[:, :, heads])) for a in (q1, k1, v1)), q_idx=rows)
+    got = np.take_along_axis(out[:, :, heads].float().cpu().numpy().astype(np.float64), rows[:, :, None, None].astype(np.int64), 1)
+    assert np.abs(got - want_o).max() < 2e-2
+    unsel = torch.ones(B, N, dtype=torch.bool, device="cuda")
+    unsel[0, idx_sel[0, :k_keep].long()] = False
+    assert torch.equal(out[unsel], out0[unsel]) and torch.equal(lse.transpose(1, 2)[unsel], lse0.transpose(1, 2)[unsel])
+    x1d, x0d = to_dev_bf16(x1), to_dev_bf16(x0)
+    assert torch.equal(x_ref[unsel], x0d[unsel]) and torch.equal(x_ref[~unsel], x1d[~unsel])
