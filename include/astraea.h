@@ -272,7 +272,7 @@ void    astraea_schedule_destroy(astraea_schedule *schedule);
  * (x_ref, LSE cache, counters, output cache) and staging buffers, and each step copies
  * the HOST inputs to the device, runs the step (score, select, refresh of x_ref,
  * sparse attention) and copies the merged output back.  The copies run on streams of
- * their own: x_cur goes first, q / k / v follow in four groups of heads, the attention
+ * their own: x_cur goes first, q / k / v follow in up to twelve groups of heads, the attention
  * of a group starts when its heads have arrived, and the group's columns of the output
  * go back while the next group is computed.  The results are those of astraea_step.
  * astraea_session_create allocates device memory (cudaMalloc) on the current device;
