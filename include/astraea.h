@@ -38,7 +38,8 @@ extern "C" {
 #define ASTRAEA_ERR_WORKSPACE_TOO_SMALL  -3
 #define ASTRAEA_ERR_CUDA                 -4  /* a CUDA call or launch failed                                      */
 #define ASTRAEA_ERR_TIMEOUT              -5  /* a bounded device-side wait gave up (seen by astraea_poll_error)   */
-#define ASTRAEA_ERR_BAD_INDEX            -6  /* an index list was out of range or not strictly ascending          */
+#define ASTRAEA_ERR_BAD_INDEX            -6  /* an index list held an entry out of range or not strictly ascending
+                                              * (found on the device; reported by astraea_poll_error)           */
 
 #define ASTRAEA_N_SKIP_CLAMP 80              /* counters saturate here so that e^n stays finite in fp32 */
 
@@ -116,7 +117,9 @@ int32_t astraea_select(const float *score, int B, int N_sel, int k, int n_always
  *   q, k, v : bf16, head_dim contiguous; element strides (batch, head, token) given per tensor.
  *             [B,N,H,d] has strides (N*H*d, d, H*d); [B,H,N,d] has (H*N*d, N*d, d).
  *             Token strides must be multiples of 8 elements, bases 16-byte aligned.
- *   q_idx   : int32 [B, M] strictly ascending token indices in [0,N); NULL => rows 0..M-1
+ *   q_idx   : int32 [B, M] strictly ascending token indices in [0,N); NULL => rows 0..M-1.  An entry out of
+ *             range, or one that does not exceed its predecessor (a duplicate, a descending step), is never
+ *             dereferenced or written: its row is skipped and astraea_poll_error reports BAD_INDEX.
  *   kv_idx  : NULL (all keys: the paper's method), or int32 [B, M_kv] token indices in [0,N): the softmax then
  *             runs over the listed keys/values only (the SelectQ&K variant of the paper's ablation study, Table 2).  Their
  *             rows are gathered into the workspace first, which must then hold
@@ -164,15 +167,17 @@ int32_t astraea_sparse_cross_attn(const void *q, const void *k, const void *v,
  * process whose device memory has been handed out in full to other owners.  This entry point keeps
  * its scratch in a fixed array inside the library image instead (ASTRAEA_NOALLOC_SCRATCH_BYTES per
  * GPU that loads the library, held until the process exits) and calls no cudaMalloc, cudaFree or
- * other allocating routine.  Arguments, arithmetic and results are those of astraea_sparse_attn
- * without the workspace pair.
- *   - Problems whose scratch need (astraea_workspace_bytes(ASTRAEA_OP_SPARSE_ATTN, ...)) exceeds
- *     ASTRAEA_NOALLOC_SCRATCH_BYTES are rejected with ASTRAEA_ERR_WORKSPACE_TOO_SMALL.
+ * other allocating routine.  Arguments (flags included), validation, arithmetic and results are those of
+ * astraea_sparse_attn without the workspace pair: the two entry points share one code path.
+ *   - Problems whose scratch need (astraea_workspace_bytes(ASTRAEA_OP_SPARSE_ATTN, ...), or
+ *     ASTRAEA_OP_SPARSE_ATTN_KV with kv_idx) exceeds ASTRAEA_NOALLOC_SCRATCH_BYTES are rejected with
+ *     ASTRAEA_ERR_WORKSPACE_TOO_SMALL.  With kv_idx that is nearly always the case: the gathered key / value
+ *     rows (2 * B * M_kv * H * d bf16) must fit the array.
  *   - The first call on a device resolves the array's device address (with that device current);
  *     make that first call before any stream capture.
  *   - All calls on a device share the one array.  It keeps the last call's contents, so each call
- *     first clears the part it uses on `stream`; calls that overlap on the GPU (different streams)
- *     race on it and must be serialised by the caller.
+ *     first clears its error word on `stream` (also a call that is then rejected for its arguments); calls
+ *     that overlap on the GPU (different streams) race on it and must be serialised by the caller.
  *   - The error word lives in that array, so astraea_poll_error cannot be pointed at it: a device-side
  *     timeout or bad index in this variant is not reported.  Callers that need the report use
  *     astraea_sparse_attn.
@@ -193,11 +198,17 @@ int32_t astraea_sparse_attn_noalloc(const void *q, const void *k, const void *v,
  *     cache[b, idx[b,r], :] = rows[b, idx[b,r], :] with ASTRAEA_SCATTER_SRC_FULL;
  * every row that is not listed is left untouched, i.e. keeps the earlier step's value.
  * The second form refreshes the reference inputs of the tokens that were computed.
- *   cache : bf16 [B, N, row_elems], in place      rows : bf16     idx : int32 [B, M], in [0,N), no duplicates
+ *   cache : bf16 [B, N, row_elems], in place      rows : bf16
+ *   idx   : int32 [B, M], strictly ascending in [0,N).  An entry out of range or not above its predecessor is
+ *           skipped (nothing is written outside the cache, no row is written twice).
+ *   err_workspace : NULL, or any workspace of this library (at least 4 bytes, 4-byte aligned): its first word is
+ *           the error word, and a skipped entry is then reported as BAD_INDEX by astraea_poll_error.  With NULL
+ *           such entries are skipped without a report.
  * M = 0 is valid.  Errors: INVALID_ARG (row_elems % 8 != 0, misaligned pointers, ...), CUDA.
  */
 int32_t astraea_scatter_reuse(void *cache, const void *rows, const int32_t *idx,
-                              int B, int N, int M, int row_elems, uint32_t flags, void *stream);
+                              int B, int N, int M, int row_elems, uint32_t flags,
+                              void *err_workspace, void *stream);
 
 /*
  * A linear layer of the compute block on the selected tokens only (Algorithm 1 lines 4-5: the query
@@ -207,7 +218,7 @@ int32_t astraea_scatter_reuse(void *cache, const void *rows, const int32_t *idx,
  * and every row of y that is not listed is left untouched, i.e. keeps the cached result of the earlier
  * step.  The gather of the rows of x and the scatter of the rows of y are fused into the GEMM.
  *   x    : bf16 [B, N, K] (with ASTRAEA_LINEAR_COMPACT_IN bf16 [B, M, K])
- *   idx  : int32 [B, M] in [0,N), no duplicates; NULL => all N rows (M ignored)
+ *   idx  : int32 [B, M] strictly ascending in [0,N); NULL => all N rows (M ignored)
  *   w    : bf16 [N_out, K] row-major (out features x in features)        bias : bf16 [N_out] or NULL
  *   y    : bf16 [B, N, N_out], rows at idx written in place; with ASTRAEA_LINEAR_COMPACT_OUT bf16 [B, M, N_out]
  *   workspace : at least astraea_workspace_bytes(ASTRAEA_OP_GATHERED_LINEAR, 0, 0, 0, 0, 0) bytes, 256-byte
@@ -216,7 +227,8 @@ int32_t astraea_scatter_reuse(void *cache, const void *rows, const int32_t *idx,
  * activations of the MLP exist for the selected rows only.
  * bf16 operands, fp32 accumulation (and fp32 GELU), one rounding to bf16 at the end.  K must be a multiple of 64, N_out
  * a multiple of 8; x, w, y 16-byte aligned.  M = 0 is valid (nothing is launched).  An index outside
- * [0,N) is not dereferenced: its row is skipped and astraea_poll_error reports BAD_INDEX.
+ * [0,N), or one that does not exceed its predecessor, is not dereferenced: its row is skipped and
+ * astraea_poll_error reports BAD_INDEX.
  * Errors: INVALID_ARG, UNSUPPORTED (unknown flags), WORKSPACE_TOO_SMALL, CUDA.
  */
 int32_t astraea_gathered_linear(const void *x, const int32_t *idx, int M, const void *w, const void *bias,

@@ -26,7 +26,9 @@
  * softmax rows sum to 1; closed forms for zero keys, constant values, a dominant
  * key, constant per-token differences, the round-robin penalty schedule;
  * permutation invariances; half-normal drift statistics; the linear layer on listed rows
- * vs a library matmul, a one-hot weight, a zero weight and pure-Python brute force.
+ * vs a library matmul, a one-hot weight, a zero weight and pure-Python brute force; the
+ * LSE scatter vs numpy indexing; a whole step at a partial budget (computed rows vs the
+ * dense library attention, cached rows / LSE / reference inputs untouched elsewhere).
  * parity unpinned: absolute score values under the paper's own (unpublished)
  * w_alpha, w_beta and its intended reading of [R1]-[R4].
  */
@@ -228,7 +230,6 @@ void oracle_scatter_lse(double *lse_cache, const double *lse_rows, const int32_t
                     lse_rows[((size_t)b * H + h) * M + r];
 }
 
-/* floor(theta * N_sel) in integer arithmetic from a permille budget [R9]. */
 /*
  * Linear layer on the selected rows (Algorithm 1 lines 4-5 and Section 3.2, "the same strategy
  * applies to the other layers of the block"): y[b, i, :] = x[b, i, :] W^T + bias for the listed
@@ -258,6 +259,7 @@ void oracle_gathered_linear(const double *x, const int32_t *idx, int M, const do
         }
 }
 
+/* floor(theta * N_sel) in integer arithmetic from a permille budget [R9]. */
 int oracle_budget_to_k(int n_sel, int theta_permille)
 {
     return (int)(((int64_t)n_sel * theta_permille) / 1000);

@@ -168,12 +168,16 @@ def scatter_lse(lse_cache, lse_rows, idx):
 
 
 def step(x_cur, x_ref, lse_cache, n_skip, q, k, v, cache, k_keep, n_always=0,
-         w_alpha=1.0, w_beta=1.0, delta_mode=0, lse_mode=0, scale=0.0):
+         w_alpha=1.0, w_beta=1.0, delta_mode=0, lse_mode=0, scale=0.0, forced_sel=None):
     """One attention block at one denoising step (Algorithm 1), all in fp64.
 
     Returns a dict with score (fp64), score_f32, idx_sel, idx_rem, n_skip (new),
     out (new cache, [B,N,H,d]), lse (new lse cache, [B,H,N]), x_ref (refreshed at
     the selected tokens: the "last computed" reference).
+
+    forced_sel [B, k_keep + n_always] (ascending; tests only): the rest of the step runs on this selection
+    instead of the oracle's own (a chained test hands over a selection that differs from the oracle's only at
+    exact near-ties of the k-th score, after having checked that); `own_idx_sel` then holds the oracle's.
     """
     B, N = x_cur.shape[:2]
     n_sel = N - n_always
@@ -181,6 +185,17 @@ def step(x_cur, x_ref, lse_cache, n_skip, q, k, v, cache, k_keep, n_always=0,
                 delta_mode=delta_mode, lse_mode=lse_mode)
     s32 = s64.astype(np.float32)
     idx_sel, idx_rem, n_new = select(s32, k_keep, n_always, n_skip)
+    own = idx_sel
+    if forced_sel is not None:
+        idx_sel = _i32(forced_sel)
+        assert idx_sel.shape == own.shape
+        chosen = np.zeros((B, N), dtype=bool)
+        for b in range(B):
+            chosen[b, idx_sel[b]] = True
+        idx_rem = np.stack([np.flatnonzero(~chosen[b, :n_sel]) for b in range(B)]).astype(np.int32)
+        if n_skip is not None:
+            n_old = np.asarray(n_skip, dtype=np.int64)
+            n_new = np.where(chosen[:, :n_sel], 0, np.minimum(n_old + 1, 80)).astype(np.int32)
     if idx_sel.shape[1]:
         o, l, _ = sparse_attn(q, k, v, q_idx=idx_sel, scale=scale)
         out = scatter_reuse(cache, o, idx_sel)
@@ -191,4 +206,4 @@ def step(x_cur, x_ref, lse_cache, n_skip, q, k, v, cache, k_keep, n_always=0,
         lse_new = np.array(lse_cache, dtype=np.float64, copy=True)
         xr = np.array(x_ref, dtype=np.float64, copy=True)
     return dict(score=s64, score_f32=s32, idx_sel=idx_sel, idx_rem=idx_rem, n_skip=n_new,
-                out=out, lse=lse_new, x_ref=xr)
+                out=out, lse=lse_new, x_ref=xr, own_idx_sel=own)

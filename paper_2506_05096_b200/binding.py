@@ -62,7 +62,7 @@ def lib() -> ctypes.CDLL:
                                                                                c_i, c_i, c_i, c_i, c_i, c_f, c_u, c_p, c_sz, c_p]
         L.astraea_sparse_attn_noalloc.argtypes = [c_p, c_p, c_p] + [c_i64] * 9 + [c_p, c_i, c_p, c_i, c_p, c_p,
                                                                                  c_i, c_i, c_i, c_i, c_f, c_u, c_p]
-        L.astraea_scatter_reuse.argtypes = [c_p, c_p, c_p, c_i, c_i, c_i, c_i, c_u, c_p]
+        L.astraea_scatter_reuse.argtypes = [c_p, c_p, c_p, c_i, c_i, c_i, c_i, c_u, c_p, c_p]
         L.astraea_gathered_linear.argtypes = [c_p, c_p, c_i, c_p, c_p, c_p, c_i, c_i, c_i, c_i, c_u, c_p, c_sz, c_p]
         L.astraea_step.argtypes = [c_p] * 11 + [c_i] * 6 + [c_f, c_f, c_i, c_i, c_p, c_sz, c_p]
         L.astraea_schedule_create.argtypes = [ctypes.POINTER(c_p), c_i, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p,
@@ -165,8 +165,10 @@ def astraea_sparse_cross_attn(q, k, v, q_strides, k_strides, v_strides, q_idx, M
                                            _ptr(workspace), workspace.numel() if workspace is not None else 0, _stream(stream)))
 
 
-def astraea_scatter_reuse(cache, rows, idx, B, N, M, row_elems, flags=0, stream=None) -> None:
-    _check(lib().astraea_scatter_reuse(_ptr(cache), _ptr(rows), _ptr(idx), B, N, M, row_elems, flags, _stream(stream)))
+def astraea_scatter_reuse(cache, rows, idx, B, N, M, row_elems, flags=0, workspace=None, stream=None) -> None:
+    """workspace (optional): any workspace tensor; bad index entries are then reported by astraea_poll_error."""
+    _check(lib().astraea_scatter_reuse(_ptr(cache), _ptr(rows), _ptr(idx), B, N, M, row_elems, flags,
+                                       _ptr(workspace), _stream(stream)))
 
 
 def astraea_gathered_linear(x, idx, M, w, bias, y, B, N, K, N_out, flags=0, workspace=None, stream=None) -> None:

@@ -34,6 +34,30 @@ int32_t check_launch(const char *what) {
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+void *tensor_map_encoder() {
+    static void *const fn = [] {                   // function-local static: initialised once, thread-safe
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            ptr = nullptr;
+        return ptr;
+    }();
+    return fn;
+}
+
+int sm_count() {
+    static int cached[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 148;
+    int n = __atomic_load_n(&cached[dev], __ATOMIC_RELAXED);
+    if (n > 0) return n;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+    if (n > kMaxSMs) n = kMaxSMs;
+    __atomic_store_n(&cached[dev], n, __ATOMIC_RELAXED);
+    return n;
+}
+
 }  // namespace astraea
 
 using namespace astraea;
@@ -170,38 +194,20 @@ int32_t astraea_sparse_attn_noalloc(const void *q, const void *k, const void *v,
                                     void *out, float *lse_out,
                                     int B, int H, int N, int d, float scale, uint32_t flags, void *stream)
 {
-    (void)M_kv;
-    REQUIRE(B > 0 && H > 0 && N > 0 && d > 0, "astraea_sparse_attn_noalloc: B, H, N, d must be positive");
-    REQUIRE(M >= 0 && M <= N, "astraea_sparse_attn_noalloc: M=%d outside [0, N=%d]", M, N);
-    if (d != 64 && d != 72 && d != 128)
-        return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_sparse_attn_noalloc: head_dim %d not in {64, 72, 128}", d);
-    if (kv_idx) return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_sparse_attn_noalloc: kv_idx (select-Q-and-K ablation) is not built");
-    if (flags & ~ASTRAEA_ATTN_COMPACT_OUT) return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_sparse_attn_noalloc: unknown flags 0x%x", flags);
-    REQUIRE(q && k && v && out, "astraea_sparse_attn_noalloc: null q, k, v or out");
-    REQUIRE(aligned16(q) && aligned16(k) && aligned16(v) && aligned16(out), "astraea_sparse_attn_noalloc: q, k, v, out must be 16-byte aligned");
-    REQUIRE(q_sn % 8 == 0 && k_sn % 8 == 0 && v_sn % 8 == 0 && q_sh % 8 == 0 && k_sh % 8 == 0 && v_sh % 8 == 0 &&
-            q_sb % 8 == 0 && k_sb % 8 == 0 && v_sb % 8 == 0,
-            "astraea_sparse_attn_noalloc: strides must be multiples of 8 elements (16 bytes)");
-    REQUIRE(q_sn >= d && k_sn >= d && v_sn >= d && q_sh > 0 && k_sh > 0 && v_sh > 0 && q_sb >= 0 && k_sb >= 0 && v_sb >= 0,
-            "astraea_sparse_attn_noalloc: strides must be positive and token stride >= head_dim");
-    REQUIRE(scale >= 0.f, "astraea_sparse_attn_noalloc: scale must be >= 0 (0 selects 1/sqrt(d))");
-    if (M == 0) return ASTRAEA_OK;
-    AttnArgs a;
-    a.q = q; a.k = k; a.v = v;
-    a.q_sb = q_sb; a.q_sh = q_sh; a.q_sn = q_sn;
-    a.k_sb = k_sb; a.k_sh = k_sh; a.k_sn = k_sn;
-    a.v_sb = v_sb; a.v_sh = v_sh; a.v_sn = v_sn;
-    a.q_idx = q_idx; a.M = M; a.out = out; a.lse_out = lse_out;
-    a.B = B; a.H = H; a.N = N; a.d = d;
-    a.scale = (scale == 0.f) ? 1.0f / sqrtf((float)d) : scale;
-    a.flags = flags;
-    a.err_word = nullptr;
-    a.N_tok = N;
-    return launch_sparse_attn_noalloc(a, (cudaStream_t)stream);
+    // the scratch is the library's own fixed array: resolve its address on this device (first call: set-up), clear
+    // the error word the last call may have left, then run the ordinary entry with it as the workspace
+    void *scratch = nullptr;
+    int32_t rc = noalloc_scratch_address(&scratch);
+    if (rc != ASTRAEA_OK) return rc;
+    cudaError_t e = cudaMemsetAsync(scratch, 0, 256, (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_sparse_attn_noalloc: clearing the scratch failed: %s", cudaGetErrorString(e));
+    return sparse_attn_entry("astraea_sparse_attn_noalloc", 0, q, k, v, q_sb, q_sh, q_sn, k_sb, k_sh, k_sn, v_sb, v_sh, v_sn,
+                             q_idx, M, kv_idx, M_kv, out, lse_out, B, H, N, d, scale, flags, scratch,
+                             ASTRAEA_NOALLOC_SCRATCH_BYTES, stream);
 }
 
 int32_t astraea_scatter_reuse(void *cache, const void *rows, const int32_t *idx,
-                              int B, int N, int M, int row_elems, uint32_t flags, void *stream)
+                              int B, int N, int M, int row_elems, uint32_t flags, void *err_workspace, void *stream)
 {
     REQUIRE(B > 0 && N > 0 && row_elems > 0, "astraea_scatter_reuse: B, N, row_elems must be positive");
     REQUIRE(M >= 0 && M <= N, "astraea_scatter_reuse: M=%d outside [0, N=%d]", M, N);
@@ -210,7 +216,8 @@ int32_t astraea_scatter_reuse(void *cache, const void *rows, const int32_t *idx,
     if (M == 0) return ASTRAEA_OK;
     REQUIRE(cache && rows && idx, "astraea_scatter_reuse: null cache, rows or idx");
     REQUIRE(aligned16(cache) && aligned16(rows), "astraea_scatter_reuse: cache / rows must be 16-byte aligned");
-    return launch_scatter(cache, rows, idx, B, N, M, row_elems, flags, (cudaStream_t)stream);
+    REQUIRE((reinterpret_cast<uintptr_t>(err_workspace) & 3u) == 0, "astraea_scatter_reuse: err_workspace must be 4-byte aligned");
+    return launch_scatter(cache, rows, idx, B, N, M, row_elems, flags, reinterpret_cast<int *>(err_workspace), (cudaStream_t)stream);
 }
 
 int32_t astraea_gathered_linear(const void *x, const int32_t *idx, int M, const void *w, const void *bias,
@@ -264,7 +271,7 @@ int32_t astraea_step(const void *x_cur, void *x_ref, float *lse_cache, int32_t *
                              lse_cache, B, H, N, d, 0.f, 0u, ws, attn_ws, stream);
     if (rc != ASTRAEA_OK) return rc;
     // the reference inputs of the tokens that were computed become the current inputs
-    return astraea_scatter_reuse(x_ref, x_cur, idx_sel, B, N, M, D, ASTRAEA_SCATTER_SRC_FULL, stream);
+    return astraea_scatter_reuse(x_ref, x_cur, idx_sel, B, N, M, D, ASTRAEA_SCATTER_SRC_FULL, ws, stream);
 }
 
 int32_t astraea_poll_error(void *workspace, void *stream)
@@ -276,7 +283,7 @@ int32_t astraea_poll_error(void *workspace, void *stream)
     if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_poll_error: %s", cudaGetErrorString(e));
     if (word != 0) cudaMemset(workspace, 0, sizeof(int));
     if (word == kErrTimeout) return fail(ASTRAEA_ERR_TIMEOUT, "a bounded device-side wait gave up");
-    if (word == kErrBadIndex) return fail(ASTRAEA_ERR_BAD_INDEX, "an index was out of range");
+    if (word == kErrBadIndex) return fail(ASTRAEA_ERR_BAD_INDEX, "an index list held an entry out of range or not strictly ascending");
     return ASTRAEA_OK;
 }
 
@@ -468,7 +475,7 @@ int32_t astraea_step_host(astraea_session *s, const void *x_cur, const void *q, 
         rc = astraea_select(s->score, B, N_sel, k_keep, n_always, s->idx_sel, s->idx_rem, s->n_skip, ws + attn_ws,
                             s->workspace_bytes - attn_ws, s->stream);
     if (rc == ASTRAEA_OK)
-        rc = astraea_scatter_reuse(s->x_ref, s->x_cur, s->idx_sel, B, N, M, D, ASTRAEA_SCATTER_SRC_FULL, s->stream);
+        rc = astraea_scatter_reuse(s->x_ref, s->x_cur, s->idx_sel, B, N, M, D, ASTRAEA_SCATTER_SRC_FULL, s->workspace, s->stream);
     if (rc != ASTRAEA_OK) return rc;
     for (int g = 0; g < groups; ++g) {
         e = cudaStreamWaitEvent(s->stream, s->ev_in[g], 0);

@@ -404,7 +404,11 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     int tok = -1;
     if (m < p.M) {
         tok = p.q_idx ? __ldg(p.q_idx + (size_t)b * p.M + m) : m;
-        if ((unsigned)tok >= (unsigned)p.N_tok) { if (par == 0) atomicExch(p.err_word, kErrBadIndex); tok = -1; }
+        // an entry out of range, or one that does not exceed its predecessor (two rows would race on one output
+        // row), is reported and its row is not written
+        const bool bad = (unsigned)tok >= (unsigned)p.N_tok ||
+                         (p.q_idx && m > 0 && __ldg(p.q_idx + (size_t)b * p.M + m - 1) >= tok);
+        if (bad) { if (par == 0 && p.err_word) atomicExch(p.err_word, kErrBadIndex); tok = -1; }
     }
 
     st.m_ref = -INFINITY;
@@ -741,17 +745,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-EncodeTiledFn get_encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void *ptr = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(ptr);
-    }
-    return fn;
-}
+EncodeTiledFn get_encode_fn() { return reinterpret_cast<EncodeTiledFn>(tensor_map_encoder()); }
 
 // K or V as a 4-D tensor (d, N, H, B) with 128-byte-swizzled boxes of 64 columns x 128 tokens
 int32_t make_kv_map(CUtensorMap *map, const void *base, int B, int H, int N, int d,
@@ -787,13 +781,14 @@ int32_t launch_dh(const AttnArgs &a, cudaStream_t stream)
         rc = make_kv_map(&mvt, a.v, a.B, a.H, a.N, a.d, a.v_sb, a.v_sh, a.v_sn, true, C::kBlockN);
         if (rc != ASTRAEA_OK) return rc;
     }
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(sparse_attn_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess ||
-            cudaFuncSetAttribute(sparse_attn_kernel<C>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess)
-            return check_launch("astraea_sparse_attn (shared memory attribute)");
-        attr_set = true;
-    }
+    static PerDeviceOnce attrs;                   // one per kernel instantiation; the attributes are per device
+    if (attrs.run([] {
+            cudaError_t e = cudaFuncSetAttribute(sparse_attn_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+            if (e == cudaSuccess)
+                e = cudaFuncSetAttribute(sparse_attn_kernel<C>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+            return e;
+        }) != cudaSuccess)
+        return check_launch("astraea_sparse_attn (shared memory attribute)");
     Params p;
     p.q = reinterpret_cast<const __nv_bfloat16 *>(a.q);
     p.q_sb = a.q_sb; p.q_sh = a.q_sh; p.q_sn = a.q_sn;
@@ -851,7 +846,8 @@ int32_t launch_sparse_attn_kv(AttnArgs a, const int32_t *kv_idx, int M_kv, void 
     uint4 *kc = reinterpret_cast<uint4 *>(ws + 256), *vc = reinterpret_cast<uint4 *>(ws + 256 + one);
     const int vec = a.d / 8;
     const long long total = (long long)a.B * M_kv * a.H * vec;
-    const int grid = (int)((total + 255) / 256 < (long long)kNumSMs * 16 ? (total + 255) / 256 : (long long)kNumSMs * 16);
+    const long long cap = (long long)sm_count() * 16;
+    const int grid = (int)((total + 255) / 256 < cap ? (total + 255) / 256 : cap);
     gather_kv_kernel<<<grid, 256, 0, stream>>>(kc, reinterpret_cast<const __nv_bfloat16 *>(a.k), a.k_sb, a.k_sh, a.k_sn,
                                                kv_idx, a.B, a.H, a.N, M_kv, vec, a.err_word);
     gather_kv_kernel<<<grid, 256, 0, stream>>>(vc, reinterpret_cast<const __nv_bfloat16 *>(a.v), a.v_sb, a.v_sh, a.v_sn,
@@ -871,38 +867,25 @@ int32_t launch_sparse_attn_kv(AttnArgs a, const int32_t *kv_idx, int M_kv, void 
 // the symbol, never a device address: the address comes from cudaGetSymbolAddress, per device.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[ASTRAEA_NOALLOC_SCRATCH_BYTES];
 
-int32_t launch_sparse_attn_noalloc(AttnArgs a, cudaStream_t stream)
+int32_t noalloc_scratch_address(void **scratch_out)
 {
-    const size_t need = attn_workspace_bytes(a.B, a.H, a.N, a.M, a.d);
-    if (need > ASTRAEA_NOALLOC_SCRATCH_BYTES)
-        return fail(ASTRAEA_ERR_WORKSPACE_TOO_SMALL,
-                    "astraea_sparse_attn_noalloc: this problem needs %zu bytes of scratch, the built-in scratch holds %d; "
-                    "use astraea_sparse_attn with a caller workspace", need, ASTRAEA_NOALLOC_SCRATCH_BYTES);
     // one-time set-up per device (with that device current): resolve the symbol to its device address
-    constexpr int kMaxDevices = 64;
     static void *scratch_of_device[kMaxDevices] = {};
     static std::mutex mu;
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices)
         return fail(ASTRAEA_ERR_CUDA, "astraea_sparse_attn_noalloc: no usable current device (%s)", cudaGetErrorString(e));
-    void *scratch = nullptr;
-    {
-        std::lock_guard<std::mutex> lock(mu);
-        if (!scratch_of_device[dev]) {
-            void *ptr = nullptr;
-            e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
-            if (e != cudaSuccess || !ptr)
-                return fail(ASTRAEA_ERR_CUDA, "astraea_sparse_attn_noalloc: cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
-            scratch_of_device[dev] = ptr;
-        }
-        scratch = scratch_of_device[dev];
+    std::lock_guard<std::mutex> lock(mu);
+    if (!scratch_of_device[dev]) {
+        void *ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+        if (e != cudaSuccess || !ptr)
+            return fail(ASTRAEA_ERR_CUDA, "astraea_sparse_attn_noalloc: cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
+        scratch_of_device[dev] = ptr;
     }
-    // the array keeps what the last call left: the error word must start at zero
-    e = cudaMemsetAsync(scratch, 0, need, stream);
-    if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_sparse_attn_noalloc: clearing the scratch failed: %s", cudaGetErrorString(e));
-    a.err_word = reinterpret_cast<int *>(scratch);
-    return launch_sparse_attn(a, stream);
+    *scratch_out = scratch_of_device[dev];
+    return ASTRAEA_OK;
 }
 
 // Which CTA shape finishes first.  Large CTAs (two query tiles, one per SM) are dispatched in launch order onto 148
@@ -914,22 +897,23 @@ static bool small_ctas_pay(const AttnArgs &a, double slowdown)
     const long long hb = (long long)(a.head_count > 0 ? a.head_count : a.H) * a.B;
     const int pairs = (a.M + 2 * kBlockM - 1) / (2 * kBlockM), tiles = (a.M + kBlockM - 1) / kBlockM;
     const bool light_last = a.M - (pairs - 1) * 2 * kBlockM <= kBlockM;
-    if (hb * pairs > 16 * kNumSMs) return false;                 // many rounds: the granularity does not matter
+    const int n_sm = sm_count();
+    if (hb * pairs > 16 * n_sm) return false;                    // many rounds: the granularity does not matter
     // a denoising loop repeats a few shapes: remember the last answer
     thread_local long long last_hb = -1;
     thread_local int last_M = -1;
     thread_local double last_slowdown = 0.0;
     thread_local bool last_answer = false;
     if (hb == last_hb && a.M == last_M && slowdown == last_slowdown) return last_answer;
-    double sm_busy[kNumSMs] = {};
+    double sm_busy[kMaxSMs] = {};
     for (long long c = 0; c < hb * pairs; ++c) {                 // greedy dispatch in launch order
         int best = 0;
-        for (int s = 1; s < kNumSMs; ++s) if (sm_busy[s] < sm_busy[best]) best = s;
+        for (int s = 1; s < n_sm; ++s) if (sm_busy[s] < sm_busy[best]) best = s;
         sm_busy[best] += (light_last && c % pairs == pairs - 1) ? 0.68 : 1.0;
     }
     double large = 0.0;
-    for (int s = 0; s < kNumSMs; ++s) large = sm_busy[s] > large ? sm_busy[s] : large;
-    const double small = slowdown * (double)((hb * tiles + 2 * kNumSMs - 1) / (2 * kNumSMs));
+    for (int s = 0; s < n_sm; ++s) large = sm_busy[s] > large ? sm_busy[s] : large;
+    const double small = slowdown * (double)((hb * tiles + 2 * n_sm - 1) / (2 * n_sm));
     last_hb = hb; last_M = a.M; last_slowdown = slowdown;
     last_answer = small < 0.97 * large;
     return last_answer;

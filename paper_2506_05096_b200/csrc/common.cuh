@@ -10,9 +10,35 @@
 
 namespace astraea {
 
-constexpr int kNumSMs = 148;            // B200: 2 dies x 74 SMs
+constexpr int kMaxSMs = 256;            // upper bound for per-SM host tables (a full B200 has 2 dies x 74 = 148)
+constexpr int kMaxDevices = 64;         // per-device host state is kept for device ordinals below this
 constexpr int kErrTimeout = 1;          // values of the device-side error word
 constexpr int kErrBadIndex = 2;
+
+// SMs of the current device (cudaDevAttrMultiProcessorCount, read once per device; a part with SMs fused off
+// reports fewer than 148 and every grid is sized from this).  148 if the query fails.
+int sm_count();
+
+// Runs `f` once per device (the current one) and remembers the devices on which it returned cudaSuccess:
+// cudaFuncSetAttribute and the like apply to the current device only.  Thread-safe.
+class PerDeviceOnce {
+public:
+    template <class F> cudaError_t run(F &&f) {
+        int dev = -1;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= kMaxDevices) return f();            // no slot: just do it every time
+        if (__atomic_load_n(&done_[dev], __ATOMIC_ACQUIRE)) return cudaSuccess;
+        e = f();                                                   // idempotent: two racing threads may both run it
+        if (e == cudaSuccess) __atomic_store_n(&done_[dev], 1, __ATOMIC_RELEASE);
+        return e;
+    }
+private:
+    int done_[kMaxDevices] = {};
+};
+
+// cuTensorMapEncodeTiled from the driver (looked up once, thread-safe); nullptr if the driver does not have it
+void *tensor_map_encoder();
 
 // thread-local text of the last failure
 void set_error(const char *fmt, ...);
@@ -29,7 +55,7 @@ int32_t launch_select(const float *score, int B, int N_sel, int k, int n_always,
                       int32_t *idx_rem, int32_t *n_skip, void *workspace, cudaStream_t stream);
 size_t select_workspace_bytes(int B, int N_sel);
 int32_t launch_scatter(void *cache, const void *rows, const int32_t *idx, int B, int N, int M,
-                       int row_elems, uint32_t flags, cudaStream_t stream);
+                       int row_elems, uint32_t flags, int *err_word, cudaStream_t stream);
 
 size_t linear_workspace_bytes();
 int32_t launch_gathered_linear(const void *x, const int32_t *idx, int M, const void *w, const void *bias, void *y,
@@ -51,8 +77,8 @@ struct AttnArgs {
 };
 int32_t launch_sparse_attn(const AttnArgs &a, cudaStream_t stream);
 size_t attn_workspace_bytes(int B, int H, int N, int M, int d);
-int32_t launch_sparse_attn_noalloc(AttnArgs a, cudaStream_t stream);
+int32_t noalloc_scratch_address(void **scratch_out);   // device address of the library's built-in scratch array on the current device
 size_t attn_kv_workspace_bytes(int B, int H, int M_kv, int d);
-int32_t launch_sparse_attn_kv(AttnArgs a, const int32_t *kv_idx, int M_kv, void *workspace, cudaStream_t stream);   // scratch in a static device array
+int32_t launch_sparse_attn_kv(AttnArgs a, const int32_t *kv_idx, int M_kv, void *workspace, cudaStream_t stream);   // gathers the listed K/V rows into the workspace first
 
 }  // namespace astraea

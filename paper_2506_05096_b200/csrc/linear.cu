@@ -71,12 +71,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *m, 
 }
 
 // row of x that holds the g-th listed row (all batch elements in one list): -1 past the end, -2 for an index
-// outside [0, N); *out_row is the row of y it goes to
+// outside [0, N) or one that does not exceed its predecessor; *out_row is the row of y it goes to
 __device__ __forceinline__ long long source_row(const LinParams &p, long long g, long long total, long long *out_row) {
     if (g >= total) return -1;
     const int b = (int)(g / p.M), r = (int)(g - (long long)b * p.M);
     const int tok = p.idx ? __ldg(p.idx + g) : r;
     if ((unsigned)tok >= (unsigned)p.N) return -2;
+    if (p.idx && r > 0 && __ldg(p.idx + g - 1) >= tok) return -2;      // not strictly ascending: a row would be written twice
     if (out_row) *out_row = p.compact ? g : (long long)b * p.N + tok;
     return p.compact_in ? g : (long long)b * p.N + tok;
 }
@@ -263,15 +264,8 @@ size_t linear_workspace_bytes() { return 256; }
 int32_t launch_gathered_linear(const void *x, const int32_t *idx, int M, const void *w, const void *bias, void *y,
                                int B, int N, int K, int N_out, uint32_t flags, int *err_word, cudaStream_t stream)
 {
-    static EncodeTiledFn enc = nullptr;
-    if (!enc) {
-        void *ptr = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            enc = reinterpret_cast<EncodeTiledFn>(ptr);
-        if (!enc) return fail(ASTRAEA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
-    }
+    const EncodeTiledFn enc = reinterpret_cast<EncodeTiledFn>(tensor_map_encoder());
+    if (!enc) return fail(ASTRAEA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
     // W as a 2-D tensor (K, N_out) with 128-byte-swizzled boxes of 64 columns x 256 rows
     CUtensorMap mw;
     cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)N_out};
@@ -282,12 +276,9 @@ int32_t launch_gathered_linear(const void *x, const int32_t *idx, int M, const v
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(ASTRAEA_ERR_INVALID_ARG, "astraea_gathered_linear: tensor map of W rejected (CUresult %d)", (int)r);
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(gathered_linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
-            return check_launch("astraea_gathered_linear (shared memory attribute)");
-        attr_set = true;
-    }
+    static PerDeviceOnce attrs;                   // the attribute is per device
+    if (attrs.run([] { return cudaFuncSetAttribute(gathered_linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes); }) != cudaSuccess)
+        return check_launch("astraea_gathered_linear (shared memory attribute)");
     LinParams p;
     p.x = reinterpret_cast<const __nv_bfloat16 *>(x);
     p.idx = idx;
@@ -301,7 +292,8 @@ int32_t launch_gathered_linear(const void *x, const int32_t *idx, int M, const v
     p.err_word = err_word;
     const long long rows = (long long)B * p.M;
     const long long tiles = ((rows + kBM - 1) / kBM) * ((N_out + kBN - 1) / kBN);
-    const int grid = (int)(tiles < kNumSMs ? tiles : kNumSMs);
+    const int n_sm = sm_count();
+    const int grid = (int)(tiles < n_sm ? tiles : n_sm);
     gathered_linear_kernel<<<grid, kThreads, kSmemBytes, stream>>>(mw, p);
     return check_launch("astraea_gathered_linear");
 }

@@ -21,7 +21,7 @@ __device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
 
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 scatter_kernel(uint4 *__restrict__ cache, const uint4 *__restrict__ rows, const int32_t *__restrict__ idx,
-               int B, int N, int M, int vec_per_row, int src_full)
+               int B, int N, int M, int vec_per_row, int src_full, int *__restrict__ err_word)
 {
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -31,7 +31,12 @@ scatter_kernel(uint4 *__restrict__ cache, const uint4 *__restrict__ rows, const 
         const int b = (int)(t / M);
         const int r = (int)(t - (long long)b * M);
         const int i = __ldg(idx + t);
-        if ((unsigned)i >= (unsigned)N) continue;           // never write outside the cache
+        // never write outside the cache, and never write a row twice: an entry that is out of range or does not
+        // exceed its predecessor is skipped and reported
+        if ((unsigned)i >= (unsigned)N || (r > 0 && __ldg(idx + t - 1) >= i)) {
+            if (lane == 0 && err_word) atomicExch(err_word, kErrBadIndex);
+            continue;
+        }
         const uint4 *src = rows + ((size_t)b * (src_full ? N : M) + (src_full ? i : r)) * vec_per_row;
         uint4 *dst = cache + ((size_t)b * N + i) * vec_per_row;
         for (int v = lane; v < vec_per_row; v += 32 * kUnroll) {
@@ -47,15 +52,16 @@ scatter_kernel(uint4 *__restrict__ cache, const uint4 *__restrict__ rows, const 
 }  // namespace
 
 int32_t launch_scatter(void *cache, const void *rows, const int32_t *idx, int B, int N, int M,
-                       int row_elems, uint32_t flags, cudaStream_t stream)
+                       int row_elems, uint32_t flags, int *err_word, cudaStream_t stream)
 {
     const long long total = (long long)B * M;
     if (total == 0) return ASTRAEA_OK;
     long long want = (total + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    int grid = (int)(want < (long long)kNumSMs * kBlocksPerSM ? want : (long long)kNumSMs * kBlocksPerSM);
+    const long long cap = (long long)sm_count() * kBlocksPerSM;
+    int grid = (int)(want < cap ? want : cap);
     scatter_kernel<<<grid, kWarpsPerBlock * 32, 0, stream>>>(
         reinterpret_cast<uint4 *>(cache), reinterpret_cast<const uint4 *>(rows), idx, B, N, M,
-        row_elems >> 3, (flags & ASTRAEA_SCATTER_SRC_FULL) ? 1 : 0);
+        row_elems >> 3, (flags & ASTRAEA_SCATTER_SRC_FULL) ? 1 : 0, err_word);
     return check_launch("astraea_scatter_reuse");
 }
 

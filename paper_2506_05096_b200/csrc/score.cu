@@ -112,7 +112,8 @@ int32_t launch_score(const void *x_cur, const void *x_ref, const float *lse, con
     const long long total = (long long)B * N_sel;
     if (total == 0) return ASTRAEA_OK;
     long long want = (total + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    int grid = (int)(want < (long long)kNumSMs * kBlocksPerSM ? want : (long long)kNumSMs * kBlocksPerSM);
+    const long long cap = (long long)sm_count() * kBlocksPerSM;
+    int grid = (int)(want < cap ? want : cap);
     const uint4 *xc = reinterpret_cast<const uint4 *>(x_cur);
     const uint4 *xr = reinterpret_cast<const uint4 *>(x_ref);
     dim3 block(kWarpsPerBlock * 32);

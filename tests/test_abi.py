@@ -63,9 +63,9 @@ def test_argument_errors_are_reported_before_any_launch(L):
     assert L.astraea_sparse_attn(*args(64, wsb=8)) == binding.ERR_WORKSPACE_TOO_SMALL
     assert L.astraea_sparse_attn(*args(64, qsn=60)) == binding.ERR_INVALID_ARG
     assert L.astraea_sparse_attn(*args(64, ws=ctypes.c_void_p(0x1010))) == binding.ERR_INVALID_ARG
-    assert L.astraea_scatter_reuse(p, p, p, 1, 16, 4, 12, 0, None) == binding.ERR_INVALID_ARG
-    assert L.astraea_scatter_reuse(p, p, p, 1, 16, 17, 16, 0, None) == binding.ERR_INVALID_ARG
-    assert L.astraea_scatter_reuse(p, p, p, 1, 16, 0, 16, 0, None) == binding.OK     # M = 0: nothing to do
+    assert L.astraea_scatter_reuse(p, p, p, 1, 16, 4, 12, 0, None, None) == binding.ERR_INVALID_ARG
+    assert L.astraea_scatter_reuse(p, p, p, 1, 16, 17, 16, 0, None, None) == binding.ERR_INVALID_ARG
+    assert L.astraea_scatter_reuse(p, p, p, 1, 16, 0, 16, 0, None, None) == binding.OK     # M = 0: nothing to do
     assert L.astraea_poll_error(None, None) == binding.ERR_INVALID_ARG
 
 

@@ -9,7 +9,7 @@ import torch
 
 from paper_2506_05096_b200 import binding as A
 from paper_2506_05096_b200 import synth
-from helpers import bf16_dev_to_f64, dev, f64, to_dev_bf16
+from helpers import assert_attn_close, bf16_dev_to_f64, dev, f64, to_dev_bf16
 
 pytestmark = pytest.mark.gpu
 
@@ -61,11 +61,11 @@ def test_random_attention_cases(oracle, seed):
         rows = np.take_along_axis(got, idx[:, :, None, None].astype(np.int64), 1)
         case = (d, B, H, N, M, mode, N_kv, sig, amp, fl)
         # one bf16 rounding of the output and of P: absolute for values of order one, relative beyond
-        err = np.abs(rows - want_o) / np.maximum(1.0, np.abs(want_o))
-        assert err.max() < 2e-2 and err.mean() < 2e-3, (case, err.max(), err.mean())
+        assert_attn_close(rows, want_o, what=case)
         got_lse = np.take_along_axis(lse.cpu().numpy().astype(np.float64), idx[:, None, :].astype(np.int64), 2)
-        # head_dim 64 sums the bf16-rounded probabilities on the tensor core: 2^-8 relative at worst (one dominant key)
-        lse_tol = 5e-3 if d == 64 else 1e-3
+        # head_dim 64 sums the bf16-rounded probabilities on the tensor core: 2^-8 relative at worst, where one key
+        # dominates a row (sharpened or heavy-tailed logits only); everything else keeps the 1e-3 bound
+        lse_tol = 5e-3 if (d == 64 and (amp > 1.0 or sig > 0.0)) else 1e-3
         assert (np.abs(got_lse - want_lse) / np.maximum(1.0, np.abs(want_lse))).max() < lse_tol, case
         mask = np.ones((B, N), bool)
         for b in range(B):

@@ -182,6 +182,97 @@ def test_full_step_at_keep_ratio_one_is_dense_attention(oracle):
     assert np.array_equal(res["x_ref"], x)
 
 
+def test_scatter_lse_matches_numpy_fancy_indexing(oracle):
+    """The LSE cache is [B, H, N] and its compact rows [B, H, M]: with B > 1, H > 1, M != H and N != M*H a
+    transposed or mis-strided index lands somewhere numpy's own indexing does not."""
+    rng = np.random.default_rng(21)
+    B, H, N, M = 3, 4, 19, 7
+    cache = _rand(rng, B, H, N)
+    rows = _rand(rng, B, H, M)
+    idx = np.stack([np.sort(rng.choice(N, M, replace=False)) for _ in range(B)]).astype(np.int32)
+    got = oracle.scatter_lse(cache, rows, idx)
+    want = cache.copy()
+    for b in range(B):
+        want[b][:, idx[b]] = rows[b]
+    assert np.array_equal(got, want)
+    assert not np.array_equal(got, cache)
+    # unsorted index lists are placed the same way (the scatter does not rely on the order)
+    perm = rng.permutation(M)
+    assert np.array_equal(oracle.scatter_lse(cache, rows[:, :, perm], idx[:, perm]), want)
+    # no rows: the cache comes back untouched
+    assert np.array_equal(oracle.scatter_lse(cache, np.empty((B, H, 0)), np.empty((B, 0), np.int32)), cache)
+
+
+def test_step_at_a_partial_budget_merges_computed_and_cached_state(oracle):
+    """Algorithm 1 lines 6-7 and the execution flow of Section 3.2 at 0 < k < N, with always-kept tokens and
+    B, H > 1: the selected tokens carry the dense library attention's rows and LSE, every other token keeps the
+    cached output and LSE bit for bit; the reference inputs are refreshed at the selected tokens ONLY; the
+    selection itself is the brute-force top-k of the scores, which are retyped here from the equations."""
+    rng = np.random.default_rng(22)
+    B, N_v, N_t, H, d = 2, 23, 3, 3, 8
+    N, k_keep = N_v + N_t, 9
+    x_ref = _rand(rng, B, N, H * d)
+    x_cur = x_ref + 0.3 * _rand(rng, B, N, H * d)
+    q, k, v, cache = (_rand(rng, B, N, H, d) for _ in range(4))
+    lse_cache = 0.5 * _rand(rng, B, H, N)
+    n0 = rng.integers(0, 3, (B, N_v)).astype(np.int32)
+    w_a, w_b = 2.0, 0.25
+    res = oracle.step(x_cur, x_ref, lse_cache, n0, q, k, v, cache, k_keep, n_always=N_t, w_alpha=w_a, w_beta=w_b)
+    # scores and selection from the definitions
+    s_ref = (w_a * np.exp(lse_cache).mean(1)[:, :N_v] * np.abs(x_cur - x_ref).mean(-1)[:, :N_v] + w_b * np.exp(n0))
+    assert np.abs(res["score"] - s_ref).max() < 1e-12 * np.abs(s_ref).max()
+    s32 = s_ref.astype(np.float32)
+    tq, tk, tv = (torch.from_numpy(a).permute(0, 2, 1, 3) for a in (q, k, v))
+    dense = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv).permute(0, 2, 1, 3).numpy()
+    dense_lse = np.log(np.exp(np.einsum("bihc,bjhc->bhij", q, k) / math.sqrt(d)).sum(-1))       # [B, H, N]
+    for b in range(B):
+        top, rest = _brute_select(list(map(float, s32[b])), k_keep)
+        sel = top + list(range(N_v, N))
+        assert list(res["idx_sel"][b]) == sel and list(res["idx_rem"][b]) == rest
+        unsel = np.setdiff1d(np.arange(N), sel)
+        assert len(unsel) == N_v - k_keep
+        # computed rows / cached rows of the output and of the LSE cache
+        assert np.abs(res["out"][b, sel] - dense[b, sel]).max() < 1e-12
+        assert np.array_equal(res["out"][b, unsel], cache[b, unsel])
+        assert np.abs(res["lse"][b][:, sel] - dense_lse[b][:, sel]).max() < 1e-12
+        assert np.array_equal(res["lse"][b][:, unsel], lse_cache[b][:, unsel])
+        # the cached values really differ from the computed ones, so the two branches cannot be confused
+        assert np.abs(cache[b, unsel] - dense[b, unsel]).min() > 0 and np.abs(lse_cache[b][:, unsel] - dense_lse[b][:, unsel]).min() > 0
+        # reference inputs: current inputs where computed, untouched elsewhere
+        assert np.array_equal(res["x_ref"][b, sel], x_cur[b, sel])
+        assert np.array_equal(res["x_ref"][b, unsel], x_ref[b, unsel])
+        assert np.abs(x_cur[b, unsel] - x_ref[b, unsel]).min() > 0
+        # counters
+        want_n = n0[b] + 1
+        want_n[top] = 0
+        assert np.array_equal(res["n_skip"][b], want_n)
+
+
+def test_step_with_a_forced_selection_only_swaps_the_selection(oracle):
+    """forced_sel (used by the chained GPU tests at near-ties): forcing the oracle's own selection changes nothing;
+    forcing another one moves exactly the rows, the remainder list and the counters that follow from it."""
+    rng = np.random.default_rng(23)
+    B, N, H, d, k_keep = 1, 12, 2, 4, 5
+    x_ref = _rand(rng, B, N, H * d)
+    x_cur = x_ref + _rand(rng, B, N, H * d)
+    q, k, v, cache = (_rand(rng, B, N, H, d) for _ in range(4))
+    lse = _rand(rng, B, H, N)
+    n0 = rng.integers(0, 3, (B, N)).astype(np.int32)
+    own = oracle.step(x_cur, x_ref, lse, n0, q, k, v, cache, k_keep)
+    same = oracle.step(x_cur, x_ref, lse, n0, q, k, v, cache, k_keep, forced_sel=own["idx_sel"])
+    for key in ("idx_sel", "idx_rem", "n_skip", "out", "lse", "x_ref"):
+        assert np.array_equal(own[key], same[key]), key
+    forced = np.array([[0, 3, 4, 7, 11]], np.int32)
+    res = oracle.step(x_cur, x_ref, lse, n0, q, k, v, cache, k_keep, forced_sel=forced)
+    rest = [i for i in range(N) if i not in forced[0]]
+    assert list(res["idx_rem"][0]) == rest and np.array_equal(res["own_idx_sel"], own["idx_sel"])
+    assert (res["n_skip"][0, forced[0]] == 0).all() and np.array_equal(res["n_skip"][0, rest], n0[0, rest] + 1)
+    dense, dense_lse, _ = oracle.sparse_attn(q, k, v)
+    assert np.array_equal(res["out"][0, forced[0]], dense[0, forced[0]]) and np.array_equal(res["out"][0, rest], cache[0, rest])
+    assert np.array_equal(res["lse"][0][:, forced[0]], dense_lse[0][:, forced[0]]) and np.array_equal(res["lse"][0][:, rest], lse[0][:, rest])
+    assert np.array_equal(res["x_ref"][0, forced[0]], x_cur[0, forced[0]]) and np.array_equal(res["x_ref"][0, rest], x_ref[0, rest])
+
+
 # -------------------------------------------------------------- selection pins
 def _brute_select(s, k):
     order = sorted(range(len(s)), key=lambda i: (-(s[i] if not math.isnan(s[i]) else -math.inf), i))
