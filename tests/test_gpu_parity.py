@@ -169,7 +169,7 @@ def test_scatter_reports_and_skips_bad_index_entries():
     B, N, M, R = 1, 32, 7, 64
     cache = torch.zeros(B, N, R, dtype=torch.bfloat16, device="cuda")
     rows = (torch.arange(1, M + 1, device="cuda").float()[None, :, None].expand(B, M, R)).bfloat16().contiguous()
-    idx = torch.tensor([[3, 5, 5, 4, 9, 32, 31]], dtype=torch.int32, device="cuda")     # dup 5, descending 4, 32 out of range
+    idx = torch.tensor([[3, 5, 5, 4, 9, 31, 32]], dtype=torch.int32, device="cuda")     # dup 5, descending 4, 32 out of range
     ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
     g = Guarded((B, N, R), torch.bfloat16, init=cache)
     A.astraea_scatter_reuse(g.t, rows, idx, B, N, M, R, workspace=ws)
@@ -179,7 +179,7 @@ def test_scatter_reports_and_skips_bad_index_entries():
     g.check("scatter with bad entries")
     got = g.t.float()[0, :, 0].cpu().numpy()
     want = np.zeros(N)
-    want[3], want[5], want[9], want[31] = 1, 2, 5, 7          # rows 3 (the second 5), 4 (the 4) and 6 (the 32) are skipped
+    want[3], want[5], want[9], want[31] = 1, 2, 5, 6          # rows 2 (the second 5), 3 (the 4) and 6 (the 32) are skipped
     assert np.array_equal(got, want)
     # without a workspace the same entries are skipped silently
     g2 = Guarded((B, N, R), torch.bfloat16, init=cache)
