@@ -42,6 +42,7 @@ extern "C" {
                                               * (found on the device; reported by astraea_poll_error)           */
 
 #define ASTRAEA_N_SKIP_CLAMP 80              /* counters saturate here so that e^n stays finite in fp32 */
+#define ASTRAEA_LSE_CLAMP    80              /* ASTRAEA_LSE_SUM_EXP: log values above this count as this, for the same reason */
 
 /* delta_mode of astraea_score: how the per-token input difference is reduced over channels */
 #define ASTRAEA_DELTA_MEAN_ABS    0          /* default reading: mean absolute difference */
@@ -78,6 +79,8 @@ extern "C" {
  * the softmax normaliser of the token's attention row from an earlier step, carried in
  * log domain and averaged over heads as lse_mode says; n_i counts the consecutive steps
  * in which token i was not selected (values above ASTRAEA_N_SKIP_CLAMP count as the clamp).
+ * With ASTRAEA_LSE_SUM_EXP a log value above ASTRAEA_LSE_CLAMP counts as the clamp as well: e^lse of such a row
+ * (one logit of 80 or more) would overflow fp32 and turn the scores of a whole batch row into inf / NaN.
  *   x_cur, x_ref : bf16 [B, N, D]                 lse    : fp32 [B, H, N]; NULL => S_LSE = 1
  *   n_skip       : int32 [B, N_sel]; NULL => 0    score  : out fp32 [B, N_sel]
  * Arithmetic: bf16 inputs, fp32 accumulation and result.

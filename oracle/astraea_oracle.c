@@ -13,7 +13,9 @@
  *   [R1] Delta_token is the mean ABSOLUTE difference over channels (modes for the
  *        squared and the signed mean exist as well).
  *   [R3] the "LSE score" is carried as ln(sum exp) and turned back into the sum
- *        of exponentials at scoring time (mode 1 uses the log value itself).
+ *        of exponentials at scoring time (mode 1 uses the log value itself).  The
+ *        paper's sum of exponentials has no bound, fp32 has: a log value above 80
+ *        counts as 80 (as for n_i in [R8]), so that the fp32 scores stay finite.
  *   [R4] per-head LSE scores are averaged over heads.
  *   [R8] n_i is reset to 0 when token i is selected, incremented otherwise, and
  *        clamped to 80 so that e^{n_i} stays finite in fp32.
@@ -38,6 +40,7 @@
 #include <string.h>
 
 #define ORACLE_N_CLAMP 80
+#define ORACLE_LSE_CLAMP 80.0
 
 /* ------------------------------------------------------------------ score
  * Selection metric, Eq. for S_token = w_a * S_sig + w_b * S_penalty with
@@ -71,6 +74,7 @@ void oracle_score(const double *x_cur, const double *x_ref, const double *lse,
                 double a = 0.0;
                 for (int h = 0; h < H; ++h) {
                     double l = lse[((size_t)b * H + h) * N + i];
+                    if (lse_mode == 0 && l > ORACLE_LSE_CLAMP) l = ORACLE_LSE_CLAMP;      /* [R3] */
                     a += (lse_mode == 0) ? exp(l) : l;
                 }
                 s_lse = a / (double)H;

@@ -1,9 +1,9 @@
 // astraea_score: S_token = w_alpha * S_LSE * Delta_token + w_beta * e^{n}
 // (selection-metric equations of Section 3.2; Algorithm 1 lines 1-2).
 //
-// HBM-bound: 2 * D bf16 per token are read once.  One warp owns one token row and
-// streams it with 16-byte loads, six per tensor in flight per lane; the channel reduction is a
-// per-lane fp32 partial sum followed by a warp shuffle tree.  The per-head LSE values of
+// HBM-bound: 2 * D bf16 per token are read once.  One warp (half or a quarter of one for narrow
+// rows) owns one token row and streams it with 16-byte loads, six per tensor in flight per lane; the
+// channel reduction is a per-lane fp32 partial sum followed by a shuffle tree.  The per-head LSE values of
 // the token (a strided gather of H floats, 1/d of the traffic) are averaged by the same
 // warp.  The grid is a multiple of the SM count and walks the tokens with a grid stride.
 #include "common.cuh"
@@ -42,36 +42,47 @@ __device__ __forceinline__ float accum_vec(const uint4 &a, const uint4 &b, float
     return acc;
 }
 
-template <int MODE>
+// LPR lanes share one token row: 32 for rows of 64 or more 16-byte vectors; 16 or 8 for narrower ones, so that no lane
+// of a warp is left without loads.  (Splitting the 144-vector rows of the Open-Sora shape over half-warps was
+// measured and is slower than a whole warp per row, 33.8 against 31.8 us: what bounds the kernel there is its fixed
+// launch / ramp / tail time of ~5 us on 25 us of streaming, not the load slots.)
+template <int MODE, int LPR>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 score_kernel(const uint4 *__restrict__ x_cur, const uint4 *__restrict__ x_ref,
              const float *__restrict__ lse, const int32_t *__restrict__ n_skip,
              float *__restrict__ score, int B, int N, int N_sel, int D, int H,
              float w_alpha, float w_beta, int lse_mode)
 {
+    // a kernel launched behind this one with programmatic stream serialization (the selection) may become resident
+    // and set itself up as soon as SMs free up; it still waits for this whole grid before it reads the scores
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    constexpr int kRowsPerWarp = 32 / LPR;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
+    const int sub = lane / LPR, sl = lane % LPR;          // which of the warp's rows, and the lane within that row
     const int vec_per_row = D >> 3;                       // 16-byte vectors per row
     const long long total = (long long)B * N_sel;
     const float inv_D = 1.0f / (float)D;
     const float inv_H = 1.0f / (float)H;
 
-    for (long long t = (long long)blockIdx.x * kWarpsPerBlock + warp; t < total;
-         t += (long long)gridDim.x * kWarpsPerBlock) {
-        const int b = (int)(t / N_sel);
-        const int i = (int)(t - (long long)b * N_sel);
+    for (long long t0 = ((long long)blockIdx.x * kWarpsPerBlock + warp) * kRowsPerWarp; t0 < total;
+         t0 += (long long)gridDim.x * kWarpsPerBlock * kRowsPerWarp) {
+        const long long t = t0 + sub;
+        const bool have = t < total;
+        const int b = have ? (int)(t / N_sel) : 0;
+        const int i = have ? (int)(t - (long long)b * N_sel) : 0;
         const size_t row = ((size_t)b * N + i) * vec_per_row;
         const uint4 *pc = x_cur + row;
         const uint4 *pr = x_ref + row;
 
         float acc0 = 0.f, acc1 = 0.f;
-        for (int v = lane; v < vec_per_row; v += 32 * kUnroll) {
+        for (int v = sl; have && v < vec_per_row; v += LPR * kUnroll) {
             uint4 a[kUnroll], r[kUnroll];
             // loads past the end of the row are skipped; zeros add nothing in any of the three reductions
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) a[u] = (v + 32 * u < vec_per_row) ? ld_stream(pc + v + 32 * u) : make_uint4(0, 0, 0, 0);
+            for (int u = 0; u < kUnroll; ++u) a[u] = (v + LPR * u < vec_per_row) ? ld_stream(pc + v + LPR * u) : make_uint4(0, 0, 0, 0);
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) r[u] = (v + 32 * u < vec_per_row) ? ld_stream(pr + v + 32 * u) : make_uint4(0, 0, 0, 0);
+            for (int u = 0; u < kUnroll; ++u) r[u] = (v + LPR * u < vec_per_row) ? ld_stream(pr + v + LPR * u) : make_uint4(0, 0, 0, 0);
 #pragma unroll
             for (int u = 0; u < kUnroll; u += 2) {
                 acc0 = accum_vec<MODE>(a[u], r[u], acc0);
@@ -80,20 +91,21 @@ score_kernel(const uint4 *__restrict__ x_cur, const uint4 *__restrict__ x_ref,
         }
         float acc = acc0 + acc1;
 
-        // S_LSE: mean over heads of exp(lse[b,h,i]) (or of lse itself)
+        // S_LSE: mean over heads of exp(lse[b,h,i]) (or of lse itself); the log value is clamped like the skip
+        // counters so that the exponential stays finite in fp32
         float ls = 0.f;
-        if (lse != nullptr) {
-            for (int h = lane; h < H; h += 32) {
+        if (lse != nullptr && have) {
+            for (int h = sl; h < H; h += LPR) {
                 float l = __ldg(lse + ((size_t)b * H + h) * N + i);
-                ls += (lse_mode == ASTRAEA_LSE_SUM_EXP) ? expf(l) : l;
+                ls += (lse_mode == ASTRAEA_LSE_SUM_EXP) ? expf(fminf(l, (float)ASTRAEA_LSE_CLAMP)) : l;
             }
         }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
+        for (int o = LPR / 2; o > 0; o >>= 1) {
             acc += __shfl_xor_sync(0xffffffffu, acc, o);
             ls += __shfl_xor_sync(0xffffffffu, ls, o);
         }
-        if (lane == 0) {
+        if (sl == 0 && have) {
             float delta = acc * inv_D;
             float s_lse = (lse != nullptr) ? ls * inv_H : 1.0f;
             int n = (n_skip != nullptr) ? n_skip[(size_t)b * N_sel + i] : 0;
@@ -101,6 +113,16 @@ score_kernel(const uint4 *__restrict__ x_cur, const uint4 *__restrict__ x_ref,
             score[(size_t)b * N_sel + i] = w_alpha * (s_lse * delta) + w_beta * expf((float)n);
         }
     }
+}
+
+template <int MODE>
+void launch_mode(int lpr, int grid, cudaStream_t stream, const uint4 *xc, const uint4 *xr, const float *lse, const int32_t *n_skip,
+                 float *score, int B, int N, int N_sel, int D, int H, float w_alpha, float w_beta, int lse_mode)
+{
+    dim3 block(kWarpsPerBlock * 32);
+    if (lpr == 32) score_kernel<MODE, 32><<<grid, block, 0, stream>>>(xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode);
+    else if (lpr == 16) score_kernel<MODE, 16><<<grid, block, 0, stream>>>(xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode);
+    else score_kernel<MODE, 8><<<grid, block, 0, stream>>>(xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode);
 }
 
 }  // namespace
@@ -111,21 +133,23 @@ int32_t launch_score(const void *x_cur, const void *x_ref, const float *lse, con
 {
     const long long total = (long long)B * N_sel;
     if (total == 0) return ASTRAEA_OK;
-    long long want = (total + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const int vec_per_row = D >> 3;
+    const int lpr = vec_per_row >= 64 ? 32 : vec_per_row >= 32 ? 16 : 8;     // lanes per row: every lane gets at least two vectors
+    const long long rows_per_block = (long long)kWarpsPerBlock * (32 / lpr);
+    long long want = (total + rows_per_block - 1) / rows_per_block;
     const long long cap = (long long)sm_count() * kBlocksPerSM;
     int grid = (int)(want < cap ? want : cap);
     const uint4 *xc = reinterpret_cast<const uint4 *>(x_cur);
     const uint4 *xr = reinterpret_cast<const uint4 *>(x_ref);
-    dim3 block(kWarpsPerBlock * 32);
     switch (delta_mode) {
     case ASTRAEA_DELTA_MEAN_ABS:
-        score_kernel<ASTRAEA_DELTA_MEAN_ABS><<<grid, block, 0, stream>>>(xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode);
+        launch_mode<ASTRAEA_DELTA_MEAN_ABS>(lpr, grid, stream, xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode);
         break;
     case ASTRAEA_DELTA_MEAN_SQ:
-        score_kernel<ASTRAEA_DELTA_MEAN_SQ><<<grid, block, 0, stream>>>(xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode);
+        launch_mode<ASTRAEA_DELTA_MEAN_SQ>(lpr, grid, stream, xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode);
         break;
     default:
-        score_kernel<ASTRAEA_DELTA_MEAN_SIGNED><<<grid, block, 0, stream>>>(xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode);
+        launch_mode<ASTRAEA_DELTA_MEAN_SIGNED>(lpr, grid, stream, xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode);
         break;
     }
     return check_launch("astraea_score");

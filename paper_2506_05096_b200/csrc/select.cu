@@ -7,13 +7,20 @@
 // ascending token order with a block-wide prefix scan (no atomics on output positions), so
 // equal scores go to the lower index, and updates the skip counters.
 //
-// Rows of up to 131072 tokens are handled by one thread-block cluster per batch row (up to 8
-// CTAs x 1024 threads): every thread keeps its 4, 8 or 16 consecutive keys in registers, so the
-// scores are read from memory exactly once; the per-CTA histograms are summed into the first CTA's
-// shared memory with remote (DSMEM) atomics and every CTA searches the summed histogram itself; the
-// CTAs exchange their selected counts the same way to place their outputs.  Cluster barriers are
-// hardware barriers (no spinning).  Longer rows fall back to one CTA that re-reads the row from L2
-// in every pass.  The call is latency-bound, not bandwidth-bound, at the sizes of the workloads.
+// Rows of up to 131072 tokens are handled by one thread-block cluster per batch row (up to 8 CTAs x 1024
+// threads): every thread keeps its 2, 4, 8 or 16 consecutive keys in registers, so the scores are read from
+// memory exactly once.  The digits are 12, 12 and 8 bits wide; per pass every CTA histograms its live keys in
+// shared memory, adds its non-zero counts into EVERY CTA's copy of the cluster histogram with remote (DSMEM)
+// atomics and, after one hardware cluster barrier, searches its own copy with all its threads.  The search
+// stops as soon as the bin that holds the k-th key must be taken whole (float scores: after two passes, when
+// the bin holds a single key); exact ties run all three passes.  The CTAs exchange their selected counts the
+// same way to place their outputs.  Longer rows fall back to one CTA that re-reads the row from L2 in every
+// pass (8-bit digits).  The call is latency-bound, not bandwidth-bound, at the sizes of the workloads, so the
+// cluster kernel is launched with programmatic stream serialization: its CTAs become resident and clear their
+// histograms while the kernel before them (the score kernel in a step) is still draining, and touch global
+// memory only after griddepcontrol.wait.  (One CTA per row with the keys in shared memory was measured as
+// well: 26.7 us on the 17550-token row against 16.7 us for a cluster of five, because one SM has to issue all
+// of the ~100 instructions per token.)
 #include "common.cuh"
 
 namespace astraea {
@@ -162,8 +169,16 @@ select_kernel(const float *__restrict__ score, int N_sel, int k, int n_always,
 }
 
 
+// programmatic dependent launch: wait for the kernel before this one in the stream (all of its memory operations
+// are then visible); let the kernel after this one start its own prologue
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------- cluster version (keys in registers)
 constexpr int kMaxCluster = 8;
+constexpr int kBinsWide = 4096;                  // 12-bit digits (the last digit has 8 bits and uses 256 of the bins)
+constexpr int kPasses = 3;
+constexpr size_t kClusterSmem = 2 * kPasses * kBinsWide * sizeof(uint32_t);      // own + cluster histogram per pass: 96 KB
 
 __device__ __forceinline__ uint32_t cluster_rank() {
     uint32_t r;
@@ -191,11 +206,11 @@ __global__ void __launch_bounds__(kThreads)
 select_cluster_kernel(const float *__restrict__ score, int N_sel, int k, int n_always,
                       int32_t *__restrict__ idx_sel, int32_t *__restrict__ idx_rem, int32_t *__restrict__ n_skip)
 {
-    __shared__ uint32_t hist[4][256];           // this CTA's histograms of the four passes
-    __shared__ uint32_t ghist[4][256];          // the cluster's histograms: every CTA adds its counts into every CTA's copy
-    __shared__ uint32_t cta_tot[kMaxCluster];   // packed (greater | equal << 16) totals of every CTA
-    __shared__ uint32_t warp_tot[32];
-    __shared__ uint32_t s_prefix, s_kk;
+    extern __shared__ __align__(16) uint32_t smem_hist[];      // [kPasses][kBinsWide] own counts, then [kPasses][kBinsWide] cluster counts
+    uint32_t *hist = smem_hist, *ghist = smem_hist + kPasses * kBinsWide;
+    __shared__ uint32_t cta_gt[kMaxCluster], cta_eq[kMaxCluster];   // selected-by-greater / equal totals of every CTA
+    __shared__ uint32_t warp_tot[32], warp_gt[32], warp_eq[32];
+    __shared__ uint32_t s_prefix, s_kk, s_cnt;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.y;
@@ -206,23 +221,38 @@ select_cluster_kernel(const float *__restrict__ score, int N_sel, int k, int n_a
     int32_t *nsk = n_skip ? n_skip + (size_t)b * N_sel : nullptr;
 
     const int base = ((int)rank * kThreads + tid) * ITEMS;      // this thread's consecutive tokens
+    {
+        uint4 *z = reinterpret_cast<uint4 *>(smem_hist);
+        for (int i = tid; i < (int)(kClusterSmem / 16); i += kThreads) z[i] = make_uint4(0, 0, 0, 0);
+    }
+    grid_launch_dependents();                    // the next kernel may set itself up; it waits for this one before it reads anything
+    grid_dependency_wait();                      // the scores (and whatever else the kernel before wrote) are complete
     uint32_t key[ITEMS];
+    // the counters are needed only at the very end: fetched now where the registers allow it (16 items per thread
+    // would spill), so that their latency is hidden behind the passes
+    constexpr bool kPrefetchCounters = ITEMS <= 8;
+    int32_t n_old[kPrefetchCounters ? ITEMS : 1];
 #pragma unroll
     for (int u = 0; u < ITEMS; ++u) key[u] = (base + u < N_sel) ? score_key(__ldg(s + base + u)) : 0u;
-
-    for (int i = tid; i < 4 * 256; i += kThreads) { (&ghist[0][0])[i] = 0; (&hist[0][0])[i] = 0; }
+    if constexpr (kPrefetchCounters) {
+#pragma unroll
+        for (int u = 0; u < ITEMS; ++u) n_old[u] = (nsk && base + u < N_sel) ? nsk[base + u] : 0;
+    }
     cluster_sync_all();                          // every CTA's histograms are zero before anyone adds to them
 
+    // token i is selected iff key > T, or key == T and fewer than need_eq equal keys precede it
     uint32_t T = 0xffffffffu, need_eq = 0;       // no key reaches 0xffffffff
     if (k > 0) {
         uint32_t prefix = 0, mask = 0, kk = (uint32_t)k;
 #pragma unroll 1
-        for (int pass = 0; pass < 4; ++pass) {
-            const int shift = 24 - 8 * pass;
+        for (int pass = 0; pass < kPasses; ++pass) {
+            const int shift = pass == 0 ? 20 : pass == 1 ? 8 : 0;
+            const uint32_t digit_mask = pass == 2 ? 255u : 4095u;
+            uint32_t *h = hist + pass * kBinsWide, *gh = ghist + pass * kBinsWide;
 #pragma unroll
             for (int u = 0; u < ITEMS; ++u) {
                 const bool live = (base + u < N_sel) && ((key[u] & mask) == prefix);
-                const uint32_t bin = (key[u] >> shift) & 255u;
+                const uint32_t bin = (key[u] >> shift) & digit_mask;
                 const uint32_t act = __ballot_sync(0xffffffffu, live);
                 if (act == 0) continue;
                 // the leading digits of the scores are nearly all equal: one atomic for the warp when its live keys
@@ -230,53 +260,73 @@ select_cluster_kernel(const float *__restrict__ score, int N_sel, int k, int n_a
                 const int leader = __ffs(act) - 1;
                 const uint32_t lbin = __shfl_sync(0xffffffffu, bin, leader);
                 if (__all_sync(0xffffffffu, !live || bin == lbin)) {
-                    if (lane == leader) atomicAdd(&hist[pass][lbin], (uint32_t)__popc(act));
+                    if (lane == leader) atomicAdd(&h[lbin], (uint32_t)__popc(act));
                 } else if (live) {
-                    atomicAdd(&hist[pass][bin], 1u);
+                    atomicAdd(&h[bin], 1u);
                 }
             }
             __syncthreads();
-            // thread (r, bin) adds this CTA's count of the bin into CTA r's copy, so that every CTA searches its own copy
-            for (int i = tid; i < 256 * (int)csize; i += kThreads) {
-                const uint32_t c = hist[pass][i & 255];
-                if (c != 0) remote_add(map_to_rank(&ghist[pass][i & 255], (uint32_t)i >> 8), c);
+            // this CTA's non-zero counts go into every CTA's copy, so that every CTA searches its own copy
+            const int bins = (int)digit_mask + 1;
+            for (int i = tid; i < bins; i += kThreads) {
+                const uint32_t c = h[i];
+                if (c != 0)
+                    for (uint32_t r = 0; r < csize; ++r) remote_add(map_to_rank(&gh[i], r), c);
             }
             cluster_sync_all();
-            if (warp == 0) {
-                // lane l owns bins 255-8l .. 248-8l (descending); find where the count from the top reaches kk
-                uint32_t c[8], tot = 0;
+            // search from the top: thread t owns bins top-4t .. top-4t-3 (the 256-bin pass uses the first 64 threads)
+            {
+                const int top = bins - 1 - 4 * tid;
+                uint32_t c[4] = {0, 0, 0, 0}, tot = 0;
+                if (top >= 3) {
 #pragma unroll
-                for (int j = 0; j < 8; ++j) { c[j] = ghist[pass][255 - 8 * lane - j]; tot += c[j]; }
+                    for (int j = 0; j < 4; ++j) { c[j] = gh[top - j]; tot += c[j]; }
+                }
                 uint32_t inc = tot;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
-                    uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+                    const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
                     if (lane >= o) inc += t;
                 }
-                const uint32_t exc = inc - tot;
-                if (exc < kk && inc >= kk) {
+                if (lane == 31) warp_tot[warp] = inc;
+                __syncthreads();
+                uint32_t wsum = warp_tot[lane];                  // every warp scans the 32 warp totals itself
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t t = __shfl_up_sync(0xffffffffu, wsum, o);
+                    if (lane >= o) wsum += t;
+                }
+                const uint32_t wbase = __shfl_sync(0xffffffffu, wsum, (warp + 31) & 31);
+                const uint32_t exc = (warp > 0 ? wbase : 0u) + inc - tot;
+                if (exc < kk && exc + tot >= kk) {
                     uint32_t above = exc;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
+                    for (int j = 0; j < 4; ++j) {
                         if (above + c[j] >= kk) {
-                            s_prefix = prefix | ((uint32_t)(255 - 8 * lane - j) << shift);
+                            s_prefix = prefix | ((uint32_t)(top - j) << shift);
                             s_kk = kk - above;
+                            s_cnt = c[j];
                             break;
                         }
                         above += c[j];
                     }
                 }
+                __syncthreads();
             }
-            __syncthreads();
             prefix = s_prefix;
             kk = s_kk;
-            mask |= 255u << shift;
+            mask |= digit_mask << shift;
+            if (s_cnt == kk) {
+                // the whole bin is taken: every key with these leading digits is selected, whatever follows them
+                T = prefix;                      // the smallest key of the bin, were it present
+                need_eq = 0xffffffffu;
+                break;
+            }
+            if (pass == kPasses - 1) { T = prefix; need_eq = kk; }
         }
-        T = prefix;
-        need_eq = kk;
     }
 
-    // ordered placement: token i is selected iff key > T, or key == T and fewer than need_eq equal keys precede it
+    // ordered placement
     uint32_t gt[ITEMS], eq[ITEMS], tg = 0, te = 0;
 #pragma unroll
     for (int u = 0; u < ITEMS; ++u) {
@@ -286,32 +336,31 @@ select_cluster_kernel(const float *__restrict__ score, int N_sel, int k, int n_a
         tg += gt[u];
         te += eq[u];
     }
-    const uint32_t packed = tg | (te << 16);     // a CTA holds at most 16384 tokens
-    uint32_t inc = packed;
+    uint32_t ig = tg, ie = te;                   // inclusive scans over the warp
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-        uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
-        if (lane >= o) inc += t;
+        const uint32_t a = __shfl_up_sync(0xffffffffu, ig, o), c = __shfl_up_sync(0xffffffffu, ie, o);
+        if (lane >= o) { ig += a; ie += c; }
     }
-    if (lane == 31) warp_tot[warp] = inc;
+    if (lane == 31) { warp_gt[warp] = ig; warp_eq[warp] = ie; }
     __syncthreads();
-    if (warp == 0) {
-        uint32_t w = warp_tot[lane], winc = w;
+    uint32_t wg = warp_gt[lane], we = warp_eq[lane];            // every warp scans the 32 warp totals itself
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            uint32_t t = __shfl_up_sync(0xffffffffu, winc, o);
-            if (lane >= o) winc += t;
-        }
-        warp_tot[lane] = winc - w;
-        // every CTA learns every CTA's totals
-        const uint32_t total = __shfl_sync(0xffffffffu, winc, 31);
-        if (lane < csize) remote_store(map_to_rank(&cta_tot[rank], lane), total);
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t a = __shfl_up_sync(0xffffffffu, wg, o), c = __shfl_up_sync(0xffffffffu, we, o);
+        if (lane >= o) { wg += a; we += c; }
+    }
+    const uint32_t bg = warp > 0 ? __shfl_sync(0xffffffffu, wg, warp - 1) : 0u;
+    const uint32_t be = warp > 0 ? __shfl_sync(0xffffffffu, we, warp - 1) : 0u;
+    // every CTA learns every CTA's totals (the shuffles are outside the branch: all 32 lanes must take part)
+    const uint32_t allg = __shfl_sync(0xffffffffu, wg, 31), alle = __shfl_sync(0xffffffffu, we, 31);
+    if (warp == 0 && lane < (int)csize) {
+        remote_store(map_to_rank(&cta_gt[rank], lane), allg);
+        remote_store(map_to_rank(&cta_eq[rank], lane), alle);
     }
     cluster_sync_all();
-    uint32_t G = 0, E = 0;
-    for (uint32_t r = 0; r < rank; ++r) { G += cta_tot[r] & 0xffffu; E += cta_tot[r] >> 16; }
-    const uint32_t exc = inc - packed + warp_tot[warp];
-    uint32_t pg = G + (exc & 0xffffu), pe = E + (exc >> 16);
+    uint32_t pg = bg + ig - tg, pe = be + ie - te;
+    for (uint32_t r = 0; r < rank; ++r) { pg += cta_gt[r]; pe += cta_eq[r]; }
 #pragma unroll
     for (int u = 0; u < ITEMS; ++u) {
         const int i = base + u;
@@ -320,7 +369,7 @@ select_cluster_kernel(const float *__restrict__ score, int N_sel, int k, int n_a
             const uint32_t before = pg + min(pe, need_eq);
             if (take) { if (sel) sel[before] = i; }
             else if (rem) rem[(uint32_t)i - before] = i;
-            if (nsk) nsk[i] = take ? 0 : min(nsk[i] + 1, ASTRAEA_N_SKIP_CLAMP);
+            if (nsk) nsk[i] = take ? 0 : min((kPrefetchCounters ? n_old[u] : nsk[i]) + 1, ASTRAEA_N_SKIP_CLAMP);
         }
         pg += gt[u];
         pe += eq[u];
@@ -334,18 +383,24 @@ int32_t launch_cluster(const float *score, int B, int N_sel, int k, int n_always
                        int32_t *idx_rem, int32_t *n_skip, cudaStream_t stream)
 {
     const int csize = (N_sel + ITEMS * kThreads - 1) / (ITEMS * kThreads);
+    static PerDeviceOnce attrs;                  // one per instantiation; the attribute is per device
+    if (attrs.run([] { return cudaFuncSetAttribute(select_cluster_kernel<ITEMS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   (int)kClusterSmem); }) != cudaSuccess)
+        return check_launch("astraea_select (shared memory attribute)");
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(csize, B, 1);
     cfg.blockDim = dim3(kThreads, 1, 1);
-    cfg.dynamicSmemBytes = 0;
+    cfg.dynamicSmemBytes = kClusterSmem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = csize;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;      // see grid_dependency_wait in the kernel
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     cudaError_t e = cudaLaunchKernelEx(&cfg, select_cluster_kernel<ITEMS>, score, N_sel, k, n_always, idx_sel, idx_rem, n_skip);
     if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_select: %s", cudaGetErrorString(e));
     return check_launch("astraea_select");
@@ -359,9 +414,8 @@ int32_t launch_select(const float *score, int B, int N_sel, int k, int n_always,
                       int32_t *idx_rem, int32_t *n_skip, void *, cudaStream_t stream)
 {
     if (B == 0 || (N_sel == 0 && n_always == 0)) return ASTRAEA_OK;
-#ifdef SEL_FORCE
-    if (N_sel > 0 && N_sel <= SEL_FORCE * kThreads * kMaxCluster) return launch_cluster<SEL_FORCE>(score, B, N_sel, k, n_always, idx_sel, idx_rem, n_skip, stream);
-#endif
+    if (N_sel > 0 && N_sel <= 2 * kThreads * kMaxCluster)
+        return launch_cluster<2>(score, B, N_sel, k, n_always, idx_sel, idx_rem, n_skip, stream);
     if (N_sel > 0 && N_sel <= 4 * kThreads * kMaxCluster)
         return launch_cluster<4>(score, B, N_sel, k, n_always, idx_sel, idx_rem, n_skip, stream);
     if (N_sel > 0 && N_sel <= 8 * kThreads * kMaxCluster)

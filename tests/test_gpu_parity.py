@@ -71,6 +71,23 @@ def test_score_counter_clamp(oracle):
     assert (np.abs(got - want) / want).max() < 1e-5
 
 
+def test_score_lse_clamp_keeps_fp32_scores_finite(oracle):
+    """Log values above 80 (a row with one logit of that size, as sharpened attention leaves behind) count as 80 in
+    the sum-of-exponentials mode, on the device as in the oracle; the scores stay finite and ordered."""
+    B, N, D, H = 1, 16, 64, 2
+    rng = np.random.default_rng(3)
+    x_ref = synth.f32_to_bf16_bits(rng.standard_normal((B, N, D)).astype(np.float32))
+    x_cur = synth.f32_to_bf16_bits(rng.standard_normal((B, N, D)).astype(np.float32))
+    lse = rng.uniform(-5, 5, (B, H, N)).astype(np.float32)
+    lse[0, 0, 3], lse[0, 1, 5], lse[0, :, 7], lse[0, 0, 9] = 79.5, 80.0, 95.0, 3.0e4
+    want = oracle.score(f64(x_cur), f64(x_ref), lse, None, H=H, w_alpha=1e-3, w_beta=0.0)
+    out = torch.empty(B, N, device="cuda")
+    A.astraea_score(to_dev_bf16(x_cur), to_dev_bf16(x_ref), dev(lse), None, out, B, N, N, D, H, 1e-3, 0.0)
+    got = out.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    assert (np.abs(got - want) / np.abs(want)).max() < SCORE_RTOL
+
+
 # --------------------------------------------------------------------- select
 def _select_case(oracle, s, k, n_always=0, with_n=True, with_rem=True, seed=0):
     B, n_sel = s.shape

@@ -350,6 +350,20 @@ def test_score_constant_per_token_difference_closed_form(oracle):
     assert np.allclose(big, math.exp(80.0), rtol=1e-15)
 
 
+def test_score_log_values_above_the_clamp_count_as_the_clamp(oracle):
+    """The sum-of-exponentials reading keeps the fp32 scores finite: a log value above 80 counts as 80 (a reading
+    of this build, stated next to the counter clamp); the log-mode score is not clamped."""
+    B, N, D, H = 1, 4, 8, 2
+    x_ref = np.zeros((B, N, D))
+    x_cur = np.full((B, N, D), 0.5)
+    lse = np.array([[[0.0, 79.0, 80.0, 1000.0], [0.0, 79.0, 85.0, 90.0]]])
+    s = oracle.score(x_cur, x_ref, lse, None, w_alpha=1.0, w_beta=0.0)
+    want = 0.5 * np.array([1.0, math.exp(79.0), math.exp(80.0), math.exp(80.0)])
+    assert np.abs(s[0] - want).max() <= 1e-12 * want.max() and np.isfinite(s.astype(np.float32)).all()
+    s1 = oracle.score(x_cur, x_ref, lse, None, w_alpha=1.0, w_beta=0.0, lse_mode=1)
+    assert np.abs(s1[0] - 0.5 * np.array([0.0, 79.0, 82.5, 545.0])).max() < 1e-12
+
+
 def test_score_mixed_signs_distinguish_the_three_reductions(oracle):
     x_ref = np.zeros((1, 1, 4))
     x_cur = np.array([[[1.0, -1.0, 2.0, -4.0]]])
