@@ -263,6 +263,36 @@ void oracle_gathered_linear(const double *x, const int32_t *idx, int M, const do
         }
 }
 
+/*
+ * Layer normalisation of token rows followed by a per-batch-element modulation, the element-wise step in front
+ * of every layer group of a compute block (Section 3.2: the layers of a block other than self-attention act on
+ * each token by itself, so they are evaluated for the selected tokens only):
+ *     y[r, :] = (x[r, :] - mean_r) / sqrt(var_r + eps) * (1 + scale[b, :]) + shift[b, :]
+ * with the biased variance over the D channels and no learned affine; scale / shift NULL: plain normalisation.
+ * x, y : [B, R, D] (R rows per batch element, whatever tokens they belong to); scale, shift : [B, D].
+ */
+void oracle_layernorm_modulate(const double *x, const double *scale, const double *shift, double *y,
+                               int B, int R, int D, double eps)
+{
+    for (int b = 0; b < B; ++b)
+        for (int r = 0; r < R; ++r) {
+            const double *xr = x + ((size_t)b * R + r) * D;
+            double *yr = y + ((size_t)b * R + r) * D;
+            double mean = 0.0, var = 0.0;
+            for (int c = 0; c < D; ++c) mean += xr[c];
+            mean /= (double)D;
+            for (int c = 0; c < D; ++c) var += (xr[c] - mean) * (xr[c] - mean);
+            var /= (double)D;
+            const double rstd = 1.0 / sqrt(var + eps);
+            for (int c = 0; c < D; ++c) {
+                double v = (xr[c] - mean) * rstd;
+                if (scale) v *= 1.0 + scale[(size_t)b * D + c];
+                if (shift) v += shift[(size_t)b * D + c];
+                yr[c] = v;
+            }
+        }
+}
+
 /* floor(theta * N_sel) in integer arithmetic from a permille budget [R9]. */
 int oracle_budget_to_k(int n_sel, int theta_permille)
 {

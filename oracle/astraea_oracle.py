@@ -157,6 +157,15 @@ def gathered_linear(x, w, bias=None, idx=None, y_cache=None, compact_in=False, g
     return y
 
 
+def layernorm_modulate(x, scale=None, shift=None, eps=1e-6):
+    """y = LayerNorm(x) * (1 + scale[b]) + shift[b] over the last axis (no learned affine); x: [B, R, D]."""
+    x = _f64(x)
+    B, R, D = x.shape
+    y = np.empty_like(x)
+    _load().oracle_layernorm_modulate(_p(x), _p(_f64(scale)), _p(_f64(shift)), _p(y), B, R, D, ctypes.c_double(eps))
+    return y
+
+
 def scatter_lse(lse_cache, lse_rows, idx):
     out = np.array(lse_cache, dtype=np.float64, copy=True, order="C")
     lse_rows, idx = _f64(lse_rows), _i32(idx)
@@ -207,3 +216,81 @@ def step(x_cur, x_ref, lse_cache, n_skip, q, k, v, cache, k_keep, n_always=0,
         xr = np.array(x_ref, dtype=np.float64, copy=True)
     return dict(score=s64, score_f32=s32, idx_sel=idx_sel, idx_rem=idx_rem, n_skip=n_new,
                 out=out, lse=lse_new, x_ref=xr, own_idx_sel=own)
+
+
+def take_rows(a, idx):
+    """Rows idx[b, r] of a [B, N, ...] array as [B, M, ...]."""
+    a = np.asarray(a)
+    ix = np.asarray(idx, dtype=np.int64).reshape(idx.shape + (1,) * (a.ndim - 2))
+    return np.take_along_axis(a, ix, axis=1)
+
+
+def block_step(x, x_ref, lse_cache, n_skip, y_cache, weights, text_k, text_v, H, k_keep, n_always=0,
+               w_alpha=1.0, w_beta=1.0, delta_mode=0, lse_mode=0, eps=1e-6, forced_sel=None, rounder=None):
+    """One transformer block at one denoising step with token-wise reuse (Algorithm 1 and the execution flow of
+    Section 3.2 applied to a whole compute block): the tokens are scored on the block's input and selected;
+    keys and values come from ALL tokens of the current step; the query projection, the self-attention rows, the
+    output projection, the cross-attention against the text keys / values and the MLP are evaluated for the selected
+    tokens only; every other token keeps the block's cached output.  Pre-norm block with residuals:
+
+        h  = LN(x) (1 + s1) + t1                      all tokens (keys / values need them)
+        K, V = h Wk^T + bk, h Wv^T + bv               all tokens;   Q = h[sel] Wq^T + bq
+        x1 = x[sel] + g1 * (Attn(Q, K, V) Wo^T + bo)
+        x2 = x1 + Attn(LN(x1) Wq2^T + bq2, text_k, text_v) Wo2^T + bo2
+        x3 = x2 + g3 * (GELU((LN(x2) (1 + s3) + t3) W1^T + b1) W2^T + b2)
+        y_cache[sel] = x3;  lse_cache[:, sel] = LSE of the self-attention rows;  x_ref[sel] = x[sel]
+
+    weights: dict of float64 arrays wq, bq, wk, bk, wv, bv, wo, bo, wq2, bq2, wo2, bo2, w1, b1, w2, b2 ([out, in] /
+    [out]) and the modulation vectors s1, t1, g1, s3, t3, g3 ([B, D], any of them None).  text_k, text_v: [B, N_text, H, d].
+    rounder: None, or a function applied to every intermediate tensor that the device stores as bf16 (the parity
+    tests pass the bf16 rounding there, so that the oracle follows the device's storage precision layer by layer).
+    Returns a dict: idx_sel, idx_rem, n_skip, score, y (new cache), lse, x_ref, and the intermediates.
+    """
+    rd = (lambda a: a) if rounder is None else rounder
+    x = _f64(x)
+    B, N, D = x.shape
+    d = D // H
+    n_sel = N - n_always
+    w = weights
+    s64 = score(x, x_ref, lse_cache, n_skip, n_sel=n_sel, w_alpha=w_alpha, w_beta=w_beta, delta_mode=delta_mode, lse_mode=lse_mode)
+    idx_sel, idx_rem, n_new = select(s64.astype(np.float32), k_keep, n_always, n_skip)
+    own = idx_sel
+    if forced_sel is not None:
+        idx_sel = _i32(forced_sel)
+        chosen = np.zeros((B, N), dtype=bool)
+        for b in range(B):
+            chosen[b, idx_sel[b]] = True
+        idx_rem = np.stack([np.flatnonzero(~chosen[b, :n_sel]) for b in range(B)]).astype(np.int32)
+        if n_skip is not None:
+            n_new = np.where(chosen[:, :n_sel], 0, np.minimum(np.asarray(n_skip, dtype=np.int64) + 1, 80)).astype(np.int32)
+    res = dict(score=s64, idx_sel=idx_sel, idx_rem=idx_rem, n_skip=n_new, own_idx_sel=own)
+    M = idx_sel.shape[1]
+    if M == 0:
+        res.update(y=np.array(y_cache, dtype=np.float64, copy=True), lse=np.array(lse_cache, dtype=np.float64, copy=True),
+                   x_ref=np.array(x_ref, dtype=np.float64, copy=True))
+        return res
+    h = rd(layernorm_modulate(x, w.get("s1"), w.get("t1"), eps))
+    k = rd(gathered_linear(h, w["wk"], w.get("bk")))
+    v = rd(gathered_linear(h, w["wv"], w.get("bv")))
+    q = rd(gathered_linear(h, w["wq"], w.get("bq"), idx_sel))                     # rows outside idx_sel stay zero and are never read
+    a, l, _ = sparse_attn(q.reshape(B, N, H, d), k.reshape(B, N, H, d), v.reshape(B, N, H, d), q_idx=idx_sel)
+    a = rd(a.reshape(B, M, D))
+    o = gathered_linear(a, w["wo"], w.get("bo"))
+    if w.get("g1") is not None:
+        o = o * _f64(w["g1"])[:, None, :]
+    x1 = rd(take_rows(x, idx_sel) + o)
+    h2 = rd(layernorm_modulate(x1, None, None, eps))
+    q2 = rd(gathered_linear(h2, w["wq2"], w.get("bq2")))
+    c, _, _ = sparse_attn(q2.reshape(B, M, H, d), text_k, text_v)
+    c = rd(c.reshape(B, M, D))
+    x2 = rd(x1 + gathered_linear(c, w["wo2"], w.get("bo2")))
+    h3 = rd(layernorm_modulate(x2, w.get("s3"), w.get("t3"), eps))
+    u = rd(gathered_linear(h3, w["w1"], w.get("b1"), gelu=True))
+    m = gathered_linear(u, w["w2"], w.get("b2"))
+    if w.get("g3") is not None:
+        m = m * _f64(w["g3"])[:, None, :]
+    x3 = rd(x2 + m)
+    res.update(h=h, k=k, v=v, q_rows=take_rows(q, idx_sel), attn_rows=a, x1=x1, h2=h2, q2=q2, cross_rows=c, x2=x2, h3=h3, u=u, x3=x3,
+               y=scatter_reuse(y_cache, x3, idx_sel), lse=scatter_lse(lse_cache, l, idx_sel),
+               x_ref=scatter_reuse(x_ref, take_rows(x, idx_sel), idx_sel))
+    return res

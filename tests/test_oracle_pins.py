@@ -509,3 +509,97 @@ def test_attention_flops_are_linear_in_selected_tokens_like_the_papers_tables():
             M = int(round(theta * N))
             ratio = accounting.attn_flops(B, H, M, N, d) / full
             assert abs(ratio - float(val) / float(orig)) < 2e-4, (name, theta)
+
+
+# ------------------------------------------------------------------ whole-block pins
+def _block_weights(rng, B, D, hidden, modulated=True):
+    lin = lambda o, i: rng.standard_normal((o, i)) / math.sqrt(i)
+    w = {}
+    for name, (o, i) in dict(wq=(D, D), wk=(D, D), wv=(D, D), wo=(D, D), wq2=(D, D), wo2=(D, D), w1=(hidden, D), w2=(D, hidden)).items():
+        w[name] = lin(o, i)
+        w["b" + name[1:]] = 0.1 * rng.standard_normal(o)
+    if modulated:
+        for name in ("s1", "t1", "g1", "s3", "t3", "g3"):
+            w[name] = 0.3 * rng.standard_normal((B, D))
+    return w
+
+
+def _torch_dense_block(x, w, text_k, text_v, H, eps=1e-6):
+    """The same block from torch's fp64 building blocks (layer_norm, linear, scaled_dot_product_attention, gelu)."""
+    F = torch.nn.functional
+    t = lambda a: torch.from_numpy(np.ascontiguousarray(a))
+    X = t(x)
+    B, N, D = X.shape
+    d = D // H
+    mod = lambda h, s, sh: h * (1 + t(w[s])[:, None, :]) + t(w[sh])[:, None, :] if w.get(s) is not None else h
+    heads = lambda a: a.reshape(B, -1, H, d).permute(0, 2, 1, 3)
+    h = mod(F.layer_norm(X, (D,), eps=eps), "s1", "t1")
+    q, k, v = (F.linear(h, t(w["w" + n]), t(w["b" + n])) for n in ("q", "k", "v"))
+    a = F.scaled_dot_product_attention(heads(q), heads(k), heads(v)).permute(0, 2, 1, 3).reshape(B, N, D)
+    o = F.linear(a, t(w["wo"]), t(w["bo"]))
+    x1 = X + (o * t(w["g1"])[:, None, :] if w.get("g1") is not None else o)
+    q2 = F.linear(F.layer_norm(x1, (D,), eps=eps), t(w["wq2"]), t(w["bq2"]))
+    c = F.scaled_dot_product_attention(heads(q2), t(text_k).permute(0, 2, 1, 3), t(text_v).permute(0, 2, 1, 3)).permute(0, 2, 1, 3).reshape(B, N, D)
+    x2 = x1 + F.linear(c, t(w["wo2"]), t(w["bo2"]))
+    h3 = mod(F.layer_norm(x2, (D,), eps=eps), "s3", "t3")
+    m = F.linear(F.gelu(F.linear(h3, t(w["w1"]), t(w["b1"]))), t(w["w2"]), t(w["b2"]))
+    x3 = x2 + (m * t(w["g3"])[:, None, :] if w.get("g3") is not None else m)
+    lse = torch.logsumexp(torch.einsum("bhic,bhjc->bhij", heads(q), heads(k)) / math.sqrt(d), -1)
+    return x3.numpy(), lse.numpy()
+
+
+@pytest.mark.parametrize("modulated", [True, False])
+def test_block_step_at_keep_ratio_one_is_the_dense_block_of_library_modules(oracle, modulated):
+    rng = np.random.default_rng(31)
+    B, N, H, d, N_text, hidden = 2, 14, 2, 4, 5, 20
+    D = H * d
+    x = _rand(rng, B, N, D)
+    w = _block_weights(rng, B, D, hidden, modulated)
+    tk, tv = _rand(rng, B, N_text, H, d), _rand(rng, B, N_text, H, d)
+    res = oracle.block_step(x, x + 1.0, _rand(rng, B, H, N), np.zeros((B, N), np.int32), _rand(rng, B, N, D), w, tk, tv, H, k_keep=N)
+    want, want_lse = _torch_dense_block(x, w, tk, tv, H)
+    assert np.abs(res["y"] - want).max() < 1e-11
+    assert np.abs(res["lse"] - want_lse).max() < 1e-11
+    assert np.array_equal(res["x_ref"], x) and (res["n_skip"] == 0).all()
+
+
+def test_block_step_partial_budget_computes_selected_rows_and_reuses_the_rest(oracle):
+    """Selected tokens carry the dense block's rows (keys and values come from all tokens, the other layers act per
+    token), every other token keeps the cached block output, LSE and reference input; keep-ratio 0 changes nothing."""
+    rng = np.random.default_rng(32)
+    B, N_v, N_t, H, d, N_text, hidden = 2, 17, 3, 2, 4, 6, 24
+    N, D, k_keep = N_v + N_t, H * d, 6
+    x_ref = _rand(rng, B, N, D)
+    x = x_ref + 0.4 * _rand(rng, B, N, D)
+    w = _block_weights(rng, B, D, hidden)
+    tk, tv = _rand(rng, B, N_text, H, d), _rand(rng, B, N_text, H, d)
+    y_cache, lse_cache = _rand(rng, B, N, D), 0.3 * _rand(rng, B, H, N)
+    n0 = rng.integers(0, 3, (B, N_v)).astype(np.int32)
+    res = oracle.block_step(x, x_ref, lse_cache, n0, y_cache, w, tk, tv, H, k_keep, n_always=N_t)
+    dense, dense_lse = _torch_dense_block(x, w, tk, tv, H)
+    step = oracle.step(x, x_ref, lse_cache, n0, *(np.zeros((B, N, H, d)) for _ in range(4)), k_keep, n_always=N_t)
+    assert np.array_equal(res["idx_sel"], step["idx_sel"]) and np.array_equal(res["n_skip"], step["n_skip"])   # same score / selection path
+    for b in range(B):
+        sel = res["idx_sel"][b]
+        unsel = np.setdiff1d(np.arange(N), sel)
+        assert len(sel) == k_keep + N_t and len(unsel) == N_v - k_keep
+        assert np.abs(res["y"][b, sel] - dense[b, sel]).max() < 1e-11
+        assert np.array_equal(res["y"][b, unsel], y_cache[b, unsel])
+        assert np.abs(res["lse"][b][:, sel] - dense_lse[b][:, sel]).max() < 1e-11
+        assert np.array_equal(res["lse"][b][:, unsel], lse_cache[b][:, unsel])
+        assert np.array_equal(res["x_ref"][b, sel], x[b, sel]) and np.array_equal(res["x_ref"][b, unsel], x_ref[b, unsel])
+    none = oracle.block_step(x, x_ref, lse_cache, n0[:, :N], y_cache, w, tk, tv, H, 0, n_always=0) if False else \
+        oracle.block_step(x[:, :N_v], x_ref[:, :N_v], lse_cache[:, :, :N_v], n0, y_cache[:, :N_v], w, tk, tv, H, 0)
+    assert np.array_equal(none["y"], y_cache[:, :N_v]) and np.array_equal(none["lse"], lse_cache[:, :, :N_v])
+    assert np.array_equal(none["x_ref"], x_ref[:, :N_v]) and np.array_equal(none["n_skip"], n0 + 1)
+
+
+def test_layernorm_modulate_matches_the_library_routine(oracle):
+    rng = np.random.default_rng(33)
+    B, R, D = 2, 7, 24
+    x, s, t = 3.0 * _rand(rng, B, R, D) + 1.5, _rand(rng, B, D), _rand(rng, B, D)
+    ref = torch.nn.functional.layer_norm(torch.from_numpy(x), (D,), eps=1e-5).numpy()
+    assert np.abs(oracle.layernorm_modulate(x, eps=1e-5) - ref).max() < 1e-13
+    assert np.abs(oracle.layernorm_modulate(x, s, t, eps=1e-5) - (ref * (1 + s[:, None]) + t[:, None])).max() < 1e-13
+    y = oracle.layernorm_modulate(x, eps=0.0)
+    assert np.abs(y.mean(-1)).max() < 1e-13 and np.abs(y.var(-1) - 1.0).max() < 1e-12
