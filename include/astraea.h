@@ -60,6 +60,13 @@ extern "C" {
 #define ASTRAEA_LINEAR_COMPACT_OUT 1u        /* y is [B,M,N_out] (row r of the index list), not the cache [B,N,N_out] */
 #define ASTRAEA_LINEAR_COMPACT_IN  2u        /* x is [B,M,K]: row r is the row of token idx[b,r] (output of a layer run with COMPACT_OUT) */
 #define ASTRAEA_LINEAR_GELU        4u        /* y = GELU(x W^T + bias), GELU(u) = u/2 (1 + erf(u / sqrt 2)): the first MLP layer */
+#define ASTRAEA_LINEAR_COMPACT_RES 8u        /* astraea_gathered_linear_residual: residual is [B,M,N_out] (row r of the index list) */
+/* flags of astraea_layernorm_modulate */
+#define ASTRAEA_LN_COMPACT_IN     1u         /* x is [B,M,D]: row r is the row of token idx[b,r] */
+#define ASTRAEA_LN_COMPACT_OUT    2u         /* y is [B,M,D] */
+/* flags of astraea_block_step */
+#define ASTRAEA_BLOCK_REUSE_SELECTION 1u     /* idx_sel already holds this step's selection (made by another block): no scoring,
+                                              * no selection, counters and reference inputs untouched (the Fixed-token variant) */
 /* flags of astraea_scatter_reuse */
 #define ASTRAEA_SCATTER_SRC_FULL  1u         /* rows is [B,N,row_elems]; row idx[r] of it is copied to row idx[r] of cache */
 
@@ -69,6 +76,7 @@ extern "C" {
 #define ASTRAEA_OP_STEP         3
 #define ASTRAEA_OP_SPARSE_ATTN_KV 4          /* astraea_sparse_attn with kv_idx: pass M_kv as the M argument */
 #define ASTRAEA_OP_GATHERED_LINEAR 5        /* astraea_gathered_linear (the size arguments are ignored) */
+#define ASTRAEA_OP_LAYERNORM    6            /* astraea_layernorm_modulate (the size arguments are ignored) */
 
 /*
  * Selection metric (Section 3.2 "Selection Metric"; Algorithm 1 lines 1-2):
@@ -237,6 +245,76 @@ int32_t astraea_scatter_reuse(void *cache, const void *rows, const int32_t *idx,
 int32_t astraea_gathered_linear(const void *x, const int32_t *idx, int M, const void *w, const void *bias,
                                 void *y, int B, int N, int K, int N_out, uint32_t flags,
                                 void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * The same layer with a gated residual in its epilogue (the residual connections around the layer groups of a
+ * compute block, applied to the selected rows only, Section 3.2):
+ *     y[b, idx[b,r], :] = residual[b, idx[b,r], :] + gate[b, :] * act(x[b, idx[b,r], :] W^T + bias)
+ *   residual : bf16 [B, N, N_out] (rows at idx), with ASTRAEA_LINEAR_COMPACT_RES bf16 [B, M, N_out]; NULL => none
+ *   gate     : bf16 [B, N_out] or NULL (no gate)
+ * Everything else as astraea_gathered_linear; fp32 until the one rounding to bf16 at the end.
+ */
+int32_t astraea_gathered_linear_residual(const void *x, const int32_t *idx, int M, const void *w, const void *bias,
+                                         const void *residual, const void *gate,
+                                         void *y, int B, int N, int K, int N_out, uint32_t flags,
+                                         void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Layer normalisation and modulation of token rows, the element-wise step in front of the layer groups of a compute
+ * block (Section 3.2: the layers other than self-attention act on each token by itself, so it runs for the selected
+ * rows only; in front of the key / value projections, Algorithm 1 line 4, for all rows):
+ *     y[b, idx[b,r], :] = (x[b, idx[b,r], :] - mean) / sqrt(var + eps) * (1 + scale[b, :]) + shift[b, :]
+ * with mean and the biased variance over the D channels of the row and no learned affine.
+ *   x : bf16 [B, N, D] (ASTRAEA_LN_COMPACT_IN: [B, M, D])     y : bf16 [B, N, D] (ASTRAEA_LN_COMPACT_OUT: [B, M, D])
+ *   idx : int32 [B, M] strictly ascending in [0,N); NULL => all N rows (M ignored, compact flags not allowed)
+ *   scale, shift : bf16 [B, D] or NULL
+ *   err_workspace : NULL, or any workspace of this library: bad index entries are skipped and then reported there
+ * fp32 arithmetic, one rounding to bf16.  D a multiple of 8, at most 4096; pointers 16-byte aligned.
+ * Errors: INVALID_ARG, UNSUPPORTED (D too large, unknown flags), CUDA.
+ */
+int32_t astraea_layernorm_modulate(const void *x, const int32_t *idx, int M, const void *scale, const void *shift,
+                                   void *y, int B, int N, int D, float eps, uint32_t flags,
+                                   void *err_workspace, void *stream);
+
+/*
+ * One whole compute block (self-attention, cross-attention, MLP; pre-norm, residual) at one denoising step with
+ * token-wise reuse: Algorithm 1 and the execution flow of Section 3.2 applied to every layer of the block.  The
+ * tokens are scored on the block's input x and selected (as astraea_step does); keys and values are projected from
+ * ALL tokens of the current step (Algorithm 1 line 4); the query projection (line 5), the self-attention rows (line
+ * 6), the output projection, the cross-attention against the text keys / values and the MLP run for the selected
+ * rows only, on compact buffers; the block's cached output keeps every other row (line 7).  With I = idx_sel:
+ *     h        = LN(x) (1 + s1) + t1                        all rows
+ *     K, V     = h Wk^T + bk, h Wv^T + bv                   all rows;      Q[I] = h[I] Wq^T + bq
+ *     x1       = x[I] + g1 * (Attn(Q[I], K, V) Wo^T + bo)
+ *     x2       = x1 + Attn(LN(x1) Wq2^T + bq2, text_k, text_v) Wo2^T + bo2
+ *     y_cache[I] = x2 + g3 * (GELU((LN(x2) (1 + s3) + t3) W1^T + b1) W2^T + b2)
+ *     lse_cache[:, I] = LSE of the self-attention rows;  x_ref[I] = x[I];  counters as astraea_select
+ * All tensors bf16 device memory; weights [out features, in features] row-major; biases [out]; modulation vectors
+ * [B, D]; any bias or modulation pointer may be NULL.  text_k, text_v: [B, N_text, H, d] (projected once per
+ * generation by the caller).  State (in/out): x_ref [B,N,D], lse_cache fp32 [B,H,N], n_skip int32 [B,N_sel], y_cache
+ * [B,N,D] = the block's output after the call.  score / idx_sel / idx_rem as astraea_step.
+ * workspace: astraea_block_workspace_bytes(B, H, N, d, hidden) bytes, 256-byte aligned, zero before the first use.
+ * D = H*d must be a multiple of 64 and at most 4096, hidden a multiple of 64.
+ * k_keep = 0 with no always-kept tokens: only scores and counters change.
+ * Errors: as the calls it is made of.
+ */
+typedef struct astraea_block_weights {
+    const void *wq, *bq, *wk, *bk, *wv, *bv, *wo, *bo;      /* self-attention: D x D each */
+    const void *wq2, *bq2, *wo2, *bo2;                      /* cross-attention query / output projection: D x D */
+    const void *w1, *b1, *w2, *b2;                          /* MLP: hidden x D, D x hidden */
+    const void *s1, *t1, *g1, *s3, *t3, *g3;                /* scale, shift, gate of the attention and MLP groups: [B, D] */
+    int32_t hidden;
+} astraea_block_weights;
+typedef struct astraea_block_state {
+    void *x_ref; float *lse_cache; int32_t *n_skip; void *y_cache;
+} astraea_block_state;
+size_t  astraea_block_workspace_bytes(int B, int H, int N, int d, int hidden);
+int32_t astraea_block_step(const void *x, const astraea_block_weights *weights, const astraea_block_state *state,
+                           const void *text_k, const void *text_v, int N_text,
+                           float *score, int32_t *idx_sel, int32_t *idx_rem,
+                           int B, int H, int N, int N_sel, int d, int k_keep,
+                           float w_alpha, float w_beta, int delta_mode, int lse_mode, float eps, uint32_t flags,
+                           void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * One whole step of one attention block on device buffers (Algorithm 1 with given Q, K, V):

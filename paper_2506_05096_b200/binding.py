@@ -22,18 +22,33 @@ LSE_SUM_EXP, LSE_LOG = 0, 1
 ATTN_COMPACT_OUT = 1
 ATTN_SMALL_CTAS = 2
 SCATTER_SRC_FULL = 1
-LINEAR_COMPACT_OUT, LINEAR_COMPACT_IN, LINEAR_GELU = 1, 2, 4
-OP_SELECT, OP_SPARSE_ATTN, OP_STEP, OP_SPARSE_ATTN_KV, OP_GATHERED_LINEAR = 1, 2, 3, 4, 5
+LINEAR_COMPACT_OUT, LINEAR_COMPACT_IN, LINEAR_GELU, LINEAR_COMPACT_RES = 1, 2, 4, 8
+LN_COMPACT_IN, LN_COMPACT_OUT = 1, 2
+BLOCK_REUSE_SELECTION = 1
+OP_SELECT, OP_SPARSE_ATTN, OP_STEP, OP_SPARSE_ATTN_KV, OP_GATHERED_LINEAR, OP_LAYERNORM = 1, 2, 3, 4, 5, 6
 N_SKIP_CLAMP = 80
 NOALLOC_SCRATCH_BYTES = 4096
 
 EXPORTS = [
     "astraea_score", "astraea_select", "astraea_sparse_attn", "astraea_sparse_cross_attn", "astraea_sparse_attn_noalloc", "astraea_scatter_reuse", "astraea_step",
-    "astraea_gathered_linear", "astraea_schedule_create", "astraea_schedule_launch", "astraea_schedule_destroy",
+    "astraea_gathered_linear", "astraea_gathered_linear_residual", "astraea_layernorm_modulate",
+    "astraea_block_step", "astraea_block_workspace_bytes", "astraea_schedule_create", "astraea_schedule_launch", "astraea_schedule_destroy",
     "astraea_session_create", "astraea_session_destroy", "astraea_step_host",
     "astraea_workspace_bytes", "astraea_budget_to_k", "astraea_poll_error",
     "astraea_last_error", "astraea_version",
 ]
+
+
+class BlockWeights(ctypes.Structure):
+    """struct astraea_block_weights: device pointers of one compute block's parameters."""
+    NAMES = ("wq", "bq", "wk", "bk", "wv", "bv", "wo", "bo", "wq2", "bq2", "wo2", "bo2", "w1", "b1", "w2", "b2",
+             "s1", "t1", "g1", "s3", "t3", "g3")
+    _fields_ = [(n, ctypes.c_void_p) for n in NAMES] + [("hidden", ctypes.c_int32)]
+
+
+class BlockState(ctypes.Structure):
+    """struct astraea_block_state: the cross-step state of one compute block."""
+    _fields_ = [("x_ref", ctypes.c_void_p), ("lse_cache", ctypes.c_void_p), ("n_skip", ctypes.c_void_p), ("y_cache", ctypes.c_void_p)]
 
 
 class AstraeaError(RuntimeError):
@@ -64,6 +79,12 @@ def lib() -> ctypes.CDLL:
                                                                                  c_i, c_i, c_i, c_i, c_f, c_u, c_p]
         L.astraea_scatter_reuse.argtypes = [c_p, c_p, c_p, c_i, c_i, c_i, c_i, c_u, c_p, c_p]
         L.astraea_gathered_linear.argtypes = [c_p, c_p, c_i, c_p, c_p, c_p, c_i, c_i, c_i, c_i, c_u, c_p, c_sz, c_p]
+        L.astraea_gathered_linear_residual.argtypes = [c_p, c_p, c_i, c_p, c_p, c_p, c_p, c_p, c_i, c_i, c_i, c_i, c_u, c_p, c_sz, c_p]
+        L.astraea_layernorm_modulate.argtypes = [c_p, c_p, c_i, c_p, c_p, c_p, c_i, c_i, c_i, c_f, c_u, c_p, c_p]
+        L.astraea_block_step.argtypes = [c_p, ctypes.POINTER(BlockWeights), ctypes.POINTER(BlockState), c_p, c_p, c_i, c_p, c_p, c_p,
+                                         c_i, c_i, c_i, c_i, c_i, c_i, c_f, c_f, c_i, c_i, c_f, c_u, c_p, c_sz, c_p]
+        L.astraea_block_workspace_bytes.argtypes = [c_i] * 5
+        L.astraea_block_workspace_bytes.restype = c_sz
         L.astraea_step.argtypes = [c_p] * 11 + [c_i] * 6 + [c_f, c_f, c_i, c_i, c_p, c_sz, c_p]
         L.astraea_schedule_create.argtypes = [ctypes.POINTER(c_p), c_i, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p, c_p,
                                               c_i, c_i, c_i, c_i, c_i, c_f, c_f, c_i, c_i, c_p, c_sz]
@@ -81,7 +102,7 @@ def lib() -> ctypes.CDLL:
         L.astraea_last_error.restype = ctypes.c_char_p
         L.astraea_version.restype = ctypes.c_char_p
         for name in ("astraea_score", "astraea_select", "astraea_sparse_attn", "astraea_sparse_cross_attn", "astraea_sparse_attn_noalloc", "astraea_scatter_reuse",
-                     "astraea_step", "astraea_gathered_linear", "astraea_schedule_create", "astraea_schedule_launch",
+                     "astraea_step", "astraea_gathered_linear", "astraea_gathered_linear_residual", "astraea_layernorm_modulate", "astraea_block_step", "astraea_schedule_create", "astraea_schedule_launch",
                      "astraea_session_create", "astraea_step_host", "astraea_budget_to_k",
                      "astraea_poll_error"):
             getattr(L, name).restype = ctypes.c_int32
@@ -177,6 +198,48 @@ def astraea_gathered_linear(x, idx, M, w, bias, y, B, N, K, N_out, flags=0, work
         return          # an empty index tensor has a null data pointer, which the C ABI reads as "all rows"
     _check(lib().astraea_gathered_linear(_ptr(x), _ptr(idx), M, _ptr(w), _ptr(bias), _ptr(y), B, N, K, N_out, flags,
                                          _ptr(workspace), workspace.numel() if workspace is not None else 0, _stream(stream)))
+
+
+def astraea_gathered_linear_residual(x, idx, M, w, bias, residual, gate, y, B, N, K, N_out, flags=0, workspace=None, stream=None) -> None:
+    """y[rows] = residual[rows] + gate[b] * act(x[rows] @ w.T + bias): astraea_gathered_linear with a gated residual."""
+    if idx is not None and M == 0:
+        return
+    _check(lib().astraea_gathered_linear_residual(_ptr(x), _ptr(idx), M, _ptr(w), _ptr(bias), _ptr(residual), _ptr(gate), _ptr(y),
+                                                  B, N, K, N_out, flags, _ptr(workspace),
+                                                  workspace.numel() if workspace is not None else 0, _stream(stream)))
+
+
+def astraea_layernorm_modulate(x, idx, M, scale, shift, y, B, N, D, eps=1e-6, flags=0, workspace=None, stream=None) -> None:
+    """y[rows] = LayerNorm(x[rows]) * (1 + scale[b]) + shift[b] (idx None: all rows)."""
+    if idx is not None and M == 0:
+        return
+    _check(lib().astraea_layernorm_modulate(_ptr(x), _ptr(idx), M, _ptr(scale), _ptr(shift), _ptr(y), B, N, D, eps, flags,
+                                            _ptr(workspace), _stream(stream)))
+
+
+def astraea_block_workspace_bytes(B: int, H: int, N: int, d: int, hidden: int) -> int:
+    return int(lib().astraea_block_workspace_bytes(B, H, N, d, hidden))
+
+
+def block_weights(tensors: dict, hidden: int) -> BlockWeights:
+    """A BlockWeights struct from a dict of device tensors (missing / None entries become NULL).  The caller keeps the
+    tensors alive."""
+    w = BlockWeights()
+    for n in BlockWeights.NAMES:
+        t = tensors.get(n)
+        setattr(w, n, None if t is None else t.data_ptr())
+    w.hidden = hidden
+    return w
+
+
+def astraea_block_step(x, weights: BlockWeights, x_ref, lse_cache, n_skip, y_cache, text_k, text_v, N_text,
+                       score, idx_sel, idx_rem, B, H, N, N_sel, d, k_keep, w_alpha=1.0, w_beta=1.0,
+                       delta_mode=DELTA_MEAN_ABS, lse_mode=LSE_SUM_EXP, eps=1e-6, flags=0, workspace=None, stream=None) -> None:
+    st = BlockState(x_ref.data_ptr(), lse_cache.data_ptr(), None if n_skip is None else n_skip.data_ptr(), y_cache.data_ptr())
+    _check(lib().astraea_block_step(_ptr(x), ctypes.byref(weights), ctypes.byref(st), _ptr(text_k), _ptr(text_v), N_text,
+                                    _ptr(score), _ptr(idx_sel), _ptr(idx_rem), B, H, N, N_sel, d, k_keep, w_alpha, w_beta,
+                                    delta_mode, lse_mode, eps, flags, _ptr(workspace),
+                                    workspace.numel() if workspace is not None else 0, _stream(stream)))
 
 
 def astraea_step(x_cur, x_ref, lse_cache, n_skip, q, k, v, out_cache, score, idx_sel, idx_rem,

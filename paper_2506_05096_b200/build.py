@@ -11,7 +11,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libastraea.so")
-SOURCES = ["api.cu", "score.cu", "select.cu", "scatter.cu", "attn.cu", "linear.cu"]
+SOURCES = ["api.cu", "score.cu", "select.cu", "scatter.cu", "attn.cu", "linear.cu", "elementwise.cu"]
 HEADERS = ["common.cuh", "sm100_ptx.cuh", "bounded_wait.cuh", os.path.join("..", "..", "include", "astraea.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-cudart", "static"]

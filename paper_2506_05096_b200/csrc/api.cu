@@ -81,6 +81,7 @@ size_t astraea_workspace_bytes(int op, int B, int H, int N, int M, int d) {
     case ASTRAEA_OP_SPARSE_ATTN_KV: return attn_kv_workspace_bytes(B, H, M, d);
     case ASTRAEA_OP_STEP: return attn_workspace_bytes(B, H, N, M, d) + align_up(select_workspace_bytes(B, N), 256);
     case ASTRAEA_OP_GATHERED_LINEAR: return linear_workspace_bytes();
+    case ASTRAEA_OP_LAYERNORM: return 256;
     default: return 0;
     }
 }
@@ -220,26 +221,143 @@ int32_t astraea_scatter_reuse(void *cache, const void *rows, const int32_t *idx,
     return launch_scatter(cache, rows, idx, B, N, M, row_elems, flags, reinterpret_cast<int *>(err_workspace), (cudaStream_t)stream);
 }
 
-int32_t astraea_gathered_linear(const void *x, const int32_t *idx, int M, const void *w, const void *bias,
-                                void *y, int B, int N, int K, int N_out, uint32_t flags,
-                                void *workspace, size_t workspace_bytes, void *stream)
+int32_t astraea_gathered_linear_residual(const void *x, const int32_t *idx, int M, const void *w, const void *bias,
+                                         const void *residual, const void *gate,
+                                         void *y, int B, int N, int K, int N_out, uint32_t flags,
+                                         void *workspace, size_t workspace_bytes, void *stream)
 {
     REQUIRE(B > 0 && N > 0 && K > 0 && N_out > 0, "astraea_gathered_linear: B, N, K, N_out must be positive");
     REQUIRE(!idx || (M >= 0 && M <= N), "astraea_gathered_linear: M=%d outside [0, N=%d]", M, N);
     REQUIRE(K % 64 == 0, "astraea_gathered_linear: K=%d must be a multiple of 64", K);
     REQUIRE(N_out % 8 == 0, "astraea_gathered_linear: N_out=%d must be a multiple of 8", N_out);
-    if (flags & ~(ASTRAEA_LINEAR_COMPACT_OUT | ASTRAEA_LINEAR_COMPACT_IN | ASTRAEA_LINEAR_GELU))
+    if (flags & ~(ASTRAEA_LINEAR_COMPACT_OUT | ASTRAEA_LINEAR_COMPACT_IN | ASTRAEA_LINEAR_GELU | ASTRAEA_LINEAR_COMPACT_RES))
         return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_gathered_linear: unknown flags 0x%x", flags);
-    REQUIRE(!(flags & (ASTRAEA_LINEAR_COMPACT_OUT | ASTRAEA_LINEAR_COMPACT_IN)) || idx, "astraea_gathered_linear: compact rows need an index list");
+    REQUIRE(!(flags & (ASTRAEA_LINEAR_COMPACT_OUT | ASTRAEA_LINEAR_COMPACT_IN | ASTRAEA_LINEAR_COMPACT_RES)) || idx,
+            "astraea_gathered_linear: compact rows need an index list");
+    REQUIRE(!(flags & ASTRAEA_LINEAR_COMPACT_RES) || residual, "astraea_gathered_linear: ASTRAEA_LINEAR_COMPACT_RES without a residual");
     if (!workspace || workspace_bytes < linear_workspace_bytes())
         return fail(ASTRAEA_ERR_WORKSPACE_TOO_SMALL, "astraea_gathered_linear: workspace of %zu bytes, need %zu",
                     workspace_bytes, linear_workspace_bytes());
     REQUIRE((reinterpret_cast<uintptr_t>(workspace) & 255u) == 0, "astraea_gathered_linear: workspace must be 256-byte aligned");
     if (idx && M == 0) return ASTRAEA_OK;
     REQUIRE(x && w && y, "astraea_gathered_linear: null x, w or y");
-    REQUIRE(aligned16(x) && aligned16(w) && aligned16(y) && aligned16(bias), "astraea_gathered_linear: x, w, bias, y must be 16-byte aligned");
+    REQUIRE(aligned16(x) && aligned16(w) && aligned16(y) && aligned16(bias) && aligned16(residual) && aligned16(gate),
+            "astraea_gathered_linear: x, w, bias, residual, gate, y must be 16-byte aligned");
     return launch_gathered_linear(x, idx, M, w, bias, y, B, N, K, N_out, flags, reinterpret_cast<int *>(workspace),
-                                  (cudaStream_t)stream);
+                                  (cudaStream_t)stream, residual, gate);
+}
+
+int32_t astraea_gathered_linear(const void *x, const int32_t *idx, int M, const void *w, const void *bias,
+                                void *y, int B, int N, int K, int N_out, uint32_t flags,
+                                void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (flags & ASTRAEA_LINEAR_COMPACT_RES) return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_gathered_linear: unknown flags 0x%x", flags);
+    return astraea_gathered_linear_residual(x, idx, M, w, bias, nullptr, nullptr, y, B, N, K, N_out, flags, workspace,
+                                            workspace_bytes, stream);
+}
+
+int32_t astraea_layernorm_modulate(const void *x, const int32_t *idx, int M, const void *scale, const void *shift,
+                                   void *y, int B, int N, int D, float eps, uint32_t flags,
+                                   void *err_workspace, void *stream)
+{
+    REQUIRE(B > 0 && N > 0 && D > 0, "astraea_layernorm_modulate: B, N, D must be positive");
+    REQUIRE(D % 8 == 0, "astraea_layernorm_modulate: D=%d must be a multiple of 8", D);
+    REQUIRE(!idx || (M >= 0 && M <= N), "astraea_layernorm_modulate: M=%d outside [0, N=%d]", M, N);
+    REQUIRE(eps >= 0.f, "astraea_layernorm_modulate: eps must be >= 0");
+    if (flags & ~(ASTRAEA_LN_COMPACT_IN | ASTRAEA_LN_COMPACT_OUT))
+        return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_layernorm_modulate: unknown flags 0x%x", flags);
+    REQUIRE(!flags || idx, "astraea_layernorm_modulate: compact rows need an index list");
+    if (idx && M == 0) return ASTRAEA_OK;
+    REQUIRE(x && y, "astraea_layernorm_modulate: null x or y");
+    REQUIRE(aligned16(x) && aligned16(y) && aligned16(scale) && aligned16(shift), "astraea_layernorm_modulate: pointers must be 16-byte aligned");
+    REQUIRE((reinterpret_cast<uintptr_t>(err_workspace) & 3u) == 0, "astraea_layernorm_modulate: err_workspace must be 4-byte aligned");
+    return launch_layernorm_modulate(x, idx, M, scale, shift, y, B, N, D, eps, flags, reinterpret_cast<int *>(err_workspace),
+                                     (cudaStream_t)stream);
+}
+
+// ------------------------------------------------------------------ a whole compute block
+// workspace: [256 bytes: error word] [select scratch] [5 token-sized buffers] [hidden-sized buffer]
+static size_t block_buffer_bytes(int B, int N, int width) { return align_up((size_t)B * N * width * 2, 256); }
+
+size_t astraea_block_workspace_bytes(int B, int H, int N, int d, int hidden)
+{
+    if (B <= 0 || H <= 0 || N <= 0 || d <= 0 || hidden <= 0) return 0;
+    return 256 + align_up(select_workspace_bytes(B, N), 256) + 5 * block_buffer_bytes(B, N, H * d) + block_buffer_bytes(B, N, hidden);
+}
+
+int32_t astraea_block_step(const void *x, const astraea_block_weights *w, const astraea_block_state *st,
+                           const void *text_k, const void *text_v, int N_text,
+                           float *score, int32_t *idx_sel, int32_t *idx_rem,
+                           int B, int H, int N, int N_sel, int d, int k_keep,
+                           float w_alpha, float w_beta, int delta_mode, int lse_mode, float eps, uint32_t flags,
+                           void *workspace, size_t workspace_bytes, void *stream)
+{
+    REQUIRE(x && w && st, "astraea_block_step: null x, weights or state");
+    REQUIRE(B > 0 && H > 0 && N > 0 && d > 0 && N_text > 0, "astraea_block_step: B, H, N, d, N_text must be positive");
+    REQUIRE(N_sel >= 0 && N_sel <= N, "astraea_block_step: N_sel=%d outside [0, N=%d]", N_sel, N);
+    REQUIRE(k_keep >= 0 && k_keep <= N_sel, "astraea_block_step: k_keep=%d outside [0, N_sel=%d]", k_keep, N_sel);
+    if (flags & ~ASTRAEA_BLOCK_REUSE_SELECTION) return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_block_step: unknown flags 0x%x", flags);
+    const int D = H * d, hidden = w->hidden;
+    REQUIRE(D % 64 == 0 && hidden > 0 && hidden % 64 == 0, "astraea_block_step: D=%d and hidden=%d must be multiples of 64", D, hidden);
+    REQUIRE(w->wq && w->wk && w->wv && w->wo && w->wq2 && w->wo2 && w->w1 && w->w2, "astraea_block_step: null weight matrix");
+    REQUIRE(st->x_ref && st->lse_cache && st->y_cache, "astraea_block_step: null state buffer");
+    REQUIRE(text_k && text_v, "astraea_block_step: null text keys / values");
+    const size_t need = astraea_block_workspace_bytes(B, H, N, d, hidden);
+    if (!workspace || workspace_bytes < need)
+        return fail(ASTRAEA_ERR_WORKSPACE_TOO_SMALL, "astraea_block_step: workspace of %zu bytes, need %zu", workspace_bytes, need);
+    REQUIRE((reinterpret_cast<uintptr_t>(workspace) & 255u) == 0, "astraea_block_step: workspace must be 256-byte aligned");
+    const int n_always = N - N_sel, M = k_keep + n_always;
+    REQUIRE(score && (idx_sel || M == 0), "astraea_block_step: null score or idx_sel");
+    char *ws = reinterpret_cast<char *>(workspace);
+    void *err = ws;                                     // the error word of every call below
+    char *p = ws + 256;
+    void *sel_ws = p; p += align_up(select_workspace_bytes(B, N), 256);
+    const size_t tb = block_buffer_bytes(B, N, D);
+    void *bufA = p, *bufQ = p + tb, *bufK = p + 2 * tb, *bufV = p + 3 * tb, *bufO = p + 4 * tb, *bufU = p + 5 * tb;
+    int32_t rc = ASTRAEA_OK;
+    if (!(flags & ASTRAEA_BLOCK_REUSE_SELECTION)) {
+        rc = astraea_score(x, st->x_ref, st->lse_cache, st->n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, delta_mode, lse_mode, stream);
+        if (rc == ASTRAEA_OK)
+            rc = astraea_select(score, B, N_sel, k_keep, n_always, idx_sel, idx_rem, st->n_skip, sel_ws, select_workspace_bytes(B, N), stream);
+        if (rc != ASTRAEA_OK) return rc;
+    }
+    if (M == 0) return ASTRAEA_OK;
+    const int64_t sb = (int64_t)N * D, sh = d, sn = D;
+    const int64_t tsb = (int64_t)N_text * D;
+    // self-attention group: keys / values from all tokens, everything else on the selected rows
+    rc = astraea_layernorm_modulate(x, nullptr, 0, w->s1, w->t1, bufA, B, N, D, eps, 0u, err, stream);
+    if (rc == ASTRAEA_OK) rc = astraea_gathered_linear(bufA, nullptr, 0, w->wk, w->bk, bufK, B, N, D, D, 0u, err, 256, stream);
+    if (rc == ASTRAEA_OK) rc = astraea_gathered_linear(bufA, nullptr, 0, w->wv, w->bv, bufV, B, N, D, D, 0u, err, 256, stream);
+    if (rc == ASTRAEA_OK) rc = astraea_gathered_linear(bufA, idx_sel, M, w->wq, w->bq, bufQ, B, N, D, D, 0u, err, 256, stream);
+    if (rc == ASTRAEA_OK)
+        rc = astraea_sparse_attn(bufQ, bufK, bufV, sb, sh, sn, sb, sh, sn, sb, sh, sn, idx_sel, M, nullptr, 0, bufO, st->lse_cache,
+                                 B, H, N, d, 0.f, 0u, err, 256, stream);
+    // x1 (compact, over the dead keys) = x[I] + g1 * (attention rows Wo^T + bo)
+    if (rc == ASTRAEA_OK)
+        rc = astraea_gathered_linear_residual(bufO, idx_sel, M, w->wo, w->bo, x, w->g1, bufK, B, N, D, D, ASTRAEA_LINEAR_COMPACT_OUT, err, 256, stream);
+    // cross-attention group on the compact rows
+    if (rc == ASTRAEA_OK)
+        rc = astraea_layernorm_modulate(bufK, idx_sel, M, nullptr, nullptr, bufA, B, N, D, eps, ASTRAEA_LN_COMPACT_IN | ASTRAEA_LN_COMPACT_OUT, err, stream);
+    if (rc == ASTRAEA_OK) rc = astraea_gathered_linear(bufA, idx_sel, M, w->wq2, w->bq2, bufQ, B, N, D, D, ASTRAEA_LINEAR_COMPACT_IN, err, 256, stream);
+    if (rc == ASTRAEA_OK)
+        rc = astraea_sparse_cross_attn(bufQ, text_k, text_v, sb, sh, sn, tsb, sh, sn, tsb, sh, sn, idx_sel, M, bufV, nullptr, B, H, N, N_text, d,
+                                       0.f, ASTRAEA_ATTN_COMPACT_OUT, err, 256, stream);
+    if (rc == ASTRAEA_OK)       // x2 (compact, over the dead attention rows) = x1 + cross rows Wo2^T + bo2
+        rc = astraea_gathered_linear_residual(bufV, idx_sel, M, w->wo2, w->bo2, bufK, nullptr, bufO, B, N, D, D,
+                                              ASTRAEA_LINEAR_COMPACT_IN | ASTRAEA_LINEAR_COMPACT_OUT | ASTRAEA_LINEAR_COMPACT_RES, err, 256, stream);
+    // MLP group: the hidden activations exist for the selected rows only; the result lands in the block's cache
+    if (rc == ASTRAEA_OK)
+        rc = astraea_layernorm_modulate(bufO, idx_sel, M, w->s3, w->t3, bufA, B, N, D, eps, ASTRAEA_LN_COMPACT_IN | ASTRAEA_LN_COMPACT_OUT, err, stream);
+    if (rc == ASTRAEA_OK)
+        rc = astraea_gathered_linear(bufA, idx_sel, M, w->w1, w->b1, bufU, B, N, D, hidden,
+                                     ASTRAEA_LINEAR_COMPACT_IN | ASTRAEA_LINEAR_COMPACT_OUT | ASTRAEA_LINEAR_GELU, err, 256, stream);
+    if (rc == ASTRAEA_OK)
+        rc = astraea_gathered_linear_residual(bufU, idx_sel, M, w->w2, w->b2, bufO, w->g3, st->y_cache, B, N, hidden, D,
+                                              ASTRAEA_LINEAR_COMPACT_IN | ASTRAEA_LINEAR_COMPACT_RES, err, 256, stream);
+    // the reference inputs of the tokens that were computed become the current inputs
+    if (rc == ASTRAEA_OK && !(flags & ASTRAEA_BLOCK_REUSE_SELECTION))
+        rc = astraea_scatter_reuse(st->x_ref, x, idx_sel, B, N, M, D, ASTRAEA_SCATTER_SRC_FULL, err, stream);
+    return rc;
 }
 
 int32_t astraea_step(const void *x_cur, void *x_ref, float *lse_cache, int32_t *n_skip,

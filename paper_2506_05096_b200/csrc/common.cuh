@@ -59,7 +59,10 @@ int32_t launch_scatter(void *cache, const void *rows, const int32_t *idx, int B,
 
 size_t linear_workspace_bytes();
 int32_t launch_gathered_linear(const void *x, const int32_t *idx, int M, const void *w, const void *bias, void *y,
-                               int B, int N, int K, int N_out, uint32_t flags, int *err_word, cudaStream_t stream);
+                               int B, int N, int K, int N_out, uint32_t flags, int *err_word, cudaStream_t stream,
+                               const void *residual = nullptr, const void *gate = nullptr);
+int32_t launch_layernorm_modulate(const void *x, const int32_t *idx, int M, const void *scale, const void *shift, void *y,
+                                  int B, int N, int D, float eps, uint32_t flags, int *err_word, cudaStream_t stream);
 
 struct AttnArgs {
     const void *q, *k, *v;

@@ -51,6 +51,9 @@ struct LinParams {
     int compact;                 // y is [B, M, N_out]
     int compact_in;              // x is [B, M, K]
     int gelu;                    // y = GELU(x W^T + bias), exact (erf) form
+    const __nv_bfloat16 *residual;   // added to the result after the gate; [B, N, N_out] rows at idx, or compact [B, M, N_out]
+    int res_compact;
+    const __nv_bfloat16 *gate;       // [B, N_out]: multiplies act(x W^T + bias) before the residual is added
     int *err_word;
 };
 
@@ -71,14 +74,18 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *m, 
 }
 
 // row of x that holds the g-th listed row (all batch elements in one list): -1 past the end, -2 for an index
-// outside [0, N) or one that does not exceed its predecessor; *out_row is the row of y it goes to
-__device__ __forceinline__ long long source_row(const LinParams &p, long long g, long long total, long long *out_row) {
+// outside [0, N) or one that does not exceed its predecessor; *out_row is the row of y it goes to, *res_row the row
+// of the residual, *batch the batch element
+__device__ __forceinline__ long long source_row(const LinParams &p, long long g, long long total, long long *out_row,
+                                                long long *res_row = nullptr, int *batch = nullptr) {
     if (g >= total) return -1;
     const int b = (int)(g / p.M), r = (int)(g - (long long)b * p.M);
     const int tok = p.idx ? __ldg(p.idx + g) : r;
     if ((unsigned)tok >= (unsigned)p.N) return -2;
     if (p.idx && r > 0 && __ldg(p.idx + g - 1) >= tok) return -2;      // not strictly ascending: a row would be written twice
     if (out_row) *out_row = p.compact ? g : (long long)b * p.N + tok;
+    if (res_row) *res_row = p.res_compact ? g : (long long)b * p.N + tok;
+    if (batch) *batch = b;
     return p.compact_in ? g : (long long)b * p.N + tok;
 }
 
@@ -127,10 +134,13 @@ gathered_linear_kernel(const __grid_constant__ CUtensorMap tmap_w, const LinPara
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
             const int tm = tile / tiles_n, tn = tile - tm * tiles_n;
             const int acc = it % kAccSets, n0 = tn * kBN;
-            long long out_row = -1;
-            const long long src = source_row(p, (long long)tm * kBM + row, total_rows, &out_row);
+            long long out_row = -1, res_row = -1;
+            int batch = 0;
+            const long long src = source_row(p, (long long)tm * kBM + row, total_rows, &out_row, &res_row, &batch);
             if (src == -2 && tn == 0) atomicExch(p.err_word, kErrBadIndex);
             __nv_bfloat16 *dst = (src >= 0) ? p.y + out_row * p.N_out + n0 : nullptr;
+            const __nv_bfloat16 *res = (src >= 0 && p.residual) ? p.residual + res_row * p.N_out : nullptr;
+            const __nv_bfloat16 *gate = p.gate ? p.gate + (long long)batch * p.N_out : nullptr;
             wait_bar(bar_acc_full + 8 * acc, (it / kAccSets) & 1, &abort_flag, p.err_word);
             tc_fence_after();
             if (abort_flag) dst = nullptr;
@@ -163,6 +173,24 @@ gathered_linear_kernel(const __grid_constant__ CUtensorMap tmap_w, const LinPara
                     if (p.gelu) {
 #pragma unroll
                         for (int i = 0; i < 8; ++i) f[i] = 0.5f * f[i] * (1.0f + erff(f[i] * 0.70710678118654752f));
+                    }
+                    if (gate) {
+                        const uint4 gg = __ldg(reinterpret_cast<const uint4 *>(gate + col));
+                        const uint32_t gw[4] = {gg.x, gg.y, gg.z, gg.w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            f[2 * i] *= __uint_as_float(gw[i] << 16);
+                            f[2 * i + 1] *= __uint_as_float(gw[i] & 0xffff0000u);
+                        }
+                    }
+                    if (res) {
+                        const uint4 rr = __ldg(reinterpret_cast<const uint4 *>(res + col));
+                        const uint32_t rw[4] = {rr.x, rr.y, rr.z, rr.w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            f[2 * i] += __uint_as_float(rw[i] << 16);
+                            f[2 * i + 1] += __uint_as_float(rw[i] & 0xffff0000u);
+                        }
                     }
                     uint32_t w[4];
 #pragma unroll
@@ -262,7 +290,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 size_t linear_workspace_bytes() { return 256; }
 
 int32_t launch_gathered_linear(const void *x, const int32_t *idx, int M, const void *w, const void *bias, void *y,
-                               int B, int N, int K, int N_out, uint32_t flags, int *err_word, cudaStream_t stream)
+                               int B, int N, int K, int N_out, uint32_t flags, int *err_word, cudaStream_t stream,
+                               const void *residual, const void *gate)
 {
     const EncodeTiledFn enc = reinterpret_cast<EncodeTiledFn>(tensor_map_encoder());
     if (!enc) return fail(ASTRAEA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
@@ -289,6 +318,9 @@ int32_t launch_gathered_linear(const void *x, const int32_t *idx, int M, const v
     p.compact = (flags & ASTRAEA_LINEAR_COMPACT_OUT) ? 1 : 0;
     p.compact_in = (flags & ASTRAEA_LINEAR_COMPACT_IN) ? 1 : 0;
     p.gelu = (flags & ASTRAEA_LINEAR_GELU) ? 1 : 0;
+    p.residual = reinterpret_cast<const __nv_bfloat16 *>(residual);
+    p.res_compact = (flags & ASTRAEA_LINEAR_COMPACT_RES) ? 1 : 0;
+    p.gate = reinterpret_cast<const __nv_bfloat16 *>(gate);
     p.err_word = err_word;
     const long long rows = (long long)B * p.M;
     const long long tiles = ((rows + kBM - 1) / kBM) * ((N_out + kBN - 1) / kBN);
