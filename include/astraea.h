@@ -67,6 +67,13 @@ extern "C" {
 /* flags of astraea_block_step */
 #define ASTRAEA_BLOCK_REUSE_SELECTION 1u     /* idx_sel already holds this step's selection (made by another block): no scoring,
                                               * no selection, counters and reference inputs untouched (the Fixed-token variant) */
+#define ASTRAEA_BLOCK_SELECT_QK   2u         /* keys and values of the self-attention are restricted to the selected tokens as well
+                                              * (and projected for them only): the SelectQ&K variant of the ablation study, Table 2 */
+/* variants of astraea_model_schedule_create: the rows of the ablation study (Table 2) */
+#define ASTRAEA_VARIANT_TOKEN_WISE  0        /* the paper's method: every block scores and selects its own tokens at every step */
+#define ASTRAEA_VARIANT_SELECT_QK   1        /* as above, with the self-attention also restricted to the selected keys / values */
+#define ASTRAEA_VARIANT_TIMESTEP    2        /* Timestep-level: a step computes all tokens or none (budgets must be 0 or N_sel) */
+#define ASTRAEA_VARIANT_FIXED_TOKEN 3        /* Fixed-token: block 0 selects, the other blocks of the step reuse its selection */
 /* flags of astraea_scatter_reuse */
 #define ASTRAEA_SCATTER_SRC_FULL  1u         /* rows is [B,N,row_elems]; row idx[r] of it is copied to row idx[r] of cache */
 
@@ -293,6 +300,7 @@ int32_t astraea_layernorm_modulate(const void *x, const int32_t *idx, int M, con
  * [B, D]; any bias or modulation pointer may be NULL.  text_k, text_v: [B, N_text, H, d] (projected once per
  * generation by the caller).  State (in/out): x_ref [B,N,D], lse_cache fp32 [B,H,N], n_skip int32 [B,N_sel], y_cache
  * [B,N,D] = the block's output after the call.  score / idx_sel / idx_rem as astraea_step.
+ * flags: ASTRAEA_BLOCK_REUSE_SELECTION, ASTRAEA_BLOCK_SELECT_QK (see there).
  * workspace: astraea_block_workspace_bytes(B, H, N, d, hidden) bytes, 256-byte aligned, zero before the first use.
  * D = H*d must be a multiple of 64 and at most 4096, hidden a multiple of 64.
  * k_keep = 0 with no always-kept tokens: only scores and counters change.
@@ -315,6 +323,44 @@ int32_t astraea_block_step(const void *x, const astraea_block_weights *weights, 
                            int B, int H, int N, int N_sel, int d, int k_keep,
                            float w_alpha, float w_beta, int delta_mode, int lse_mode, float eps, uint32_t flags,
                            void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * A generation as ONE CUDA graph: T denoising steps x L compute blocks (the execution flow of Section 3.2 with the
+ * per-step budgets theta_t of the search space of Section 3.3, fixed before the generation starts).  At step t block
+ * 0 reads x_in[t]; block l > 0 reads block l-1's merged output of the same step (its y_cache: computed rows + reused
+ * rows); every block keeps its own state (reference inputs, LSE cache, counters, output cache) and, per block,
+ * score / idx_sel / idx_rem buffers that hold its last selection.  `variant` picks the row of the ablation study
+ * (Table 2): the paper's token-wise method, SelectQ&K, Timestep-level (every budget 0 or N_sel: the policy
+ * astraea_timestep_level_budgets makes such a schedule from a token-wise one) or Fixed-token (block 0's selection is
+ * shared by all blocks of the step; the other blocks' counters and reference inputs are not used).
+ *   k_keep : HOST int32 [T]                     x_in : HOST array of T device pointers, bf16 [B,N,D] each
+ *   weights, states : HOST arrays of L structs  text_k, text_v : HOST arrays of L device pointers, bf16 [B,N_text,H,d]
+ *   score, idx_sel, idx_rem : HOST arrays of L device pointers (fp32 [B,N_sel]; int32 [B,N]; int32 [B,N_sel] or NULL)
+ *   workspace : astraea_block_workspace_bytes(...) bytes, shared by all blocks (they run one after the other)
+ * The first step of a generation should carry k_keep = N_sel.  The graph keeps the pointers, not the data.
+ * astraea_model_schedule_launch enqueues the whole generation with one graph launch; the last block's y_cache then
+ * holds the output of the last step.  Errors: as astraea_block_step, INVALID_ARG for a budget the variant does not
+ * allow, CUDA for a failed capture.
+ */
+typedef struct astraea_model_schedule astraea_model_schedule;
+int32_t astraea_model_schedule_create(astraea_model_schedule **schedule, int L, int T, const int32_t *k_keep,
+                                      const void *const *x_in, const astraea_block_weights *weights,
+                                      const astraea_block_state *states, const void *const *text_k,
+                                      const void *const *text_v, int N_text,
+                                      float *const *score, int32_t *const *idx_sel, int32_t *const *idx_rem,
+                                      int B, int H, int N, int N_sel, int d,
+                                      float w_alpha, float w_beta, int delta_mode, int lse_mode, float eps, int variant,
+                                      void *workspace, size_t workspace_bytes);
+int32_t astraea_model_schedule_launch(astraea_model_schedule *schedule, void *stream);
+void    astraea_model_schedule_destroy(astraea_model_schedule *schedule);
+
+/*
+ * Host policy of the Timestep-level variant (ablation study, Table 2): turns a token-wise budget schedule into one
+ * whose steps compute all tokens or none, with the same total budget up to one step: the budgets are accumulated and
+ * a step computes everything as soon as the accumulated budget covers N_sel tokens (the first step always does).
+ *   k_keep, out : HOST int32 [T] (may be the same array).  Returns the number of computed steps, or INVALID_ARG.
+ */
+int32_t astraea_timestep_level_budgets(const int32_t *k_keep, int T, int N_sel, int32_t *out);
 
 /*
  * One whole step of one attention block on device buffers (Algorithm 1 with given Q, K, V):

@@ -226,7 +226,8 @@ def take_rows(a, idx):
 
 
 def block_step(x, x_ref, lse_cache, n_skip, y_cache, weights, text_k, text_v, H, k_keep, n_always=0,
-               w_alpha=1.0, w_beta=1.0, delta_mode=0, lse_mode=0, eps=1e-6, forced_sel=None, rounder=None):
+               w_alpha=1.0, w_beta=1.0, delta_mode=0, lse_mode=0, eps=1e-6, forced_sel=None, rounder=None,
+               select_qk=False, shared_sel=None):
     """One transformer block at one denoising step with token-wise reuse (Algorithm 1 and the execution flow of
     Section 3.2 applied to a whole compute block): the tokens are scored on the block's input and selected;
     keys and values come from ALL tokens of the current step; the query projection, the self-attention rows, the
@@ -244,6 +245,9 @@ def block_step(x, x_ref, lse_cache, n_skip, y_cache, weights, text_k, text_v, H,
     [out]) and the modulation vectors s1, t1, g1, s3, t3, g3 ([B, D], any of them None).  text_k, text_v: [B, N_text, H, d].
     rounder: None, or a function applied to every intermediate tensor that the device stores as bf16 (the parity
     tests pass the bf16 rounding there, so that the oracle follows the device's storage precision layer by layer).
+    select_qk: the SelectQ&K variant of the ablation study (Table 2): the self-attention's keys and values are
+    restricted to the selected tokens as well.  shared_sel [B, M]: the Fixed-token variant: the selection was made by
+    another block of this step; nothing is scored here, counters and reference inputs stay as they are.
     Returns a dict: idx_sel, idx_rem, n_skip, score, y (new cache), lse, x_ref, and the intermediates.
     """
     rd = (lambda a: a) if rounder is None else rounder
@@ -252,9 +256,14 @@ def block_step(x, x_ref, lse_cache, n_skip, y_cache, weights, text_k, text_v, H,
     d = D // H
     n_sel = N - n_always
     w = weights
-    s64 = score(x, x_ref, lse_cache, n_skip, n_sel=n_sel, w_alpha=w_alpha, w_beta=w_beta, delta_mode=delta_mode, lse_mode=lse_mode)
-    idx_sel, idx_rem, n_new = select(s64.astype(np.float32), k_keep, n_always, n_skip)
-    own = idx_sel
+    if shared_sel is not None:
+        idx_sel = own = _i32(shared_sel)
+        s64, idx_rem, forced_sel = None, None, None
+        n_new = None if n_skip is None else np.array(n_skip, dtype=np.int32, copy=True)
+    else:
+        s64 = score(x, x_ref, lse_cache, n_skip, n_sel=n_sel, w_alpha=w_alpha, w_beta=w_beta, delta_mode=delta_mode, lse_mode=lse_mode)
+        idx_sel, idx_rem, n_new = select(s64.astype(np.float32), k_keep, n_always, n_skip)
+        own = idx_sel
     if forced_sel is not None:
         idx_sel = _i32(forced_sel)
         chosen = np.zeros((B, N), dtype=bool)
@@ -270,10 +279,11 @@ def block_step(x, x_ref, lse_cache, n_skip, y_cache, weights, text_k, text_v, H,
                    x_ref=np.array(x_ref, dtype=np.float64, copy=True))
         return res
     h = rd(layernorm_modulate(x, w.get("s1"), w.get("t1"), eps))
-    k = rd(gathered_linear(h, w["wk"], w.get("bk")))
-    v = rd(gathered_linear(h, w["wv"], w.get("bv")))
-    q = rd(gathered_linear(h, w["wq"], w.get("bq"), idx_sel))                     # rows outside idx_sel stay zero and are never read
-    a, l, _ = sparse_attn(q.reshape(B, N, H, d), k.reshape(B, N, H, d), v.reshape(B, N, H, d), q_idx=idx_sel)
+    kv_rows = idx_sel if select_qk else None                                      # rows outside a list stay zero and are never read
+    k = rd(gathered_linear(h, w["wk"], w.get("bk"), kv_rows))
+    v = rd(gathered_linear(h, w["wv"], w.get("bv"), kv_rows))
+    q = rd(gathered_linear(h, w["wq"], w.get("bq"), idx_sel))
+    a, l, _ = sparse_attn(q.reshape(B, N, H, d), k.reshape(B, N, H, d), v.reshape(B, N, H, d), q_idx=idx_sel, kv_idx=kv_rows)
     a = rd(a.reshape(B, M, D))
     o = gathered_linear(a, w["wo"], w.get("bo"))
     if w.get("g1") is not None:
@@ -292,5 +302,46 @@ def block_step(x, x_ref, lse_cache, n_skip, y_cache, weights, text_k, text_v, H,
     x3 = rd(x2 + m)
     res.update(h=h, k=k, v=v, q_rows=take_rows(q, idx_sel), attn_rows=a, x1=x1, h2=h2, q2=q2, cross_rows=c, x2=x2, h3=h3, u=u, x3=x3,
                y=scatter_reuse(y_cache, x3, idx_sel), lse=scatter_lse(lse_cache, l, idx_sel),
-               x_ref=scatter_reuse(x_ref, take_rows(x, idx_sel), idx_sel))
+               x_ref=(np.array(x_ref, dtype=np.float64, copy=True) if shared_sel is not None
+                      else scatter_reuse(x_ref, take_rows(x, idx_sel), idx_sel)))
     return res
+
+
+def timestep_level_budgets(k_keep, n_sel):
+    """Host policy of the Timestep-level variant (ablation study, Table 2): every step computes all tokens or none.
+    The token-wise budgets are accumulated; a step computes everything once the accumulated budget covers all n_sel
+    tokens, and the first step always does."""
+    out, carry = [], 0
+    for t, k in enumerate(k_keep):
+        carry += int(k)
+        if t == 0 or (n_sel > 0 and carry >= n_sel):
+            out.append(n_sel)
+            carry = max(0, carry - n_sel)
+        else:
+            out.append(0)
+    return out
+
+
+VARIANT_TOKEN_WISE, VARIANT_SELECT_QK, VARIANT_TIMESTEP, VARIANT_FIXED_TOKEN = 0, 1, 2, 3
+
+
+def model_step(x_in, blocks, states, text_k, text_v, H, k_keep, n_always=0, variant=0, forced_sels=None, rounder=None, **kw):
+    """One denoising step through L compute blocks (execution flow of Section 3.2): block 0 reads x_in, block l > 0
+    the merged output (computed + reused rows) of block l-1.  blocks: list of weight dicts; states: list of dicts
+    with x_ref, lse, n_skip, y.  variant: the rows of the ablation study (Table 2): 0 token-wise (every block scores and
+    selects), 1 SelectQ&K, 2 Timestep-level (k_keep must be 0 or all), 3 Fixed-token (block 0's selection is shared by
+    the other blocks of the step).  forced_sels: per block, a selection to adopt (tests, near-ties).  Returns the list
+    of per-block result dicts; `states` is not modified."""
+    n_sel = np.asarray(x_in).shape[1] - n_always
+    if variant == VARIANT_TIMESTEP:
+        assert k_keep in (0, n_sel), "the Timestep-level variant computes all tokens or none"
+    outs, x = [], x_in
+    for l, (w, st) in enumerate(zip(blocks, states)):
+        shared = outs[0]["idx_sel"] if (variant == VARIANT_FIXED_TOKEN and l > 0) else None
+        forced = None if forced_sels is None else forced_sels[l]
+        r = block_step(x, st["x_ref"], st["lse"], st["n_skip"], st["y"], w, text_k[l], text_v[l], H, k_keep, n_always,
+                       forced_sel=None if shared is not None else forced, rounder=rounder,
+                       select_qk=(variant == VARIANT_SELECT_QK), shared_sel=shared, **kw)
+        outs.append(r)
+        x = r["y"] if rounder is None else rounder(r["y"])
+    return outs

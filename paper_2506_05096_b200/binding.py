@@ -24,7 +24,8 @@ ATTN_SMALL_CTAS = 2
 SCATTER_SRC_FULL = 1
 LINEAR_COMPACT_OUT, LINEAR_COMPACT_IN, LINEAR_GELU, LINEAR_COMPACT_RES = 1, 2, 4, 8
 LN_COMPACT_IN, LN_COMPACT_OUT = 1, 2
-BLOCK_REUSE_SELECTION = 1
+BLOCK_REUSE_SELECTION, BLOCK_SELECT_QK = 1, 2
+VARIANT_TOKEN_WISE, VARIANT_SELECT_QK, VARIANT_TIMESTEP, VARIANT_FIXED_TOKEN = 0, 1, 2, 3
 OP_SELECT, OP_SPARSE_ATTN, OP_STEP, OP_SPARSE_ATTN_KV, OP_GATHERED_LINEAR, OP_LAYERNORM = 1, 2, 3, 4, 5, 6
 N_SKIP_CLAMP = 80
 NOALLOC_SCRATCH_BYTES = 4096
@@ -32,7 +33,8 @@ NOALLOC_SCRATCH_BYTES = 4096
 EXPORTS = [
     "astraea_score", "astraea_select", "astraea_sparse_attn", "astraea_sparse_cross_attn", "astraea_sparse_attn_noalloc", "astraea_scatter_reuse", "astraea_step",
     "astraea_gathered_linear", "astraea_gathered_linear_residual", "astraea_layernorm_modulate",
-    "astraea_block_step", "astraea_block_workspace_bytes", "astraea_schedule_create", "astraea_schedule_launch", "astraea_schedule_destroy",
+    "astraea_block_step", "astraea_block_workspace_bytes", "astraea_model_schedule_create", "astraea_model_schedule_launch",
+    "astraea_model_schedule_destroy", "astraea_timestep_level_budgets", "astraea_schedule_create", "astraea_schedule_launch", "astraea_schedule_destroy",
     "astraea_session_create", "astraea_session_destroy", "astraea_step_host",
     "astraea_workspace_bytes", "astraea_budget_to_k", "astraea_poll_error",
     "astraea_last_error", "astraea_version",
@@ -83,6 +85,13 @@ def lib() -> ctypes.CDLL:
         L.astraea_layernorm_modulate.argtypes = [c_p, c_p, c_i, c_p, c_p, c_p, c_i, c_i, c_i, c_f, c_u, c_p, c_p]
         L.astraea_block_step.argtypes = [c_p, ctypes.POINTER(BlockWeights), ctypes.POINTER(BlockState), c_p, c_p, c_i, c_p, c_p, c_p,
                                          c_i, c_i, c_i, c_i, c_i, c_i, c_f, c_f, c_i, c_i, c_f, c_u, c_p, c_sz, c_p]
+        L.astraea_model_schedule_create.argtypes = [ctypes.POINTER(c_p), c_i, c_i, c_p, c_p, ctypes.POINTER(BlockWeights),
+                                                    ctypes.POINTER(BlockState), c_p, c_p, c_i, c_p, c_p, c_p,
+                                                    c_i, c_i, c_i, c_i, c_i, c_f, c_f, c_i, c_i, c_f, c_i, c_p, c_sz]
+        L.astraea_model_schedule_launch.argtypes = [c_p, c_p]
+        L.astraea_model_schedule_destroy.argtypes = [c_p]
+        L.astraea_model_schedule_destroy.restype = None
+        L.astraea_timestep_level_budgets.argtypes = [c_p, c_i, c_i, c_p]
         L.astraea_block_workspace_bytes.argtypes = [c_i] * 5
         L.astraea_block_workspace_bytes.restype = c_sz
         L.astraea_step.argtypes = [c_p] * 11 + [c_i] * 6 + [c_f, c_f, c_i, c_i, c_p, c_sz, c_p]
@@ -102,7 +111,8 @@ def lib() -> ctypes.CDLL:
         L.astraea_last_error.restype = ctypes.c_char_p
         L.astraea_version.restype = ctypes.c_char_p
         for name in ("astraea_score", "astraea_select", "astraea_sparse_attn", "astraea_sparse_cross_attn", "astraea_sparse_attn_noalloc", "astraea_scatter_reuse",
-                     "astraea_step", "astraea_gathered_linear", "astraea_gathered_linear_residual", "astraea_layernorm_modulate", "astraea_block_step", "astraea_schedule_create", "astraea_schedule_launch",
+                     "astraea_step", "astraea_gathered_linear", "astraea_gathered_linear_residual", "astraea_layernorm_modulate", "astraea_block_step", "astraea_model_schedule_create", "astraea_model_schedule_launch",
+                     "astraea_timestep_level_budgets", "astraea_schedule_create", "astraea_schedule_launch",
                      "astraea_session_create", "astraea_step_host", "astraea_budget_to_k",
                      "astraea_poll_error"):
             getattr(L, name).restype = ctypes.c_int32
@@ -253,6 +263,55 @@ def astraea_step(x_cur, x_ref, lse_cache, n_skip, q, k, v, out_cache, score, idx
 
 def astraea_poll_error(workspace, stream=None) -> None:
     _check(lib().astraea_poll_error(_ptr(workspace), _stream(stream)))
+
+
+def astraea_timestep_level_budgets(k_keep, N_sel: int):
+    """The all-or-nothing schedule of the Timestep-level variant made from a token-wise one (host policy)."""
+    T = len(k_keep)
+    src = (ctypes.c_int32 * T)(*[int(a) for a in k_keep])
+    out = (ctypes.c_int32 * T)()
+    rc = lib().astraea_timestep_level_budgets(src, T, N_sel, out)
+    if rc < 0:
+        raise AstraeaError(rc, lib().astraea_last_error().decode())
+    return list(out)
+
+
+class ModelSchedule:
+    """A generation of T steps x L compute blocks as one CUDA graph (astraea_model_schedule_*).
+    x_in: list of T device tensors; weights: list of L (dict of device tensors, hidden); states: list of L dicts with
+    x_ref, lse_cache, n_skip, y_cache, score, idx_sel, idx_rem (idx_rem may be None); text_k / text_v: lists of L tensors."""
+
+    def __init__(self, k_keep, x_in, weights, states, text_k, text_v, N_text, B, H, N, N_sel, d, w_alpha=1.0, w_beta=1.0,
+                 delta_mode=DELTA_MEAN_ABS, lse_mode=LSE_SUM_EXP, eps=1e-6, variant=VARIANT_TOKEN_WISE, workspace=None):
+        T, L = len(k_keep), len(weights)
+        assert len(x_in) == T and len(states) == L and len(text_k) == L and len(text_v) == L
+        self._keep = (list(x_in), weights, states, list(text_k), list(text_v), workspace)   # the graph keeps pointers
+        kk = (ctypes.c_int32 * T)(*[int(a) for a in k_keep])
+        xs = (ctypes.c_void_p * T)(*[t.data_ptr() for t in x_in])
+        W = (BlockWeights * L)(*[block_weights(w, hidden) for (w, hidden) in weights])
+        S = (BlockState * L)(*[BlockState(s["x_ref"].data_ptr(), s["lse_cache"].data_ptr(), s["n_skip"].data_ptr(), s["y_cache"].data_ptr())
+                               for s in states])
+        ptrs = lambda lst: (ctypes.c_void_p * L)(*[None if t is None else t.data_ptr() for t in lst])
+        rem = None if all(s.get("idx_rem") is None for s in states) else ptrs([s.get("idx_rem") for s in states])
+        self._h = ctypes.c_void_p()
+        _check(lib().astraea_model_schedule_create(ctypes.byref(self._h), L, T, kk, xs, W, S, ptrs(text_k), ptrs(text_v), N_text,
+                                                   ptrs([s["score"] for s in states]), ptrs([s["idx_sel"] for s in states]), rem,
+                                                   B, H, N, N_sel, d, w_alpha, w_beta, delta_mode, lse_mode, eps, variant,
+                                                   _ptr(workspace), workspace.numel() if workspace is not None else 0))
+
+    def launch(self, stream=None) -> None:
+        _check(lib().astraea_model_schedule_launch(self._h, _stream(stream)))
+
+    def close(self) -> None:
+        if getattr(self, "_h", None):
+            lib().astraea_model_schedule_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 class Schedule:

@@ -276,13 +276,17 @@ int32_t astraea_layernorm_modulate(const void *x, const int32_t *idx, int M, con
 }
 
 // ------------------------------------------------------------------ a whole compute block
-// workspace: [256 bytes: error word] [select scratch] [5 token-sized buffers] [hidden-sized buffer]
+// workspace: [256 bytes: error word | gathered keys and values of the SelectQ&K variant] [select scratch]
+//            [5 token-sized buffers] [hidden-sized buffer]
+// (the first part is laid out as the workspace of astraea_sparse_attn with kv_idx, so that every call of the block
+// shares the one error word at the very start)
 static size_t block_buffer_bytes(int B, int N, int width) { return align_up((size_t)B * N * width * 2, 256); }
 
 size_t astraea_block_workspace_bytes(int B, int H, int N, int d, int hidden)
 {
     if (B <= 0 || H <= 0 || N <= 0 || d <= 0 || hidden <= 0) return 0;
-    return 256 + align_up(select_workspace_bytes(B, N), 256) + 5 * block_buffer_bytes(B, N, H * d) + block_buffer_bytes(B, N, hidden);
+    return align_up(attn_kv_workspace_bytes(B, H, N, d), 256) + align_up(select_workspace_bytes(B, N), 256) +
+           5 * block_buffer_bytes(B, N, H * d) + block_buffer_bytes(B, N, hidden);
 }
 
 int32_t astraea_block_step(const void *x, const astraea_block_weights *w, const astraea_block_state *st,
@@ -296,7 +300,8 @@ int32_t astraea_block_step(const void *x, const astraea_block_weights *w, const 
     REQUIRE(B > 0 && H > 0 && N > 0 && d > 0 && N_text > 0, "astraea_block_step: B, H, N, d, N_text must be positive");
     REQUIRE(N_sel >= 0 && N_sel <= N, "astraea_block_step: N_sel=%d outside [0, N=%d]", N_sel, N);
     REQUIRE(k_keep >= 0 && k_keep <= N_sel, "astraea_block_step: k_keep=%d outside [0, N_sel=%d]", k_keep, N_sel);
-    if (flags & ~ASTRAEA_BLOCK_REUSE_SELECTION) return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_block_step: unknown flags 0x%x", flags);
+    if (flags & ~(ASTRAEA_BLOCK_REUSE_SELECTION | ASTRAEA_BLOCK_SELECT_QK))
+        return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_block_step: unknown flags 0x%x", flags);
     const int D = H * d, hidden = w->hidden;
     REQUIRE(D % 64 == 0 && hidden > 0 && hidden % 64 == 0, "astraea_block_step: D=%d and hidden=%d must be multiples of 64", D, hidden);
     REQUIRE(w->wq && w->wk && w->wv && w->wo && w->wq2 && w->wo2 && w->w1 && w->w2, "astraea_block_step: null weight matrix");
@@ -310,10 +315,11 @@ int32_t astraea_block_step(const void *x, const astraea_block_weights *w, const 
     REQUIRE(score && (idx_sel || M == 0), "astraea_block_step: null score or idx_sel");
     char *ws = reinterpret_cast<char *>(workspace);
     void *err = ws;                                     // the error word of every call below
-    char *p = ws + 256;
+    char *p = ws + align_up(attn_kv_workspace_bytes(B, H, N, d), 256);
     void *sel_ws = p; p += align_up(select_workspace_bytes(B, N), 256);
     const size_t tb = block_buffer_bytes(B, N, D);
     void *bufA = p, *bufQ = p + tb, *bufK = p + 2 * tb, *bufV = p + 3 * tb, *bufO = p + 4 * tb, *bufU = p + 5 * tb;
+    const bool select_qk = (flags & ASTRAEA_BLOCK_SELECT_QK) != 0;
     int32_t rc = ASTRAEA_OK;
     if (!(flags & ASTRAEA_BLOCK_REUSE_SELECTION)) {
         rc = astraea_score(x, st->x_ref, st->lse_cache, st->n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, delta_mode, lse_mode, stream);
@@ -326,12 +332,17 @@ int32_t astraea_block_step(const void *x, const astraea_block_weights *w, const 
     const int64_t tsb = (int64_t)N_text * D;
     // self-attention group: keys / values from all tokens, everything else on the selected rows
     rc = astraea_layernorm_modulate(x, nullptr, 0, w->s1, w->t1, bufA, B, N, D, eps, 0u, err, stream);
-    if (rc == ASTRAEA_OK) rc = astraea_gathered_linear(bufA, nullptr, 0, w->wk, w->bk, bufK, B, N, D, D, 0u, err, 256, stream);
-    if (rc == ASTRAEA_OK) rc = astraea_gathered_linear(bufA, nullptr, 0, w->wv, w->bv, bufV, B, N, D, D, 0u, err, 256, stream);
+    // (SelectQ&K: keys and values of the selected tokens only, so only their rows are projected)
+    const int32_t *kv_rows = select_qk ? idx_sel : nullptr;
+    if (rc == ASTRAEA_OK) rc = astraea_gathered_linear(bufA, kv_rows, M, w->wk, w->bk, bufK, B, N, D, D, 0u, err, 256, stream);
+    if (rc == ASTRAEA_OK) rc = astraea_gathered_linear(bufA, kv_rows, M, w->wv, w->bv, bufV, B, N, D, D, 0u, err, 256, stream);
     if (rc == ASTRAEA_OK) rc = astraea_gathered_linear(bufA, idx_sel, M, w->wq, w->bq, bufQ, B, N, D, D, 0u, err, 256, stream);
-    if (rc == ASTRAEA_OK)
+    if (rc == ASTRAEA_OK && !select_qk)
         rc = astraea_sparse_attn(bufQ, bufK, bufV, sb, sh, sn, sb, sh, sn, sb, sh, sn, idx_sel, M, nullptr, 0, bufO, st->lse_cache,
                                  B, H, N, d, 0.f, 0u, err, 256, stream);
+    if (rc == ASTRAEA_OK && select_qk)       // the listed key / value rows are gathered into the head of the workspace
+        rc = astraea_sparse_attn(bufQ, bufK, bufV, sb, sh, sn, sb, sh, sn, sb, sh, sn, idx_sel, M, idx_sel, M, bufO, st->lse_cache,
+                                 B, H, N, d, 0.f, 0u, ws, attn_kv_workspace_bytes(B, H, N, d), stream);
     // x1 (compact, over the dead keys) = x[I] + g1 * (attention rows Wo^T + bo)
     if (rc == ASTRAEA_OK)
         rc = astraea_gathered_linear_residual(bufO, idx_sel, M, w->wo, w->bo, x, w->g1, bufK, B, N, D, D, ASTRAEA_LINEAR_COMPACT_OUT, err, 256, stream);
@@ -471,6 +482,104 @@ int32_t astraea_schedule_launch(astraea_schedule *s, void *stream)
     REQUIRE(s && s->exec, "astraea_schedule_launch: null schedule");
     cudaError_t e = cudaGraphLaunch(s->exec, (cudaStream_t)stream);
     if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_schedule_launch: %s", cudaGetErrorString(e));
+    return ASTRAEA_OK;
+}
+
+// ------------------------------------------------------------------ a generation (T steps x L blocks) as one CUDA graph
+struct astraea_model_schedule {
+    cudaGraph_t graph;
+    cudaGraphExec_t exec;
+    int L, T;
+};
+
+void astraea_model_schedule_destroy(astraea_model_schedule *s)
+{
+    if (!s) return;
+    if (s->exec) cudaGraphExecDestroy(s->exec);
+    if (s->graph) cudaGraphDestroy(s->graph);
+    delete s;
+}
+
+int32_t astraea_timestep_level_budgets(const int32_t *k_keep, int T, int N_sel, int32_t *out)
+{
+    if (!k_keep || !out || T <= 0 || N_sel < 0) return fail(ASTRAEA_ERR_INVALID_ARG, "astraea_timestep_level_budgets: bad arguments");
+    long long carry = 0;
+    int computed = 0;
+    for (int t = 0; t < T; ++t) {
+        if (k_keep[t] < 0 || k_keep[t] > N_sel) return fail(ASTRAEA_ERR_INVALID_ARG, "astraea_timestep_level_budgets: k_keep[%d]=%d outside [0, N_sel=%d]", t, k_keep[t], N_sel);
+        carry += k_keep[t];
+        if (t == 0 || (N_sel > 0 && carry >= N_sel)) {
+            out[t] = N_sel;
+            carry -= N_sel;
+            if (carry < 0) carry = 0;          // the first step computes everything whatever its budget was
+            ++computed;
+        } else {
+            out[t] = 0;
+        }
+    }
+    return computed;
+}
+
+int32_t astraea_model_schedule_create(astraea_model_schedule **schedule, int L, int T, const int32_t *k_keep,
+                                      const void *const *x_in, const astraea_block_weights *weights,
+                                      const astraea_block_state *states, const void *const *text_k,
+                                      const void *const *text_v, int N_text,
+                                      float *const *score, int32_t *const *idx_sel, int32_t *const *idx_rem,
+                                      int B, int H, int N, int N_sel, int d,
+                                      float w_alpha, float w_beta, int delta_mode, int lse_mode, float eps, int variant,
+                                      void *workspace, size_t workspace_bytes)
+{
+    REQUIRE(schedule, "astraea_model_schedule_create: null schedule pointer");
+    *schedule = nullptr;
+    REQUIRE(L > 0 && T > 0 && k_keep && x_in && weights && states && text_k && text_v && score && idx_sel,
+            "astraea_model_schedule_create: L, T must be positive and the arrays non-null");
+    REQUIRE(N_sel >= 0 && N_sel <= N, "astraea_model_schedule_create: N_sel=%d outside [0, N=%d]", N_sel, N);
+    if (variant < ASTRAEA_VARIANT_TOKEN_WISE || variant > ASTRAEA_VARIANT_FIXED_TOKEN)
+        return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_model_schedule_create: unknown variant %d", variant);
+    for (int t = 0; t < T; ++t) {
+        REQUIRE(k_keep[t] >= 0 && k_keep[t] <= N_sel, "astraea_model_schedule_create: k_keep[%d]=%d outside [0, N_sel=%d]", t, k_keep[t], N_sel);
+        REQUIRE(variant != ASTRAEA_VARIANT_TIMESTEP || k_keep[t] == 0 || k_keep[t] == N_sel,
+                "astraea_model_schedule_create: the Timestep-level variant computes all tokens or none, k_keep[%d]=%d", t, k_keep[t]);
+        REQUIRE(x_in[t], "astraea_model_schedule_create: null input pointer at step %d", t);
+    }
+    for (int l = 0; l < L; ++l)
+        REQUIRE(text_k[l] && text_v[l] && score[l] && idx_sel[l], "astraea_model_schedule_create: null pointer for block %d", l);
+    astraea_model_schedule *s = new (std::nothrow) astraea_model_schedule();
+    if (!s) return fail(ASTRAEA_ERR_CUDA, "astraea_model_schedule_create: out of host memory");
+    s->graph = nullptr; s->exec = nullptr; s->L = L; s->T = T;
+    cudaStream_t cap = nullptr;
+    cudaError_t e = cudaStreamCreateWithFlags(&cap, cudaStreamNonBlocking);
+    if (e != cudaSuccess) { delete s; return fail(ASTRAEA_ERR_CUDA, "astraea_model_schedule_create: %s", cudaGetErrorString(e)); }
+    e = cudaStreamBeginCapture(cap, cudaStreamCaptureModeThreadLocal);
+    int32_t rc = ASTRAEA_OK;
+    if (e == cudaSuccess) {
+        const uint32_t base = variant == ASTRAEA_VARIANT_SELECT_QK ? ASTRAEA_BLOCK_SELECT_QK : 0u;
+        for (int t = 0; t < T && rc == ASTRAEA_OK; ++t)
+            for (int l = 0; l < L && rc == ASTRAEA_OK; ++l) {
+                const bool shared = variant == ASTRAEA_VARIANT_FIXED_TOKEN && l > 0;      // block 0's selection serves the whole step
+                rc = astraea_block_step(l == 0 ? x_in[t] : states[l - 1].y_cache, &weights[l], &states[l], text_k[l], text_v[l], N_text,
+                                        score[l], shared ? idx_sel[0] : idx_sel[l], idx_rem ? idx_rem[l] : nullptr,
+                                        B, H, N, N_sel, d, k_keep[t], w_alpha, w_beta, delta_mode, lse_mode, eps,
+                                        base | (shared ? ASTRAEA_BLOCK_REUSE_SELECTION : 0u), workspace, workspace_bytes, cap);
+            }
+        e = cudaStreamEndCapture(cap, &s->graph);          // also ends a capture that a failed step left open
+    }
+    if (e == cudaSuccess && rc == ASTRAEA_OK) e = cudaGraphInstantiate(&s->exec, s->graph, 0);
+    cudaStreamDestroy(cap);
+    if (rc != ASTRAEA_OK) { astraea_model_schedule_destroy(s); return rc; }
+    if (e != cudaSuccess) {
+        astraea_model_schedule_destroy(s);
+        return fail(ASTRAEA_ERR_CUDA, "astraea_model_schedule_create (graph capture): %s", cudaGetErrorString(e));
+    }
+    *schedule = s;
+    return ASTRAEA_OK;
+}
+
+int32_t astraea_model_schedule_launch(astraea_model_schedule *s, void *stream)
+{
+    REQUIRE(s && s->exec, "astraea_model_schedule_launch: null schedule");
+    cudaError_t e = cudaGraphLaunch(s->exec, (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_model_schedule_launch: %s", cudaGetErrorString(e));
     return ASTRAEA_OK;
 }
 

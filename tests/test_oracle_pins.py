@@ -603,3 +603,76 @@ def test_layernorm_modulate_matches_the_library_routine(oracle):
     assert np.abs(oracle.layernorm_modulate(x, s, t, eps=1e-5) - (ref * (1 + s[:, None]) + t[:, None])).max() < 1e-13
     y = oracle.layernorm_modulate(x, eps=0.0)
     assert np.abs(y.mean(-1)).max() < 1e-13 and np.abs(y.var(-1) - 1.0).max() < 1e-12
+
+
+# ------------------------------------------------------------------ variants of the ablation study, several blocks
+def test_timestep_level_budgets_compute_all_or_nothing_with_the_same_total(oracle):
+    for seed, T, n in ((0, 12, 100), (1, 50, 17550), (2, 7, 1)):
+        rng = np.random.default_rng(seed)
+        k = [n] + [int(v) for v in rng.integers(0, n + 1, T - 1)]
+        out = oracle.timestep_level_budgets(k, n)
+        assert out[0] == n and set(out) <= {0, n}
+        assert abs(sum(out) - sum(k)) < n or sum(k) < n                  # the total budget is kept up to one step
+        # a schedule that is all-or-nothing already comes back unchanged
+        assert oracle.timestep_level_budgets(out, n) == out
+    assert oracle.timestep_level_budgets([10, 5, 5, 0, 9, 1], 10) == [10, 0, 10, 0, 0, 10]
+    assert oracle.timestep_level_budgets([3, 3, 3], 10) == [10, 0, 0]    # the first step computes everything whatever its budget
+
+
+def test_select_qk_block_is_the_block_on_the_selected_tokens_alone(oracle):
+    """SelectQ&K (Table 2): with keys and values restricted to the selected tokens, the selected rows of the block are
+    the dense block evaluated on the sub-sequence of selected tokens."""
+    rng = np.random.default_rng(41)
+    B, N, H, d, N_text, hidden, k_keep = 1, 15, 2, 4, 4, 16, 6
+    D = H * d
+    x = _rand(rng, B, N, D)
+    w = _block_weights(rng, B, D, hidden)
+    tk, tv = _rand(rng, B, N_text, H, d), _rand(rng, B, N_text, H, d)
+    y_cache = _rand(rng, B, N, D)
+    res = oracle.block_step(x, x + 0.5 * _rand(rng, B, N, D), _rand(rng, B, H, N), np.zeros((B, N), np.int32), y_cache, w, tk, tv, H,
+                            k_keep, select_qk=True)
+    sel = res["idx_sel"][0]
+    dense_sub, lse_sub = _torch_dense_block(x[:, sel], w, tk, tv, H)
+    assert np.abs(res["y"][0, sel] - dense_sub[0]).max() < 1e-11
+    assert np.abs(res["lse"][0][:, sel] - lse_sub[0]).max() < 1e-11
+    unsel = np.setdiff1d(np.arange(N), sel)
+    assert np.array_equal(res["y"][0, unsel], y_cache[0, unsel])
+
+
+def test_model_step_chains_blocks_and_the_variants_differ_as_the_ablation_describes(oracle):
+    rng = np.random.default_rng(42)
+    B, N, H, d, N_text, hidden, L, k_keep = 1, 16, 2, 4, 3, 16, 3, 7
+    D = H * d
+    x = _rand(rng, B, N, D)
+    blocks = [_block_weights(rng, B, D, hidden) for _ in range(L)]
+    tks, tvs = [_rand(rng, B, N_text, H, d) for _ in range(L)], [_rand(rng, B, N_text, H, d) for _ in range(L)]
+    states = [dict(x_ref=_rand(rng, B, N, D), lse=_rand(rng, B, H, N), n_skip=rng.integers(0, 3, (B, N)).astype(np.int32),
+                   y=_rand(rng, B, N, D)) for _ in range(L)]
+    # token-wise: the chain of single blocks, each reading the merged output of the one before
+    outs = oracle.model_step(x, blocks, states, tks, tvs, H, k_keep)
+    xin = x
+    for l in range(L):
+        r = oracle.block_step(xin, states[l]["x_ref"], states[l]["lse"], states[l]["n_skip"], states[l]["y"], blocks[l], tks[l], tvs[l], H, k_keep)
+        for key in ("idx_sel", "y", "lse", "x_ref", "n_skip"):
+            assert np.array_equal(outs[l][key], r[key]), (l, key)
+        xin = r["y"]
+    assert any(not np.array_equal(outs[0]["idx_sel"], outs[l]["idx_sel"]) for l in range(1, L))       # blocks select on their own
+    # Fixed-token: every block of the step works on block 0's selection; later blocks keep counters and references
+    fx = oracle.model_step(x, blocks, states, tks, tvs, H, k_keep, variant=oracle.VARIANT_FIXED_TOKEN)
+    assert np.array_equal(fx[0]["y"], outs[0]["y"])
+    for l in range(1, L):
+        assert np.array_equal(fx[l]["idx_sel"], fx[0]["idx_sel"])
+        assert np.array_equal(fx[l]["n_skip"], states[l]["n_skip"]) and np.array_equal(fx[l]["x_ref"], states[l]["x_ref"])
+        unsel = np.setdiff1d(np.arange(N), fx[0]["idx_sel"][0])
+        assert np.array_equal(fx[l]["y"][0, unsel], states[l]["y"][0, unsel])
+    # Timestep-level: a step computes everything (the dense model) or nothing (every cache as it was)
+    full = oracle.model_step(x, blocks, states, tks, tvs, H, N, variant=oracle.VARIANT_TIMESTEP)
+    xin = x
+    for l in range(L):
+        xin, _ = _torch_dense_block(xin, blocks[l], tks[l], tvs[l], H)
+        assert np.abs(full[l]["y"] - xin).max() < 1e-10
+    none = oracle.model_step(x, blocks, states, tks, tvs, H, 0, variant=oracle.VARIANT_TIMESTEP)
+    for l in range(L):
+        assert np.array_equal(none[l]["y"], states[l]["y"]) and np.array_equal(none[l]["lse"], states[l]["lse"])
+    with pytest.raises(AssertionError):
+        oracle.model_step(x, blocks, states, tks, tvs, H, 5, variant=oracle.VARIANT_TIMESTEP)
