@@ -97,3 +97,13 @@ def test_argument_errors_of_the_next_layer_entry_points(L):
     assert sched(keep=(ctypes.c_int32 * 2)(4, 4), wsb=8) == binding.ERR_WORKSPACE_TOO_SMALL
     assert L.astraea_schedule_launch(None, None) == binding.ERR_INVALID_ARG
     L.astraea_schedule_destroy(None)                                                       # a null handle is ignored
+
+
+def test_timestep_level_policy_matches_the_oracles(L, oracle):
+    import numpy as np
+    for seed, T, n in ((0, 12, 100), (1, 50, 17550), (2, 7, 1), (3, 30, 118800)):
+        rng = np.random.default_rng(seed)
+        k = [n] + [int(v) for v in rng.integers(0, n + 1, T - 1)]
+        assert binding.astraea_timestep_level_budgets(k, n) == oracle.timestep_level_budgets(k, n)
+    with pytest.raises(binding.AstraeaError):
+        binding.astraea_timestep_level_budgets([5, 11], 10)

@@ -369,3 +369,96 @@ def test_block_step_cogvideox_shape_sampled_rows_layer_by_layer(oracle):
     rows = np.unique(np.concatenate([[0, 127, 128, 255, 256, M // 2, M - 257, M - 256, M - 1], rng.choice(M, 23, replace=False)]))
     tok, want_y_rows = check_layers(oracle, bits, t, x_bits, idx, tk_bits, tv_bits, B, H, N, d, rows=rows, heads=[0, H // 2, H - 1])
     _close(oracle.take_rows(bf16_dev_to_f64(y), tok), want_y_rows, "y")
+
+
+# ------------------------------------------------------------------ a generation of T steps x L blocks as one graph
+@pytest.mark.parametrize("variant", [A.VARIANT_TOKEN_WISE, A.VARIANT_SELECT_QK, A.VARIANT_TIMESTEP, A.VARIANT_FIXED_TOKEN])
+def test_model_schedule_two_blocks_six_steps_against_the_oracle(oracle, variant):
+    """The four rows of the ablation study (Table 2) as scheduled runs of 2 blocks x 6 steps.  The graph of the first
+    t+1 steps, replayed from fresh state, must leave in every block the state that the oracle's block produces from the
+    state the graph of the first t steps left (teacher forcing from graph to graph, block by block: block 1 is fed the
+    device's output of block 0 of the same step)."""
+    rng = np.random.default_rng(200 + variant)
+    B, H, d, N_v, N_t, N_text, hidden, L, T = 1, 2, 64, 300, 12, 20, 256, 2, 6
+    N, D = N_v + N_t, H * d
+    budgets = [N_v, N_v * 40 // 100, N_v * 25 // 100, 0, N_v * 60 // 100, N_v * 30 // 100]
+    if variant == A.VARIANT_TIMESTEP:
+        budgets = A.astraea_timestep_level_budgets([N_v, 120, 100, 90, 200, 130], N_v)
+        assert budgets == oracle.timestep_level_budgets([N_v, 120, 100, 90, 200, 130], N_v) and 0 in budgets and budgets.count(N_v) >= 2
+    blocks = [make_block(rng, B, H, d, hidden, N_text) for _ in range(L)]
+    Wd = [({n: to_dev_bf16(a) for n, a in bits.items()}, hidden) for bits, _, _ in blocks]
+    Wf = [{n: f64(a) for n, a in bits.items()} for bits, _, _ in blocks]
+    tk, tv = [to_dev_bf16(b[1]) for b in blocks], [to_dev_bf16(b[2]) for b in blocks]
+    tkf, tvf = [f64(b[1]) for b in blocks], [f64(b[2]) for b in blocks]
+    xs = [_bits(rng, B, N, D)]
+    for t in range(1, T):
+        xs.append(synth.drift_step(xs[-1], 700 + t, 0.1, False))
+    dx = [to_dev_bf16(a) for a in xs]
+    cache0 = [_bits(rng, B, N, D) for _ in range(L)]
+    rd = lambda a: synth.bf16_to_f64(synth.f32_to_bf16_bits(a.astype(np.float32)))
+
+    def fresh():
+        return [dict(x_ref=to_dev_bf16(xs[0]), lse_cache=torch.zeros(B, H, N, device="cuda"),
+                     n_skip=torch.zeros(B, N_v, dtype=torch.int32, device="cuda"), y_cache=to_dev_bf16(cache0[l]),
+                     score=torch.zeros(B, N_v, device="cuda"), idx_sel=torch.zeros(B, N, dtype=torch.int32, device="cuda"),
+                     idx_rem=torch.zeros(B, N_v, dtype=torch.int32, device="cuda")) for l in range(L)]
+
+    def host(states):
+        return [dict(x_ref=bf16_dev_to_f64(s["x_ref"]), lse=s["lse_cache"].cpu().numpy().astype(np.float64),
+                     n_skip=s["n_skip"].cpu().numpy().copy(), y=bf16_dev_to_f64(s["y_cache"]),
+                     score=s["score"].cpu().numpy().astype(np.float64), idx_sel=s["idx_sel"].cpu().numpy().copy()) for s in states]
+
+    ws = torch.zeros(A.astraea_block_workspace_bytes(B, H, N, d, hidden), dtype=torch.uint8, device="cuda")
+    prev = host(fresh())
+    for t in range(T):
+        st = fresh()
+        sched = A.ModelSchedule(budgets[:t + 1], dx[:t + 1], Wd, st, tk, tv, N_text, B, H, N, N_v, d, variant=variant, workspace=ws)
+        sched.launch()
+        A.astraea_poll_error(ws)
+        sched.close()
+        now = host(st)
+        k_keep = budgets[t]
+        M = k_keep + N_t
+        x_in = f64(xs[t])
+        shared = None
+        for l in range(L):
+            what = (variant, t, l)
+            fixed_later = variant == A.VARIANT_FIXED_TOKEN and l > 0
+            got_sel = (now[0] if fixed_later else now[l])["idx_sel"].reshape(-1)[:B * M].reshape(B, M)
+            res = oracle.block_step(x_in, prev[l]["x_ref"], prev[l]["lse"], prev[l]["n_skip"], prev[l]["y"], Wf[l], tkf[l], tvf[l], H, k_keep,
+                                    n_always=N_t, rounder=rd, select_qk=(variant == A.VARIANT_SELECT_QK), shared_sel=shared if fixed_later else None)
+            if not fixed_later:
+                rel = np.abs(now[l]["score"] - res["score"]) / np.abs(res["score"])
+                assert rel.max() < 1e-5, what
+                if not np.array_equal(got_sel, res["idx_sel"]):
+                    # near-ties of the k-th score only; then the oracle adopts the device's (valid) selection
+                    for b in range(B):
+                        assert (np.diff(got_sel[b]) > 0).all() and np.array_equal(got_sel[b][k_keep:], np.arange(N_v, N)), what
+                        kth = np.sort(res["score"][b])[::-1][k_keep - 1]
+                        diff = np.setxor1d(got_sel[b], res["idx_sel"][b])
+                        assert (np.abs(res["score"][b][diff] - kth) <= 1e-6 * abs(kth)).all(), what
+                    res = oracle.block_step(x_in, prev[l]["x_ref"], prev[l]["lse"], prev[l]["n_skip"], prev[l]["y"], Wf[l], tkf[l], tvf[l], H,
+                                            k_keep, n_always=N_t, rounder=rd, select_qk=(variant == A.VARIANT_SELECT_QK), forced_sel=got_sel)
+                assert np.array_equal(now[l]["n_skip"], res["n_skip"]), what
+            else:
+                assert np.array_equal(now[l]["n_skip"], prev[l]["n_skip"]), what             # a later block of a Fixed-token step
+            assert np.array_equal(now[l]["x_ref"], res["x_ref"]), what
+            sel_mask = np.zeros((B, N), bool)
+            for b in range(B):
+                sel_mask[b, got_sel[b]] = True
+            err = np.abs(now[l]["y"] - res["y"]) / np.maximum(1.0, np.abs(res["y"]))
+            assert err.max() < 6e-2 and err.mean() < 4e-3, (what, err.max(), err.mean())
+            assert np.array_equal(now[l]["y"][~sel_mask], prev[l]["y"][~sel_mask]), what     # reuse: bit for bit
+            assert np.abs(now[l]["lse"] - res["lse"]).max() < 2e-2, what
+            assert np.array_equal(now[l]["lse"].transpose(0, 2, 1)[~sel_mask], prev[l]["lse"].transpose(0, 2, 1)[~sel_mask]), what
+            if M:
+                assert np.abs(now[l]["y"][sel_mask] - prev[l]["y"][sel_mask]).max() > 1e-3, what    # the selected rows did change
+            if variant == A.VARIANT_FIXED_TOKEN and l == 0:
+                shared = got_sel
+            x_in = now[l]["y"]                       # block l + 1 reads the device's merged output of block l
+        prev = now
+    # a Timestep-level schedule refuses partial budgets
+    if variant == A.VARIANT_TIMESTEP:
+        with pytest.raises(A.AstraeaError) as e:
+            A.ModelSchedule([N_v, 7], dx[:2], Wd, fresh(), tk, tv, N_text, B, H, N, N_v, d, variant=variant, workspace=ws)
+        assert e.value.code == A.ERR_INVALID_ARG
