@@ -440,6 +440,17 @@ int32_t astraea_budget_to_k(int n_sel, int theta_permille);
  */
 int32_t astraea_poll_error(void *workspace, void *stream);
 
+/*
+ * Self-test of the failure detection: every wait inside the tensor-core kernels (on a copy, an MMA, another warp) is
+ * bounded; when one runs out the kernel raises ASTRAEA_ERR_TIMEOUT in its workspace's error word, lets its remaining
+ * waits return at once and exits in order.  This call runs that give-up path in isolation: one warp waits for at most
+ * limit_us microseconds (1 .. 1000) on a barrier that nothing ever arrives at, then returns.  Afterwards
+ * astraea_poll_error(workspace) reports ASTRAEA_ERR_TIMEOUT and the context and the workspace remain usable.
+ *   gave_up : optional device int32, set to 1 by the kernel when its wait ran out
+ * (The paper has no counterpart: this is a property of the library.)
+ */
+int32_t astraea_selftest_wait(void *workspace, int limit_us, int32_t *gave_up, void *stream);
+
 const char *astraea_last_error(void);
 const char *astraea_version(void);
 

@@ -36,7 +36,7 @@ EXPORTS = [
     "astraea_block_step", "astraea_block_workspace_bytes", "astraea_model_schedule_create", "astraea_model_schedule_launch",
     "astraea_model_schedule_destroy", "astraea_timestep_level_budgets", "astraea_schedule_create", "astraea_schedule_launch", "astraea_schedule_destroy",
     "astraea_session_create", "astraea_session_destroy", "astraea_step_host",
-    "astraea_workspace_bytes", "astraea_budget_to_k", "astraea_poll_error",
+    "astraea_workspace_bytes", "astraea_budget_to_k", "astraea_poll_error", "astraea_selftest_wait",
     "astraea_last_error", "astraea_version",
 ]
 
@@ -108,6 +108,8 @@ def lib() -> ctypes.CDLL:
         L.astraea_workspace_bytes.restype = c_sz
         L.astraea_budget_to_k.argtypes = [c_i, c_i]
         L.astraea_poll_error.argtypes = [c_p, c_p]
+        L.astraea_selftest_wait.argtypes = [c_p, c_i, c_p, c_p]
+        L.astraea_selftest_wait.restype = ctypes.c_int32
         L.astraea_last_error.restype = ctypes.c_char_p
         L.astraea_version.restype = ctypes.c_char_p
         for name in ("astraea_score", "astraea_select", "astraea_sparse_attn", "astraea_sparse_cross_attn", "astraea_sparse_attn_noalloc", "astraea_scatter_reuse",
@@ -259,6 +261,11 @@ def astraea_step(x_cur, x_ref, lse_cache, n_skip, q, k, v, out_cache, score, idx
                               _ptr(out_cache), _ptr(score), _ptr(idx_sel), _ptr(idx_rem),
                               B, H, N, N_sel, d, k_keep, w_alpha, w_beta, delta_mode, lse_mode,
                               _ptr(workspace), workspace.numel() if workspace is not None else 0, _stream(stream)))
+
+
+def astraea_selftest_wait(workspace, limit_us=200, gave_up=None, stream=None) -> None:
+    """Runs the give-up path of the bounded device-side waits in isolation (see include/astraea.h)."""
+    _check(lib().astraea_selftest_wait(_ptr(workspace), limit_us, _ptr(gave_up), _stream(stream)))
 
 
 def astraea_poll_error(workspace, stream=None) -> None:

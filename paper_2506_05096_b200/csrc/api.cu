@@ -403,6 +403,13 @@ int32_t astraea_step(const void *x_cur, void *x_ref, float *lse_cache, int32_t *
     return astraea_scatter_reuse(x_ref, x_cur, idx_sel, B, N, M, D, ASTRAEA_SCATTER_SRC_FULL, ws, stream);
 }
 
+int32_t astraea_selftest_wait(void *workspace, int limit_us, int32_t *gave_up, void *stream)
+{
+    REQUIRE(workspace, "astraea_selftest_wait: null workspace");
+    REQUIRE(limit_us > 0 && limit_us <= 1000, "astraea_selftest_wait: limit_us=%d outside [1, 1000]", limit_us);
+    return launch_wait_selftest(reinterpret_cast<int *>(workspace), (uint64_t)limit_us * 1000ull, gave_up, (cudaStream_t)stream);
+}
+
 int32_t astraea_poll_error(void *workspace, void *stream)
 {
     REQUIRE(workspace, "astraea_poll_error: null workspace");

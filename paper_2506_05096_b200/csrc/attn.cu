@@ -888,6 +888,33 @@ int32_t noalloc_scratch_address(void **scratch_out)
     return ASTRAEA_OK;
 }
 
+// ---------------------------------------------------------------- self-test of the bounded wait
+// One warp waits, with the given limit, on an mbarrier that is initialised and that nothing ever arrives at: the wait
+// must give up, raise the error word and return, and the context must stay usable.  This is the give-up path that
+// every tcgen05 kernel of the library takes when a copy or an MMA never completes, run where nothing else is at stake.
+namespace {
+__global__ void __launch_bounds__(32) wait_selftest_kernel(int *err_word, uint64_t limit_ns, int *gave_up)
+{
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        ptx::mbar_init(ptx::smem_u32(&bar), 1);
+        ptx::fence_barrier_init();
+    }
+    __syncwarp();
+    wait_bar(ptx::smem_u32(&bar), 0, &abort_flag, err_word, limit_ns);
+    __syncwarp();
+    if (threadIdx.x == 0 && gave_up) *gave_up = abort_flag;
+}
+}  // namespace
+
+int32_t launch_wait_selftest(int *err_word, uint64_t limit_ns, int *gave_up, cudaStream_t stream)
+{
+    wait_selftest_kernel<<<1, 32, 0, stream>>>(err_word, limit_ns, gave_up);
+    return check_launch("astraea_selftest_wait");
+}
+
 // Which CTA shape finishes first.  Large CTAs (two query tiles, one per SM) are dispatched in launch order onto 148
 // SMs; the last one of every (head, batch) is cheaper when it holds one query tile only (0.68 of a full one,
 // measured).  Small CTAs (one query tile, two per SM) all cost the same: `slowdown` times a large one, because two

@@ -16,7 +16,8 @@ __device__ __forceinline__ bool elect_one() {
 
 // Bounded mbarrier wait.  Gives up after the limit, or at once when another wait of this CTA
 // already gave up; the caller carries on (its results are void, the error word says so).
-__device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err_word) {
+__device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err_word,
+                                         uint64_t limit_ns = kWaitLimitNs) {
     using namespace ptx;
     if (mbar_try_wait(bar, parity)) return;
     if (*abort_flag) return;
@@ -25,7 +26,7 @@ __device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, volatile
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 255u) == 0) {
             if (*abort_flag) return;
-            if (globaltimer_ns() - t0 > kWaitLimitNs) {
+            if (globaltimer_ns() - t0 > limit_ns) {
                 *abort_flag = 1;
                 atomicExch(err_word, kErrTimeout);
                 return;

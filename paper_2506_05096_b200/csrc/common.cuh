@@ -80,6 +80,7 @@ struct AttnArgs {
 };
 int32_t launch_sparse_attn(const AttnArgs &a, cudaStream_t stream);
 size_t attn_workspace_bytes(int B, int H, int N, int M, int d);
+int32_t launch_wait_selftest(int *err_word, uint64_t limit_ns, int *gave_up, cudaStream_t stream);
 int32_t noalloc_scratch_address(void **scratch_out);   // device address of the library's built-in scratch array on the current device
 size_t attn_kv_workspace_bytes(int B, int H, int M_kv, int d);
 int32_t launch_sparse_attn_kv(AttnArgs a, const int32_t *kv_idx, int M_kv, void *workspace, cudaStream_t stream);   // gathers the listed K/V rows into the workspace first

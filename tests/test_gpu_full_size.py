@@ -232,3 +232,88 @@ def test_hunyuan_shaped_consecutive_steps_full_size(oracle):
     assert torch.equal(out[unsel], out0[unsel]) and torch.equal(lse.transpose(1, 2)[unsel], lse0.transpose(1, 2)[unsel])
     x1d, x0d = to_dev_bf16(x1), to_dev_bf16(x0)
     assert torch.equal(x_ref[unsel], x0d[unsel]) and torch.equal(x_ref[~unsel], x1d[~unsel])
+
+
+def test_hunyuan_shaped_fifty_consecutive_steps_full_size(oracle):
+    """The 50-step drifting-latent workload at the full HunyuanVideo shape (118800 tokens, 24 heads of 128): a dense
+    step 0 from empty caches, then 49 steps at keep-ratio 0.6 with the real LSE / x_ref / counter chain.  The latents
+    drift on the device (seeded generator: inputs, not arithmetic of the method).  At steps 0, 1, 25 and 49 the step is
+    checked with the oracle started from the device's state before it: sampled scores, the whole selection and the
+    counters bit for bit on the device's scores, sampled attention rows, reuse and refresh bit for bit.  At the end the
+    penalty term must have kept every token from being skipped for longer than its bound."""
+    w = synth.WORKLOADS["hunyuan"]
+    B, N, H, d, D, N_sel = w.B, w.N, w.H, w.d, w.D, w.N_v
+    T, theta, checks = 50, 600, (0, 1, 25, 49)
+    g = torch.Generator(device="cuda").manual_seed(11)
+    rng = np.random.default_rng(12)
+
+    def drift(t, sigma, preserve):
+        inv = 1.0 / math.sqrt(1.0 + sigma * sigma) if preserve else 1.0
+        flat = t.view(-1, D)
+        for r0 in range(0, flat.shape[0], 16384):
+            r1 = min(flat.shape[0], r0 + 16384)
+            eps = torch.randn(r1 - r0, D, device="cuda", generator=g)
+            flat[r0:r1] = ((flat[r0:r1].float() + sigma * eps) * inv).to(torch.bfloat16)
+
+    x, q, k, v = (torch.randn(B, N, D, device="cuda", generator=g, dtype=torch.bfloat16) for _ in range(4))
+    x_ref = x.clone()
+    out = torch.zeros(B, N, H, d, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros(B, H, N, device="cuda")
+    n_skip = torch.zeros(B, N_sel, dtype=torch.int32, device="cuda")
+    score = torch.empty(B, N_sel, device="cuda")
+    idx_sel = torch.empty(B, N, dtype=torch.int32, device="cuda")
+    idx_rem = torch.empty(B, N_sel, dtype=torch.int32, device="cuda")
+    ws = A.new_workspace(A.OP_STEP, B, H, N, N, d)
+    w_alpha = 1.0 / N
+    heads = [0, H - 1]
+    f = lambda t: t.float().cpu().numpy().astype(np.float64)
+    max_sig = 0.0
+    for t in range(T):
+        if t > 0:
+            drift(x, 0.05, False)
+            for a in (q, k, v):
+                drift(a, 0.05, True)
+        k_keep = N_sel if t == 0 else w.k_of(theta)
+        check = t in checks
+        if check:
+            x_ref0, out0, lse0, n0 = x_ref.clone(), out.clone(), lse.clone(), n_skip.clone()
+        A.astraea_step(x, x_ref, lse, n_skip, q, k, v, out, score, idx_sel, idx_rem, B, H, N, N_sel, d, k_keep,
+                       w_alpha=w_alpha, workspace=ws)
+        if not check:
+            continue
+        A.astraea_poll_error(ws)
+        # scores on sampled tokens, from the device's state before the step
+        pick = np.sort(rng.choice(N_sel, 1024, replace=False))
+        pk = torch.from_numpy(pick).cuda()
+        want_s = oracle.score(f(x[:, pk]), f(x_ref0[:, pk]), f(lse0[:, :, pk]), n0[:, pk].cpu().numpy(), n_sel=len(pick), w_alpha=w_alpha)
+        got_score = score.cpu().numpy()
+        assert (np.abs(got_score[:, pick].astype(np.float64) - want_s) / np.abs(want_s)).max() < 1e-5, t
+        n0_h = n0.cpu().numpy()
+        max_sig = max(max_sig, float((got_score.astype(np.float64) - np.exp(np.minimum(n0_h, 80))).max()))
+        # the whole selection and the counters, bit for bit on the device's scores
+        want_sel, want_rem, want_n = oracle.select(got_score, k_keep, 0, n0_h)
+        got_sel = idx_sel.cpu().numpy()[:, :k_keep]
+        assert np.array_equal(got_sel, want_sel) and np.array_equal(n_skip.cpu().numpy(), want_n), t
+        assert np.array_equal(idx_rem.cpu().numpy()[:, :N_sel - k_keep], want_rem), t
+        # sampled attention rows (first and last rows of the first, a middle and the last CTA, and random ones)
+        rows = stratified_rows(rng, got_sel[0], 16)[None]
+        rw = torch.from_numpy(rows[0]).long().cuda()
+        qh, kh, vh = (f(a.view(B, N, H, d)[:, :, heads]) for a in (q, k, v))
+        want_o, want_l, _ = oracle.sparse_attn(qh, kh, vh, q_idx=rows)
+        del qh, kh, vh
+        assert_attn_close(f(out[:, rw][:, :, heads]), want_o, what=("step", t))
+        assert np.abs(f(lse[:, heads][:, :, rw]) - want_l).max() < 1e-3, t
+        # reuse and refresh, bit for bit, over the whole tensors
+        sel = torch.zeros(B, N, dtype=torch.bool, device="cuda")
+        sel[0, idx_sel[0, :k_keep].long()] = True
+        assert torch.equal(out[~sel], out0[~sel]) and torch.equal(lse.transpose(1, 2)[~sel], lse0.transpose(1, 2)[~sel]), t
+        assert torch.equal(x_ref[~sel], x_ref0[~sel]) and torch.equal(x_ref[sel], x[sel]), t
+        if t > 0:
+            assert not torch.equal(out[sel][:4096], out0[sel][:4096]), t              # the selected rows were recomputed
+        del x_ref0, out0, lse0, n0
+    A.astraea_poll_error(ws)
+    # Penalty term (Section 3.2, S_penalty = e^n with w_beta = 1): at a keep-ratio of one half or more the tokens that
+    # were skipped (at most 40 % of them) outrank every token that was just computed as soon as e^n exceeds the largest
+    # significance term + 1, so no counter can pass that n
+    bound = max(1, int(math.ceil(math.log(1.0 + max(max_sig, 0.0)))))
+    assert int(n_skip.max().item()) <= bound, (int(n_skip.max().item()), bound, max_sig)

@@ -427,6 +427,29 @@ def test_attn_bad_index_is_reported_not_dereferenced():
     assert torch.equal(out[0, 2:], torch.ones_like(out[0, 2:]))
 
 
+def test_bounded_wait_runs_out_reports_timeout_and_the_workspace_stays_usable(oracle):
+    """Failure detection without a fault: a wait on a barrier that nothing arrives at gives up after its limit (200
+    microseconds here), the error word says TIMEOUT, and the very same workspace then serves a normal attention call."""
+    B, H, N, d, M = 1, 2, 300, 64, 77
+    ws = A.new_workspace(A.OP_SPARSE_ATTN, B, H, N, M, d)
+    gave_up = torch.zeros(1, dtype=torch.int32, device="cuda")
+    A.astraea_selftest_wait(ws, 200, gave_up)
+    with pytest.raises(A.AstraeaError) as e:
+        A.astraea_poll_error(ws)
+    assert e.value.code == A.ERR_TIMEOUT and int(gave_up.item()) == 1
+    A.astraea_poll_error(ws)                 # the word was cleared
+    rng = np.random.default_rng(4)
+    q, k, v = (synth.f32_to_bf16_bits(rng.standard_normal((B, N, H, d)).astype(np.float32)) for _ in range(3))
+    idx = np.sort(rng.choice(N, M, replace=False)).astype(np.int32)[None]
+    out = torch.zeros(B, M, H, d, dtype=torch.bfloat16, device="cuda")
+    s_ = A.bhnd_strides(N, H, d)
+    A.astraea_sparse_attn(to_dev_bf16(q), to_dev_bf16(k), to_dev_bf16(v), s_, s_, s_, dev(idx), M, out, None, B, H, N, d,
+                          flags=A.ATTN_COMPACT_OUT, workspace=ws)
+    A.astraea_poll_error(ws)
+    want, _, _ = oracle.sparse_attn(f64(q), f64(k), f64(v), q_idx=idx)
+    assert_attn_close(bf16_dev_to_f64(out), want)
+
+
 def test_attn_duplicate_and_descending_indices_are_reported_and_written_once():
     """q_idx must be strictly ascending: a duplicate would make two rows race on one output row.  The offending
     entries are skipped (their rows keep the cache), the others are computed, BAD_INDEX is reported."""
