@@ -42,9 +42,14 @@ NOMINAL_BF16_TFLOPS, NOMINAL_HBM_GBS = 2250.0, 8000.0     # the part's nominal d
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the attention kernel, from the ncu captures summarised
 # in profiles/ (workload -> theta_permille -> (bytes, file)); None where not captured at that size.
 NCU_TRAFFIC = {
-    "cogvideox": {500: (324246784, "profiles/sparse_attn_d64_cogvideox.md")},
-    "sweep": {250: (1285133616, "profiles/sparse_attn_d128_sweep.md")},
+    "cogvideox": {500: (324454400, "profiles/sparse_attn_d64_cogvideox.md")},
+    "opensora": {400: (207461376, "profiles/sparse_attn_d72_opensora.md")},
+    "sweep": {250: (1299120184, "profiles/sparse_attn_d128_sweep.md")},
 }
+# The headline launch (sweep shape, keep-ratio 0.5) holds too much for a multi-pass capture: its traffic is the
+# keep-ratio-0.25 capture scaled by the compulsory bytes (the traffic is Q and output rows of M tokens plus K and V of
+# N tokens, each read through L2 at the same hit rate)
+NCU_TRAFFIC_SCALED_FROM = {"sweep": 250}
 
 
 def measured_peaks():
@@ -299,6 +304,11 @@ def kernel_report(w, theta, parts, peaks, long_region=False, pair_ms=None):
         return {"ms": float(ms), "GB/s": gbs, "frac_hbm": gbs / hbm, "frac_hbm_nominal": gbs / NOMINAL_HBM_GBS}
 
     traffic = NCU_TRAFFIC.get(w.name, {}).get(theta)
+    if traffic is None and w.name in NCU_TRAFFIC_SCALED_FROM:
+        th0 = NCU_TRAFFIC_SCALED_FROM[w.name]
+        b0, src = NCU_TRAFFIC[w.name][th0]
+        ratio = accounting.attn_min_bytes(B, H, M, N, d) / accounting.attn_min_bytes(B, H, w.M_of(th0), N, d)
+        traffic = (int(b0 * ratio), "%s (keep-ratio %.2f capture x %.3f = ratio of the compulsory bytes)" % (src, th0 / 1000, ratio))
     roofline = {"bound": "tensor", "kernel": "sparse_attn_kernel<%d>" % d, "achieved": achieved,
                 "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
                 "peak_kind": "%s burst bf16" % peaks["source"],
@@ -319,6 +329,128 @@ def kernel_report(w, theta, parts, peaks, long_region=False, pair_ms=None):
                "sparse_attn": {"ms": attn_ms, "TFLOP/s": achieved},
                "scatter_reuse(x_ref)": hbm_entry(cb, parts[3])}
     return roofline, kernels
+
+
+def block_leg(torch, A, w, thetas, peaks, hidden_mult=4, N_text=226, reps=5):
+    """The whole compute block (astraea_block_step: score, select, K/V projections of all rows, query projection,
+    self-attention, output projection, cross-attention and MLP on the selected rows) at several keep-ratios, and its
+    layers one by one at the first of them.  Keep-ratio 1000 is the dense block."""
+    B, N, H, d, D, N_sel, n_always = w.B, w.N, w.H, w.d, w.D, w.N_v, w.N_t
+    hidden = hidden_mult * D
+    g = torch.Generator(device="cuda").manual_seed(99)
+    rn = lambda *s, scale=1.0: (scale * torch.randn(*s, device="cuda", generator=g)).to(torch.bfloat16)
+    W = {}
+    for name, (o, i) in dict(wq=(D, D), wk=(D, D), wv=(D, D), wo=(D, D), wq2=(D, D), wo2=(D, D), w1=(hidden, D), w2=(D, hidden)).items():
+        W[name] = rn(o, i, scale=1 / math.sqrt(i))
+        W["b" + name[1:]] = rn(o, scale=0.1)
+    for name in ("s1", "t1", "g1", "s3", "t3", "g3"):
+        W[name] = rn(B, D, scale=0.3)
+    tk, tv = rn(B, N_text, H, d), rn(B, N_text, H, d)
+    xs = [rn(B, N, D), None]
+    xs[1] = (xs[0].float() + 0.05 * torch.randn(B, N, D, device="cuda", generator=g)).to(torch.bfloat16)
+    x_ref = xs[0].clone()
+    lse = torch.zeros(B, H, N, device="cuda")
+    n_skip = torch.zeros(B, N_sel, dtype=torch.int32, device="cuda")
+    y = torch.zeros(B, N, D, dtype=torch.bfloat16, device="cuda")
+    score = torch.empty(B, N_sel, device="cuda")
+    idx_sel = torch.empty(B, N, dtype=torch.int32, device="cuda")
+    ws = torch.zeros(A.astraea_block_workspace_bytes(B, H, N, d, hidden), dtype=torch.uint8, device="cuda")
+    bw = A.block_weights(W, hidden)
+    w_alpha = float(1.0 / N)
+
+    def run(t, k_keep):
+        A.astraea_block_step(xs[t & 1], bw, x_ref, lse, n_skip, y, tk, tv, N_text, score, idx_sel, None, B, H, N, N_sel, d, k_keep,
+                             w_alpha=w_alpha, workspace=ws)
+
+    run(0, N_sel)                                  # dense first step fills the caches
+    A.astraea_poll_error(ws)
+    out = {"shape": {"B": B, "N": N, "D": D, "H": H, "d": d, "hidden": hidden, "N_text": N_text}, "keep_ratios": {}}
+    for th in thetas:
+        k_keep = w.k_of(th)
+        M = k_keep + n_always
+        for t in range(2):
+            run(t + 1, k_keep)
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+        torch.cuda.synchronize()
+        evs[0].record()
+        for t in range(reps):
+            run(t + 1, k_keep)
+            evs[t + 1].record()
+        torch.cuda.synchronize()
+        A.astraea_poll_error(ws)
+        ms = float(np.median([evs[i].elapsed_time(evs[i + 1]) for i in range(reps)]))
+        # algorithmic flops of the block as built: K/V projections of all rows, the rest on M rows
+        fl = (2 * 2 * B * N * D * D                                    # K, V
+              + 2 * B * M * D * D * 4                                  # Q, out-projection, cross-attention query and output projection
+              + 2 * 2 * B * M * D * hidden                             # MLP
+              + accounting.attn_flops(B, H, M, N, d) + accounting.attn_flops(B, H, M, N_text, d))
+        out["keep_ratios"][str(th)] = {"ms": ms, "M": M, "TFLOP/s": fl / (ms * 1e-3) / 1e12,
+                                       "frac_bf16_peak": fl / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"], "flops": fl}
+    dense = out["keep_ratios"].get("1000")
+    if dense:
+        for th, e in out["keep_ratios"].items():
+            e["speedup_vs_dense_block"] = dense["ms"] / e["ms"]
+            e["flops_vs_dense_block"] = e["flops"] / dense["flops"]
+    # the layers one by one at the middle keep-ratio (the same calls astraea_block_step makes, buffers of their own)
+    th = thetas[len(thetas) // 2]
+    k_keep = w.k_of(th)
+    M = k_keep + n_always
+    run(1, k_keep)
+    idx = idx_sel.view(-1)[:B * M].view(B, M)
+    z = lambda *s: torch.zeros(*s, dtype=torch.bfloat16, device="cuda")
+    h, kk, vv, qq, a = z(B, N, D), z(B, N, D), z(B, N, D), z(B, N, D), z(B, N, D)
+    x1, h2, c, x2, u = z(B, M, D), z(B, M, D), z(B, M, D), z(B, M, D), z(B, M, hidden)
+    st, ts = A.bhnd_strides(N, H, d), A.bhnd_strides(N_text, H, d)
+    x = xs[0]
+    CI, CO, CR = A.LINEAR_COMPACT_IN, A.LINEAR_COMPACT_OUT, A.LINEAR_COMPACT_RES
+    layers = [
+        ("layernorm+modulate (all rows)", 2 * B * N * D * 2, None, lambda: A.astraea_layernorm_modulate(x, None, 0, W["s1"], W["t1"], h, B, N, D, workspace=ws)),
+        ("K projection (all rows)", None, 2 * B * N * D * D, lambda: A.astraea_gathered_linear(h, None, 0, W["wk"], W["bk"], kk, B, N, D, D, workspace=ws)),
+        ("V projection (all rows)", None, 2 * B * N * D * D, lambda: A.astraea_gathered_linear(h, None, 0, W["wv"], W["bv"], vv, B, N, D, D, workspace=ws)),
+        ("Q projection (selected rows)", None, 2 * B * M * D * D, lambda: A.astraea_gathered_linear(h, idx, M, W["wq"], W["bq"], qq, B, N, D, D, workspace=ws)),
+        ("self-attention (selected rows x all keys)", None, accounting.attn_flops(B, H, M, N, d),
+         lambda: A.astraea_sparse_attn(qq, kk, vv, st, st, st, idx, M, a, lse, B, H, N, d, workspace=ws)),
+        ("output projection + gated residual", None, 2 * B * M * D * D,
+         lambda: A.astraea_gathered_linear_residual(a, idx, M, W["wo"], W["bo"], x, W["g1"], x1, B, N, D, D, flags=CO, workspace=ws)),
+        ("layernorm (selected rows)", 2 * B * M * D * 2, None,
+         lambda: A.astraea_layernorm_modulate(x1, idx, M, None, None, h2, B, N, D, flags=A.LN_COMPACT_IN | A.LN_COMPACT_OUT, workspace=ws)),
+        ("cross-attention query projection", None, 2 * B * M * D * D, lambda: A.astraea_gathered_linear(h2, idx, M, W["wq2"], W["bq2"], qq, B, N, D, D, flags=CI, workspace=ws)),
+        ("cross-attention (selected rows x text keys)", None, accounting.attn_flops(B, H, M, N_text, d),
+         lambda: A.astraea_sparse_cross_attn(qq, tk, tv, st, ts, ts, idx, M, c, None, B, H, N, N_text, d, flags=A.ATTN_COMPACT_OUT, workspace=ws)),
+        ("cross-attention output projection + residual", None, 2 * B * M * D * D,
+         lambda: A.astraea_gathered_linear_residual(c, idx, M, W["wo2"], W["bo2"], x1, None, x2, B, N, D, D, flags=CI | CO | CR, workspace=ws)),
+        ("layernorm+modulate (selected rows)", 2 * B * M * D * 2, None,
+         lambda: A.astraea_layernorm_modulate(x2, idx, M, W["s3"], W["t3"], h2, B, N, D, flags=A.LN_COMPACT_IN | A.LN_COMPACT_OUT, workspace=ws)),
+        ("MLP up-projection + GELU", None, 2 * B * M * D * hidden,
+         lambda: A.astraea_gathered_linear(h2, idx, M, W["w1"], W["b1"], u, B, N, D, hidden, flags=CI | CO | A.LINEAR_GELU, workspace=ws)),
+        ("MLP down-projection + gated residual + scatter", None, 2 * B * M * D * hidden,
+         lambda: A.astraea_gathered_linear_residual(u, idx, M, W["w2"], W["b2"], x2, W["g3"], y, B, N, hidden, D, flags=CI | CR, workspace=ws)),
+    ]
+    per = {}
+    for name, nbytes, fl, fn in layers:
+        for _ in range(2):
+            fn()
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+        torch.cuda.synchronize()
+        evs[0].record()
+        for i in range(reps):
+            fn()
+            evs[i + 1].record()
+        torch.cuda.synchronize()
+        ms = float(np.median([evs[i].elapsed_time(evs[i + 1]) for i in range(reps)]))
+        e = {"ms": ms}
+        if fl:
+            e["TFLOP/s"] = fl / (ms * 1e-3) / 1e12
+            e["frac_bf16_peak"] = e["TFLOP/s"] / peaks["bf16_tflops"]
+        if nbytes:
+            e["GB/s"] = nbytes / ms / 1e6
+            e["frac_hbm"] = e["GB/s"] / peaks["hbm_gbs"]
+        per[name] = e
+    A.astraea_poll_error(ws)
+    out["layers_at_keep_ratio_%d" % th] = per
+    out["layers_note"] = ("each layer timed alone in a loop over one buffer set (inputs of the small layers stay in L2); the block "
+                          "figures above are whole astraea_block_step calls on alternating inputs")
+    return out
 
 
 def e2e_leg(torch, A, w, theta, steps, barrier):
@@ -374,6 +506,7 @@ def main():
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-workloads", action="store_true", help="headline only")
     ap.add_argument("--no-next", action="store_true", help="skip the query projection of the selected rows (astraea_gathered_linear)")
+    ap.add_argument("--no-block", action="store_true", help="skip the whole-block leg (astraea_block_step on the CogVideoX shape)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -588,6 +721,10 @@ def main():
         if not args.no_e2e:
             dt, fl, info = e2e_leg(torch, A, hw, 600, 3, barrier)
             workloads["hunyuan"]["600"]["e2e"] = {"value": fl / dt / 1e12, "unit": UNIT, **info, "ms_per_step": 1e3 * dt / 3}
+    block = None
+    if not args.no_block and extras:
+        block = block_leg(torch, A, synth.WORKLOADS["cogvideox"], (1000, 500, 250), peaks)
+        torch.cuda.empty_cache()
     sampler.stop()
 
     cpu = None
@@ -608,7 +745,7 @@ def main():
                                     "all": attn_fracs},
                 "worst_hbm_frac": {"value": hbm_fracs[worst_h], "where": worst_h, "of": "measured copy bandwidth",
                                    "of_nominal_8000": hbm_fracs[worst_h] * peaks["hbm_gbs"] / NOMINAL_HBM_GBS, "all": hbm_fracs},
-                "keep_ratio_sweep": sweep, "workloads": workloads, "next": nxt, "e2e": e2e, "cpu_baseline": cpu,
+                "keep_ratio_sweep": sweep, "workloads": workloads, "next": nxt, "block": block, "e2e": e2e, "cpu_baseline": cpu,
                 "bench_seconds": time.perf_counter() - t_start}
         print(json.dumps(line))
     if world > 1:

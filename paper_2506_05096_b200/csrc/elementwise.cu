@@ -3,9 +3,9 @@
 // element-wise step in front of them runs for the selected tokens only; in front of the key / value projections it
 // runs for all tokens).
 //
-// HBM-bound: every row is read once and written once.  One warp owns one row and keeps it in registers (16-byte
-// loads, all in flight at once), takes the mean and then the centred sum of squares from the registers (two passes over
-// registers, one over memory), normalises, modulates and stores.  fp32 arithmetic, one rounding to bf16 at the end.
+// HBM-bound: every row is read once and written once.  One warp owns one row and keeps it packed in registers (16-byte
+// loads, all in flight at once), takes mean and variance from the registers in one pass over shifted data, then
+// normalises, modulates and stores in a second pass over the registers.  fp32 arithmetic, one rounding to bf16 at the end.
 #include "common.cuh"
 
 namespace astraea {
@@ -28,8 +28,10 @@ __device__ __forceinline__ void unpack8(const uint4 &v, float (&f)[8]) {
 }
 
 // VPL: 16-byte vectors per lane (compile-time bound of the register array; vec_per_row <= 32 * VPL)
+// (two or three blocks per SM: the row stays packed in registers and is unpacked again in every pass, instead of being
+// kept as 8 * VPL floats, which would leave room for one block per SM only and too few bytes in flight)
 template <int VPL>
-__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+__global__ void __launch_bounds__(kWarpsPerBlock * 32, VPL <= 8 ? 3 : 2)
 layernorm_modulate_kernel(const uint4 *__restrict__ x, const int32_t *__restrict__ idx, int M, const uint4 *__restrict__ scale,
                           const uint4 *__restrict__ shift, uint4 *__restrict__ y, int B, int N, int vec_per_row, float eps,
                           int compact_in, int compact_out, int *__restrict__ err_word)
@@ -49,29 +51,23 @@ layernorm_modulate_kernel(const uint4 *__restrict__ x, const int32_t *__restrict
         uint4 v[VPL];
 #pragma unroll
         for (int u = 0; u < VPL; ++u) v[u] = (lane + 32 * u < vec_per_row) ? ld_stream(src + lane + 32 * u) : make_uint4(0, 0, 0, 0);
-        float sum = 0.f;
-#pragma unroll
-        for (int u = 0; u < VPL; ++u) {
-            float f[8];
-            unpack8(v[u], f);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) sum += f[i];               // vectors past the end are zero
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-        const float mean = sum * inv_D;
-        float sq = 0.f;
+        // mean and variance in one pass over the packed registers, on data shifted by the row's first element: the
+        // shift takes the cancellation out of E[(x - x0)^2] - (E[x - x0])^2 whenever the mean is large against the spread
+        const float x0 = __shfl_sync(0xffffffffu, __uint_as_float(v[0].x << 16), 0);
+        float s1 = 0.f, s2 = 0.f;
 #pragma unroll
         for (int u = 0; u < VPL; ++u) {
             if (lane + 32 * u < vec_per_row) {
                 float f[8];
                 unpack8(v[u], f);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) sq = fmaf(f[i] - mean, f[i] - mean, sq);
+                for (int i = 0; i < 8; ++i) { const float c = f[i] - x0; s1 += c; s2 = fmaf(c, c, s2); }
             }
         }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+        for (int o = 16; o > 0; o >>= 1) { s1 += __shfl_xor_sync(0xffffffffu, s1, o); s2 += __shfl_xor_sync(0xffffffffu, s2, o); }
+        const float ms = s1 * inv_D, mean = x0 + ms;
+        const float sq = fmaxf(s2 - s1 * ms, 0.f);                 // sum of squares about the mean
         const float rstd = rsqrtf(sq * inv_D + eps);
 #pragma unroll
         for (int u = 0; u < VPL; ++u) {
