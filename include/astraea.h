@@ -107,6 +107,26 @@ int32_t astraea_score(const void *x_cur, const void *x_ref, const float *lse, co
                       float w_alpha, float w_beta, int delta_mode, int lse_mode, void *stream);
 
 /*
+ * The selection metric when the heads (and with them the channels, D = H*d) are sharded over several GPUs (the
+ * multi-GPU scalability experiment of Section 4; the paper does not name its scheme: here every GPU owns a
+ * contiguous range of heads with the full-length keys / values, outputs and LSE values of those heads).  S_token is a
+ * product of two sums that run over all channels and all heads, so each shard contributes raw partial sums,
+ *     part[0, b, i] = sum over the shard's channels of |x_cur - x_ref| (or its square, or the signed difference)
+ *     part[1, b, i] = sum over the shard's heads of exp(min(lse, ASTRAEA_LSE_CLAMP)) (or of lse in the log mode),
+ * the partial sums of all shards are added up (ONE all-reduce of 2*B*N_sel floats), and astraea_score_combine turns
+ * the totals into S_token = w_alpha * (part[1] / H) * (part[0] / D) + w_beta * e^n on every GPU alike, so that the
+ * (deterministic) selection that follows is identical everywhere.
+ *   x_cur, x_ref : bf16 [B, N, D_local]    lse : fp32 [B, H_local, N] or NULL (part[1] = 0)
+ *   part         : out fp32 [2, B, N_sel]
+ * astraea_score_combine: D, H are the TOTAL channel and head counts; has_lse = 0 => S_LSE = 1; n_skip may be NULL.
+ * Errors: as astraea_score.
+ */
+int32_t astraea_score_partial(const void *x_cur, const void *x_ref, const float *lse, float *part,
+                              int B, int N, int N_sel, int D_local, int H_local, int delta_mode, int lse_mode, void *stream);
+int32_t astraea_score_combine(const float *part, const int32_t *n_skip, float *score, int B, int N_sel, int D, int H,
+                              int has_lse, float w_alpha, float w_beta, void *stream);
+
+/*
  * TopK(S_token, theta) -> I_sel, I_remain (Algorithm 1 line 3): the k largest scores of
  * each batch row.  Deterministic: equal scores go to the lower token index, -0 equals +0,
  * NaN ranks below every number.  Both index lists come out ascending by token index; the

@@ -81,6 +81,31 @@ def score(x_cur, x_ref, lse=None, n_skip=None, n_sel=None, H=1, w_alpha=1.0, w_b
     return out
 
 
+def score_partial(x_cur, x_ref, lse=None, n_sel=None, delta_mode=0, lse_mode=0):
+    """The two sums behind the selection metric over a shard of the channels / heads (head-sharded multi-GPU form):
+    (sum over the given channels of the difference term, sum over the given heads of exp(min(lse, 80)) or of lse).
+    Plain numpy; float64 [2, B, n_sel]."""
+    x_cur, x_ref = _f64(x_cur), _f64(x_ref)
+    B, N, D = x_cur.shape
+    n_sel = N if n_sel is None else n_sel
+    diff = (x_cur - x_ref)[:, :n_sel]
+    a = np.abs(diff).sum(-1) if delta_mode == 0 else (diff * diff).sum(-1) if delta_mode == 1 else diff.sum(-1)
+    if lse is None:
+        b = np.zeros((B, n_sel))
+    else:
+        l = _f64(lse)[:, :, :n_sel]
+        b = np.exp(np.minimum(l, 80.0)).sum(1) if lse_mode == 0 else l.sum(1)
+    return np.stack([a, b])
+
+
+def score_combine(part, n_skip, D, H, has_lse=True, w_alpha=1.0, w_beta=1.0):
+    """S_token from the partial sums added up over all shards: w_alpha (part[1]/H)(part[0]/D) + w_beta e^min(n, 80)."""
+    part = _f64(part)
+    n = np.zeros(part.shape[1:], dtype=np.int64) if n_skip is None else np.minimum(np.asarray(n_skip, dtype=np.int64), 80)
+    s_lse = part[1] / H if has_lse else 1.0
+    return w_alpha * s_lse * (part[0] / D) + w_beta * np.exp(n.astype(np.float64))
+
+
 def select(score_f32, k, n_always=0, n_skip=None):
     """Top-k per batch row on float32 scores.  Returns (idx_sel, idx_rem, n_skip_new)."""
     s = np.ascontiguousarray(score_f32, dtype=np.float32)

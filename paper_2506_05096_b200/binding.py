@@ -31,7 +31,7 @@ N_SKIP_CLAMP = 80
 NOALLOC_SCRATCH_BYTES = 4096
 
 EXPORTS = [
-    "astraea_score", "astraea_select", "astraea_sparse_attn", "astraea_sparse_cross_attn", "astraea_sparse_attn_noalloc", "astraea_scatter_reuse", "astraea_step",
+    "astraea_score", "astraea_score_partial", "astraea_score_combine", "astraea_select", "astraea_sparse_attn", "astraea_sparse_cross_attn", "astraea_sparse_attn_noalloc", "astraea_scatter_reuse", "astraea_step",
     "astraea_gathered_linear", "astraea_gathered_linear_residual", "astraea_layernorm_modulate",
     "astraea_block_step", "astraea_block_workspace_bytes", "astraea_model_schedule_create", "astraea_model_schedule_launch",
     "astraea_model_schedule_destroy", "astraea_timestep_level_budgets", "astraea_schedule_create", "astraea_schedule_launch", "astraea_schedule_destroy",
@@ -72,6 +72,9 @@ def lib() -> ctypes.CDLL:
         c_i, c_f, c_p, c_sz, c_i64, c_u = (ctypes.c_int, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t,
                                            ctypes.c_int64, ctypes.c_uint32)
         L.astraea_score.argtypes = [c_p, c_p, c_p, c_p, c_p, c_i, c_i, c_i, c_i, c_i, c_f, c_f, c_i, c_i, c_p]
+        L.astraea_score_partial.argtypes = [c_p, c_p, c_p, c_p, c_i, c_i, c_i, c_i, c_i, c_i, c_i, c_p]
+        L.astraea_score_combine.argtypes = [c_p, c_p, c_p, c_i, c_i, c_i, c_i, c_i, c_f, c_f, c_p]
+        L.astraea_score_partial.restype = L.astraea_score_combine.restype = ctypes.c_int32
         L.astraea_select.argtypes = [c_p, c_i, c_i, c_i, c_i, c_p, c_p, c_p, c_p, c_sz, c_p]
         L.astraea_sparse_attn.argtypes = [c_p, c_p, c_p] + [c_i64] * 9 + [c_p, c_i, c_p, c_i, c_p, c_p,
                                                                          c_i, c_i, c_i, c_i, c_f, c_u, c_p, c_sz, c_p]
@@ -165,6 +168,19 @@ def astraea_score(x_cur, x_ref, lse, n_skip, score, B, N, N_sel, D, H, w_alpha=1
                   delta_mode=DELTA_MEAN_ABS, lse_mode=LSE_SUM_EXP, stream=None) -> None:
     _check(lib().astraea_score(_ptr(x_cur), _ptr(x_ref), _ptr(lse), _ptr(n_skip), _ptr(score),
                                B, N, N_sel, D, H, w_alpha, w_beta, delta_mode, lse_mode, _stream(stream)))
+
+
+def astraea_score_partial(x_cur, x_ref, lse, part, B, N, N_sel, D_local, H_local, delta_mode=DELTA_MEAN_ABS, lse_mode=LSE_SUM_EXP,
+                          stream=None) -> None:
+    """Raw partial sums of the selection metric over a shard of the channels / heads: part is fp32 [2, B, N_sel]."""
+    _check(lib().astraea_score_partial(_ptr(x_cur), _ptr(x_ref), _ptr(lse), _ptr(part), B, N, N_sel, D_local, H_local,
+                                       delta_mode, lse_mode, _stream(stream)))
+
+
+def astraea_score_combine(part, n_skip, score, B, N_sel, D, H, has_lse=True, w_alpha=1.0, w_beta=1.0, stream=None) -> None:
+    """S_token from the partial sums added up over all shards (D, H: total channel and head counts)."""
+    _check(lib().astraea_score_combine(_ptr(part), _ptr(n_skip), _ptr(score), B, N_sel, D, H, 1 if has_lse else 0,
+                                       w_alpha, w_beta, _stream(stream)))
 
 
 def astraea_select(score, B, N_sel, k, n_always, idx_sel, idx_rem, n_skip, workspace, stream=None) -> None:

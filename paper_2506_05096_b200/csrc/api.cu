@@ -101,6 +101,28 @@ int32_t astraea_score(const void *x_cur, const void *x_ref, const float *lse, co
                         lse_mode, (cudaStream_t)stream);
 }
 
+int32_t astraea_score_partial(const void *x_cur, const void *x_ref, const float *lse, float *part,
+                              int B, int N, int N_sel, int D_local, int H_local, int delta_mode, int lse_mode, void *stream)
+{
+    REQUIRE(B > 0 && N > 0 && D_local > 0 && H_local > 0, "astraea_score_partial: B, N, D_local, H_local must be positive");
+    REQUIRE(N_sel >= 0 && N_sel <= N, "astraea_score_partial: N_sel=%d outside [0, N=%d]", N_sel, N);
+    REQUIRE(D_local % 8 == 0, "astraea_score_partial: D_local=%d must be a multiple of 8 (16-byte rows)", D_local);
+    REQUIRE(x_cur && x_ref && part, "astraea_score_partial: null x_cur, x_ref or part");
+    REQUIRE(aligned16(x_cur) && aligned16(x_ref), "astraea_score_partial: x_cur / x_ref must be 16-byte aligned");
+    if (delta_mode < 0 || delta_mode > 2 || lse_mode < 0 || lse_mode > 1)
+        return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_score_partial: unknown delta_mode %d or lse_mode %d", delta_mode, lse_mode);
+    return launch_score(x_cur, x_ref, lse, nullptr, nullptr, B, N, N_sel, D_local, H_local, 0.f, 0.f, delta_mode, lse_mode,
+                        (cudaStream_t)stream, part);
+}
+
+int32_t astraea_score_combine(const float *part, const int32_t *n_skip, float *score, int B, int N_sel, int D, int H,
+                              int has_lse, float w_alpha, float w_beta, void *stream)
+{
+    REQUIRE(B > 0 && N_sel >= 0 && D > 0 && H > 0, "astraea_score_combine: bad sizes");
+    REQUIRE((part && score) || N_sel == 0, "astraea_score_combine: null part or score");
+    return launch_score_combine(part, n_skip, score, B, N_sel, D, H, has_lse ? 1 : 0, w_alpha, w_beta, (cudaStream_t)stream);
+}
+
 int32_t astraea_select(const float *score, int B, int N_sel, int k, int n_always,
                        int32_t *idx_sel, int32_t *idx_rem, int32_t *n_skip,
                        void *workspace, size_t workspace_bytes, void *stream)

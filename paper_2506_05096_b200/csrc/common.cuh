@@ -50,7 +50,9 @@ inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 // kernel launchers (one per .cu file)
 int32_t launch_score(const void *x_cur, const void *x_ref, const float *lse, const int32_t *n_skip,
                      float *score, int B, int N, int N_sel, int D, int H, float w_alpha, float w_beta,
-                     int delta_mode, int lse_mode, cudaStream_t stream);
+                     int delta_mode, int lse_mode, cudaStream_t stream, float *part = nullptr);
+int32_t launch_score_combine(const float *part, const int32_t *n_skip, float *score, int B, int N_sel, int D, int H,
+                             int has_lse, float w_alpha, float w_beta, cudaStream_t stream);
 int32_t launch_select(const float *score, int B, int N_sel, int k, int n_always, int32_t *idx_sel,
                       int32_t *idx_rem, int32_t *n_skip, void *workspace, cudaStream_t stream);
 size_t select_workspace_bytes(int B, int N_sel);

@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 score_kernel(const uint4 *__restrict__ x_cur, const uint4 *__restrict__ x_ref,
              const float *__restrict__ lse, const int32_t *__restrict__ n_skip,
              float *__restrict__ score, int B, int N, int N_sel, int D, int H,
-             float w_alpha, float w_beta, int lse_mode)
+             float w_alpha, float w_beta, int lse_mode, float *__restrict__ part)
 {
     // a kernel launched behind this one with programmatic stream serialization (the selection) may become resident
     // and set itself up as soon as SMs free up; it still waits for this whole grid before it reads the scores
@@ -105,7 +105,11 @@ score_kernel(const uint4 *__restrict__ x_cur, const uint4 *__restrict__ x_ref,
             acc += __shfl_xor_sync(0xffffffffu, acc, o);
             ls += __shfl_xor_sync(0xffffffffu, ls, o);
         }
-        if (sl == 0 && have) {
+        if (sl == 0 && have && part != nullptr) {
+            // a shard of the channels / heads: the raw sums, to be added up over the shards before they are combined
+            part[(size_t)b * N_sel + i] = acc;
+            part[((size_t)B + b) * N_sel + i] = ls;
+        } else if (sl == 0 && have) {
             float delta = acc * inv_D;
             float s_lse = (lse != nullptr) ? ls * inv_H : 1.0f;
             int n = (n_skip != nullptr) ? n_skip[(size_t)b * N_sel + i] : 0;
@@ -117,19 +121,44 @@ score_kernel(const uint4 *__restrict__ x_cur, const uint4 *__restrict__ x_ref,
 
 template <int MODE>
 void launch_mode(int lpr, int grid, cudaStream_t stream, const uint4 *xc, const uint4 *xr, const float *lse, const int32_t *n_skip,
-                 float *score, int B, int N, int N_sel, int D, int H, float w_alpha, float w_beta, int lse_mode)
+                 float *score, int B, int N, int N_sel, int D, int H, float w_alpha, float w_beta, int lse_mode, float *part)
 {
     dim3 block(kWarpsPerBlock * 32);
-    if (lpr == 32) score_kernel<MODE, 32><<<grid, block, 0, stream>>>(xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode);
-    else if (lpr == 16) score_kernel<MODE, 16><<<grid, block, 0, stream>>>(xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode);
-    else score_kernel<MODE, 8><<<grid, block, 0, stream>>>(xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode);
+    if (lpr == 32) score_kernel<MODE, 32><<<grid, block, 0, stream>>>(xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode, part);
+    else if (lpr == 16) score_kernel<MODE, 16><<<grid, block, 0, stream>>>(xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode, part);
+    else score_kernel<MODE, 8><<<grid, block, 0, stream>>>(xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode, part);
+}
+
+// score[b, i] = w_alpha * (sum of exp(lse) / H) * (sum of differences / D) + w_beta * e^n from the summed partial sums
+__global__ void __launch_bounds__(256)
+score_combine_kernel(const float *__restrict__ part, const int32_t *__restrict__ n_skip, float *__restrict__ score,
+                     long long total, float inv_D, float inv_H, int has_lse, float w_alpha, float w_beta)
+{
+    for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (long long)gridDim.x * blockDim.x) {
+        const float delta = part[t] * inv_D;
+        const float s_lse = has_lse ? part[total + t] * inv_H : 1.0f;
+        int n = n_skip ? n_skip[t] : 0;
+        n = min(n, ASTRAEA_N_SKIP_CLAMP);
+        score[t] = w_alpha * (s_lse * delta) + w_beta * expf((float)n);
+    }
 }
 
 }  // namespace
 
+int32_t launch_score_combine(const float *part, const int32_t *n_skip, float *score, int B, int N_sel, int D, int H,
+                             int has_lse, float w_alpha, float w_beta, cudaStream_t stream)
+{
+    const long long total = (long long)B * N_sel;
+    if (total == 0) return ASTRAEA_OK;
+    const long long want = (total + 255) / 256, cap = (long long)sm_count() * 8;
+    score_combine_kernel<<<(int)(want < cap ? want : cap), 256, 0, stream>>>(part, n_skip, score, total, 1.0f / (float)D, 1.0f / (float)H,
+                                                                             has_lse, w_alpha, w_beta);
+    return check_launch("astraea_score_combine");
+}
+
 int32_t launch_score(const void *x_cur, const void *x_ref, const float *lse, const int32_t *n_skip,
                      float *score, int B, int N, int N_sel, int D, int H, float w_alpha, float w_beta,
-                     int delta_mode, int lse_mode, cudaStream_t stream)
+                     int delta_mode, int lse_mode, cudaStream_t stream, float *part)
 {
     const long long total = (long long)B * N_sel;
     if (total == 0) return ASTRAEA_OK;
@@ -143,13 +172,13 @@ int32_t launch_score(const void *x_cur, const void *x_ref, const float *lse, con
     const uint4 *xr = reinterpret_cast<const uint4 *>(x_ref);
     switch (delta_mode) {
     case ASTRAEA_DELTA_MEAN_ABS:
-        launch_mode<ASTRAEA_DELTA_MEAN_ABS>(lpr, grid, stream, xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode);
+        launch_mode<ASTRAEA_DELTA_MEAN_ABS>(lpr, grid, stream, xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode, part);
         break;
     case ASTRAEA_DELTA_MEAN_SQ:
-        launch_mode<ASTRAEA_DELTA_MEAN_SQ>(lpr, grid, stream, xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode);
+        launch_mode<ASTRAEA_DELTA_MEAN_SQ>(lpr, grid, stream, xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode, part);
         break;
     default:
-        launch_mode<ASTRAEA_DELTA_MEAN_SIGNED>(lpr, grid, stream, xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode);
+        launch_mode<ASTRAEA_DELTA_MEAN_SIGNED>(lpr, grid, stream, xc, xr, lse, n_skip, score, B, N, N_sel, D, H, w_alpha, w_beta, lse_mode, part);
         break;
     }
     return check_launch("astraea_score");

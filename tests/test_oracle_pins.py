@@ -676,3 +676,25 @@ def test_model_step_chains_blocks_and_the_variants_differ_as_the_ablation_descri
         assert np.array_equal(none[l]["y"], states[l]["y"]) and np.array_equal(none[l]["lse"], states[l]["lse"])
     with pytest.raises(AssertionError):
         oracle.model_step(x, blocks, states, tks, tvs, H, 5, variant=oracle.VARIANT_TIMESTEP)
+
+
+def test_partial_scores_of_head_shards_add_up_to_the_score(oracle):
+    """Head-sharded form: the selection metric from partial sums over contiguous head ranges equals the unsharded one."""
+    rng = np.random.default_rng(51)
+    B, N, N_sel, H, d = 2, 21, 18, 6, 4
+    D = H * d
+    x_ref = _rand(rng, B, N, D)
+    x_cur = x_ref + 0.3 * _rand(rng, B, N, D)
+    lse = _rand(rng, B, H, N)
+    lse[0, 2, 5] = 95.0                                   # above the clamp
+    n = rng.integers(0, 4, (B, N_sel)).astype(np.int32)
+    for delta_mode in (0, 1, 2):
+        for lse_mode in (0, 1):
+            want = oracle.score(x_cur, x_ref, lse, n, n_sel=N_sel, w_alpha=0.7, w_beta=0.2, delta_mode=delta_mode, lse_mode=lse_mode)
+            for bounds in ([0, 6], [0, 2, 6], [0, 1, 3, 4, 6]):
+                part = sum(oracle.score_partial(x_cur[:, :, h0 * d:h1 * d], x_ref[:, :, h0 * d:h1 * d], lse[:, h0:h1], N_sel, delta_mode, lse_mode)
+                           for h0, h1 in zip(bounds[:-1], bounds[1:]))
+                got = oracle.score_combine(part, n, D, H, True, 0.7, 0.2)
+                assert np.abs(got - want).max() <= 1e-12 * np.abs(want).max()
+    got = oracle.score_combine(oracle.score_partial(x_cur, x_ref, None, N_sel), None, D, H, False)
+    assert np.abs(got - oracle.score(x_cur, x_ref, None, None, n_sel=N_sel)).max() < 1e-12
