@@ -7,14 +7,14 @@
 // 256-row x 256-column output tiles (column tiles of one row tile are neighbours in the walk, so the
 // gathered rows stay in L2 while W, which is small, lives there anyway).  A tile is two 128-row sub-tiles
 // that share every W tile in shared memory.  Warp roles:
-//   warps 0-7   epilogue: one thread per output row; TMEM -> registers -> (+ bias, GELU) -> bf16 -> the row
-//               of y that idx names (fused scatter);
-//   warps 8-15  gather of the A operand: the listed rows of x, 64 columns (128 bytes) per pipeline stage,
+//   warps 0-15  epilogue: two threads per output row (128 columns each); TMEM -> registers -> (+ bias, GELU, gate,
+//               residual) -> bf16 -> the row of y that idx names (fused scatter);
+//   warps 16-23 gather of the A operand: the listed rows of x, 64 columns (128 bytes) per pipeline stage,
 //               by 16-byte cp.async into the 128-byte-swizzled layout the MMA reads (rows past the end
 //               are zero-filled); the copies arrive on the stage's barrier by themselves, so a thread never
 //               waits for its own copies, only for a free stage;
-//   warp 16     TMA producer of the B operand: a 256 x 64 tile of W per stage (rows past N_out read as zero);
-//   warp 17     tcgen05.mma issuer: per stage four 128 x 256 x 16 SS MMAs into each sub-tile's accumulator.
+//   warp 24     TMA producer of the B operand: a 256 x 64 tile of W per stage (rows past N_out read as zero);
+//   warp 25     tcgen05.mma issuer: per stage four 128 x 256 x 16 SS MMAs into each sub-tile's accumulator.
 // Stages: 3 x (2 x 16 KB of A + 32 KB of W); TMEM: two accumulators of 256 columns.  Every mbarrier wait
 // is bounded; on a timeout the CTA raises the error word, the remaining waits return at once, and the
 // CTA runs out.
@@ -35,7 +35,11 @@ constexpr int kBM = 128 * kMSub, kBN = 256, kBK = 64;
 constexpr int kStages = (kMSub == 2) ? 3 : 4;
 constexpr int kAccSets = 2 / kMSub;                      // accumulator sets in TMEM: two sets let the epilogue run under the next main loop
 constexpr int kASubBytes = 128 * kBK * 2, kABytes = kMSub * kASubBytes, kBBytes = kBN * kBK * 2;
-constexpr int kEpiWarps = 4 * kMSub, kGatherWarps = 4 * kMSub;
+// Epilogue warps: four per sub-tile cover its 128 rows (one TMEM lane quarter each); kEpiSplit such groups share the 256
+// columns of the accumulator.  Two: the epilogue is not hidden under the next tile's main loop (TMEM is full), so its
+// time counts in full, and bias, GELU (erf), gate and residual make it a third to a half of a tile's time with one group.
+constexpr int kEpiSplit = 2;
+constexpr int kEpiWarps = 4 * kMSub * kEpiSplit, kGatherWarps = 4 * kMSub;
 constexpr int kThreads = (kEpiWarps + kGatherWarps + 2) * 32;
 constexpr int kTmaWarp = kEpiWarps + kGatherWarps, kMmaWarp = kTmaWarp + 1;
 constexpr int kSmemBytes = kStages * (kABytes + kBBytes) + 256 + 1024;
@@ -128,8 +132,11 @@ gathered_linear_kernel(const __grid_constant__ CUtensorMap tmap_w, const LinPara
 
     if (warp < kEpiWarps) {
         // ------------------------------------------------ epilogue
-        const int row = warp * 32 + lane;                      // row of the CTA tile; sub-tile warp / 4, TMEM lanes by warp % 4
-        const uint32_t t_row = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (warp >> 2) * kAccCols;
+        // row of the CTA tile: sub-tile (warp / 4) % kMSub, TMEM lanes by warp % 4; columns [c0, c0 + kBN / kEpiSplit) by warp / (4 kMSub)
+        const int sub = (warp >> 2) % kMSub, part = warp / (4 * kMSub);
+        const int row = sub * 128 + (warp & 3) * 32 + lane;
+        const int c0 = part * (kBN / kEpiSplit);
+        const uint32_t t_row = tmem + ((uint32_t)((warp & 3) * 32) << 16) + sub * kAccCols;
         int it = 0;
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
             const int tm = tile / tiles_n, tn = tile - tm * tiles_n;
@@ -137,7 +144,7 @@ gathered_linear_kernel(const __grid_constant__ CUtensorMap tmap_w, const LinPara
             long long out_row = -1, res_row = -1;
             int batch = 0;
             const long long src = source_row(p, (long long)tm * kBM + row, total_rows, &out_row, &res_row, &batch);
-            if (src == -2 && tn == 0) atomicExch(p.err_word, kErrBadIndex);
+            if (src == -2 && tn == 0 && part == 0) atomicExch(p.err_word, kErrBadIndex);
             __nv_bfloat16 *dst = (src >= 0) ? p.y + out_row * p.N_out + n0 : nullptr;
             const __nv_bfloat16 *res = (src >= 0 && p.residual) ? p.residual + res_row * p.N_out : nullptr;
             const __nv_bfloat16 *gate = p.gate ? p.gate + (long long)batch * p.N_out : nullptr;
@@ -145,11 +152,11 @@ gathered_linear_kernel(const __grid_constant__ CUtensorMap tmap_w, const LinPara
             tc_fence_after();
             if (abort_flag) dst = nullptr;
 #pragma unroll 1
-            for (int c = 0; c < kBN; c += 32) {
+            for (int c = c0; c < c0 + kBN / kEpiSplit; c += 32) {
                 uint32_t o[32];
                 tmem_ld32(t_row + acc * kMSub * kAccCols + c, o);
                 tc_wait_ld();
-                if (c + 32 == kBN) {                     // the accumulator has been read: the MMA warp may reuse it
+                if (c + 32 == c0 + kBN / kEpiSplit) {    // this thread's part of the accumulator has been read: the MMA warp may reuse it
                     tc_fence_before();
                     mbar_arrive(bar_acc_empty + 8 * acc);
                 }
