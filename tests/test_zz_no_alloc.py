@@ -48,6 +48,24 @@ def test_noalloc_entry_matches_the_workspace_entry_on_two_calls_in_a_row(oracle)
         assert torch.equal(got[mask], cache[mask])
 
 
+def test_noalloc_entry_takes_the_same_flags_and_refuses_what_does_not_fit_its_scratch():
+    """The two entry points share one validation and launch path: the CTA-shape flag is accepted, and a kv_idx
+    problem whose gathered key / value rows do not fit the built-in scratch is refused with WORKSPACE_TOO_SMALL."""
+    B, H, N, d, M = 1, 2, 400, 64, 100
+    q, k, v, cache, idx = _inputs(3, B, H, N, d, M)
+    s = A.bhnd_strides(N, H, d)
+    want, got = cache.clone(), cache.clone()
+    ws = A.new_workspace(A.OP_SPARSE_ATTN, B, H, N, M, d)
+    A.astraea_sparse_attn(q, k, v, s, s, s, idx, M, want, None, B, H, N, d, flags=A.ATTN_SMALL_CTAS, workspace=ws)
+    A.astraea_sparse_attn_noalloc(q, k, v, s, s, s, idx, M, got, None, B, H, N, d, flags=A.ATTN_SMALL_CTAS)
+    torch.cuda.synchronize()
+    assert torch.equal(got.view(torch.int16), want.view(torch.int16))
+    with pytest.raises(A.AstraeaError) as e:
+        A.astraea_sparse_attn_noalloc(q, k, v, s, s, s, idx, M, got, None, B, H, N, d, kv_idx=idx, M_kv=M)
+    assert e.value.code == A.ERR_WORKSPACE_TOO_SMALL
+    assert A.astraea_workspace_bytes(A.OP_SPARSE_ATTN_KV, B, H, N, M, d) > A.NOALLOC_SCRATCH_BYTES
+
+
 def test_noalloc_entry_rejects_bad_arguments_like_the_workspace_entry():
     z = torch.zeros(1, 64, 1, 64, dtype=torch.bfloat16, device="cuda")
     s = A.bhnd_strides(64, 1, 64)
