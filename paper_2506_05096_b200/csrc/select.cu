@@ -225,6 +225,7 @@ select_cluster_kernel(const float *__restrict__ score, int N_sel, int k, int n_a
         uint4 *z = reinterpret_cast<uint4 *>(smem_hist);
         for (int i = tid; i < (int)(kClusterSmem / 16); i += kThreads) z[i] = make_uint4(0, 0, 0, 0);
     }
+    cluster_sync_all();                          // every CTA's histograms are zero before anyone adds to them (still ahead of the wait)
     grid_launch_dependents();                    // the next kernel may set itself up; it waits for this one before it reads anything
     grid_dependency_wait();                      // the scores (and whatever else the kernel before wrote) are complete
     uint32_t key[ITEMS];
@@ -238,7 +239,6 @@ select_cluster_kernel(const float *__restrict__ score, int N_sel, int k, int n_a
 #pragma unroll
         for (int u = 0; u < ITEMS; ++u) n_old[u] = (nsk && base + u < N_sel) ? nsk[base + u] : 0;
     }
-    cluster_sync_all();                          // every CTA's histograms are zero before anyone adds to them
 
     // token i is selected iff key > T, or key == T and fewer than need_eq equal keys precede it
     uint32_t T = 0xffffffffu, need_eq = 0;       // no key reaches 0xffffffff
