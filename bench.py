@@ -482,9 +482,10 @@ def e2e_leg(torch, A, w, theta, steps, barrier):
         sess.step_host(host["x_cur"], host["q"], host["k"], host["v"], host_out, k_keep, w_alpha, 1.0)
     torch.cuda.synchronize()
     dt = time.perf_counter() - t0
+    h2d = sess.last_h2d_bytes()             # x_cur, k, v in full; of the pinned q only the selected rows
     sess.close()
     flops = accounting.attn_flops(B, w.H, k_keep + w.N_t, N, w.d)
-    return dt, flops * steps, {"h2d_bytes_per_step": 4 * tb, "d2h_bytes_per_step": tb, "steps": steps,
+    return dt, flops * steps, {"h2d_bytes_per_step": h2d, "d2h_bytes_per_step": tb, "steps": steps,
                                "api": "astraea_step_host (pinned host buffers)"}
 
 

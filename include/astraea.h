@@ -437,7 +437,8 @@ void    astraea_schedule_destroy(astraea_schedule *schedule);
  * astraea_session_create allocates device memory (cudaMalloc) on the current device;
  * the first step of a session must be run with k_keep = N_sel (all tokens computed) to
  * fill the caches, as the paper's denoising loop does at its first timestep.
- *   x_cur, q, k, v : host bf16 [B,N,D] (pinned memory gives asynchronous copies)
+ *   x_cur, q, k, v : host bf16 [B,N,D] (pinned memory gives asynchronous copies; from a pinned q only the rows of
+ *                    the selected tokens cross the bus: the rest of q is never read)
  *   out            : host bf16 [B,N,D], receives X_out,t (computed + cached rows)
  * astraea_step_host synchronises the session's streams before it returns.
  */
@@ -447,6 +448,8 @@ void    astraea_session_destroy(astraea_session *session);
 int32_t astraea_step_host(astraea_session *session, const void *x_cur, const void *q, const void *k,
                           const void *v, void *out, int k_keep,
                           float w_alpha, float w_beta, int delta_mode, int lse_mode);
+/* Host-to-device bytes that the last astraea_step_host of the session moved (0 before the first step). */
+size_t  astraea_session_last_h2d_bytes(const astraea_session *session);
 
 /* Scratch size for an op (bytes); 0 for unknown ops.  H, d, M may be 0 where the op does not use them. */
 size_t  astraea_workspace_bytes(int op, int B, int H, int N, int M, int d);

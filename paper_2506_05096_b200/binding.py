@@ -35,7 +35,7 @@ EXPORTS = [
     "astraea_gathered_linear", "astraea_gathered_linear_residual", "astraea_layernorm_modulate",
     "astraea_block_step", "astraea_block_workspace_bytes", "astraea_model_schedule_create", "astraea_model_schedule_launch",
     "astraea_model_schedule_destroy", "astraea_timestep_level_budgets", "astraea_schedule_create", "astraea_schedule_launch", "astraea_schedule_destroy",
-    "astraea_session_create", "astraea_session_destroy", "astraea_step_host",
+    "astraea_session_create", "astraea_session_destroy", "astraea_step_host", "astraea_session_last_h2d_bytes",
     "astraea_workspace_bytes", "astraea_budget_to_k", "astraea_poll_error", "astraea_selftest_wait",
     "astraea_last_error", "astraea_version",
 ]
@@ -107,6 +107,8 @@ def lib() -> ctypes.CDLL:
         L.astraea_session_destroy.argtypes = [c_p]
         L.astraea_session_destroy.restype = None
         L.astraea_step_host.argtypes = [c_p, c_p, c_p, c_p, c_p, c_p, c_i, c_f, c_f, c_i, c_i]
+        L.astraea_session_last_h2d_bytes.argtypes = [c_p]
+        L.astraea_session_last_h2d_bytes.restype = c_sz
         L.astraea_workspace_bytes.argtypes = [c_i] * 6
         L.astraea_workspace_bytes.restype = c_sz
         L.astraea_budget_to_k.argtypes = [c_i, c_i]
@@ -386,6 +388,10 @@ class Session:
             assert not t.is_cuda and t.is_contiguous()
         _check(lib().astraea_step_host(self._h, _ptr(x_cur), _ptr(q), _ptr(k), _ptr(v), _ptr(out), k_keep,
                                        w_alpha, w_beta, delta_mode, lse_mode))
+
+    def last_h2d_bytes(self) -> int:
+        """Host-to-device bytes of the last step (a pinned q contributes only its selected rows)."""
+        return int(lib().astraea_session_last_h2d_bytes(self._h))
 
     def close(self) -> None:
         if self._h:

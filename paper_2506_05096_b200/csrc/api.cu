@@ -627,10 +627,14 @@ struct astraea_session {
     size_t workspace_bytes;
     cudaStream_t stream;            // score, select, attention, refresh
     cudaStream_t copy_in, copy_out; // host -> device and device -> host copies, overlapped with the compute stream
+    cudaStream_t gather;            // zero-copy fetches of the selected q rows from a pinned host buffer
+    cudaEvent_t ev_sel;             // the selection of this step is known
+    cudaEvent_t ev_q[kHostGroups];  // the selected q rows of a head group have arrived
     cudaEvent_t ev_x;               // x_cur has arrived
     cudaEvent_t ev_in[kHostGroups]; // q, k, v of a head group have arrived
     cudaEvent_t ev_attn[kHostGroups];   // attention of a head group is done
     int steps;
+    size_t last_h2d_bytes;          // host-to-device bytes of the last step
 };
 
 void astraea_session_destroy(astraea_session *s)
@@ -640,11 +644,13 @@ void astraea_session_destroy(astraea_session *s)
                     s->n_skip, s->idx_sel, s->idx_rem, s->workspace};
     for (void *p : bufs) if (p) cudaFree(p);
     if (s->ev_x) cudaEventDestroy(s->ev_x);
+    if (s->ev_sel) cudaEventDestroy(s->ev_sel);
     for (int g = 0; g < kHostGroups; ++g) {
+        if (s->ev_q[g]) cudaEventDestroy(s->ev_q[g]);
         if (s->ev_in[g]) cudaEventDestroy(s->ev_in[g]);
         if (s->ev_attn[g]) cudaEventDestroy(s->ev_attn[g]);
     }
-    cudaStream_t streams[] = {s->stream, s->copy_in, s->copy_out};
+    cudaStream_t streams[] = {s->stream, s->copy_in, s->copy_out, s->gather};
     for (cudaStream_t st : streams) if (st) cudaStreamDestroy(st);
     delete s;
 }
@@ -664,8 +670,11 @@ int32_t astraea_session_create(astraea_session **session, int B, int H, int N, i
     cudaError_t e = cudaStreamCreateWithFlags(&s->stream, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&s->copy_in, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&s->copy_out, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&s->gather, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&s->ev_x, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&s->ev_sel, cudaEventDisableTiming);
     for (int g = 0; g < kHostGroups; ++g) {
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&s->ev_q[g], cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&s->ev_in[g], cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&s->ev_attn[g], cudaEventDisableTiming);
     }
@@ -691,6 +700,8 @@ int32_t astraea_session_create(astraea_session **session, int B, int H, int N, i
     return ASTRAEA_OK;
 }
 
+size_t astraea_session_last_h2d_bytes(const astraea_session *s) { return s ? s->last_h2d_bytes : 0; }
+
 int32_t astraea_step_host(astraea_session *s, const void *x_cur, const void *q, const void *k,
                           const void *v, void *out, int k_keep,
                           float w_alpha, float w_beta, int delta_mode, int lse_mode)
@@ -706,14 +717,31 @@ int32_t astraea_step_host(astraea_session *s, const void *x_cur, const void *q, 
     const int groups = H < kHostGroups ? H : kHostGroups;
     auto head_lo = [&](int g) { return (int)((long long)H * g / groups); };
 
-    // copy-in stream: x_cur first (the score needs nothing else), then q, k, v by head group
+    // Only the M selected rows of q are ever read.  When q sits in pinned host memory that the device can address, it
+    // is not copied: once the selection is known a kernel fetches just the listed rows over the bus (zero-copy reads
+    // of whole 2*D-byte rows), which takes (N - M) / N of one tensor off the host-to-device traffic that bounds the step.
+    // Worth it only while the bus bounds the step: the fetch kernels share the SMs with the attention, and on a step
+    // whose attention takes longer than its transfers (the HunyuanVideo shape: 95 -> 101 ms) they only delay it.
+    // Rough rates: 1e15 flop/s for the attention, 5e10 bytes/s for the bus.
+    const void *q_mapped = nullptr;
+    const double attn_s = 4.0 * B * H * (double)M * N * d / 1e15, bus_s = 4.0 * (double)s->tensor_bytes / 5e10;
+    if (M < N && M > 0 && attn_s < bus_s) {
+        cudaPointerAttributes attr;
+        if (cudaPointerGetAttributes(&attr, q) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer)
+            q_mapped = attr.devicePointer;
+        else
+            cudaGetLastError();               // pageable memory: not an error, the rows are copied as before
+    }
+    s->last_h2d_bytes = s->tensor_bytes * 3 + (q_mapped ? (size_t)B * M * D * 2 : s->tensor_bytes);
+
+    // copy-in stream: x_cur first (the score needs nothing else), then (q,) k, v by head group
     cudaError_t e = cudaMemcpyAsync(s->x_cur, x_cur, s->tensor_bytes, cudaMemcpyHostToDevice, s->copy_in);
     if (e == cudaSuccess) e = cudaEventRecord(s->ev_x, s->copy_in);
     for (int g = 0; g < groups && e == cudaSuccess; ++g) {
         const size_t off = (size_t)head_lo(g) * d * 2, width = (size_t)(head_lo(g + 1) - head_lo(g)) * d * 2;
         const void *src[3] = {q, k, v};
         void *dst[3] = {s->q, s->k, s->v};
-        for (int i = 0; i < 3 && e == cudaSuccess; ++i)
+        for (int i = q_mapped ? 1 : 0; i < 3 && e == cudaSuccess; ++i)
             e = cudaMemcpy2DAsync(static_cast<char *>(dst[i]) + off, pitch, static_cast<const char *>(src[i]) + off, pitch,
                                   width, rows, cudaMemcpyHostToDevice, s->copy_in);
         if (e == cudaSuccess) e = cudaEventRecord(s->ev_in[g], s->copy_in);
@@ -733,8 +761,25 @@ int32_t astraea_step_host(astraea_session *s, const void *x_cur, const void *q, 
     if (rc == ASTRAEA_OK)
         rc = astraea_scatter_reuse(s->x_ref, s->x_cur, s->idx_sel, B, N, M, D, ASTRAEA_SCATTER_SRC_FULL, s->workspace, s->stream);
     if (rc != ASTRAEA_OK) return rc;
+    if (q_mapped) {
+        // the selected rows of q, straight from the host buffer, head group by head group on a stream of its own (so
+        // that a group's attention waits for its own columns only and the fetches run under the attention of the
+        // groups before)
+        e = cudaEventRecord(s->ev_sel, s->stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(s->gather, s->ev_sel, 0);
+        for (int g = 0; g < groups && e == cudaSuccess; ++g) {
+            const size_t off = (size_t)head_lo(g) * d * 2;
+            rc = launch_scatter(static_cast<char *>(s->q) + off, static_cast<const char *>(q_mapped) + off, s->idx_sel, B, N, M,
+                                (head_lo(g + 1) - head_lo(g)) * d, ASTRAEA_SCATTER_SRC_FULL, reinterpret_cast<int *>(s->workspace),
+                                s->gather, D);
+            if (rc != ASTRAEA_OK) return rc;
+            e = cudaEventRecord(s->ev_q[g], s->gather);
+        }
+        if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_step_host (fetch of the selected q rows): %s", cudaGetErrorString(e));
+    }
     for (int g = 0; g < groups; ++g) {
         e = cudaStreamWaitEvent(s->stream, s->ev_in[g], 0);
+        if (e == cudaSuccess && q_mapped) e = cudaStreamWaitEvent(s->stream, s->ev_q[g], 0);
         if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_step_host: %s", cudaGetErrorString(e));
         if (M > 0) {
             AttnArgs a;
@@ -762,6 +807,7 @@ int32_t astraea_step_host(astraea_session *s, const void *x_cur, const void *q, 
     }
     e = cudaStreamSynchronize(s->copy_out);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s->copy_in);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s->gather);
     if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_step_host (copy out): %s", cudaGetErrorString(e));
     s->steps++;
     return astraea_poll_error(s->workspace, s->stream);

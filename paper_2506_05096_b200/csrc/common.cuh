@@ -57,7 +57,7 @@ int32_t launch_select(const float *score, int B, int N_sel, int k, int n_always,
                       int32_t *idx_rem, int32_t *n_skip, void *workspace, cudaStream_t stream);
 size_t select_workspace_bytes(int B, int N_sel);
 int32_t launch_scatter(void *cache, const void *rows, const int32_t *idx, int B, int N, int M,
-                       int row_elems, uint32_t flags, int *err_word, cudaStream_t stream);
+                       int row_elems, uint32_t flags, int *err_word, cudaStream_t stream, int pitch_elems = 0);   // pitch 0: rows are dense
 
 size_t linear_workspace_bytes();
 int32_t launch_gathered_linear(const void *x, const int32_t *idx, int M, const void *w, const void *bias, void *y,

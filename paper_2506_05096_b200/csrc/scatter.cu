@@ -24,8 +24,10 @@ __device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
 template <int LPR>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 scatter_kernel(uint4 *__restrict__ cache, const uint4 *__restrict__ rows, const int32_t *__restrict__ idx,
-               int B, int N, int M, int vec_per_row, int src_full, int *__restrict__ err_word)
+               int B, int N, int M, int vec_per_row, int pitch_vec, int src_full, int *__restrict__ err_word)
 {
+    // vec_per_row 16-byte vectors are copied per row; rows are pitch_vec vectors apart in both tensors (a column slice
+    // of wider rows when pitch_vec > vec_per_row: the caller offsets the base pointers to the slice's first column)
     constexpr int kRowsPerWarp = 32 / LPR;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -44,8 +46,8 @@ scatter_kernel(uint4 *__restrict__ cache, const uint4 *__restrict__ rows, const 
             if (sl == 0 && err_word) atomicExch(err_word, kErrBadIndex);
             continue;
         }
-        const uint4 *src = rows + ((size_t)b * (src_full ? N : M) + (src_full ? i : r)) * vec_per_row;
-        uint4 *dst = cache + ((size_t)b * N + i) * vec_per_row;
+        const uint4 *src = rows + ((size_t)b * (src_full ? N : M) + (src_full ? i : r)) * pitch_vec;
+        uint4 *dst = cache + ((size_t)b * N + i) * pitch_vec;
         for (int v = sl; v < vec_per_row; v += LPR * kUnroll) {
             uint4 a[kUnroll];
 #pragma unroll
@@ -59,8 +61,9 @@ scatter_kernel(uint4 *__restrict__ cache, const uint4 *__restrict__ rows, const 
 }  // namespace
 
 int32_t launch_scatter(void *cache, const void *rows, const int32_t *idx, int B, int N, int M,
-                       int row_elems, uint32_t flags, int *err_word, cudaStream_t stream)
+                       int row_elems, uint32_t flags, int *err_word, cudaStream_t stream, int pitch_elems)
 {
+    const int pitch_vec = (pitch_elems > 0 ? pitch_elems : row_elems) >> 3;
     const long long total = (long long)B * M;
     if (total == 0) return ASTRAEA_OK;
     const int vec_per_row = row_elems >> 3;
@@ -72,9 +75,9 @@ int32_t launch_scatter(void *cache, const void *rows, const int32_t *idx, int B,
     uint4 *c = reinterpret_cast<uint4 *>(cache);
     const uint4 *rw = reinterpret_cast<const uint4 *>(rows);
     const int full = (flags & ASTRAEA_SCATTER_SRC_FULL) ? 1 : 0;
-    if (lpr == 32) scatter_kernel<32><<<grid, kWarpsPerBlock * 32, 0, stream>>>(c, rw, idx, B, N, M, vec_per_row, full, err_word);
-    else if (lpr == 16) scatter_kernel<16><<<grid, kWarpsPerBlock * 32, 0, stream>>>(c, rw, idx, B, N, M, vec_per_row, full, err_word);
-    else scatter_kernel<8><<<grid, kWarpsPerBlock * 32, 0, stream>>>(c, rw, idx, B, N, M, vec_per_row, full, err_word);
+    if (lpr == 32) scatter_kernel<32><<<grid, kWarpsPerBlock * 32, 0, stream>>>(c, rw, idx, B, N, M, vec_per_row, pitch_vec, full, err_word);
+    else if (lpr == 16) scatter_kernel<16><<<grid, kWarpsPerBlock * 32, 0, stream>>>(c, rw, idx, B, N, M, vec_per_row, pitch_vec, full, err_word);
+    else scatter_kernel<8><<<grid, kWarpsPerBlock * 32, 0, stream>>>(c, rw, idx, B, N, M, vec_per_row, pitch_vec, full, err_word);
     return check_launch("astraea_scatter_reuse");
 }
 
