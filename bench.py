@@ -338,7 +338,7 @@ def kernel_report(w, theta, parts, peaks, long_region=False, pair_ms=None):
     return roofline, kernels
 
 
-def block_leg(torch, A, w, thetas, peaks, hidden_mult=4, N_text=226, reps=5):
+def block_leg(torch, A, w, thetas, peaks, sampler, hidden_mult=4, N_text=226, reps=5):
     """The whole compute block (astraea_block_step: score, select, K/V projections of all rows, query projection,
     self-attention, output projection, cross-attention and MLP on the selected rows) at several keep-ratios, and its
     layers one by one at the first of them.  Keep-ratio 1000 is the dense block."""
@@ -380,11 +380,13 @@ def block_leg(torch, A, w, thetas, peaks, hidden_mult=4, N_text=226, reps=5):
             run(t + 1, k_keep)
         evs = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
         torch.cuda.synchronize()
+        m0 = sampler.mark()
         evs[0].record()
         for t in range(reps):
             run(t + 1, k_keep)
             evs[t + 1].record()
         torch.cuda.synchronize()
+        m1 = sampler.mark()
         A.astraea_poll_error(ws)
         ms = float(np.median([evs[i].elapsed_time(evs[i + 1]) for i in range(reps)]))
         # algorithmic flops of the block as built: K/V projections of all rows, the rest on M rows
@@ -393,7 +395,8 @@ def block_leg(torch, A, w, thetas, peaks, hidden_mult=4, N_text=226, reps=5):
               + 2 * 2 * B * M * D * hidden                             # MLP
               + accounting.attn_flops(B, H, M, N, d) + accounting.attn_flops(B, H, M, N_text, d))
         out["keep_ratios"][str(th)] = {"ms": ms, "M": M, "TFLOP/s": fl / (ms * 1e-3) / 1e12,
-                                       "frac_bf16_peak": fl / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"], "flops": fl}
+                                       "frac_bf16_peak": fl / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"], "flops": fl,
+                                       "clocks": sampler.summary(m0, m1) if m1 > m0 else None}
     dense = out["keep_ratios"].get("1000")
     if dense:
         for th, e in out["keep_ratios"].items():
@@ -461,6 +464,70 @@ def block_leg(torch, A, w, thetas, peaks, hidden_mult=4, N_text=226, reps=5):
     return out
 
 
+def model_leg(torch, A, w, theta, sampler, L=2, T=8, hidden_mult=4, N_text=226, reps=3):
+    """A generation of T steps x L compute blocks as ONE CUDA graph (astraea_model_schedule_*), for the four rows of the
+    ablation study (Table 2): token-wise selection, SelectQ&K, Timestep-level and Fixed-token, all made from the same
+    budget schedule (dense step 0, then keep-ratio theta), next to the all-dense schedule of the same size."""
+    B, N, H, d, D, N_sel, n_always = w.B, w.N, w.H, w.d, w.D, w.N_v, w.N_t
+    hidden = hidden_mult * D
+    g = torch.Generator(device="cuda").manual_seed(123)
+    rn = lambda *s, scale=1.0: (scale * torch.randn(*s, device="cuda", generator=g)).to(torch.bfloat16)
+    Ws = []
+    for _ in range(L):
+        W = {}
+        for name, (o, i) in dict(wq=(D, D), wk=(D, D), wv=(D, D), wo=(D, D), wq2=(D, D), wo2=(D, D), w1=(hidden, D), w2=(D, hidden)).items():
+            W[name] = rn(o, i, scale=1 / math.sqrt(i))
+            W["b" + name[1:]] = rn(o, scale=0.1)
+        for name in ("s1", "t1", "g1", "s3", "t3", "g3"):
+            W[name] = rn(B, D, scale=0.3)
+        Ws.append((W, hidden))
+    tk, tv = [rn(B, N_text, H, d) for _ in range(L)], [rn(B, N_text, H, d) for _ in range(L)]
+    x0 = rn(B, N, D)
+    x1 = (x0.float() + 0.05 * torch.randn(B, N, D, device="cuda", generator=g)).to(torch.bfloat16)
+    x_in = [x0 if t % 2 == 0 else x1 for t in range(T)]
+    states = [dict(x_ref=x0.clone(), lse_cache=torch.zeros(B, H, N, device="cuda"),
+                   n_skip=torch.zeros(B, N_sel, dtype=torch.int32, device="cuda"),
+                   y_cache=torch.zeros(B, N, D, dtype=torch.bfloat16, device="cuda"),
+                   score=torch.zeros(B, N_sel, device="cuda"), idx_sel=torch.zeros(B, N, dtype=torch.int32, device="cuda"),
+                   idx_rem=None) for _ in range(L)]
+    ws = torch.zeros(A.astraea_block_workspace_bytes(B, H, N, d, hidden), dtype=torch.uint8, device="cuda")
+    k_keep = w.k_of(theta)
+    token_wise = [N_sel] + [k_keep] * (T - 1)
+    schedules = [("dense", A.VARIANT_TOKEN_WISE, [N_sel] * T),
+                 ("token-wise (Astraea)", A.VARIANT_TOKEN_WISE, token_wise),
+                 ("SelectQ&K", A.VARIANT_SELECT_QK, token_wise),
+                 ("Timestep-level", A.VARIANT_TIMESTEP, A.astraea_timestep_level_budgets(token_wise, N_sel)),
+                 ("Fixed-token", A.VARIANT_FIXED_TOKEN, token_wise)]
+    out = {"shape": {"B": B, "N": N, "D": D, "H": H, "d": d, "hidden": hidden, "N_text": N_text, "blocks": L, "steps": T},
+           "keep_ratio_permille": theta, "schedules": {}}
+    for name, variant, budgets in schedules:
+        sched = A.ModelSchedule(budgets, x_in, Ws, states, tk, tv, N_text, B, H, N, N_sel, d, w_alpha=float(1.0 / N),
+                                variant=variant, workspace=ws)
+        cool_down(torch)
+        sched.launch()
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+        torch.cuda.synchronize()
+        m0 = sampler.mark()
+        evs[0].record()
+        for i in range(reps):
+            sched.launch()
+            evs[i + 1].record()
+        torch.cuda.synchronize()
+        m1 = sampler.mark()
+        A.astraea_poll_error(ws)
+        sched.close()
+        ms = float(np.median([evs[i].elapsed_time(evs[i + 1]) for i in range(reps)]))
+        out["schedules"][name] = {"ms_per_generation": ms, "ms_per_step_and_block": ms / (T * L),
+                                  "tokens_computed_fraction": float(sum(b + n_always for b in budgets)) / (T * N),
+                                  "budgets": [int(b) for b in budgets], "clocks": sampler.summary(m0, m1) if m1 > m0 else None}
+    dense = out["schedules"]["dense"]["ms_per_generation"]
+    for e in out["schedules"].values():
+        e["speedup_vs_dense"] = dense / e["ms_per_generation"]
+    out["note"] = ("one graph launch per generation; SelectQ&K gathers the selected K / V rows in a pass of its own before the "
+                   "attention (twice the K / V bytes of those rows through HBM); Fixed-token scores and selects in block 0 only")
+    return out
+
+
 def e2e_leg(torch, A, w, theta, steps, barrier):
     """The same step through astraea_step_host: pinned host buffers in, merged output back, every step."""
     B, N, D = w.B, w.N, w.D
@@ -515,6 +582,7 @@ def main():
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-workloads", action="store_true", help="headline only")
     ap.add_argument("--no-next", action="store_true", help="skip the query projection of the selected rows (astraea_gathered_linear)")
+    ap.add_argument("--no-model", action="store_true", help="skip the scheduled generations (astraea_model_schedule_*: 2 blocks x 8 steps, four variants); --no-block skips them too")
     ap.add_argument("--no-block", action="store_true", help="skip the whole-block leg (astraea_block_step on the CogVideoX shape)")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -584,7 +652,11 @@ def main():
     # the whole compute block on the CogVideoX shape (head_dim 64 as well: before the long legs for the same reason)
     block = None
     if not args.no_block and extras:
-        block = block_leg(torch, A, synth.WORKLOADS["cogvideox"], (1000, 500, 250), peaks)
+        block = block_leg(torch, A, synth.WORKLOADS["cogvideox"], (1000, 500, 250), peaks, sampler)
+        torch.cuda.empty_cache()
+    model = None
+    if not args.no_model and not args.no_block and extras:
+        model = model_leg(torch, A, synth.WORKLOADS["cogvideox"], 500, sampler)
         torch.cuda.empty_cache()
 
     # ------------------------------------------------------------ headline: K consecutive steps, device-resident inputs
@@ -764,7 +836,7 @@ def main():
                                     "all": attn_fracs},
                 "worst_hbm_frac": {"value": hbm_fracs[worst_h], "where": worst_h, "of": "measured copy bandwidth",
                                    "of_nominal_8000": hbm_fracs[worst_h] * peaks["hbm_gbs"] / NOMINAL_HBM_GBS, "all": hbm_fracs},
-                "keep_ratio_sweep": sweep, "workloads": workloads, "next": nxt, "block": block, "e2e": e2e, "cpu_baseline": cpu,
+                "keep_ratio_sweep": sweep, "workloads": workloads, "next": nxt, "block": block, "model_schedules": model, "e2e": e2e, "cpu_baseline": cpu,
                 "bench_seconds": time.perf_counter() - t_start}
         print(json.dumps(line))
     if world > 1:
