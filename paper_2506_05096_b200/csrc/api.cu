@@ -625,7 +625,10 @@ struct astraea_session {
     int32_t *n_skip, *idx_sel, *idx_rem;
     void *workspace;
     size_t workspace_bytes;
-    cudaStream_t stream;            // score, select, attention, refresh
+    cudaStream_t stream;            // score, select, refresh, attention of the even head groups
+    cudaStream_t stream2;           // attention of the odd head groups: the CTAs of one group fill the SMs that the last,
+                                    // partial wave of the group before leaves idle (two heads of 128 query tiles are 1.73
+                                    // waves of CTAs: one after the other every group would pay for 2)
     cudaStream_t copy_in, copy_out; // host -> device and device -> host copies, overlapped with the compute stream
     cudaStream_t gather;            // zero-copy fetches of the selected q rows from a pinned host buffer
     cudaEvent_t ev_sel;             // the selection of this step is known
@@ -650,7 +653,7 @@ void astraea_session_destroy(astraea_session *s)
         if (s->ev_in[g]) cudaEventDestroy(s->ev_in[g]);
         if (s->ev_attn[g]) cudaEventDestroy(s->ev_attn[g]);
     }
-    cudaStream_t streams[] = {s->stream, s->copy_in, s->copy_out, s->gather};
+    cudaStream_t streams[] = {s->stream, s->stream2, s->copy_in, s->copy_out, s->gather};
     for (cudaStream_t st : streams) if (st) cudaStreamDestroy(st);
     delete s;
 }
@@ -668,6 +671,7 @@ int32_t astraea_session_create(astraea_session **session, int B, int H, int N, i
     s->tensor_bytes = (size_t)B * N * H * d * 2;
     s->workspace_bytes = astraea_workspace_bytes(ASTRAEA_OP_STEP, B, H, N, N, d);
     cudaError_t e = cudaStreamCreateWithFlags(&s->stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&s->stream2, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&s->copy_in, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&s->copy_out, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&s->gather, cudaStreamNonBlocking);
@@ -761,12 +765,14 @@ int32_t astraea_step_host(astraea_session *s, const void *x_cur, const void *q, 
     if (rc == ASTRAEA_OK)
         rc = astraea_scatter_reuse(s->x_ref, s->x_cur, s->idx_sel, B, N, M, D, ASTRAEA_SCATTER_SRC_FULL, s->workspace, s->stream);
     if (rc != ASTRAEA_OK) return rc;
+    e = cudaEventRecord(s->ev_sel, s->stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s->stream2, s->ev_sel, 0);
+    if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_step_host: %s", cudaGetErrorString(e));
     if (q_mapped) {
         // the selected rows of q, straight from the host buffer, head group by head group on a stream of its own (so
         // that a group's attention waits for its own columns only and the fetches run under the attention of the
         // groups before)
-        e = cudaEventRecord(s->ev_sel, s->stream);
-        if (e == cudaSuccess) e = cudaStreamWaitEvent(s->gather, s->ev_sel, 0);
+        e = cudaStreamWaitEvent(s->gather, s->ev_sel, 0);
         for (int g = 0; g < groups && e == cudaSuccess; ++g) {
             const size_t off = (size_t)head_lo(g) * d * 2;
             rc = launch_scatter(static_cast<char *>(s->q) + off, static_cast<const char *>(q_mapped) + off, s->idx_sel, B, N, M,
@@ -778,8 +784,9 @@ int32_t astraea_step_host(astraea_session *s, const void *x_cur, const void *q, 
         if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_step_host (fetch of the selected q rows): %s", cudaGetErrorString(e));
     }
     for (int g = 0; g < groups; ++g) {
-        e = cudaStreamWaitEvent(s->stream, s->ev_in[g], 0);
-        if (e == cudaSuccess && q_mapped) e = cudaStreamWaitEvent(s->stream, s->ev_q[g], 0);
+        cudaStream_t cs = (g & 1) ? s->stream2 : s->stream;
+        e = cudaStreamWaitEvent(cs, s->ev_in[g], 0);
+        if (e == cudaSuccess && q_mapped) e = cudaStreamWaitEvent(cs, s->ev_q[g], 0);
         if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_step_host: %s", cudaGetErrorString(e));
         if (M > 0) {
             AttnArgs a;
@@ -793,10 +800,10 @@ int32_t astraea_step_host(astraea_session *s, const void *x_cur, const void *q, 
             a.flags = 0;
             a.err_word = reinterpret_cast<int *>(s->workspace);
             a.head_begin = head_lo(g); a.head_count = head_lo(g + 1) - head_lo(g);
-            rc = launch_sparse_attn(a, s->stream);
+            rc = launch_sparse_attn(a, cs);
             if (rc != ASTRAEA_OK) return rc;
         }
-        e = cudaEventRecord(s->ev_attn[g], s->stream);
+        e = cudaEventRecord(s->ev_attn[g], cs);
         // copy-out stream: the group's columns of the output cache (computed and reused rows alike)
         if (e == cudaSuccess) e = cudaStreamWaitEvent(s->copy_out, s->ev_attn[g], 0);
         const size_t off = (size_t)head_lo(g) * d * 2, width = (size_t)(head_lo(g + 1) - head_lo(g)) * d * 2;
@@ -808,6 +815,8 @@ int32_t astraea_step_host(astraea_session *s, const void *x_cur, const void *q, 
     e = cudaStreamSynchronize(s->copy_out);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s->copy_in);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s->gather);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s->stream2);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s->stream);      // the refresh of x_ref runs beside the attention
     if (e != cudaSuccess) return fail(ASTRAEA_ERR_CUDA, "astraea_step_host (copy out): %s", cudaGetErrorString(e));
     s->steps++;
     return astraea_poll_error(s->workspace, s->stream);
