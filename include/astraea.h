@@ -56,6 +56,8 @@ extern "C" {
 #define ASTRAEA_ATTN_COMPACT_OUT  1u         /* out is [B,M,H,d] and lse_out [B,H,M] (row r of the index list), not the caches */
 #define ASTRAEA_ATTN_SMALL_CTAS   2u         /* head_dim 64 / 72: one 128-row query tile per CTA, two CTAs per SM, whatever the
                                               * launch-time estimate says (without the flag the library picks the faster shape) */
+#define ASTRAEA_ATTN_WHOLE_KEYS   4u         /* every CTA runs over all keys: the last, partial round of CTAs is never split by keys
+                                              * (see `workspace` of astraea_sparse_attn) */
 /* flags of astraea_gathered_linear */
 #define ASTRAEA_LINEAR_COMPACT_OUT 1u        /* y is [B,M,N_out] (row r of the index list), not the cache [B,N,N_out] */
 #define ASTRAEA_LINEAR_COMPACT_IN  2u        /* x is [B,M,K]: row r is the row of token idx[b,r] (output of a layer run with COMPACT_OUT) */
@@ -165,8 +167,12 @@ int32_t astraea_select(const float *score, int B, int N_sel, int k, int n_always
  *   out     : bf16 [B, N, H, d]  (or [B, M, H, d] compact)
  *   lse_out : fp32 [B, H, N]     (or [B, H, M] compact); may be NULL
  *   scale   : 0 => 1/sqrt(d)
- *   workspace : at least astraea_workspace_bytes(ASTRAEA_OP_SPARSE_ATTN, B, H, N, M, d) bytes,
- *               256-byte aligned; its first word is an error word (see astraea_poll_error)
+ *   workspace : 256-byte aligned, at least 256 bytes (with kv_idx: see above); its first word is an error word (see
+ *               astraea_poll_error).  With astraea_workspace_bytes(ASTRAEA_OP_SPARSE_ATTN, B, H, N, M, d) bytes (a few
+ *               tens of MB at most) a launch of only a few rounds of CTAs may split the keys of its last, partial round:
+ *               each of those CTAs is replaced by 2..8 CTAs that take a share of the keys each and leave fp32 rows
+ *               in the workspace, which a second kernel merges (out = sum_i exp(lse_i - lse) out_i).  Results agree
+ *               with the unsplit launch to fp32 rounding.  A workspace serves one call at a time.
  * Arithmetic: bf16 operands, fp32 logits, softmax and accumulation; probabilities are
  * rounded to bf16 before the P.V product; outputs rounded to bf16.
  * M = 0 is valid: nothing is launched and the caches are untouched.
@@ -180,6 +186,15 @@ int32_t astraea_sparse_attn(const void *q, const void *k, const void *v,
                             void *out, float *lse_out,
                             int B, int H, int N, int d, float scale, uint32_t flags,
                             void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * The launch schedule astraea_sparse_attn would pick for a problem (host logic only, no GPU work): small_ctas = 1 when
+ * it launches one query tile per CTA; otherwise the last split_units CTAs are replaced by `split` CTAs each that share
+ * the keys (split = 1, split_units = 0: every CTA runs over all keys).  workspace_bytes as given to astraea_sparse_attn.
+ * Errors: INVALID_ARG, UNSUPPORTED.
+ */
+int32_t astraea_sparse_attn_plan(int B, int H, int N, int M, int d, uint32_t flags, size_t workspace_bytes,
+                                 int32_t *small_ctas, int32_t *split_units, int32_t *split);
 
 /*
  * Cross-attention of the selected rows (Section 3.2: the layers of a block other than self-attention are
@@ -207,9 +222,10 @@ int32_t astraea_sparse_cross_attn(const void *q, const void *k, const void *v,
  * GPU that loads the library, held until the process exits) and calls no cudaMalloc, cudaFree or
  * other allocating routine.  Arguments (flags included), validation, arithmetic and results are those of
  * astraea_sparse_attn without the workspace pair: the two entry points share one code path.
- *   - Problems whose scratch need (astraea_workspace_bytes(ASTRAEA_OP_SPARSE_ATTN, ...), or
- *     ASTRAEA_OP_SPARSE_ATTN_KV with kv_idx) exceeds ASTRAEA_NOALLOC_SCRATCH_BYTES are rejected with
- *     ASTRAEA_ERR_WORKSPACE_TOO_SMALL.  With kv_idx that is nearly always the case: the gathered key / value
+ *   - Without kv_idx the 256 bytes every launch needs fit the array: nothing is rejected for its size, and
+ *     the launch never splits its last round of CTAs by keys (there is no room for the shares).  With kv_idx a problem
+ *     whose need (astraea_workspace_bytes(ASTRAEA_OP_SPARSE_ATTN_KV, ...)) exceeds ASTRAEA_NOALLOC_SCRATCH_BYTES is
+ *     rejected with ASTRAEA_ERR_WORKSPACE_TOO_SMALL, which is nearly always the case: the gathered key / value
  *     rows (2 * B * M_kv * H * d bf16) must fit the array.
  *   - The first call on a device resolves the array's device address (with that device current);
  *     make that first call before any stream capture.

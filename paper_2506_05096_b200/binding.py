@@ -21,6 +21,7 @@ DELTA_MEAN_ABS, DELTA_MEAN_SQ, DELTA_MEAN_SIGNED = 0, 1, 2
 LSE_SUM_EXP, LSE_LOG = 0, 1
 ATTN_COMPACT_OUT = 1
 ATTN_SMALL_CTAS = 2
+ATTN_WHOLE_KEYS = 4
 SCATTER_SRC_FULL = 1
 LINEAR_COMPACT_OUT, LINEAR_COMPACT_IN, LINEAR_GELU, LINEAR_COMPACT_RES = 1, 2, 4, 8
 LN_COMPACT_IN, LN_COMPACT_OUT = 1, 2
@@ -31,7 +32,7 @@ N_SKIP_CLAMP = 80
 NOALLOC_SCRATCH_BYTES = 4096
 
 EXPORTS = [
-    "astraea_score", "astraea_score_partial", "astraea_score_combine", "astraea_select", "astraea_sparse_attn", "astraea_sparse_cross_attn", "astraea_sparse_attn_noalloc", "astraea_scatter_reuse", "astraea_step",
+    "astraea_score", "astraea_score_partial", "astraea_score_combine", "astraea_select", "astraea_sparse_attn", "astraea_sparse_attn_plan", "astraea_sparse_cross_attn", "astraea_sparse_attn_noalloc", "astraea_scatter_reuse", "astraea_step",
     "astraea_gathered_linear", "astraea_gathered_linear_residual", "astraea_layernorm_modulate",
     "astraea_block_step", "astraea_block_workspace_bytes", "astraea_model_schedule_create", "astraea_model_schedule_launch",
     "astraea_model_schedule_destroy", "astraea_timestep_level_budgets", "astraea_schedule_create", "astraea_schedule_launch", "astraea_schedule_destroy",
@@ -82,6 +83,8 @@ def lib() -> ctypes.CDLL:
                                                                                c_i, c_i, c_i, c_i, c_i, c_f, c_u, c_p, c_sz, c_p]
         L.astraea_sparse_attn_noalloc.argtypes = [c_p, c_p, c_p] + [c_i64] * 9 + [c_p, c_i, c_p, c_i, c_p, c_p,
                                                                                  c_i, c_i, c_i, c_i, c_f, c_u, c_p]
+        L.astraea_sparse_attn_plan.argtypes = [c_i, c_i, c_i, c_i, c_i, c_u, c_sz, c_p, c_p, c_p]
+        L.astraea_sparse_attn_plan.restype = ctypes.c_int32
         L.astraea_scatter_reuse.argtypes = [c_p, c_p, c_p, c_i, c_i, c_i, c_i, c_u, c_p, c_p]
         L.astraea_gathered_linear.argtypes = [c_p, c_p, c_i, c_p, c_p, c_p, c_i, c_i, c_i, c_i, c_u, c_p, c_sz, c_p]
         L.astraea_gathered_linear_residual.argtypes = [c_p, c_p, c_i, c_p, c_p, c_p, c_p, c_p, c_i, c_i, c_i, c_i, c_u, c_p, c_sz, c_p]
@@ -197,6 +200,15 @@ def astraea_sparse_attn(q, k, v, q_strides, k_strides, v_strides, q_idx, M, out,
                                      _ptr(q_idx), M, _ptr(kv_idx), M_kv, _ptr(out), _ptr(lse_out),
                                      B, H, N, d, scale, flags, _ptr(workspace),
                                      workspace.numel() if workspace is not None else 0, _stream(stream)))
+
+
+def astraea_sparse_attn_plan(B, H, N, M, d, flags=0, workspace_bytes=None) -> dict:
+    """The launch schedule astraea_sparse_attn would pick (host logic only).  workspace_bytes None: the full size."""
+    if workspace_bytes is None:
+        workspace_bytes = astraea_workspace_bytes(OP_SPARSE_ATTN, B, H, N, M, d)
+    r = (ctypes.c_int32 * 3)()
+    _check(lib().astraea_sparse_attn_plan(B, H, N, M, d, flags, workspace_bytes, ctypes.byref(r, 0), ctypes.byref(r, 4), ctypes.byref(r, 8)))
+    return {"small_ctas": bool(r[0]), "split_units": int(r[1]), "split": int(r[2])}
 
 
 def astraea_sparse_attn_noalloc(q, k, v, q_strides, k_strides, v_strides, q_idx, M, out, lse_out, B, H, N, d,

@@ -152,7 +152,7 @@ static int32_t sparse_attn_entry(const char *fn, int N_kv, const void *q, const 
     REQUIRE(M >= 0 && M <= N, "%s: M=%d outside [0, N=%d]", fn, M, N);
     if (d != 64 && d != 72 && d != 128)
         return fail(ASTRAEA_ERR_UNSUPPORTED, "%s: head_dim %d not in {64, 72, 128}", fn, d);
-    if (flags & ~(ASTRAEA_ATTN_COMPACT_OUT | ASTRAEA_ATTN_SMALL_CTAS)) return fail(ASTRAEA_ERR_UNSUPPORTED, "%s: unknown flags 0x%x", fn, flags);
+    if (flags & ~(ASTRAEA_ATTN_COMPACT_OUT | ASTRAEA_ATTN_SMALL_CTAS | ASTRAEA_ATTN_WHOLE_KEYS)) return fail(ASTRAEA_ERR_UNSUPPORTED, "%s: unknown flags 0x%x", fn, flags);
     REQUIRE(q && k && v && out, "%s: null q, k, v or out", fn);
     REQUIRE(aligned16(q) && aligned16(k) && aligned16(v) && aligned16(out), "%s: q, k, v, out must be 16-byte aligned", fn);
     REQUIRE(q_sn % 8 == 0 && k_sn % 8 == 0 && v_sn % 8 == 0 && q_sh % 8 == 0 && k_sh % 8 == 0 && v_sh % 8 == 0 &&
@@ -161,7 +161,8 @@ static int32_t sparse_attn_entry(const char *fn, int N_kv, const void *q, const 
     REQUIRE(q_sn >= d && k_sn >= d && v_sn >= d && q_sh > 0 && k_sh > 0 && v_sh > 0 && q_sb >= 0 && k_sb >= 0 && v_sb >= 0,
             "%s: strides must be positive and token stride >= head_dim", fn);
     REQUIRE(scale >= 0.f, "%s: scale must be >= 0 (0 selects 1/sqrt(d))", fn);
-    const size_t ws_need = kv_idx ? attn_kv_workspace_bytes(B, H, M_kv, d) : attn_workspace_bytes(B, H, N, M, d);
+    // without kv_idx the error word is all a launch needs; what lies behind it lets the launch split its last round of CTAs
+    const size_t ws_need = kv_idx ? attn_kv_workspace_bytes(B, H, M_kv, d) : 256;
     if (!workspace || workspace_bytes < ws_need)
         return fail(ASTRAEA_ERR_WORKSPACE_TOO_SMALL, "%s: workspace of %zu bytes, need %zu", fn,
                     workspace_bytes, ws_need);
@@ -180,6 +181,7 @@ static int32_t sparse_attn_entry(const char *fn, int N_kv, const void *q, const 
     a.N_tok = N;
     if (N_kv > 0) a.N = N_kv;          // keys and values of another sequence: N stays the token count of q / out
     if (kv_idx) return launch_sparse_attn_kv(a, kv_idx, M_kv, workspace, (cudaStream_t)stream);
+    if (workspace_bytes > 256) { a.split_ws = static_cast<char *>(workspace) + 256; a.split_ws_bytes = workspace_bytes - 256; }
     return launch_sparse_attn(a, (cudaStream_t)stream);
 }
 
@@ -194,6 +196,22 @@ int32_t astraea_sparse_attn(const void *q, const void *k, const void *v,
 {
     return sparse_attn_entry("astraea_sparse_attn", 0, q, k, v, q_sb, q_sh, q_sn, k_sb, k_sh, k_sn, v_sb, v_sh, v_sn,
                              q_idx, M, kv_idx, M_kv, out, lse_out, B, H, N, d, scale, flags, workspace, workspace_bytes, stream);
+}
+
+int32_t astraea_sparse_attn_plan(int B, int H, int N, int M, int d, uint32_t flags, size_t workspace_bytes,
+                                 int32_t *small_ctas, int32_t *split_units, int32_t *split)
+{
+    REQUIRE(B > 0 && H > 0 && N > 0 && M >= 0 && M <= N, "astraea_sparse_attn_plan: bad sizes");
+    REQUIRE(small_ctas && split_units && split, "astraea_sparse_attn_plan: null result pointer");
+    if (d != 64 && d != 72 && d != 128) return fail(ASTRAEA_ERR_UNSUPPORTED, "astraea_sparse_attn_plan: head_dim %d not in {64, 72, 128}", d);
+    AttnArgs a = {};
+    a.B = B; a.H = H; a.N = N; a.N_tok = N; a.M = M; a.d = d; a.flags = flags;
+    static char nowhere;                       // never dereferenced: the plan only asks whether there is room
+    if (workspace_bytes > 256) { a.split_ws = &nowhere; a.split_ws_bytes = workspace_bytes - 256; }
+    int s = 0, u = 0, k = 1;
+    if (M > 0) attn_plan(a, &s, &u, &k);
+    *small_ctas = s; *split_units = u; *split = k;
+    return ASTRAEA_OK;
 }
 
 int32_t astraea_sparse_cross_attn(const void *q, const void *k, const void *v,
@@ -298,16 +316,23 @@ int32_t astraea_layernorm_modulate(const void *x, const int32_t *idx, int M, con
 }
 
 // ------------------------------------------------------------------ a whole compute block
-// workspace: [256 bytes: error word | gathered keys and values of the SelectQ&K variant] [select scratch]
+// workspace: [256 bytes: error word | gathered keys and values of the SelectQ&K variant, or the key shares of a split
+//             self-attention launch] [select scratch]
 //            [5 token-sized buffers] [hidden-sized buffer]
 // (the first part is laid out as the workspace of astraea_sparse_attn with kv_idx, so that every call of the block
 // shares the one error word at the very start)
 static size_t block_buffer_bytes(int B, int N, int width) { return align_up((size_t)B * N * width * 2, 256); }
+// the head of the block's workspace serves the self-attention: gathered keys / values (SelectQ&K) or the key shares of a split launch
+static size_t block_attn_region_bytes(int B, int H, int N, int d)
+{
+    const size_t kv = attn_kv_workspace_bytes(B, H, N, d), plain = attn_workspace_bytes(B, H, N, N, d);
+    return align_up(kv > plain ? kv : plain, 256);
+}
 
 size_t astraea_block_workspace_bytes(int B, int H, int N, int d, int hidden)
 {
     if (B <= 0 || H <= 0 || N <= 0 || d <= 0 || hidden <= 0) return 0;
-    return align_up(attn_kv_workspace_bytes(B, H, N, d), 256) + align_up(select_workspace_bytes(B, N), 256) +
+    return block_attn_region_bytes(B, H, N, d) + align_up(select_workspace_bytes(B, N), 256) +
            5 * block_buffer_bytes(B, N, H * d) + block_buffer_bytes(B, N, hidden);
 }
 
@@ -337,7 +362,7 @@ int32_t astraea_block_step(const void *x, const astraea_block_weights *w, const 
     REQUIRE(score && (idx_sel || M == 0), "astraea_block_step: null score or idx_sel");
     char *ws = reinterpret_cast<char *>(workspace);
     void *err = ws;                                     // the error word of every call below
-    char *p = ws + align_up(attn_kv_workspace_bytes(B, H, N, d), 256);
+    char *p = ws + block_attn_region_bytes(B, H, N, d);
     void *sel_ws = p; p += align_up(select_workspace_bytes(B, N), 256);
     const size_t tb = block_buffer_bytes(B, N, D);
     void *bufA = p, *bufQ = p + tb, *bufK = p + 2 * tb, *bufV = p + 3 * tb, *bufO = p + 4 * tb, *bufU = p + 5 * tb;
@@ -361,7 +386,7 @@ int32_t astraea_block_step(const void *x, const astraea_block_weights *w, const 
     if (rc == ASTRAEA_OK) rc = astraea_gathered_linear(bufA, idx_sel, M, w->wq, w->bq, bufQ, B, N, D, D, 0u, err, 256, stream);
     if (rc == ASTRAEA_OK && !select_qk)
         rc = astraea_sparse_attn(bufQ, bufK, bufV, sb, sh, sn, sb, sh, sn, sb, sh, sn, idx_sel, M, nullptr, 0, bufO, st->lse_cache,
-                                 B, H, N, d, 0.f, 0u, err, 256, stream);
+                                 B, H, N, d, 0.f, 0u, ws, block_attn_region_bytes(B, H, N, d), stream);
     if (rc == ASTRAEA_OK && select_qk)       // the listed key / value rows are gathered into the head of the workspace
         rc = astraea_sparse_attn(bufQ, bufK, bufV, sb, sh, sn, sb, sh, sn, sb, sh, sn, idx_sel, M, idx_sel, M, bufO, st->lse_cache,
                                  B, H, N, d, 0.f, 0u, ws, attn_kv_workspace_bytes(B, H, N, d), stream);

@@ -133,6 +133,12 @@ struct Params {
     int compact;
     int h0;                      // first head of this launch
     int *err_word;
+    // The grid is one-dimensional: CTA id -> (query-tile group x, head y, batch z), x fastest.  CTAs [0, n_full) take
+    // their rows against all keys.  Every later group of `split` CTAs shares one such unit and splits its KEY tiles
+    // evenly: each writes normalised fp32 rows and their LSE to part_o / part_lse, which merge_parts_kernel combines.
+    int tiles_x, heads;
+    int n_full, split;
+    float *part_o, *part_lse;    // [part][kTilesM * 128 rows][head_dim] and [part][kTilesM * 128 rows]
 };
 
 __device__ __forceinline__ float ex2(float x) {
@@ -365,7 +371,8 @@ __device__ __forceinline__ void pass_sync() {
 // tile: its query tile; par: which key tiles it takes (j = par, par + kSplit, ...)
 template <class C>
 __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, int tile, int par, uint8_t *sQ_gen, uint32_t tmem,
-                                             int m_base, int h, int b, int n_tiles, volatile int *abort_flag, volatile int *redo_flag, float2 *xchg)
+                                             int m_base, int h, int b, int n_tiles, int key0, int part,
+                                             volatile int *abort_flag, volatile int *redo_flag, float2 *xchg)
 {
     const int wtid = threadIdx.x & 127;
     const int warp = __shfl_sync(0xffffffffu, wtid >> 5, 0);       // warp-uniform
@@ -397,7 +404,8 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     st.t_s0 = t_row + tile * C::kSBufs * C::kBlockN;
     st.t_o = t_row + C::kColO + tile * C::kOStride;
     st.bar_s = bar.s + 32 * tile; st.bar_p = bar.p + 32 * tile; st.bar_done = bar.done + 8 * tile;
-    st.N = p.N; st.abort_flag = abort_flag; st.err_word = p.err_word;
+    st.N = p.N - key0;                                           // keys from this CTA's first key tile on
+    st.abort_flag = abort_flag; st.err_word = p.err_word;
     st.ref_x = &xchg[wtid].x; st.ref_bar = 3 + tile; st.redo_flag = redo_flag;
 
     const int m = m_base + wtid;
@@ -466,6 +474,35 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     constexpr int ncol = C::kMain / 2;                           // O columns this thread writes
     const int col0 = par * ncol;
     const float inv_l = 1.0f / l_sum;
+    if (part >= 0) {
+        // a share of the keys only: the normalised row and its LSE go to the workspace in fp32 (every row of the tile,
+        // listed or not; the merge knows which ones count).  A CTA that gave up marks its rows with NaN.
+        const size_t prow = (size_t)part * (C::kTilesM * kBlockM) + tile * kBlockM + wtid;
+        float *po = p.part_o + prow * C::kDH;
+        if (par == 0)
+            p.part_lse[prow] = *abort_flag ? __int_as_float(0x7fc00000) : st.m_ref * p.scale + st.shift * 0.6931471805599453f + logf(l_sum);
+#pragma unroll
+        for (int cc = 0; cc < ncol; cc += 32) {
+            const int c = col0 + cc;
+            uint32_t o[32];
+            tmem_ld32(st.t_o + c, o);
+            tc_wait_ld();
+#pragma unroll
+            for (int v = 0; v < 8; ++v)
+                *reinterpret_cast<float4 *>(po + c + v * 4) = make_float4(__uint_as_float(o[4 * v]) * inv_l, __uint_as_float(o[4 * v + 1]) * inv_l,
+                                                                           __uint_as_float(o[4 * v + 2]) * inv_l, __uint_as_float(o[4 * v + 3]) * inv_l);
+        }
+        if (C::kTail && par == kSplit - 1) {
+            uint32_t o[8];
+            tmem_ld8(st.t_o + C::kMain, o);
+            tc_wait_ld();
+#pragma unroll
+            for (int v = 0; v < 2; ++v)
+                *reinterpret_cast<float4 *>(po + C::kMain + v * 4) = make_float4(__uint_as_float(o[4 * v]) * inv_l, __uint_as_float(o[4 * v + 1]) * inv_l,
+                                                                                  __uint_as_float(o[4 * v + 2]) * inv_l, __uint_as_float(o[4 * v + 3]) * inv_l);
+        }
+        return;
+    }
     __nv_bfloat16 *dst = nullptr;
     if (tok >= 0 && !*abort_flag) {
         const size_t orow = p.compact ? ((size_t)b * p.M + m) : ((size_t)b * p.N_tok + tok);
@@ -538,9 +575,19 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 
     const int tid = threadIdx.x;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);        // warp-uniform
-    const int m0 = blockIdx.x * (kTilesM * kBlockM), h = p.h0 + blockIdx.y, b = blockIdx.z;
     constexpr int kBlockN = C::kBlockN;
-    const int n_tiles = (p.N + kBlockN - 1) / kBlockN;
+    int unit = blockIdx.x, kpart = 0, ksplit = 1;
+    int part = -1;                                                 // >= 0: this CTA takes a share of the keys only
+    if (unit >= p.n_full) {
+        part = unit - p.n_full;
+        kpart = part % p.split; ksplit = p.split;
+        unit = p.n_full + part / p.split;
+    }
+    const int m0 = (unit % p.tiles_x) * (kTilesM * kBlockM), h = p.h0 + (unit / p.tiles_x) % p.heads, b = unit / (p.tiles_x * p.heads);
+    const int n_tiles_all = (p.N + kBlockN - 1) / kBlockN;
+    const int tile0 = n_tiles_all * kpart / ksplit;                // first key tile of this CTA (split <= 8: no overflow)
+    const int n_tiles = n_tiles_all * (kpart + 1) / ksplit - tile0;
+    const int key0 = tile0 * kBlockN;
     // the last CTA of a head may have rows in its first query tile only: the second tile's warps and MMAs are skipped
     const int q_tiles = (m0 + kBlockM < p.M) ? kTilesM : 1;
 
@@ -582,7 +629,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         const int wg = warp >> 2;
         const int tile = wg / kSplit, par = wg % kSplit;
         if (tile < q_tiles)
-            softmax_role<C>(p, bar, tile, par, smem_gen + tile * C::kQTileBytes, tmem, m0 + tile * kBlockM, h, b, n_tiles,
+            softmax_role<C>(p, bar, tile, par, smem_gen + tile * C::kQTileBytes, tmem, m0 + tile * kBlockM, h, b, n_tiles, key0, part,
                              &abort_flag, &redo_flag, xchg[tile]);
         else pass_sync<C>();
     } else if (warp == kProducerWarp) {
@@ -600,9 +647,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                 mbar_arrive_expect_tx(bar.kf + 8 * st, C::kLoadBytes);
 #pragma unroll
                 for (int ch = 0; ch < C::kChunks; ++ch)
-                    tma_load_4d(sK + st * C::kTileBytes + ch * C::kChunkBytes, &tmap_k, bar.kf + 8 * st, ch * 64, j * kBlockN, h, b);
+                    tma_load_4d(sK + st * C::kTileBytes + ch * C::kChunkBytes, &tmap_k, bar.kf + 8 * st, ch * 64, key0 + j * kBlockN, h, b);
                 if (C::kTail)
-                    tma_load_4d(sK + st * C::kTileBytes + C::kChunks * C::kChunkBytes, &tmap_k_tail, bar.kf + 8 * st, C::kMain, j * kBlockN, h, b);
+                    tma_load_4d(sK + st * C::kTileBytes + C::kChunks * C::kChunkBytes, &tmap_k_tail, bar.kf + 8 * st, C::kMain, key0 + j * kBlockN, h, b);
             }
             __syncwarp();
         };
@@ -613,9 +660,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                 mbar_arrive_expect_tx(bar.vf + 8 * st, C::kLoadBytes);
 #pragma unroll
                 for (int ch = 0; ch < C::kChunks; ++ch)
-                    tma_load_4d(sV + st * C::kTileBytes + ch * C::kChunkBytes, &tmap_v, bar.vf + 8 * st, ch * 64, j * kBlockN, h, b);
+                    tma_load_4d(sV + st * C::kTileBytes + ch * C::kChunkBytes, &tmap_v, bar.vf + 8 * st, ch * 64, key0 + j * kBlockN, h, b);
                 if (C::kTail)
-                    tma_load_4d(sV + st * C::kTileBytes + C::kChunks * C::kChunkBytes, &tmap_v_tail, bar.vf + 8 * st, C::kMain, j * kBlockN, h, b);
+                    tma_load_4d(sV + st * C::kTileBytes + C::kChunks * C::kChunkBytes, &tmap_v_tail, bar.vf + 8 * st, C::kMain, key0 + j * kBlockN, h, b);
             }
             __syncwarp();
         };
@@ -740,6 +787,60 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     if (warp == kIssuerWarp) tmem_dealloc(tmem, kTmemCols);
 }
 
+// Combines the key shares of the split units: row = sum_i w_i row_i with w_i = exp(lse_i - LSE), LSE = log sum_i exp(lse_i)
+// (each share is a complete softmax over its own keys).  One thread per (row, 8 columns); grid (head_dim / 8, units).
+template <int DH, int ROWS>
+__global__ void __launch_bounds__(ROWS) merge_parts_kernel(const Params p)
+{
+    constexpr int kChunksRow = DH / 8;
+    const int unit = p.n_full + blockIdx.y;
+    const int m0 = (unit % p.tiles_x) * ROWS, h = p.h0 + (unit / p.tiles_x) % p.heads, b = unit / (p.tiles_x * p.heads);
+    const int idx = blockIdx.x * ROWS + threadIdx.x;
+    const int r = idx / kChunksRow, c = idx - r * kChunksRow;
+    const int m = m0 + r;
+    if (m >= p.M) return;
+    const int tok = p.q_idx ? __ldg(p.q_idx + (size_t)b * p.M + m) : m;
+    if ((unsigned)tok >= (unsigned)p.N_tok || (p.q_idx && m > 0 && __ldg(p.q_idx + (size_t)b * p.M + m - 1) >= tok)) return;   // reported by the attention kernel
+    const size_t part0 = (size_t)blockIdx.y * p.split;
+    float lse[8], mx = -INFINITY;
+    bool gave_up = false;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        lse[i] = -INFINITY;
+        if (i < p.split) {
+            lse[i] = __ldg(p.part_lse + (part0 + i) * ROWS + r);
+            gave_up |= lse[i] != lse[i];
+            mx = fmaxf(mx, lse[i]);
+        }
+    }
+    if (gave_up) return;                                            // a share was not finished (a wait ran out): the row stays as it is
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, wsum = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        if (i < p.split) {
+            const float w = __expf(lse[i] - mx);
+            wsum += w;
+            const float4 *src = reinterpret_cast<const float4 *>(p.part_o + ((part0 + i) * ROWS + r) * DH + c * 8);
+            const float4 a = __ldg(src), d = __ldg(src + 1);
+            acc[0] += w * a.x; acc[1] += w * a.y; acc[2] += w * a.z; acc[3] += w * a.w;
+            acc[4] += w * d.x; acc[5] += w * d.y; acc[6] += w * d.z; acc[7] += w * d.w;
+        }
+    }
+    const float inv = 1.0f / wsum;
+    uint32_t w4[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        __nv_bfloat162 v2 = __floats2bfloat162_rn(acc[2 * i] * inv, acc[2 * i + 1] * inv);
+        w4[i] = *reinterpret_cast<uint32_t *>(&v2);
+    }
+    const size_t orow = p.compact ? ((size_t)b * p.M + m) : ((size_t)b * p.N_tok + tok);
+    *reinterpret_cast<uint4 *>(p.out + (orow * p.H + h) * DH + c * 8) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+    if (p.lse_out && c == 0) {
+        const size_t li = p.compact ? (((size_t)b * p.H + h) * p.M + m) : (((size_t)b * p.H + h) * p.N_tok + tok);
+        p.lse_out[li] = mx + logf(wsum);
+    }
+}
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -765,8 +866,16 @@ int32_t make_kv_map(CUtensorMap *map, const void *base, int B, int H, int N, int
     return ASTRAEA_OK;
 }
 
+// The last, partial round of CTAs of a launch: its `units` CTAs are replaced by `split` CTAs each, every one with a
+// share of the key tiles, and merged afterwards (split 1: nothing is split).
+struct SplitPlan { int units = 0, split = 1; };
+
+constexpr int kMaxSplit = 8;                 // shares per unit
+constexpr int kMaxSplitParts = 2 * 148;      // shares per launch (what the workspace holds)
+constexpr int kMinSplitKeyTiles = 16;        // key tiles per share at least
+
 template <int DH, int TM>
-int32_t launch_dh(const AttnArgs &a, cudaStream_t stream)
+int32_t launch_dh(const AttnArgs &a, cudaStream_t stream, SplitPlan plan = SplitPlan())
 {
     using C = Cfg<DH, TM>;
     CUtensorMap mk, mv, mkt, mvt;
@@ -801,14 +910,44 @@ int32_t launch_dh(const AttnArgs &a, cudaStream_t stream)
     p.compact = (a.flags & ASTRAEA_ATTN_COMPACT_OUT) ? 1 : 0;
     p.err_word = a.err_word;
     p.h0 = a.head_begin;
-    dim3 grid((a.M + TM * kBlockM - 1) / (TM * kBlockM), a.head_count > 0 ? a.head_count : a.H, a.B);
+    p.tiles_x = (a.M + TM * kBlockM - 1) / (TM * kBlockM);
+    p.heads = a.head_count > 0 ? a.head_count : a.H;
+    const long long units = (long long)p.tiles_x * p.heads * a.B;
+    if (units + (long long)plan.units * (plan.split - 1) > 0x7fffffffll) return fail(ASTRAEA_ERR_INVALID_ARG, "astraea_sparse_attn: too many CTAs");
+    const bool split = TM == 2 && plan.split > 1 && plan.units > 0;
+    p.n_full = (int)units - (split ? plan.units : 0);
+    p.split = split ? plan.split : 1;
+    p.part_o = p.part_lse = nullptr;
+    if (split) {
+        // workspace behind the error word: the LSEs of all shares, then their rows
+        const size_t parts = (size_t)plan.units * plan.split, rows = parts * (TM * kBlockM);
+        p.part_lse = reinterpret_cast<float *>(static_cast<char *>(a.split_ws));
+        p.part_o = p.part_lse + (rows + 63) / 64 * 64;
+    }
+    const unsigned grid = (unsigned)(p.n_full + (split ? plan.units * plan.split : 0));
     sparse_attn_kernel<C><<<grid, C::kThreads, C::kSmemBytes, stream>>>(mk, mv, mkt, mvt, p);
+    if (split) {
+        static_assert((TM * kBlockM * (DH / 8)) % (TM * kBlockM) == 0, "whole blocks per unit");
+        merge_parts_kernel<DH, TM * kBlockM><<<dim3(DH / 8, plan.units), TM * kBlockM, 0, stream>>>(p);
+    }
     return check_launch("astraea_sparse_attn");
 }
 
 }  // namespace
 
-size_t attn_workspace_bytes(int, int, int, int, int) { return 256; }
+// 256 bytes for the error word; behind them room for the key shares of a split last round of CTAs (fp32 rows and
+// LSEs), an upper bound over every M' <= M of the same problem
+static size_t split_bytes(long long parts, int d) { return (size_t)parts * (2 * kBlockM) * ((size_t)d * 4 + 4) + 256; }
+static int max_split_of(int N) { const int s = ((N + 63) / 64) / kMinSplitKeyTiles; return s > kMaxSplit ? kMaxSplit : s; }
+
+size_t attn_workspace_bytes(int B, int H, int N, int M, int d)
+{
+    const int s_max = max_split_of(N);
+    if (s_max < 2 || M <= 0) return 256;
+    const long long units = (long long)B * H * ((M + 2 * kBlockM - 1) / (2 * kBlockM));
+    const long long parts = units * s_max < kMaxSplitParts ? units * s_max : kMaxSplitParts;
+    return 256 + split_bytes(parts, d);
+}
 
 // ---------------------------------------------------------------- gathered keys / values
 // The "select Q and K" ablation of the paper restricts keys and values to listed tokens.  The listed K and V
@@ -915,44 +1054,104 @@ int32_t launch_wait_selftest(int *err_word, uint64_t limit_ns, int *gave_up, cud
     return check_launch("astraea_selftest_wait");
 }
 
-// Which CTA shape finishes first.  Large CTAs (two query tiles, one per SM) are dispatched in launch order onto 148
-// SMs; the last one of every (head, batch) is cheaper when it holds one query tile only (0.68 of a full one,
-// measured).  Small CTAs (one query tile, two per SM) all cost the same: `slowdown` times a large one, because two
-// share the SM (measured: 1.05 at head_dim 64, 1.17 at 72).  The difference matters for launches of a few rounds.
-static bool small_ctas_pay(const AttnArgs &a, double slowdown)
+// Which launch finishes first.  Large CTAs (two query tiles, one per SM) are dispatched in launch order onto the SMs;
+// the last one of every (head, batch) is cheaper when it holds one query tile only (0.68 of a full one, measured).
+// Their last round is usually partial: its CTAs can each be replaced by `split` CTAs with a share of the keys (a share
+// costs its part of the unit plus ~3 % for the query gather, the pipeline fill and the fp32 rows it writes), merged by
+// a small kernel afterwards.  Small CTAs (one query tile, two per SM, head_dim 64 / 72) all cost the same: `slowdown`
+// times a large one, because two share the SM (measured: 1.05 at head_dim 64, 1.17 at 72).  All of this matters for
+// launches of a few rounds only.
+namespace {
+struct Schedule { bool small = false; SplitPlan plan; };
+
+double finish_time(long long units, int pairs, bool light_last, int n_sm, int tail_units, int split)
 {
+    // greedy dispatch in launch order: every CTA goes to the SM that is free first (a binary min-heap of busy times)
+    double heap[kMaxSMs] = {};
+    double finish = 0.0;
+    auto put = [&](double cost) {
+        const double t = heap[0] + cost;
+        finish = t > finish ? t : finish;
+        int i = 0;
+        for (;;) {                                               // replace the root and sift it down
+            const int l = 2 * i + 1, r = l + 1;
+            int m = l;
+            if (l >= n_sm) break;
+            if (r < n_sm && heap[r] < heap[l]) m = r;
+            if (heap[m] >= t) break;
+            heap[i] = heap[m];
+            i = m;
+        }
+        heap[i] = t;
+    };
+    for (long long c = 0; c < units; ++c) {
+        const double cost = (light_last && c % pairs == pairs - 1) ? 0.68 : 1.0;
+        if (c < units - tail_units) put(cost);
+        else for (int i = 0; i < split; ++i) put(cost / split + 0.03);
+    }
+    return finish;
+}
+
+Schedule choose_schedule(const AttnArgs &a, double slowdown /* 0: no small CTAs */)
+{
+    Schedule out;
     const long long hb = (long long)(a.head_count > 0 ? a.head_count : a.H) * a.B;
     const int pairs = (a.M + 2 * kBlockM - 1) / (2 * kBlockM), tiles = (a.M + kBlockM - 1) / kBlockM;
     const bool light_last = a.M - (pairs - 1) * 2 * kBlockM <= kBlockM;
     const int n_sm = sm_count();
-    if (hb * pairs > 16 * n_sm) return false;                    // many rounds: the granularity does not matter
-    // a denoising loop repeats a few shapes: remember the last answer
-    thread_local long long last_hb = -1;
-    thread_local int last_M = -1;
-    thread_local double last_slowdown = 0.0;
-    thread_local bool last_answer = false;
-    if (hb == last_hb && a.M == last_M && slowdown == last_slowdown) return last_answer;
-    double sm_busy[kMaxSMs] = {};
-    for (long long c = 0; c < hb * pairs; ++c) {                 // greedy dispatch in launch order
-        int best = 0;
-        for (int s = 1; s < n_sm; ++s) if (sm_busy[s] < sm_busy[best]) best = s;
-        sm_busy[best] += (light_last && c % pairs == pairs - 1) ? 0.68 : 1.0;
+    const long long units = hb * pairs;
+    if (units > 16 * n_sm) return out;                           // many rounds: the granularity does not matter
+    // a denoising loop repeats a few shapes: remember the last answers
+    struct Memo { long long hb = -1; int M = -1, N = -1, n_sm = 0; double slowdown = 0.0; size_t ws = 0; Schedule answer; };
+    constexpr int kMemo = 16;
+    thread_local Memo memo[kMemo];
+    thread_local int memo_next = 0;
+    const size_t ws_key = (a.flags & ASTRAEA_ATTN_WHOLE_KEYS) ? 0 : a.split_ws_bytes;
+    for (const Memo &e : memo)
+        if (e.hb == hb && e.M == a.M && e.N == a.N && e.n_sm == n_sm && e.slowdown == slowdown && e.ws == ws_key) return e.answer;
+    double best = finish_time(units, pairs, light_last, n_sm, 0, 1);
+    const double whole = best;
+    const int tail = (int)(units % n_sm);
+    if (a.split_ws && tail > 0 && !(a.flags & ASTRAEA_ATTN_WHOLE_KEYS)) {
+        for (int s = 2; s <= max_split_of(a.N); ++s) {
+            if ((long long)tail * s > kMaxSplitParts || split_bytes((long long)tail * s, a.d) > a.split_ws_bytes) break;
+            const double t = finish_time(units, pairs, light_last, n_sm, tail, s);
+            if (t < 0.98 * whole && t < best) { best = t; out.plan.units = tail; out.plan.split = s; }
+        }
     }
-    double large = 0.0;
-    for (int s = 0; s < n_sm; ++s) large = sm_busy[s] > large ? sm_busy[s] : large;
-    const double small = slowdown * (double)((hb * tiles + 2 * n_sm - 1) / (2 * n_sm));
-    last_hb = hb; last_M = a.M; last_slowdown = slowdown;
-    last_answer = small < 0.97 * large;
-    return last_answer;
+    if (slowdown > 0.0) {
+        const double small = slowdown * (double)((hb * tiles + 2 * n_sm - 1) / (2 * n_sm));
+        if (small < 0.97 * best) { out.small = true; out.plan = SplitPlan(); }
+    }
+    Memo &e = memo[memo_next];
+    memo_next = (memo_next + 1) % kMemo;
+    e.hb = hb; e.M = a.M; e.N = a.N; e.n_sm = n_sm; e.slowdown = slowdown; e.ws = ws_key; e.answer = out;
+    return out;
+}
+}  // namespace
+
+void attn_plan(const AttnArgs &a, int *small_ctas, int *split_units, int *split)
+{
+    const bool force_small = (a.flags & ASTRAEA_ATTN_SMALL_CTAS) != 0 && a.d != 128;
+    const Schedule sc = force_small ? Schedule() : choose_schedule(a, a.d == 64 ? 1.05 : a.d == 72 ? 1.17 : 0.0);
+    *small_ctas = (force_small || sc.small) ? 1 : 0;
+    *split_units = *small_ctas ? 0 : sc.plan.units;
+    *split = *small_ctas ? 1 : sc.plan.split;
 }
 
 int32_t launch_sparse_attn(const AttnArgs &a, cudaStream_t stream)
 {
     const bool force_small = (a.flags & ASTRAEA_ATTN_SMALL_CTAS) != 0;
     switch (a.d) {
-    case 64: return (force_small || small_ctas_pay(a, 1.05)) ? launch_dh<64, 1>(a, stream) : launch_dh<64, 2>(a, stream);
-    case 72: return (force_small || small_ctas_pay(a, 1.17)) ? launch_dh<72, 1>(a, stream) : launch_dh<72, 2>(a, stream);
-    case 128: return launch_dh<128, 2>(a, stream);
+    case 64: {
+        const Schedule sc = force_small ? Schedule() : choose_schedule(a, 1.05);
+        return (force_small || sc.small) ? launch_dh<64, 1>(a, stream) : launch_dh<64, 2>(a, stream, sc.plan);
+    }
+    case 72: {
+        const Schedule sc = force_small ? Schedule() : choose_schedule(a, 1.17);
+        return (force_small || sc.small) ? launch_dh<72, 1>(a, stream) : launch_dh<72, 2>(a, stream, sc.plan);
+    }
+    case 128: return launch_dh<128, 2>(a, stream, choose_schedule(a, 0.0).plan);
     default: return fail(ASTRAEA_ERR_UNSUPPORTED, "head_dim %d is not supported", a.d);
     }
 }

@@ -79,8 +79,14 @@ struct AttnArgs {
     uint32_t flags;
     int *err_word;
     int head_begin = 0, head_count = 0;   // a sub-range of the H heads (head_count 0: all); strides and H stay those of the full tensors
+    // room for the key shares of a split last round of CTAs (256-byte aligned; NULL: the launch is never split).  Two
+    // launches that may run at the same time must not share it.
+    void *split_ws = nullptr;
+    size_t split_ws_bytes = 0;
 };
 int32_t launch_sparse_attn(const AttnArgs &a, cudaStream_t stream);
+// the schedule launch_sparse_attn would pick (host logic only; uses B, H / head_count, N, M, d, flags, split_ws, split_ws_bytes)
+void attn_plan(const AttnArgs &a, int *small_ctas, int *split_units, int *split);
 size_t attn_workspace_bytes(int B, int H, int N, int M, int d);
 int32_t launch_wait_selftest(int *err_word, uint64_t limit_ns, int *gave_up, cudaStream_t stream);
 int32_t noalloc_scratch_address(void **scratch_out);   // device address of the library's built-in scratch array on the current device

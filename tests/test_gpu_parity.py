@@ -213,7 +213,8 @@ def test_scatter_with_no_rows_leaves_cache_alone():
 
 
 # ------------------------------------------------------------------ attention
-def _attn_case(oracle, B, H, N, d, M, seed, layout="bnhd", compact=False, dense=False, scale=0.0, amp=1.0, small_ctas=False):
+def _attn_case(oracle, B, H, N, d, M, seed, layout="bnhd", compact=False, dense=False, scale=0.0, amp=1.0, small_ctas=False,
+               whole_keys=False, expect_split=None):
     rng = np.random.default_rng(seed)
     # amp sharpens the logits only (q, k); values and the cache stay N(0,1)
     q, k, v, cache = (synth.f32_to_bf16_bits((a * rng.standard_normal((B, N, H, d))).astype(np.float32)) for a in (amp, amp, 1.0, 1.0))
@@ -238,9 +239,12 @@ def _attn_case(oracle, B, H, N, d, M, seed, layout="bnhd", compact=False, dense=
         g_lse = Guarded((B, H, N), torch.float32, init=dev(lse_cache0))
     out, lse = g_out.t, g_lse.t
     ws = A.new_workspace(A.OP_SPARSE_ATTN, B, H, N, M, d)
+    flags = (A.ATTN_COMPACT_OUT if compact else 0) | (A.ATTN_SMALL_CTAS if small_ctas else 0) | (A.ATTN_WHOLE_KEYS if whole_keys else 0)
+    if expect_split is not None:
+        plan = A.astraea_sparse_attn_plan(B, H, N, M, d, flags=flags, workspace_bytes=ws.numel())
+        assert (plan["split"], plan["small_ctas"]) == (expect_split, False) and (plan["split_units"] > 0) == (expect_split > 1), plan
     A.astraea_sparse_attn(qd, kd, vd, qs, ks, vs, None if idx is None else dev(idx), M, out, lse, B, H, N, d,
-                          scale=scale, flags=(A.ATTN_COMPACT_OUT if compact else 0) | (A.ATTN_SMALL_CTAS if small_ctas else 0),
-                          workspace=ws)
+                          scale=scale, flags=flags, workspace=ws)
     A.astraea_poll_error(ws)
     g_out.check(("attention out", B, H, N, d, M))
     g_lse.check(("attention lse", B, H, N, d, M))
@@ -293,6 +297,22 @@ def test_attn_one_query_tile_per_cta_shape(oracle, d):
     _attn_case(oracle, 1, 2, 129, d, 129, seed=74, dense=True, small_ctas=True)
     _attn_case(oracle, 1, 2, 900, d, 600, seed=75, amp=12.0, small_ctas=True)
     _attn_case(oracle, 1, 1, 1, d, 1, seed=76, small_ctas=True)
+
+
+@pytest.mark.parametrize("d", [64, 72, 128])
+def test_attn_last_round_split_by_keys(oracle, d):
+    """Launches of less than one round of CTAs and 32+ key tiles: every CTA is replaced by 2-8 CTAs with a share of the
+    keys each, whose fp32 rows a second kernel merges.  Ragged last key tile, a last CTA with one query tile, shares
+    of unequal length, a compact output, the head-major layout, logits that make the shares redo their work."""
+    _attn_case(oracle, 1, 3, 2100, d, 700, seed=300 + d, expect_split=2)
+    _attn_case(oracle, 2, 2, 64 * 53 + 7, d, 300, seed=301 + d, expect_split=3)
+    _attn_case(oracle, 1, 2, 64 * 130 + 33, d, 129, seed=302 + d, expect_split=8)
+    _attn_case(oracle, 1, 2, 4200, d, 520, seed=303 + d, compact=True, expect_split=4)
+    _attn_case(oracle, 1, 2, 2100, d, 260, seed=304 + d, layout="bhnd", expect_split=2)
+    _attn_case(oracle, 1, 2, 2100, d, 600, seed=305 + d, amp=12.0, expect_split=2)
+    _attn_case(oracle, 1, 2, 2100, d, 2100, seed=306 + d, dense=True, expect_split=2)
+    # the same launch with every CTA over all keys
+    _attn_case(oracle, 1, 3, 2100, d, 700, seed=300 + d, whole_keys=True, expect_split=1)
 
 
 def test_attn_many_key_tiles_exercise_every_stage_phase(oracle):
