@@ -275,6 +275,27 @@ class Block:
         parts = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(4)] for e in evs])
         return total_ms, parts.mean(axis=0), parts
 
+    def timed_plain_copy(self, k_keep, steps=10, t_base=1):
+        """The yardstick for the refresh of x_ref on the small shapes: torch's contiguous device-to-device copy of as
+        many bytes (M rows of the OTHER input set, which the step has not just read), launched right behind the step's
+        own calls and timed the same way."""
+        torch, w = self.torch, self.w
+        M = k_keep + w.N_t
+        if M == 0:
+            return None
+        n = w.B * M * w.D
+        dst = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
+        self.step(t_base, k_keep)
+        for t in range(steps):
+            self.step(t_base + 1 + t, k_keep)
+            src = self.sets[(t_base + 2 + t) % len(self.sets)]["x_cur"].view(-1)[:n]
+            evs[t][0].record()
+            dst.copy_(src)
+            evs[t][1].record()
+        torch.cuda.synchronize()
+        return float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
+
     def timed_pair(self, k_keep, steps=10, t_base=1):
         """Mean time of score + select launched back to back (whole steps run; events around the pair only)."""
         torch = self.torch
@@ -284,6 +305,14 @@ class Block:
             self.step(t_base + 1 + t, k_keep, pair_ev=evs[t])
         torch.cuda.synchronize()
         return float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
+
+
+def add_copy_yardstick(kernels, copy_ms):
+    """Next to the refresh of x_ref: what torch's plain copy of as many bytes takes in the same place."""
+    if copy_ms:
+        e = kernels["scatter_reuse(x_ref)"]
+        e["torch_copy_of_as_many_bytes_ms"] = copy_ms
+        e["time_vs_torch_copy"] = e["ms"] / copy_ms
 
 
 def cool_down(torch, seconds=0.5):
@@ -645,6 +674,7 @@ def main():
                 m1 = sampler.mark()
                 A.astraea_poll_error(b2.ws)
                 rl, kn = kernel_report(ww, th, pp, peaks, pair_ms=b2.timed_pair(ww.k_of(th)))
+                add_copy_yardstick(kn, b2.timed_plain_copy(ww.k_of(th)))
                 entry = {"config": config_of(ww, th, world), "ms_per_step": tot / n_st, "steps": n_st,
                          "step_tflops": accounting.attn_flops(ww.B, ww.H, ww.M_of(th), ww.N, ww.d) / (tot / n_st * 1e-3) / 1e12,
                          "roofline": rl, "kernels": kn, "clocks": sampler.summary(m0, m1)}
@@ -686,6 +716,8 @@ def main():
     value = replicas.throughput(job_flops, total_ms) / 1e12
     pair_ms = blk.timed_pair(k_keep) if extras else None
     roofline, kernels = kernel_report(w, theta, parts, peaks, pair_ms=pair_ms)
+    if extras:
+        add_copy_yardstick(kernels, blk.timed_plain_copy(k_keep))
     kernels["hbm_peaks_gbs"] = {"measured": peaks["hbm_gbs"], "nominal": NOMINAL_HBM_GBS}
     clocks = sampler.summary(c0, c1) if c1 > c0 else sampler.summary()
     attn_fracs["%s@%d" % (w.name, theta)] = roofline["frac"]
