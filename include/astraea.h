@@ -202,6 +202,7 @@ int32_t astraea_sparse_attn_plan(int B, int H, int N, int M, int d, uint32_t fla
  * astraea_sparse_attn, but keys and values come from another sequence of N_kv tokens (the text tokens),
  *     out[b, i, h, :] = Softmax(q[b, i, h, :] K[b, :, h, :]^T * scale) V[b, :, h, :]   for i in q_idx,
  * k, v : bf16 [B, N_kv, H, d] through their stride triples; q, out, lse_out, q_idx, M, flags, workspace as above
+ *        (the keys that a launch may split are the N_kv ones: size the workspace with N_kv in place of N for that)
  * (N is the token count of q and out).  There is no kv_idx form.  Errors as astraea_sparse_attn.
  */
 int32_t astraea_sparse_cross_attn(const void *q, const void *k, const void *v,

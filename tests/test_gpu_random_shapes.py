@@ -25,10 +25,10 @@ def test_random_attention_cases(oracle, seed):
     for _ in range(8):
         d = rnd.choice([64, 72, 128])
         B, H = rnd.choice([1, 2]), rnd.choice([1, 2, 3])
-        N = rnd.choice([1, 2, 63, 64, 65, 127, 128, 129, 191, 192, 193, 255, 257, 300, 640, 777])
+        N = rnd.choice([1, 2, 63, 64, 65, 127, 128, 129, 191, 192, 193, 255, 257, 300, 640, 777, 1100, 2150])   # 1024+ keys: the launch may split them
         M = rnd.randint(1, N)
         mode = rnd.choice(["self", "self", "cross", "kv"])
-        N_kv = rnd.choice([1, 5, 64, 100, 226, 300]) if mode == "cross" else N
+        N_kv = rnd.choice([1, 5, 64, 100, 226, 300, 1300]) if mode == "cross" else N
         fl = A.ATTN_SMALL_CTAS if (d != 128 and rnd.random() < 0.4) else 0   # the other CTA shape of head_dim 64 / 72
         sig = rnd.choice([0.0, 0.0, 0.5, 1.0])                       # per-token lognormal norms: heavy-tailed logits
         amp = rnd.choice([1.0, 1.0, 2.0, 12.0])                      # 12: the speculation limit is passed, the CTAs redo
@@ -45,7 +45,7 @@ def test_random_attention_cases(oracle, seed):
         out, lse = to_dev_bf16(cache), torch.zeros(B, H, N, device="cuda")
         sq_, sk_ = A.bhnd_strides(N, H, d), A.bhnd_strides(N_kv, H, d)
         if mode == "cross":
-            ws = A.new_workspace(A.OP_SPARSE_ATTN, B, H, N, M, d)
+            ws = A.new_workspace(A.OP_SPARSE_ATTN, B, H, max(N, N_kv), M, d)     # room for a split over the N_kv keys
             A.astraea_sparse_cross_attn(to_dev_bf16(q), to_dev_bf16(k), to_dev_bf16(v), sq_, sk_, sk_, dev(idx), M, out, lse,
                                         B, H, N, N_kv, d, flags=fl, workspace=ws)
         elif mode == "kv":
