@@ -42,7 +42,9 @@ constexpr int kEpiSplit = 2;
 constexpr int kEpiWarps = 4 * kMSub * kEpiSplit, kGatherWarps = 4 * kMSub;
 constexpr int kThreads = (kEpiWarps + kGatherWarps + 2) * 32;
 constexpr int kTmaWarp = kEpiWarps + kGatherWarps, kMmaWarp = kTmaWarp + 1;
-constexpr int kSmemBytes = kStages * (kABytes + kBBytes) + 256 + 1024;
+constexpr int kEpiStageBytes = 32 * 64;                  // per epilogue warp: 32 rows x 32 bf16 columns on their way to / from global memory
+constexpr int kSmemBytes = kStages * (kABytes + kBBytes) + 256 + kEpiWarps * kEpiStageBytes + 1024;
+static_assert(kSmemBytes <= 227 * 1024, "shared memory of one CTA");
 constexpr uint32_t kAccCols = kBN, kTmemCols = 2 * kBN;
 
 struct LinParams {
@@ -137,6 +139,7 @@ gathered_linear_kernel(const __grid_constant__ CUtensorMap tmap_w, const LinPara
         const int row = sub * 128 + (warp & 3) * 32 + lane;
         const int c0 = part * (kBN / kEpiSplit);
         const uint32_t t_row = tmem + ((uint32_t)((warp & 3) * 32) << 16) + sub * kAccCols;
+        uint8_t *stage = smem_raw + (bars + 256 - smem_u32(smem_raw)) + warp * kEpiStageBytes;
         int it = 0;
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
             const int tm = tile / tiles_n, tn = tile - tm * tiles_n;
@@ -145,14 +148,44 @@ gathered_linear_kernel(const __grid_constant__ CUtensorMap tmap_w, const LinPara
             int batch = 0;
             const long long src = source_row(p, (long long)tm * kBM + row, total_rows, &out_row, &res_row, &batch);
             if (src == -2 && tn == 0 && part == 0) atomicExch(p.err_word, kErrBadIndex);
-            __nv_bfloat16 *dst = (src >= 0) ? p.y + out_row * p.N_out + n0 : nullptr;
-            const __nv_bfloat16 *res = (src >= 0 && p.residual) ? p.residual + res_row * p.N_out : nullptr;
+            if (src < 0) { out_row = -1; res_row = -1; }
+            if (!p.residual) res_row = -1;
             const __nv_bfloat16 *gate = p.gate ? p.gate + (long long)batch * p.N_out : nullptr;
             wait_bar(bar_acc_full + 8 * acc, (it / kAccSets) & 1, &abort_flag, p.err_word);
             tc_fence_after();
-            if (abort_flag) dst = nullptr;
+            if (abort_flag) out_row = -1;
+            // Global memory is touched in a transposed layout: a thread owns a row of the accumulator, so a warp that
+            // stored its rows directly would touch 32 lines per instruction, 16 bytes in each (measured: ~9 us of a
+            // 36 us tile, 16 us with a residual).  Instead lane l moves the 16-byte piece l & 3 of rows (l >> 2) + 8 j:
+            // 64 contiguous bytes per row, 8 rows per instruction, through 2 KB of shared memory per warp (pieces
+            // swizzled by the row so that both directions are free of bank conflicts).
+            const int q = lane & 3;
 #pragma unroll 1
             for (int c = c0; c < c0 + kBN / kEpiSplit; c += 32) {
+                const int colq = n0 + c + q * 8;                    // the 8 columns this lane moves
+                uint32_t rw[16];                                    // this thread's row of the residual: 32 bf16
+                if (p.residual) {
+                    uint4 rr[4];
+#pragma unroll
+                    for (int jj = 0; jj < 4; ++jj) {
+                        const int r = (lane >> 2) + 8 * jj;
+                        const long long rrow = __shfl_sync(0xffffffffu, res_row, r);
+                        rr[jj] = (rrow >= 0 && colq < p.N_out) ? __ldg(reinterpret_cast<const uint4 *>(p.residual + rrow * p.N_out + colq))
+                                                                : make_uint4(0, 0, 0, 0);
+                    }
+#pragma unroll
+                    for (int jj = 0; jj < 4; ++jj) {
+                        const int r = (lane >> 2) + 8 * jj;
+                        *reinterpret_cast<uint4 *>(stage + r * 64 + ((q ^ ((r >> 1) & 3)) << 4)) = rr[jj];
+                    }
+                    __syncwarp();
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        const uint4 t = *reinterpret_cast<const uint4 *>(stage + lane * 64 + ((v ^ ((lane >> 1) & 3)) << 4));
+                        rw[4 * v] = t.x; rw[4 * v + 1] = t.y; rw[4 * v + 2] = t.z; rw[4 * v + 3] = t.w;
+                    }
+                    __syncwarp();
+                }
                 uint32_t o[32];
                 tmem_ld32(t_row + acc * kMSub * kAccCols + c, o);
                 tc_wait_ld();
@@ -160,43 +193,41 @@ gathered_linear_kernel(const __grid_constant__ CUtensorMap tmap_w, const LinPara
                     tc_fence_before();
                     mbar_arrive(bar_acc_empty + 8 * acc);
                 }
-                if (dst == nullptr) continue;
 #pragma unroll
                 for (int v = 0; v < 4; ++v) {
                     const int col = n0 + c + v * 8;
-                    if (col >= p.N_out) break;           // N_out is a multiple of 8
                     float f[8];
 #pragma unroll
                     for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(o[v * 8 + i]);
-                    if (p.bias) {
-                        const uint4 bb = __ldg(reinterpret_cast<const uint4 *>(p.bias + col));
-                        const uint32_t bw[4] = {bb.x, bb.y, bb.z, bb.w};
+                    if (col < p.N_out) {                 // N_out is a multiple of 8; columns past it are never stored
+                        if (p.bias) {
+                            const uint4 bb = __ldg(reinterpret_cast<const uint4 *>(p.bias + col));
+                            const uint32_t bw[4] = {bb.x, bb.y, bb.z, bb.w};
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            f[2 * i] += __uint_as_float(bw[i] << 16);
-                            f[2 * i + 1] += __uint_as_float(bw[i] & 0xffff0000u);
+                            for (int i = 0; i < 4; ++i) {
+                                f[2 * i] += __uint_as_float(bw[i] << 16);
+                                f[2 * i + 1] += __uint_as_float(bw[i] & 0xffff0000u);
+                            }
                         }
-                    }
-                    if (p.gelu) {
+                        if (p.gelu) {
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) f[i] = 0.5f * f[i] * (1.0f + erff(f[i] * 0.70710678118654752f));
-                    }
-                    if (gate) {
-                        const uint4 gg = __ldg(reinterpret_cast<const uint4 *>(gate + col));
-                        const uint32_t gw[4] = {gg.x, gg.y, gg.z, gg.w};
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            f[2 * i] *= __uint_as_float(gw[i] << 16);
-                            f[2 * i + 1] *= __uint_as_float(gw[i] & 0xffff0000u);
+                            for (int i = 0; i < 8; ++i) f[i] = 0.5f * f[i] * (1.0f + erff(f[i] * 0.70710678118654752f));
                         }
-                    }
-                    if (res) {
-                        const uint4 rr = __ldg(reinterpret_cast<const uint4 *>(res + col));
-                        const uint32_t rw[4] = {rr.x, rr.y, rr.z, rr.w};
+                        if (gate) {
+                            const uint4 gg = __ldg(reinterpret_cast<const uint4 *>(gate + col));
+                            const uint32_t gw[4] = {gg.x, gg.y, gg.z, gg.w};
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            f[2 * i] += __uint_as_float(rw[i] << 16);
-                            f[2 * i + 1] += __uint_as_float(rw[i] & 0xffff0000u);
+                            for (int i = 0; i < 4; ++i) {
+                                f[2 * i] *= __uint_as_float(gw[i] << 16);
+                                f[2 * i + 1] *= __uint_as_float(gw[i] & 0xffff0000u);
+                            }
+                        }
+                        if (p.residual) {
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                f[2 * i] += __uint_as_float(rw[4 * v + i] << 16);
+                                f[2 * i + 1] += __uint_as_float(rw[4 * v + i] & 0xffff0000u);
+                            }
                         }
                     }
                     uint32_t w[4];
@@ -205,8 +236,17 @@ gathered_linear_kernel(const __grid_constant__ CUtensorMap tmap_w, const LinPara
                         __nv_bfloat162 v2 = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
                         w[i] = *reinterpret_cast<uint32_t *>(&v2);
                     }
-                    *reinterpret_cast<uint4 *>(dst + c + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<uint4 *>(stage + lane * 64 + ((v ^ ((lane >> 1) & 3)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
+                __syncwarp();
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    const int r = (lane >> 2) + 8 * jj;
+                    const long long orow = __shfl_sync(0xffffffffu, out_row, r);
+                    const uint4 t = *reinterpret_cast<const uint4 *>(stage + r * 64 + ((q ^ ((r >> 1) & 3)) << 4));
+                    if (orow >= 0 && colq < p.N_out) *reinterpret_cast<uint4 *>(p.y + orow * p.N_out + colq) = t;
+                }
+                __syncwarp();
             }
         }
     } else if (warp < kEpiWarps + kGatherWarps) {
