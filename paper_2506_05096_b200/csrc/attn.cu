@@ -3,7 +3,8 @@
 // Section 3.2 "Sparse Attention").
 //
 // One CTA per (256 selected queries, head, batch): two 128-row query tiles that share every
-// K/V tile of 64 keys.  Warp roles:
+// K/V tile of 64 keys.  (The CTAs of a launch's last, partial round may instead be replaced by several CTAs
+// each, every one with a share of the key tiles; merge_parts_kernel combines their rows: see SplitPlan.)  Warp roles:
 //   softmax warpgroups (one thread per query row), two per query tile: gather the tile's Q rows into
 //              128B-swizzled shared memory, then per key tile read S from TMEM, exponentiate in the log2
 //              domain against a reference maximum, write P (bf16) back to TMEM over S, and at the end
@@ -1100,6 +1101,10 @@ Schedule choose_schedule(const AttnArgs &a, double slowdown /* 0: no small CTAs 
     const bool light_last = a.M - (pairs - 1) * 2 * kBlockM <= kBlockM;
     const int n_sm = sm_count();
     const long long units = hb * pairs;
+    // a handful of key tiles (cross-attention over the text tokens): a CTA is mostly set-up (barriers, TMEM, the query
+    // gather, the epilogue), which two small CTAs per SM overlap with each other's key loop (measured on 226 keys,
+    // 9001 queries x 48 heads: 121 against 137 us)
+    if (slowdown > 0.0 && (a.N + 63) / 64 <= 8 && tiles > 1) { out.small = true; return out; }
     if (units > 16 * n_sm) return out;                           // many rounds: the granularity does not matter
     // a denoising loop repeats a few shapes: remember the last answers
     struct Memo { long long hb = -1; int M = -1, N = -1, n_sm = 0; double slowdown = 0.0; size_t ws = 0; Schedule answer; };
