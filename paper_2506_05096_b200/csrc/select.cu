@@ -233,11 +233,45 @@ select_cluster_kernel(const float *__restrict__ score, int N_sel, int k, int n_a
     // would spill), so that their latency is hidden behind the passes
     constexpr bool kPrefetchCounters = ITEMS <= 8;
     int32_t n_old[kPrefetchCounters ? ITEMS : 1];
+    // a thread's tokens are consecutive: 16-byte accesses where the row's alignment and the thread's range allow them
+    constexpr int kVec = ITEMS >= 4 ? 4 : ITEMS;
+    const bool whole = base + ITEMS <= N_sel;
+    const bool vec_s = whole && (reinterpret_cast<uintptr_t>(s + base) & (kVec * 4 - 1)) == 0;
+    const bool vec_n = whole && nsk && (reinterpret_cast<uintptr_t>(nsk + base) & (kVec * 4 - 1)) == 0;
+    if (vec_s) {
 #pragma unroll
-    for (int u = 0; u < ITEMS; ++u) key[u] = (base + u < N_sel) ? score_key(__ldg(s + base + u)) : 0u;
+        for (int u = 0; u < ITEMS; u += kVec) {
+            float f[kVec];
+            if constexpr (kVec == 4) {
+                const float4 v = __ldg(reinterpret_cast<const float4 *>(s + base + u));
+                f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
+            } else {
+                const float2 v = __ldg(reinterpret_cast<const float2 *>(s + base + u));
+                f[0] = v.x; f[1] = v.y;
+            }
+#pragma unroll
+            for (int j = 0; j < kVec; ++j) key[u + j] = score_key(f[j]);
+        }
+    } else {
+#pragma unroll
+        for (int u = 0; u < ITEMS; ++u) key[u] = (base + u < N_sel) ? score_key(__ldg(s + base + u)) : 0u;
+    }
     if constexpr (kPrefetchCounters) {
+        if (vec_n) {
 #pragma unroll
-        for (int u = 0; u < ITEMS; ++u) n_old[u] = (nsk && base + u < N_sel) ? nsk[base + u] : 0;
+            for (int u = 0; u < ITEMS; u += kVec) {
+                if constexpr (kVec == 4) {
+                    const int4 v = *reinterpret_cast<const int4 *>(nsk + base + u);
+                    n_old[u] = v.x; n_old[u + 1] = v.y; n_old[u + 2] = v.z; n_old[u + 3] = v.w;
+                } else {
+                    const int2 v = *reinterpret_cast<const int2 *>(nsk + base + u);
+                    n_old[u] = v.x; n_old[u + 1] = v.y;
+                }
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < ITEMS; ++u) n_old[u] = (nsk && base + u < N_sel) ? nsk[base + u] : 0;
+        }
     }
 
     // token i is selected iff key > T, or key == T and fewer than need_eq equal keys precede it
@@ -327,15 +361,14 @@ select_cluster_kernel(const float *__restrict__ score, int N_sel, int k, int n_a
     }
 
     // ordered placement
-    uint32_t gt[ITEMS], eq[ITEMS], tg = 0, te = 0;
+    uint32_t gtm = 0, eqm = 0;                   // bit u: this thread's token u has a key above / equal to T
 #pragma unroll
     for (int u = 0; u < ITEMS; ++u) {
         const bool in = base + u < N_sel;
-        gt[u] = in && key[u] > T;
-        eq[u] = in && key[u] == T;
-        tg += gt[u];
-        te += eq[u];
+        gtm |= (uint32_t)(in && key[u] > T) << u;
+        eqm |= (uint32_t)(in && key[u] == T) << u;
     }
+    const uint32_t tg = __popc(gtm), te = __popc(eqm);
     uint32_t ig = tg, ie = te;                   // inclusive scans over the warp
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -362,17 +395,35 @@ select_cluster_kernel(const float *__restrict__ score, int N_sel, int k, int n_a
     uint32_t pg = bg + ig - tg, pe = be + ie - te;
     for (uint32_t r = 0; r < rank; ++r) { pg += cta_gt[r]; pe += cta_eq[r]; }
 #pragma unroll
-    for (int u = 0; u < ITEMS; ++u) {
-        const int i = base + u;
-        if (i < N_sel) {
-            const bool take = gt[u] || (eq[u] && pe < need_eq);
-            const uint32_t before = pg + min(pe, need_eq);
-            if (take) { if (sel) sel[before] = i; }
-            else if (rem) rem[(uint32_t)i - before] = i;
-            if (nsk) nsk[i] = take ? 0 : min((kPrefetchCounters ? n_old[u] : nsk[i]) + 1, ASTRAEA_N_SKIP_CLAMP);
+    for (int u0 = 0; u0 < ITEMS; u0 += kVec) {
+        int32_t cnt[kVec];                       // the counters of this group of tokens: old, then new
+        if (vec_n) {
+            if constexpr (kPrefetchCounters) {
+#pragma unroll
+                for (int j = 0; j < kVec; ++j) cnt[j] = n_old[u0 + j];
+            } else if constexpr (kVec == 4) {    // not fetched ahead: one 16-byte load per four
+                const int4 v = *reinterpret_cast<const int4 *>(nsk + base + u0);
+                cnt[0] = v.x; cnt[1] = v.y; cnt[2] = v.z; cnt[3] = v.w;
+            }
         }
-        pg += gt[u];
-        pe += eq[u];
+#pragma unroll
+        for (int j = 0; j < kVec; ++j) {
+            const int u = u0 + j, i = base + u;
+            if (i < N_sel) {
+                const bool take = ((gtm >> u) & 1u) || (((eqm >> u) & 1u) && pe < need_eq);
+                const uint32_t before = pg + min(pe, need_eq);
+                if (take) { if (sel) sel[before] = i; }
+                else if (rem) rem[(uint32_t)i - before] = i;
+                if (vec_n) cnt[j] = take ? 0 : min(cnt[j] + 1, ASTRAEA_N_SKIP_CLAMP);
+                else if (nsk) nsk[i] = take ? 0 : min((kPrefetchCounters ? n_old[u] : nsk[i]) + 1, ASTRAEA_N_SKIP_CLAMP);
+            }
+            pg += (gtm >> u) & 1u;
+            pe += (eqm >> u) & 1u;
+        }
+        if (vec_n) {
+            if constexpr (kVec == 4) *reinterpret_cast<int4 *>(nsk + base + u0) = make_int4(cnt[0], cnt[1], cnt[2], cnt[3]);
+            else *reinterpret_cast<int2 *>(nsk + base + u0) = make_int2(cnt[0], cnt[1]);
+        }
     }
     if (rank == 0) for (int t = tid; t < n_always; t += kThreads) sel[k + t] = N_sel + t;
     // no barrier at the end: the last remote accesses (the totals above) were complete at the barrier before the placement
