@@ -394,6 +394,19 @@ select_cluster_kernel(const float *__restrict__ score, int N_sel, int k, int n_a
     cluster_sync_all();
     uint32_t pg = bg + ig - tg, pe = be + ie - te;
     for (uint32_t r = 0; r < rank; ++r) { pg += cta_gt[r]; pe += cta_eq[r]; }
+    // With 8 or 16 tokens per thread a warp's direct stores of the two index lists would touch 32 lines per instruction
+    // (a thread's entries are consecutive, the lanes are 32 or 64 bytes apart).  The warp's tokens are consecutive, and
+    // so are their places in both lists: the entries are first put in order into the warp's piece of the histogram
+    // memory (idle since the last cluster barrier; nobody writes it remotely any more), then copied out by whole lines.
+    constexpr bool kStage = ITEMS >= 8;
+    int32_t *stage = reinterpret_cast<int32_t *>(smem_hist) + warp * (32 * ITEMS);
+    static_assert(!kStage || (size_t)kThreads * ITEMS * sizeof(int32_t) <= kClusterSmem, "the staged lists fit the histogram memory");
+    const uint32_t before0 = pg + min(pe, need_eq);              // selected tokens ahead of this thread's first token
+    const uint32_t takes = tg + min(te, need_eq > pe ? need_eq - pe : 0u);
+    const uint32_t w_sel0 = __shfl_sync(0xffffffffu, before0, 0);
+    const uint32_t w_sel_n = __shfl_sync(0xffffffffu, before0 + takes, 31) - w_sel0;     // selected tokens of the warp
+    const int w_tok0 = base - lane * ITEMS;                      // the warp's first token
+    const uint32_t w_rem0 = (uint32_t)w_tok0 - w_sel0;
 #pragma unroll
     for (int u0 = 0; u0 < ITEMS; u0 += kVec) {
         int32_t cnt[kVec];                       // the counters of this group of tokens: old, then new
@@ -412,8 +425,13 @@ select_cluster_kernel(const float *__restrict__ score, int N_sel, int k, int n_a
             if (i < N_sel) {
                 const bool take = ((gtm >> u) & 1u) || (((eqm >> u) & 1u) && pe < need_eq);
                 const uint32_t before = pg + min(pe, need_eq);
-                if (take) { if (sel) sel[before] = i; }
-                else if (rem) rem[(uint32_t)i - before] = i;
+                if constexpr (kStage) {
+                    if (take) stage[before - w_sel0] = i;
+                    else stage[w_sel_n + ((uint32_t)i - before - w_rem0)] = i;
+                } else {
+                    if (take) { if (sel) sel[before] = i; }
+                    else if (rem) rem[(uint32_t)i - before] = i;
+                }
                 if (vec_n) cnt[j] = take ? 0 : min(cnt[j] + 1, ASTRAEA_N_SKIP_CLAMP);
                 else if (nsk) nsk[i] = take ? 0 : min((kPrefetchCounters ? n_old[u] : nsk[i]) + 1, ASTRAEA_N_SKIP_CLAMP);
             }
@@ -424,6 +442,13 @@ select_cluster_kernel(const float *__restrict__ score, int N_sel, int k, int n_a
             if constexpr (kVec == 4) *reinterpret_cast<int4 *>(nsk + base + u0) = make_int4(cnt[0], cnt[1], cnt[2], cnt[3]);
             else *reinterpret_cast<int2 *>(nsk + base + u0) = make_int2(cnt[0], cnt[1]);
         }
+    }
+    if constexpr (kStage) {
+        __syncwarp();
+        const int w_tok_n = min(max(N_sel - w_tok0, 0), 32 * ITEMS);      // tokens of this warp
+        const uint32_t w_rem_n = (uint32_t)w_tok_n - w_sel_n;
+        if (sel) for (uint32_t j = lane; j < w_sel_n; j += 32) sel[w_sel0 + j] = stage[j];
+        if (rem) for (uint32_t j = lane; j < w_rem_n; j += 32) rem[w_rem0 + j] = stage[w_sel_n + j];
     }
     if (rank == 0) for (int t = tid; t < n_always; t += kThreads) sel[k + t] = N_sel + t;
     // no barrier at the end: the last remote accesses (the totals above) were complete at the barrier before the placement
