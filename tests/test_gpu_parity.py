@@ -495,6 +495,36 @@ def test_attn_duplicate_and_descending_indices_are_reported_and_written_once():
     assert bool((out[0, untouched.cuda()] == 3.0).all())
 
 
+def test_attn_bad_indices_in_a_launch_that_is_split_by_keys():
+    """The same rule where the CTAs take shares of the keys and a second kernel merges them: the merge skips the rows
+    that the attention kernel reported, writes the others, and the rows in between keep the cache."""
+    B, H, N, d, M = 1, 2, 2100, 64, 300
+    g = torch.Generator(device="cpu").manual_seed(6)
+    q, k, v = (torch.randn(B, N, H, d, generator=g).bfloat16().cuda() for _ in range(3))
+    s = A.bhnd_strides(N, H, d)
+    ws = A.new_workspace(A.OP_SPARSE_ATTN, B, H, N, M, d)
+    assert A.astraea_sparse_attn_plan(B, H, N, M, d, workspace_bytes=ws.numel())["split"] == 2
+    good = (torch.arange(M, dtype=torch.int32) * 7).view(1, M).cuda()
+    want, want_lse = torch.full((B, N, H, d), 3.0, dtype=torch.bfloat16, device="cuda"), torch.full((B, H, N), -7.0, device="cuda")
+    A.astraea_sparse_attn(q, k, v, s, s, s, good, M, want, want_lse, B, H, N, d, workspace=ws)
+    A.astraea_poll_error(ws)
+    bad = good.clone()
+    bad[0, 10] = bad[0, 9]                       # a duplicate
+    bad[0, 200] = 5                              # a descending step
+    bad[0, 299] = N + 3                          # out of range
+    out, lse = torch.full((B, N, H, d), 3.0, dtype=torch.bfloat16, device="cuda"), torch.full((B, H, N), -7.0, device="cuda")
+    A.astraea_sparse_attn(q, k, v, s, s, s, bad, M, out, lse, B, H, N, d, workspace=ws)
+    with pytest.raises(A.AstraeaError) as e:
+        A.astraea_poll_error(ws)
+    assert e.value.code == A.ERR_BAD_INDEX
+    ok_rows = [r for r in range(M) if r not in (10, 200, 299)]
+    toks = good[0, ok_rows].long()
+    assert torch.equal(out[0, toks], want[0, toks]) and torch.equal(lse[0][:, toks], want_lse[0][:, toks])
+    untouched = torch.ones(N, dtype=torch.bool, device="cuda")
+    untouched[toks] = False
+    assert bool((out[0, untouched] == 3.0).all()) and bool((lse[0][:, untouched] == -7.0).all())
+
+
 # ------------------------------------------------------------- the whole step
 def _step_case(oracle, w, seed, theta, steps=1):
     inp = synth.make_step_inputs(w, seed)
