@@ -61,7 +61,8 @@ extern "C" {
 /* flags of astraea_gathered_linear */
 #define ASTRAEA_LINEAR_COMPACT_OUT 1u        /* y is [B,M,N_out] (row r of the index list), not the cache [B,N,N_out] */
 #define ASTRAEA_LINEAR_COMPACT_IN  2u        /* x is [B,M,K]: row r is the row of token idx[b,r] (output of a layer run with COMPACT_OUT) */
-#define ASTRAEA_LINEAR_GELU        4u        /* y = GELU(x W^T + bias), GELU(u) = u/2 (1 + erf(u / sqrt 2)): the first MLP layer */
+#define ASTRAEA_LINEAR_GELU        4u        /* y = GELU(x W^T + bias), GELU(u) = u/2 (1 + erf(u / sqrt 2)): the first MLP layer
+                                              * (erf in fp32 to 6e-7 absolute, before the one rounding to bf16) */
 #define ASTRAEA_LINEAR_COMPACT_RES 8u        /* astraea_gathered_linear_residual: residual is [B,M,N_out] (row r of the index list) */
 /* flags of astraea_layernorm_modulate */
 #define ASTRAEA_LN_COMPACT_IN     1u         /* x is [B,M,D]: row r is the row of token idx[b,r] */
