@@ -262,7 +262,8 @@ class Block:
             ev[4].record()
 
     def timed(self, k_keep, steps, warmup, barrier, t_base=1):
-        """`steps` consecutive steps after `warmup` untimed ones; returns (total ms, mean ms of the four calls)."""
+        """`steps` consecutive steps after `warmup` untimed ones; returns (total ms, median ms of each of the four calls
+        over the steps, all the per-step times)."""
         torch = self.torch
         for t in range(warmup):
             self.step(t_base + t, k_keep)
@@ -273,7 +274,7 @@ class Block:
         barrier()
         total_ms = evs[0][0].elapsed_time(evs[-1][4])
         parts = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(4)] for e in evs])
-        return total_ms, parts.mean(axis=0), parts
+        return total_ms, np.median(parts, axis=0), parts
 
     def timed_plain_copy(self, k_keep, steps=10, t_base=1):
         """The yardstick for the refresh of x_ref on the small shapes: torch's contiguous device-to-device copy of as
@@ -297,14 +298,14 @@ class Block:
         return float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
 
     def timed_pair(self, k_keep, steps=10, t_base=1):
-        """Mean time of score + select launched back to back (whole steps run; events around the pair only)."""
+        """Median time of score + select launched back to back (whole steps run; events around the pair only)."""
         torch = self.torch
         evs = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
         self.step(t_base, k_keep)
         for t in range(steps):
             self.step(t_base + 1 + t, k_keep, pair_ev=evs[t])
         torch.cuda.synchronize()
-        return float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
+        return float(np.median([e[0].elapsed_time(e[1]) for e in evs]))
 
 
 def add_copy_yardstick(kernels, copy_ms):
@@ -332,8 +333,9 @@ def attn_schedule(w, theta):
     return plan
 
 
-def kernel_report(w, theta, parts, peaks, long_region=False, pair_ms=None):
-    """Per-kernel figures of one step: times, achieved rates and fractions of the measured and nominal peaks."""
+def kernel_report(w, theta, parts, peaks, long_region=False, pair_ms=None, all_parts=None, stat="median"):
+    """Per-kernel figures of one step: times (the median over the timed steps; with all_parts also the minimum and the
+    number of launches), achieved rates and fractions of the measured and nominal peaks."""
     B, N, H, d, D, N_sel = w.B, w.N, w.H, w.d, w.D, w.N_v
     k_keep = w.k_of(theta)
     M = k_keep + w.N_t
@@ -374,6 +376,11 @@ def kernel_report(w, theta, parts, peaks, long_region=False, pair_ms=None):
                                 "sum_of_the_two_alone_ms": float(parts[0] + parts[1])},
                "sparse_attn": {"ms": attn_ms, "TFLOP/s": achieved, "schedule": attn_schedule(w, theta)},
                "scatter_reuse(x_ref)": hbm_entry(cb, parts[3])}
+    if all_parts is not None:
+        for i, n in enumerate(("score", "select", "sparse_attn", "scatter_reuse(x_ref)")):
+            kernels[n]["min_ms"] = float(np.min(all_parts[:, i]))
+            kernels[n]["launches_timed"] = int(all_parts.shape[0])
+            kernels[n]["of"] = stat
     return roofline, kernels
 
 
@@ -667,13 +674,13 @@ def main():
             b2.step(0, ww.N_v)
             workloads[name] = {}
             for th in thetas:
-                n_st = 20
+                n_st = 20                     # 80 ms at most: with 50 steps (0.2 s) the power cap already pulls the clock down inside the leg
                 cool_down(torch)
                 m0 = sampler.mark()
-                tot, pp, _ = b2.timed(ww.k_of(th), n_st, 3, barrier)
+                tot, pp, allp = b2.timed(ww.k_of(th), n_st, 3, barrier)
                 m1 = sampler.mark()
                 A.astraea_poll_error(b2.ws)
-                rl, kn = kernel_report(ww, th, pp, peaks, pair_ms=b2.timed_pair(ww.k_of(th)))
+                rl, kn = kernel_report(ww, th, pp, peaks, pair_ms=b2.timed_pair(ww.k_of(th), steps=20), all_parts=allp)
                 add_copy_yardstick(kn, b2.timed_plain_copy(ww.k_of(th)))
                 entry = {"config": config_of(ww, th, world), "ms_per_step": tot / n_st, "steps": n_st,
                          "step_tflops": accounting.attn_flops(ww.B, ww.H, ww.M_of(th), ww.N, ww.d) / (tot / n_st * 1e-3) / 1e12,
@@ -707,7 +714,7 @@ def main():
     k_keep = w.k_of(theta)
     M = k_keep + n_always
     c0 = sampler.mark()
-    total_ms, parts, _ = blk.timed(k_keep, args.steps, args.warmup, barrier)
+    total_ms, parts, all_parts = blk.timed(k_keep, args.steps, args.warmup, barrier)
     c1 = sampler.mark()
     A.astraea_poll_error(blk.ws)
     flops = accounting.attn_flops(B, H, M, N, d)
@@ -715,7 +722,8 @@ def main():
     ms_per_step = total_ms / args.steps
     value = replicas.throughput(job_flops, total_ms) / 1e12
     pair_ms = blk.timed_pair(k_keep) if extras else None
-    roofline, kernels = kernel_report(w, theta, parts, peaks, pair_ms=pair_ms)
+    # the headline's roofline divides by the kernel's AVERAGE launch duration over the timed steps
+    roofline, kernels = kernel_report(w, theta, all_parts.mean(axis=0), peaks, pair_ms=pair_ms, all_parts=all_parts, stat="mean")
     if extras:
         add_copy_yardstick(kernels, blk.timed_plain_copy(k_keep))
     kernels["hbm_peaks_gbs"] = {"measured": peaks["hbm_gbs"], "nominal": NOMINAL_HBM_GBS}
@@ -838,8 +846,8 @@ def main():
             m1 = sampler.mark()
             A.astraea_poll_error(b2.ws)
             allp = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(4)] for e in evs])
-            pp = allp.mean(axis=0)
-            rl, kn = kernel_report(hw, th, pp, peaks, long_region=True, pair_ms=b2.timed_pair(hw.k_of(th), steps=3, t_base=0))
+            pp = np.median(allp, axis=0)
+            rl, kn = kernel_report(hw, th, pp, peaks, long_region=True, pair_ms=b2.timed_pair(hw.k_of(th), steps=3, t_base=0), all_parts=allp)
             step_ms = allp.sum(axis=1)
             n_max = int(b2.n_skip.max().item())
             workloads["hunyuan"][str(th)] = {
