@@ -379,21 +379,39 @@ __device__ __forceinline__ void softmax_role(const Params &p, const Bars &bar, i
     const int warp = __shfl_sync(0xffffffffu, wtid >> 5, 0);       // warp-uniform
     // gather this tile's Q rows (swizzled, K-major): 16-byte units, unit c of row r
     constexpr int kMainUnits = C::kMain / 8, kUnits = kMainUnits + (C::kTail ? 2 : 0);
-    for (int v = par * 128 + wtid; v < kBlockM * kUnits; v += 128 * kSplit) {     // the warpgroups of a tile share the rows
+    // (the warpgroups of a tile share the rows; all index loads first, then all row loads, then the stores, so that the
+    // two dependent round trips to memory are paid once and not once per unit)
+    constexpr int kGatherIters = kBlockM * kUnits / (128 * kSplit);
+    static_assert(kBlockM * kUnits % (128 * kSplit) == 0, "whole iterations of the Q gather");
+    int gtok[kGatherIters];
+#pragma unroll
+    for (int it = 0; it < kGatherIters; ++it) {
+        const int v = par * 128 + wtid + it * 128 * kSplit;
         const int r = v / kUnits, c = v - r * kUnits;
         const int m = m_base + r;
-        uint4 val = make_uint4(0, 0, 0, 0);
-        if (m < p.M && c * 8 < C::kDH) {                 // the upper half of the tail chunk stays zero
-            const int tok = p.q_idx ? __ldg(p.q_idx + (size_t)b * p.M + m) : m;
-            if ((unsigned)tok < (unsigned)p.N_tok) {
-                const __nv_bfloat16 *src = p.q + (size_t)b * p.q_sb + (size_t)tok * p.q_sn + (size_t)h * p.q_sh + c * 8;
-                val = __ldg(reinterpret_cast<const uint4 *>(src));
-            }
+        gtok[it] = -1;
+        if (m < p.M && c * 8 < C::kDH)                   // the upper half of the tail chunk stays zero
+            gtok[it] = p.q_idx ? __ldg(p.q_idx + (size_t)b * p.M + m) : m;
+    }
+    uint4 gval[kGatherIters];
+#pragma unroll
+    for (int it = 0; it < kGatherIters; ++it) {
+        const int v = par * 128 + wtid + it * 128 * kSplit;
+        const int c = v % kUnits;
+        gval[it] = make_uint4(0, 0, 0, 0);
+        if ((unsigned)gtok[it] < (unsigned)p.N_tok) {
+            const __nv_bfloat16 *src = p.q + (size_t)b * p.q_sb + (size_t)gtok[it] * p.q_sn + (size_t)h * p.q_sh + c * 8;
+            gval[it] = __ldg(reinterpret_cast<const uint4 *>(src));
         }
+    }
+#pragma unroll
+    for (int it = 0; it < kGatherIters; ++it) {
+        const int v = par * 128 + wtid + it * 128 * kSplit;
+        const int r = v / kUnits, c = v - r * kUnits;
         uint32_t off;
         if (c < kMainUnits) off = (c >> 3) * C::kQChunkBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4);          // 128-byte swizzle
         else off = C::kChunks * C::kQChunkBytes + r * 32 + ((((c - kMainUnits) & 1) ^ ((r >> 2) & 1)) << 4);   // 32-byte swizzle
-        *reinterpret_cast<uint4 *>(sQ_gen + off) = val;
+        *reinterpret_cast<uint4 *>(sQ_gen + off) = gval[it];
     }
     fence_proxy_async_smem();
     mbar_arrive(bar.q + 8 * tile);
@@ -643,12 +661,35 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             mbar_init(bar.done + 8 * t, 1);
             for (int u = 0; u < 4; ++u) { mbar_init(bar.s + 32 * t + 8 * u, 1); mbar_init(bar.p + 32 * t + 8 * u, 128); }
         }
-        // a K/V stage is free once the issuer of every active query tile has committed its MMAs on it
-        for (int s = 0; s < C::kStagesK; ++s) { mbar_init(bar.kf + 8 * s, 1); mbar_init(bar.ke + 8 * s, q_tiles); }
-        for (int s = 0; s < C::kStagesV; ++s) { mbar_init(bar.vf + 8 * s, 1); mbar_init(bar.ve + 8 * s, q_tiles); }
         fence_barrier_init();
     }
     constexpr int kProducerWarp = C::kSoftmaxWarps, kIssuerWarp = C::kSoftmaxWarps + 1;
+    // The producer warp sets up the K/V stage barriers itself and sends for the first kAhead K tiles and the first V
+    // tile at once: their flight then runs under the TMEM allocation, the CTA-wide barrier and the gather of the Q rows
+    // (nobody else touches these barriers or the stages before that barrier).
+    if (warp == kProducerWarp) {
+        if (elect_one()) {
+            // a K/V stage is free once the issuer of every active query tile has committed its MMAs on it
+            for (int s = 0; s < C::kStagesK; ++s) { mbar_init(bar.kf + 8 * s, 1); mbar_init(bar.ke + 8 * s, q_tiles); }
+            for (int s = 0; s < C::kStagesV; ++s) { mbar_init(bar.vf + 8 * s, 1); mbar_init(bar.ve + 8 * s, q_tiles); }
+            fence_barrier_init();
+            for (int j = 0; j < kAhead && j < n_tiles; ++j) {
+                mbar_arrive_expect_tx(bar.kf + 8 * j, C::kLoadBytes);
+#pragma unroll
+                for (int ch = 0; ch < C::kChunks; ++ch)
+                    tma_load_4d(sK + j * C::kTileBytes + ch * C::kChunkBytes, &tmap_k, bar.kf + 8 * j, ch * 64, key0 + j * kBlockN, h, b);
+                if (C::kTail)
+                    tma_load_4d(sK + j * C::kTileBytes + C::kChunks * C::kChunkBytes, &tmap_k_tail, bar.kf + 8 * j, C::kMain, key0 + j * kBlockN, h, b);
+            }
+            mbar_arrive_expect_tx(bar.vf, C::kLoadBytes);
+#pragma unroll
+            for (int ch = 0; ch < C::kChunks; ++ch)
+                tma_load_4d(sV + ch * C::kChunkBytes, &tmap_v, bar.vf, ch * 64, key0, h, b);
+            if (C::kTail)
+                tma_load_4d(sV + C::kChunks * C::kChunkBytes, &tmap_v_tail, bar.vf, C::kMain, key0, h, b);
+        }
+        __syncwarp();
+    }
     if (warp == kIssuerWarp) {
         tmem_alloc(smem_u32(&tmem_slot), kTmemCols);
         tmem_relinquish();
@@ -703,10 +744,11 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         // K runs kAhead tiles ahead of V: K_{j+kAhead} is consumed next to V_j.  The max-only pass needs no V.
         auto produce_pass = [&](int pass) {
             const int gk0 = pass * n_tiles, gv0 = (pass == kExact) ? n_tiles : 0;
-            for (int j = 0; j < kAhead && j < n_tiles; ++j) load_k(gk0 + j, j);
+            const bool sent = pass == kSpeculate;        // the first K tiles and V tile of this pass are on their way already
+            for (int j = 0; j < kAhead && j < n_tiles; ++j) if (!sent) load_k(gk0 + j, j);
             for (int j = 0; j < n_tiles; ++j) {
                 if (j + kAhead < n_tiles) load_k(gk0 + j + kAhead, j + kAhead);
-                if (pass != kMaxOnly) load_v(gv0 + j, j);
+                if (pass != kMaxOnly && !(sent && j == 0)) load_v(gv0 + j, j);
             }
         };
         produce_pass(kSpeculate);
