@@ -42,9 +42,9 @@ NOMINAL_BF16_TFLOPS, NOMINAL_HBM_GBS = 2250.0, 8000.0     # the part's nominal d
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the attention kernel, from the ncu captures summarised
 # in profiles/ (workload -> theta_permille -> (bytes, file)); None where not captured at that size.
 NCU_TRAFFIC = {
-    "cogvideox": {500: (276513024 + 48443136, "profiles/sparse_attn_d64_cogvideox.md")},
-    "opensora": {400: (183240448 + 24986880, "profiles/sparse_attn_d72_opensora.md")},
-    "sweep": {250: (1134856000 + 112798976, "profiles/sparse_attn_d128_sweep.md")},
+    "cogvideox": {500: (276493056 + 47539200, "profiles/sparse_attn_d64_cogvideox.md")},
+    "opensora": {400: (183320320 + 24948736, "profiles/sparse_attn_d72_opensora.md")},
+    "sweep": {250: (1142801000 + 112186368, "profiles/sparse_attn_d128_sweep.md")},
 }
 # The headline launch (sweep shape, keep-ratio 0.5) holds too much for a multi-pass capture: its traffic is the
 # keep-ratio-0.25 capture scaled by the compulsory bytes (the traffic is Q and output rows of M tokens plus K and V of
