@@ -134,6 +134,31 @@ def test_select_q_and_k_ablation_is_attention_on_the_subset(oracle):
 
 
 # ------------------------------------------------------------------ reuse pins
+def test_attention_over_all_keys_is_the_lse_weighted_mix_of_attentions_over_a_partition(oracle):
+    """Softmax attention over a union of disjoint key sets: out = sum_i exp(lse_i - lse) out_i and lse = log sum_i
+    exp(lse_i) (the identity behind every split of the keys).  Pins the LSE output together with kv_idx: a wrong sign,
+    base or scale in the LSE, or keys taken from the wrong rows, breaks the identity."""
+    rng = np.random.default_rng(31)
+    B, N, H, d, M = 2, 90, 2, 16, 11
+    q, k, v = (rng.standard_normal((B, N, H, d)) for _ in range(3))
+    q_idx = np.stack([np.sort(rng.choice(N, M, replace=False)) for _ in range(B)]).astype(np.int32)
+    o_all, lse_all, _ = oracle.sparse_attn(q, k, v, q_idx=q_idx, scale=0.3)
+    perm = np.stack([rng.permutation(N) for _ in range(B)])
+    cuts = [0, 17, 18, 60, N]
+    outs, lses = [], []
+    for a, b_ in zip(cuts[:-1], cuts[1:]):
+        kv = np.sort(perm[:, a:b_], axis=1).astype(np.int32)
+        o, l, _ = oracle.sparse_attn(q, k, v, q_idx=q_idx, kv_idx=kv, scale=0.3)
+        outs.append(o)
+        lses.append(l)
+    lses = np.stack(lses)                                   # [parts, B, H, M]
+    lse = np.log(np.exp(lses).sum(axis=0))
+    w = np.exp(lses - lse[None])                            # [parts, B, H, M]
+    mix = sum(w[i].transpose(0, 2, 1)[..., None] * outs[i] for i in range(len(outs)))
+    assert np.abs(lse - lse_all).max() < 1e-12
+    assert np.abs(mix - o_all).max() < 1e-12
+
+
 def test_keep_ratio_zero_returns_cache_unchanged(oracle):
     rng = np.random.default_rng(9)
     B, N, H, d = 2, 12, 2, 4
